@@ -1,0 +1,130 @@
+"""ctypes loader for the CPU oracle (``tf_oracle.cpp``).
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT: only ``tests/``, the smoke check and the benchmark's
+CPU-baseline leg import this package.  It imports nothing from the CUDA package and the CUDA
+package imports nothing from here.
+
+Arrays are numpy, C-contiguous, shape ``[rows, cols]``; bf16 tensors travel as ``uint16`` bit
+patterns.  Every function returns freshly allocated outputs.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "tf_oracle.cpp"
+_LIB = _HERE / "libtf_oracle.so"
+
+F32, BF16 = 0, 1
+_NP = {F32: np.float32, BF16: np.uint16}
+
+
+def build(force: bool = False) -> Path:
+    """Compile the oracle with g++ (no fast-math, no CUDA) unless an up-to-date build exists."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
+        subprocess.run(
+            ["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-pthread", "-o", str(tmp), str(_SRC)],
+            check=True,
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(str(build()))
+        vp, i64, f32, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_float, ctypes.c_int
+        lib.oracle_softmax.argtypes = [vp, vp, vp, i64, i64, i32, i32]
+        lib.oracle_softmax.restype = i32
+        lib.oracle_layernorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, i32]
+        lib.oracle_layernorm.restype = i32
+        lib.oracle_rmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, i32]
+        lib.oracle_rmsnorm.restype = i32
+        lib.oracle_bf16_from_double.argtypes = [vp, vp, i64]
+        lib.oracle_bf16_from_double.restype = None
+        lib.oracle_bf16_to_double.argtypes = [vp, vp, i64]
+        lib.oracle_bf16_to_double.restype = None
+        _lib = lib
+    return _lib
+
+
+def _check(a: np.ndarray, dt: int, name: str) -> np.ndarray:
+    if a.dtype != _NP[dt] or not a.flags.c_contiguous:
+        raise TypeError(f"{name}: want C-contiguous {_NP[dt].__name__}, got {a.dtype}")
+    return a
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def softmax(x: np.ndarray, dt: int, want64: bool = False, nthreads: int = 1):
+    """Row softmax.  Returns ``y`` (and the unrounded float64 result if ``want64``)."""
+    _check(x, dt, "x")
+    rows, cols = x.shape
+    y = np.empty_like(x)
+    y64 = np.empty((rows, cols), np.float64) if want64 else None
+    rc = _load().oracle_softmax(_p(x), _p(y), _p(y64), rows, cols, dt, nthreads)
+    if rc:
+        raise ValueError("oracle_softmax: bad argument")
+    return (y, y64) if want64 else y
+
+
+def layernorm(x, gamma, beta, eps: float, dt: int, want64: bool = False, nthreads: int = 1):
+    """Row LayerNorm.  Returns ``(y, mean_f32, rstd_f32)`` plus ``(y64, stats64[rows, 2])`` if ``want64``."""
+    _check(x, dt, "x"), _check(gamma, dt, "gamma"), _check(beta, dt, "beta")
+    rows, cols = x.shape
+    if gamma.shape != (cols,) or beta.shape != (cols,):
+        raise ValueError("gamma/beta must have shape [cols]")
+    y = np.empty_like(x)
+    mean = np.empty(rows, np.float32)
+    rstd = np.empty(rows, np.float32)
+    y64 = np.empty((rows, cols), np.float64) if want64 else None
+    st = np.empty((rows, 2), np.float64) if want64 else None
+    rc = _load().oracle_layernorm(_p(x), _p(gamma), _p(beta), _p(y), _p(y64), _p(mean), _p(rstd), _p(st),
+                                  rows, cols, eps, dt, nthreads)
+    if rc:
+        raise ValueError("oracle_layernorm: bad argument")
+    return (y, mean, rstd, y64, st) if want64 else (y, mean, rstd)
+
+
+def rmsnorm(x, w, eps: float, dt: int, want64: bool = False, nthreads: int = 1):
+    """Row RMSNorm.  Returns ``(y, rstd_f32)`` plus ``(y64, rstd64[rows])`` if ``want64``."""
+    _check(x, dt, "x"), _check(w, dt, "w")
+    rows, cols = x.shape
+    if w.shape != (cols,):
+        raise ValueError("w must have shape [cols]")
+    y = np.empty_like(x)
+    rstd = np.empty(rows, np.float32)
+    y64 = np.empty((rows, cols), np.float64) if want64 else None
+    st = np.empty(rows, np.float64) if want64 else None
+    rc = _load().oracle_rmsnorm(_p(x), _p(w), _p(y), _p(y64), _p(rstd), _p(st), rows, cols, eps, dt, nthreads)
+    if rc:
+        raise ValueError("oracle_rmsnorm: bad argument")
+    return (y, rstd, y64, st) if want64 else (y, rstd)
+
+
+def bf16_from_double(v: np.ndarray) -> np.ndarray:
+    """Round float64 values to bf16 bit patterns (nearest-even, subnormals kept)."""
+    v = np.ascontiguousarray(v, np.float64)
+    out = np.empty(v.shape, np.uint16)
+    _load().oracle_bf16_from_double(_p(v), _p(out), v.size)
+    return out
+
+
+def bf16_to_double(h: np.ndarray) -> np.ndarray:
+    """Widen bf16 bit patterns to float64 (exact)."""
+    h = np.ascontiguousarray(h, np.uint16)
+    out = np.empty(h.shape, np.float64)
+    _load().oracle_bf16_to_double(_p(h), _p(out), h.size)
+    return out
