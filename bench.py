@@ -1,0 +1,442 @@
+#!/usr/bin/env python
+"""Benchmark of the row-wise reduce-then-normalise library on B200.
+
+Default run (``python bench.py [--gpus N --steps K --warmup W]``): one step = one pass of the hot path
+(``tf_layernorm_fwd`` through the C ABI) over one bf16 [8192, 4096] batch that is already resident in HBM.
+Prints ONE JSON line: achieved HBM GB/s (algorithmic bytes / device time), the roofline fraction against the
+measured copy bandwidth of this machine, the end-to-end figure with host<->device copies inside the timed region, and
+the CPU oracle timed on this machine's host cores as a reported baseline.
+
+``--impl reference`` times the CPU oracle alone (the reference arm).
+``--table configs|sweep`` measures the other configurations / the shape sweep and writes a table (not a bench line).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+NOMINAL_HBM_GBS = 8000.0          # the "~8 TB/s" the 80% bar is quoted against
+FALLBACK_HBM_GBS = 6650.0         # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+L2_BYTES = 126 << 20
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
+# profiles/; None until a capture of that kernel exists.
+NCU_TRAFFIC_BYTES = {
+    "layernorm_bf16_8192x4096": None,
+}
+
+
+def measured_peak():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------------------
+# clocks: sampled through NVML while the timed region runs (reading only)
+# ---------------------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, cuda_index: int, period_s: float = 0.004):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:        # CUDA and NVML may number the GPUs differently: match by UUID
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(cuda_index).uuid)
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(cuda_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+        self.period = period_s
+
+    def sample(self):
+        if self._h is None:
+            return
+        try:
+            self.samples.append(int(self._nv.nvmlDeviceGetClockInfo(self._h, self._nv.NVML_CLOCK_SM)))
+            mask = int(self._nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+            for bit, name in self.REASONS.items():
+                if mask & bit and name != "gpu_idle":
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self.sample()
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+        self.sample()
+
+    def summary(self) -> dict:
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------------------------------------
+# one workload on one device
+# ---------------------------------------------------------------------------------------------------------
+class DeviceCase:
+    """K rotating (x, y) buffer sets of one workload in HBM, so that no launch finds its lines in L2."""
+
+    def __init__(self, w, data, device, min_total_bytes=1 << 30, max_sets=128):
+        import torch
+        from paper_2512_09196_b200 import inputs
+        self.w, self.torch = w, torch
+        tdt = torch.float32 if w.dt == inputs.F32 else torch.bfloat16
+
+        def dev(a):
+            t = torch.from_numpy(a)
+            return (t.view(torch.bfloat16) if w.dt == inputs.BF16 else t).to(device)
+
+        x0 = dev(data["x"])
+        foot = 2 * x0.numel() * x0.element_size()
+        self.sets = max(2, min(max_sets, -(-min_total_bytes // foot)))
+        if foot >= 4 * L2_BYTES:
+            self.sets = 2
+        self.x = [x0] + [x0.clone() for _ in range(self.sets - 1)]
+        self.y = [torch.empty_like(x0) for _ in range(self.sets)]
+        self.params = {k: dev(v) for k, v in data.items() if k != "x"}
+        rows = x0.shape[0]
+        self.mean = torch.empty(rows, dtype=torch.float32, device=device)
+        self.rstd = torch.empty(rows, dtype=torch.float32, device=device)
+        self.i = 0
+        self.bytes_per_step = w.algorithmic_bytes(rows)
+        self.footprint = foot
+        _ = tdt
+
+    def step(self):
+        import paper_2512_09196_b200 as tf
+        k = self.i % self.sets
+        self.i += 1
+        w = self.w
+        if w.op == "softmax":
+            tf.tf_softmax_fwd(self.x[k], self.y[k])
+        elif w.op == "layernorm":
+            tf.tf_layernorm_fwd(self.x[k], self.params["gamma"], self.params["beta"], w.eps, self.y[k], self.mean, self.rstd)
+        else:
+            tf.tf_rmsnorm_fwd(self.x[k], self.params["w"], w.eps, self.y[k])
+
+    def time_steps(self, steps: int, warmup: int) -> float:
+        """Milliseconds for `steps` back-to-back launches (CUDA events on the launching stream)."""
+        torch = self.torch
+        for _ in range(warmup):
+            self.step()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(steps):
+            self.step()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+
+
+def time_oracle(w, data, rows: int, reps: int = 1) -> float:
+    """Seconds (best of reps) for the single-threaded oracle on the first `rows` rows."""
+    import oracle
+    x = data["x"][:rows]
+    best = float("inf")
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        if w.op == "softmax":
+            oracle.softmax(x, w.dt)
+        elif w.op == "layernorm":
+            oracle.layernorm(x, data["gamma"], data["beta"], w.eps, w.dt)
+        else:
+            oracle.rmsnorm(x, data["w"], w.eps, w.dt)
+        best = min(best, time.perf_counter() - t0)
+    return best
+
+
+def cpu_baseline(w, data, budget_s: float = 15.0) -> dict:
+    """The oracle as it stands, one thread, on a bounded sample of the workload."""
+    probe_rows = max(1, min(w.rows, 64))
+    t_probe = max(time_oracle(w, data, probe_rows), 1e-6)
+    rows = int(max(1, min(w.rows, probe_rows * budget_s / 3 / t_probe)))
+    reps = 3 if rows == w.rows else 1
+    t = time_oracle(w, data, rows, reps)
+    gbs = w.algorithmic_bytes(rows) / t / 1e9
+    sample = (f"full batch [{rows}, {w.cols}], best of {reps}" if rows == w.rows
+              else f"first {rows} of {w.rows} rows, one pass, scaled per byte")
+    return {"value": gbs, "unit": "GB/s", "cores": 1, "cores_available": os.cpu_count(), "kind": "oracle", "sample": sample,
+            "seconds": t}
+
+
+# ---------------------------------------------------------------------------------------------------------
+# end to end: pinned host buffers, H2D + kernel + D2H inside the timed region
+# ---------------------------------------------------------------------------------------------------------
+def time_e2e(w, data, device, steps: int, warmup: int):
+    import torch
+    import paper_2512_09196_b200 as tf
+    from paper_2512_09196_b200 import inputs
+
+    def pin(a):
+        t = torch.from_numpy(a)
+        return (t.view(torch.bfloat16) if w.dt == inputs.BF16 else t).pin_memory()
+
+    hx = pin(data["x"])
+    hp = {k: pin(v) for k, v in data.items() if k != "x"}
+    hy = torch.empty_like(hx).pin_memory()
+    rows = hx.shape[0]
+    hmean = torch.empty(rows, dtype=torch.float32).pin_memory()
+    hrstd = torch.empty(rows, dtype=torch.float32).pin_memory()
+    dx = torch.empty_like(hx, device=device)
+    dy = torch.empty_like(dx)
+    dp = {k: torch.empty_like(v, device=device) for k, v in hp.items()}
+    dmean = torch.empty(rows, dtype=torch.float32, device=device)
+    drstd = torch.empty(rows, dtype=torch.float32, device=device)
+    h2d = hx.numel() * hx.element_size() + sum(v.numel() * v.element_size() for v in hp.values())
+    d2h = hy.numel() * hy.element_size() + (8 * rows if w.op == "layernorm" else 0)
+
+    def step():
+        dx.copy_(hx, non_blocking=True)
+        for k in hp:
+            dp[k].copy_(hp[k], non_blocking=True)
+        if w.op == "softmax":
+            tf.tf_softmax_fwd(dx, dy)
+        elif w.op == "layernorm":
+            tf.tf_layernorm_fwd(dx, dp["gamma"], dp["beta"], w.eps, dy, dmean, drstd)
+            hmean.copy_(dmean, non_blocking=True)
+            hrstd.copy_(drstd, non_blocking=True)
+        else:
+            tf.tf_rmsnorm_fwd(dx, dp["w"], w.eps, dy)
+        hy.copy_(dy, non_blocking=True)
+
+    for _ in range(warmup):
+        step()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(steps):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b), h2d, d2h
+
+
+# ---------------------------------------------------------------------------------------------------------
+# arms
+# ---------------------------------------------------------------------------------------------------------
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2512_09196_b200 as tf
+    from paper_2512_09196_b200 import inputs
+
+    rank, local_rank, world = dist_env()
+    if args.gpus != world and world > 1:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+
+    # weak scaling: every rank owns one full batch (rows are independent; there is no exchange step)
+    base = inputs.config(1)
+    w = inputs.Workload(base.name, base.op, base.dt, base.rows, base.cols, seed=base.seed + 1000 * rank, x_mean=base.x_mean,
+                        x_std=base.x_std, eps=base.eps, scale=base.scale, shift=base.shift)
+    data = w.generate()
+    case = DeviceCase(w, data, device)
+    tuned = tf.tf_tune(w.op, w.rows, w.cols, w.dt) if not args.no_tune else {"plan": tf.tf_query_choice(w.op, w.rows, w.cols, w.dt)}
+
+    steps, warmup = args.steps, max(args.warmup, 3)
+    for _ in range(warmup):
+        case.step()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = tf.tf_launch_count()
+    with ClockSampler(local_rank) as clk:
+        start.record()
+        for _ in range(steps):
+            case.step()
+        end.record()
+        torch.cuda.synchronize()
+    launches = tf.tf_launch_count() - launches0
+    ms = start.elapsed_time(end)
+    if world > 1:
+        t = torch.tensor([ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        ms = float(t.item())
+    tf.tf_device_status()
+
+    e2e_steps = max(3, min(steps, 20))
+    e2e_ms, h2d, d2h = time_e2e(w, data, device, e2e_steps, 3)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        bytes_step = case.bytes_per_step
+        value = world * bytes_step * steps / (ms * 1e-3) / 1e9
+        per_launch_gbs = bytes_step / (ms * 1e-3 / steps) / 1e9
+        line = {
+            "metric": "achieved HBM GB/s (algorithmic bytes / device time)", "value": value, "unit": "GB/s",
+            "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "op": w.op, "storage": w.dtype_name, "rows_per_gpu": w.rows, "cols": w.cols,
+                       "algorithmic_bytes_per_step": bytes_step, "plan": tuned["plan"],
+                       "l2": f"rotating {case.sets} buffer sets ({case.sets * case.footprint / 1e9:.2f} GB) > 126 MB L2",
+                       "sharding": "independent row batches per GPU, no collective"},
+            "pct_of_nominal_8000": 100 * per_launch_gbs / NOMINAL_HBM_GBS,
+            "pct_of_measured_peak": 100 * per_launch_gbs / peak,
+            "roofline": {"bound": "hbm", "achieved": per_launch_gbs, "peak": peak, "peak_kind": f"of {peak_kind}",
+                         "unit": "GB/s", "frac": per_launch_gbs / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+            "e2e": {"value": world * bytes_step * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                    "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": launches,
+            "clocks": clk.summary(),
+            "tune": {k: tuned[k] for k in tuned if k != "plan"},
+        }
+        line["cpu_baseline"] = cpu_baseline(w, data) if world == 1 else None
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on this machine's host cores."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    from paper_2512_09196_b200 import inputs
+    w = inputs.config(1)
+    data = w.generate()
+    steps, warmup = args.steps, args.warmup
+    probe = max(time_oracle(w, data, 64), 1e-6) / 64                      # seconds per row
+    budget = 120.0 / max(1, steps + warmup)
+    rows = int(max(1, min(w.rows, min(0.25, budget) / probe)))
+    for _ in range(warmup):
+        time_oracle(w, data, rows)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        time_oracle(w, data, rows)
+    sec = time.perf_counter() - t0
+    value = w.algorithmic_bytes(rows) * steps / sec / 1e9
+    sample = f"first {rows} of {w.rows} rows per step"
+    print(json.dumps({
+        "impl": "reference", "metric": "achieved HBM GB/s (algorithmic bytes / device time)", "value": value, "unit": "GB/s",
+        "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": 1e3 * sec / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "op": w.op, "storage": w.dtype_name, "rows_per_step": rows, "cols": w.cols},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# tables: the other configurations and the shape sweep (not bench lines)
+# ---------------------------------------------------------------------------------------------------------
+def run_table(args):
+    import torch
+    import paper_2512_09196_b200 as tf
+    from paper_2512_09196_b200 import inputs
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    peak, peak_kind = measured_peak()
+    if args.table == "configs":
+        points = [inputs.config(i) for i in range(4)]
+    else:
+        points = inputs.sweep()
+        if args.filter:
+            points = [p for p in points if args.filter in p.name]
+    out_dir = ROOT / "gpurun_out"
+    out_dir.mkdir(exist_ok=True)
+    rows_out = []
+    for w in points:
+        data = w.generate()
+        case = DeviceCase(w, data, device)
+        heur = tf.tf_query_choice(w.op, w.rows, w.cols, w.dt)
+        reps = max(20, min(400, int(0.05 / max(1e-6, case.bytes_per_step / 5e12))))
+        tf.tf_clear_cache()
+        ms_h = case.time_steps(reps, 5)
+        tuned = tf.tf_tune(w.op, w.rows, w.cols, w.dt) if not args.no_tune else {"plan": heur, "timed": 0}
+        ms_t = case.time_steps(reps, 5)
+        us = 1e3 * ms_t / reps
+        gbs = case.bytes_per_step / (us * 1e-6) / 1e9
+        row = {"workload": w.name, "op": w.op, "dtype": w.dtype_name, "rows": w.rows, "cols": w.cols,
+               "bytes": case.bytes_per_step, "heuristic_plan": heur, "heuristic_us": 1e3 * ms_h / reps,
+               "plan": tuned["plan"], "timed_candidates": tuned.get("timed"), "us": us, "gbs": gbs,
+               "pct_of_8000": 100 * gbs / NOMINAL_HBM_GBS, f"pct_of_{peak_kind}_{peak:.0f}": 100 * gbs / peak}
+        if args.cpu:
+            cb = cpu_baseline(w, data, budget_s=6.0)
+            row["oracle_gbs"], row["oracle_sample"] = cb["value"], cb["sample"]
+        rows_out.append(row)
+        print(json.dumps(row), flush=True)
+        del case
+        torch.cuda.empty_cache()
+    (out_dir / f"table_{args.table}.json").write_text(json.dumps(rows_out, indent=1))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--table", choices=["configs", "sweep"], default=None)
+    ap.add_argument("--filter", default=None)
+    ap.add_argument("--no-tune", action="store_true")
+    ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 10 if args.steps is None else args.steps
+        args.warmup = 3 if args.warmup is None else args.warmup
+        return run_reference(args)
+    args.steps = 5000 if args.steps is None else args.steps
+    args.warmup = 50 if args.warmup is None else args.warmup
+    import __graft_entry__
+    __graft_entry__.build()
+    if args.table:
+        return run_table(args)
+    run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

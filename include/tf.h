@@ -1,0 +1,111 @@
+/* tf.h — C ABI of libtf.so: fused row-wise reduce-then-normalise forward kernels for NVIDIA B200
+ * (sm_100a), with a measure-and-keep tuner.
+ *
+ * The ops are the memory-bound kernel class the TritonForge paper's loop is aimed at (Section 2 lists
+ * "softmax variants" and fused operators among the hand-optimised Triton kernels it wants to automate);
+ * the paper defines none of them, so each declaration below states the standard definition it computes.
+ * tf_tune is that paper's Algorithm 1 in miniature: candidates are proposed, run, timed on the device
+ * and kept only if the measured time improves on the best so far.
+ *
+ * Conventions for every *_fwd entry point
+ *   Memory     All tensor pointers are DEVICE memory owned by the caller, on the current CUDA device.
+ *              The library keeps no reference after the call returns and allocates nothing.
+ *   Layout     x and y are dense row-major [rows, cols] (row stride = cols); gamma/beta/weight are [cols];
+ *              mean/rstd are [rows], always fp32.  x, y and the parameters share one element type `dt`.
+ *   Alignment  Any.  A 16-byte aligned x, y and parameters with cols * sizeof(element) a multiple of 16
+ *              unlock the vectorised and TMA-staged variants; anything else runs on the generic variant.
+ *   Aliasing   y == x (exactly) is allowed; partial overlap is undefined.
+ *   Async      Work is enqueued on `cuda_stream` (a cudaStream_t; NULL = the default stream) and the call
+ *              returns without synchronising.
+ *   Numerics   Arithmetic in fp32, one round-to-nearest-even conversion to the output type at the end,
+ *              subnormal results kept (never flushed to zero).
+ *   Errors     Return codes only; arguments are checked before any CUDA call.  rows == 0 is a no-op.
+ *   Threads    Entry points may be called from several host threads.
+ */
+#ifndef TF_H_
+#define TF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TF_OK = 0,
+    TF_ERR_INVALID_ARG = 1,   /* null required pointer, rows < 0, cols <= 0, bad enum, eps negative or NaN */
+    TF_ERR_UNSUPPORTED = 2,   /* size overflow, or a forced plan that cannot run this shape */
+    TF_ERR_CUDA = 3,          /* a CUDA call failed: see tf_last_cuda_error() */
+    TF_ERR_TIMEOUT = 4,       /* a bounded device-side wait gave up: see tf_device_status() */
+    TF_ERR_NOMEM = 5          /* tf_tune could not allocate its scratch tensors */
+} tf_status;
+
+typedef enum { TF_F32 = 0, TF_BF16 = 1 } tf_dtype;
+typedef enum { TF_OP_SOFTMAX = 0, TF_OP_LAYERNORM = 1, TF_OP_RMSNORM = 2 } tf_op;
+
+/* Softmax over the last axis: y[r,j] = exp(x[r,j] - m_r) / sum_k exp(x[r,k] - m_r), m_r = max_k x[r,k].
+ * No temperature.  A mask is expressed in the data: x = -inf gives exactly +0; a row that is -inf
+ * throughout gives +0 everywhere (not NaN). */
+tf_status tf_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
+
+/* LayerNorm: mu_r = mean_j x[r,j]; var_r = mean_j (x[r,j] - mu_r)^2 (divisor cols);
+ * rstd_r = 1/sqrt(var_r + eps); y[r,j] = (x[r,j] - mu_r) * rstd_r * gamma[j] + beta[j].
+ * gamma and beta are required.  mean and rstd are optional outputs (NULL to skip). */
+tf_status tf_layernorm_fwd(const void* x, const void* gamma, const void* beta, void* y, float* mean, float* rstd,
+                           int64_t rows, int64_t cols, float eps, tf_dtype dt, void* cuda_stream);
+
+/* RMSNorm: rrms_r = 1/sqrt(mean_j x[r,j]^2 + eps); y[r,j] = x[r,j] * rrms_r * weight[j], rounded once.
+ * weight is required; rstd (= rrms) is an optional output. */
+tf_status tf_rmsnorm_fwd(const void* x, const void* weight, void* y, float* rstd, int64_t rows, int64_t cols,
+                         float eps, tf_dtype dt, void* cuda_stream);
+
+/* Measure-and-keep tuning for one (op, rows, cols, dt) on the current device (Algorithm 1 of the paper,
+ * with the hand-written launch plans as proposals): starting from the heuristic plan as incumbent, every
+ * candidate plan that can launch is run on library-owned scratch tensors, its output is checked against
+ * the incumbent's, it is timed with CUDA events (3 warm-up + 5 timed launches, median; the paper's
+ * Section 3.4 protocol) on rotating buffers larger than L2, and it replaces the incumbent only if it is
+ * at least 2% faster.  The winner is cached in memory (and in the file named by the TF_TUNE_CACHE
+ * environment variable, if set) and used by later *_fwd calls with the same key.  Blocking; allocates and
+ * frees its own scratch; assumes 16-byte aligned tensors. */
+tf_status tf_tune(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);
+
+/* Result of the last tf_tune on this thread: number of candidates timed, median microseconds of the
+ * heuristic plan and of the winner.  Any pointer may be NULL. */
+tf_status tf_tune_report(int* candidates_timed, float* heuristic_us, float* best_us);
+
+const char* tf_status_string(tf_status s);
+
+/* cudaError_t value behind the most recent TF_ERR_CUDA on the calling thread (0 if none). */
+int tf_last_cuda_error(void);
+
+/* Synchronises the current device, then returns TF_ERR_TIMEOUT if any kernel since the last call gave up
+ * on a bounded wait (its output rows are then undefined), else TF_OK.  Clears the flag. */
+tf_status tf_device_status(void);
+
+/* ---- test and bench hooks ------------------------------------------------------------------------- */
+
+/* Plans are written as "variant:key=value,..." e.g. "cta:threads=256,vpt=2", "warp:lanes=8,vpt=1,rpg=4",
+ * "tma:threads=512,cluster=4,stages=1", "stream:threads=256".  tf_force_plan makes every later call of `op`
+ * use that plan (NULL or "" returns to automatic choice); a forced plan that cannot run a given shape
+ * makes the call return TF_ERR_UNSUPPORTED. */
+tf_status tf_force_plan(tf_op op, const char* plan);
+
+/* Writes the plan the dispatcher would use now for this problem (forced > tuned > heuristic), assuming
+ * 16-byte aligned tensors if aligned != 0. */
+tf_status tf_query_choice(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int aligned, char* buf, size_t n);
+
+/* Number of candidate plans tf_tune would consider for this problem, and the index-th of them as text. */
+int tf_candidate_count(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);
+tf_status tf_candidate(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int index, char* buf, size_t n);
+
+/* Forgets every tuned plan (in memory only). */
+void tf_clear_cache(void);
+
+/* Number of kernels this library has launched since it was loaded (all threads). */
+int64_t tf_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TF_H_ */

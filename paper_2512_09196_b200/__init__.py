@@ -1,0 +1,193 @@
+"""Row-wise softmax / LayerNorm / RMSNorm forward kernels for B200 behind a C ABI (``libtf.so``).
+
+This module is the thin binding: it marshals torch tensors (used only as device memory and for the
+current stream) into the C calls declared in ``include/tf.h`` and does no arithmetic of its own.
+There is no fallback: if ``libtf.so`` has not been built, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+_HERE = Path(__file__).resolve().parent
+LIB_PATH = _HERE / "libtf.so"
+
+TF_F32, TF_BF16 = 0, 1
+TF_OP_SOFTMAX, TF_OP_LAYERNORM, TF_OP_RMSNORM = 0, 1, 2
+OP_CODE = {"softmax": TF_OP_SOFTMAX, "layernorm": TF_OP_LAYERNORM, "rmsnorm": TF_OP_RMSNORM}
+TF_OK = 0
+STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3: "TF_ERR_CUDA", 4: "TF_ERR_TIMEOUT",
+                5: "TF_ERR_NOMEM"}
+
+# every symbol include/tf.h declares
+EXPORTS = ("tf_softmax_fwd", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_report", "tf_status_string",
+           "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
+           "tf_candidate", "tf_clear_cache", "tf_launch_count")
+
+
+class TfError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        detail = ""
+        if status == 3 and _lib is not None:
+            detail = f" (cudaError {_lib.tf_last_cuda_error()})"
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}{detail}")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built (``python -m paper_2512_09196_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(f"{LIB_PATH} is missing: build it first (python -m paper_2512_09196_b200.build); "
+                               "there is no fallback path")
+        L = ctypes.CDLL(str(LIB_PATH))
+        vp, i64, i32, f32, cp, sz = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float, ctypes.c_char_p,
+                                     ctypes.c_size_t)
+        L.tf_softmax_fwd.argtypes = [vp, vp, i64, i64, i32, vp]
+        L.tf_layernorm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, vp]
+        L.tf_rmsnorm_fwd.argtypes = [vp, vp, vp, vp, i64, i64, f32, i32, vp]
+        L.tf_tune.argtypes = [i32, i64, i64, i32]
+        L.tf_tune_report.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(f32)]
+        L.tf_status_string.argtypes = [i32]
+        L.tf_status_string.restype = cp
+        L.tf_last_cuda_error.argtypes = []
+        L.tf_device_status.argtypes = []
+        L.tf_force_plan.argtypes = [i32, cp]
+        L.tf_query_choice.argtypes = [i32, i64, i64, i32, i32, ctypes.c_char_p, sz]
+        L.tf_candidate_count.argtypes = [i32, i64, i64, i32]
+        L.tf_candidate.argtypes = [i32, i64, i64, i32, i32, ctypes.c_char_p, sz]
+        L.tf_clear_cache.argtypes = []
+        L.tf_clear_cache.restype = None
+        L.tf_launch_count.argtypes = []
+        L.tf_launch_count.restype = i64
+        for name in ("tf_softmax_fwd", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_report",
+                     "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice",
+                     "tf_candidate_count", "tf_candidate"):
+            getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def _dt(t) -> int:
+    import torch
+    if t.dtype == torch.float32:
+        return TF_F32
+    if t.dtype == torch.bfloat16:
+        return TF_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}: fp32 and bf16 only")
+
+
+def _check2d(x, name="x"):
+    if not x.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if x.dim() != 2 or not x.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous [rows, cols] tensor")
+
+
+def _stream(x) -> int:
+    import torch
+    return torch.cuda.current_stream(x.device).cuda_stream
+
+
+def _ok(status: int, where: str):
+    if status != TF_OK:
+        raise TfError(status, where)
+
+
+def tf_softmax_fwd(x, y=None):
+    """Softmax over the last axis of a contiguous CUDA [rows, cols] tensor (fp32 or bf16); ``y`` may alias ``x``."""
+    import torch
+    _check2d(x)
+    if y is None:
+        y = torch.empty_like(x)
+    rows, cols = x.shape
+    with torch.cuda.device(x.device):
+        _ok(lib().tf_softmax_fwd(x.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)), "tf_softmax_fwd")
+    return y
+
+
+def tf_layernorm_fwd(x, gamma, beta, eps: float, y=None, mean=None, rstd=None, want_stats: bool = True):
+    """LayerNorm forward; returns ``(y, mean, rstd)`` (fp32 [rows] statistics, or None if ``want_stats`` is False
+    and none were passed in)."""
+    import torch
+    _check2d(x)
+    rows, cols = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    if want_stats and mean is None:
+        mean = torch.empty(rows, dtype=torch.float32, device=x.device)
+    if want_stats and rstd is None:
+        rstd = torch.empty(rows, dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        _ok(lib().tf_layernorm_fwd(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(),
+                                   mean.data_ptr() if mean is not None else None,
+                                   rstd.data_ptr() if rstd is not None else None,
+                                   rows, cols, eps, _dt(x), _stream(x)), "tf_layernorm_fwd")
+    return y, mean, rstd
+
+
+def tf_rmsnorm_fwd(x, weight, eps: float, y=None, rstd=None, want_rstd: bool = False):
+    """RMSNorm forward; returns ``(y, rstd)`` (``rstd`` is None unless requested or passed in)."""
+    import torch
+    _check2d(x)
+    rows, cols = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    if want_rstd and rstd is None:
+        rstd = torch.empty(rows, dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        _ok(lib().tf_rmsnorm_fwd(x.data_ptr(), weight.data_ptr(), y.data_ptr(),
+                                 rstd.data_ptr() if rstd is not None else None, rows, cols, eps, _dt(x), _stream(x)),
+            "tf_rmsnorm_fwd")
+    return y, rstd
+
+
+def tf_tune(op, rows: int, cols: int, dt: int) -> dict:
+    """Times the candidate plans for this problem on the current device, caches the winner, and returns
+    ``{"timed": n, "heuristic_us": a, "best_us": b, "plan": "..."}``."""
+    code = OP_CODE[op] if isinstance(op, str) else int(op)
+    _ok(lib().tf_tune(code, rows, cols, dt), "tf_tune")
+    n, a, b = ctypes.c_int(), ctypes.c_float(), ctypes.c_float()
+    lib().tf_tune_report(ctypes.byref(n), ctypes.byref(a), ctypes.byref(b))
+    return {"timed": n.value, "heuristic_us": a.value, "best_us": b.value, "plan": tf_query_choice(code, rows, cols, dt)}
+
+
+def tf_force_plan(op, plan: str | None):
+    code = OP_CODE[op] if isinstance(op, str) else int(op)
+    _ok(lib().tf_force_plan(code, plan.encode() if plan else None), "tf_force_plan")
+
+
+def tf_query_choice(op, rows: int, cols: int, dt: int, aligned: bool = True) -> str:
+    code = OP_CODE[op] if isinstance(op, str) else int(op)
+    buf = ctypes.create_string_buffer(256)
+    _ok(lib().tf_query_choice(code, rows, cols, dt, int(aligned), buf, 256), "tf_query_choice")
+    return buf.value.decode()
+
+
+def tf_candidates(op, rows: int, cols: int, dt: int) -> list[str]:
+    code = OP_CODE[op] if isinstance(op, str) else int(op)
+    n = lib().tf_candidate_count(code, rows, cols, dt)
+    if n < 0:
+        raise TfError(1, "tf_candidate_count")
+    out = []
+    buf = ctypes.create_string_buffer(256)
+    for i in range(n):
+        _ok(lib().tf_candidate(code, rows, cols, dt, i, buf, 256), "tf_candidate")
+        out.append(buf.value.decode())
+    return out
+
+
+def tf_device_status():
+    _ok(lib().tf_device_status(), "tf_device_status")
+
+
+def tf_clear_cache():
+    lib().tf_clear_cache()
+
+
+def tf_launch_count() -> int:
+    return int(lib().tf_launch_count())

@@ -1,0 +1,624 @@
+// C ABI of libtf.so: argument checks, plan choice (forced > tuned > heuristic), the measure-and-keep tuner
+// and its cache.  The kernels live in tf_rowreg.cu, tf_tma.cu and tf_stream.cu.
+#include <algorithm>
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "../../include/tf.h"
+#include "tf_common.cuh"
+
+namespace tf {
+namespace {
+
+// ------------------------------------------------------------------------------------------------
+// process-wide state
+// ------------------------------------------------------------------------------------------------
+__device__ int g_status_word;               // set by kernels whose bounded waits gave up
+
+thread_local int t_last_cuda_error = 0;
+thread_local int t_tune_timed = 0;
+thread_local float t_tune_heur_us = 0.f, t_tune_best_us = 0.f;
+std::atomic<int64_t> g_launches{0};
+
+std::mutex g_mu;                            // guards everything below
+struct DevState { DeviceInfo info; int* status = nullptr; bool ok = false; };
+DevState g_dev[64];
+bool g_forced[OP_COUNT] = {false, false, false};
+Plan g_forced_plan[OP_COUNT];
+using Key = std::tuple<int, int, int, int64_t, int64_t>;      // device, op, dt, rows, cols
+std::map<Key, Plan> g_cache;
+bool g_cache_file_loaded = false;
+
+tf_status cuda_fail(cudaError_t e) {
+    t_last_cuda_error = static_cast<int>(e);
+    cudaGetLastError();                     // launch-configuration errors are not sticky: clear them
+    return TF_ERR_CUDA;
+}
+
+// Per-device facts, read once.  No allocation: the status word is a __device__ variable of this module.
+tf_status device_state(DevState** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return TF_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DevState& d = g_dev[dev];
+    if (!d.ok) {
+        int sms = 0, smem = 0;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) return cuda_fail(e);
+        void* p = nullptr;
+        if ((e = cudaGetSymbolAddress(&p, g_status_word)) != cudaSuccess) return cuda_fail(e);
+        d.info.ordinal = dev; d.info.sms = sms; d.info.smem_optin = smem; d.info.max_cluster = kMaxCluster;
+        d.status = static_cast<int*>(p);
+        d.ok = true;
+    }
+    *out = &d;
+    return TF_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// plans as text
+// ------------------------------------------------------------------------------------------------
+const char* kVariantName[V_COUNT] = {"warp", "cta", "tma", "stream", "pipe"};
+
+std::string plan_to_string(const Plan& p) {
+    char b[160];
+    switch (p.variant) {
+        case V_WARP: snprintf(b, sizeof b, "warp:threads=%d,lanes=%d,vpt=%d,rpg=%d,persist=%d", p.threads, p.lanes, p.vpt, p.rpg, p.persist); break;
+        case V_CTA: snprintf(b, sizeof b, "cta:threads=%d,vpt=%d,cluster=%d,persist=%d", p.threads, p.vpt, p.cluster, p.persist); break;
+        case V_TMA: snprintf(b, sizeof b, "tma:threads=%d,cluster=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.cluster, p.stages, p.chunk, p.persist); break;
+        case V_PIPE: snprintf(b, sizeof b, "pipe:threads=%d,lanes=%d,vpt=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.lanes, p.vpt, p.stages, p.chunk, p.persist); break;
+        default: snprintf(b, sizeof b, "stream:threads=%d,lanes=%d,persist=%d", p.threads, p.lanes, p.persist); break;
+    }
+    return b;
+}
+
+bool plan_from_string(const char* s, Plan& out) {
+    Plan p;
+    const char* colon = strchr(s, ':');
+    std::string name = colon ? std::string(s, colon - s) : std::string(s);
+    int v = -1;
+    for (int i = 0; i < V_COUNT; ++i) if (name == kVariantName[i]) v = i;
+    if (v < 0) return false;
+    p.variant = v;
+    if (v == V_STREAM) p.lanes = 0;
+    if (v == V_PIPE) { p.persist = 1; p.stages = 4; p.chunk = 32768; }
+    const char* q = colon ? colon + 1 : s + strlen(s);
+    while (*q) {
+        const char* eq = strchr(q, '=');
+        if (!eq) return false;
+        std::string key(q, eq - q);
+        char* end = nullptr;
+        long val = strtol(eq + 1, &end, 10);
+        if (end == eq + 1) return false;
+        if (key == "threads") p.threads = val; else if (key == "lanes") p.lanes = val; else if (key == "vpt") p.vpt = val;
+        else if (key == "rpg") p.rpg = val; else if (key == "cluster") p.cluster = val; else if (key == "stages") p.stages = val;
+        else if (key == "chunk") p.chunk = val; else if (key == "persist") p.persist = val; else return false;
+        q = (*end == ',') ? end + 1 : end;
+        if (*end && *end != ',') return false;
+    }
+    if (p.persist < 0) return false;
+    out = p;
+    return true;
+}
+
+// ------------------------------------------------------------------------------------------------
+// plan support / launch
+// ------------------------------------------------------------------------------------------------
+bool supports(const Plan& p, const Args& a, const DeviceInfo& d) {
+    switch (p.variant) {
+        case V_WARP: return supports_warp(p, a, d);
+        case V_CTA: return supports_cta(p, a, d);
+        case V_TMA: return supports_tma(p, a, d);
+        case V_STREAM: return supports_stream(p, a, d);
+        case V_PIPE: return supports_pipe(p, a, d);
+    }
+    return false;
+}
+
+cudaError_t launch(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    switch (p.variant) {
+        case V_WARP: return launch_warp(p, a, d, st);
+        case V_CTA: return launch_cta(p, a, d, st);
+        case V_TMA: return launch_tma(p, a, d, st);
+        case V_PIPE: return launch_pipe(p, a, d, st);
+        default: return launch_stream(p, a, d, st);
+    }
+}
+
+int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+}  // namespace
+
+cudaError_t ensure_max_smem(const void* fn, const DeviceInfo& d) {
+    static std::mutex mu;
+    static std::map<std::pair<const void*, int>, bool> done;
+    std::lock_guard<std::mutex> lk(mu);
+    bool& ok = done[std::make_pair(fn, d.ordinal)];
+    if (ok) return cudaSuccess;
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, fn);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin - static_cast<int>(fa.sharedSizeBytes));
+    if (e == cudaSuccess) ok = true;
+    return e;
+}
+
+namespace {
+
+// Default plan by row size (bytes); tf_tune may overturn it.
+Plan heuristic(const Args& a, const DeviceInfo& d) {
+    Plan p;
+    const int64_t row_bytes = a.cols * elem_size(a.dt);
+    if (!vector_ok(a)) {
+        p.variant = V_STREAM;
+        p.lanes = (a.cols <= 2048) ? 32 : 0;
+        p.threads = (a.cols <= 2048) ? 256 : (a.cols <= 65536 ? 512 : 1024);
+        return p;
+    }
+    const int64_t nvec = row_bytes / 16;
+    if (nvec <= 128) {
+        p.variant = V_WARP;
+        p.threads = 256;
+        if (nvec <= 8) { p.lanes = 8; p.vpt = 1; p.rpg = 4; }
+        else if (nvec <= 16) { p.lanes = 16; p.vpt = 1; p.rpg = 4; }
+        else if (nvec <= 32) { p.lanes = 32; p.vpt = 1; p.rpg = 4; }
+        else if (nvec <= 64) { p.lanes = 32; p.vpt = 2; p.rpg = 2; }
+        else { p.lanes = 32; p.vpt = 4; p.rpg = 1; }
+        return p;
+    }
+    if (nvec <= 8192) {
+        p.variant = V_CTA;
+        if (nvec <= 1024) { p.vpt = 2; p.threads = std::max(64, round_up(static_cast<int>((nvec + 1) / 2), 32)); }
+        else if (nvec <= 2048) { p.vpt = 4; p.threads = round_up(static_cast<int>((nvec + 3) / 4), 32); }
+        else if (nvec <= 4096) { p.vpt = 8; p.threads = round_up(static_cast<int>((nvec + 7) / 8), 32); }
+        else { p.vpt = 8; p.cluster = 2; p.threads = round_up(static_cast<int>((nvec + 15) / 16), 32); }
+        return p;
+    }
+    // long rows: shared-memory staging, slices of at most 64 KiB
+    p.variant = V_TMA;
+    p.threads = 512;
+    p.stages = 1;
+    p.chunk = 8192;
+    int cl = 1;
+    while (cl < kMaxCluster && row_bytes > static_cast<int64_t>(cl) * 65536) cl *= 2;
+    p.cluster = cl;
+    if (!supports_tma(p, a, d)) {           // longer than a full cluster of shared memory can hold
+        Plan s;
+        s.variant = V_STREAM; s.lanes = 0; s.threads = 1024;
+        return s;
+    }
+    return p;
+}
+
+// The finite proposal list of the tuner: launch geometries around the row size.  Only plans whose geometry
+// holds the row are returned.
+std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
+    std::vector<Plan> out;
+    auto add = [&](Plan p) {
+        if (!supports(p, a, d)) return;
+        const std::string s = plan_to_string(p);
+        for (const Plan& q : out) if (plan_to_string(q) == s) return;
+        out.push_back(p);
+    };
+    add(heuristic(a, d));
+    if (!vector_ok(a)) {
+        for (int lanes : {32, 0}) for (int th : {128, 256, 512, 1024}) { Plan p; p.variant = V_STREAM; p.lanes = lanes; p.threads = th; add(p); }
+        return out;
+    }
+    const int64_t nvec = a.cols * elem_size(a.dt) / 16;
+    // warp-group variants
+    for (int lanes : {8, 16, 32})
+        for (int vpt : {1, 2, 4, 8})
+            for (int rpg : {1, 2, 4}) {
+                if (nvec > static_cast<int64_t>(lanes) * vpt) continue;
+                if (nvec * 2 <= static_cast<int64_t>(lanes) * vpt && !(lanes == 8 && vpt == 1)) continue;   // over half idle
+                for (int th : {128, 256}) {
+                    Plan p; p.variant = V_WARP; p.lanes = lanes; p.vpt = vpt; p.rpg = rpg; p.threads = th;
+                    add(p);
+                    p.persist = 8; add(p);
+                }
+            }
+    // CTA / cluster register variants
+    for (int cl : {1, 2, 4, 8})
+        for (int vpt : {1, 2, 4, 8}) {
+            const int64_t per = (nvec + cl - 1) / cl;
+            const int64_t th = (per + vpt - 1) / vpt;
+            if (th > 1024 || th < 48) continue;
+            Plan p; p.variant = V_CTA; p.cluster = cl; p.vpt = vpt; p.threads = round_up(static_cast<int>(th), 32);
+            add(p);
+            if (a.rows > 4LL * d.sms) { p.persist = std::max(1, 2048 / p.threads); add(p); }
+        }
+    // persistent pipeline: (lanes, vpt) that hold the row, ring shapes that fit one or two CTAs per SM
+    {
+        const int combos[][2] = {{8, 1}, {16, 1}, {32, 1}, {32, 2}, {32, 4}, {32, 8}, {64, 2}, {64, 4}, {64, 8}, {128, 2},
+                                 {128, 4}, {128, 8}, {256, 2}, {256, 4}, {256, 8}, {512, 4}};
+        const int64_t row_bytes = nvec * 16;
+        const int64_t param_bytes = a.op == OP_SOFTMAX ? 0 : row_bytes * (a.op == OP_LAYERNORM ? 2 : 1);
+        for (const auto& c : combos) {
+            const int64_t cap = static_cast<int64_t>(c[0]) * c[1];
+            if (nvec > cap || (nvec * 2 <= cap && c[0] != 8)) continue;
+            for (int th : {256, 512}) {
+                if (th < c[0]) continue;
+                for (int persist : {1, 2})
+                    for (int stage_bytes : {16384, 32768, 65536}) {
+                        if (stage_bytes < row_bytes) continue;
+                        const int64_t budget = (persist == 1 ? 200 : 98) * 1024 - param_bytes;
+                        const int stages = static_cast<int>(std::min<int64_t>(8, budget / stage_bytes));
+                        if (stages < 2) continue;
+                        Plan p; p.variant = V_PIPE; p.lanes = c[0]; p.vpt = c[1]; p.threads = th; p.persist = persist;
+                        p.chunk = stage_bytes; p.stages = stages;
+                        add(p);
+                        if (stages >= 6) { p.stages = stages / 2; add(p); }
+                    }
+            }
+        }
+    }
+    // shared-memory staged variants
+    if (nvec >= 512)
+        for (int cl : {1, 2, 4, 8}) {
+            const int64_t slice = (nvec + cl - 1) / cl * 16;
+            if (slice < 8192) continue;
+            for (int th : {256, 512, 1024})
+                for (int chunk : {8192, 32768}) {
+                    Plan p; p.variant = V_TMA; p.cluster = cl; p.threads = th; p.chunk = chunk; p.stages = 1;
+                    add(p);
+                    if (slice * 2 <= 100 * 1024 && a.rows > 2LL * d.sms) { p.stages = 2; p.persist = std::max(1, static_cast<int>(200 * 1024 / (2 * slice))); add(p); }
+                }
+        }
+    return out;
+}
+
+// ------------------------------------------------------------------------------------------------
+// tune cache
+// ------------------------------------------------------------------------------------------------
+void load_cache_file_locked() {
+    if (g_cache_file_loaded) return;
+    g_cache_file_loaded = true;
+    const char* path = getenv("TF_TUNE_CACHE");
+    if (!path || !*path) return;
+    FILE* f = fopen(path, "r");
+    if (!f) return;
+    char line[512];
+    while (fgets(line, sizeof line, f)) {
+        int dev, op, dt; long long rows, cols; char plan[256];
+        if (sscanf(line, "%d %d %d %lld %lld %255s", &dev, &op, &dt, &rows, &cols, plan) != 6) continue;
+        Plan p;
+        if (op < 0 || op >= OP_COUNT || (dt != DT_F32 && dt != DT_BF16) || !plan_from_string(plan, p)) continue;
+        g_cache[Key(dev, op, dt, rows, cols)] = p;
+    }
+    fclose(f);
+}
+
+void save_cache_file_locked() {
+    const char* path = getenv("TF_TUNE_CACHE");
+    if (!path || !*path) return;
+    FILE* f = fopen(path, "w");
+    if (!f) return;
+    for (const auto& kv : g_cache)
+        fprintf(f, "%d %d %d %lld %lld %s\n", std::get<0>(kv.first), std::get<1>(kv.first), std::get<2>(kv.first),
+                static_cast<long long>(std::get<3>(kv.first)), static_cast<long long>(std::get<4>(kv.first)),
+                plan_to_string(kv.second).c_str());
+    fclose(f);
+}
+
+// forced > tuned (if it still fits: the tuner assumed aligned tensors) > heuristic
+Plan choose(const Args& a, const DeviceInfo& d, bool* forced) {
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (g_forced[a.op]) { *forced = true; return g_forced_plan[a.op]; }
+        load_cache_file_locked();
+        auto it = g_cache.find(Key(d.ordinal, a.op, a.dt, a.rows, a.cols));
+        if (it != g_cache.end() && supports(it->second, a, d)) return it->second;
+    }
+    return heuristic(a, d);
+}
+
+tf_status run(const Args& a0, void* stream) {
+    if (a0.rows == 0) return TF_OK;
+    DevState* ds = nullptr;
+    tf_status s = device_state(&ds);
+    if (s != TF_OK) return s;
+    Args a = a0;
+    a.status = ds->status;
+    bool forced = false;
+    const Plan p = choose(a, ds->info, &forced);
+    if (!supports(p, a, ds->info)) return TF_ERR_UNSUPPORTED;
+    cudaError_t e = launch(p, a, ds->info, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TF_OK : cuda_fail(e);
+}
+
+bool bad_shape(int64_t rows, int64_t cols, int dt) {  // dt arrives as an int so that out-of-range enum values are caught
+    return rows < 0 || cols <= 0 || (dt != DT_F32 && dt != DT_BF16); }
+bool too_big(int64_t rows, int64_t cols) { return rows > 0 && cols > (INT64_MAX / 8) / rows; }
+bool bad_eps(float eps) { return !(eps >= 0.f) || std::isinf(eps); }
+
+// ------------------------------------------------------------------------------------------------
+// tuner helpers (device side)
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t hash32(uint64_t i) {
+    uint64_t z = i + 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return static_cast<uint32_t>((z ^ (z >> 31)) >> 32);
+}
+
+// Scratch contents for timing: lo + (hi - lo) * u, u a hash of the index in [0, 1).
+template <int DT>
+__global__ void k_fill(void* out, int64_t n, float lo, float hi, uint64_t salt) {
+    using E = Elem<DT>;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n; i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const float u = static_cast<float>(hash32(i + salt) >> 8) * (1.0f / 16777216.0f);
+        static_cast<typename E::scalar*>(out)[i] = E::from_float(lo + (hi - lo) * u);
+    }
+}
+
+// Counts elements where two outputs of the same problem disagree by more than two plans of this library
+// legitimately can (each is within the parity tolerance of the exact result).
+template <int DT>
+__global__ void k_mismatch(const void* a, const void* b, int64_t n, unsigned long long* count) {
+    using E = Elem<DT>;
+    unsigned long long local = 0;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n; i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const float x = E::to_float(static_cast<const typename E::scalar*>(a)[i]);
+        const float y = E::to_float(static_cast<const typename E::scalar*>(b)[i]);
+        const float tol = (DT == DT_F32 ? 2e-5f : 1.6e-2f) * fmaxf(fabsf(x), fabsf(y)) + 1e-5f;
+        if (!(fabsf(x - y) <= tol)) ++local;
+    }
+    if (local) atomicAdd(count, local);
+}
+
+struct Scratch {
+    std::vector<void*> ptrs;
+    ~Scratch() { for (void* p : ptrs) cudaFree(p); }
+    void* get(size_t bytes) {
+        void* p = nullptr;
+        if (cudaMalloc(&p, std::max<size_t>(bytes, 16)) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        ptrs.push_back(p);
+        return p;
+    }
+};
+
+}  // namespace
+}  // namespace tf
+
+using namespace tf;
+
+extern "C" {
+
+tf_status tf_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols, tf_dtype dt, void* stream) {
+    if (bad_shape(rows, cols, dt) || (rows > 0 && (!x || !y))) return TF_ERR_INVALID_ARG;
+    if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
+    Args a{OP_SOFTMAX, dt, x, nullptr, nullptr, y, nullptr, nullptr, rows, cols, 0.f, nullptr};
+    return run(a, stream);
+}
+
+tf_status tf_layernorm_fwd(const void* x, const void* gamma, const void* beta, void* y, float* mean, float* rstd,
+                           int64_t rows, int64_t cols, float eps, tf_dtype dt, void* stream) {
+    if (bad_shape(rows, cols, dt) || bad_eps(eps) || !gamma || !beta || (rows > 0 && (!x || !y))) return TF_ERR_INVALID_ARG;
+    if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
+    Args a{OP_LAYERNORM, dt, x, gamma, beta, y, mean, rstd, rows, cols, eps, nullptr};
+    return run(a, stream);
+}
+
+tf_status tf_rmsnorm_fwd(const void* x, const void* weight, void* y, float* rstd, int64_t rows, int64_t cols, float eps,
+                         tf_dtype dt, void* stream) {
+    if (bad_shape(rows, cols, dt) || bad_eps(eps) || !weight || (rows > 0 && (!x || !y))) return TF_ERR_INVALID_ARG;
+    if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
+    Args a{OP_RMSNORM, dt, x, weight, nullptr, y, nullptr, rstd, rows, cols, eps, nullptr};
+    return run(a, stream);
+}
+
+tf_status tf_tune(tf_op op_, int64_t rows, int64_t cols, tf_dtype dt_) {
+    const int op = op_, dt = dt_;
+    if (op < 0 || op >= OP_COUNT || bad_shape(rows, cols, dt) || rows == 0) return TF_ERR_INVALID_ARG;
+    if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
+    DevState* ds = nullptr;
+    tf_status s = device_state(&ds);
+    if (s != TF_OK) return s;
+    const DeviceInfo& dev = ds->info;
+    const int es = elem_size(dt);
+    const size_t tensor_bytes = static_cast<size_t>(rows) * cols * es;
+    // K rotating (x, y) sets so that a timed batch never re-touches lines still in L2 (> 2x its size in total)
+    const size_t want = 256u << 20;
+    const int K = static_cast<int>(std::min<size_t>(64, std::max<size_t>(1, (want + 2 * tensor_bytes - 1) / (2 * tensor_bytes))));
+
+    Scratch sc;
+    std::vector<void*> xs(K), ys(K);
+    for (int k = 0; k < K; ++k) { xs[k] = sc.get(tensor_bytes); ys[k] = sc.get(tensor_bytes); if (!xs[k] || !ys[k]) return TF_ERR_NOMEM; }
+    void* yref = sc.get(tensor_bytes);
+    void* p0 = sc.get(static_cast<size_t>(cols) * es);
+    void* p1 = sc.get(static_cast<size_t>(cols) * es);
+    float* mean = static_cast<float*>(sc.get(static_cast<size_t>(rows) * 4));
+    float* rstd = static_cast<float*>(sc.get(static_cast<size_t>(rows) * 4));
+    unsigned long long* mism = static_cast<unsigned long long*>(sc.get(8));
+    if (!yref || !p0 || !p1 || !mean || !rstd || !mism) return TF_ERR_NOMEM;
+
+    cudaStream_t st = nullptr;
+    cudaEvent_t ev[2] = {nullptr, nullptr};
+    cudaError_t e;
+    if ((e = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+    auto cleanup = [&]() { if (ev[0]) cudaEventDestroy(ev[0]); if (ev[1]) cudaEventDestroy(ev[1]); cudaStreamDestroy(st); };
+    if ((e = cudaEventCreate(&ev[0])) != cudaSuccess || (e = cudaEventCreate(&ev[1])) != cudaSuccess) { cleanup(); return cuda_fail(e); }
+
+    const int64_t n = rows * cols;
+    const int fill_grid = static_cast<int>(std::min<int64_t>((n + 255) / 256, static_cast<int64_t>(dev.sms) * 16));
+    for (int k = 0; k < K; ++k) {
+        if (dt == DT_F32) k_fill<DT_F32><<<fill_grid, 256, 0, st>>>(xs[k], n, -4.f, 4.f, 1000003ull * k);
+        else k_fill<DT_BF16><<<fill_grid, 256, 0, st>>>(xs[k], n, -4.f, 4.f, 1000003ull * k);
+    }
+    const int pgrid = static_cast<int>(std::min<int64_t>((cols + 255) / 256, 1024));
+    if (dt == DT_F32) { k_fill<DT_F32><<<pgrid, 256, 0, st>>>(p0, cols, 0.5f, 1.5f, 7); k_fill<DT_F32><<<pgrid, 256, 0, st>>>(p1, cols, -0.5f, 0.5f, 11); }
+    else { k_fill<DT_BF16><<<pgrid, 256, 0, st>>>(p0, cols, 0.5f, 1.5f, 7); k_fill<DT_BF16><<<pgrid, 256, 0, st>>>(p1, cols, -0.5f, 0.5f, 11); }
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) { cleanup(); return cuda_fail(e); }
+
+    auto args_for = [&](int k, void* y) {
+        Args a{op, dt, xs[k], p0, p1, y, op == OP_LAYERNORM ? mean : nullptr, op == OP_LAYERNORM ? rstd : nullptr,
+               rows, cols, op == OP_SOFTMAX ? 0.f : 1e-5f, ds->status};
+        return a;
+    };
+    // BuildRun: can it launch, and does it reproduce the incumbent's output?
+    auto runs_and_matches = [&](const Plan& p, bool is_reference) -> bool {
+        void* y = is_reference ? yref : ys[0];
+        if (launch(p, args_for(0, y), dev, st) != cudaSuccess) { cudaGetLastError(); return false; }
+        if (cudaStreamSynchronize(st) != cudaSuccess) return false;
+        int flag = 0;                                        // a bounded wait gave up: the candidate is dropped
+        if (cudaMemcpy(&flag, ds->status, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) return false;
+        if (flag != 0) { cudaMemset(ds->status, 0, sizeof flag); return false; }
+        if (is_reference) return true;
+        cudaMemsetAsync(mism, 0, 8, st);
+        const int g = static_cast<int>(std::min<int64_t>((n + 255) / 256, static_cast<int64_t>(dev.sms) * 16));
+        if (dt == DT_F32) k_mismatch<DT_F32><<<g, 256, 0, st>>>(ys[0], yref, n, mism);
+        else k_mismatch<DT_BF16><<<g, 256, 0, st>>>(ys[0], yref, n, mism);
+        unsigned long long h = 1;
+        if (cudaMemcpyAsync(&h, mism, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return false;
+        return h == 0;
+    };
+    // Profile: 3 warm-up + 5 timed batches of K launches (one per buffer set), CUDA events, median per launch.
+    auto profile = [&](const Plan& p, float* us) -> bool {
+        float t[5];
+        for (int rep = 0; rep < 8; ++rep) {
+            if (rep >= 3) cudaEventRecord(ev[0], st);
+            for (int k = 0; k < K; ++k)
+                if (launch(p, args_for(k, ys[k]), dev, st) != cudaSuccess) { cudaGetLastError(); return false; }
+            if (rep >= 3) {
+                cudaEventRecord(ev[1], st);
+                if (cudaEventSynchronize(ev[1]) != cudaSuccess) return false;
+                float ms = 0.f;
+                cudaEventElapsedTime(&ms, ev[0], ev[1]);
+                t[rep - 3] = ms * 1000.f / K;
+            }
+        }
+        std::sort(t, t + 5);
+        *us = t[2];
+        return true;
+    };
+
+    const Args probe = args_for(0, ys[0]);
+    Plan best = heuristic(probe, dev);
+    float best_us = 0.f;
+    int timed = 0;
+    if (!supports(best, probe, dev) || !runs_and_matches(best, true) || !profile(best, &best_us)) { cleanup(); return cuda_fail(cudaGetLastError()); }
+    ++timed;
+    const float heur_us = best_us;
+    const std::string best0 = plan_to_string(best);
+    for (const Plan& c : candidates(probe, dev)) {
+        if (plan_to_string(c) == best0) continue;
+        float us = 0.f;
+        if (!runs_and_matches(c, false)) continue;          // failed BuildRun: dropped, never cached
+        if (!profile(c, &us)) continue;
+        ++timed;
+        if (us < 0.98f * best_us) { best = c; best_us = us; }       // Arbiter: accept only a measured improvement
+    }
+    cleanup();
+    t_tune_timed = timed; t_tune_heur_us = heur_us; t_tune_best_us = best_us;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        load_cache_file_locked();
+        g_cache[Key(dev.ordinal, op, dt, rows, cols)] = best;
+        save_cache_file_locked();
+    }
+    return TF_OK;
+}
+
+tf_status tf_tune_report(int* candidates_timed, float* heuristic_us, float* best_us) {
+    if (candidates_timed) *candidates_timed = t_tune_timed;
+    if (heuristic_us) *heuristic_us = t_tune_heur_us;
+    if (best_us) *best_us = t_tune_best_us;
+    return TF_OK;
+}
+
+const char* tf_status_string(tf_status s) {
+    switch (s) {
+        case TF_OK: return "ok";
+        case TF_ERR_INVALID_ARG: return "invalid argument";
+        case TF_ERR_UNSUPPORTED: return "unsupported size or plan";
+        case TF_ERR_CUDA: return "CUDA error";
+        case TF_ERR_TIMEOUT: return "device-side wait timed out";
+        case TF_ERR_NOMEM: return "out of device memory";
+    }
+    return "unknown status";
+}
+
+int tf_last_cuda_error(void) { return t_last_cuda_error; }
+
+tf_status tf_device_status(void) {
+    DevState* ds = nullptr;
+    tf_status s = device_state(&ds);
+    if (s != TF_OK) return s;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e);
+    int h = 0, zero = 0;
+    if ((e = cudaMemcpy(&h, ds->status, sizeof h, cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(e);
+    if (h != 0 && (e = cudaMemcpy(ds->status, &zero, sizeof zero, cudaMemcpyHostToDevice)) != cudaSuccess) return cuda_fail(e);
+    return h == 0 ? TF_OK : TF_ERR_TIMEOUT;
+}
+
+tf_status tf_force_plan(tf_op op_, const char* plan) {
+    const int op = op_;
+    if (op < 0 || op >= OP_COUNT) return TF_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!plan || !*plan) { g_forced[op] = false; return TF_OK; }
+    Plan p;
+    if (!plan_from_string(plan, p)) return TF_ERR_INVALID_ARG;
+    g_forced_plan[op] = p;
+    g_forced[op] = true;
+    return TF_OK;
+}
+
+static bool fake_args(tf_op op_, int64_t rows, int64_t cols, tf_dtype dt_, int aligned, Args* a) {
+    const int op = op_, dt = dt_;
+    if (op < 0 || op >= OP_COUNT || bad_shape(rows, cols, dt)) return false;
+    const void* base = reinterpret_cast<const void*>(static_cast<uintptr_t>(aligned ? 256 : 258));
+    *a = Args{op, dt, base, base, base, const_cast<void*>(base), nullptr, nullptr, rows, cols, 0.f, nullptr};
+    return true;
+}
+
+tf_status tf_query_choice(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int aligned, char* buf, size_t n) {
+    Args a;
+    if (!buf || n == 0 || !fake_args(op, rows, cols, dt, aligned, &a)) return TF_ERR_INVALID_ARG;
+    DevState* ds = nullptr;
+    tf_status s = device_state(&ds);
+    if (s != TF_OK) return s;
+    bool forced = false;
+    snprintf(buf, n, "%s", plan_to_string(choose(a, ds->info, &forced)).c_str());
+    return TF_OK;
+}
+
+int tf_candidate_count(tf_op op, int64_t rows, int64_t cols, tf_dtype dt) {
+    Args a;
+    DevState* ds = nullptr;
+    if (!fake_args(op, rows, cols, dt, 1, &a) || device_state(&ds) != TF_OK) return -1;
+    return static_cast<int>(candidates(a, ds->info).size());
+}
+
+tf_status tf_candidate(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int index, char* buf, size_t n) {
+    Args a;
+    if (!buf || n == 0 || !fake_args(op, rows, cols, dt, 1, &a)) return TF_ERR_INVALID_ARG;
+    DevState* ds = nullptr;
+    tf_status s = device_state(&ds);
+    if (s != TF_OK) return s;
+    const std::vector<Plan> c = candidates(a, ds->info);
+    if (index < 0 || index >= static_cast<int>(c.size())) return TF_ERR_INVALID_ARG;
+    snprintf(buf, n, "%s", plan_to_string(c[index]).c_str());
+    return TF_OK;
+}
+
+void tf_clear_cache(void) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_cache.clear();
+}
+
+int64_t tf_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,155 @@
+// Device-side building blocks shared by the kernel files: 16-byte vector access, bf16 <-> fp32,
+// the exponential used by softmax, warp and CTA reductions, and the per-op partial-combine rules.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tf_plan.h"
+
+namespace tf {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kNegInf = -__builtin_huge_valf();
+
+// ---------------------------------------------------------------------------------------------
+// Element traits: a 16-byte vector holds NE elements.
+// ---------------------------------------------------------------------------------------------
+template <int DT> struct Elem;
+
+template <> struct Elem<DT_F32> {
+    static constexpr int NE = 4;
+    static constexpr int SIZE = 4;
+    using scalar = float;
+    static __device__ __forceinline__ void unpack(const uint4& v, float (&f)[NE]) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&f)[NE]) {
+        return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+    }
+    static __device__ __forceinline__ float to_float(float s) { return s; }
+    static __device__ __forceinline__ float from_float(float f) { return f; }
+};
+
+template <> struct Elem<DT_BF16> {
+    static constexpr int NE = 8;
+    static constexpr int SIZE = 2;
+    using scalar = uint16_t;
+    // a bf16 is the upper half of an fp32: widening is a shift (exact)
+    static __device__ __forceinline__ void unpack(const uint4& v, float (&f)[NE]) {
+        f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xFFFF0000u);
+        f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xFFFF0000u);
+        f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xFFFF0000u);
+        f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xFFFF0000u);
+    }
+    // round-to-nearest-even, subnormals kept (cvt.rn.bf16x2.f32)
+    static __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+        __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&p);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&f)[NE]) {
+        return make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+    }
+    static __device__ __forceinline__ float to_float(uint16_t s) { return __uint_as_float(static_cast<uint32_t>(s) << 16); }
+    static __device__ __forceinline__ uint16_t from_float(float f) {
+        __nv_bfloat16 b = __float2bfloat16_rn(f);
+        return *reinterpret_cast<uint16_t*>(&b);
+    }
+};
+
+// ---------------------------------------------------------------------------------------------
+// Global memory access.  x is read once and y written once: both bypass L1 allocation / are marked
+// streaming so that they do not push the (re-read) parameter vectors out of the caches.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 ld_param(const uint4* p) { return __ldg(p); }
+
+// 2^t with subnormal results kept (no .ftz): ex2.approx.f32, relative error about 2^-22.  Used once per row.
+__device__ __forceinline__ float ex2(float t) {
+    float r;
+    asm("ex2.approx.f32 %0, %1;" : "=f"(r) : "f"(t));
+    return r;
+}
+// 2^t as a single MUFU operation; results below 2^-126 are flushed to zero.  The softmax paths use it
+// per element on exponents that carry a bias of +kExpBias (folded into the constant of the FMA that forms
+// the exponent): the largest term is then 2^64, a term is only flushed when its true value is below
+// 2^-190 (zero in fp32 and bf16 anyway), and the bias cancels in e / sum(e) -- the final, non-flushing
+// multiply by 1/sum produces subnormal outputs correctly.
+constexpr float kExpBias = 64.0f;
+__device__ __forceinline__ float ex2_ftz(float t) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
+    return r;
+}
+// Exponent offset of a slice whose maximum is m: exponents are x*log2e + exp_offset(m).  One rounding,
+// shared by every element of the slice, so it cancels between numerator and denominator.
+__device__ __forceinline__ float exp_offset(float m) { return (m == kNegInf) ? 0.f : fmaf(-m, kLog2e, kExpBias); }
+
+// Largest element of a 16-byte vector (NaNs are ignored, as by fmaxf).
+template <int DT> __device__ __forceinline__ float vec_max(const uint4& v) {
+    if constexpr (DT == DT_F32) {
+        return fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)), fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
+    } else {
+        const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&v.x), b = *reinterpret_cast<const __nv_bfloat162*>(&v.y);
+        const __nv_bfloat162 c = *reinterpret_cast<const __nv_bfloat162*>(&v.z), d = *reinterpret_cast<const __nv_bfloat162*>(&v.w);
+        const __nv_bfloat162 m = __hmax2(__hmax2(a, b), __hmax2(c, d));
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(&m);
+        return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Reductions.
+// ---------------------------------------------------------------------------------------------
+struct SumOp { static __device__ __forceinline__ float apply(float a, float b) { return a + b; } static __device__ __forceinline__ float identity() { return 0.f; } };
+struct MaxOp { static __device__ __forceinline__ float apply(float a, float b) { return fmaxf(a, b); } static __device__ __forceinline__ float identity() { return kNegInf; } };
+
+template <class Op, int LANES>
+__device__ __forceinline__ float group_reduce(float v) {      // all LANES lanes of the group get the result
+#pragma unroll
+    for (int o = LANES / 2; o > 0; o >>= 1) v = Op::apply(v, __shfl_xor_sync(0xFFFFFFFFu, v, o, LANES));
+    return v;
+}
+
+// CTA-wide reduction through `buf` (>= 32 floats of shared memory, private to this call site until the
+// next __syncthreads after a later use of a DIFFERENT buffer).  Every thread gets the result.
+template <class Op>
+__device__ __forceinline__ float cta_reduce(float v, float* buf) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+    v = group_reduce<Op, 32>(v);
+    if (lane == 0) buf[warp] = v;
+    __syncthreads();
+    float r = (lane < nwarp) ? buf[lane] : Op::identity();
+    return group_reduce<Op, 32>(r);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Combining per-slice partial results of one row (used across the CTAs of a cluster).
+// ---------------------------------------------------------------------------------------------
+
+// softmax: partial k is (o_k, s_k) with o_k = exp_offset(slice max) (+inf marks an all -inf slice) and
+// s_k = sum_j 2^(x_j*log2e + o_k).  With O = min_k o_k (the offset of the row maximum) the row total is
+// S = sum_k s_k * 2^(O - o_k), and slice k's terms rescale by 2^(O - o_k): every exponent is then
+// x_j*log2e + O, the same expression in numerator and denominator.
+__device__ __forceinline__ float softmax_rescale(float O, float ok) { return (ok == -kNegInf) ? 0.f : ex2(O - ok); }
+
+// LayerNorm (Chan et al. pairwise update): (n, mean, M2) of the union of two disjoint slices.
+struct MomentPartial { float n, mean, m2; };
+__device__ __forceinline__ MomentPartial chan_combine(const MomentPartial& a, const MomentPartial& b) {
+    if (b.n == 0.f) return a;
+    if (a.n == 0.f) return b;
+    const float n = a.n + b.n, d = b.mean - a.mean, f = b.n / n;
+    return MomentPartial{n, fmaf(d, f, a.mean), a.m2 + b.m2 + d * d * a.n * f};
+}
+
+}  // namespace tf

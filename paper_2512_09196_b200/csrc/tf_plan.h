@@ -1,0 +1,80 @@
+// Launch plans: which hand-written variant runs a problem and with what geometry.  Host and device.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tf {
+
+enum : int { DT_F32 = 0, DT_BF16 = 1 };
+enum : int { OP_SOFTMAX = 0, OP_LAYERNORM = 1, OP_RMSNORM = 2, OP_COUNT = 3 };
+
+enum Variant : int {
+    V_WARP = 0,     // a group of 8/16/32 lanes holds one row in registers; several rows per warp for narrow rows
+    V_CTA = 1,      // a CTA (or a cluster of CTAs) holds one row in registers; 16-byte coalesced loads
+    V_TMA = 2,      // each CTA of a cluster stages its slice of the row in shared memory with bulk async copies
+    V_STREAM = 3,   // generic: scalar accesses, several passes over the row, any alignment and length
+    V_PIPE = 4,     // persistent CTAs: a producer thread streams row tiles into a shared-memory ring, consumer warps normalise
+    V_COUNT = 5
+};
+
+struct Plan {
+    int variant = V_STREAM;
+    int threads = 256;   // CTA size
+    int lanes = 32;      // V_WARP / V_PIPE: threads per row
+    int vpt = 1;         // V_WARP / V_CTA / V_PIPE: 16-byte vectors held per thread
+    int rpg = 1;         // V_WARP: rows a group has in flight per iteration
+    int cluster = 1;     // V_CTA / V_TMA: CTAs sharing one row
+    int stages = 1;      // V_TMA / V_PIPE: shared-memory ring depth
+    int chunk = 8192;    // V_TMA: bytes per bulk copy (one mbarrier each); V_PIPE: bytes per stage
+    int persist = 0;     // 0: grid covers all rows once; k > 0: k CTAs per SM looping over rows (V_PIPE: always >= 1)
+};
+
+struct Args {
+    int op, dt;
+    const void* x;
+    const void* p0;      // gamma (LayerNorm) / weight (RMSNorm)
+    const void* p1;      // beta (LayerNorm)
+    void* y;
+    float* mean;         // LayerNorm, nullable
+    float* rstd;         // LayerNorm / RMSNorm, nullable
+    int64_t rows, cols;
+    float eps;
+    int* status;         // device word that bounded waits set when they give up
+};
+
+struct DeviceInfo {
+    int ordinal = -1;
+    int sms = 0;
+    int smem_optin = 0;          // max dynamic shared memory per CTA, bytes
+    int max_cluster = 8;
+};
+
+// Geometry limits shared by the dispatcher and the kernels.
+constexpr int kMaxCluster = 8;
+constexpr int kMaxChunks = 32;       // bulk copies (mbarriers) per slice
+constexpr int kMaxStages = 3;
+
+// One launcher per kernel family.  `supports_*` is the host-side check that the plan's geometry can hold
+// the row; `launch_*` enqueues on `stream` and returns the launch error.
+bool supports_warp(const Plan&, const Args&, const DeviceInfo&);
+bool supports_cta(const Plan&, const Args&, const DeviceInfo&);
+bool supports_tma(const Plan&, const Args&, const DeviceInfo&);
+bool supports_stream(const Plan&, const Args&, const DeviceInfo&);
+bool supports_pipe(const Plan&, const Args&, const DeviceInfo&);
+cudaError_t launch_warp(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+cudaError_t launch_cta(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+cudaError_t launch_tma(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+cudaError_t launch_stream(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+cudaError_t launch_pipe(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+
+// Raises a kernel's dynamic shared-memory limit to the device's opt-in maximum, once per kernel and device.
+cudaError_t ensure_max_smem(const void* fn, const DeviceInfo&);
+
+inline int elem_size(int dt) { return dt == DT_F32 ? 4 : 2; }
+inline bool vector_ok(const Args& a) {          // 16-byte vectors usable on every tensor
+    auto al = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+    return (a.cols * elem_size(a.dt)) % 16 == 0 && al(a.x) && al(a.y) && al(a.p0) && al(a.p1);
+}
+
+}  // namespace tf

@@ -1,0 +1,254 @@
+"""GPU parity: every variant forced explicitly and the automatic choice, both dtypes, edge shapes, against the
+CPU oracle, through the C ABI."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_09196_b200 as tf
+from paper_2512_09196_b200 import inputs
+from paper_2512_09196_b200.inputs import BF16, F32, Workload
+import parity
+
+pytestmark = pytest.mark.gpu
+
+OPS = ("softmax", "layernorm", "rmsnorm")
+EPS = {"softmax": 0.0, "layernorm": 1e-5, "rmsnorm": 1e-6}
+
+
+def wl(op, dt, rows, cols, seed=7, **kw):
+    kw.setdefault("x_mean", 0.3)
+    kw.setdefault("x_std", 2.0)
+    return Workload(f"{op}-{dt}-{rows}x{cols}", op, dt, rows, cols, seed=seed, eps=EPS[op], **kw)
+
+
+@pytest.fixture(autouse=True)
+def _auto_plans():
+    yield
+    for op in OPS:
+        tf.tf_force_plan(op, None)
+
+
+# ------------------------------------------------------------------ automatic choice over edge shapes
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("cols", [1, 2, 3, 7, 8, 31, 32, 33, 64, 100, 256, 1000, 1001, 1024, 4096, 4097, 5120, 12288, 40000])
+def test_auto_edge_cols(op, dt, cols):
+    for rows in (1, 37):
+        fails = parity.parity(wl(op, dt, rows, cols, seed=cols))
+        assert not fails, f"{tf.tf_query_choice(op, rows, cols, dt, (cols * (4 if dt == F32 else 2)) % 16 == 0)}: {fails}"
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("rows", [2, 147, 148, 149, 1000])
+def test_auto_edge_rows(op, rows):
+    for dt, cols in ((F32, 520), (BF16, 2048)):
+        assert not parity.parity(wl(op, dt, rows, cols, seed=rows))
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_long_rows_take_the_cluster_path(op, dt):
+    cols = 131072 if dt == BF16 else 65536 + 64
+    w = wl(op, dt, 21, cols)
+    assert tf.tf_query_choice(op, 21, cols, dt).startswith("tma:")
+    assert not parity.parity(w)
+    w2 = wl(op, dt, 3, 1 << 20)          # 2-4 MiB rows: more than a cluster of shared memory holds
+    assert tf.tf_query_choice(op, 3, 1 << 20, dt).startswith(("tma:", "stream:"))
+    assert not parity.parity(w2)
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_misaligned_base_and_inplace(op, dt):
+    for cols in (64, 1000, 4096):
+        w = wl(op, dt, 19, cols)
+        assert not parity.parity(w, offset=1), "misaligned base"
+        assert not parity.parity(w, inplace=True), "in place"
+        assert not parity.parity(w, offset=3, inplace=True), "misaligned and in place"
+
+
+def test_rows_zero_is_a_noop_and_bad_args_are_rejected():
+    x = torch.empty((0, 16), device="cuda")
+    tf.tf_softmax_fwd(x)
+    L = tf.lib()
+    buf = torch.zeros(64, device="cuda")
+    p = buf.data_ptr()
+    assert L.tf_softmax_fwd(None, p, 2, 8, 0, None) == 1
+    assert L.tf_softmax_fwd(p, p, -1, 8, 0, None) == 1
+    assert L.tf_softmax_fwd(p, p, 2, 0, 0, None) == 1
+    assert L.tf_softmax_fwd(p, p, 2, 8, 5, None) == 1
+    assert L.tf_layernorm_fwd(p, None, p, p, None, None, 2, 8, 1e-5, 0, None) == 1
+    assert L.tf_layernorm_fwd(p, p, p, p, None, None, 2, 8, -1.0, 0, None) == 1
+    assert L.tf_layernorm_fwd(p, p, p, p, None, None, 2, 8, float("nan"), 0, None) == 1
+    assert L.tf_rmsnorm_fwd(p, None, p, None, 2, 8, 1e-6, 0, None) == 1
+    assert L.tf_softmax_fwd(p, p, 1 << 40, 1 << 40, 0, None) == 2
+    assert L.tf_tune(7, 2, 8, 0) == 1
+    assert L.tf_force_plan(0, b"nonsense:threads=3") == 1
+    assert L.tf_status_string(2) == b"unsupported size or plan"
+
+
+# ------------------------------------------------------------------ special values
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_softmax_masks_fully_masked_rows_and_subnormals(dt):
+    for cols, plan in ((64, None), (4096, None), (131072, None), (4096, "stream:threads=256,lanes=0")):
+        tf.tf_force_plan("softmax", plan)
+        w = Workload("m", "softmax", dt, 24, cols, seed=5, x_std=10.0, mask_step=max(1, cols // 16 + 3))
+        data = w.generate()
+        x = data["x"]
+        ninf = np.float32(-np.inf) if dt == F32 else np.uint16(0xFF80)
+        x[3, :] = ninf                                     # fully masked row -> all +0
+        x[5, : cols // 2] = ninf                           # masked head instead of tail
+        x[7, ::2] = ninf                                   # alternating
+        x[9, 0] = np.float32(75.0) if dt == F32 else np.uint16(0x4296)   # 75.0: pushes much of the row to e^-88 and below
+        got, ref = parity.run_gpu(w, data), parity.run_oracle(w, data)
+        assert not parity.check(w, data, got, ref)
+        assert not got["y"][3].any()
+        if dt == BF16 and cols >= 4096:
+            sub = (ref["y"] > 0) & (ref["y"] < 0x0080)
+            assert sub.any(), "the case is meant to produce bf16 subnormal outputs"
+
+
+@pytest.mark.parametrize("op", ["layernorm", "rmsnorm"])
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_norm_degenerate_rows(op, dt):
+    for cols in (8, 512, 8192):
+        w = wl(op, dt, 6, cols)
+        data = w.generate()
+        x = data["x"]
+        x[1, :] = x[1, 0]                                  # constant row: variance 0
+        x[2, :] = 0                                        # all zeros
+        if dt == F32:
+            x[3, :] *= np.float32(1e4)
+        got, ref = parity.run_gpu(w, data), parity.run_oracle(w, data)
+        assert not parity.check(w, data, got, ref)
+
+
+def test_rmsnorm_outliers_and_optional_rstd():
+    w = Workload("o", "rmsnorm", BF16, 64, 8192, seed=2, eps=1e-6, outlier_p=0.01, outlier_factor=100.0,
+                 scale=("normal", 1.0, 0.1))
+    assert not parity.parity(w)
+    assert not parity.parity(w, rms_rstd=False)
+
+
+def test_nan_row_does_not_leak_into_other_rows():
+    w = wl("softmax", F32, 8, 1024)
+    data = w.generate()
+    data["x"][4, 100] = np.nan
+    got, ref = parity.run_gpu(w, data), parity.run_oracle(w, data)
+    keep = [r for r in range(8) if r != 4]
+    sub = {"x": data["x"][keep]}
+    assert not parity.check(w, sub, {"y": got["y"][keep]}, {"y": ref["y"][keep], "y64": ref["y64"][keep]})
+    assert np.isnan(got["y"][4]).any()
+
+
+# ------------------------------------------------------------------ every variant, forced
+
+WARP_PLANS = [(l, v, r) for (l, v, r) in [(8, 1, 1), (8, 1, 2), (8, 1, 4), (8, 2, 1), (8, 2, 2), (16, 1, 1), (16, 1, 2),
+                                           (16, 1, 4), (16, 2, 1), (16, 2, 2), (32, 1, 1), (32, 1, 2), (32, 1, 4),
+                                           (32, 2, 1), (32, 2, 2), (32, 4, 1), (32, 4, 2), (32, 8, 1)]]
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_forced_warp_variants(op, dt):
+    ne = 4 if dt == F32 else 8
+    for lanes, vpt, rpg in WARP_PLANS:
+        cap = lanes * vpt                               # vectors the group can hold
+        for nvec in {cap, max(1, cap - 1), max(1, cap // 2 + 1)}:
+            for threads, persist in ((128, 0), (256, 1)):
+                tf.tf_force_plan(op, f"warp:threads={threads},lanes={lanes},vpt={vpt},rpg={rpg},persist={persist}")
+                fails = parity.parity(wl(op, dt, 301, nvec * ne, seed=nvec))
+                assert not fails, (lanes, vpt, rpg, nvec, threads, fails)
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+def test_forced_cta_variants(op, dt, cluster):
+    ne = 4 if dt == F32 else 8
+    for vpt in (1, 2, 4, 8):
+        for threads in (64, 256) + ((1024,) if vpt <= 2 else (512,)):
+            cap = threads * vpt * cluster
+            for nvec in {cap, cap - 1, cap - threads - 3, max(1, cap // 2 + 5)}:
+                if nvec < 1:
+                    continue
+                for persist in (0, 1):
+                    tf.tf_force_plan(op, f"cta:threads={threads},vpt={vpt},cluster={cluster},persist={persist}")
+                    rows = 9 if persist == 0 else 700
+                    fails = parity.parity(wl(op, dt, rows if nvec < 4096 else 5, nvec * ne, seed=nvec))
+                    assert not fails, (vpt, threads, cluster, nvec, persist, fails)
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+def test_forced_tma_variants(op, dt, cluster):
+    ne = 4 if dt == F32 else 8
+    for nvec in (cluster * 512, cluster * 4096 - 1, cluster * 2048 + 77, 1000):
+        for threads, stages, chunk, persist, rows in ((128, 1, 4096, 0, 7), (512, 1, 8192, 0, 7), (1024, 2, 32768, 1, 400),
+                                                       (256, 3, 16384, 1, 900), (256, 2, 1024, 2, 1300)):
+            tf.tf_force_plan(op, f"tma:threads={threads},cluster={cluster},stages={stages},chunk={chunk},persist={persist}")
+            fails = parity.parity(wl(op, dt, rows if nvec <= 4096 else min(rows, 300), nvec * ne, seed=nvec))
+            assert not fails, (cluster, nvec, threads, stages, chunk, persist, fails)
+
+
+PIPE_COMBOS = [(8, 1), (16, 1), (32, 1), (32, 2), (32, 4), (32, 8), (64, 2), (64, 4), (64, 8), (128, 2), (128, 4), (128, 8),
+               (256, 2), (256, 4), (256, 8), (512, 4)]
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_forced_pipe_variants(op, dt):
+    ne = 4 if dt == F32 else 8
+    for lanes, vpt in PIPE_COMBOS:
+        cap = lanes * vpt
+        for threads in (256, 512):
+            if threads < lanes or (vpt == 8 and threads > 256):
+                continue
+            for nvec in {cap, max(1, cap - 1), max(1, cap // 2 + 1)}:
+                for stages, chunk, persist, rows in ((2, 16384, 1, 77), (4, 32768, 1, 3000), (3, 65536, 2, 1301), (8, 8192, 1, 5000)):
+                    if chunk < nvec * 16:
+                        chunk = 65536
+                    plan = f"pipe:threads={threads},lanes={lanes},vpt={vpt},stages={stages},chunk={chunk},persist={persist}"
+                    tf.tf_force_plan(op, plan)
+                    w = wl(op, dt, rows if nvec * 16 <= 8192 else max(40, rows // 8), nvec * ne, seed=nvec)
+                    try:
+                        fails = parity.parity(w)
+                    except tf.TfError as e:
+                        assert e.status == 2, plan                     # ring does not fit shared memory: refused, not wrong
+                        continue
+                    assert not fails, (plan, nvec, fails)
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_forced_stream_variants(op, dt):
+    for lanes in (32, 0):
+        for threads in (64, 1024):
+            for cols in (1, 5, 999, 4099):
+                tf.tf_force_plan(op, f"stream:threads={threads},lanes={lanes},persist=0")
+                assert not parity.parity(wl(op, dt, 41, cols, seed=cols), offset=1)
+            tf.tf_force_plan(op, f"stream:threads={threads},lanes={lanes},persist=1")
+            assert not parity.parity(wl(op, dt, 5000, 40, seed=1))
+
+
+def test_forced_plan_that_cannot_hold_the_row_is_refused():
+    tf.tf_force_plan("softmax", "warp:threads=256,lanes=8,vpt=1,rpg=1")
+    x = torch.zeros((4, 4096), device="cuda")
+    with pytest.raises(tf.TfError) as e:
+        tf.tf_softmax_fwd(x)
+    assert e.value.status == 2
+    tf.tf_force_plan("softmax", "cta:threads=64,vpt=1,cluster=1")
+    with pytest.raises(tf.TfError):
+        tf.tf_softmax_fwd(x)
+    tf.tf_force_plan("softmax", "tma:threads=256,cluster=1,stages=3,chunk=8192")
+    with pytest.raises(tf.TfError):
+        tf.tf_softmax_fwd(torch.zeros((2, 1 << 16), device="cuda"))        # 3 x 256 KiB of shared memory
+    tf.tf_force_plan("softmax", "warp:threads=256,lanes=8,vpt=1,rpg=1")
+    xu = torch.zeros(4 * 32 + 1, device="cuda")[1:].view(4, 32)             # misaligned: vector plans refuse
+    with pytest.raises(tf.TfError):
+        tf.tf_softmax_fwd(xu)
