@@ -90,7 +90,27 @@ def _check2d(x, name="x"):
 
 def _stream(x) -> int:
     import torch
-    return torch.cuda.current_stream(x.device).cuda_stream
+    try:                                    # raw handle of the current stream without building a Stream object
+        return torch._C._cuda_getCurrentRawStream(x.device.index)
+    except AttributeError:
+        return torch.cuda.current_stream(x.device).cuda_stream
+
+
+class _on_device:
+    """Makes x's device current for the call; free when it already is."""
+    __slots__ = ("guard",)
+
+    def __init__(self, x):
+        import torch
+        self.guard = None if x.device.index == torch.cuda.current_device() else torch.cuda.device(x.device)
+
+    def __enter__(self):
+        if self.guard is not None:
+            self.guard.__enter__()
+
+    def __exit__(self, *exc):
+        if self.guard is not None:
+            self.guard.__exit__(*exc)
 
 
 def _ok(status: int, where: str):
@@ -105,7 +125,7 @@ def tf_softmax_fwd(x, y=None):
     if y is None:
         y = torch.empty_like(x)
     rows, cols = x.shape
-    with torch.cuda.device(x.device):
+    with _on_device(x):
         _ok(lib().tf_softmax_fwd(x.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)), "tf_softmax_fwd")
     return y
 
@@ -122,7 +142,7 @@ def tf_layernorm_fwd(x, gamma, beta, eps: float, y=None, mean=None, rstd=None, w
         mean = torch.empty(rows, dtype=torch.float32, device=x.device)
     if want_stats and rstd is None:
         rstd = torch.empty(rows, dtype=torch.float32, device=x.device)
-    with torch.cuda.device(x.device):
+    with _on_device(x):
         _ok(lib().tf_layernorm_fwd(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(),
                                    mean.data_ptr() if mean is not None else None,
                                    rstd.data_ptr() if rstd is not None else None,
@@ -139,7 +159,7 @@ def tf_rmsnorm_fwd(x, weight, eps: float, y=None, rstd=None, want_rstd: bool = F
         y = torch.empty_like(x)
     if want_rstd and rstd is None:
         rstd = torch.empty(rows, dtype=torch.float32, device=x.device)
-    with torch.cuda.device(x.device):
+    with _on_device(x):
         _ok(lib().tf_rmsnorm_fwd(x.data_ptr(), weight.data_ptr(), y.data_ptr(),
                                  rstd.data_ptr() if rstd is not None else None, rows, cols, eps, _dt(x), _stream(x)),
             "tf_rmsnorm_fwd")

@@ -167,15 +167,27 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         return p;
     }
     const int64_t nvec = row_bytes / 16;
-    if (nvec <= 128) {
-        p.variant = V_WARP;
-        p.threads = 256;
-        if (nvec <= 8) { p.lanes = 8; p.vpt = 1; p.rpg = 4; }
-        else if (nvec <= 16) { p.lanes = 16; p.vpt = 1; p.rpg = 4; }
-        else if (nvec <= 32) { p.lanes = 32; p.vpt = 1; p.rpg = 4; }
-        else if (nvec <= 64) { p.lanes = 32; p.vpt = 2; p.rpg = 2; }
-        else { p.lanes = 32; p.vpt = 4; p.rpg = 1; }
-        return p;
+    if (nvec <= 4096) {
+        // rows up to 64 KiB: the persistent self-feeding pipeline, one CTA of 512 threads per SM, two stages per unit
+        p.variant = V_PIPE;
+        p.threads = 512; p.persist = 1; p.stages = 2;
+        if (nvec <= 8) { p.lanes = 8; p.vpt = 1; }
+        else if (nvec <= 16) { p.lanes = 16; p.vpt = 1; }
+        else if (nvec <= 32) { p.lanes = 32; p.vpt = 1; }
+        else if (nvec <= 64) { p.lanes = 32; p.vpt = 2; }
+        else if (nvec <= 128) { p.lanes = 32; p.vpt = 4; }
+        else if (nvec <= 256) { p.lanes = 32; p.vpt = 8; }
+        else if (nvec <= 512) { p.lanes = 64; p.vpt = 8; }
+        else if (nvec <= 1024) { p.lanes = 128; p.vpt = 8; }
+        else if (nvec <= 2048) { p.lanes = 256; p.vpt = 8; }
+        else { p.lanes = 512; p.vpt = 8; }
+        const int ut = p.lanes < 32 ? 32 : p.lanes;
+        const int64_t pass_bytes = row_bytes * (ut / p.lanes);
+        const int64_t param_bytes = a.op == OP_SOFTMAX ? 0 : row_bytes * (a.op == OP_LAYERNORM ? 2 : 1);
+        const int64_t per_stage = (200 * 1024 - param_bytes) / (p.threads / ut) / p.stages;
+        p.chunk = static_cast<int>(std::max<int64_t>(pass_bytes, std::min<int64_t>(16384, per_stage) / pass_bytes * pass_bytes));
+        if (supports_pipe(p, a, d)) return p;
+        p = Plan();
     }
     if (nvec <= 8192) {
         p.variant = V_CTA;
@@ -239,27 +251,29 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
             add(p);
             if (a.rows > 4LL * d.sms) { p.persist = std::max(1, 2048 / p.threads); add(p); }
         }
-    // persistent pipeline: (lanes, vpt) that hold the row, ring shapes that fit one or two CTAs per SM
+    // persistent self-feeding pipeline: (lanes, vpt) that hold the row; rings that fit one or two CTAs per SM
     {
         const int combos[][2] = {{8, 1}, {16, 1}, {32, 1}, {32, 2}, {32, 4}, {32, 8}, {64, 2}, {64, 4}, {64, 8}, {128, 2},
-                                 {128, 4}, {128, 8}, {256, 2}, {256, 4}, {256, 8}, {512, 4}};
+                                 {128, 4}, {128, 8}, {256, 2}, {256, 4}, {256, 8}, {512, 4}, {512, 8}};
         const int64_t row_bytes = nvec * 16;
         const int64_t param_bytes = a.op == OP_SOFTMAX ? 0 : row_bytes * (a.op == OP_LAYERNORM ? 2 : 1);
         for (const auto& c : combos) {
             const int64_t cap = static_cast<int64_t>(c[0]) * c[1];
             if (nvec > cap || (nvec * 2 <= cap && c[0] != 8)) continue;
+            const int ut = c[0] < 32 ? 32 : c[0];
+            const int64_t pass_bytes = row_bytes * (ut / c[0]);
             for (int th : {256, 512}) {
-                if (th < c[0]) continue;
-                for (int persist : {1, 2})
-                    for (int stage_bytes : {16384, 32768, 65536}) {
-                        if (stage_bytes < row_bytes) continue;
-                        const int64_t budget = (persist == 1 ? 200 : 98) * 1024 - param_bytes;
-                        const int stages = static_cast<int>(std::min<int64_t>(8, budget / stage_bytes));
-                        if (stages < 2) continue;
+                if (th < ut) continue;
+                const int units = th / ut;
+                for (int persist : {1, 2, 4})
+                    for (int stages : {2, 3, 4}) {
+                        const int64_t budget = (persist == 1 ? 200 : (persist == 2 ? 98 : 48)) * 1024 - param_bytes;
+                        int64_t chunk = std::min<int64_t>(32768, budget / units / stages) / pass_bytes * pass_bytes;
+                        if (chunk < pass_bytes) continue;
                         Plan p; p.variant = V_PIPE; p.lanes = c[0]; p.vpt = c[1]; p.threads = th; p.persist = persist;
-                        p.chunk = stage_bytes; p.stages = stages;
+                        p.chunk = static_cast<int>(chunk); p.stages = stages;
                         add(p);
-                        if (stages >= 6) { p.stages = stages / 2; add(p); }
+                        if (chunk >= 4 * pass_bytes && chunk > 4096) { p.chunk = static_cast<int>(chunk / 2 / pass_bytes * pass_bytes); add(p); }
                     }
             }
         }
@@ -512,12 +526,16 @@ tf_status tf_tune(tf_op op_, int64_t rows, int64_t cols, tf_dtype dt_) {
     ++timed;
     const float heur_us = best_us;
     const std::string best0 = plan_to_string(best);
+    const char* log_env = getenv("TF_LOG");
+    const bool log = log_env && *log_env && *log_env != '0';
+    if (log) fprintf(stderr, "tf_tune: %8.2f us  %s (heuristic)\n", best_us, best0.c_str());
     for (const Plan& c : candidates(probe, dev)) {
         if (plan_to_string(c) == best0) continue;
         float us = 0.f;
         if (!runs_and_matches(c, false)) continue;          // failed BuildRun: dropped, never cached
         if (!profile(c, &us)) continue;
         ++timed;
+        if (log) fprintf(stderr, "tf_tune: %8.2f us  %s\n", us, plan_to_string(c).c_str());
         if (us < 0.98f * best_us) { best = c; best_us = us; }       // Arbiter: accept only a measured improvement
     }
     cleanup();

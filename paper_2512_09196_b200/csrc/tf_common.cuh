@@ -60,6 +60,46 @@ template <> struct Elem<DT_BF16> {
 };
 
 // ---------------------------------------------------------------------------------------------
+// Packed pairs of fp32 (Blackwell's .f32x2 arithmetic: one instruction, two IEEE results, no flushing).
+// The row arithmetic below is written on pairs, which halves its FP instruction count.
+// ---------------------------------------------------------------------------------------------
+struct F2 { unsigned long long v; };
+__device__ __forceinline__ F2 f2(float lo, float hi) { F2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "f"(lo), "f"(hi)); return r; }
+__device__ __forceinline__ F2 f2(float both) { return f2(both, both); }
+__device__ __forceinline__ void split(F2 a, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a.v)); }
+__device__ __forceinline__ float hsum(F2 a) { float lo, hi; split(a, lo, hi); return lo + hi; }
+__device__ __forceinline__ F2 fma2(F2 a, F2 b, F2 c) { F2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v)); return r; }
+__device__ __forceinline__ F2 add2(F2 a, F2 b) { F2 r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r; }
+__device__ __forceinline__ F2 sub2(F2 a, F2 b) { F2 r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r; }
+__device__ __forceinline__ F2 mul2(F2 a, F2 b) { F2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r; }
+
+// A 16-byte vector as NP pairs.
+template <int DT> struct Pairs;
+template <> struct Pairs<DT_F32> {
+    static constexpr int NP = 2;
+    static __device__ __forceinline__ void unpack(const uint4& v, F2 (&p)[NP]) {
+        p[0] = f2(__uint_as_float(v.x), __uint_as_float(v.y));
+        p[1] = f2(__uint_as_float(v.z), __uint_as_float(v.w));
+    }
+    static __device__ __forceinline__ uint4 pack(const F2 (&p)[NP]) {
+        float a, b, c, d;
+        split(p[0], a, b); split(p[1], c, d);
+        return make_uint4(__float_as_uint(a), __float_as_uint(b), __float_as_uint(c), __float_as_uint(d));
+    }
+};
+template <> struct Pairs<DT_BF16> {
+    static constexpr int NP = 4;
+    static __device__ __forceinline__ F2 widen(uint32_t w) { return f2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u)); }
+    static __device__ __forceinline__ void unpack(const uint4& v, F2 (&p)[NP]) {
+        p[0] = widen(v.x); p[1] = widen(v.y); p[2] = widen(v.z); p[3] = widen(v.w);
+    }
+    static __device__ __forceinline__ uint32_t narrow(F2 a) { float lo, hi; split(a, lo, hi); return Elem<DT_BF16>::pack2(lo, hi); }
+    static __device__ __forceinline__ uint4 pack(const F2 (&p)[NP]) {
+        return make_uint4(narrow(p[0]), narrow(p[1]), narrow(p[2]), narrow(p[3]));
+    }
+};
+
+// ---------------------------------------------------------------------------------------------
 // Global memory access.  x is read once and y written once: both bypass L1 allocation / are marked
 // streaming so that they do not push the (re-read) parameter vectors out of the caches.
 // ---------------------------------------------------------------------------------------------
@@ -91,6 +131,7 @@ __device__ __forceinline__ float ex2_ftz(float t) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
     return r;
 }
+__device__ __forceinline__ F2 ex2_ftz2(F2 t) { float lo, hi; split(t, lo, hi); return f2(ex2_ftz(lo), ex2_ftz(hi)); }
 // Exponent offset of a slice whose maximum is m: exponents are x*log2e + exp_offset(m).  One rounding,
 // shared by every element of the slice, so it cancels between numerator and denominator.
 __device__ __forceinline__ float exp_offset(float m) { return (m == kNegInf) ? 0.f : fmaf(-m, kLog2e, kExpBias); }

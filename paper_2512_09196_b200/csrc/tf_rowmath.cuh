@@ -1,6 +1,6 @@
-// Register-level row arithmetic shared by the variants that hold a row (or a slice) in registers:
-// the per-op math on NV 16-byte vectors per thread, parameterised by how partials are reduced across
-// the threads that share the row and by where the affine parameters come from.
+// Register-level row arithmetic shared by the variants that hold a row (or a slice of one) in registers:
+// the per-op math on NV 16-byte vectors per thread, written on packed fp32 pairs, parameterised by how
+// partials are reduced across the threads that share the data and by where the affine parameters come from.
 #pragma once
 
 #include "tf_common.cuh"
@@ -15,7 +15,7 @@ template <int DT> __device__ __forceinline__ uint4 fill_vec(int op) {
     return make_uint4(0, 0, 0, 0);
 }
 
-// Reducers: how a per-thread partial becomes the value for everything this group holds.
+// Reducers: how a per-thread partial becomes the value for everything the group holds.
 template <int LANES> struct GroupRed {
     __device__ __forceinline__ float sum(float v, int) const { return group_reduce<SumOp, LANES>(v); }
     __device__ __forceinline__ float max(float v, int) const { return group_reduce<MaxOp, LANES>(v); }
@@ -26,7 +26,7 @@ struct CtaRed {
     __device__ __forceinline__ float max(float v, int slot) const { return cta_reduce<MaxOp>(v, buf + 32 * slot); }
 };
 
-// Parameter access: either held in registers (V_WARP) or fetched from L1/L2 when the normalise pass needs them.
+// Parameter access: held in registers, or fetched (L1/L2 or shared memory) when the normalise pass needs them.
 template <int NV> struct HeldParams {
     uint4 g[NV], b[NV];
     __device__ __forceinline__ uint4 gamma(int v) const { return g[v]; }
@@ -40,88 +40,143 @@ struct LazyParams {
     __device__ __forceinline__ uint4 beta(int v) const { return ld_param(p1 + first + v * stride); }
 };
 
-// ---- single-group math: the group holds the entire row -----------------------------------------------
-// raw[v] invalid => filled with -inf (softmax) / 0 (norms).  slot0 alternates between calls so that a CTA
-// reducer never reuses a shared buffer that slow threads may still be reading.
+// ---- slice math ---------------------------------------------------------------------------------------
+// A group holds one SLICE of a row (possibly the whole row) as NV vectors per thread; invalid vectors are
+// filled with -inf (softmax) / 0 (norms).  Inside the slice the statistics are exact two-pass ones.  Slices
+// of one row that live in groups which cannot shuffle with one another (the warps of a multi-warp unit, the
+// CTAs of a cluster) are merged afterwards: (offset, sum) for softmax, (mean, M2) with Chan's update for
+// LayerNorm, the plain sum of squares for RMSNorm.
+struct Part { float a, b; };
+struct Total { float a, b; };        // softmax: (rescale of my slice, 1/S); LayerNorm: (mean, rstd); RMSNorm: (rrms, rrms)
+
+// `slot0` picks the reducer's shared buffers (CTA reducers alternate them between rows).  `w` receives the
+// widened values (softmax: the exponentials) for slice_finish.
+template <int OP, int DT, int NV, class Red>
+__device__ __forceinline__ Part slice_stats(const uint4 (&raw)[NV], const bool (&valid)[NV], const Red& red, int slot0,
+                                            float n_slice, F2 (&w)[NV][Pairs<DT>::NP]) {
+    using P = Pairs<DT>;
+    constexpr int NP = P::NP;
+    if constexpr (OP == OP_SOFTMAX) {
+        float m = kNegInf;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) m = fmaxf(m, vec_max<DT>(raw[v]));
+        m = red.max(m, slot0);
+        const F2 off = f2(exp_offset(m)), l2e = f2(kLog2e);
+        F2 s = f2(0.f);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            P::unpack(raw[v], w[v]);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) { w[v][i] = ex2_ftz2(fma2(w[v][i], l2e, off)); s = add2(s, w[v][i]); }
+        }
+        return Part{(m == kNegInf) ? -kNegInf : exp_offset(m), red.sum(hsum(s), slot0 + 1)};
+    } else if constexpr (OP == OP_LAYERNORM) {
+        F2 s = f2(0.f);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            P::unpack(raw[v], w[v]);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) s = add2(s, w[v][i]);
+        }
+        const float tot = red.sum(hsum(s), slot0);
+        const float mean = (n_slice > 0.f) ? tot / n_slice : 0.f;
+        const F2 mm = f2(mean);
+        F2 m2 = f2(0.f);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            if (valid[v]) {
+#pragma unroll
+                for (int i = 0; i < NP; ++i) { const F2 d = sub2(w[v][i], mm); m2 = fma2(d, d, m2); }
+            }
+        }
+        return Part{mean, red.sum(hsum(m2), slot0 + 1)};
+    } else {
+        F2 ss = f2(0.f);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            P::unpack(raw[v], w[v]);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) ss = fma2(w[v][i], w[v][i], ss);
+        }
+        return Part{red.sum(hsum(ss), slot0), 0.f};
+    }
+}
+
+// Merges K slice partials (read through get(k), element counts through count(k)) in slice order, so that
+// every holder of the same partials computes bit-identical totals.
+template <int OP, class Get, class Count>
+__device__ __forceinline__ Total combine_parts(int K, int mine, const Get& get, const Count& count, float n, float eps) {
+    if constexpr (OP == OP_SOFTMAX) {
+        float O = -kNegInf;
+        for (int k = 0; k < K; ++k) O = fminf(O, get(k).a);
+        float S = 0.f;
+        for (int k = 0; k < K; ++k) { const Part p = get(k); S = fmaf(p.b, softmax_rescale(O, p.a), S); }
+        return Total{softmax_rescale(O, get(mine).a), (S == 0.f) ? 0.f : 1.0f / S};
+    } else if constexpr (OP == OP_LAYERNORM) {
+        MomentPartial acc{0.f, 0.f, 0.f};
+        for (int k = 0; k < K; ++k) { const Part p = get(k); acc = chan_combine(acc, MomentPartial{count(k), p.a, p.b}); }
+        return Total{acc.mean, 1.0f / sqrtf(acc.m2 / n + eps)};
+    } else {
+        float tot = 0.f;
+        for (int k = 0; k < K; ++k) tot += get(k).a;
+        const float rr = 1.0f / sqrtf(tot / n + eps);
+        return Total{rr, rr};
+    }
+}
+
+// The single-slice case of combine_parts (the group holds the whole row).
+template <int OP>
+__device__ __forceinline__ Total total_of(const Part& p, float n, float eps) {
+    if constexpr (OP == OP_SOFTMAX) return Total{1.0f, (p.b == 0.f) ? 0.f : 1.0f / p.b};
+    else if constexpr (OP == OP_LAYERNORM) return Total{p.a, 1.0f / sqrtf(p.b / n + eps)};
+    else { const float rr = 1.0f / sqrtf(p.a / n + eps); return Total{rr, rr}; }
+}
+
+// SINGLE: the slice is the whole row, so softmax needs no slice rescale.
+template <int OP, int DT, int NV, bool SINGLE, class Par>
+__device__ __forceinline__ void slice_finish(const bool (&valid)[NV], F2 (&w)[NV][Pairs<DT>::NP], const Total& t, const Par& par,
+                                             uint4 (&out)[NV]) {
+    using P = Pairs<DT>;
+    constexpr int NP = P::NP;
+    const F2 ta = f2(t.a), tb = f2(t.b);
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        if constexpr (OP == OP_SOFTMAX) {
+            // two factors when slices are merged: the slice rescale may be subnormal (a slice far below the row
+            // maximum) while 1/S carries 2^-bias; their product could lose the subnormal bits.
+#pragma unroll
+            for (int i = 0; i < NP; ++i) w[v][i] = SINGLE ? mul2(w[v][i], tb) : mul2(mul2(w[v][i], ta), tb);
+            out[v] = P::pack(w[v]);
+        } else if constexpr (OP == OP_LAYERNORM) {
+            if (valid[v]) {
+                F2 g[NP], b[NP];
+                P::unpack(par.gamma(v), g);
+                P::unpack(par.beta(v), b);
+#pragma unroll
+                for (int i = 0; i < NP; ++i) w[v][i] = fma2(mul2(sub2(w[v][i], ta), tb), g[i], b[i]);
+            }
+            out[v] = P::pack(w[v]);
+        } else {
+            if (valid[v]) {
+                F2 g[NP];
+                P::unpack(par.gamma(v), g);
+#pragma unroll
+                for (int i = 0; i < NP; ++i) w[v][i] = mul2(mul2(w[v][i], ta), g[i]);
+            }
+            out[v] = P::pack(w[v]);
+        }
+    }
+}
+
+// Whole row in one group: statistics, totals and outputs in one call.  st0/st1: mean & rstd (LayerNorm), rrms (RMSNorm).
 template <int OP, int DT, int NV, class Red, class Par>
 __device__ __forceinline__ void row_math(const uint4 (&raw)[NV], const bool (&valid)[NV], const Red& red, const Par& par,
                                          int slot0, float n, float eps, uint4 (&out)[NV], float& st0, float& st1) {
-    using E = Elem<DT>;
-    constexpr int NE = E::NE;
-    if constexpr (OP == OP_SOFTMAX) {
-        float f[NV][NE];
-        float m = kNegInf;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            E::unpack(raw[v], f[v]);
-#pragma unroll
-            for (int e = 0; e < NE; ++e) m = fmaxf(m, f[v][e]);
-        }
-        m = red.max(m, slot0);
-        const float off = exp_offset(m);
-        float s = 0.f;
-#pragma unroll
-        for (int v = 0; v < NV; ++v)
-#pragma unroll
-            for (int e = 0; e < NE; ++e) { f[v][e] = ex2_ftz(fmaf(f[v][e], kLog2e, off)); s += f[v][e]; }
-        s = red.sum(s, slot0 + 1);
-        const float inv = (s == 0.f) ? 0.f : 1.0f / s;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-#pragma unroll
-            for (int e = 0; e < NE; ++e) f[v][e] *= inv;
-            out[v] = E::pack(f[v]);
-        }
-    } else if constexpr (OP == OP_LAYERNORM) {
-        float s = 0.f;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            float f[NE]; E::unpack(raw[v], f);
-#pragma unroll
-            for (int e = 0; e < NE; ++e) s += f[e];
-        }
-        const float mean = red.sum(s, slot0) / n;
-        float m2 = 0.f;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            float f[NE]; E::unpack(raw[v], f);
-            if (valid[v]) {
-#pragma unroll
-                for (int e = 0; e < NE; ++e) { const float d = f[e] - mean; m2 = fmaf(d, d, m2); }
-            }
-        }
-        const float var = red.sum(m2, slot0 + 1) / n;
-        const float rstd = 1.0f / sqrtf(var + eps);
-        st0 = mean; st1 = rstd;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            float f[NE], g[NE], b[NE];
-            E::unpack(raw[v], f);
-            if (valid[v]) { E::unpack(par.gamma(v), g); E::unpack(par.beta(v), b); }
-#pragma unroll
-            for (int e = 0; e < NE; ++e) f[e] = valid[v] ? fmaf((f[e] - mean) * rstd, g[e], b[e]) : 0.f;
-            out[v] = E::pack(f);
-        }
-    } else {
-        float ss = 0.f;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            float f[NE]; E::unpack(raw[v], f);
-#pragma unroll
-            for (int e = 0; e < NE; ++e) ss = fmaf(f[e], f[e], ss);
-        }
-        const float rr = 1.0f / sqrtf(red.sum(ss, slot0) / n + eps);
-        st0 = rr; st1 = rr;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            float f[NE], w[NE];
-            E::unpack(raw[v], f);
-            if (valid[v]) E::unpack(par.gamma(v), w);
-#pragma unroll
-            for (int e = 0; e < NE; ++e) f[e] = valid[v] ? (f[e] * rr) * w[e] : 0.f;
-            out[v] = E::pack(f);
-        }
-    }
+    F2 w[NV][Pairs<DT>::NP];
+    const Part part = slice_stats<OP, DT, NV>(raw, valid, red, slot0, n, w);
+    const Total t = total_of<OP>(part, n, eps);
+    st0 = t.a; st1 = t.b;
+    slice_finish<OP, DT, NV, true>(valid, w, t, par, out);
 }
 
 }  // namespace tf

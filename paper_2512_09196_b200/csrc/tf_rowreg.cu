@@ -129,106 +129,18 @@ __global__ void __launch_bounds__(cta_max_threads(VPT)) k_cta(const KArgs a, con
         } else {
             cg::cluster_group cl = cg::this_cluster();
             const int par_buf = it & 1;
-            auto push = [&](float p0v, float p1v) {
-                if (t < cs) {
-                    float* dst = cl.map_shared_rank(&xch[par_buf][rank][0], t);
-                    dst[0] = p0v; dst[1] = p1v;
-                }
-                cl.sync();                                               // release our writes, acquire the peers'
-            };
-            if constexpr (OP == OP_SOFTMAX) {
-                float f[VPT][NE];
-                float m = kNegInf;
-#pragma unroll
-                for (int v = 0; v < VPT; ++v) {
-                    E::unpack(raw[v], f[v]);
-#pragma unroll
-                    for (int e = 0; e < NE; ++e) m = fmaxf(m, f[v][e]);
-                }
-                m = red.max(m, slot0);
-                const float ok = exp_offset(m);
-                float s = 0.f;
-#pragma unroll
-                for (int v = 0; v < VPT; ++v)
-#pragma unroll
-                    for (int e = 0; e < NE; ++e) { f[v][e] = ex2_ftz(fmaf(f[v][e], kLog2e, ok)); s += f[v][e]; }
-                s = red.sum(s, slot0 + 1);
-                push((m == kNegInf) ? -kNegInf : ok, s);
-                float O = -kNegInf;
-                for (int k = 0; k < cs; ++k) O = fminf(O, xch[par_buf][k][0]);
-                float S = 0.f;
-                for (int k = 0; k < cs; ++k) S = fmaf(xch[par_buf][k][1], softmax_rescale(O, xch[par_buf][k][0]), S);
-                // two factors: 2^(O - ok) may be subnormal (a slice far below the row maximum) and 1/S carries 2^-bias
-                const float f1 = (m == kNegInf) ? 0.f : softmax_rescale(O, ok);
-                const float inv = (S == 0.f) ? 0.f : 1.0f / S;
-#pragma unroll
-                for (int v = 0; v < VPT; ++v) {
-#pragma unroll
-                    for (int e = 0; e < NE; ++e) f[v][e] = (f[v][e] * f1) * inv;
-                    out[v] = E::pack(f[v]);
-                }
-            } else if constexpr (OP == OP_LAYERNORM) {
-                float s = 0.f;
-#pragma unroll
-                for (int v = 0; v < VPT; ++v) {
-                    float f[NE]; E::unpack(raw[v], f);
-#pragma unroll
-                    for (int e = 0; e < NE; ++e) s += f[e];
-                }
-                const float nk = static_cast<float>(len) * NE;
-                const float tot = red.sum(s, slot0);
-                const float mk = (len > 0) ? tot / nk : 0.f;
-                float m2 = 0.f;
-#pragma unroll
-                for (int v = 0; v < VPT; ++v) {
-                    float f[NE]; E::unpack(raw[v], f);
-                    if (valid[v]) {
-#pragma unroll
-                        for (int e = 0; e < NE; ++e) { const float d = f[e] - mk; m2 = fmaf(d, d, m2); }
-                    }
-                }
-                m2 = red.sum(m2, slot0 + 1);
-                push(mk, m2);
-                MomentPartial acc{0.f, 0.f, 0.f};
-                for (int k = 0; k < cs; ++k) {
-                    const float n_k = static_cast<float>(max(0, min(per, a.nvec - k * per))) * NE;
-                    acc = chan_combine(acc, MomentPartial{n_k, xch[par_buf][k][0], xch[par_buf][k][1]});
-                }
-                const float mean = acc.mean, rstd = 1.0f / sqrtf(acc.m2 / a.n + a.eps);
-                st0 = mean; st1 = rstd;
-#pragma unroll
-                for (int v = 0; v < VPT; ++v) {
-                    float f[NE], g[NE], b[NE];
-                    E::unpack(raw[v], f);
-                    if (valid[v]) { E::unpack(par.gamma(v), g); E::unpack(par.beta(v), b); }
-#pragma unroll
-                    for (int e = 0; e < NE; ++e) f[e] = valid[v] ? fmaf((f[e] - mean) * rstd, g[e], b[e]) : 0.f;
-                    out[v] = E::pack(f);
-                }
-            } else {
-                float ss = 0.f;
-#pragma unroll
-                for (int v = 0; v < VPT; ++v) {
-                    float f[NE]; E::unpack(raw[v], f);
-#pragma unroll
-                    for (int e = 0; e < NE; ++e) ss = fmaf(f[e], f[e], ss);
-                }
-                ss = red.sum(ss, slot0);
-                push(ss, 0.f);
-                float tot = 0.f;
-                for (int k = 0; k < cs; ++k) tot += xch[par_buf][k][0];
-                const float rr = 1.0f / sqrtf(tot / a.n + a.eps);
-                st0 = rr; st1 = rr;
-#pragma unroll
-                for (int v = 0; v < VPT; ++v) {
-                    float f[NE], w[NE];
-                    E::unpack(raw[v], f);
-                    if (valid[v]) E::unpack(par.gamma(v), w);
-#pragma unroll
-                    for (int e = 0; e < NE; ++e) f[e] = valid[v] ? (f[e] * rr) * w[e] : 0.f;
-                    out[v] = E::pack(f);
-                }
+            F2 w[VPT][Pairs<DT>::NP];
+            const Part part = slice_stats<OP, DT, VPT>(raw, valid, red, slot0, static_cast<float>(len) * NE, w);
+            if (t < cs) {                                             // push my partial into every CTA of the cluster
+                float* dst = cl.map_shared_rank(&xch[par_buf][rank][0], t);
+                dst[0] = part.a; dst[1] = part.b;
             }
+            cl.sync();                                                // release our writes, acquire the peers'
+            const Total tot = combine_parts<OP>(
+                cs, rank, [&](int k) { return Part{xch[par_buf][k][0], xch[par_buf][k][1]}; },
+                [&](int k) { return static_cast<float>(max(0, min(per, a.nvec - k * per))) * NE; }, a.n, a.eps);
+            st0 = tot.a; st1 = tot.b;
+            slice_finish<OP, DT, VPT, false>(valid, w, tot, par, out);
         }
 #pragma unroll
         for (int v = 0; v < VPT; ++v)

@@ -19,7 +19,7 @@
 #include <algorithm>
 #include <mutex>
 
-#include "tf_common.cuh"
+#include "tf_rowmath.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -83,7 +83,8 @@ template <int DT> __device__ __forceinline__ bool all_neg_inf(const uint4& v) {
 template <int OP, int DT>
 __global__ void __launch_bounds__(1024) k_tma(const TArgs a) {
     using E = Elem<DT>;
-    constexpr int NE = E::NE;
+    using P = Pairs<DT>;
+    constexpr int NE = E::NE, NP = P::NP;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ __align__(8) uint64_t mbar[kMaxStages][kMaxChunks];
     __shared__ float red_buf[4 * 32];
@@ -146,115 +147,116 @@ __global__ void __launch_bounds__(1024) k_tma(const TArgs a) {
         };
         float st0 = 0.f, st1 = 0.f;
 
+        auto wait_chunk = [&](int c) {
+            if (!mbar_wait(&mbar[stage][c], parity)) { failed = true; mbar_wait(&mbar[stage][c], parity); }
+        };
+        auto slice_count = [&](int k) { return static_cast<float>(max(0, min(per, a.nvec - k * per))) * NE; };
+        auto get_part = [&](int k) { return Part{xch[xb][k][0], xch[xb][k][1]}; };
+        const F2 l2e = f2(kLog2e);
+
         if constexpr (OP == OP_SOFTMAX) {
             // pass 1 (consumes chunks as they land): slice max
             float m = kNegInf;
             for (int c = 0; c < nchunk; ++c) {
-                if (!mbar_wait(&mbar[stage][c], parity)) { failed = true; mbar_wait(&mbar[stage][c], parity); }
+                wait_chunk(c);
                 const int end = min(len, (c + 1) * a.cv);
 #pragma unroll 4
                 for (int v = c * a.cv + t; v < end; v += T) m = fmaxf(m, vec_max<DT>(buf[v]));
             }
             m = cta_reduce<MaxOp>(m, rb0);
-            const float ok = exp_offset(m);
-            // pass 2: slice sum of 2^(x*log2e + ok); vectors that are -inf throughout contribute nothing
-            float s = 0.f;
+            // pass 2: slice sum of 2^(x*log2e + off); vectors that are -inf throughout contribute nothing
+            const F2 off = f2(exp_offset(m));
+            F2 s2 = f2(0.f);
 #pragma unroll 4
             for (int v = t; v < len; v += T) {
                 const uint4 raw = buf[v];
                 if (!all_neg_inf<DT>(raw)) {
-                    float f[NE]; E::unpack(raw, f);
+                    F2 w[NP]; P::unpack(raw, w);
 #pragma unroll
-                    for (int e = 0; e < NE; ++e) s += ex2_ftz(fmaf(f[e], kLog2e, ok));
+                    for (int i = 0; i < NP; ++i) s2 = add2(s2, ex2_ftz2(fma2(w[i], l2e, off)));
                 }
             }
-            s = cta_reduce<SumOp>(s, rb1);
-            push((m == kNegInf) ? -kNegInf : ok, s);
+            const float s = cta_reduce<SumOp>(hsum(s2), rb1);
+            push((m == kNegInf) ? -kNegInf : exp_offset(m), s);
             float O = -kNegInf;
             for (int k = 0; k < cs; ++k) O = fminf(O, xch[xb][k][0]);
             float S = 0.f;
             for (int k = 0; k < cs; ++k) S = fmaf(xch[xb][k][1], softmax_rescale(O, xch[xb][k][0]), S);
             const float inv = (S == 0.f) ? 0.f : 1.0f / S;
             // pass 3: y = 2^(x*log2e + O) / S with the row-wide offset O; store
+            const F2 O2 = f2(O), inv2 = f2(inv);
 #pragma unroll 4
             for (int v = t; v < len; v += T) {
                 const uint4 raw = buf[v];
                 uint4 out = make_uint4(0, 0, 0, 0);
                 if (!all_neg_inf<DT>(raw) && inv != 0.f) {
-                    float f[NE]; E::unpack(raw, f);
+                    F2 w[NP]; P::unpack(raw, w);
 #pragma unroll
-                    for (int e = 0; e < NE; ++e) f[e] = ex2_ftz(fmaf(f[e], kLog2e, O)) * inv;
-                    out = E::pack(f);
+                    for (int i = 0; i < NP; ++i) w[i] = mul2(ex2_ftz2(fma2(w[i], l2e, O2)), inv2);
+                    out = P::pack(w);
                 }
                 st_stream(yr + v, out);
             }
         } else if constexpr (OP == OP_LAYERNORM) {
-            float s = 0.f;
+            F2 s2 = f2(0.f);
             for (int c = 0; c < nchunk; ++c) {
-                if (!mbar_wait(&mbar[stage][c], parity)) { failed = true; mbar_wait(&mbar[stage][c], parity); }
+                wait_chunk(c);
                 const int end = min(len, (c + 1) * a.cv);
 #pragma unroll 4
                 for (int v = c * a.cv + t; v < end; v += T) {
-                    float f[NE]; E::unpack(buf[v], f);
+                    F2 w[NP]; P::unpack(buf[v], w);
 #pragma unroll
-                    for (int e = 0; e < NE; ++e) s += f[e];
+                    for (int i = 0; i < NP; ++i) s2 = add2(s2, w[i]);
                 }
             }
-            s = cta_reduce<SumOp>(s, rb0);
-            const float nk = static_cast<float>(len) * NE;
-            const float mk = (len > 0) ? s / nk : 0.f;
-            float m2 = 0.f;
+            const float s = cta_reduce<SumOp>(hsum(s2), rb0);
+            const float mk = (len > 0) ? s / slice_count(rank) : 0.f;
+            const F2 mk2 = f2(mk);
+            F2 q2 = f2(0.f);
 #pragma unroll 4
             for (int v = t; v < len; v += T) {
-                float f[NE]; E::unpack(buf[v], f);
+                F2 w[NP]; P::unpack(buf[v], w);
 #pragma unroll
-                for (int e = 0; e < NE; ++e) { const float d = f[e] - mk; m2 = fmaf(d, d, m2); }
+                for (int i = 0; i < NP; ++i) { const F2 d = sub2(w[i], mk2); q2 = fma2(d, d, q2); }
             }
-            m2 = cta_reduce<SumOp>(m2, rb1);
-            push(mk, m2);
-            MomentPartial acc{0.f, 0.f, 0.f};
-            for (int k = 0; k < cs; ++k) {
-                const float n_k = static_cast<float>(max(0, min(per, a.nvec - k * per))) * NE;
-                acc = chan_combine(acc, MomentPartial{n_k, xch[xb][k][0], xch[xb][k][1]});
-            }
-            const float mean = acc.mean, rstd = 1.0f / sqrtf(acc.m2 / a.n + a.eps);
-            st0 = mean; st1 = rstd;
+            push(mk, cta_reduce<SumOp>(hsum(q2), rb1));
+            const Total tot = combine_parts<OP>(cs, rank, get_part, slice_count, a.n, a.eps);
+            st0 = tot.a; st1 = tot.b;
+            const F2 mean2 = f2(tot.a), rstd2 = f2(tot.b);
 #pragma unroll 2
             for (int v = t; v < len; v += T) {
-                float f[NE], g[NE], b[NE];
-                E::unpack(buf[v], f);
-                E::unpack(ld_param(a.p0 + first + v), g);
-                E::unpack(ld_param(a.p1 + first + v), b);
+                F2 w[NP], g[NP], b[NP];
+                P::unpack(buf[v], w);
+                P::unpack(ld_param(a.p0 + first + v), g);
+                P::unpack(ld_param(a.p1 + first + v), b);
 #pragma unroll
-                for (int e = 0; e < NE; ++e) f[e] = fmaf((f[e] - mean) * rstd, g[e], b[e]);
-                st_stream(yr + v, E::pack(f));
+                for (int i = 0; i < NP; ++i) w[i] = fma2(mul2(sub2(w[i], mean2), rstd2), g[i], b[i]);
+                st_stream(yr + v, P::pack(w));
             }
         } else {
-            float ss = 0.f;
+            F2 q2 = f2(0.f);
             for (int c = 0; c < nchunk; ++c) {
-                if (!mbar_wait(&mbar[stage][c], parity)) { failed = true; mbar_wait(&mbar[stage][c], parity); }
+                wait_chunk(c);
                 const int end = min(len, (c + 1) * a.cv);
 #pragma unroll 4
                 for (int v = c * a.cv + t; v < end; v += T) {
-                    float f[NE]; E::unpack(buf[v], f);
+                    F2 w[NP]; P::unpack(buf[v], w);
 #pragma unroll
-                    for (int e = 0; e < NE; ++e) ss = fmaf(f[e], f[e], ss);
+                    for (int i = 0; i < NP; ++i) q2 = fma2(w[i], w[i], q2);
                 }
             }
-            ss = cta_reduce<SumOp>(ss, rb0);
-            push(ss, 0.f);
-            float tot = 0.f;
-            for (int k = 0; k < cs; ++k) tot += xch[xb][k][0];
-            const float rr = 1.0f / sqrtf(tot / a.n + a.eps);
-            st0 = rr; st1 = rr;
+            push(cta_reduce<SumOp>(hsum(q2), rb0), 0.f);
+            const Total tot = combine_parts<OP>(cs, rank, get_part, slice_count, a.n, a.eps);
+            st0 = tot.a; st1 = tot.b;
+            const F2 rr2 = f2(tot.a);
 #pragma unroll 4
             for (int v = t; v < len; v += T) {
-                float f[NE], w[NE];
-                E::unpack(buf[v], f);
-                E::unpack(ld_param(a.p0 + first + v), w);
+                F2 w[NP], g[NP];
+                P::unpack(buf[v], w);
+                P::unpack(ld_param(a.p0 + first + v), g);
 #pragma unroll
-                for (int e = 0; e < NE; ++e) f[e] = (f[e] * rr) * w[e];
-                st_stream(yr + v, E::pack(f));
+                for (int i = 0; i < NP; ++i) w[i] = mul2(mul2(w[i], rr2), g[i]);
+                st_stream(yr + v, P::pack(w));
             }
         }
         if (t == 0 && rank == 0) {

@@ -197,31 +197,35 @@ def test_forced_tma_variants(op, dt, cluster):
 
 
 PIPE_COMBOS = [(8, 1), (16, 1), (32, 1), (32, 2), (32, 4), (32, 8), (64, 2), (64, 4), (64, 8), (128, 2), (128, 4), (128, 8),
-               (256, 2), (256, 4), (256, 8), (512, 4)]
+               (256, 2), (256, 4), (256, 8), (512, 4), (512, 8)]
 
 
 @pytest.mark.parametrize("op", OPS)
 @pytest.mark.parametrize("dt", [F32, BF16])
 def test_forced_pipe_variants(op, dt):
     ne = 4 if dt == F32 else 8
-    for lanes, vpt in PIPE_COMBOS:
+    ran = 0
+    for ci, (lanes, vpt) in enumerate(PIPE_COMBOS):
         cap = lanes * vpt
-        for threads in (256, 512):
-            if threads < lanes or (vpt == 8 and threads > 256):
+        ut = max(32, lanes)
+        threads = 512 if ci % 2 else max(256, ut)
+        # rows chosen so that a unit wraps its ring several times and the last tile is ragged
+        for nvec, stages, chunk, persist, rows in ((cap, 2, 4096, 1, 4001), (max(1, cap - 1), 3, 16384, 2, 2999),
+                                                   (max(1, cap // 2 + 1), 1, 2048, 1, 1777), (cap, 4, 512, 8, 77)):
+            chunk = max(chunk, nvec * 16 * (ut // lanes))
+            plan = f"pipe:threads={threads},lanes={lanes},vpt={vpt},stages={stages},chunk={chunk},persist={persist}"
+            tf.tf_force_plan(op, plan)
+            if nvec * 16 > 8192:
+                rows = max(40, rows // 16)
+            w = wl(op, dt, rows, nvec * ne, seed=nvec)
+            try:
+                fails = parity.parity(w)
+            except tf.TfError as e:
+                assert e.status == 2, plan                     # ring does not fit shared memory: refused, not wrong
                 continue
-            for nvec in {cap, max(1, cap - 1), max(1, cap // 2 + 1)}:
-                for stages, chunk, persist, rows in ((2, 16384, 1, 77), (4, 32768, 1, 3000), (3, 65536, 2, 1301), (8, 8192, 1, 5000)):
-                    if chunk < nvec * 16:
-                        chunk = 65536
-                    plan = f"pipe:threads={threads},lanes={lanes},vpt={vpt},stages={stages},chunk={chunk},persist={persist}"
-                    tf.tf_force_plan(op, plan)
-                    w = wl(op, dt, rows if nvec * 16 <= 8192 else max(40, rows // 8), nvec * ne, seed=nvec)
-                    try:
-                        fails = parity.parity(w)
-                    except tf.TfError as e:
-                        assert e.status == 2, plan                     # ring does not fit shared memory: refused, not wrong
-                        continue
-                    assert not fails, (plan, nvec, fails)
+            ran += 1
+            assert not fails, (plan, nvec, fails)
+    assert ran >= 40
 
 
 @pytest.mark.parametrize("op", OPS)
