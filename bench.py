@@ -31,7 +31,9 @@ L2_BYTES = 126 << 20
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/; None until a capture of that kernel exists.
 NCU_TRAFFIC_BYTES = {
-    "layernorm_bf16_8192x4096": None,
+    # profiles/k_pipe_layernorm_bf16_8192x4096.md: 67.16 MB read (= the algorithmic reads) + 9.48 MB written inside the
+    # kernel; the other 57.7 MB of y are still dirty in the 126 MB L2 when an isolated launch ends
+    "layernorm_bf16_8192x4096": 67157760 + 9477888,
 }
 
 
@@ -288,11 +290,13 @@ def run_ours(args):
     torch.cuda.synchronize()
     launches0 = tf.tf_launch_count()
     with ClockSampler(local_rank) as clk:
+        torch.cuda.nvtx.range_push("BIG_OP")         # the label the paper's profiling step filters on (Section 3.3)
         start.record()
         for _ in range(steps):
             case.step()
         end.record()
         torch.cuda.synchronize()
+        torch.cuda.nvtx.range_pop()
     launches = tf.tf_launch_count() - launches0
     ms = start.elapsed_time(end)
     if world > 1:
@@ -414,6 +418,35 @@ def run_table(args):
     (out_dir / f"table_{args.table}.json").write_text(json.dumps(rows_out, indent=1))
 
 
+def run_case(args):
+    """A few launches of one op/shape (for profiler captures): --case op:dtype:rows:cols or --case config:<i>[:rows]."""
+    import torch
+    import paper_2512_09196_b200 as tf
+    from paper_2512_09196_b200 import inputs
+    torch.cuda.set_device(0)
+    parts = args.case.split(":")
+    if parts[0] == "config":
+        w = inputs.config(int(parts[1]))
+        if len(parts) > 2:
+            w = inputs.Workload(w.name, w.op, w.dt, int(parts[2]), w.cols, seed=w.seed, x_mean=w.x_mean, x_std=w.x_std, eps=w.eps,
+                                outlier_p=w.outlier_p, outlier_factor=w.outlier_factor, mask_step=w.mask_step, scale=w.scale,
+                                shift=w.shift)
+    else:
+        op, dt, rows, cols = parts
+        eps = {"softmax": 0.0, "layernorm": 1e-5, "rmsnorm": 1e-6}[op]
+        w = inputs.Workload(f"case_{op}_{dt}_{rows}x{cols}", op, inputs.F32 if dt == "f32" else inputs.BF16, int(rows), int(cols),
+                            seed=int(cols), eps=eps)
+    case = DeviceCase(w, w.generate(), torch.device("cuda", 0), min_total_bytes=0)
+    if args.plan:
+        tf.tf_force_plan(w.op, args.plan)
+    elif not args.no_tune:
+        tf.tf_tune(w.op, w.rows, w.cols, w.dt)
+    ms = case.time_steps(args.steps, max(1, args.warmup))
+    tf.tf_device_status()
+    print(json.dumps({"case": w.name, "plan": args.plan or tf.tf_query_choice(w.op, w.rows, w.cols, w.dt), "launches": args.steps,
+                      "us_per_launch": 1e3 * ms / args.steps, "gbs": case.bytes_per_step / (ms * 1e-3 / args.steps) / 1e9}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -424,6 +457,8 @@ def main():
     ap.add_argument("--filter", default=None)
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
+    ap.add_argument("--case", default=None, help="op:dtype:rows:cols or config:<i>[:rows] -- a few launches of one shape")
+    ap.add_argument("--plan", default=None, help="with --case: force this launch plan")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 10 if args.steps is None else args.steps
@@ -433,6 +468,8 @@ def main():
     args.warmup = 50 if args.warmup is None else args.warmup
     import __graft_entry__
     __graft_entry__.build()
+    if args.case:
+        return run_case(args)
     if args.table:
         return run_table(args)
     run_ours(args)

@@ -1,0 +1,93 @@
+"""Parity at the full sizes of the fixed configurations, in the launch configuration the bench times (the tuned
+plan): configurations 0-2 are compared on every row, block by block; the 2 GiB masked softmax on sampled rows
+(each row is an independent problem, so a row sample is an exact check of those rows)."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_09196_b200 as tf
+from paper_2512_09196_b200 import inputs
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_full(w, data):
+    dt = w.dt
+    x = parity.to_dev(data["x"], dt)
+    out = {}
+    if w.op == "softmax":
+        out["y"] = tf.tf_softmax_fwd(x)
+    elif w.op == "layernorm":
+        y, mean, rstd = tf.tf_layernorm_fwd(x, parity.to_dev(data["gamma"], dt), parity.to_dev(data["beta"], dt), w.eps)
+        out.update(y=y, mean=mean.cpu().numpy(), rstd=rstd.cpu().numpy())
+    else:
+        y, rstd = tf.tf_rmsnorm_fwd(x, parity.to_dev(data["w"], dt), w.eps, want_rstd=True)
+        out.update(y=y, rstd=rstd.cpu().numpy())
+    torch.cuda.synchronize()
+    tf.tf_device_status()
+    return out
+
+
+def _check_rows(w, data, got, rows):
+    """Oracle + comparison on the given row indices (a slice or an index array)."""
+    sub = dict(data)
+    sub["x"] = np.ascontiguousarray(data["x"][rows])
+    g = {"y": parity.to_host(got["y"][rows], w.dt)}
+    for k in ("mean", "rstd"):
+        if k in got:
+            g[k] = got[k][rows]
+    return parity.check(w, sub, g, parity.run_oracle(w, sub, nthreads=16))
+
+
+@pytest.mark.parametrize("i", [0, 1, 2])
+def test_full_configuration_every_row(i):
+    w = inputs.config(i)
+    tf.tf_tune(w.op, w.rows, w.cols, w.dt)
+    data = w.generate()
+    got = _run_full(w, data)
+    block = max(1, (1 << 23) // w.cols)
+    for r0 in range(0, w.rows, block):
+        fails = _check_rows(w, data, got, slice(r0, min(w.rows, r0 + block)))
+        assert not fails, (w.name, tf.tf_query_choice(w.op, w.rows, w.cols, w.dt), r0, fails)
+
+
+def test_masked_softmax_2gib_sampled_rows():
+    w = inputs.config(3)
+    tf.tf_tune(w.op, w.rows, w.cols, w.dt)
+    data = w.generate()
+    got = _run_full(w, data)
+    rows = np.unique(np.concatenate([np.arange(0, w.rows, 61), [0, 1, 2047, 2048, w.rows - 2, w.rows - 1]]))
+    fails = _check_rows(w, data, got, rows)
+    assert not fails, (tf.tf_query_choice(w.op, w.rows, w.cols, w.dt), fails)
+    # properties that hold for every row: masked tail is +0 everywhere, nothing else is NaN, rows sum to about 1
+    y = got["y"]
+    assert not torch.isnan(y).any()
+    sums = y.float().sum(dim=1)
+    assert (sums > 0.97).all() and (sums < 1.03).all()
+    for r in (1, 1000, 4095):
+        k = (r * 32) % w.cols
+        assert (y[r, w.cols - k:].view(torch.int16) == 0).all()
+
+
+def test_tune_is_idempotent_and_candidates_all_pass_parity():
+    w = inputs.Workload("tune_case", "layernorm", inputs.BF16, 600, 2048, seed=9, x_mean=0.5, x_std=3.0, eps=1e-5)
+    tf.tf_clear_cache()
+    first = tf.tf_tune(w.op, w.rows, w.cols, w.dt)
+    cands = tf.tf_candidates(w.op, w.rows, w.cols, w.dt)
+    assert first["plan"] in cands and first["timed"] >= 2 and first["best_us"] <= first["heuristic_us"] * 1.0001
+    assert tf.tf_query_choice(w.op, w.rows, w.cols, w.dt) == first["plan"]          # later calls hit the cache
+    second = tf.tf_tune(w.op, w.rows, w.cols, w.dt)
+    assert second["plan"] in cands
+    data = w.generate()
+    ref = parity.run_oracle(w, data)
+    try:
+        for plan in cands[:: max(1, len(cands) // 24)]:
+            tf.tf_force_plan(w.op, plan)
+            fails = parity.check(w, data, parity.run_gpu(w, data), ref)
+            assert not fails, (plan, fails)
+    finally:
+        tf.tf_force_plan(w.op, None)
+        tf.tf_clear_cache()

@@ -178,7 +178,7 @@ def test_forced_cta_variants(op, dt, cluster):
                     continue
                 for persist in (0, 1):
                     tf.tf_force_plan(op, f"cta:threads={threads},vpt={vpt},cluster={cluster},persist={persist}")
-                    rows = 9 if persist == 0 else 700
+                    rows = 9 if persist == 0 else min(700, max(160, (1 << 20) // (nvec * ne)))   # > 148 clusters' worth
                     fails = parity.parity(wl(op, dt, rows if nvec < 4096 else 5, nvec * ne, seed=nvec))
                     assert not fails, (vpt, threads, cluster, nvec, persist, fails)
 
@@ -192,7 +192,8 @@ def test_forced_tma_variants(op, dt, cluster):
         for threads, stages, chunk, persist, rows in ((128, 1, 4096, 0, 7), (512, 1, 8192, 0, 7), (1024, 2, 32768, 1, 400),
                                                        (256, 3, 16384, 1, 900), (256, 2, 1024, 2, 1300)):
             tf.tf_force_plan(op, f"tma:threads={threads},cluster={cluster},stages={stages},chunk={chunk},persist={persist}")
-            fails = parity.parity(wl(op, dt, rows if nvec <= 4096 else min(rows, 300), nvec * ne, seed=nvec))
+            rows = min(rows, max(7 if persist == 0 else 2 * 148 // cluster + 9, (1 << 21) // (nvec * ne)))
+            fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec))
             assert not fails, (cluster, nvec, threads, stages, chunk, persist, fails)
 
 
