@@ -11,7 +11,7 @@ HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 INCLUDE = HERE.parent / "include"
 LIB = HERE / "libtf.so"
-SOURCES = ["tf_api.cu", "tf_rowreg.cu", "tf_tma.cu", "tf_stream.cu", "tf_pipe.cu"]
+SOURCES = ["tf_api.cu", "tf_rowreg.cu", "tf_tma.cu", "tf_stream.cu", "tf_pipe.cu", "tf_ring.cu", "tf_pipe_softmax.cu", "tf_pipe_layernorm.cu", "tf_pipe_rmsnorm.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-Xcompiler", "-fPIC"]
 
 
@@ -51,7 +51,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
             raise RuntimeError(f"nvcc failed on {src}:\n{r.stdout}\n{r.stderr}")
         return r.stderr
 
-    with ThreadPoolExecutor(max_workers=4) as ex:
+    with ThreadPoolExecutor(max_workers=8) as ex:
         logs = list(ex.map(compile_one, jobs))
     if verbose:
         sys.stderr.write("\n".join(logs))

@@ -68,7 +68,7 @@ tf_status device_state(DevState** out) {
 // ------------------------------------------------------------------------------------------------
 // plans as text
 // ------------------------------------------------------------------------------------------------
-const char* kVariantName[V_COUNT] = {"warp", "cta", "tma", "stream", "pipe"};
+const char* kVariantName[V_COUNT] = {"warp", "cta", "tma", "stream", "pipe", "ring"};
 
 std::string plan_to_string(const Plan& p) {
     char b[160];
@@ -76,7 +76,8 @@ std::string plan_to_string(const Plan& p) {
         case V_WARP: snprintf(b, sizeof b, "warp:threads=%d,lanes=%d,vpt=%d,rpg=%d,persist=%d", p.threads, p.lanes, p.vpt, p.rpg, p.persist); break;
         case V_CTA: snprintf(b, sizeof b, "cta:threads=%d,vpt=%d,cluster=%d,persist=%d", p.threads, p.vpt, p.cluster, p.persist); break;
         case V_TMA: snprintf(b, sizeof b, "tma:threads=%d,cluster=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.cluster, p.stages, p.chunk, p.persist); break;
-        case V_PIPE: snprintf(b, sizeof b, "pipe:threads=%d,lanes=%d,vpt=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.lanes, p.vpt, p.stages, p.chunk, p.persist); break;
+        case V_PIPE: snprintf(b, sizeof b, "pipe:threads=%d,lanes=%d,vpt=%d,rpg=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.lanes, p.vpt, p.rpg, p.stages, p.chunk, p.persist); break;
+        case V_RING: snprintf(b, sizeof b, "ring:threads=%d,vpt=%d,cluster=%d,stages=%d,persist=%d", p.threads, p.vpt, p.cluster, p.stages, p.persist); break;
         default: snprintf(b, sizeof b, "stream:threads=%d,lanes=%d,persist=%d", p.threads, p.lanes, p.persist); break;
     }
     return b;
@@ -92,6 +93,7 @@ bool plan_from_string(const char* s, Plan& out) {
     p.variant = v;
     if (v == V_STREAM) p.lanes = 0;
     if (v == V_PIPE) { p.persist = 1; p.stages = 4; p.chunk = 32768; }
+    if (v == V_RING) { p.persist = 1; p.stages = 2; }
     const char* q = colon ? colon + 1 : s + strlen(s);
     while (*q) {
         const char* eq = strchr(q, '=');
@@ -121,6 +123,7 @@ bool supports(const Plan& p, const Args& a, const DeviceInfo& d) {
         case V_TMA: return supports_tma(p, a, d);
         case V_STREAM: return supports_stream(p, a, d);
         case V_PIPE: return supports_pipe(p, a, d);
+        case V_RING: return supports_ring(p, a, d);
     }
     return false;
 }
@@ -132,6 +135,7 @@ cudaError_t launch(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream
         case V_CTA: return launch_cta(p, a, d, st);
         case V_TMA: return launch_tma(p, a, d, st);
         case V_PIPE: return launch_pipe(p, a, d, st);
+        case V_RING: return launch_ring(p, a, d, st);
         default: return launch_stream(p, a, d, st);
     }
 }
@@ -197,7 +201,19 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         else { p.vpt = 8; p.cluster = 2; p.threads = round_up(static_cast<int>((nvec + 15) / 16), 32); }
         return p;
     }
-    // long rows: shared-memory staging, slices of at most 64 KiB
+    // long rows: persistent clusters with a prefetch ring, slices of at most 64 KiB (4 vectors per thread)
+    {
+        Plan r;
+        r.variant = V_RING; r.vpt = 4; r.stages = 2;
+        int cl = 1;
+        while (cl < kMaxCluster && row_bytes > static_cast<int64_t>(cl) * 65536) cl *= 2;
+        r.cluster = cl;
+        const int64_t per = (nvec + cl - 1) / cl;
+        r.threads = std::min(1024, round_up(static_cast<int>((per + 3) / 4), 32));
+        r.persist = std::max(1, std::min(2, static_cast<int>(200 * 1024 / (2 * per * 16))));
+        if (supports_ring(r, a, d)) return r;
+    }
+    // fallback for long rows: shared-memory staging with re-reads from shared memory
     p.variant = V_TMA;
     p.threads = 512;
     p.stages = 1;
@@ -261,16 +277,17 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
             const int64_t cap = static_cast<int64_t>(c[0]) * c[1];
             if (nvec > cap || (nvec * 2 <= cap && c[0] != 8)) continue;
             const int ut = c[0] < 32 ? 32 : c[0];
-            const int64_t pass_bytes = row_bytes * (ut / c[0]);
+            for (int rpg : {1, 2})
             for (int th : {256, 512}) {
-                if (th < ut) continue;
+                if (th < ut || (rpg == 2 && (c[1] > 4 || nvec != cap))) continue;
+                const int64_t pass_bytes = row_bytes * (ut / c[0]) * rpg;
                 const int units = th / ut;
                 for (int persist : {1, 2, 4})
                     for (int stages : {2, 3, 4}) {
                         const int64_t budget = (persist == 1 ? 200 : (persist == 2 ? 98 : 48)) * 1024 - param_bytes;
                         int64_t chunk = std::min<int64_t>(32768, budget / units / stages) / pass_bytes * pass_bytes;
                         if (chunk < pass_bytes) continue;
-                        Plan p; p.variant = V_PIPE; p.lanes = c[0]; p.vpt = c[1]; p.threads = th; p.persist = persist;
+                        Plan p; p.variant = V_PIPE; p.lanes = c[0]; p.vpt = c[1]; p.rpg = rpg; p.threads = th; p.persist = persist;
                         p.chunk = static_cast<int>(chunk); p.stages = stages;
                         add(p);
                         if (chunk >= 4 * pass_bytes && chunk > 4096) { p.chunk = static_cast<int>(chunk / 2 / pass_bytes * pass_bytes); add(p); }
@@ -278,6 +295,23 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
             }
         }
     }
+    // persistent cluster ring for long rows
+    if (nvec >= 2048)
+        for (int cl : {1, 2, 4, 8})
+            for (int vpt : {2, 4, 8}) {
+                const int64_t per = (nvec + cl - 1) / cl;
+                const int64_t th = (per + vpt - 1) / vpt;
+                if (th > (vpt <= 4 ? 1024 : 512) || th < 128) continue;
+                for (int stages : {2, 3}) {
+                    const int64_t ring_bytes = stages * per * 16;
+                    if (ring_bytes > 200 * 1024) continue;
+                    Plan p; p.variant = V_RING; p.cluster = cl; p.vpt = vpt; p.threads = round_up(static_cast<int>(th), 32); p.stages = stages;
+                    const int fit = static_cast<int>(std::min<int64_t>({8, 200 * 1024 / ring_bytes, 2048 / p.threads}));
+                    p.persist = std::max(1, fit);
+                    add(p);
+                    if (fit > 1) { p.persist = 1; add(p); }
+                }
+            }
     // shared-memory staged variants
     if (nvec >= 512)
         for (int cl : {1, 2, 4, 8}) {

@@ -1,0 +1,252 @@
+// V_PIPE: persistent self-feeding pipeline for rows that fit a shared-memory stage (128 B .. 64 KiB).
+//
+// Rows are dense and row-major, so a tile of R consecutive rows is one contiguous range of global memory
+// and arrives with one bulk asynchronous copy (cp.async.bulk global -> shared, completion counted on an
+// mbarrier; no multicast).  A CTA is a set of independent UNITS (a warp, or a few warps for wide rows); each
+// unit owns a small ring of stages and walks its own sequence of tiles: wait for a stage, take the rows into
+// registers, reduce, and -- as soon as the reduction has consumed the stage -- let its first lane refill
+// that same stage with the unit's tile after next, then normalise and write y with 16-byte streaming stores.
+// There is no producer warp and no "empty" barrier: the refill is issued by a thread that has just finished
+// with the data.  The bytes in flight are the rings (up to ~200 KiB per SM), not what the register file can
+// hold, and no unit ever waits for another.  HBM sees each element once in and once out.
+//
+// Inside a unit a row belongs to LANES threads: 8 or 16 (a warp then covers 4 or 2 rows at a time), 32, or
+// several warps that merge their partials (max,sum | mean,M2 | sum of squares) through shared memory and one
+// named barrier per row.  LayerNorm / RMSNorm parameters are copied to shared memory once per CTA.
+//
+// The kernel is launched with programmatic stream serialisation: its prologue (barrier init) overlaps the
+// tail of the previous kernel in the stream, and griddepcontrol.wait orders every global access after it.
+//
+// All mbarrier waits are bounded by a clock budget; a unit that gives up records TF_ERR_TIMEOUT in the status
+// word, stops issuing copies and finishes its loop without waiting again (control flow stays uniform, so no
+// named barrier is left hanging).
+#pragma once
+
+#include "tf_rowmath.cuh"
+
+namespace tf {
+namespace pipe {
+
+struct PArgs {
+    const uint4* x;
+    const uint4* p0;
+    const uint4* p1;
+    uint4* y;
+    float* mean;
+    float* rstd;
+    int64_t rows;
+    int nvec;          // 16-byte vectors per row
+    float n, eps;
+    int tile_rows;     // rows per stage of a unit
+    int nstage;        // stages per unit
+    int* status;
+};
+
+constexpr int kPipeMaxBarriers = 128;                    // units x stages per CTA
+constexpr long long kPipeWaitBudget = 400000000LL;      // about 0.2 s
+
+__device__ __forceinline__ uint32_t sm_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void bar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sm_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool bar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(sm_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, long long budget) {   // false: gave up
+    if (bar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!bar_try_wait(bar, parity))
+        if (clock64() - t0 > budget) return false;
+    return true;
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(sm_u32(dst)), "l"(src), "r"(bytes), "r"(sm_u32(bar)) : "memory");
+}
+
+// Parameters staged in shared memory: gamma at [0, nvec), beta at [nvec, 2 nvec).
+struct SmemParams {
+    const uint4* base;
+    int nvec, first, stride;
+    __device__ __forceinline__ uint4 gamma(int v) const { return base[first + v * stride]; }
+    __device__ __forceinline__ uint4 beta(int v) const { return base[nvec + first + v * stride]; }
+};
+
+constexpr int kPipeMaxThreads = 512;
+
+// RPG: rows of the same columns a thread carries through one pass (parameters, barriers and shuffle latency are
+// shared by them).  FULL: the row fills LANES x VPL vectors exactly, so no vector needs a predicate.
+template <int OP, int DT, int LANES, int VPL, int RPG, bool FULL>
+__global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
+    using E = Elem<DT>;
+    constexpr int NE = E::NE;
+    constexpr int UT = LANES < 32 ? 32 : LANES;          // threads per unit
+    constexpr int RPP = UT / LANES;                      // rows a unit takes per pass
+    constexpr int W = UT / 32;                           // warps per unit
+    constexpr int RPU = RPP * RPG;                       // rows a unit takes per pass
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    __shared__ __align__(8) uint64_t full_bar[kPipeMaxBarriers];
+    __shared__ float xch[W > 1 ? (kPipeMaxThreads / UT) * 2 * RPG * W * 2 : 1];     // [unit][parity][row][warp][2]
+
+    const int t = threadIdx.x;
+    const int units = blockDim.x / UT;
+    const int unit = t / UT, ut = t % UT;               // unit index, thread index within the unit
+    const int sub = ut / LANES, lane = ut % LANES;      // row slot within a pass, lane within the row
+    const int S = a.nstage;
+    const size_t tile_vecs = static_cast<size_t>(a.tile_rows) * a.nvec;
+    uint4* const ring = reinterpret_cast<uint4*>(dyn_smem) + tile_vecs * S * unit;
+    uint4* const params = reinterpret_cast<uint4*>(dyn_smem) + tile_vecs * S * units;
+    uint64_t* const bars = full_bar + unit * S;
+    const int64_t num_tiles = (a.rows + a.tile_rows - 1) / a.tile_rows;
+    const int64_t gu = static_cast<int64_t>(blockIdx.x) * units + unit;          // global unit index
+    const int64_t GU = static_cast<int64_t>(gridDim.x) * units;
+
+    if (ut == 0) {
+        for (int s = 0; s < S; ++s) bar_init(&bars[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // everything below may read what the previous kernel wrote
+
+    auto issue = [&](int64_t tile, int s) {              // first thread of the unit only
+        const int64_t row0 = tile * a.tile_rows;
+        const int rows_here = static_cast<int>(min(static_cast<int64_t>(a.tile_rows), a.rows - row0));
+        const uint32_t bytes = static_cast<uint32_t>(rows_here) * a.nvec * 16u;
+        bar_expect_tx(&bars[s], bytes);
+        bulk_load(ring + tile_vecs * s, a.x + row0 * a.nvec, bytes, &bars[s]);
+    };
+    if (ut == 0)
+        for (int s = 0; s < S; ++s) {
+            const int64_t tile = gu + s * GU;
+            if (tile < num_tiles) issue(tile, s);
+        }
+    if (OP != OP_SOFTMAX) {
+        for (int i = t; i < a.nvec; i += blockDim.x) {
+            params[i] = ld_param(a.p0 + i);
+            if (OP == OP_LAYERNORM) params[a.nvec + i] = ld_param(a.p1 + i);
+        }
+    }
+    __syncthreads();                                      // barriers initialised, parameters staged
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    bool valid[VPL];
+#pragma unroll
+    for (int v = 0; v < VPL; ++v) valid[v] = FULL || (lane + v * LANES) < a.nvec;
+    const GroupRed<(LANES < 32 ? LANES : 32)> red;
+    const SmemParams par{params, a.nvec, lane, LANES};
+    const uint4 fill = fill_vec<DT>(OP);
+    // element count of warp w's slice of a row (multi-warp units): lanes 32w .. 32w+31 own vectors l + v*LANES
+    auto slice_count = [&](int w) {
+        int c = 0;
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) c += max(0, min(32, a.nvec - (w * 32 + v * LANES)));
+        return static_cast<float>(c * NE);
+    };
+    const int my_warp = ut >> 5;
+    const float my_count = (W > 1) ? slice_count(my_warp) : a.n;
+    (void)my_warp;
+
+    bool failed = false;
+    int i = 0, xpar = 0;
+    for (int64_t tile = gu; tile < num_tiles; tile += GU, ++i) {
+        const int s = i % S;
+        if (!failed && !bar_wait(&bars[s], static_cast<uint32_t>(i / S) & 1u, kPipeWaitBudget)) {
+            failed = true;
+            atomicExch(a.status, 4);
+            bar_wait(&bars[s], static_cast<uint32_t>(i / S) & 1u, kPipeWaitBudget);    // one more bounded wait for the copy
+        }
+        const int64_t row0 = tile * a.tile_rows;
+        const int rows_here = static_cast<int>(min(static_cast<int64_t>(a.tile_rows), a.rows - row0));
+        const uint4* stage = ring + tile_vecs * s;
+        const int64_t next = tile + static_cast<int64_t>(S) * GU;
+        // same trip count for every thread of the unit; slots past the tile compute on fill values and store nothing
+        for (int r0 = 0; r0 < rows_here; r0 += RPU) {
+            int r[RPG];
+            bool live[RPG];
+            uint4 raw[RPG][VPL], out[RPG][VPL];
+#pragma unroll
+            for (int q = 0; q < RPG; ++q) {
+                r[q] = r0 + q * RPP + sub;
+                live[q] = (RPU == 1) || r[q] < rows_here;
+                const uint4* xr = stage + static_cast<size_t>(live[q] ? r[q] : 0) * a.nvec + lane;
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) raw[q][v] = (live[q] && valid[v]) ? xr[v * LANES] : fill;
+            }
+            F2 w[RPG][VPL][Pairs<DT>::NP];
+            Part part[RPG];
+#pragma unroll
+            for (int q = 0; q < RPG; ++q) part[q] = slice_stats<OP, DT, VPL, decltype(red), FULL>(raw[q], valid, red, 0, my_count, w[q]);
+            Total tot[RPG];
+            if constexpr (W > 1) {
+                float* slot = xch + ((unit * 2 + xpar) * RPG) * W * 2;
+                if ((ut & 31) == 0) {
+#pragma unroll
+                    for (int q = 0; q < RPG; ++q) { slot[(q * W + my_warp) * 2] = part[q].a; slot[(q * W + my_warp) * 2 + 1] = part[q].b; }
+                }
+                asm volatile("bar.sync %0, %1;" ::"r"(1 + unit), "r"(UT) : "memory");
+#pragma unroll
+                for (int q = 0; q < RPG; ++q)
+                    tot[q] = combine_parts<OP>(W, my_warp, [&](int k) { return Part{slot[(q * W + k) * 2], slot[(q * W + k) * 2 + 1]}; },
+                                               slice_count, a.n, a.eps);
+                xpar ^= 1;
+            } else {
+#pragma unroll
+                for (int q = 0; q < RPG; ++q) tot[q] = total_of<OP>(part[q], a.n, a.eps);
+            }
+            // The reductions above consumed every value this unit read from the stage (shuffle results and the
+            // named barrier both depend on all of its loads): after the tile's last pass the stage is refilled.
+            if (r0 + RPU >= rows_here && ut == 0 && !failed && next < num_tiles) issue(next, s);
+            slice_finish_rows<OP, DT, VPL, RPG, (W == 1), FULL>(valid, w, tot, par, out);
+#pragma unroll
+            for (int q = 0; q < RPG; ++q) {
+                if (live[q]) {
+                    const int64_t row = row0 + r[q];
+                    uint4* yr = a.y + row * a.nvec + lane;
+#pragma unroll
+                    for (int v = 0; v < VPL; ++v)
+                        if (valid[v]) st_stream(yr + v * LANES, out[q][v]);
+                    if (lane == 0) {
+                        if (OP == OP_LAYERNORM && a.mean) a.mean[row] = tot[q].a;
+                        if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = tot[q].b;
+                    }
+                }
+            }
+        }
+    }
+}
+
+using PipeFn = void (*)(const PArgs);
+
+template <int OP, int DT> PipeFn pick_pipe(int lanes, int vpl, int rpg, bool full) {
+#define TF_P(L, V)                                                                     \
+    if (lanes == L && vpl == V) {                                                      \
+        if (rpg == 1) return full ? k_pipe<OP, DT, L, V, 1, true> : k_pipe<OP, DT, L, V, 1, false>; \
+        if (rpg == 2 && V <= 4 && full) return k_pipe<OP, DT, L, (V <= 4 ? V : 1), 2, true>;       \
+        return nullptr;                                                                \
+    }
+    TF_P(8, 1) TF_P(16, 1) TF_P(32, 1) TF_P(32, 2) TF_P(32, 4) TF_P(32, 8)
+    TF_P(64, 2) TF_P(64, 4) TF_P(64, 8) TF_P(128, 2) TF_P(128, 4) TF_P(128, 8) TF_P(256, 2) TF_P(256, 4) TF_P(256, 8)
+    TF_P(512, 4) TF_P(512, 8)
+#undef TF_P
+    return nullptr;
+}
+
+template <int OP> PipeFn pipe_fn_op(int dt, int lanes, int vpl, int rpg, bool full) {
+    return dt == DT_F32 ? pick_pipe<OP, DT_F32>(lanes, vpl, rpg, full) : pick_pipe<OP, DT_BF16>(lanes, vpl, rpg, full);
+}
+
+// one translation unit per op instantiates the kernels
+PipeFn pipe_fn_softmax(int dt, int lanes, int vpl, int rpg, bool full);
+PipeFn pipe_fn_layernorm(int dt, int lanes, int vpl, int rpg, bool full);
+PipeFn pipe_fn_rmsnorm(int dt, int lanes, int vpl, int rpg, bool full);
+
+}  // namespace pipe
+}  // namespace tf

@@ -15,7 +15,8 @@ enum Variant : int {
     V_TMA = 2,      // each CTA of a cluster stages its slice of the row in shared memory with bulk async copies
     V_STREAM = 3,   // generic: scalar accesses, several passes over the row, any alignment and length
     V_PIPE = 4,     // persistent CTAs: a producer thread streams row tiles into a shared-memory ring, consumer warps normalise
-    V_COUNT = 5
+    V_RING = 5,     // persistent clusters: each CTA prefetches its slice of a long row into a shared-memory ring, registers hold it
+    V_COUNT = 6
 };
 
 struct Plan {
@@ -62,11 +63,13 @@ bool supports_cta(const Plan&, const Args&, const DeviceInfo&);
 bool supports_tma(const Plan&, const Args&, const DeviceInfo&);
 bool supports_stream(const Plan&, const Args&, const DeviceInfo&);
 bool supports_pipe(const Plan&, const Args&, const DeviceInfo&);
+bool supports_ring(const Plan&, const Args&, const DeviceInfo&);
 cudaError_t launch_warp(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_cta(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_tma(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_stream(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_pipe(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+cudaError_t launch_ring(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 
 // Raises a kernel's dynamic shared-memory limit to the device's opt-in maximum, once per kernel and device.
 cudaError_t ensure_max_smem(const void* fn, const DeviceInfo&);

@@ -51,7 +51,8 @@ struct Total { float a, b; };        // softmax: (rescale of my slice, 1/S); Lay
 
 // `slot0` picks the reducer's shared buffers (CTA reducers alternate them between rows).  `w` receives the
 // widened values (softmax: the exponentials) for slice_finish.
-template <int OP, int DT, int NV, class Red>
+// ALLV: every vector of every thread is valid (the row fills the group exactly), so no predicate is needed.
+template <int OP, int DT, int NV, class Red, bool ALLV = false>
 __device__ __forceinline__ Part slice_stats(const uint4 (&raw)[NV], const bool (&valid)[NV], const Red& red, int slot0,
                                             float n_slice, F2 (&w)[NV][Pairs<DT>::NP]) {
     using P = Pairs<DT>;
@@ -84,7 +85,7 @@ __device__ __forceinline__ Part slice_stats(const uint4 (&raw)[NV], const bool (
         F2 m2 = f2(0.f);
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
-            if (valid[v]) {
+            if (ALLV || valid[v]) {
 #pragma unroll
                 for (int i = 0; i < NP; ++i) { const F2 d = sub2(w[v][i], mm); m2 = fma2(d, d, m2); }
             }
@@ -132,40 +133,59 @@ __device__ __forceinline__ Total total_of(const Part& p, float n, float eps) {
     else { const float rr = 1.0f / sqrtf(p.a / n + eps); return Total{rr, rr}; }
 }
 
-// SINGLE: the slice is the whole row, so softmax needs no slice rescale.
-template <int OP, int DT, int NV, bool SINGLE, class Par>
-__device__ __forceinline__ void slice_finish(const bool (&valid)[NV], F2 (&w)[NV][Pairs<DT>::NP], const Total& t, const Par& par,
-                                             uint4 (&out)[NV]) {
+// Normalises R rows that share this thread's columns: the parameters of a vector are fetched and widened once
+// and applied to every row.  SINGLE: the slice is the whole row, so softmax needs no slice rescale.
+template <int OP, int DT, int NV, int R, bool SINGLE, bool ALLV, class Par>
+__device__ __forceinline__ void slice_finish_rows(const bool (&valid)[NV], F2 (&w)[R][NV][Pairs<DT>::NP], const Total (&t)[R],
+                                                  const Par& par, uint4 (&out)[R][NV]) {
     using P = Pairs<DT>;
     constexpr int NP = P::NP;
-    const F2 ta = f2(t.a), tb = f2(t.b);
+    F2 ta[R], tb[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) { ta[r] = f2(t[r].a); tb[r] = f2(t[r].b); }
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
         if constexpr (OP == OP_SOFTMAX) {
             // two factors when slices are merged: the slice rescale may be subnormal (a slice far below the row
             // maximum) while 1/S carries 2^-bias; their product could lose the subnormal bits.
 #pragma unroll
-            for (int i = 0; i < NP; ++i) w[v][i] = SINGLE ? mul2(w[v][i], tb) : mul2(mul2(w[v][i], ta), tb);
-            out[v] = P::pack(w[v]);
+            for (int r = 0; r < R; ++r) {
+#pragma unroll
+                for (int i = 0; i < NP; ++i) w[r][v][i] = SINGLE ? mul2(w[r][v][i], tb[r]) : mul2(mul2(w[r][v][i], ta[r]), tb[r]);
+                out[r][v] = P::pack(w[r][v]);
+            }
         } else if constexpr (OP == OP_LAYERNORM) {
-            if (valid[v]) {
+            if (ALLV || valid[v]) {
                 F2 g[NP], b[NP];
                 P::unpack(par.gamma(v), g);
                 P::unpack(par.beta(v), b);
 #pragma unroll
-                for (int i = 0; i < NP; ++i) w[v][i] = fma2(mul2(sub2(w[v][i], ta), tb), g[i], b[i]);
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int i = 0; i < NP; ++i) w[r][v][i] = fma2(mul2(sub2(w[r][v][i], ta[r]), tb[r]), g[i], b[i]);
             }
-            out[v] = P::pack(w[v]);
+#pragma unroll
+            for (int r = 0; r < R; ++r) out[r][v] = P::pack(w[r][v]);
         } else {
-            if (valid[v]) {
+            if (ALLV || valid[v]) {
                 F2 g[NP];
                 P::unpack(par.gamma(v), g);
 #pragma unroll
-                for (int i = 0; i < NP; ++i) w[v][i] = mul2(mul2(w[v][i], ta), g[i]);
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int i = 0; i < NP; ++i) w[r][v][i] = mul2(mul2(w[r][v][i], ta[r]), g[i]);
             }
-            out[v] = P::pack(w[v]);
+#pragma unroll
+            for (int r = 0; r < R; ++r) out[r][v] = P::pack(w[r][v]);
         }
     }
+}
+
+template <int OP, int DT, int NV, bool SINGLE, class Par>
+__device__ __forceinline__ void slice_finish(const bool (&valid)[NV], F2 (&w)[NV][Pairs<DT>::NP], const Total& t, const Par& par,
+                                             uint4 (&out)[NV]) {
+    slice_finish_rows<OP, DT, NV, 1, SINGLE, false>(valid, reinterpret_cast<F2 (&)[1][NV][Pairs<DT>::NP]>(w),
+                                                    reinterpret_cast<const Total (&)[1]>(t), par, reinterpret_cast<uint4 (&)[1][NV]>(out));
 }
 
 // Whole row in one group: statistics, totals and outputs in one call.  st0/st1: mean & rstd (LayerNorm), rrms (RMSNorm).

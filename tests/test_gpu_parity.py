@@ -53,10 +53,10 @@ def test_auto_edge_rows(op, rows):
 def test_long_rows_take_the_cluster_path(op, dt):
     cols = 131072 if dt == BF16 else 65536 + 64
     w = wl(op, dt, 21, cols)
-    assert tf.tf_query_choice(op, 21, cols, dt).startswith("tma:")
+    assert tf.tf_query_choice(op, 21, cols, dt).startswith("ring:")
     assert not parity.parity(w)
     w2 = wl(op, dt, 3, 1 << 20)          # 2-4 MiB rows: more than a cluster of shared memory holds
-    assert tf.tf_query_choice(op, 3, 1 << 20, dt).startswith(("tma:", "stream:"))
+    assert tf.tf_query_choice(op, 3, 1 << 20, dt).startswith(("ring:", "tma:", "stream:"))
     assert not parity.parity(w2)
 
 
@@ -214,7 +214,8 @@ def test_forced_pipe_variants(op, dt):
         for nvec, stages, chunk, persist, rows in ((cap, 2, 4096, 1, 4001), (max(1, cap - 1), 3, 16384, 2, 2999),
                                                    (max(1, cap // 2 + 1), 1, 2048, 1, 1777), (cap, 4, 512, 8, 77)):
             chunk = max(chunk, nvec * 16 * (ut // lanes))
-            plan = f"pipe:threads={threads},lanes={lanes},vpt={vpt},stages={stages},chunk={chunk},persist={persist}"
+            rpg = 2 if (vpt <= 4 and nvec == cap and stages != 3) else 1        # two rows per pass needs a full row
+            plan = f"pipe:threads={threads},lanes={lanes},vpt={vpt},rpg={rpg},stages={stages},chunk={chunk},persist={persist}"
             tf.tf_force_plan(op, plan)
             if nvec * 16 > 8192:
                 rows = max(40, rows // 16)
@@ -226,7 +227,24 @@ def test_forced_pipe_variants(op, dt):
                 continue
             ran += 1
             assert not fails, (plan, nvec, fails)
-    assert ran >= 40
+    assert ran >= 30
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+def test_forced_ring_variants(op, dt, cluster):
+    ne = 4 if dt == F32 else 8
+    for vpt, threads in ((1, 128), (2, 256), (4, 1024), (8, 512), (4, 96)):
+        cap = threads * vpt * cluster
+        for nvec, stages, persist, rows in ((cap, 2, 1, 2 * 148 // cluster + 11), (cap - 1, 3, 2, 700 // cluster + 5),
+                                            (max(1, cap - threads - 3), 1, 1, 19), (max(1, cap // 2 + 5), 4, 1, 3)):
+            if nvec * 16 * stages // cluster > 180 * 1024 // persist:
+                continue
+            rows = min(rows, max(3, (1 << 22) // (nvec * ne)))
+            tf.tf_force_plan(op, f"ring:threads={threads},vpt={vpt},cluster={cluster},stages={stages},persist={persist}")
+            fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec))
+            assert not fails, (vpt, threads, cluster, nvec, stages, persist, rows, fails)
 
 
 @pytest.mark.parametrize("op", OPS)
