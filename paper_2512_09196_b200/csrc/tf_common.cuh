@@ -149,6 +149,12 @@ template <int DT> __device__ __forceinline__ float vec_max(const uint4& v) {
     }
 }
 
+// Programmatic dependent launch: every kernel is launched with programmatic stream serialisation, so its
+// CTAs may be scheduled while the previous kernel of the stream drains.  pdl_wait() orders all later global
+// accesses after that kernel's completion; pdl_trigger() lets the next kernel start being scheduled.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------------------------------------
 // Reductions.
 // ---------------------------------------------------------------------------------------------

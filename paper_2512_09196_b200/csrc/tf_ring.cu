@@ -84,6 +84,7 @@ __device__ __forceinline__ void rbulk_load(void* dst, const void* src, uint32_t 
 }
 
 constexpr int ring_max_threads(int vpt) { return vpt <= 4 ? 1024 : 512; }
+__device__ __forceinline__ bool valid_at(int idx, int len) { return idx < len; }
 
 template <int OP, int DT, int VPT>
 __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
@@ -132,7 +133,18 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
 #pragma unroll
     for (int v = 0; v < VPT; ++v) valid[v] = (t + v * T) < len;
     const CtaRed red{red_buf};
-    const LazyParams par{a.p0, a.p1, first + t, T};
+    // A persistent CTA always owns the same columns: with few vectors per thread their parameters live in
+    // registers for the whole kernel; otherwise they are fetched from L1/L2 when the normalise pass needs them.
+    constexpr bool kHeld = (VPT <= 4) && OP != OP_SOFTMAX;
+    HeldParams<kHeld ? VPT : 1> held;
+    if constexpr (kHeld) {
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            held.g[v] = valid_at(t + v * T, len) ? ld_param(a.p0 + first + t + v * T) : make_uint4(0, 0, 0, 0);
+            held.b[v] = (OP == OP_LAYERNORM && valid_at(t + v * T, len)) ? ld_param(a.p1 + first + t + v * T) : make_uint4(0, 0, 0, 0);
+        }
+    }
+    const LazyParams lazy{a.p0, a.p1, first + t, T};
     const uint4 fill = fill_vec<DT>(OP);
     auto slice_count = [&](int k) { return static_cast<float>(max(0, min(per, a.nvec - k * per))) * NE; };
 
@@ -166,7 +178,8 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
             __syncthreads();
         }
         const Total tot = combine_parts<OP>(cs, rank, [&](int k) { return Part{xch[xb][k][0], xch[xb][k][1]}; }, slice_count, a.n, a.eps);
-        slice_finish<OP, DT, VPT, false>(valid, w, tot, par, out);
+        if constexpr (kHeld) slice_finish<OP, DT, VPT, false>(valid, w, tot, held, out);
+        else slice_finish<OP, DT, VPT, false>(valid, w, tot, lazy, out);
         uint4* yr = a.y + row * a.nvec + first + t;
 #pragma unroll
         for (int v = 0; v < VPT; ++v)

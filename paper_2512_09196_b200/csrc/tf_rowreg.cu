@@ -41,6 +41,8 @@ constexpr int cta_max_threads(int vpt) { return vpt <= 2 ? 1024 : 512; }
 // =====================================================================================================
 template <int OP, int DT, int LANES, int VPT, int RPG>
 __global__ void __launch_bounds__(kWarpMaxThreads) k_warp(const KArgs a) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x % LANES;
     const int gpc = blockDim.x / LANES;                                   // groups per CTA
     const int64_t g = static_cast<int64_t>(blockIdx.x) * gpc + threadIdx.x / LANES;
@@ -97,6 +99,8 @@ __global__ void __launch_bounds__(cta_max_threads(VPT)) k_cta(const KArgs a, con
     __shared__ float red_buf[4 * 32];
     __shared__ float xch[2][kMaxCluster][2];          // partials pushed by the peers, double-buffered by row parity
 
+    pdl_wait();
+    pdl_trigger();
     const int T = blockDim.x, t = threadIdx.x;
     const int rank = CLUSTER ? static_cast<int>(blockIdx.x % cs) : 0;
     const int64_t cluster_id = CLUSTER ? blockIdx.x / cs : blockIdx.x;
@@ -221,8 +225,16 @@ cudaError_t launch_warp(const Plan& p, const Args& a, const DeviceInfo& d, cudaS
     int64_t grid = (a.rows + rows_per_cta - 1) / rows_per_cta;
     if (p.persist > 0) grid = std::min<int64_t>(grid, static_cast<int64_t>(p.persist) * d.sms);
     grid = std::min<int64_t>(grid, 0x7FFFFFFF);
-    fn<<<static_cast<unsigned>(grid), p.threads, 0, st>>>(make_kargs(a));
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(p.threads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, make_kargs(a));
 }
 
 bool supports_cta(const Plan& p, const Args& a, const DeviceInfo& d) {
@@ -246,11 +258,13 @@ cudaError_t launch_cta(const Plan& p, const Args& a, const DeviceInfo& d, cudaSt
     cfg.blockDim = dim3(p.threads);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = p.cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = p.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = p.cluster > 1 ? 1 : 0;
+    cfg.numAttrs = p.cluster > 1 ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, fn, make_kargs(a), p.cluster);
 }
 

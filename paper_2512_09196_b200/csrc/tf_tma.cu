@@ -105,6 +105,8 @@ __global__ void __launch_bounds__(1024) k_tma(const TArgs a) {
             for (int c = 0; c < nchunk; ++c) mbar_init(&mbar[s][c], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    pdl_wait();
+    pdl_trigger();
     __syncthreads();
     if (cs > 1) cl.sync();                 // all CTAs of the cluster resident before any remote shared-memory write
 
@@ -330,11 +332,13 @@ cudaError_t launch_tma(const Plan& p, const Args& a, const DeviceInfo& d, cudaSt
     cfg.blockDim = dim3(p.threads);
     cfg.dynamicSmemBytes = g.smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = p.cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = p.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = p.cluster > 1 ? 1 : 0;
+    cfg.numAttrs = p.cluster > 1 ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, fn, k);
 }
 

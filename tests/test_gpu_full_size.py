@@ -91,3 +91,23 @@ def test_tune_is_idempotent_and_candidates_all_pass_parity():
     finally:
         tf.tf_force_plan(w.op, None)
         tf.tf_clear_cache()
+
+
+def test_host_pipeline_matches_single_call():
+    """The overlapped host path (row blocks on three streams) gives exactly the single-call result."""
+    from paper_2512_09196_b200.host import HostPipeline
+    w = inputs.Workload("host_case", "layernorm", inputs.BF16, 1037, 2048, seed=4, x_mean=0.5, x_std=3.0, eps=1e-5)
+    data = w.generate()
+    pin = lambda a: torch.from_numpy(a).view(torch.bfloat16).pin_memory()
+    hx, hg, hb = pin(data["x"]), pin(data["gamma"]), pin(data["beta"])
+    hy = torch.empty_like(hx).pin_memory()
+    hmean, hrstd = torch.empty(w.rows).pin_memory(), torch.empty(w.rows).pin_memory()
+    dev = torch.device("cuda", 0)
+    dp = {"gamma": torch.empty_like(hg, device=dev), "beta": torch.empty_like(hb, device=dev)}
+    pipe = HostPipeline("layernorm", w.rows, w.cols, torch.bfloat16, dev, blocks=5)
+    for _ in range(2):
+        pipe.run(hx, hy, {"gamma": hg, "beta": hb}, dp, w.eps, hmean, hrstd)
+    torch.cuda.synchronize()
+    tf.tf_device_status()
+    got = {"y": hy.view(torch.uint16).numpy(), "mean": hmean.numpy(), "rstd": hrstd.numpy()}
+    assert not parity.check(w, data, got, parity.run_oracle(w, data))
