@@ -68,7 +68,7 @@ tf_status device_state(DevState** out) {
 // ------------------------------------------------------------------------------------------------
 // plans as text
 // ------------------------------------------------------------------------------------------------
-const char* kVariantName[V_COUNT] = {"warp", "cta", "tma", "stream", "pipe", "ring"};
+const char* kVariantName[V_COUNT] = {"warp", "cta", "tma", "stream", "pipe", "ring", "twopass"};
 
 std::string plan_to_string(const Plan& p) {
     char b[160];
@@ -78,6 +78,7 @@ std::string plan_to_string(const Plan& p) {
         case V_TMA: snprintf(b, sizeof b, "tma:threads=%d,cluster=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.cluster, p.stages, p.chunk, p.persist); break;
         case V_PIPE: snprintf(b, sizeof b, "pipe:threads=%d,lanes=%d,vpt=%d,rpg=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.lanes, p.vpt, p.rpg, p.stages, p.chunk, p.persist); break;
         case V_RING: snprintf(b, sizeof b, "ring:threads=%d,vpt=%d,cluster=%d,stages=%d,persist=%d", p.threads, p.vpt, p.cluster, p.stages, p.persist); break;
+        case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,persist=%d", p.threads, p.persist); break;
         default: snprintf(b, sizeof b, "stream:threads=%d,lanes=%d,persist=%d", p.threads, p.lanes, p.persist); break;
     }
     return b;
@@ -124,6 +125,7 @@ bool supports(const Plan& p, const Args& a, const DeviceInfo& d) {
         case V_STREAM: return supports_stream(p, a, d);
         case V_PIPE: return supports_pipe(p, a, d);
         case V_RING: return supports_ring(p, a, d);
+        case V_TWOPASS: return supports_twopass(p, a, d);
     }
     return false;
 }
@@ -136,6 +138,7 @@ cudaError_t launch(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream
         case V_TMA: return launch_tma(p, a, d, st);
         case V_PIPE: return launch_pipe(p, a, d, st);
         case V_RING: return launch_ring(p, a, d, st);
+        case V_TWOPASS: return launch_twopass(p, a, d, st);
         default: return launch_stream(p, a, d, st);
     }
 }
@@ -201,7 +204,13 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         else { p.vpt = 8; p.cluster = 2; p.threads = round_up(static_cast<int>((nvec + 15) / 16), 32); }
         return p;
     }
-    // long rows: persistent clusters with a prefetch ring, slices of at most 64 KiB (4 vectors per thread)
+    // long rows: two streamed passes for LayerNorm (its parameters make register-resident slices costly) and for
+    // everything beyond 128 KiB; persistent clusters with a prefetch ring in between
+    if (a.op == OP_LAYERNORM || nvec > 8192) {
+        Plan s;
+        s.variant = V_TWOPASS; s.threads = 512;
+        return s;
+    }
     {
         Plan r;
         r.variant = V_RING; r.vpt = 4; r.stages = 2;
@@ -223,7 +232,7 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
     p.cluster = cl;
     if (!supports_tma(p, a, d)) {           // longer than a full cluster of shared memory can hold
         Plan s;
-        s.variant = V_STREAM; s.lanes = 0; s.threads = 1024;
+        s.variant = V_TWOPASS; s.threads = 1024;
         return s;
     }
     return p;
@@ -295,6 +304,10 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
             }
         }
     }
+    // two streamed passes (second from L2) for long rows
+    if (nvec >= 1024)
+        for (int th : {256, 512, 1024})
+            for (int persist : {0, 2048 / th}) { Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = persist; add(p); }
     // persistent cluster ring for long rows
     if (nvec >= 2048)
         for (int cl : {1, 2, 4, 8})

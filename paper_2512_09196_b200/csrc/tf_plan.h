@@ -16,7 +16,8 @@ enum Variant : int {
     V_STREAM = 3,   // generic: scalar accesses, several passes over the row, any alignment and length
     V_PIPE = 4,     // persistent CTAs: a producer thread streams row tiles into a shared-memory ring, consumer warps normalise
     V_RING = 5,     // persistent clusters: each CTA prefetches its slice of a long row into a shared-memory ring, registers hold it
-    V_COUNT = 6
+    V_TWOPASS = 6,  // CTA per row, the row streamed twice with vector loads (second time from L2); any row length
+    V_COUNT = 7
 };
 
 struct Plan {
@@ -64,12 +65,14 @@ bool supports_tma(const Plan&, const Args&, const DeviceInfo&);
 bool supports_stream(const Plan&, const Args&, const DeviceInfo&);
 bool supports_pipe(const Plan&, const Args&, const DeviceInfo&);
 bool supports_ring(const Plan&, const Args&, const DeviceInfo&);
+bool supports_twopass(const Plan&, const Args&, const DeviceInfo&);
 cudaError_t launch_warp(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_cta(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_tma(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_stream(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_pipe(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_ring(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+cudaError_t launch_twopass(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 
 // Raises a kernel's dynamic shared-memory limit to the device's opt-in maximum, once per kernel and device.
 cudaError_t ensure_max_smem(const void* fn, const DeviceInfo&);

@@ -53,10 +53,10 @@ def test_auto_edge_rows(op, rows):
 def test_long_rows_take_the_cluster_path(op, dt):
     cols = 131072 if dt == BF16 else 65536 + 64
     w = wl(op, dt, 21, cols)
-    assert tf.tf_query_choice(op, 21, cols, dt).startswith("ring:")
+    assert tf.tf_query_choice(op, 21, cols, dt).startswith(("ring:", "twopass:"))
     assert not parity.parity(w)
     w2 = wl(op, dt, 3, 1 << 20)          # 2-4 MiB rows: more than a cluster of shared memory holds
-    assert tf.tf_query_choice(op, 3, 1 << 20, dt).startswith(("ring:", "tma:", "stream:"))
+    assert tf.tf_query_choice(op, 3, 1 << 20, dt).startswith(("ring:", "tma:", "twopass:"))
     assert not parity.parity(w2)
 
 
@@ -245,6 +245,26 @@ def test_forced_ring_variants(op, dt, cluster):
             tf.tf_force_plan(op, f"ring:threads={threads},vpt={vpt},cluster={cluster},stages={stages},persist={persist}")
             fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec))
             assert not fails, (vpt, threads, cluster, nvec, stages, persist, rows, fails)
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_forced_twopass_variants(op, dt):
+    ne = 4 if dt == F32 else 8
+    for threads, persist in ((32, 0), (256, 1), (1024, 0)):
+        for nvec, rows in ((1, 5), (threads * 4, 9), (threads * 4 + 1, 9), (threads * 9 - 3, 300), (70001, 3)):
+            tf.tf_force_plan(op, f"twopass:threads={threads},persist={persist}")
+            fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec))
+            assert not fails, (threads, persist, nvec, rows, fails)
+    if op == "softmax":                                    # masks, a fully masked row and outputs in the subnormal range
+        tf.tf_force_plan(op, "twopass:threads=256,persist=0")
+        w = Workload("m", "softmax", dt, 12, 40000, seed=5, x_std=10.0, mask_step=3001)
+        data = w.generate()
+        ninf = np.float32(-np.inf) if dt == F32 else np.uint16(0xFF80)
+        data["x"][3, :] = ninf
+        data["x"][5, :20000] = ninf
+        data["x"][7, 0] = np.float32(75.0) if dt == F32 else np.uint16(0x4296)
+        assert not parity.check(w, data, parity.run_gpu(w, data), parity.run_oracle(w, data))
 
 
 @pytest.mark.parametrize("op", OPS)
