@@ -149,6 +149,13 @@ template <int DT> __device__ __forceinline__ float vec_max(const uint4& v) {
     }
 }
 
+// Per-row scalars (1/n, 1/sqrt(var + eps), 1/sum) use the approximate MUFU forms: their relative error is about
+// 2^-22, two orders below the 1e-5 tolerance, and the IEEE sequences would cost 10-20 instructions per row in
+// every thread, which matters for rows of a few hundred bytes.  None of them flushes subnormals.
+__device__ __forceinline__ float fast_div(float a, float b) { return __fdividef(a, b); }      // |b| < 2^126
+__device__ __forceinline__ float fast_rsqrt(float v) { return rsqrtf(v); }
+__device__ __forceinline__ float fast_rcp(float v) { return __frcp_rn(v); }
+
 // Programmatic dependent launch: every kernel is launched with programmatic stream serialisation, so its
 // CTAs may be scheduled while the previous kernel of the stream drains.  pdl_wait() orders all later global
 // accesses after that kernel's completion; pdl_trigger() lets the next kernel start being scheduled.
@@ -195,7 +202,7 @@ struct MomentPartial { float n, mean, m2; };
 __device__ __forceinline__ MomentPartial chan_combine(const MomentPartial& a, const MomentPartial& b) {
     if (b.n == 0.f) return a;
     if (a.n == 0.f) return b;
-    const float n = a.n + b.n, d = b.mean - a.mean, f = b.n / n;
+    const float n = a.n + b.n, d = b.mean - a.mean, f = fast_div(b.n, n);
     return MomentPartial{n, fmaf(d, f, a.mean), a.m2 + b.m2 + d * d * a.n * f};
 }
 

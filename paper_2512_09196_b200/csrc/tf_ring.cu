@@ -249,11 +249,10 @@ cudaError_t launch_ring(const Plan& p, const Args& a, const DeviceInfo& d, cudaS
     cfg.blockDim = dim3(p.threads);
     cfg.dynamicSmemBytes = ring_smem(p, a);
     cfg.stream = st;
-    cudaLaunchAttribute attr[2];
+    // No programmatic early launch here: a persistent cluster that could only be placed after the previous
+    // kernel has drained would start late with a full share of rows and double the kernel's duration.
+    cudaLaunchAttribute attr[1];
     int na = 0;
-    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[na].val.programmaticStreamSerializationAllowed = 1;
-    ++na;
     if (p.cluster > 1) {
         attr[na].id = cudaLaunchAttributeClusterDimension;
         attr[na].val.clusterDim.x = p.cluster; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;

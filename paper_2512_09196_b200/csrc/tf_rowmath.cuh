@@ -80,7 +80,7 @@ __device__ __forceinline__ Part slice_stats(const uint4 (&raw)[NV], const bool (
             for (int i = 0; i < NP; ++i) s = add2(s, w[v][i]);
         }
         const float tot = red.sum(hsum(s), slot0);
-        const float mean = (n_slice > 0.f) ? tot / n_slice : 0.f;
+        const float mean = (n_slice > 0.f) ? fast_div(tot, n_slice) : 0.f;
         const F2 mm = f2(mean);
         F2 m2 = f2(0.f);
 #pragma unroll
@@ -112,15 +112,15 @@ __device__ __forceinline__ Total combine_parts(int K, int mine, const Get& get, 
         for (int k = 0; k < K; ++k) O = fminf(O, get(k).a);
         float S = 0.f;
         for (int k = 0; k < K; ++k) { const Part p = get(k); S = fmaf(p.b, softmax_rescale(O, p.a), S); }
-        return Total{softmax_rescale(O, get(mine).a), (S == 0.f) ? 0.f : 1.0f / S};
+        return Total{softmax_rescale(O, get(mine).a), (S == 0.f) ? 0.f : fast_rcp(S)};
     } else if constexpr (OP == OP_LAYERNORM) {
         MomentPartial acc{0.f, 0.f, 0.f};
         for (int k = 0; k < K; ++k) { const Part p = get(k); acc = chan_combine(acc, MomentPartial{count(k), p.a, p.b}); }
-        return Total{acc.mean, 1.0f / sqrtf(acc.m2 / n + eps)};
+        return Total{acc.mean, fast_rsqrt(fast_div(acc.m2, n) + eps)};
     } else {
         float tot = 0.f;
         for (int k = 0; k < K; ++k) tot += get(k).a;
-        const float rr = 1.0f / sqrtf(tot / n + eps);
+        const float rr = fast_rsqrt(fast_div(tot, n) + eps);
         return Total{rr, rr};
     }
 }
@@ -128,9 +128,9 @@ __device__ __forceinline__ Total combine_parts(int K, int mine, const Get& get, 
 // The single-slice case of combine_parts (the group holds the whole row).
 template <int OP>
 __device__ __forceinline__ Total total_of(const Part& p, float n, float eps) {
-    if constexpr (OP == OP_SOFTMAX) return Total{1.0f, (p.b == 0.f) ? 0.f : 1.0f / p.b};
-    else if constexpr (OP == OP_LAYERNORM) return Total{p.a, 1.0f / sqrtf(p.b / n + eps)};
-    else { const float rr = 1.0f / sqrtf(p.a / n + eps); return Total{rr, rr}; }
+    if constexpr (OP == OP_SOFTMAX) return Total{1.0f, (p.b == 0.f) ? 0.f : fast_rcp(p.b)};
+    else if constexpr (OP == OP_LAYERNORM) return Total{p.a, fast_rsqrt(fast_div(p.b, n) + eps)};
+    else { const float rr = fast_rsqrt(fast_div(p.a, n) + eps); return Total{rr, rr}; }
 }
 
 // Normalises R rows that share this thread's columns: the parameters of a vector are fetched and widened once

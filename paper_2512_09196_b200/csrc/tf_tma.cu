@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(1024) k_tma(const TArgs a) {
             for (int k = 0; k < cs; ++k) O = fminf(O, xch[xb][k][0]);
             float S = 0.f;
             for (int k = 0; k < cs; ++k) S = fmaf(xch[xb][k][1], softmax_rescale(O, xch[xb][k][0]), S);
-            const float inv = (S == 0.f) ? 0.f : 1.0f / S;
+            const float inv = (S == 0.f) ? 0.f : fast_rcp(S);
             // pass 3: y = 2^(x*log2e + O) / S with the row-wide offset O; store
             const F2 O2 = f2(O), inv2 = f2(inv);
 #pragma unroll 4
@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(1024) k_tma(const TArgs a) {
                 }
             }
             const float s = cta_reduce<SumOp>(hsum(s2), rb0);
-            const float mk = (len > 0) ? s / slice_count(rank) : 0.f;
+            const float mk = (len > 0) ? fast_div(s, slice_count(rank)) : 0.f;
             const F2 mk2 = f2(mk);
             F2 q2 = f2(0.f);
 #pragma unroll 4

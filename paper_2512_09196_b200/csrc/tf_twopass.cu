@@ -114,7 +114,7 @@ __global__ void __launch_bounds__(1024) k_twopass(const WArgs a) {
                     for (int i = 0; i < NP; ++i) s2 = add2(s2, w[u][i]);
                 }
                 const float nc = static_cast<float>(cnt);
-                const float mc = hsum(s2) / nc;                // cnt > 0: base < nvec
+                const float mc = fast_div(hsum(s2), nc);                // cnt > 0: base < nvec
                 const F2 mc2 = f2(mc);
                 F2 d2 = f2(0.f);
 #pragma unroll
@@ -142,15 +142,15 @@ __global__ void __launch_bounds__(1024) k_twopass(const WArgs a) {
             const float O = exp_offset(M);
             const float mine = (s_max == kNegInf) ? 0.f : s_sum * ex2(O - s_off);       // O <= s_off: factor <= 1
             const float S = cta_reduce<SumOp>(mine, rb + 32);
-            ta = O; tb = (S == 0.f) ? 0.f : 1.0f / S;
+            ta = O; tb = (S == 0.f) ? 0.f : fast_rcp(S);
         } else if constexpr (OP == OP_LAYERNORM) {
-            const float mean = cta_reduce<SumOp>(c_n * c_mean, rb) / a.n;
+            const float mean = fast_div(cta_reduce<SumOp>(c_n * c_mean, rb), a.n);
             const float d = c_mean - mean;
             const float m2 = cta_reduce<SumOp>(fmaf(c_n * d, d, c_m2), rb + 32);          // sum of M2_t + n_t (mean_t - mean)^2
-            ta = mean; tb = 1.0f / sqrtf(m2 / a.n + a.eps);
+            ta = mean; tb = fast_rsqrt(fast_div(m2, a.n) + a.eps);
         } else {
             const float tot = cta_reduce<SumOp>(hsum(q2), rb);
-            ta = tb = 1.0f / sqrtf(tot / a.n + a.eps);
+            ta = tb = fast_rsqrt(fast_div(tot, a.n) + a.eps);
         }
         if (t == 0) {
             if (OP == OP_LAYERNORM && a.mean) a.mean[row] = ta;
