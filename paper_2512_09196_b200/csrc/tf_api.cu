@@ -68,7 +68,7 @@ tf_status device_state(DevState** out) {
 // ------------------------------------------------------------------------------------------------
 // plans as text
 // ------------------------------------------------------------------------------------------------
-const char* kVariantName[V_COUNT] = {"warp", "cta", "tma", "stream", "pipe", "ring", "twopass"};
+const char* kVariantName[V_COUNT] = {"warp", "cta", "tma", "stream", "pipe", "ring", "twopass", "split"};
 
 std::string plan_to_string(const Plan& p) {
     char b[160];
@@ -79,6 +79,7 @@ std::string plan_to_string(const Plan& p) {
         case V_PIPE: snprintf(b, sizeof b, "pipe:threads=%d,lanes=%d,vpt=%d,rpg=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.lanes, p.vpt, p.rpg, p.stages, p.chunk, p.persist); break;
         case V_RING: snprintf(b, sizeof b, "ring:threads=%d,vpt=%d,cluster=%d,stages=%d,persist=%d", p.threads, p.vpt, p.cluster, p.stages, p.persist); break;
         case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,persist=%d", p.threads, p.persist); break;
+        case V_SPLIT: snprintf(b, sizeof b, "split:threads=%d,splits=%d", p.threads, p.cluster); break;
         default: snprintf(b, sizeof b, "stream:threads=%d,lanes=%d,persist=%d", p.threads, p.lanes, p.persist); break;
     }
     return b;
@@ -104,7 +105,7 @@ bool plan_from_string(const char* s, Plan& out) {
         long val = strtol(eq + 1, &end, 10);
         if (end == eq + 1) return false;
         if (key == "threads") p.threads = val; else if (key == "lanes") p.lanes = val; else if (key == "vpt") p.vpt = val;
-        else if (key == "rpg") p.rpg = val; else if (key == "cluster") p.cluster = val; else if (key == "stages") p.stages = val;
+        else if (key == "rpg") p.rpg = val; else if (key == "cluster" || key == "splits") p.cluster = val; else if (key == "stages") p.stages = val;
         else if (key == "chunk") p.chunk = val; else if (key == "persist") p.persist = val; else return false;
         q = (*end == ',') ? end + 1 : end;
         if (*end && *end != ',') return false;
@@ -126,6 +127,7 @@ bool supports(const Plan& p, const Args& a, const DeviceInfo& d) {
         case V_PIPE: return supports_pipe(p, a, d);
         case V_RING: return supports_ring(p, a, d);
         case V_TWOPASS: return supports_twopass(p, a, d);
+        case V_SPLIT: return supports_split(p, a, d);
     }
     return false;
 }
@@ -139,6 +141,7 @@ cudaError_t launch(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream
         case V_PIPE: return launch_pipe(p, a, d, st);
         case V_RING: return launch_ring(p, a, d, st);
         case V_TWOPASS: return launch_twopass(p, a, d, st);
+        case V_SPLIT: return launch_split(p, a, d, st);
         default: return launch_stream(p, a, d, st);
     }
 }
@@ -174,6 +177,14 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         return p;
     }
     const int64_t nvec = row_bytes / 16;
+    if (a.rows <= 4 && row_bytes >= 256 * 1024) {
+        // a handful of very long rows: even a cluster per row would leave most SMs idle, so cut the rows into
+        // segments of at least 4 KiB, about two CTAs per SM (for more rows the second launch costs more than it saves)
+        Plan s;
+        s.variant = V_SPLIT; s.threads = 256;
+        s.cluster = static_cast<int>(std::max<int64_t>(2, std::min<int64_t>(nvec / 256, 2 * d.sms / a.rows)));
+        if (supports_split(s, a, d)) return s;
+    }
     if (nvec <= 4096) {
         // rows up to 64 KiB: the persistent self-feeding pipeline, one CTA of 512 threads per SM, two stages per unit
         p.variant = V_PIPE;
@@ -304,6 +315,14 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
             }
         }
     }
+    // few long rows: segments over many CTAs
+    if (a.rows * 2 <= d.sms && nvec >= 1024)
+        for (int mult : {1, 2, 4})
+            for (int th : {256, 512}) {
+                Plan p; p.variant = V_SPLIT; p.threads = th;
+                p.cluster = static_cast<int>(std::max<int64_t>(2, std::min<int64_t>(nvec / 128, static_cast<int64_t>(mult) * d.sms / a.rows)));
+                add(p);
+            }
     // two streamed passes (second from L2) for long rows
     if (nvec >= 1024)
         for (int th : {256, 512, 1024})

@@ -17,7 +17,8 @@ enum Variant : int {
     V_PIPE = 4,     // persistent CTAs: a producer thread streams row tiles into a shared-memory ring, consumer warps normalise
     V_RING = 5,     // persistent clusters: each CTA prefetches its slice of a long row into a shared-memory ring, registers hold it
     V_TWOPASS = 6,  // CTA per row, the row streamed twice with vector loads (second time from L2); any row length
-    V_COUNT = 7
+    V_SPLIT = 7,    // few very long rows: a row cut into segments over many CTAs, partials merged through global scratch
+    V_COUNT = 8
 };
 
 struct Plan {
@@ -26,7 +27,7 @@ struct Plan {
     int lanes = 32;      // V_WARP / V_PIPE: threads per row
     int vpt = 1;         // V_WARP / V_CTA / V_PIPE: 16-byte vectors held per thread
     int rpg = 1;         // V_WARP: rows a group has in flight per iteration
-    int cluster = 1;     // V_CTA / V_TMA: CTAs sharing one row
+    int cluster = 1;     // V_CTA / V_TMA / V_RING: CTAs sharing one row; V_SPLIT: segments per row
     int stages = 1;      // V_TMA / V_PIPE: shared-memory ring depth
     int chunk = 8192;    // V_TMA: bytes per bulk copy (one mbarrier each); V_PIPE: bytes per stage
     int persist = 0;     // 0: grid covers all rows once; k > 0: k CTAs per SM looping over rows (V_PIPE: always >= 1)
@@ -66,6 +67,7 @@ bool supports_stream(const Plan&, const Args&, const DeviceInfo&);
 bool supports_pipe(const Plan&, const Args&, const DeviceInfo&);
 bool supports_ring(const Plan&, const Args&, const DeviceInfo&);
 bool supports_twopass(const Plan&, const Args&, const DeviceInfo&);
+bool supports_split(const Plan&, const Args&, const DeviceInfo&);
 cudaError_t launch_warp(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_cta(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_tma(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
@@ -73,6 +75,10 @@ cudaError_t launch_stream(const Plan&, const Args&, const DeviceInfo&, cudaStrea
 cudaError_t launch_pipe(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_ring(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_twopass(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+cudaError_t launch_split(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+// The split plan with caller-provided scratch (split_scratch_bytes() of device memory).
+cudaError_t launch_split_with_scratch(const Plan&, const Args&, void* scratch, cudaStream_t);
+size_t split_scratch_bytes(const Plan&, const Args&);
 
 // Raises a kernel's dynamic shared-memory limit to the device's opt-in maximum, once per kernel and device.
 cudaError_t ensure_max_smem(const void* fn, const DeviceInfo&);

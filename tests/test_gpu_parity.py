@@ -53,10 +53,10 @@ def test_auto_edge_rows(op, rows):
 def test_long_rows_take_the_cluster_path(op, dt):
     cols = 131072 if dt == BF16 else 65536 + 64
     w = wl(op, dt, 21, cols)
-    assert tf.tf_query_choice(op, 21, cols, dt).startswith(("ring:", "twopass:"))
+    assert tf.tf_query_choice(op, 21, cols, dt).startswith(("ring:", "twopass:", "split:"))
     assert not parity.parity(w)
     w2 = wl(op, dt, 3, 1 << 20)          # 2-4 MiB rows: more than a cluster of shared memory holds
-    assert tf.tf_query_choice(op, 3, 1 << 20, dt).startswith(("ring:", "tma:", "twopass:"))
+    assert tf.tf_query_choice(op, 3, 1 << 20, dt).startswith(("ring:", "tma:", "twopass:", "split:"))
     assert not parity.parity(w2)
 
 
@@ -264,6 +264,30 @@ def test_forced_twopass_variants(op, dt):
         data["x"][3, :] = ninf
         data["x"][5, :20000] = ninf
         data["x"][7, 0] = np.float32(75.0) if dt == F32 else np.uint16(0x4296)
+        assert not parity.check(w, data, parity.run_gpu(w, data), parity.run_oracle(w, data))
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_forced_split_variants_and_few_long_rows(op, dt):
+    ne = 4 if dt == F32 else 8
+    for threads, splits, nvec, rows in ((32, 2, 5, 3), (256, 7, 4099, 4), (512, 64, 40000, 2), (1024, 300, 70001, 1), (128, 8, 8, 5)):
+        tf.tf_force_plan(op, f"split:threads={threads},splits={splits}")
+        fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec))
+        assert not fails, (threads, splits, nvec, rows, fails)
+    tf.tf_force_plan(op, None)
+    for rows, cols in ((1, 262144), (3, 524288), (8, 131072), (64, 32768)):  # what a decode-time vocabulary softmax looks like
+        if rows <= 4:
+            assert tf.tf_query_choice(op, rows, cols, dt).startswith("split:")
+        assert not parity.parity(wl(op, dt, rows, cols, seed=rows))
+    if op == "softmax":
+        tf.tf_force_plan(op, "split:threads=256,splits=16")
+        w = Workload("m", "softmax", dt, 6, 40000, seed=5, x_std=10.0, mask_step=3001)
+        data = w.generate()
+        ninf = np.float32(-np.inf) if dt == F32 else np.uint16(0xFF80)
+        data["x"][1, :] = ninf                                   # fully masked row
+        data["x"][2, :30000] = ninf                              # whole segments masked
+        data["x"][3, 0] = np.float32(75.0) if dt == F32 else np.uint16(0x4296)
         assert not parity.check(w, data, parity.run_gpu(w, data), parity.run_oracle(w, data))
 
 
