@@ -9,7 +9,10 @@
  *
  * Conventions for every *_fwd entry point
  *   Memory     All tensor pointers are DEVICE memory owned by the caller, on the current CUDA device.
- *              The library keeps no reference after the call returns and allocates nothing.
+ *              The library keeps no reference after the call returns.  It allocates nothing, with one
+ *              exception: for a handful of very long rows (rows <= 4, >= 256 KiB each) the split-row plan takes
+ *              8 bytes per row segment from the stream-ordered allocator (cudaMallocAsync / cudaFreeAsync on the
+ *              caller's stream) for the duration of the call.
  *   Layout     x and y are dense row-major [rows, cols] (row stride = cols); gamma/beta/weight are [cols];
  *              mean/rstd are [rows], always fp32.  x, y and the parameters share one element type `dt`.
  *   Alignment  Any.  A 16-byte aligned x, y and parameters with cols * sizeof(element) a multiple of 16
@@ -59,6 +62,25 @@ tf_status tf_layernorm_fwd(const void* x, const void* gamma, const void* beta, v
  * weight is required; rstd (= rrms) is an optional output. */
 tf_status tf_rmsnorm_fwd(const void* x, const void* weight, void* y, float* rstd, int64_t rows, int64_t cols,
                          float eps, tf_dtype dt, void* cuda_stream);
+
+/* Softmax (same definition and conventions as tf_softmax_fwd) for callers that must not trigger a device
+ * allocation: a process that handed all free device memory to its own pool at start-up (a later driver
+ * allocation could fail or stall there), or a latency-critical loop in which an allocation call may
+ * synchronise the device.  The paper has no counterpart; this exists for deployment.
+ * It always runs the split-row plan (each row cut into segments over many CTAs, one 8-byte partial per
+ * segment) with the partials in a fixed 64 KiB array inside the library (room for 8192 partials; every GPU
+ * that loads the library holds it until the process exits).  It calls no cudaMalloc / cudaFree or any other
+ * allocating routine.
+ *   Limits   rows <= 8192; x and y 16-byte aligned and cols * sizeof(element) a multiple of 16.  Anything else
+ *            returns TF_ERR_UNSUPPORTED and launches nothing.  Long rows are its purpose; short ones work
+ *            but are served better by tf_softmax_fwd.
+ *   Set-up   The first call on a device looks up the array's device address (with that device current).  Make
+ *            that first call before any stream capture begins.
+ *   Sharing  Every call on a device uses the same array, which keeps the previous call's partials.  Nothing in
+ *            it needs clearing (each call overwrites every partial it later reads), but two calls whose
+ *            kernels can overlap on the GPU (different streams without an ordering between them) race on it:
+ *            order such calls yourself. */
+tf_status tf_softmax_fwd_noalloc(const void* x, void* y, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
 
 /* Measure-and-keep tuning for one (op, rows, cols, dt) on the current device (Algorithm 1 of the paper,
  * with the hand-written launch plans as proposals): starting from the heuristic plan as incumbent, every

@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_report", "tf_status_string",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_report", "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
 
@@ -48,6 +48,7 @@ def lib() -> ctypes.CDLL:
         vp, i64, i32, f32, cp, sz = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float, ctypes.c_char_p,
                                      ctypes.c_size_t)
         L.tf_softmax_fwd.argtypes = [vp, vp, i64, i64, i32, vp]
+        L.tf_softmax_fwd_noalloc.argtypes = [vp, vp, i64, i64, i32, vp]
         L.tf_layernorm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_rmsnorm_fwd.argtypes = [vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_tune.argtypes = [i32, i64, i64, i32]
@@ -64,7 +65,7 @@ def lib() -> ctypes.CDLL:
         L.tf_clear_cache.restype = None
         L.tf_launch_count.argtypes = []
         L.tf_launch_count.restype = i64
-        for name in ("tf_softmax_fwd", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_report",
+        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_report",
                      "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice",
                      "tf_candidate_count", "tf_candidate"):
             getattr(L, name).restype = i32
@@ -127,6 +128,19 @@ def tf_softmax_fwd(x, y=None):
     rows, cols = x.shape
     with _on_device(x):
         _ok(lib().tf_softmax_fwd(x.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)), "tf_softmax_fwd")
+    return y
+
+
+def tf_softmax_fwd_noalloc(x, y):
+    """Softmax through the entry point that never allocates device memory: for processes that gave all free device
+    memory to their own pool at start-up, or loops that cannot afford an allocation call's possible synchronisation.
+    ``y`` must be preallocated (it may alias ``x``); rows <= 8192, 16-byte aligned tensors.  Calls that may overlap on
+    the GPU share one fixed scratch array inside the library and must be ordered by the caller."""
+    _check2d(x)
+    _check2d(y, "y")
+    rows, cols = x.shape
+    with _on_device(x):
+        _ok(lib().tf_softmax_fwd_noalloc(x.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)), "tf_softmax_fwd_noalloc")
     return y
 
 

@@ -150,6 +150,9 @@ int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 }  // namespace
 
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+void remember_cuda_error(cudaError_t e) { cuda_fail(e); }
+
 cudaError_t ensure_max_smem(const void* fn, const DeviceInfo& d) {
     static std::mutex mu;
     static std::map<std::pair<const void*, int>, bool> done;

@@ -80,6 +80,10 @@ cudaError_t launch_split(const Plan&, const Args&, const DeviceInfo&, cudaStream
 cudaError_t launch_split_with_scratch(const Plan&, const Args&, void* scratch, cudaStream_t);
 size_t split_scratch_bytes(const Plan&, const Args&);
 
+// Bookkeeping shared with the C ABI layer: count kernel launches; remember the CUDA error behind a TF_ERR_CUDA.
+void count_launches(int n);
+void remember_cuda_error(cudaError_t e);
+
 // Raises a kernel's dynamic shared-memory limit to the device's opt-in maximum, once per kernel and device.
 cudaError_t ensure_max_smem(const void* fn, const DeviceInfo&);
 

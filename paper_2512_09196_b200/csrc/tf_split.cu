@@ -152,3 +152,71 @@ cudaError_t launch_split(const Plan& p, const Args& a, const DeviceInfo&, cudaSt
 }
 
 }  // namespace tf
+
+// =====================================================================================================
+// tf_softmax_fwd_noalloc: the split plan with its scratch in a fixed device array of this module
+// =====================================================================================================
+#include <mutex>
+
+#include "../../include/tf.h"
+
+namespace tf {
+namespace {
+
+// Room for this many (row, segment) partials: 8192 x 8 bytes = 64 KiB, held by every GPU that loads the library
+// until the process exits.
+constexpr int kStaticPartials = 8192;
+static __device__ __align__(256) float2 g_static_partials[kStaticPartials];
+
+struct StaticScratch { void* ptr = nullptr; int sms = 0; bool ready = false; };
+std::mutex g_static_mu;
+StaticScratch g_static[64];
+
+// Once per device, with that device current: the device address of the array (in host code its name is only a
+// stand-in, not something a kernel can be given) and the SM count.  Allocates nothing.
+cudaError_t static_scratch(StaticScratch** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    StaticScratch& s = g_static[dev];
+    if (!s.ready) {
+        void* p = nullptr;
+        if ((e = cudaGetSymbolAddress(&p, g_static_partials)) != cudaSuccess) return e;
+        int sms = 0;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        s.ptr = p; s.sms = sms; s.ready = true;
+    }
+    *out = &s;
+    return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace tf
+
+extern "C" tf_status tf_softmax_fwd_noalloc(const void* x, void* y, int64_t rows, int64_t cols, tf_dtype dt_, void* stream) {
+    using namespace tf;
+    const int dt = dt_;
+    if (rows < 0 || cols <= 0 || (dt != DT_F32 && dt != DT_BF16) || (rows > 0 && (!x || !y))) return TF_ERR_INVALID_ARG;
+    if (rows == 0) return TF_OK;
+    Args a{OP_SOFTMAX, dt, x, nullptr, nullptr, y, nullptr, nullptr, rows, cols, 0.f, nullptr};
+    if (!vector_ok(a)) return TF_ERR_UNSUPPORTED;                 // needs 16-byte aligned x, y and cols * size % 16 == 0
+    if (rows > kStaticPartials) return TF_ERR_UNSUPPORTED;        // more rows than the fixed scratch has partials for
+    StaticScratch* sc = nullptr;
+    cudaError_t e = static_scratch(&sc);
+    if (e != cudaSuccess) { remember_cuda_error(e); return TF_ERR_CUDA; }
+    // about two CTAs per SM, segments of at least 4 KiB, and never more partials than the array holds
+    const int64_t nvec = cols * elem_size(dt) / 16;
+    int64_t splits = std::max<int64_t>(1, 2 * static_cast<int64_t>(sc->sms) / rows);
+    splits = std::min<int64_t>(splits, std::max<int64_t>(1, nvec / 256));
+    splits = std::min<int64_t>(splits, kStaticPartials / rows);
+    Plan p;
+    p.variant = V_SPLIT; p.threads = 256; p.cluster = static_cast<int>(splits);
+    DeviceInfo d;
+    if (!supports_split(p, a, d)) return TF_ERR_UNSUPPORTED;
+    count_launches(2);
+    e = launch_split_with_scratch(p, a, sc->ptr, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { remember_cuda_error(e); return TF_ERR_CUDA; }
+    return TF_OK;
+}
