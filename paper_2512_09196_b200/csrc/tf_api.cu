@@ -52,12 +52,13 @@ tf_status device_state(DevState** out) {
     std::lock_guard<std::mutex> lk(g_mu);
     DevState& d = g_dev[dev];
     if (!d.ok) {
-        int sms = 0, smem = 0;
+        int sms = 0, smem = 0, l2 = 0;
         if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return cuda_fail(e);
         if ((e = cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev)) != cudaSuccess) return cuda_fail(e);
         void* p = nullptr;
         if ((e = cudaGetSymbolAddress(&p, g_status_word)) != cudaSuccess) return cuda_fail(e);
-        d.info.ordinal = dev; d.info.sms = sms; d.info.smem_optin = smem; d.info.max_cluster = kMaxCluster;
+        d.info.ordinal = dev; d.info.sms = sms; d.info.smem_optin = smem; d.info.max_cluster = kMaxCluster; d.info.l2_bytes = l2;
         d.status = static_cast<int*>(p);
         d.ok = true;
     }

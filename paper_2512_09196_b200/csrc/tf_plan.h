@@ -51,6 +51,7 @@ struct DeviceInfo {
     int sms = 0;
     int smem_optin = 0;          // max dynamic shared memory per CTA, bytes
     int max_cluster = 8;
+    int l2_bytes = 0;            // L2 cache size
 };
 
 // Geometry limits shared by the dispatcher and the kernels.

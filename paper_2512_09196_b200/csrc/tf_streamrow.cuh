@@ -160,7 +160,9 @@ __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const u
     const int T = blockDim.x, t = threadIdx.x;
     const uint4 fill = fill_vec<DT>(OP);
     const F2 ta2 = f2(sc.a), tb2 = f2(sc.b), l2e = f2(kLog2e);
-    for (int64_t base = t; base < nvec; base += static_cast<int64_t>(T) * U) {
+    // back to front: the end of the segment is what pass A touched last, hence what L2 most likely still holds
+    const int64_t step = static_cast<int64_t>(T) * U;
+    for (int64_t base = (nvec - 1) / step * step + t; base >= 0; base -= step) {
         uint4 raw[U];
         bool ok[U];
 #pragma unroll

@@ -3,7 +3,7 @@
 // A CTA owns a row.  Pass A streams the row from HBM and keeps only per-thread running statistics in
 // registers -- (max offset, sum) rescaled online for softmax, (n, mean, M2) merged chunk by chunk with Chan's
 // update for LayerNorm, the sum of squares for RMSNorm -- so no cross-thread communication happens inside the
-// row; one CTA-wide merge follows.  Pass B streams the row again, this time from L2 (a row is at most a few
+// row; one CTA-wide merge follows.  Pass B streams the row again, back to front, this time from L2 (a row is at most a few
 // MiB and was just read; the loads of pass A carry an L2 evict-last policy, those of pass B an
 // evict-first one), normalises and writes y with streaming stores.  HBM still sees x once and y once.
 // There is no shared-memory staging, no cluster and no limit on the row length; many resident CTAs with
