@@ -268,7 +268,8 @@ def run_ours(args):
                         x_std=base.x_std, eps=base.eps, scale=base.scale, shift=base.shift)
     data = w.generate()
     case = DeviceCase(w, data, device)
-    tuned = tf.tf_tune(w.op, w.rows, w.cols, w.dt) if not args.no_tune else {"plan": tf.tf_query_choice(w.op, w.rows, w.cols, w.dt)}
+    like = (case.x[0], case.params.get("gamma", case.params.get("w")), case.params.get("beta"))
+    tuned = tf.tf_tune(w.op, w.rows, w.cols, w.dt, like=like) if not args.no_tune else {"plan": tf.tf_query_choice(w.op, w.rows, w.cols, w.dt)}
 
     steps, warmup = args.steps, max(args.warmup, 3)
     for _ in range(warmup):
@@ -390,7 +391,8 @@ def run_table(args):
         reps = max(20, min(400, int(0.05 / max(1e-6, case.bytes_per_step / 5e12))))
         tf.tf_clear_cache()
         ms_h = case.time_steps(reps, 5)
-        tuned = tf.tf_tune(w.op, w.rows, w.cols, w.dt) if not args.no_tune else {"plan": heur, "timed": 0}
+        like = (case.x[0], case.params.get("gamma", case.params.get("w")), case.params.get("beta"))
+        tuned = tf.tf_tune(w.op, w.rows, w.cols, w.dt, like=like) if not args.no_tune else {"plan": heur, "timed": 0}
         ms_t = case.time_steps(reps, 5)
         us = 1e3 * ms_t / reps
         gbs = case.bytes_per_step / (us * 1e-6) / 1e9
@@ -443,7 +445,7 @@ def run_case(args):
     if args.plan:
         tf.tf_force_plan(w.op, args.plan)
     elif not args.no_tune:
-        tf.tf_tune(w.op, w.rows, w.cols, w.dt)
+        tf.tf_tune(w.op, w.rows, w.cols, w.dt, like=(case.x[0], case.params.get("gamma", case.params.get("w")), case.params.get("beta")))
     ms = case.time_steps(args.steps, max(1, args.warmup))
     tf.tf_device_status()
     print(json.dumps({"case": w.name, "plan": args.plan or tf.tf_query_choice(w.op, w.rows, w.cols, w.dt), "launches": args.steps,

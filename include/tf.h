@@ -92,6 +92,13 @@ tf_status tf_softmax_fwd_noalloc(const void* x, void* y, int64_t rows, int64_t c
  * frees its own scratch; assumes 16-byte aligned tensors. */
 tf_status tf_tune(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);
 
+/* The same loop, timed on the caller's data instead of synthetic values: the contents of x (device, [rows, cols])
+ * and, if given, of the parameter vectors p0 (gamma / weight) and p1 (beta) are copied into the tuner's scratch
+ * tensors; the caller's tensors are only read.  Worth it when the data changes the cost, e.g. a masked softmax
+ * whose -inf tails cost no exponentials.  (The paper's loop likewise profiles on the kernel's own test inputs,
+ * Section 3.2.) */
+tf_status tf_tune_like(tf_op op, const void* x, const void* p0, const void* p1, int64_t rows, int64_t cols, tf_dtype dt);
+
 /* Result of the last tf_tune on this thread: number of candidates timed, median microseconds of the
  * heuristic plan and of the winner.  Any pointer may be NULL. */
 tf_status tf_tune_report(int* candidates_timed, float* heuristic_us, float* best_us);

@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_report", "tf_status_string",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
 
@@ -52,6 +52,7 @@ def lib() -> ctypes.CDLL:
         L.tf_layernorm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_rmsnorm_fwd.argtypes = [vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_tune.argtypes = [i32, i64, i64, i32]
+        L.tf_tune_like.argtypes = [i32, vp, vp, vp, i64, i64, i32]
         L.tf_tune_report.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(f32)]
         L.tf_status_string.argtypes = [i32]
         L.tf_status_string.restype = cp
@@ -65,7 +66,7 @@ def lib() -> ctypes.CDLL:
         L.tf_clear_cache.restype = None
         L.tf_launch_count.argtypes = []
         L.tf_launch_count.restype = i64
-        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_report",
+        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report",
                      "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice",
                      "tf_candidate_count", "tf_candidate"):
             getattr(L, name).restype = i32
@@ -180,11 +181,17 @@ def tf_rmsnorm_fwd(x, weight, eps: float, y=None, rstd=None, want_rstd: bool = F
     return y, rstd
 
 
-def tf_tune(op, rows: int, cols: int, dt: int) -> dict:
+def tf_tune(op, rows: int, cols: int, dt: int, like=None) -> dict:
     """Times the candidate plans for this problem on the current device, caches the winner, and returns
-    ``{"timed": n, "heuristic_us": a, "best_us": b, "plan": "..."}``."""
+    ``{"timed": n, "heuristic_us": a, "best_us": b, "plan": "..."}``.  ``like=(x, p0, p1)`` (CUDA tensors, p0/p1 may be
+    None) times on a copy of the caller's data instead of synthetic values."""
     code = OP_CODE[op] if isinstance(op, str) else int(op)
-    _ok(lib().tf_tune(code, rows, cols, dt), "tf_tune")
+    if like is None:
+        _ok(lib().tf_tune(code, rows, cols, dt), "tf_tune")
+    else:
+        x, p0, p1 = like
+        _ok(lib().tf_tune_like(code, x.data_ptr(), p0.data_ptr() if p0 is not None else None,
+                               p1.data_ptr() if p1 is not None else None, rows, cols, dt), "tf_tune_like")
     n, a, b = ctypes.c_int(), ctypes.c_float(), ctypes.c_float()
     lib().tf_tune_report(ctypes.byref(n), ctypes.byref(a), ctypes.byref(b))
     return {"timed": n.value, "heuristic_us": a.value, "best_us": b.value, "plan": tf_query_choice(code, rows, cols, dt)}

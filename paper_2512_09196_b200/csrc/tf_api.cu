@@ -503,8 +503,8 @@ tf_status tf_rmsnorm_fwd(const void* x, const void* weight, void* y, float* rstd
     return run(a, stream);
 }
 
-tf_status tf_tune(tf_op op_, int64_t rows, int64_t cols, tf_dtype dt_) {
-    const int op = op_, dt = dt_;
+// x_like / p0_like / p1_like: device tensors whose contents the timing input is copied from (NULL: synthetic).
+static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const void* x_like, const void* p0_like, const void* p1_like) {
     if (op < 0 || op >= OP_COUNT || bad_shape(rows, cols, dt) || rows == 0) return TF_ERR_INVALID_ARG;
     if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
     DevState* ds = nullptr;
@@ -538,12 +538,15 @@ tf_status tf_tune(tf_op op_, int64_t rows, int64_t cols, tf_dtype dt_) {
     const int64_t n = rows * cols;
     const int fill_grid = static_cast<int>(std::min<int64_t>((n + 255) / 256, static_cast<int64_t>(dev.sms) * 16));
     for (int k = 0; k < K; ++k) {
-        if (dt == DT_F32) k_fill<DT_F32><<<fill_grid, 256, 0, st>>>(xs[k], n, -4.f, 4.f, 1000003ull * k);
+        if (x_like) cudaMemcpyAsync(xs[k], x_like, tensor_bytes, cudaMemcpyDeviceToDevice, st);
+        else if (dt == DT_F32) k_fill<DT_F32><<<fill_grid, 256, 0, st>>>(xs[k], n, -4.f, 4.f, 1000003ull * k);
         else k_fill<DT_BF16><<<fill_grid, 256, 0, st>>>(xs[k], n, -4.f, 4.f, 1000003ull * k);
     }
     const int pgrid = static_cast<int>(std::min<int64_t>((cols + 255) / 256, 1024));
     if (dt == DT_F32) { k_fill<DT_F32><<<pgrid, 256, 0, st>>>(p0, cols, 0.5f, 1.5f, 7); k_fill<DT_F32><<<pgrid, 256, 0, st>>>(p1, cols, -0.5f, 0.5f, 11); }
     else { k_fill<DT_BF16><<<pgrid, 256, 0, st>>>(p0, cols, 0.5f, 1.5f, 7); k_fill<DT_BF16><<<pgrid, 256, 0, st>>>(p1, cols, -0.5f, 0.5f, 11); }
+    if (p0_like) cudaMemcpyAsync(p0, p0_like, static_cast<size_t>(cols) * es, cudaMemcpyDeviceToDevice, st);
+    if (p1_like) cudaMemcpyAsync(p1, p1_like, static_cast<size_t>(cols) * es, cudaMemcpyDeviceToDevice, st);
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess) { cleanup(); return cuda_fail(e); }
 
     auto args_for = [&](int k, void* y) {
@@ -617,6 +620,15 @@ tf_status tf_tune(tf_op op_, int64_t rows, int64_t cols, tf_dtype dt_) {
         save_cache_file_locked();
     }
     return TF_OK;
+}
+
+tf_status tf_tune(tf_op op, int64_t rows, int64_t cols, tf_dtype dt) {
+    return tune_impl(op, rows, cols, dt, nullptr, nullptr, nullptr);
+}
+
+tf_status tf_tune_like(tf_op op, const void* x, const void* p0, const void* p1, int64_t rows, int64_t cols, tf_dtype dt) {
+    if (!x) return TF_ERR_INVALID_ARG;
+    return tune_impl(op, rows, cols, dt, x, p0, p1);
 }
 
 tf_status tf_tune_report(int* candidates_timed, float* heuristic_us, float* best_us) {
