@@ -79,7 +79,7 @@ std::string plan_to_string(const Plan& p) {
         case V_TMA: snprintf(b, sizeof b, "tma:threads=%d,cluster=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.cluster, p.stages, p.chunk, p.persist); break;
         case V_PIPE: snprintf(b, sizeof b, "pipe:threads=%d,lanes=%d,vpt=%d,rpg=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.lanes, p.vpt, p.rpg, p.stages, p.chunk, p.persist); break;
         case V_RING: snprintf(b, sizeof b, "ring:threads=%d,vpt=%d,cluster=%d,stages=%d,persist=%d", p.threads, p.vpt, p.cluster, p.stages, p.persist); break;
-        case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,persist=%d", p.threads, p.persist); break;
+        case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,cache=%d,persist=%d", p.threads, p.chunk, p.persist); break;
         case V_SPLIT: snprintf(b, sizeof b, "split:threads=%d,splits=%d", p.threads, p.cluster); break;
         default: snprintf(b, sizeof b, "stream:threads=%d,lanes=%d,persist=%d", p.threads, p.lanes, p.persist); break;
     }
@@ -97,6 +97,7 @@ bool plan_from_string(const char* s, Plan& out) {
     if (v == V_STREAM) p.lanes = 0;
     if (v == V_PIPE) { p.persist = 1; p.stages = 4; p.chunk = 32768; }
     if (v == V_RING) { p.persist = 1; p.stages = 2; }
+    if (v == V_TWOPASS) p.chunk = 0;
     const char* q = colon ? colon + 1 : s + strlen(s);
     while (*q) {
         const char* eq = strchr(q, '=');
@@ -107,7 +108,7 @@ bool plan_from_string(const char* s, Plan& out) {
         if (end == eq + 1) return false;
         if (key == "threads") p.threads = val; else if (key == "lanes") p.lanes = val; else if (key == "vpt") p.vpt = val;
         else if (key == "rpg") p.rpg = val; else if (key == "cluster" || key == "splits") p.cluster = val; else if (key == "stages") p.stages = val;
-        else if (key == "chunk") p.chunk = val; else if (key == "persist") p.persist = val; else return false;
+        else if (key == "chunk" || key == "cache") p.chunk = val; else if (key == "persist") p.persist = val; else return false;
         q = (*end == ',') ? end + 1 : end;
         if (*end && *end != ',') return false;
     }
@@ -223,7 +224,7 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
     // everything beyond 128 KiB; persistent clusters with a prefetch ring in between
     if (a.op == OP_LAYERNORM || nvec > 8192) {
         Plan s;
-        s.variant = V_TWOPASS; s.threads = 512;
+        s.variant = V_TWOPASS; s.threads = 512; s.chunk = 49152;
         return s;
     }
     {
@@ -247,7 +248,7 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
     p.cluster = cl;
     if (!supports_tma(p, a, d)) {           // longer than a full cluster of shared memory can hold
         Plan s;
-        s.variant = V_TWOPASS; s.threads = 1024;
+        s.variant = V_TWOPASS; s.threads = 1024; s.chunk = 0;
         return s;
     }
     return p;
@@ -330,7 +331,13 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
     // two streamed passes (second from L2) for long rows
     if (nvec >= 1024)
         for (int th : {256, 512, 1024})
-            for (int persist : {0, 2048 / th}) { Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = persist; add(p); }
+            for (int persist : {0, 2048 / th})
+                for (int cache : {0, 1}) {
+                    // cache: what shared memory offers each of the 2048 / th CTAs of an SM, at most the row
+                    Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = persist;
+                    p.chunk = cache ? static_cast<int>(std::min<int64_t>(nvec * 16, (200 * 1024 / (2048 / th)) / 16 * 16)) : 0;
+                    add(p);
+                }
     // persistent cluster ring for long rows
     if (nvec >= 2048)
         for (int cl : {1, 2, 4, 8})

@@ -100,9 +100,12 @@ template <int OP, int DT> struct Running {
     }
 };
 
-// Pass A over `nvec` vectors starting at xs (all threads of the CTA take part).
+// Pass A over `nvec` vectors starting at xs (all threads of the CTA take part).  The first `cache_vecs` vectors
+// are also parked in shared memory (`cache`), each by the thread that will want it back in pass B -- the same
+// thread meets the same vectors in both passes, so no barrier is needed between them.
 template <int OP, int DT>
-__device__ __forceinline__ Running<OP, DT> stream_stats(const uint4* xs, int64_t nvec, uint64_t policy) {
+__device__ __forceinline__ Running<OP, DT> stream_stats(const uint4* xs, int64_t nvec, uint64_t policy, uint4* cache = nullptr,
+                                                        int64_t cache_vecs = 0) {
     constexpr int U = kStreamU;
     const int T = blockDim.x, t = threadIdx.x;
     const uint4 fill = fill_vec<DT>(OP);
@@ -114,6 +117,11 @@ __device__ __forceinline__ Running<OP, DT> stream_stats(const uint4* xs, int64_t
         for (int u = 0; u < U; ++u) {
             ok[u] = base + static_cast<int64_t>(u) * T < nvec;
             raw[u] = ok[u] ? ld_hint(xs + base + static_cast<int64_t>(u) * T, policy) : fill;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t idx = base + static_cast<int64_t>(u) * T;
+            if (idx < cache_vecs) cache[idx] = raw[u];          // cache_vecs <= nvec
         }
         run.update(raw, ok);
     }
@@ -154,7 +162,8 @@ __device__ __forceinline__ RowScale scale_of_row(const Part& p, float n, float e
 // Pass B over `nvec` vectors: xs/ys point at the segment, g/b at the parameters of its first column.
 template <int OP, int DT>
 __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const uint4* g, const uint4* b, int64_t nvec,
-                                             const RowScale& sc, uint64_t policy) {
+                                             const RowScale& sc, uint64_t policy, const uint4* cache = nullptr,
+                                             int64_t cache_vecs = 0) {
     using P = Pairs<DT>;
     constexpr int NP = P::NP, U = kStreamU;
     const int T = blockDim.x, t = threadIdx.x;
@@ -167,8 +176,9 @@ __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const u
         bool ok[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            ok[u] = base + static_cast<int64_t>(u) * T < nvec;
-            raw[u] = ok[u] ? ld_hint(xs + base + static_cast<int64_t>(u) * T, policy) : fill;
+            const int64_t idx = base + static_cast<int64_t>(u) * T;
+            ok[u] = idx < nvec;
+            raw[u] = !ok[u] ? fill : (idx < cache_vecs ? cache[idx] : ld_hint(xs + idx, policy));
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {

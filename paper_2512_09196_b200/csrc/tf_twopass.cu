@@ -5,7 +5,9 @@
 // update for LayerNorm, the sum of squares for RMSNorm -- so no cross-thread communication happens inside the
 // row; one CTA-wide merge follows.  Pass B streams the row again, back to front, this time from L2 (a row is at most a few
 // MiB and was just read; the loads of pass A carry an L2 evict-last policy, those of pass B an
-// evict-first one), normalises and writes y with streaming stores.  HBM still sees x once and y once.
+// evict-first one), normalises and writes y with streaming stores.  The head of the row -- the part pass A read
+// first and L2 is most likely to have dropped -- can be parked in shared memory instead (plan field `cache`).
+// HBM still sees x once and y once.
 // There is no shared-memory staging, no cluster and no limit on the row length; many resident CTAs with
 // several independent loads per thread keep the memory system busy.
 #include <algorithm>
@@ -24,26 +26,29 @@ struct WArgs {
     float* rstd;
     int64_t rows;
     int64_t nvec;
+    int64_t cache_vecs;   // vectors at the head of a row parked in shared memory between the passes
     float n, eps;
 };
 
 template <int OP, int DT>
 __global__ void __launch_bounds__(1024) k_twopass(const WArgs a) {
     __shared__ float red_buf[4 * 32];
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    uint4* const cache = reinterpret_cast<uint4*>(dyn_smem);
     pdl_wait();
     pdl_trigger();
     const uint64_t keep = policy_evict_last(), last = policy_evict_first();     // pass A keeps x in L2, pass B lets it go
     int it = 0;
     for (int64_t row = blockIdx.x; row < a.rows; row += gridDim.x, ++it) {
         const uint4* xr = a.x + row * a.nvec;
-        const Running<OP, DT> run = stream_stats<OP, DT>(xr, a.nvec, keep);
+        const Running<OP, DT> run = stream_stats<OP, DT>(xr, a.nvec, keep, cache, a.cache_vecs);
         const Part part = merge_running<OP, DT>(run, a.n, red_buf + 64 * (it & 1));
         const RowScale sc = scale_of_row<OP>(part, a.n, a.eps);
         if (threadIdx.x == 0) {
             if (OP == OP_LAYERNORM && a.mean) a.mean[row] = sc.a;
             if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = sc.b;
         }
-        stream_apply<OP, DT>(xr, a.y + row * a.nvec, a.p0, a.p1, a.nvec, sc, last);
+        stream_apply<OP, DT>(xr, a.y + row * a.nvec, a.p0, a.p1, a.nvec, sc, last, cache, a.cache_vecs);
     }
 }
 
@@ -63,8 +68,10 @@ TwoFn two_fn(int op, int dt) {
 
 }  // namespace
 
-bool supports_twopass(const Plan& p, const Args& a, const DeviceInfo&) {
-    return vector_ok(a) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0;
+// Plan field `chunk`: bytes of each row's head kept in shared memory between the passes (0 = none).
+bool supports_twopass(const Plan& p, const Args& a, const DeviceInfo& d) {
+    return vector_ok(a) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0 && p.chunk >= 0 && p.chunk % 16 == 0 &&
+           (d.smem_optin == 0 || p.chunk + 2048 <= d.smem_optin);
 }
 
 cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
@@ -78,7 +85,13 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
     k.y = static_cast<uint4*>(a.y); k.mean = a.mean; k.rstd = a.rstd; k.rows = a.rows;
     k.nvec = a.cols * elem_size(a.dt) / 16;
     k.n = static_cast<float>(a.cols); k.eps = a.eps;
+    k.cache_vecs = std::min<int64_t>(k.nvec, p.chunk / 16);
+    if (p.chunk > 0) {
+        cudaError_t e = ensure_max_smem(reinterpret_cast<const void*>(fn), d);
+        if (e != cudaSuccess) return e;
+    }
     cudaLaunchConfig_t cfg = {};
+    cfg.dynamicSmemBytes = static_cast<size_t>(k.cache_vecs) * 16;
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
     cfg.blockDim = dim3(p.threads);
     cfg.stream = st;
