@@ -87,7 +87,9 @@ tf_status tf_softmax_fwd_noalloc(const void* x, void* y, int64_t rows, int64_t c
  * candidate plan that can launch is run on library-owned scratch tensors, its output is checked against
  * the incumbent's, it is timed with CUDA events (3 warm-up + 5 timed launches, median; the paper's
  * Section 3.4 protocol) on rotating buffers larger than L2, and it replaces the incumbent only if it is
- * at least 2% faster.  The winner is cached in memory (and in the file named by the TF_TUNE_CACHE
+ * at least 2% faster.  After the fixed proposal list, one-parameter neighbours of the best plan are tried in
+ * rounds (the rule-based stand-in for Algorithm 1's refinement hint) until a round brings no improvement, at
+ * most 8 rounds (the paper's iteration cap).  The winner is cached in memory (and in the file named by the TF_TUNE_CACHE
  * environment variable, if set) and used by later *_fwd calls with the same key.  Blocking; allocates and
  * frees its own scratch; assumes 16-byte aligned tensors. */
 tf_status tf_tune(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);

@@ -370,6 +370,32 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
     return out;
 }
 
+// One-parameter variations of a plan (unsupported ones are filtered by the caller).
+std::vector<Plan> neighbours(const Plan& b) {
+    std::vector<Plan> out;
+    auto with = [&](auto edit) { Plan p = b; edit(p); out.push_back(p); };
+    for (int th : {b.threads / 2, b.threads - 64, b.threads - 32, b.threads + 32, b.threads + 64, b.threads * 2})
+        if (th >= 32 && th <= 1024 && th % 32 == 0 && th != b.threads) with([&](Plan& p) { p.threads = th; });
+    for (int pe : {b.persist - 1, b.persist + 1, b.persist * 2, 0})
+        if (pe >= 0 && pe <= 32 && pe != b.persist) with([&](Plan& p) { p.persist = pe; });
+    if (b.variant == V_PIPE || b.variant == V_RING || b.variant == V_TMA)
+        for (int st : {b.stages - 1, b.stages + 1})
+            if (st >= 1 && st <= 8) with([&](Plan& p) { p.stages = st; });
+    if (b.variant == V_PIPE || b.variant == V_TMA || b.variant == V_TWOPASS)
+        for (int ch : {b.chunk / 2 / 16 * 16, b.chunk * 3 / 4 / 16 * 16, b.chunk * 3 / 2 / 16 * 16, b.chunk * 2})
+            if (ch >= 0 && ch != b.chunk && ch <= 220 * 1024) with([&](Plan& p) { p.chunk = ch; });
+    if (b.variant == V_PIPE || b.variant == V_WARP)
+        for (int r : {1, 2, 4})
+            if (r != b.rpg) with([&](Plan& p) { p.rpg = r; });
+    if (b.variant == V_SPLIT)
+        for (int sp : {b.cluster / 2, b.cluster * 3 / 4, b.cluster * 3 / 2, b.cluster * 2})
+            if (sp >= 1 && sp != b.cluster) with([&](Plan& p) { p.cluster = sp; });
+    if (b.variant == V_CTA || b.variant == V_RING || b.variant == V_TMA)
+        for (int cl : {b.cluster / 2, b.cluster * 2})
+            if (cl >= 1 && cl <= kMaxCluster && cl != b.cluster) with([&](Plan& p) { p.cluster = cl; });
+    return out;
+}
+
 // ------------------------------------------------------------------------------------------------
 // tune cache
 // ------------------------------------------------------------------------------------------------
@@ -609,14 +635,29 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
     const char* log_env = getenv("TF_LOG");
     const bool log = log_env && *log_env && *log_env != '0';
     if (log) fprintf(stderr, "tf_tune: %8.2f us  %s (heuristic)\n", best_us, best0.c_str());
-    for (const Plan& c : candidates(probe, dev)) {
-        if (plan_to_string(c) == best0) continue;
+    std::vector<std::string> seen{best0};
+    // One proposal through BuildRun -> Profile -> Arbiter.  Returns true when the proposal was accepted.
+    auto consider = [&](const Plan& c) -> bool {
+        const std::string name = plan_to_string(c);
+        if (std::find(seen.begin(), seen.end(), name) != seen.end()) return false;
+        seen.push_back(name);
         float us = 0.f;
-        if (!runs_and_matches(c, false)) continue;          // failed BuildRun: dropped, never cached
-        if (!profile(c, &us)) continue;
+        if (!supports(c, probe, dev) || !runs_and_matches(c, false)) return false;   // failed BuildRun: dropped, never cached
+        if (!profile(c, &us)) return false;
         ++timed;
-        if (log) fprintf(stderr, "tf_tune: %8.2f us  %s\n", us, plan_to_string(c).c_str());
-        if (us < 0.98f * best_us) { best = c; best_us = us; }       // Arbiter: accept only a measured improvement
+        if (log) fprintf(stderr, "tf_tune: %8.2f us  %s\n", us, name.c_str());
+        if (us < 0.98f * best_us) { best = c; best_us = us; return true; }             // Arbiter: accept only a measured improvement
+        return false;
+    };
+    // Proposals: the fixed list of launch geometries around the row size.
+    for (const Plan& c : candidates(probe, dev)) consider(c);
+    // Targeted refinement (Algorithm 1's RefineHint, rule-based): one-parameter neighbours of the best plan so far,
+    // repeated while a round still brings a measured improvement, at most 8 rounds (the paper's iteration cap).
+    for (int round = 0; round < 8; ++round) {
+        bool improved = false;
+        for (const Plan& c : neighbours(best)) improved |= consider(c);
+        if (log) fprintf(stderr, "tf_tune: refinement round %d: %s\n", round + 1, improved ? "continue" : "finish");
+        if (!improved) break;                                                            // diminishing returns: finish
     }
     cleanup();
     t_tune_timed = timed; t_tune_heur_us = heur_us; t_tune_best_us = best_us;
