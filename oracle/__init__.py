@@ -10,6 +10,8 @@ patterns.  Every function returns freshly allocated outputs.
 from __future__ import annotations
 
 import ctypes
+import fcntl
+import hashlib
 import os
 import subprocess
 from pathlib import Path
@@ -25,14 +27,19 @@ _NP = {F32: np.float32, BF16: np.uint16}
 
 
 def build(force: bool = False) -> Path:
-    """Compile the oracle with g++ (no fast-math, no CUDA) unless an up-to-date build exists."""
-    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
-        tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
-        subprocess.run(
-            ["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-pthread", "-o", str(tmp), str(_SRC)],
-            check=True,
-        )
-        os.replace(tmp, _LIB)
+    """Compile the oracle with g++ (no fast-math, no CUDA) unless a build of the same source exists."""
+    stamp = _HERE / ".libtf_oracle.stamp"
+    digest = hashlib.sha256(_SRC.read_bytes()).hexdigest()
+    with open(_HERE / ".build.lock", "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        if force or not _LIB.exists() or not stamp.exists() or stamp.read_text().strip() != digest:
+            tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
+            subprocess.run(
+                ["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-pthread", "-o", str(tmp), str(_SRC)],
+                check=True,
+            )
+            os.replace(tmp, _LIB)
+            stamp.write_text(digest)
     return _LIB
 
 

@@ -1,6 +1,8 @@
 """Builds libtf.so (the C-ABI library) in-tree with nvcc for sm_100a."""
 from __future__ import annotations
 
+import fcntl
+import hashlib
 import os
 import subprocess
 import sys
@@ -22,46 +24,77 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found")
 
 
-def _stale(target: Path, deps) -> bool:
-    if not target.exists():
-        return True
-    t = target.stat().st_mtime
-    return any(Path(d).stat().st_mtime > t for d in deps)
+def _digest(paths, extra=()) -> str:
+    """Content hash of the inputs of a build step (file times do not survive a copy of the tree)."""
+    h = hashlib.sha256()
+    for x in extra:
+        h.update(str(x).encode())
+    for p in sorted(map(str, paths)):
+        h.update(p.rsplit("/", 1)[-1].encode())
+        h.update(Path(p).read_bytes())
+    return h.hexdigest()
+
+
+def _stale(target: Path, stamp: Path, digest: str) -> bool:
+    return not target.exists() or not stamp.exists() or stamp.read_text().strip() != digest
+
+
+class _Lock:
+    """One builder at a time (several ranks may import the package at once)."""
+
+    def __init__(self, path: Path):
+        self.path = path
+
+    def __enter__(self):
+        self.f = open(self.path, "w")
+        fcntl.flock(self.f, fcntl.LOCK_EX)
+
+    def __exit__(self, *exc):
+        fcntl.flock(self.f, fcntl.LOCK_UN)
+        self.f.close()
 
 
 def build(force: bool = False, verbose: bool = False) -> Path:
-    """Compile every .cu file to an object (in parallel) and link libtf.so.  Incremental by mtime."""
+    """Compile every .cu file to an object (in parallel) and link libtf.so.  A step is redone when the content of
+    its inputs (source, headers, flags) changed."""
     headers = list(CSRC.glob("*.h")) + list(CSRC.glob("*.cuh")) + list(INCLUDE.glob("*.h"))
     objdir = HERE / "build"
     objdir.mkdir(exist_ok=True)
-    nvcc = _nvcc()
-    jobs = []
-    for src in SOURCES:
-        obj = objdir / (src[:-3] + ".o")
-        if force or _stale(obj, [CSRC / src, *headers]):
-            jobs.append((src, obj))
+    with _Lock(objdir / ".lock"):
+        nvcc = _nvcc()
+        jobs = []
+        for src in SOURCES:
+            obj = objdir / (src[:-3] + ".o")
+            stamp = objdir / (src[:-3] + ".stamp")
+            digest = _digest([CSRC / src, *headers], NVCC_FLAGS)
+            if force or _stale(obj, stamp, digest):
+                jobs.append((src, obj, stamp, digest))
 
-    def compile_one(job):
-        src, obj = job
-        cmd = [nvcc, *NVCC_FLAGS, "-I", str(INCLUDE), "-c", str(CSRC / src), "-o", str(obj)]
+        def compile_one(job):
+            src, obj, stamp, digest = job
+            cmd = [nvcc, *NVCC_FLAGS, "-I", str(INCLUDE), "-c", str(CSRC / src), "-o", str(obj)]
+            if verbose:
+                cmd.insert(1, "-Xptxas=-v")
+            r = subprocess.run(cmd, capture_output=True, text=True)
+            if r.returncode:
+                raise RuntimeError(f"nvcc failed on {src}:\n{r.stdout}\n{r.stderr}")
+            stamp.write_text(digest)
+            return r.stderr
+
+        with ThreadPoolExecutor(max_workers=8) as ex:
+            logs = list(ex.map(compile_one, jobs))
         if verbose:
-            cmd.insert(1, "-Xptxas=-v")
-        r = subprocess.run(cmd, capture_output=True, text=True)
-        if r.returncode:
-            raise RuntimeError(f"nvcc failed on {src}:\n{r.stdout}\n{r.stderr}")
-        return r.stderr
-
-    with ThreadPoolExecutor(max_workers=8) as ex:
-        logs = list(ex.map(compile_one, jobs))
-    if verbose:
-        sys.stderr.write("\n".join(logs))
-    objs = [objdir / (s[:-3] + ".o") for s in SOURCES]
-    if force or jobs or _stale(LIB, objs):
-        tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
-        r = subprocess.run([nvcc, "-shared", "-o", str(tmp), *map(str, objs)], capture_output=True, text=True)
-        if r.returncode:
-            raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
-        os.replace(tmp, LIB)
+            sys.stderr.write("\n".join(logs))
+        objs = [objdir / (s[:-3] + ".o") for s in SOURCES]
+        link_digest = _digest(objs)
+        link_stamp = objdir / "libtf.stamp"
+        if force or jobs or _stale(LIB, link_stamp, link_digest):
+            tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
+            r = subprocess.run([nvcc, "-shared", "-o", str(tmp), *map(str, objs)], capture_output=True, text=True)
+            if r.returncode:
+                raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
+            os.replace(tmp, LIB)
+            link_stamp.write_text(link_digest)
     return LIB
 
 

@@ -10,6 +10,8 @@ bf16 tensors are ``uint16`` bit patterns; view them with ``torch.from_numpy(a).v
 from __future__ import annotations
 
 import ctypes
+import fcntl
+import hashlib
 import os
 import subprocess
 from dataclasses import dataclass, field
@@ -28,11 +30,17 @@ OPS = ("softmax", "layernorm", "rmsnorm")
 
 
 def build(force: bool = False) -> Path:
-    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
-        tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
-        subprocess.run(["gcc", "-std=c11", "-O2", "-fopenmp", "-fPIC", "-shared", "-o", str(tmp), str(_SRC), "-lm"],
-                       check=True)
-        os.replace(tmp, _LIB)
+    """Compile the generator with gcc + OpenMP unless a build of the same source exists."""
+    stamp = _HERE / ".libtf_inputs.stamp"
+    digest = hashlib.sha256(_SRC.read_bytes()).hexdigest()
+    with open(_HERE / ".build.lock", "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        if force or not _LIB.exists() or not stamp.exists() or stamp.read_text().strip() != digest:
+            tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
+            subprocess.run(["gcc", "-std=c11", "-O2", "-fopenmp", "-fPIC", "-shared", "-o", str(tmp), str(_SRC), "-lm"],
+                           check=True)
+            os.replace(tmp, _LIB)
+            stamp.write_text(digest)
     return _LIB
 
 
