@@ -43,36 +43,6 @@ struct PArgs {
 };
 
 constexpr int kPipeMaxBarriers = 128;                    // units x stages per CTA
-constexpr long long kPipeWaitBudget = 400000000LL;      // about 0.2 s
-
-__device__ __forceinline__ uint32_t sm_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void bar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sm_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void bar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool bar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(sm_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity, long long budget) {   // false: gave up
-    if (bar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!bar_try_wait(bar, parity))
-        if (clock64() - t0 > budget) return false;
-    return true;
-}
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(sm_u32(dst)), "l"(src), "r"(bytes), "r"(sm_u32(bar)) : "memory");
-}
-
 // Parameters staged in shared memory: gamma at [0, nvec), beta at [nvec, 2 nvec).
 struct SmemParams {
     const uint4* base;
@@ -111,17 +81,17 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     const int64_t GU = static_cast<int64_t>(gridDim.x) * units;
 
     if (ut == 0) {
-        for (int s = 0; s < S; ++s) bar_init(&bars[s], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int s = 0; s < S; ++s) mbar_init(&bars[s], 1);
+        mbar_fence_init();
     }
-    asm volatile("griddepcontrol.wait;" ::: "memory");   // everything below may read what the previous kernel wrote
+    pdl_wait();   // everything below may read what the previous kernel wrote
 
     auto issue = [&](int64_t tile, int s) {              // first thread of the unit only
         const int64_t row0 = tile * a.tile_rows;
         const int rows_here = static_cast<int>(min(static_cast<int64_t>(a.tile_rows), a.rows - row0));
         const uint32_t bytes = static_cast<uint32_t>(rows_here) * a.nvec * 16u;
-        bar_expect_tx(&bars[s], bytes);
-        bulk_load(ring + tile_vecs * s, a.x + row0 * a.nvec, bytes, &bars[s]);
+        mbar_expect_tx(&bars[s], bytes);
+        bulk_g2s(ring + tile_vecs * s, a.x + row0 * a.nvec, bytes, &bars[s]);
     };
     if (ut == 0)
         for (int s = 0; s < S; ++s) {
@@ -135,7 +105,7 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
         }
     }
     __syncthreads();                                      // barriers initialised, parameters staged
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    pdl_trigger();
 
     bool valid[VPL];
 #pragma unroll
@@ -158,10 +128,10 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     int i = 0, xpar = 0;
     for (int64_t tile = gu; tile < num_tiles; tile += GU, ++i) {
         const int s = i % S;
-        if (!failed && !bar_wait(&bars[s], static_cast<uint32_t>(i / S) & 1u, kPipeWaitBudget)) {
+        if (!failed && !mbar_wait(&bars[s], static_cast<uint32_t>(i / S) & 1u)) {
             failed = true;
             atomicExch(a.status, 4);
-            bar_wait(&bars[s], static_cast<uint32_t>(i / S) & 1u, kPipeWaitBudget);    // one more bounded wait for the copy
+            mbar_wait(&bars[s], static_cast<uint32_t>(i / S) & 1u);    // one more bounded wait for the copy
         }
         const int64_t row0 = tile * a.tile_rows;
         const int rows_here = static_cast<int>(min(static_cast<int64_t>(a.tile_rows), a.rows - row0));

@@ -45,44 +45,14 @@ struct RArgs {
 };
 
 constexpr int kRingMaxStages = 4;
-constexpr long long kRingWaitBudget = 400000000LL;      // about 0.2 s
-
-__device__ __forceinline__ uint32_t rs_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void rbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(rs_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void rbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(rs_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool rbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(rs_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool rbar_wait(uint64_t* bar, uint32_t parity) {
-    if (rbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!rbar_try_wait(bar, parity))
-        if (clock64() - t0 > kRingWaitBudget) return false;
-    return true;
-}
 // Remote 8-byte store into CTA `rank`'s copy of `slot`, counted on that CTA's copy of `bar`.
 __device__ __forceinline__ void push_partial(float* slot, uint64_t* bar, uint32_t rank, float a, float b) {
     uint32_t rslot, rbar;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rslot) : "r"(rs_u32(slot)), "r"(rank));
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(rs_u32(bar)), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rslot) : "r"(smem_u32(slot)), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(smem_u32(bar)), "r"(rank));
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
                  ::"r"(rslot), "f"(a), "f"(b), "r"(rbar) : "memory");
 }
-__device__ __forceinline__ void rbulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(rs_u32(dst)), "l"(src), "r"(bytes), "r"(rs_u32(bar)) : "memory");
-}
-
 constexpr int ring_max_threads(int vpt) { return vpt <= 4 ? 1024 : 512; }
 __device__ __forceinline__ bool valid_at(int idx, int len) { return idx < len; }
 
@@ -106,19 +76,19 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
     cg::cluster_group cl = cg::this_cluster();
 
     if (t == 0) {
-        for (int s = 0; s < S; ++s) rbar_init(&full_bar[s], 1);
-        rbar_init(&xch_bar[0], 1);
-        rbar_init(&xch_bar[1], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int s = 0; s < S; ++s) mbar_init(&full_bar[s], 1);
+        mbar_init(&xch_bar[0], 1);
+        mbar_init(&xch_bar[1], 1);
+        mbar_fence_init();
     }
-    asm volatile("griddepcontrol.wait;" ::: "memory");             // global reads below follow the previous kernel
+    pdl_wait();             // global reads below follow the previous kernel
     auto issue = [&](int64_t row, int s) {                           // thread 0 only; a slice may need several copies
         if (len == 0) return;
         const char* src = reinterpret_cast<const char*>(a.x + row * a.nvec + first);
         char* dst = reinterpret_cast<char*>(ring + static_cast<size_t>(s) * per);
         const uint32_t bytes = static_cast<uint32_t>(len) * 16u;
-        rbar_expect_tx(&full_bar[s], bytes);
-        for (uint32_t off = 0; off < bytes; off += 65536u) rbulk_load(dst + off, src + off, min(65536u, bytes - off), &full_bar[s]);
+        mbar_expect_tx(&full_bar[s], bytes);
+        for (uint32_t off = 0; off < bytes; off += 65536u) bulk_g2s(dst + off, src + off, min(65536u, bytes - off), &full_bar[s]);
     };
     if (t == 0)
         for (int s = 0; s < S; ++s) {
@@ -127,7 +97,7 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
         }
     __syncthreads();
     if (cs > 1) cl.sync();                 // every CTA of the cluster is resident (barriers initialised) before any remote store
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    pdl_trigger();
 
     bool valid[VPT];
 #pragma unroll
@@ -152,10 +122,10 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
     int it = 0;
     for (int64_t row = cluster_id; row < a.rows; row += num_clusters, ++it) {
         const int s = it % S;
-        if (len > 0 && !failed && !rbar_wait(&full_bar[s], static_cast<uint32_t>(it / S) & 1u)) {
+        if (len > 0 && !failed && !mbar_wait(&full_bar[s], static_cast<uint32_t>(it / S) & 1u)) {
             failed = true;
             atomicExch(a.status, 4);
-            rbar_wait(&full_bar[s], static_cast<uint32_t>(it / S) & 1u);      // one more bounded wait for the copy in flight
+            mbar_wait(&full_bar[s], static_cast<uint32_t>(it / S) & 1u);      // one more bounded wait for the copy in flight
         }
         const uint4* buf = ring + static_cast<size_t>(s) * per + t;
         uint4 raw[VPT], out[VPT];
@@ -170,9 +140,9 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
         // A peer can be at most one row ahead of this CTA (it needs this CTA's partial to finish a row), so two
         // slot buffers suffice; every CTA receives exactly cs pushes per row, all of them before it can leave the loop.
         if (cs > 1) {
-            if (t == 0) rbar_expect_tx(&xch_bar[xb], static_cast<uint32_t>(cs) * 8u);
+            if (t == 0) mbar_expect_tx(&xch_bar[xb], static_cast<uint32_t>(cs) * 8u);
             if (t < cs) push_partial(&xch[xb][rank][0], &xch_bar[xb], static_cast<uint32_t>(t), part.a, part.b);
-            if (!rbar_wait(&xch_bar[xb], static_cast<uint32_t>(it >> 1) & 1u) && !failed) { failed = true; atomicExch(a.status, 4); }
+            if (!mbar_wait(&xch_bar[xb], static_cast<uint32_t>(it >> 1) & 1u) && !failed) { failed = true; atomicExch(a.status, 4); }
         } else {
             if (t == 0) { xch[xb][0][0] = part.a; xch[xb][0][1] = part.b; }
             __syncthreads();
