@@ -408,11 +408,21 @@ def run_table(args):
         torch.cuda.synchronize()
         copy_us = 1e3 * ca.elapsed_time(cb) / reps
         copy_gbs = 2 * case.x[0].numel() * case.x[0].element_size() / (copy_us * 1e-6) / 1e9
+        # and the library's own streaming copy (same load/store style as the row kernels)
+        for k in range(min(5, case.sets)):
+            tf.tf_copy(case.x[k], case.y[k])
+        torch.cuda.synchronize()
+        ca.record()
+        for k in range(reps):
+            tf.tf_copy(case.x[k % case.sets], case.y[k % case.sets])
+        cb.record()
+        torch.cuda.synchronize()
+        tf_copy_gbs = 2 * case.x[0].numel() * case.x[0].element_size() / (ca.elapsed_time(cb) / reps * 1e-3) / 1e9
         row = {"workload": w.name, "op": w.op, "dtype": w.dtype_name, "rows": w.rows, "cols": w.cols,
                "bytes": case.bytes_per_step, "heuristic_plan": heur, "heuristic_us": 1e3 * ms_h / reps,
                "plan": tuned["plan"], "timed_candidates": tuned.get("timed"), "us": us, "gbs": gbs,
                "pct_of_8000": 100 * gbs / NOMINAL_HBM_GBS, f"pct_of_{peak_kind}_{peak:.0f}": 100 * gbs / peak,
-               "copy_us": copy_us, "copy_gbs": copy_gbs}
+               "copy_us": copy_us, "copy_gbs": copy_gbs, "tf_copy_gbs": tf_copy_gbs}
         if args.cpu:
             cb = cpu_baseline(w, data, budget_s=6.0)
             row["oracle_gbs"], row["oracle_sample"] = cb["value"], cb["sample"]

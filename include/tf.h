@@ -105,6 +105,21 @@ tf_status tf_tune_like(tf_op op, const void* x, const void* p0, const void* p1, 
  * heuristic plan and of the winner.  Any pointer may be NULL. */
 tf_status tf_tune_report(int* candidates_timed, float* heuristic_us, float* best_us);
 
+/* ---- calibration kernels --------------------------------------------------------------------------- */
+
+/* Device copy of `bytes` bytes written in the same load/store style as the row kernels (16-byte streaming
+ * accesses, four in flight per thread, one contiguous block per CTA, programmatic launch): the practical ceiling for "bytes in, bytes out" on
+ * this GPU at a given size, which the bench prints beside every result.  x and y must not overlap.  Any
+ * alignment (the vector path needs both 16-byte aligned). */
+tf_status tf_copy(const void* x, void* y, int64_t bytes, void* cuda_stream);
+
+/* y[i] = sin(x[i]) over n elements: the element-wise kernel of the paper's Case Study 1, whose only tuning knob is
+ * its launch geometry (the paper's baseline used blocks of 4 elements; the fix was an autotune over block sizes).
+ * threads per CTA (multiple of 32, <= 1024) and 16-byte vectors per thread (1, 2, 4 or 8) are that knob here -- a
+ * CTA covers threads x vectors_per_thread vectors, its "block size"; 0 selects the defaults (256, 4).
+ * fp32 arithmetic with full range reduction, one rounding to the storage type.  y == x is allowed. */
+tf_status tf_sin_fwd(const void* x, void* y, int64_t n, tf_dtype dt, int threads, int vectors_per_thread, void* cuda_stream);
+
 const char* tf_status_string(tf_status s);
 
 /* cudaError_t value behind the most recent TF_ERR_CUDA on the calling thread (0 if none). */

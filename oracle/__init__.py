@@ -57,6 +57,8 @@ def _load():
         lib.oracle_layernorm.restype = i32
         lib.oracle_rmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, i32]
         lib.oracle_rmsnorm.restype = i32
+        lib.oracle_sin.argtypes = [vp, vp, vp, i64, i32]
+        lib.oracle_sin.restype = i32
         lib.oracle_bf16_from_double.argtypes = [vp, vp, i64]
         lib.oracle_bf16_from_double.restype = None
         lib.oracle_bf16_to_double.argtypes = [vp, vp, i64]
@@ -119,6 +121,16 @@ def rmsnorm(x, w, eps: float, dt: int, want64: bool = False, nthreads: int = 1):
     if rc:
         raise ValueError("oracle_rmsnorm: bad argument")
     return (y, rstd, y64, st) if want64 else (y, rstd)
+
+
+def sin(x: np.ndarray, dt: int, want64: bool = False):
+    """Element-wise sine of any-shape array.  Returns ``y`` (and the unrounded float64 result if ``want64``)."""
+    _check(x, dt, "x")
+    y = np.empty_like(x)
+    y64 = np.empty(x.shape, np.float64) if want64 else None
+    if _load().oracle_sin(_p(x), _p(y), _p(y64), x.size, dt):
+        raise ValueError("oracle_sin: bad argument")
+    return (y, y64) if want64 else y
 
 
 def bf16_from_double(v: np.ndarray) -> np.ndarray:

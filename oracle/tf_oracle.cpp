@@ -19,7 +19,10 @@
 // Pins (tests that hold this file to something other than itself): closed forms and hand rows,
 // row-sum / shift / scale invariants, the eps closed forms for variance and RMS, brute force in
 // long double on tiny rows, agreement with torch-CPU float64 library routines before rounding, and
-// for the bf16 codec an exhaustive walk over all 65,536 patterns and every midpoint.  tf_tune has
+// for the bf16 codec an exhaustive walk over all 65,536 patterns and every midpoint.  The element-wise
+// sine (the kernel of the paper's Case Study 1, used as a calibration workload) is std::sin in double;
+// it is pinned by sin(+-0), oddness, the double-angle identity, the small-angle series and libm
+// through another route.  tf_tune has
 // no oracle function here: which candidate wins is hardware-dependent ("parity unpinned" for the
 // winner's identity; its output is checked like any other launch).
 
@@ -210,6 +213,17 @@ int oracle_rmsnorm(const void* x, const void* w, void* y, double* y64, float* rs
     if (bad(rows, cols, dt) || !x || !w) return -1;
     const double e = static_cast<double>(eps);
     for_rows(rows, nthreads, [=](int64_t r) { rmsnorm_row(x, w, y, y64, rstd, stats64, cols, e, dt, r); });
+    return 0;
+}
+
+// Element-wise sine (the kernel of the paper's Case Study 1): y_i = sin(x_i) in double, rounded once.
+int oracle_sin(const void* x, void* y, double* y64, int64_t n, int dt) {
+    if (n < 0 || (dt != F32 && dt != BF16) || !x) return -1;
+    for (int64_t i = 0; i < n; ++i) {
+        const double v = std::sin(load(x, i, dt));
+        if (y64) y64[i] = v;
+        if (y) store(y, i, dt, v);
+    }
     return 0;
 }
 

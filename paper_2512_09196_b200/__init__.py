@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_status_string",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
 
@@ -52,6 +52,8 @@ def lib() -> ctypes.CDLL:
         L.tf_layernorm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_rmsnorm_fwd.argtypes = [vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_tune.argtypes = [i32, i64, i64, i32]
+        L.tf_copy.argtypes = [vp, vp, i64, vp]
+        L.tf_sin_fwd.argtypes = [vp, vp, i64, i32, i32, i32, vp]
         L.tf_tune_like.argtypes = [i32, vp, vp, vp, i64, i64, i32]
         L.tf_tune_report.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(f32)]
         L.tf_status_string.argtypes = [i32]
@@ -66,7 +68,7 @@ def lib() -> ctypes.CDLL:
         L.tf_clear_cache.restype = None
         L.tf_launch_count.argtypes = []
         L.tf_launch_count.restype = i64
-        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report",
+        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd",
                      "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice",
                      "tf_candidate_count", "tf_candidate"):
             getattr(L, name).restype = i32
@@ -142,6 +144,31 @@ def tf_softmax_fwd_noalloc(x, y):
     rows, cols = x.shape
     with _on_device(x):
         _ok(lib().tf_softmax_fwd_noalloc(x.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)), "tf_softmax_fwd_noalloc")
+    return y
+
+
+def tf_copy(x, y=None):
+    """Calibration copy of a contiguous CUDA tensor with the library's own streaming kernel."""
+    import torch
+    if not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x must be a contiguous CUDA tensor")
+    if y is None:
+        y = torch.empty_like(x)
+    with _on_device(x):
+        _ok(lib().tf_copy(x.data_ptr(), y.data_ptr(), x.numel() * x.element_size(), _stream(x)), "tf_copy")
+    return y
+
+
+def tf_sin_fwd(x, y=None, threads: int = 0, vectors_per_thread: int = 0):
+    """Element-wise sine of a contiguous CUDA tensor (fp32 or bf16); ``threads`` and ``vectors_per_thread`` (1, 2, 4, 8)
+    are the launch geometry (0 = defaults)."""
+    import torch
+    if not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x must be a contiguous CUDA tensor")
+    if y is None:
+        y = torch.empty_like(x)
+    with _on_device(x):
+        _ok(lib().tf_sin_fwd(x.data_ptr(), y.data_ptr(), x.numel(), _dt(x), threads, vectors_per_thread, _stream(x)), "tf_sin_fwd")
     return y
 
 

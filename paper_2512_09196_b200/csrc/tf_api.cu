@@ -307,12 +307,13 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
                 if (th < ut || (rpg == 2 && (c[1] > 4 || nvec != cap))) continue;
                 const int64_t pass_bytes = row_bytes * (ut / c[0]) * rpg;
                 const int units = th / ut;
-                for (int persist : {1, 2, 4})
+                for (int persist : {1, 2, 4, 0, -2})          // 0 / -2: non-persistent grids with rings sized for 3 / 2 CTAs per SM
                     for (int stages : {2, 3, 4}) {
-                        const int64_t budget = (persist == 1 ? 200 : (persist == 2 ? 98 : 48)) * 1024 - param_bytes;
+                        if (persist <= 0 && stages == 4) continue;
+                        const int64_t budget = (persist == 1 ? 200 : (persist == 2 ? 98 : (persist == 4 ? 48 : (persist == 0 ? 64 : 98)))) * 1024 - param_bytes;
                         int64_t chunk = std::min<int64_t>(32768, budget / units / stages) / pass_bytes * pass_bytes;
                         if (chunk < pass_bytes) continue;
-                        Plan p; p.variant = V_PIPE; p.lanes = c[0]; p.vpt = c[1]; p.rpg = rpg; p.threads = th; p.persist = persist;
+                        Plan p; p.variant = V_PIPE; p.lanes = c[0]; p.vpt = c[1]; p.rpg = rpg; p.threads = th; p.persist = std::max(0, persist);
                         p.chunk = static_cast<int>(chunk); p.stages = stages;
                         add(p);
                         if (chunk >= 4 * pass_bytes && chunk > 4096) { p.chunk = static_cast<int>(chunk / 2 / pass_bytes * pass_bytes); add(p); }

@@ -39,7 +39,7 @@ bool pipe_geometry(const Plan& p, const Args& a, const DeviceInfo& d, PipeGeomet
     g.smem = static_cast<size_t>(units) * p.stages * rows * row_bytes + param_bytes;
     if (rows * row_bytes >= (1 << 20)) return false;          // mbarrier transaction-count limit
     const size_t static_smem = 8 * kPipeMaxBarriers + 1024 + 1024;
-    return g.smem + static_smem <= static_cast<size_t>(d.smem_optin) / std::max(1, p.persist);
+    return g.smem + static_smem <= static_cast<size_t>(d.smem_optin) / std::max(1, p.persist);      // persist = 0: any ring that fits
 }
 
 }  // namespace
@@ -49,7 +49,7 @@ bool supports_pipe(const Plan& p, const Args& a, const DeviceInfo& d) {
     const int ut = p.lanes < 32 ? 32 : p.lanes;
     if (p.threads % ut || p.rpg < 1 || !pipe_fn(a.op, a.dt, p.lanes, p.vpt, p.rpg, row_fills(p, a))) return false;
     const int units = p.threads / ut;
-    if (p.stages < 1 || units * p.stages > kPipeMaxBarriers || p.persist < 1 || p.persist > 8 || p.chunk < 16) return false;
+    if (p.stages < 1 || units * p.stages > kPipeMaxBarriers || p.persist < 0 || p.persist > 8 || p.chunk < 16) return false;
     if (ut > 32 && units > 15) return false;                  // one named barrier per multi-warp unit
     const int64_t nvec = a.cols * elem_size(a.dt) / 16;
     if (nvec > static_cast<int64_t>(p.lanes) * p.vpt) return false;
@@ -66,7 +66,11 @@ cudaError_t launch_pipe(const Plan& p, const Args& a, const DeviceInfo& d, cudaS
     const int ut = p.lanes < 32 ? 32 : p.lanes;
     const int units = p.threads / ut;
     const int64_t tiles = (a.rows + g.tile_rows - 1) / g.tile_rows;
-    const int64_t grid = std::min<int64_t>((tiles + units - 1) / units, static_cast<int64_t>(p.persist) * d.sms);
+    // persist = k: k CTAs per SM walk all tiles.  persist = 0: as many CTAs as it takes for every unit to get at most
+    // `stages` tiles, all requested in its prologue -- no refill, the hardware replaces finished CTAs.
+    int64_t grid = (tiles + units - 1) / units;
+    if (p.persist > 0) grid = std::min<int64_t>(grid, static_cast<int64_t>(p.persist) * d.sms);
+    else grid = std::min<int64_t>((grid + p.stages - 1) / p.stages, 0x7FFFFFFF);
     PArgs k;
     k.x = static_cast<const uint4*>(a.x); k.p0 = static_cast<const uint4*>(a.p0); k.p1 = static_cast<const uint4*>(a.p1);
     k.y = static_cast<uint4*>(a.y); k.mean = a.mean; k.rstd = a.rstd; k.rows = a.rows;

@@ -193,6 +193,29 @@ def test_rmsnorm_closed_form_and_scale_equivariance():
     np.testing.assert_array_equal(s[0], [1.0, 1.0, 1.0])
 
 
+# ------------------------------------------------------------------ element-wise sine (calibration kernel)
+
+def test_sin_closed_forms_symmetry_and_library():
+    x = f32([0.0, -0.0, 0.5, 1.0, 2.0, 3.0, 10.0, 100.0, 1e6, -7.25])
+    y, y64 = oracle.sin(x, F32, want64=True)
+    assert y[0] == 0.0 and not np.signbit(y[0]) and np.signbit(y[1])             # sin(+-0) = +-0
+    # closed forms at exactly representable arguments of the half-angle chain: sin(2a) = 2 sin a cos a, sin^2 + cos^2 = 1
+    a = x.astype(np.float64)
+    s_half, c_half = np.sin(a / 2), np.cos(a / 2)
+    np.testing.assert_allclose(y64, 2 * s_half * c_half, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(y64, [math.sin(float(v)) for v in x], rtol=1e-15)       # libm through Python, value by value
+    _, neg = oracle.sin(f32(-a), F32, want64=True)
+    np.testing.assert_array_equal(neg, -y64)                                        # odd
+    assert (np.abs(y64) <= 1).all()
+    # small-angle series: sin x = x - x^3/6 + x^5/120 - ... for |x| <= 2^-10 agrees to 1e-16 relative
+    small = f32([2.0 ** -10, 2.0 ** -15, -2.0 ** -20])
+    _, ys = oracle.sin(small, F32, want64=True)
+    sd = small.astype(np.float64)
+    np.testing.assert_allclose(ys, sd - sd ** 3 / 6 + sd ** 5 / 120, rtol=1e-15)
+    yb, yb64 = oracle.sin(bf([0.5, 1.5]), BF16, want64=True)
+    np.testing.assert_array_equal(yb, oracle.bf16_from_double(yb64))
+
+
 # ------------------------------------------------------------------ brute force on tiny rows (long double)
 
 def test_bruteforce_longdouble_tiny_rows():
