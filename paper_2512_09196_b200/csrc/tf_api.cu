@@ -295,16 +295,20 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
     // persistent self-feeding pipeline: (lanes, vpt) that hold the row; rings that fit one or two CTAs per SM
     {
         const int combos[][2] = {{8, 1}, {16, 1}, {32, 1}, {32, 2}, {32, 4}, {32, 8}, {64, 2}, {64, 4}, {64, 8}, {128, 2},
-                                 {128, 4}, {128, 8}, {256, 2}, {256, 4}, {256, 8}, {512, 4}, {512, 8}};
+                                 {128, 4}, {128, 8}, {256, 2}, {256, 4}, {256, 8}, {512, 4}, {512, 8},
+                                 {160, 4}, {160, 8}, {320, 4}, {192, 8}, {384, 4}, {384, 8}};
         const int64_t row_bytes = nvec * 16;
         const int64_t param_bytes = a.op == OP_SOFTMAX ? 0 : row_bytes * (a.op == OP_LAYERNORM ? 2 : 1);
         for (const auto& c : combos) {
             const int64_t cap = static_cast<int64_t>(c[0]) * c[1];
             if (nvec > cap || (nvec * 2 <= cap && c[0] != 8)) continue;
             const int ut = c[0] < 32 ? 32 : c[0];
+            const bool odd = (ut & (ut - 1)) != 0;                 // 160, 192, 320, 384: only worth it when the row fills them
+            if (odd && nvec != cap) continue;
             for (int rpg : {1, 2})
-            for (int th : {256, 512}) {
-                if (th < ut || (rpg == 2 && (c[1] > 4 || nvec != cap))) continue;
+            for (int th0 : {256, 512}) {
+                const int th = th0 / ut * ut;                       // CTA = whole units
+                if (th < ut || (odd && th0 == 256 && 512 / ut * ut == th) || (rpg == 2 && (c[1] > 4 || nvec != cap))) continue;
                 const int64_t pass_bytes = row_bytes * (ut / c[0]) * rpg;
                 const int units = th / ut;
                 for (int persist : {1, 2, 4, 0, -2})          // 0 / -2: non-persistent grids with rings sized for 3 / 2 CTAs per SM

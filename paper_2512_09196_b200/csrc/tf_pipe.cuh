@@ -205,6 +205,8 @@ template <int OP, int DT> PipeFn pick_pipe(int lanes, int vpl, int rpg, bool ful
     TF_P(8, 1) TF_P(16, 1) TF_P(32, 1) TF_P(32, 2) TF_P(32, 4) TF_P(32, 8)
     TF_P(64, 2) TF_P(64, 4) TF_P(64, 8) TF_P(128, 2) TF_P(128, 4) TF_P(128, 8) TF_P(256, 2) TF_P(256, 4) TF_P(256, 8)
     TF_P(512, 4) TF_P(512, 8)
+    // rows of 5120 and 12288 elements (640 / 1280 / 1536 / 3072 vectors) fill these exactly
+    TF_P(160, 4) TF_P(160, 8) TF_P(320, 4) TF_P(192, 8) TF_P(384, 4) TF_P(384, 8)
 #undef TF_P
     return nullptr;
 }

@@ -198,7 +198,7 @@ def test_forced_tma_variants(op, dt, cluster):
 
 
 PIPE_COMBOS = [(8, 1), (16, 1), (32, 1), (32, 2), (32, 4), (32, 8), (64, 2), (64, 4), (64, 8), (128, 2), (128, 4), (128, 8),
-               (256, 2), (256, 4), (256, 8), (512, 4), (512, 8)]
+               (256, 2), (256, 4), (256, 8), (512, 4), (512, 8), (160, 4), (160, 8), (320, 4), (192, 8), (384, 4), (384, 8)]
 
 
 @pytest.mark.parametrize("op", OPS)
@@ -209,7 +209,7 @@ def test_forced_pipe_variants(op, dt):
     for ci, (lanes, vpt) in enumerate(PIPE_COMBOS):
         cap = lanes * vpt
         ut = max(32, lanes)
-        threads = 512 if ci % 2 else max(256, ut)
+        threads = (512 if ci % 2 else max(256, ut)) // ut * ut
         # rows chosen so that a unit wraps its ring several times and the last tile is ragged
         for nvec, stages, chunk, persist, rows in ((cap, 2, 4096, 1, 4001), (max(1, cap - 1), 3, 16384, 2, 2999),
                                                    (max(1, cap // 2 + 1), 1, 2048, 1, 1777), (cap, 4, 512, 8, 77)):
