@@ -59,6 +59,8 @@ def _load():
         lib.oracle_rmsnorm.restype = i32
         lib.oracle_sin.argtypes = [vp, vp, vp, i64, i32]
         lib.oracle_sin.restype = i32
+        lib.oracle_bvecmat.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i32, i32]
+        lib.oracle_bvecmat.restype = i32
         lib.oracle_bf16_from_double.argtypes = [vp, vp, i64]
         lib.oracle_bf16_from_double.restype = None
         lib.oracle_bf16_to_double.argtypes = [vp, vp, i64]
@@ -131,6 +133,22 @@ def sin(x: np.ndarray, dt: int, want64: bool = False):
     if _load().oracle_sin(_p(x), _p(y), _p(y64), x.size, dt):
         raise ValueError("oracle_sin: bad argument")
     return (y, y64) if want64 else y
+
+
+def bvecmat(a: np.ndarray, b: np.ndarray, dt: int, want64: bool = False, nthreads: int = 1):
+    """C[m,n] = sum_k a[m,k] * b[m,n,k].  Returns ``c`` plus ``(c64, scale64)`` if ``want64``, where
+    ``scale64[m,n] = sum_k |a[m,k] * b[m,n,k]|``."""
+    _check(a, dt, "a"), _check(b, dt, "b")
+    if a.ndim != 2 or b.ndim != 3 or b.shape[0] != a.shape[0] or b.shape[2] != a.shape[1]:
+        raise ValueError("want a [M, K] and b [M, N, K]")
+    M, K = a.shape
+    N = b.shape[1]
+    c = np.empty((M, N), _NP[dt])
+    c64 = np.empty((M, N), np.float64) if want64 else None
+    sc = np.empty((M, N), np.float64) if want64 else None
+    if _load().oracle_bvecmat(_p(a), _p(b), _p(c), _p(c64), _p(sc), M, N, K, dt, nthreads):
+        raise ValueError("oracle_bvecmat: bad argument")
+    return (c, c64, sc) if want64 else c
 
 
 def bf16_from_double(v: np.ndarray) -> np.ndarray:

@@ -22,7 +22,10 @@
 // for the bf16 codec an exhaustive walk over all 65,536 patterns and every midpoint.  The element-wise
 // sine (the kernel of the paper's Case Study 1, used as a calibration workload) is std::sin in double;
 // it is pinned by sin(+-0), oddness, the double-angle identity, the small-angle series and libm
-// through another route.  tf_tune has
+// through another route.  The batched vector-matrix product (the paper's Case Study 2) is the plain
+// triple loop in double; it is pinned by all-ones and ramp closed forms, unit-vector selection, an
+// index-order trap (B[m,n,k] versus B[m,k,n] and A[m,k] versus A[n,k]), exact integer brute force,
+// linearity, and numpy's float64 einsum.  tf_tune has
 // no oracle function here: which candidate wins is hardware-dependent ("parity unpinned" for the
 // winner's identity; its output is checked like any other launch).
 
@@ -224,6 +227,28 @@ int oracle_sin(const void* x, void* y, double* y64, int64_t n, int dt) {
         if (y64) y64[i] = v;
         if (y) store(y, i, dt, v);
     }
+    return 0;
+}
+
+// Batched vector-matrix product (the paper's Case Study 2):  C[m,n] = sum_k A[m,k] * B[m,n,k],
+// A [M,K], B [M,N,K] (k fastest), C [M,N].  Inputs widened exactly, products and the running sum in
+// double in increasing k, one rounding to the output type.  scale64 (nullable) receives
+// sum_k |A[m,k] * B[m,n,k]|, the quantity any summation-order error bound is stated against.
+int oracle_bvecmat(const void* A, const void* B, void* C, double* c64, double* scale64, int64_t M, int64_t N,
+                   int64_t K, int dt, int nthreads) {
+    if (M < 0 || N < 0 || K <= 0 || (dt != F32 && dt != BF16) || ((M > 0 && N > 0) && (!A || !B))) return -1;
+    for_rows(M * N, nthreads, [=](int64_t r) {
+        const int64_t m = r / N;
+        double s = 0.0, t = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            const double p = load(A, m * K + k, dt) * load(B, r * K + k, dt);
+            s += p;
+            t += std::fabs(p);
+        }
+        if (c64) c64[r] = s;
+        if (scale64) scale64[r] = t;
+        if (C) store(C, r, dt, s);
+    });
     return 0;
 }
 
