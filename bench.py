@@ -433,6 +433,78 @@ def run_table(args):
     (out_dir / f"table_{args.table}.json").write_text(json.dumps(rows_out, indent=1))
 
 
+def run_vecmat_table(args):
+    """Batched vector-matrix product (the paper's second case study) over the K sweep: automatic geometry, every forced
+    geometry, and torch's library routine for the same contraction as context.  B is far larger than L2."""
+    import torch
+    import paper_2512_09196_b200 as tf
+    from paper_2512_09196_b200 import inputs
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak()
+    points = inputs.vecmat_sweep()
+    if args.filter:
+        points = [p for p in points if args.filter in p.name]
+    out_dir = ROOT / "gpurun_out"
+    out_dir.mkdir(exist_ok=True)
+
+    def timed(fn, reps):
+        for _ in range(5):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return 1e3 * a.elapsed_time(b) / reps
+
+    rows_out = []
+    for w in points:
+        data = w.generate()
+        conv = (lambda t: t.view(torch.bfloat16)) if w.dt == inputs.BF16 else (lambda t: t)
+        A, B = conv(torch.from_numpy(data["a"])).cuda(), conv(torch.from_numpy(data["b"])).cuda()
+        C = torch.empty((w.M, w.N), dtype=A.dtype, device="cuda")
+        nbytes = w.algorithmic_bytes()
+        reps = max(20, min(200, int(0.05 / (nbytes / 5e12))))
+        us_auto = timed(lambda: tf.tf_bvecmat_fwd(A, B, C), reps)
+        grid, kvec = {}, w.K * w.elem_size // 16
+        if not args.no_tune:
+            for threads in (128, 256, 512, 1024):
+                for lanes in (4, 8, 16, 32):
+                    if w.dt == inputs.F32 and lanes <= kvec and (lanes == 32 or kvec <= 16 * lanes):
+                        for rows in (1, 2, 4):
+                            grid[f"{threads},{lanes},{rows},0"] = timed(lambda: tf.tf_bvecmat_fwd(A, B, C, threads, lanes, rows), reps)
+                if w.dt == inputs.BF16 and threads < 1024:
+                    for rows in (16, 32):
+                        for ks in (1, 2, 4, 8):
+                            if ks * 32 <= threads:
+                                grid[f"{threads},0,{rows},{ks}"] = timed(lambda: tf.tf_bvecmat_fwd(A, B, C, threads, 0, rows, ks), reps)
+        best = min(grid, key=grid.get) if grid else None
+        us_lib = timed(lambda: torch.bmm(B, A.unsqueeze(-1)), max(5, reps // 4))
+        tf.tf_device_status()
+        row = {"workload": w.name, "dtype": w.dtype_name, "M": w.M, "N": w.N, "K": w.K, "bytes": nbytes, "us": us_auto,
+               "gbs": nbytes / us_auto / 1e3, f"pct_of_{peak_kind}_{peak:.0f}": 100 * nbytes / us_auto / 1e3 / peak,
+               "best_geometry": best, "best_us": grid.get(best), "best_gbs": nbytes / grid[best] / 1e3 if best else None,
+               "torch_bmm_us": us_lib, "torch_bmm_gbs": nbytes / us_lib / 1e3,
+               "grid_us": {k: round(v, 2) for k, v in sorted(grid.items(), key=lambda kv: kv[1])[:8]}}
+        if args.cpu:
+            import numpy as np
+            import oracle
+            sub = max(1, min(w.N, int(2e8 / (w.M * w.K))))
+            sub_b = np.ascontiguousarray(data["b"][:, :sub])
+            t0 = time.perf_counter()
+            oracle.bvecmat(data["a"], sub_b, w.dt, nthreads=os.cpu_count() or 1)
+            dt_s = time.perf_counter() - t0
+            row["oracle_gbs"] = (w.M * w.K + w.M * sub * w.K + w.M * sub) * w.elem_size / dt_s / 1e9
+            row["oracle_sample"] = f"first {sub} of {w.N} columns n of every batch entry"
+        rows_out.append(row)
+        print(json.dumps(row), flush=True)
+        del A, B, C
+        torch.cuda.empty_cache()
+    (out_dir / "table_vecmat.json").write_text(json.dumps(rows_out, indent=1))
+
+
 def run_case(args):
     """A few launches of one op/shape (for profiler captures): --case op:dtype:rows:cols or --case config:<i>[:rows]."""
     import torch
@@ -440,6 +512,28 @@ def run_case(args):
     from paper_2512_09196_b200 import inputs
     torch.cuda.set_device(0)
     parts = args.case.split(":")
+    if parts[0] == "vecmat":                  # vecmat:dtype:M:N:K[:threads:lanes:rows:ksplit]
+        dt = inputs.F32 if parts[1] == "f32" else inputs.BF16
+        M, N, K = (int(v) for v in parts[2:5])
+        knobs = [int(v) for v in parts[5:9]] + [0] * (4 - len(parts[5:9]))
+        w = inputs.VecMat(f"case_bvecmat_{parts[1]}_{M}x{N}x{K}", dt, M, N, K, seed=K)
+        data = w.generate()
+        conv = (lambda t: t.view(torch.bfloat16)) if dt == inputs.BF16 else (lambda t: t)
+        A, B = conv(torch.from_numpy(data["a"])).cuda(), conv(torch.from_numpy(data["b"])).cuda()
+        C = torch.empty((M, N), dtype=A.dtype, device="cuda")
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(max(1, args.warmup)):
+            tf.tf_bvecmat_fwd(A, B, C, *knobs)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(args.steps):
+            tf.tf_bvecmat_fwd(A, B, C, *knobs)
+        b.record()
+        torch.cuda.synchronize()
+        us = 1e3 * a.elapsed_time(b) / args.steps
+        print(json.dumps({"case": w.name, "knobs": knobs, "launches": args.steps, "us_per_launch": us,
+                          "gbs": w.algorithmic_bytes() / us / 1e3}))
+        return
     if parts[0] == "config":
         w = inputs.config(int(parts[1]))
         if len(parts) > 2:
@@ -468,7 +562,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--table", choices=["configs", "sweep"], default=None)
+    ap.add_argument("--table", choices=["configs", "sweep", "vecmat"], default=None)
     ap.add_argument("--filter", default=None)
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
@@ -485,6 +579,8 @@ def main():
     __graft_entry__.build()
     if args.case:
         return run_case(args)
+    if args.table == "vecmat":
+        return run_vecmat_table(args)
     if args.table:
         return run_table(args)
     run_ours(args)

@@ -120,6 +120,25 @@ tf_status tf_copy(const void* x, void* y, int64_t bytes, void* cuda_stream);
  * fp32 arithmetic with full range reduction, one rounding to the storage type.  y == x is allowed. */
 tf_status tf_sin_fwd(const void* x, void* y, int64_t n, tf_dtype dt, int threads, int vectors_per_thread, void* cuda_stream);
 
+/* ---- second memory-bound workload -------------------------------------------------------------------- */
+
+/* Batched vector-matrix product (the paper's Case Study 2, "GEMV restructuring"):
+ *     C[m,n] = sum_{k<K} A[m,k] * B[m,n,k]
+ * A is [M, K], B is [M, N, K] with k contiguous, C is [M, N]; all dense, device memory, one element type.
+ * Products are exact in fp32, accumulation is fp32, C gets one round-to-nearest-even conversion.  B is read once:
+ * the operation is bound by HBM bandwidth.  Launch geometry, every knob 0 = automatic:
+ *   threads  per CTA, a multiple of 32, at most 1024;
+ *   lanes    per row group on the plain path (4, 8, 16 or 32); bf16 with lanes = 0 takes the tensor-core path;
+ *   rows     consecutive n that share one load of the A[m,:] pieces: 1, 2 or 4 per lane group on the plain path,
+ *            16 or 32 per warp on the tensor-core path;
+ *   ksplit   warps of a CTA that share a row group along k on the tensor-core path (1, 2, 4 or 8).
+ * 16-byte aligned A and B with K * sizeof(element) a multiple of 16 take a vector path, anything else a scalar one.
+ * Errors: TF_ERR_INVALID_ARG for a null pointer with M*N > 0, K <= 0, an unknown element type or a knob outside its
+ * set; TF_ERR_UNSUPPORTED when the grid would exceed 2^31 - 1 CTAs.  Asynchronous on cuda_stream; allocates nothing;
+ * A, B, C stay the caller's. */
+tf_status tf_bvecmat_fwd(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, tf_dtype dt, int threads,
+                         int lanes, int rows, int ksplit, void* cuda_stream);
+
 const char* tf_status_string(tf_status s);
 
 /* cudaError_t value behind the most recent TF_ERR_CUDA on the calling thread (0 if none). */

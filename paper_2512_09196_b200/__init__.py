@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_status_string",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
 
@@ -53,6 +53,7 @@ def lib() -> ctypes.CDLL:
         L.tf_rmsnorm_fwd.argtypes = [vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_tune.argtypes = [i32, i64, i64, i32]
         L.tf_copy.argtypes = [vp, vp, i64, vp]
+        L.tf_bvecmat_fwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp]
         L.tf_sin_fwd.argtypes = [vp, vp, i64, i32, i32, i32, vp]
         L.tf_tune_like.argtypes = [i32, vp, vp, vp, i64, i64, i32]
         L.tf_tune_report.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(f32)]
@@ -68,7 +69,7 @@ def lib() -> ctypes.CDLL:
         L.tf_clear_cache.restype = None
         L.tf_launch_count.argtypes = []
         L.tf_launch_count.restype = i64
-        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd",
+        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd",
                      "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice",
                      "tf_candidate_count", "tf_candidate"):
             getattr(L, name).restype = i32
@@ -170,6 +171,24 @@ def tf_sin_fwd(x, y=None, threads: int = 0, vectors_per_thread: int = 0):
     with _on_device(x):
         _ok(lib().tf_sin_fwd(x.data_ptr(), y.data_ptr(), x.numel(), _dt(x), threads, vectors_per_thread, _stream(x)), "tf_sin_fwd")
     return y
+
+
+def tf_bvecmat_fwd(a, b, c=None, threads: int = 0, lanes: int = 0, rows: int = 0, ksplit: int = 0):
+    """C[m,n] = sum_k A[m,k] * B[m,n,k] for contiguous CUDA tensors a [M, K], b [M, N, K] (fp32 or bf16)."""
+    import torch
+    if not (a.is_cuda and b.is_cuda and a.is_contiguous() and b.is_contiguous()) or a.dim() != 2 or b.dim() != 3:
+        raise ValueError("a must be a contiguous CUDA [M, K] tensor and b a contiguous CUDA [M, N, K] tensor")
+    M, K = a.shape
+    if b.shape[0] != M or b.shape[2] != K or b.dtype != a.dtype:
+        raise ValueError("shape or dtype mismatch between a and b")
+    N = b.shape[1]
+    if c is None:
+        c = torch.empty((M, N), dtype=a.dtype, device=a.device)
+    with _on_device(a):
+        _ok(lib().tf_bvecmat_fwd(a.data_ptr(), b.data_ptr(), c.data_ptr(), M, N, K, _dt(a), threads, lanes, rows, ksplit,
+                                 _stream(a)),
+            "tf_bvecmat_fwd")
+    return c
 
 
 def tf_layernorm_fwd(x, gamma, beta, eps: float, y=None, mean=None, rstd=None, want_stats: bool = True):

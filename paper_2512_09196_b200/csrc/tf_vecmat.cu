@@ -1,0 +1,325 @@
+// Batched vector-matrix product of the paper's Case Study 2:  C[m,n] = sum_k A[m,k] * B[m,n,k].
+//
+// B ([M, N, K], k contiguous) is read exactly once and dominates the traffic, so this is a streamed reduction bound by
+// HBM (every element of B meets one multiply-add).  Viewed as M*N rows of length K, each row is dotted with the vector
+// A[m,:] of its batch entry.  Measured on B200: the B stream alone runs at about 7.0 TB/s, and what holds a kernel below
+// that is the traffic of the A pieces through L1/L2, one 16-byte A load for every 16-byte B load when each row fetches
+// its own.  So both paths below let one A load serve several rows:
+//   plain path (fp32, and bf16 when forced): a group of 4..32 lanes owns R consecutive n of one m; per step it loads
+//     U vectors of A[m,:] once and the matching vectors of its R rows, accumulates in packed fp32 pairs, reduces with
+//     shuffles, writes R elements of C;
+//   tensor-core path (bf16): a warp owns RT tiles of 16 consecutive n and feeds m16n8k16 multiply-accumulates straight
+//     from the packed words it loaded (see below).
+// One contiguous block of rows per CTA, as many CTAs as there are blocks.
+#include <algorithm>
+
+#include "../../include/tf.h"
+#include "tf_common.cuh"
+
+namespace tf {
+namespace {
+
+// Lane group of LANES lanes, R rows, U vectors per row and step.  All loops have warp-uniform trip counts.
+template <int DT, int LANES, int R, int U>
+__global__ void __launch_bounds__(1024) k_vecmat(const uint4* __restrict__ A, const uint4* __restrict__ B,
+                                                 typename Elem<DT>::scalar* __restrict__ C, int64_t N, int kvec, int tiles_per_m, int64_t tiles) {
+    using P = Pairs<DT>;
+    constexpr int NP = P::NP;
+    pdl_wait();
+    pdl_trigger();
+    const int lane = threadIdx.x % LANES;
+    const int64_t tile = static_cast<int64_t>(blockIdx.x) * (blockDim.x / LANES) + threadIdx.x / LANES;
+    const bool tile_live = tile < tiles;                          // every lane runs the loop: shuffles need the whole warp
+    const int64_t m = tile_live ? tile / tiles_per_m : 0;
+    const int64_t n0 = tile_live ? (tile - m * tiles_per_m) * R : 0;
+    const int64_t out = m * N + n0;
+    const int n_left = tile_live ? static_cast<int>(N - n0 < R ? N - n0 : R) : 0;
+    const uint4* a = A + m * kvec;
+    const uint4* b[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) b[r] = B + (out + (r < n_left ? r : 0)) * kvec;
+    F2 acc[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) acc[r] = f2(0.f);
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+#pragma unroll(R == 2 ? 2 : 1)                                  // measured: R = 2 gains from a second step in flight, R = 1 and 4 lose occupancy
+    for (int v0 = lane; v0 < kvec; v0 += LANES * U) {
+        uint4 bv[R][U], av[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int v = v0 + u * LANES;
+            const bool ok = v < kvec;
+            av[u] = ok && tile_live ? ld_param(a + v) : zero;
+#pragma unroll
+            for (int r = 0; r < R; ++r) bv[r][u] = ok && r < n_left ? ld_stream(b[r] + v) : zero;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            F2 y[NP];
+            P::unpack(av[u], y);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                F2 x[NP];
+                P::unpack(bv[r][u], x);
+#pragma unroll
+                for (int i = 0; i < NP; ++i) acc[r] = fma2(x[i], y[i], acc[r]);
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const float dot = group_reduce<SumOp, LANES>(hsum(acc[r]));
+        if (lane == 0 && r < n_left) C[out + r] = Elem<DT>::from_float(dot);
+    }
+}
+
+// bf16 through the tensor cores.  Unpacking bf16 pairs and issuing fp32 multiply-adds per element costs instruction
+// slots that a 7 TB/s stream does not leave; m16n8k16 multiply-accumulates take the packed pairs as they arrive.
+// A warp owns RT tiles of 16 consecutive n of one batch entry.  Lane (g, t) = (lane / 4, lane % 4) loads 16-byte vectors
+// of rows g and g + 8 of each tile and the matching vector of A[m,:]; since a sum over k does not care which k sits in
+// which slot of the fragment, the four 32-bit words of a vector serve directly as the (k-slot 2t, 2t+8) words of two
+// fragments, and the words of the A[m,:] vector, the same for every g, as the column operand: every output column holds
+// the same dot product and column 0 is kept.  Products are exact in fp32; each step's four multiply-accumulates start
+// from zero and the step totals are added in ordinary fp32, so the result does not lean on how the tensor core rounds
+// long chains.  With few tiles, `ksplit` warps of a CTA share a tile group along k and combine through shared memory.
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int WARPS, int RT>
+__global__ void __launch_bounds__(WARPS * 32) k_vecmat_mma(const uint4* __restrict__ A, const uint4* __restrict__ B, uint16_t* __restrict__ C,
+                                                           int64_t N, int kvec, int ksplit, int tiles_per_m, int64_t tiles) {
+    constexpr int ROWS = 16 * RT;                                 // n per warp
+    __shared__ float part[WARPS][ROWS];
+    pdl_wait();
+    pdl_trigger();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int64_t tile = static_cast<int64_t>(blockIdx.x) * (WARPS / ksplit) + warp / ksplit;
+    const int kw = warp % ksplit;
+    const bool tile_live = tile < tiles;
+    const int64_t m = tile_live ? tile / tiles_per_m : 0;
+    const int64_t n0 = tile_live ? (tile - m * tiles_per_m) * ROWS : 0;
+    const int64_t out = m * N + n0;
+    const int n_left = tile_live ? static_cast<int>(N - n0 < ROWS ? N - n0 : ROWS) : 0;
+    const uint4* a = A + m * kvec;
+    const uint4* b[RT][2];                                        // row g + 8*h of tile q is local row 16*q + 8*h + g
+#pragma unroll
+    for (int q = 0; q < RT; ++q)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int row = 16 * q + 8 * h + g;
+            b[q][h] = B + (out + (row < n_left ? row : 0)) * kvec;
+        }
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    float acc[RT][2];
+#pragma unroll
+    for (int q = 0; q < RT; ++q) acc[q][0] = acc[q][1] = 0.f;
+    const int steps = (kvec + 7) / 8;                             // a step is 8 vectors = 64 elements of every row
+#pragma unroll 2
+    for (int s = kw; s < steps; s += ksplit) {                    // trip count is the same for every lane of a warp
+        uint4 r[RT][2][2], v[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int vi = s * 8 + j * 4 + t;
+            const bool ok = vi < kvec;
+            v[j] = ok && tile_live ? ld_param(a + vi) : zero;
+#pragma unroll
+            for (int q = 0; q < RT; ++q)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) r[q][h][j] = ok && 16 * q + 8 * h + g < n_left ? ld_stream(b[q][h] + vi) : zero;
+        }
+#pragma unroll
+        for (int q = 0; q < RT; ++q) {
+            float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                mma_bf16_16816(c, r[q][0][j].x, r[q][1][j].x, r[q][0][j].y, r[q][1][j].y, v[j].x, v[j].y);
+                mma_bf16_16816(c, r[q][0][j].z, r[q][1][j].z, r[q][0][j].w, r[q][1][j].w, v[j].z, v[j].w);
+            }
+            acc[q][0] += c[0];
+            acc[q][1] += c[2];
+        }
+    }
+    if (ksplit == 1) {
+        if (t == 0) {
+#pragma unroll
+            for (int q = 0; q < RT; ++q)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int row = 16 * q + 8 * h + g;
+                    if (row < n_left) C[out + row] = Elem<DT_BF16>::from_float(acc[q][h]);
+                }
+        }
+        return;                                                   // uniform over the CTA: ksplit is a launch constant
+    }
+    if (t == 0) {
+#pragma unroll
+        for (int q = 0; q < RT; ++q)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) part[warp][16 * q + 8 * h + g] = acc[q][h];
+    }
+    __syncthreads();
+    if (kw == 0) {
+        for (int row = lane; row < n_left; row += 32) {
+            float sum = 0.f;
+            for (int i = 0; i < ksplit; ++i) sum += part[warp + i][row];
+            C[out + row] = Elem<DT_BF16>::from_float(sum);
+        }
+    }
+}
+
+// Any alignment, any K: a warp per row, scalar accesses.
+template <int DT>
+__global__ void __launch_bounds__(1024) k_vecmat_scalar(const typename Elem<DT>::scalar* A, const typename Elem<DT>::scalar* B,
+                                                        typename Elem<DT>::scalar* C, int64_t rows, int64_t N, int64_t K) {
+    using E = Elem<DT>;
+    const int lane = threadIdx.x & 31;
+    const int64_t r = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const bool live = r < rows;
+    const int64_t rr = live ? r : 0;
+    float acc = 0.f;
+    for (int64_t k = lane; k < K; k += 32) acc = fmaf(E::to_float(B[rr * K + k]), E::to_float(A[(rr / N) * K + k]), acc);
+    acc = group_reduce<SumOp, 32>(acc);
+    if (live && lane == 0) C[r] = E::from_float(acc);
+}
+
+bool al16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <class... T>
+cudaError_t launch_pdl(void (*fn)(T...), int64_t grid, int threads, cudaStream_t st, T... args) {
+    if (grid > 0x7FFFFFFF) return cudaErrorInvalidConfiguration;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(threads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, args...);
+}
+
+int sm_count() {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms;
+}
+
+// Warps wanted: about four waves of fully occupied SMs, so that the last, partly filled wave is a small part of the
+// run (the partial-wave tail that the paper's case study removes with a tunable grid).
+int64_t warps_wanted(int sms) { return 4LL * 64 * sms; }
+
+
+template <int DT, int LANES, int R>
+cudaError_t launch_plain_lr(int threads, cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t kvec) {
+    constexpr int U = R == 1 ? 4 : R == 2 ? 2 : 1;
+    using S = typename Elem<DT>::scalar;
+    const int64_t tiles_per_m = (N + R - 1) / R, tiles = M * tiles_per_m;
+    if (tiles_per_m > 0x7FFFFFFF || kvec > 0x7FFFFFF0) return cudaErrorInvalidConfiguration;
+    const int gpc = threads / LANES;
+    return launch_pdl(k_vecmat<DT, LANES, R, U>, (tiles + gpc - 1) / gpc, threads, st, static_cast<const uint4*>(A),
+                      static_cast<const uint4*>(B), static_cast<S*>(C), N, static_cast<int>(kvec), static_cast<int>(tiles_per_m), tiles);
+}
+
+template <int DT, int LANES>
+cudaError_t launch_plain_l(int rows, int threads, cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t kvec) {
+    switch (rows) {
+        case 1: return launch_plain_lr<DT, LANES, 1>(threads, st, A, B, C, M, N, kvec);
+        case 2: return launch_plain_lr<DT, LANES, 2>(threads, st, A, B, C, M, N, kvec);
+        default: return launch_plain_lr<DT, LANES, 4>(threads, st, A, B, C, M, N, kvec);
+    }
+}
+
+template <int DT>
+cudaError_t launch_plain(int lanes, int rows, int threads, cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N,
+                         int64_t kvec) {
+    const int sms = sm_count();
+    // Measured on the K sweep: rows of up to 4 KiB run best with two rows per group sharing each A load and two
+    // vectors per lane and step; longer rows with one row per group and four vectors in flight per lane.
+    if (lanes == 0) lanes = kvec <= 8 ? 4 : kvec <= 16 ? 8 : kvec <= 32 ? 16 : 32;
+    if (rows == 0) rows = (kvec <= 256 && N >= 2 && M * ((N + 1) / 2) * lanes / 32 >= warps_wanted(sms) / 4) ? 2 : 1;
+    switch (lanes) {
+        case 4: return launch_plain_l<DT, 4>(rows, threads, st, A, B, C, M, N, kvec);
+        case 8: return launch_plain_l<DT, 8>(rows, threads, st, A, B, C, M, N, kvec);
+        case 16: return launch_plain_l<DT, 16>(rows, threads, st, A, B, C, M, N, kvec);
+        default: return launch_plain_l<DT, 32>(rows, threads, st, A, B, C, M, N, kvec);
+    }
+}
+
+template <int WARPS, int RT>
+cudaError_t launch_mma_wr(cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t kvec, int ksplit) {
+    const int64_t tiles_per_m = (N + 16 * RT - 1) / (16 * RT), tiles = M * tiles_per_m;
+    if (tiles_per_m > 0x7FFFFFFF || kvec > 0x7FFFFFF0) return cudaErrorInvalidConfiguration;
+    if (ksplit > WARPS) ksplit = WARPS;
+    const int tpc = WARPS / ksplit;
+    return launch_pdl(k_vecmat_mma<WARPS, RT>, (tiles + tpc - 1) / tpc, WARPS * 32, st, static_cast<const uint4*>(A),
+                      static_cast<const uint4*>(B), static_cast<uint16_t*>(C), N, static_cast<int>(kvec), ksplit, static_cast<int>(tiles_per_m), tiles);
+}
+
+cudaError_t launch_mma(int rows, int ksplit, int threads, cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N,
+                       int64_t kvec) {
+    const int sms = sm_count();
+    const int64_t steps = (kvec + 7) / 8;
+    if (rows == 0) rows = (steps <= 2 && N >= 32 && M * ((N + 31) / 32) >= warps_wanted(sms)) ? 32 : 16;
+    if (ksplit == 0) {
+        // Measured on the K sweep: from 512 elements per row on, two warps sharing a tile along k beat one (shorter
+        // dependent chains of steps per warp); beyond that k is cut only until one wave of resident warps exists.
+        const int64_t tiles = M * ((N + rows - 1) / rows);
+        ksplit = steps >= 8 ? 2 : 1;
+        while (ksplit < 8 && ksplit * 32 < threads && tiles * ksplit < 32LL * sms && steps >= 4 * ksplit) ksplit *= 2;
+    }
+    if (rows == 32)
+        return threads <= 128 ? launch_mma_wr<4, 2>(st, A, B, C, M, N, kvec, ksplit)
+             : threads <= 256 ? launch_mma_wr<8, 2>(st, A, B, C, M, N, kvec, ksplit)
+                              : launch_mma_wr<16, 2>(st, A, B, C, M, N, kvec, ksplit);
+    return threads <= 128 ? launch_mma_wr<4, 1>(st, A, B, C, M, N, kvec, ksplit)
+         : threads <= 256 ? launch_mma_wr<8, 1>(st, A, B, C, M, N, kvec, ksplit)
+                          : launch_mma_wr<16, 1>(st, A, B, C, M, N, kvec, ksplit);
+}
+
+}  // namespace
+}  // namespace tf
+
+using namespace tf;
+
+extern "C" tf_status tf_bvecmat_fwd(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K, tf_dtype dt_, int threads,
+                                    int lanes, int rows, int ksplit, void* stream) {
+    const int dt = dt_;
+    if (M < 0 || N < 0 || K <= 0 || (dt != DT_F32 && dt != DT_BF16)) return TF_ERR_INVALID_ARG;
+    if (M > 0 && N > 0 && (!A || !B || !C)) return TF_ERR_INVALID_ARG;
+    if (threads == 0) threads = 128;
+    const bool tensor = dt == DT_BF16 && lanes == 0;              // a forced `lanes` selects the plain path
+    if (threads < 32 || threads > 1024 || threads % 32 || (lanes != 0 && lanes != 4 && lanes != 8 && lanes != 16 && lanes != 32) ||
+        (ksplit != 0 && ksplit != 1 && ksplit != 2 && ksplit != 4 && ksplit != 8))
+        return TF_ERR_INVALID_ARG;
+    if (tensor ? (rows != 0 && rows != 16 && rows != 32) : (rows != 0 && rows != 1 && rows != 2 && rows != 4))
+        return TF_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return TF_OK;
+    if (N > INT64_MAX / M || K > (INT64_MAX / 8) / (M * N)) return TF_ERR_UNSUPPORTED;
+    const int64_t nrows = M * N;
+    const int es = elem_size(dt);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    count_launches(1);
+    if (al16(A) && al16(B) && (K * es) % 16 == 0) {
+        const int64_t kvec = K * es / 16;
+        if (tensor) e = launch_mma(rows, ksplit, threads, st, A, B, C, M, N, kvec);
+        else if (dt == DT_F32) e = launch_plain<DT_F32>(lanes, rows, threads, st, A, B, C, M, N, kvec);
+        else e = launch_plain<DT_BF16>(lanes, rows, threads, st, A, B, C, M, N, kvec);
+    } else {
+        const int64_t grid = (nrows + threads / 32 - 1) / (threads / 32);
+        if (grid > 0x7FFFFFFF) return TF_ERR_UNSUPPORTED;
+        if (dt == DT_F32)
+            k_vecmat_scalar<DT_F32><<<static_cast<unsigned>(grid), threads, 0, st>>>(static_cast<const float*>(A), static_cast<const float*>(B), static_cast<float*>(C), nrows, N, K);
+        else
+            k_vecmat_scalar<DT_BF16><<<static_cast<unsigned>(grid), threads, 0, st>>>(static_cast<const uint16_t*>(A), static_cast<const uint16_t*>(B), static_cast<uint16_t*>(C), nrows, N, K);
+        e = cudaGetLastError();
+    }
+    if (e == cudaErrorInvalidConfiguration) return TF_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) { remember_cuda_error(e); return TF_ERR_CUDA; }
+    return TF_OK;
+}

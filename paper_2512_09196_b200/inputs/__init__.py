@@ -1,4 +1,4 @@
-"""Seeded synthetic workloads (numpy, host memory) for the three row-wise ops.
+"""Seeded synthetic workloads (numpy, host memory) for the three row-wise ops and the batched vector-matrix product.
 
 Data generation only: nothing here computes a softmax or a norm.  The generator is a small C file
 (``gen.c``, built with gcc + OpenMP) so that the 2 GiB workload is produced in seconds; every element
@@ -200,3 +200,50 @@ def shard_rows(rows: int, rank: int, world: int) -> tuple[int, int]:
     q, r = divmod(rows, world)
     n = q + (1 if rank < r else 0)
     return rank * q + min(rank, r), n
+
+
+@dataclass(frozen=True)
+class VecMat:
+    """One point of the batched vector-matrix workload  C[m,n] = sum_k A[m,k] * B[m,n,k]:  A [M, K] ~ N(0, 1),
+    B [M, N, K] ~ N(0, 1) (streams 0 and 1 of the counter-based generator)."""
+    name: str
+    dt: int
+    M: int
+    N: int
+    K: int
+    seed: int
+
+    @property
+    def elem_size(self) -> int:
+        return ELEM_SIZE[self.dt]
+
+    @property
+    def dtype_name(self) -> str:
+        return "f32" if self.dt == F32 else "bf16"
+
+    def algorithmic_bytes(self) -> int:
+        """A in once, B in once, C out once."""
+        return (self.M * self.K + self.M * self.N * self.K + self.M * self.N) * self.elem_size
+
+    def generate(self) -> dict:
+        return {"a": normal((self.M, self.K), self.dt, self.seed, 0, 0.0, 1.0),
+                "b": normal((self.M, self.N, self.K), self.dt, self.seed, 1, 0.0, 1.0)}
+
+
+VECMAT_KS = (64, 256, 1000, 1024, 4096, 16384)
+VECMAT_BYTES = 512 << 20
+
+
+def vecmat_point(dt: int, K: int, M: int = 64, b_bytes: int = VECMAT_BYTES) -> VecMat:
+    """N = floor(b_bytes / (M * K * elem_size)): B holds about b_bytes whatever K is."""
+    N = max(1, b_bytes // (M * K * ELEM_SIZE[dt]))
+    return VecMat(f"bvecmat_{'f32' if dt == F32 else 'bf16'}_{M}x{N}x{K}", dt, M, N, K, seed=K)
+
+
+def vecmat_headline() -> VecMat:
+    """bf16, B = 1.5 GiB: the traffic that the paper's reported runtime and memory throughput for this kernel imply."""
+    return VecMat("bvecmat_bf16_96x2048x4096", BF16, 96, 2048, 4096, seed=96)
+
+
+def vecmat_sweep():
+    return [vecmat_headline()] + [vecmat_point(dt, K) for dt in (F32, BF16) for K in VECMAT_KS]
