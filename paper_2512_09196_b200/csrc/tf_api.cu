@@ -79,7 +79,7 @@ std::string plan_to_string(const Plan& p) {
         case V_TMA: snprintf(b, sizeof b, "tma:threads=%d,cluster=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.cluster, p.stages, p.chunk, p.persist); break;
         case V_PIPE: snprintf(b, sizeof b, "pipe:threads=%d,lanes=%d,vpt=%d,rpg=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.lanes, p.vpt, p.rpg, p.stages, p.chunk, p.persist); break;
         case V_RING: snprintf(b, sizeof b, "ring:threads=%d,vpt=%d,cluster=%d,stages=%d,persist=%d", p.threads, p.vpt, p.cluster, p.stages, p.persist); break;
-        case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,cache=%d,persist=%d", p.threads, p.chunk, p.persist); break;
+        case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,cache=%d,persist=%d,regcap=%d", p.threads, p.chunk, p.persist, p.rpg == 2 ? 1 : 0); break;
         case V_SPLIT: snprintf(b, sizeof b, "split:threads=%d,splits=%d", p.threads, p.cluster); break;
         default: snprintf(b, sizeof b, "stream:threads=%d,lanes=%d,persist=%d", p.threads, p.lanes, p.persist); break;
     }
@@ -108,7 +108,7 @@ bool plan_from_string(const char* s, Plan& out) {
         if (end == eq + 1) return false;
         if (key == "threads") p.threads = val; else if (key == "lanes") p.lanes = val; else if (key == "vpt") p.vpt = val;
         else if (key == "rpg") p.rpg = val; else if (key == "cluster" || key == "splits") p.cluster = val; else if (key == "stages") p.stages = val;
-        else if (key == "chunk" || key == "cache") p.chunk = val; else if (key == "persist") p.persist = val; else return false;
+        else if (key == "chunk" || key == "cache") p.chunk = val; else if (key == "persist") p.persist = val; else if (key == "regcap") p.rpg = val ? 2 : 1; else return false;
         q = (*end == ',') ? end + 1 : end;
         if (*end && *end != ',') return false;
     }
@@ -342,6 +342,7 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
                     Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = persist;
                     p.chunk = cache ? static_cast<int>(std::min<int64_t>(nvec * 16, (200 * 1024 / (2048 / th)) / 16 * 16)) : 0;
                     add(p);
+                    if (th <= 768 && persist == 0) { p.rpg = 2; add(p); }      // 40-register form: 1536 resident threads per SM
                 }
     // persistent cluster ring for long rows
     if (nvec >= 2048)
@@ -392,6 +393,7 @@ std::vector<Plan> neighbours(const Plan& b) {
     if (b.variant == V_PIPE || b.variant == V_WARP)
         for (int r : {1, 2, 4})
             if (r != b.rpg) with([&](Plan& p) { p.rpg = r; });
+    if (b.variant == V_TWOPASS) with([&](Plan& p) { p.rpg = b.rpg == 2 ? 1 : 2; });
     if (b.variant == V_SPLIT)
         for (int sp : {b.cluster / 2, b.cluster * 3 / 4, b.cluster * 3 / 2, b.cluster * 2})
             if (sp >= 1 && sp != b.cluster) with([&](Plan& p) { p.cluster = sp; });

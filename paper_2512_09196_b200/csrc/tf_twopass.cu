@@ -30,8 +30,10 @@ struct WArgs {
     float n, eps;
 };
 
-template <int OP, int DT>
-__global__ void __launch_bounds__(1024) k_twopass(const WArgs a) {
+// MAXT / MINB: the launch bounds.  Besides the unconstrained form (1024, 0) there are (768, 2) and (512, 3), which hold
+// the kernel to 40 registers so that 1536 threads are resident per SM instead of 1024-1280.
+template <int OP, int DT, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB) k_twopass(const WArgs a) {
     __shared__ float red_buf[4 * 32];
     extern __shared__ __align__(16) unsigned char dyn_smem[];
     uint4* const cache = reinterpret_cast<uint4*>(dyn_smem);
@@ -54,28 +56,36 @@ __global__ void __launch_bounds__(1024) k_twopass(const WArgs a) {
 
 using TwoFn = void (*)(const WArgs);
 
-TwoFn two_fn(int op, int dt) {
+template <int MAXT, int MINB>
+TwoFn two_fn_b(int op, int dt) {
     switch (op * 2 + dt) {
-        case 0: return k_twopass<OP_SOFTMAX, DT_F32>;
-        case 1: return k_twopass<OP_SOFTMAX, DT_BF16>;
-        case 2: return k_twopass<OP_LAYERNORM, DT_F32>;
-        case 3: return k_twopass<OP_LAYERNORM, DT_BF16>;
-        case 4: return k_twopass<OP_RMSNORM, DT_F32>;
-        case 5: return k_twopass<OP_RMSNORM, DT_BF16>;
+        case 0: return k_twopass<OP_SOFTMAX, DT_F32, MAXT, MINB>;
+        case 1: return k_twopass<OP_SOFTMAX, DT_BF16, MAXT, MINB>;
+        case 2: return k_twopass<OP_LAYERNORM, DT_F32, MAXT, MINB>;
+        case 3: return k_twopass<OP_LAYERNORM, DT_BF16, MAXT, MINB>;
+        case 4: return k_twopass<OP_RMSNORM, DT_F32, MAXT, MINB>;
+        case 5: return k_twopass<OP_RMSNORM, DT_BF16, MAXT, MINB>;
     }
     return nullptr;
 }
 
+TwoFn two_fn(int op, int dt, int threads, bool capped) {
+    if (capped && threads <= 512) return two_fn_b<512, 3>(op, dt);
+    if (capped && threads <= 768) return two_fn_b<768, 2>(op, dt);
+    return two_fn_b<1024, 0>(op, dt);
+}
+
 }  // namespace
 
-// Plan field `chunk`: bytes of each row's head kept in shared memory between the passes (0 = none).
+// Plan field `chunk`: bytes of each row's head kept in shared memory between the passes (0 = none); `rpg` = 2 selects
+// the register-capped build (threads <= 768).
 bool supports_twopass(const Plan& p, const Args& a, const DeviceInfo& d) {
-    return vector_ok(a) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0 && p.chunk >= 0 && p.chunk % 16 == 0 &&
+    return vector_ok(a) && (p.rpg == 1 || (p.rpg == 2 && p.threads <= 768)) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0 && p.chunk >= 0 && p.chunk % 16 == 0 &&
            (d.smem_optin == 0 || p.chunk + 2048 <= d.smem_optin);
 }
 
 cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
-    TwoFn fn = two_fn(a.op, a.dt);
+    TwoFn fn = two_fn(a.op, a.dt, p.threads, p.rpg == 2);
     if (!fn) return cudaErrorInvalidValue;
     int64_t grid = a.rows;
     if (p.persist > 0) grid = std::min<int64_t>(grid, static_cast<int64_t>(p.persist) * d.sms);

@@ -251,11 +251,11 @@ def test_forced_ring_variants(op, dt, cluster):
 @pytest.mark.parametrize("dt", [F32, BF16])
 def test_forced_twopass_variants(op, dt):
     ne = 4 if dt == F32 else 8
-    for threads, persist in ((32, 0), (256, 1), (1024, 0)):
+    for threads, persist, regcap in ((32, 0, 0), (256, 1, 0), (1024, 0, 0), (512, 0, 1), (768, 0, 1), (96, 2, 1)):
         for nvec, rows in ((1, 5), (threads * 4, 9), (threads * 4 + 1, 9), (threads * 9 - 3, 300), (70001, 3)):
-            tf.tf_force_plan(op, f"twopass:threads={threads},persist={persist}")
+            tf.tf_force_plan(op, f"twopass:threads={threads},persist={persist},regcap={regcap}")
             fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec))
-            assert not fails, (threads, persist, nvec, rows, fails)
+            assert not fails, (threads, persist, regcap, nvec, rows, fails)
     if op == "softmax":                                    # masks, a fully masked row and outputs in the subnormal range
         tf.tf_force_plan(op, "twopass:threads=256,persist=0")
         w = Workload("m", "softmax", dt, 12, 40000, seed=5, x_std=10.0, mask_step=3001)
