@@ -41,6 +41,7 @@ template <int OP, int DT> struct Running {
     float s_off = 0.f, s_sum = 0.f, s_max = kNegInf;
     float c_n = 0.f, c_mean = 0.f, c_m2 = 0.f;
     F2 q2 = f2(0.f);
+    int64_t live_end = 0;            // softmax: one past the last vector of THIS thread that held anything but -inf
 
     __device__ __forceinline__ void update(const uint4 (&raw)[kStreamU], const bool (&ok)[kStreamU]) {
         using P = Pairs<DT>;
@@ -122,6 +123,7 @@ __device__ __forceinline__ Running<OP, DT> stream_stats(const uint4* xs, int64_t
         for (int u = 0; u < U; ++u) {
             const int64_t idx = base + static_cast<int64_t>(u) * T;
             if (idx < cache_vecs) cache[idx] = raw[u];          // cache_vecs <= nvec
+            if (OP == OP_SOFTMAX && ok[u] && !all_neg_inf_vec<DT>(raw[u])) run.live_end = idx + 1;
         }
         run.update(raw, ok);
     }
@@ -160,10 +162,12 @@ __device__ __forceinline__ RowScale scale_of_row(const Part& p, float n, float e
 }
 
 // Pass B over `nvec` vectors: xs/ys point at the segment, g/b at the parameters of its first column.
+// live_end: this thread's Running::live_end when the same thread ran pass A over the same vectors (softmax): vectors
+// from there on are known to be all -inf, so their zeros are written without reading x again.
 template <int OP, int DT>
 __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const uint4* g, const uint4* b, int64_t nvec,
                                              const RowScale& sc, uint64_t policy, const uint4* cache = nullptr,
-                                             int64_t cache_vecs = 0) {
+                                             int64_t cache_vecs = 0, int64_t live_end = INT64_MAX) {
     using P = Pairs<DT>;
     constexpr int NP = P::NP, U = kStreamU;
     const int T = blockDim.x, t = threadIdx.x;
@@ -178,7 +182,7 @@ __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const u
         for (int u = 0; u < U; ++u) {
             const int64_t idx = base + static_cast<int64_t>(u) * T;
             ok[u] = idx < nvec;
-            raw[u] = !ok[u] ? fill : (idx < cache_vecs ? cache[idx] : ld_hint(xs + idx, policy));
+            raw[u] = (!ok[u] || idx >= live_end) ? fill : (idx < cache_vecs ? cache[idx] : ld_hint(xs + idx, policy));
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {

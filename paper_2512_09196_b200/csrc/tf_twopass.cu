@@ -50,7 +50,8 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass(const WArgs a) {
             if (OP == OP_LAYERNORM && a.mean) a.mean[row] = sc.a;
             if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = sc.b;
         }
-        stream_apply<OP, DT>(xr, a.y + row * a.nvec, a.p0, a.p1, a.nvec, sc, last, cache, a.cache_vecs);
+        stream_apply<OP, DT>(xr, a.y + row * a.nvec, a.p0, a.p1, a.nvec, sc, last, cache, a.cache_vecs,
+                             OP == OP_SOFTMAX ? run.live_end : INT64_MAX);
     }
 }
 
