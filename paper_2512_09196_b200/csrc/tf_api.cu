@@ -78,7 +78,7 @@ std::string plan_to_string(const Plan& p) {
         case V_CTA: snprintf(b, sizeof b, "cta:threads=%d,vpt=%d,cluster=%d,persist=%d", p.threads, p.vpt, p.cluster, p.persist); break;
         case V_TMA: snprintf(b, sizeof b, "tma:threads=%d,cluster=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.cluster, p.stages, p.chunk, p.persist); break;
         case V_PIPE: snprintf(b, sizeof b, "pipe:threads=%d,lanes=%d,vpt=%d,rpg=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.lanes, p.vpt, p.rpg, p.stages, p.chunk, p.persist); break;
-        case V_RING: snprintf(b, sizeof b, "ring:threads=%d,vpt=%d,cluster=%d,stages=%d,persist=%d", p.threads, p.vpt, p.cluster, p.stages, p.persist); break;
+        case V_RING: snprintf(b, sizeof b, "ring:threads=%d,vpt=%d,cluster=%d,stages=%d,persist=%d,psmem=%d", p.threads, p.vpt, p.cluster, p.stages, p.persist, p.rpg == 2 ? 1 : 0); break;
         case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,cache=%d,persist=%d,regcap=%d", p.threads, p.chunk, p.persist, p.rpg == 2 ? 1 : 0); break;
         case V_SPLIT: snprintf(b, sizeof b, "split:threads=%d,splits=%d", p.threads, p.cluster); break;
         default: snprintf(b, sizeof b, "stream:threads=%d,lanes=%d,persist=%d", p.threads, p.lanes, p.persist); break;
@@ -108,7 +108,7 @@ bool plan_from_string(const char* s, Plan& out) {
         if (end == eq + 1) return false;
         if (key == "threads") p.threads = val; else if (key == "lanes") p.lanes = val; else if (key == "vpt") p.vpt = val;
         else if (key == "rpg") p.rpg = val; else if (key == "cluster" || key == "splits") p.cluster = val; else if (key == "stages") p.stages = val;
-        else if (key == "chunk" || key == "cache") p.chunk = val; else if (key == "persist") p.persist = val; else if (key == "regcap") p.rpg = val ? 2 : 1; else return false;
+        else if (key == "chunk" || key == "cache") p.chunk = val; else if (key == "persist") p.persist = val; else if (key == "regcap" || key == "psmem") p.rpg = val ? 2 : 1; else return false;
         q = (*end == ',') ? end + 1 : end;
         if (*end && *end != ',') return false;
     }
@@ -359,6 +359,14 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
                     p.persist = std::max(1, fit);
                     add(p);
                     if (fit > 1) { p.persist = 1; add(p); }
+                    if (vpt == 8 && a.op != OP_SOFTMAX)                    // parameter slices in shared memory behind the ring
+                        for (int st : {1, stages}) {
+                            const int64_t all_bytes = (st + (a.op == OP_LAYERNORM ? 2 : 1)) * per * 16;
+                            if (all_bytes > 200 * 1024 || (st == 1 && stages != 2)) continue;
+                            p.rpg = 2; p.stages = st;
+                            p.persist = std::max(1, static_cast<int>(std::min<int64_t>({8, 200 * 1024 / all_bytes, 2048 / p.threads})));
+                            add(p);
+                        }
                 }
             }
     // shared-memory staged variants
@@ -393,7 +401,7 @@ std::vector<Plan> neighbours(const Plan& b) {
     if (b.variant == V_PIPE || b.variant == V_WARP)
         for (int r : {1, 2, 4})
             if (r != b.rpg) with([&](Plan& p) { p.rpg = r; });
-    if (b.variant == V_TWOPASS) with([&](Plan& p) { p.rpg = b.rpg == 2 ? 1 : 2; });
+    if (b.variant == V_TWOPASS || b.variant == V_RING) with([&](Plan& p) { p.rpg = b.rpg == 2 ? 1 : 2; });
     if (b.variant == V_SPLIT)
         for (int sp : {b.cluster / 2, b.cluster * 3 / 4, b.cluster * 3 / 2, b.cluster * 2})
             if (sp >= 1 && sp != b.cluster) with([&](Plan& p) { p.cluster = sp; });

@@ -56,7 +56,9 @@ __device__ __forceinline__ void push_partial(float* slot, uint64_t* bar, uint32_
 constexpr int ring_max_threads(int vpt) { return vpt <= 4 ? 1024 : 512; }
 __device__ __forceinline__ bool valid_at(int idx, int len) { return idx < len; }
 
-template <int OP, int DT, int VPT>
+// PSMEM: the CTA's slice of gamma/beta (weight) is copied into shared memory once, behind the ring, instead of being
+// fetched from L1/L2 for every row: for long LayerNorm rows the parameters are twice the bytes of x on the L2-to-SM path.
+template <int OP, int DT, int VPT, bool PSMEM>
 __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
     using E = Elem<DT>;
     constexpr int NE = E::NE;
@@ -115,6 +117,17 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
         }
     }
     const LazyParams lazy{a.p0, a.p1, first + t, T};
+    uint4* const pg = ring + static_cast<size_t>(S) * per;        // behind the ring: gamma slice, then beta slice
+    uint4* const pb = pg + per;
+    if constexpr (PSMEM) {
+#pragma unroll
+        for (int v = 0; v < VPT; ++v)
+            if (valid[v]) {
+                pg[t + v * T] = ld_param(a.p0 + first + t + v * T);
+                if (OP == OP_LAYERNORM) pb[t + v * T] = ld_param(a.p1 + first + t + v * T);
+            }
+    }
+    const SmemParams inshared{pg, pb, t, T};
     const uint4 fill = fill_vec<DT>(OP);
     auto slice_count = [&](int k) { return static_cast<float>(max(0, min(per, a.nvec - k * per))) * NE; };
 
@@ -149,6 +162,7 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
         }
         const Total tot = combine_parts<OP>(cs, rank, [&](int k) { return Part{xch[xb][k][0], xch[xb][k][1]}; }, slice_count, a.n, a.eps);
         if constexpr (kHeld) slice_finish<OP, DT, VPT, false>(valid, w, tot, held, out);
+        else if constexpr (PSMEM) slice_finish<OP, DT, VPT, false>(valid, w, tot, inshared, out);
         else slice_finish<OP, DT, VPT, false>(valid, w, tot, lazy, out);
         uint4* yr = a.y + row * a.nvec + first + t;
 #pragma unroll
@@ -163,24 +177,28 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
 
 using RingFn = void (*)(const RArgs);
 
-template <int OP, int DT> RingFn pick_ring(int vpt) {
+template <int OP, int DT> RingFn pick_ring(int vpt, bool psmem) {
+    if (psmem) {                       // only where the parameters are not already held in registers
+        if (OP != OP_SOFTMAX && vpt == 8) return k_ring<OP, DT, 8, (OP != OP_SOFTMAX)>;
+        return nullptr;
+    }
     switch (vpt) {
-        case 1: return k_ring<OP, DT, 1>;
-        case 2: return k_ring<OP, DT, 2>;
-        case 4: return k_ring<OP, DT, 4>;
-        case 8: return k_ring<OP, DT, 8>;
+        case 1: return k_ring<OP, DT, 1, false>;
+        case 2: return k_ring<OP, DT, 2, false>;
+        case 4: return k_ring<OP, DT, 4, false>;
+        case 8: return k_ring<OP, DT, 8, false>;
     }
     return nullptr;
 }
 
-RingFn ring_fn(int op, int dt, int vpt) {
+RingFn ring_fn(int op, int dt, int vpt, bool psmem) {
     switch (op * 2 + dt) {
-        case 0: return pick_ring<OP_SOFTMAX, DT_F32>(vpt);
-        case 1: return pick_ring<OP_SOFTMAX, DT_BF16>(vpt);
-        case 2: return pick_ring<OP_LAYERNORM, DT_F32>(vpt);
-        case 3: return pick_ring<OP_LAYERNORM, DT_BF16>(vpt);
-        case 4: return pick_ring<OP_RMSNORM, DT_F32>(vpt);
-        case 5: return pick_ring<OP_RMSNORM, DT_BF16>(vpt);
+        case 0: return pick_ring<OP_SOFTMAX, DT_F32>(vpt, psmem);
+        case 1: return pick_ring<OP_SOFTMAX, DT_BF16>(vpt, psmem);
+        case 2: return pick_ring<OP_LAYERNORM, DT_F32>(vpt, psmem);
+        case 3: return pick_ring<OP_LAYERNORM, DT_BF16>(vpt, psmem);
+        case 4: return pick_ring<OP_RMSNORM, DT_F32>(vpt, psmem);
+        case 5: return pick_ring<OP_RMSNORM, DT_BF16>(vpt, psmem);
     }
     return nullptr;
 }
@@ -188,7 +206,8 @@ RingFn ring_fn(int op, int dt, int vpt) {
 size_t ring_smem(const Plan& p, const Args& a) {
     const int64_t nvec = a.cols * elem_size(a.dt) / 16;
     const int64_t per = (nvec + p.cluster - 1) / p.cluster;
-    return static_cast<size_t>(p.stages) * per * 16;
+    const int nparam = p.rpg == 2 ? (a.op == OP_LAYERNORM ? 2 : 1) : 0;      // rpg = 2: parameter slices in shared memory
+    return static_cast<size_t>(p.stages + nparam) * per * 16;
 }
 
 }  // namespace
@@ -196,7 +215,7 @@ size_t ring_smem(const Plan& p, const Args& a) {
 bool supports_ring(const Plan& p, const Args& a, const DeviceInfo& d) {
     if (!vector_ok(a) || p.threads < 32 || p.threads % 32 || p.threads > ring_max_threads(p.vpt)) return false;
     if (p.cluster < 1 || p.cluster > kMaxCluster || p.cluster > d.max_cluster || (p.cluster & (p.cluster - 1))) return false;
-    if (p.stages < 1 || p.stages > kRingMaxStages || p.persist < 1 || p.persist > 8 || !ring_fn(a.op, a.dt, p.vpt)) return false;
+    if (p.stages < 1 || p.stages > kRingMaxStages || p.persist < 1 || p.persist > 8 || (p.rpg != 1 && p.rpg != 2) || !ring_fn(a.op, a.dt, p.vpt, p.rpg == 2)) return false;
     const int64_t nvec = a.cols * elem_size(a.dt) / 16;
     if (nvec > 0x7FFFFFFF) return false;
     const int64_t per = (nvec + p.cluster - 1) / p.cluster;
@@ -205,7 +224,7 @@ bool supports_ring(const Plan& p, const Args& a, const DeviceInfo& d) {
 }
 
 cudaError_t launch_ring(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
-    RingFn fn = ring_fn(a.op, a.dt, p.vpt);
+    RingFn fn = ring_fn(a.op, a.dt, p.vpt, p.rpg == 2);
     if (!fn) return cudaErrorInvalidValue;
     cudaError_t e = ensure_max_smem(reinterpret_cast<const void*>(fn), d);
     if (e != cudaSuccess) return e;

@@ -40,6 +40,16 @@ struct LazyParams {
     __device__ __forceinline__ uint4 beta(int v) const { return ld_param(p1 + first + v * stride); }
 };
 
+// Parameters copied once into shared memory by the thread that will use them (a persistent CTA always owns the same
+// columns): no barrier is needed between the copy and the reads.
+struct SmemParams {
+    const uint4* g;
+    const uint4* b;
+    int first, stride;
+    __device__ __forceinline__ uint4 gamma(int v) const { return g[first + v * stride]; }
+    __device__ __forceinline__ uint4 beta(int v) const { return b[first + v * stride]; }
+};
+
 // ---- slice math ---------------------------------------------------------------------------------------
 // A group holds one SLICE of a row (possibly the whole row) as NV vectors per thread; invalid vectors are
 // filled with -inf (softmax) / 0 (norms).  Inside the slice the statistics are exact two-pass ones.  Slices
