@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
                 if (OP == OP_LAYERNORM) pb[t + v * T] = ld_param(a.p1 + first + t + v * T);
             }
     }
-    const SmemParams inshared{pg, pb, t, T};
+    const OwnedSmemParams inshared{pg, pb, t, T};
     const uint4 fill = fill_vec<DT>(OP);
     auto slice_count = [&](int k) { return static_cast<float>(max(0, min(per, a.nvec - k * per))) * NE; };
 

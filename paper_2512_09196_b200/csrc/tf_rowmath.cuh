@@ -42,7 +42,7 @@ struct LazyParams {
 
 // Parameters copied once into shared memory by the thread that will use them (a persistent CTA always owns the same
 // columns): no barrier is needed between the copy and the reads.
-struct SmemParams {
+struct OwnedSmemParams {
     const uint4* g;
     const uint4* b;
     int first, stride;
