@@ -61,6 +61,8 @@ def _load():
         lib.oracle_sin.restype = i32
         lib.oracle_bvecmat.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i32, i32]
         lib.oracle_bvecmat.restype = i32
+        lib.oracle_add.argtypes = [vp, vp, vp, vp, i64, i32]
+        lib.oracle_add.restype = i32
         lib.oracle_bf16_from_double.argtypes = [vp, vp, i64]
         lib.oracle_bf16_from_double.restype = None
         lib.oracle_bf16_to_double.argtypes = [vp, vp, i64]
@@ -149,6 +151,30 @@ def bvecmat(a: np.ndarray, b: np.ndarray, dt: int, want64: bool = False, nthread
     if _load().oracle_bvecmat(_p(a), _p(b), _p(c), _p(c64), _p(sc), M, N, K, dt, nthreads):
         raise ValueError("oracle_bvecmat: bad argument")
     return (c, c64, sc) if want64 else c
+
+
+def add(x: np.ndarray, r: np.ndarray, dt: int, want64: bool = False):
+    """h = x + r rounded once to the storage type (the residual add of a fused add-and-normalise)."""
+    _check(x, dt, "x"), _check(r, dt, "r")
+    if x.shape != r.shape:
+        raise ValueError("x and r must have the same shape")
+    h = np.empty_like(x)
+    h64 = np.empty(x.shape, np.float64) if want64 else None
+    if _load().oracle_add(_p(x), _p(r), _p(h), _p(h64), x.size, dt):
+        raise ValueError("oracle_add: bad argument")
+    return (h, h64) if want64 else h
+
+
+def add_layernorm(x, r, gamma, beta, eps: float, dt: int, want64: bool = False, nthreads: int = 1):
+    """Fused residual add + LayerNorm: ``h = add(x, r)`` then ``layernorm(h)``.  Returns ``(h,) + layernorm(h, ...)``."""
+    h = add(x, r, dt)
+    return (h,) + tuple(layernorm(h, gamma, beta, eps, dt, want64=want64, nthreads=nthreads))
+
+
+def add_rmsnorm(x, r, w, eps: float, dt: int, want64: bool = False, nthreads: int = 1):
+    """Fused residual add + RMSNorm: ``h = add(x, r)`` then ``rmsnorm(h)``.  Returns ``(h,) + rmsnorm(h, ...)``."""
+    h = add(x, r, dt)
+    return (h,) + tuple(rmsnorm(h, w, eps, dt, want64=want64, nthreads=nthreads))
 
 
 def bf16_from_double(v: np.ndarray) -> np.ndarray:

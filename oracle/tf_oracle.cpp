@@ -25,7 +25,10 @@
 // through another route.  The batched vector-matrix product (the paper's Case Study 2) is the plain
 // triple loop in double; it is pinned by all-ones and ramp closed forms, unit-vector selection, an
 // index-order trap (B[m,n,k] versus B[m,k,n] and A[m,k] versus A[n,k]), exact integer brute force,
-// linearity, and numpy's float64 einsum.  tf_tune has
+// linearity, and numpy's float64 einsum.  The residual add that precedes a fused add-and-normalise
+// (h = x + r, rounded once to the storage type; the norm is then the ordinary one applied to h) is
+// pinned by exact small sums, x + 0, x - x, commutativity, bf16 ties to even, and torch's CPU add.
+// tf_tune has
 // no oracle function here: which candidate wins is hardware-dependent ("parity unpinned" for the
 // winner's identity; its output is checked like any other launch).
 
@@ -249,6 +252,20 @@ int oracle_bvecmat(const void* A, const void* B, void* C, double* c64, double* s
         if (scale64) scale64[r] = t;
         if (C) store(C, r, dt, s);
     });
+    return 0;
+}
+
+// Residual add of a fused add-and-normalise:  h_i = x_i + r_i in double (exact for every pair of
+// fp32 or bf16 inputs whose exponents differ by less than 29), rounded once to the storage type.
+// Reading: the statistics and the output of the norm that follows are computed from this ROUNDED h,
+// i.e. the fused op equals the two ops called one after the other.
+int oracle_add(const void* x, const void* r, void* h, double* h64, int64_t n, int dt) {
+    if (n < 0 || (dt != F32 && dt != BF16) || (n > 0 && (!x || !r))) return -1;
+    for (int64_t i = 0; i < n; ++i) {
+        const double v = load(x, i, dt) + load(r, i, dt);
+        if (h64) h64[i] = v;
+        if (h) store(h, i, dt, v);
+    }
     return 0;
 }
 

@@ -342,3 +342,54 @@ def test_bf16_rounds_directly_from_double():
     v = 1.0 + 2.0 ** -8 + 2.0 ** -30
     assert oracle.bf16_from_double(np.array([v]))[0] == 0x3F81
     assert np.float32(v) == np.float32(1.0 + 2.0 ** -8)
+
+
+# ------------------------------------------------------------------ residual add of the fused add-and-normalise
+
+def test_add_exact_cases_ties_and_library():
+    x = f32([1.0, 2.5, -3.0, 1e30, 0.0, -0.0, 16777216.0, 1.0])
+    r = f32([2.0, 0.25, 3.0, 1e30, 0.0, -0.0, 1.0, 2.0 ** -30])
+    h, h64 = oracle.add(x, r, F32, want64=True)
+    np.testing.assert_array_equal(h64[:4], [3.0, 2.75, 0.0, 2.0 * float(np.float32(1e30))])
+    assert not np.signbit(h[2])                                  # x + (-x) = +0 in round-to-nearest
+    assert np.signbit(h[5]) and not np.signbit(h[4])             # (-0) + (-0) = -0, (+0) + (+0) = +0
+    assert h[6] == np.float32(16777216.0)                        # 2^24 + 1 is a tie in fp32: goes to the even 2^24
+    assert h[7] == np.float32(1.0)
+    np.testing.assert_array_equal(oracle.add(r, x, F32), h)      # commutative
+    np.testing.assert_array_equal(oracle.add(x, ZEROS(8), F32)[[0, 1, 2, 3, 6, 7]], x[[0, 1, 2, 3, 6, 7]])
+    # bf16: ties to even at 1 + 2^-8 (down to 1) and 1 + 2^-7 + 2^-8 (up to 1 + 2^-6); a sum that needs more than 8 bits
+    xb = bf([1.0, 1.0 + 2.0 ** -7, 256.0, 3.0])
+    rb = bf([2.0 ** -8, 2.0 ** -8, 1.0, -3.0])
+    hb, hb64 = oracle.add(xb, rb, BF16, want64=True)
+    np.testing.assert_array_equal(hb64, [1.0 + 2.0 ** -8, 1.0 + 2.0 ** -7 + 2.0 ** -8, 257.0, 0.0])
+    np.testing.assert_array_equal(oracle.bf16_to_double(hb), [1.0, 1.0 + 2.0 ** -6, 256.0, 0.0])
+    # against torch's CPU add on random finite inputs, both types (an independent library route), and the bf16 codec
+    rng = np.random.default_rng(21)
+    a = rng.standard_normal(200_000) * np.exp(rng.uniform(-20, 20, 200_000))
+    b = rng.standard_normal(200_000) * np.exp(rng.uniform(-20, 20, 200_000))
+    np.testing.assert_array_equal(oracle.add(f32(a), f32(b), F32), (torch.from_numpy(f32(a)) + torch.from_numpy(f32(b))).numpy())
+    ab, bb = bf(a), bf(b)
+    tb = (torch.from_numpy(ab).view(torch.bfloat16) + torch.from_numpy(bb).view(torch.bfloat16)).view(torch.uint16).numpy()
+    got, got64 = oracle.add(ab, bb, BF16, want64=True)
+    np.testing.assert_array_equal(got, tb)
+    np.testing.assert_array_equal(got, oracle.bf16_from_double(oracle.bf16_to_double(ab) + oracle.bf16_to_double(bb)))
+    np.testing.assert_array_equal(got64, oracle.bf16_to_double(ab) + oracle.bf16_to_double(bb))
+
+
+def test_add_then_norm_is_the_composition():
+    rng = np.random.default_rng(22)
+    for dt, enc in ((F32, f32), (BF16, bf)):
+        x, r = enc(rng.standard_normal((5, 96)) * 3), enc(rng.standard_normal((5, 96)))
+        g, b = enc(rng.uniform(0.5, 1.5, 96)), enc(rng.standard_normal(96) * 0.1)
+        h, y, mean, rstd = oracle.add_layernorm(x, r, g, b, 1e-5, dt)
+        np.testing.assert_array_equal(h, oracle.add(x, r, dt))
+        y2, mean2, rstd2 = oracle.layernorm(h, g, b, 1e-5, dt)
+        np.testing.assert_array_equal(y, y2), np.testing.assert_array_equal(mean, mean2), np.testing.assert_array_equal(rstd, rstd2)
+        h, y, rs = oracle.add_rmsnorm(x, r, g, 1e-6, dt)
+        y2, rs2 = oracle.rmsnorm(oracle.add(x, r, dt), g, 1e-6, dt)
+        np.testing.assert_array_equal(y, y2), np.testing.assert_array_equal(rs, rs2)
+        # the statistics come from the ROUNDED h: feeding the unrounded sum would change mean in the last bits for bf16
+        if dt == BF16:
+            exact = oracle.bf16_to_double(x) + oracle.bf16_to_double(r)
+            assert np.abs(mean.astype(np.float64) - oracle.bf16_to_double(h).mean(axis=1)).max() < 1e-6
+            assert np.abs(oracle.bf16_to_double(h) - exact).max() > 0          # rounding did happen
