@@ -505,6 +505,74 @@ def run_vecmat_table(args):
     (out_dir / "table_vecmat.json").write_text(json.dumps(rows_out, indent=1))
 
 
+def run_addnorm_table(args):
+    """Fused residual add + norm against the same work as two calls (torch add into h, then the unfused op)."""
+    import torch
+    import paper_2512_09196_b200 as tf
+    from paper_2512_09196_b200 import inputs
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak()
+    out_dir = ROOT / "gpurun_out"
+    out_dir.mkdir(exist_ok=True)
+    shapes = [("rmsnorm", inputs.BF16, 16384, 4096), ("rmsnorm", inputs.BF16, 16384, 8192), ("rmsnorm", inputs.BF16, 4096, 16384),
+              ("rmsnorm", inputs.F32, 8192, 8192), ("layernorm", inputs.BF16, 16384, 4096), ("layernorm", inputs.BF16, 65536, 1024),
+              ("layernorm", inputs.F32, 16384, 4096), ("rmsnorm", inputs.BF16, 256, 8192)]
+    rows_out = []
+    for op, dt, rows, cols in shapes:
+        w = inputs.Workload(f"add_{op}_{'f32' if dt == inputs.F32 else 'bf16'}_{rows}x{cols}", op, dt, rows, cols, seed=cols,
+                            eps=1e-5 if op == "layernorm" else 1e-6)
+        data = w.generate()
+        conv = (lambda t: t.view(torch.bfloat16)) if dt == inputs.BF16 else (lambda t: t)
+        es = w.elem_size
+        sets = max(2, min(16, int((1 << 30) // (4 * rows * cols * es)) + 1))         # rotate so that no launch finds its lines in L2
+        xs = [conv(torch.from_numpy(data["x"])).cuda() for _ in range(sets)]
+        rs = [conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols + 1, 7, 0.0, 1.0))).cuda() for _ in range(sets)]
+        hs = [torch.empty_like(xs[0]) for _ in range(sets)]
+        ys = [torch.empty_like(xs[0]) for _ in range(sets)]
+        g = conv(torch.from_numpy(data["gamma"] if op == "layernorm" else data["w"])).cuda()
+        b = conv(torch.from_numpy(data["beta"])).cuda() if op == "layernorm" else None
+        tf.tf_tune(op, rows, cols, dt, like=(xs[0], g, b))
+        tuned = tf.tf_tune_add(op, rows, cols, dt)
+
+        def fused(k):
+            if op == "layernorm":
+                tf.tf_add_layernorm_fwd(xs[k], rs[k], g, b, w.eps, h=hs[k], y=ys[k], want_stats=False)
+            else:
+                tf.tf_add_rmsnorm_fwd(xs[k], rs[k], g, w.eps, h=hs[k], y=ys[k])
+
+        def unfused(k):
+            torch.add(xs[k], rs[k], out=hs[k])
+            if op == "layernorm":
+                tf.tf_layernorm_fwd(hs[k], g, b, w.eps, y=ys[k], want_stats=False)
+            else:
+                tf.tf_rmsnorm_fwd(hs[k], g, w.eps, y=ys[k])
+
+        def timed(fn, reps):
+            for k in range(5):
+                fn(k % sets)
+            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for k in range(reps):
+                fn(k % sets)
+            e.record()
+            torch.cuda.synchronize()
+            return 1e3 * a.elapsed_time(e) / reps
+
+        nbytes = 4 * rows * cols * es + (2 if op == "layernorm" else 1) * cols * es
+        reps = max(20, min(400, int(0.05 / (nbytes / 5e12))))
+        us_f, us_u = timed(fused, reps), timed(unfused, reps)
+        tf.tf_device_status()
+        row = {"workload": w.name, "op": op, "dtype": w.dtype_name, "rows": rows, "cols": cols, "bytes": nbytes, "us": us_f,
+               "gbs": nbytes / us_f / 1e3, f"pct_of_{peak_kind}_{peak:.0f}": 100 * nbytes / us_f / 1e3 / peak,
+               "unfused_us": us_u, "speedup_vs_two_calls": us_u / us_f, "tune": tuned, "base_plan": tf.tf_query_choice(op, rows, cols, dt)}
+        rows_out.append(row)
+        print(json.dumps(row), flush=True)
+        del xs, rs, hs, ys
+        torch.cuda.empty_cache()
+    (out_dir / "table_addnorm.json").write_text(json.dumps(rows_out, indent=1))
+
+
 def run_case(args):
     """A few launches of one op/shape (for profiler captures): --case op:dtype:rows:cols or --case config:<i>[:rows]."""
     import torch
@@ -562,7 +630,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--table", choices=["configs", "sweep", "vecmat"], default=None)
+    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm"], default=None)
     ap.add_argument("--filter", default=None)
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
@@ -581,6 +649,8 @@ def main():
         return run_case(args)
     if args.table == "vecmat":
         return run_vecmat_table(args)
+    if args.table == "addnorm":
+        return run_addnorm_table(args)
     if args.table:
         return run_table(args)
     run_ours(args)

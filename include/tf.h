@@ -120,6 +120,25 @@ tf_status tf_copy(const void* x, void* y, int64_t bytes, void* cuda_stream);
  * fp32 arithmetic with full range reduction, one rounding to the storage type.  y == x is allowed. */
 tf_status tf_sin_fwd(const void* x, void* y, int64_t n, tf_dtype dt, int threads, int vectors_per_thread, void* cuda_stream);
 
+/* ---- fused residual add + norm ------------------------------------------------------------------------ */
+
+/* h = x + r (fp32 add, ONE rounding to the storage type), then the LayerNorm / RMSNorm defined above applied to that
+ * rounded h: bit for bit the result of an add followed by tf_layernorm_fwd / tf_rmsnorm_fwd, with x and r read once
+ * and h and y written once.  The paper names fused operators as a class of its targets (Section 2) and defines none;
+ * this is the residual-stream update of pre-norm transformer blocks.
+ * x, r, h, y: [rows, cols] row-major, device memory, one element type; h may alias x or r, y may alias x; h and y must
+ * not overlap each other.  gamma / beta / weight, mean / rstd, eps, errors and stream behaviour as for the unfused
+ * calls, plus TF_ERR_INVALID_ARG for a null r or h.  Rows of up to 512 KiB on 16-byte aligned tensors run as one
+ * kernel; anything else as an element-wise add followed by the unfused op (same results).  Allocates nothing. */
+tf_status tf_add_layernorm_fwd(const void* x, const void* r, const void* gamma, const void* beta, void* h, void* y, float* mean,
+                               float* rstd, int64_t rows, int64_t cols, float eps, tf_dtype dt, void* cuda_stream);
+tf_status tf_add_rmsnorm_fwd(const void* x, const void* r, const void* weight, void* h, void* y, float* rstd, int64_t rows,
+                             int64_t cols, float eps, tf_dtype dt, void* cuda_stream);
+/* tf_tune for the fused form of TF_OP_LAYERNORM / TF_OP_RMSNORM: measures the register-resident plans on synthetic
+ * data and caches the fastest under its own key.  TF_ERR_UNSUPPORTED when no such plan holds the row (the two-kernel
+ * route is then used, and there is nothing to choose); TF_ERR_INVALID_ARG for TF_OP_SOFTMAX.  Blocking. */
+tf_status tf_tune_add(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);
+
 /* ---- second memory-bound workload -------------------------------------------------------------------- */
 
 /* Batched vector-matrix product (the paper's Case Study 2, "GEMV restructuring"):

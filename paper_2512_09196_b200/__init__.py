@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_status_string",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
 
@@ -53,6 +53,9 @@ def lib() -> ctypes.CDLL:
         L.tf_rmsnorm_fwd.argtypes = [vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_tune.argtypes = [i32, i64, i64, i32]
         L.tf_copy.argtypes = [vp, vp, i64, vp]
+        L.tf_add_layernorm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, vp]
+        L.tf_add_rmsnorm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, vp]
+        L.tf_tune_add.argtypes = [i32, i64, i64, i32]
         L.tf_bvecmat_fwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp]
         L.tf_sin_fwd.argtypes = [vp, vp, i64, i32, i32, i32, vp]
         L.tf_tune_like.argtypes = [i32, vp, vp, vp, i64, i64, i32]
@@ -69,7 +72,7 @@ def lib() -> ctypes.CDLL:
         L.tf_clear_cache.restype = None
         L.tf_launch_count.argtypes = []
         L.tf_launch_count.restype = i64
-        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd",
+        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add",
                      "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice",
                      "tf_candidate_count", "tf_candidate"):
             getattr(L, name).restype = i32
@@ -211,6 +214,45 @@ def tf_layernorm_fwd(x, gamma, beta, eps: float, y=None, mean=None, rstd=None, w
     return y, mean, rstd
 
 
+def tf_add_layernorm_fwd(x, r, gamma, beta, eps: float, h=None, y=None, want_stats: bool = True):
+    """Fused residual add + LayerNorm: ``h = x + r`` (rounded to the storage type), ``y = layernorm(h)``.
+    Returns ``(h, y, mean, rstd)``; pass ``h=r`` to update the residual stream in place."""
+    import torch
+    _check2d(x)
+    _check2d(r, "r")
+    rows, cols = x.shape
+    if r.shape != x.shape or r.dtype != x.dtype:
+        raise ValueError("r must match x")
+    h = torch.empty_like(x) if h is None else h
+    y = torch.empty_like(x) if y is None else y
+    mean = torch.empty(rows, dtype=torch.float32, device=x.device) if want_stats else None
+    rstd = torch.empty(rows, dtype=torch.float32, device=x.device) if want_stats else None
+    with _on_device(x):
+        _ok(lib().tf_add_layernorm_fwd(x.data_ptr(), r.data_ptr(), gamma.data_ptr(), beta.data_ptr(), h.data_ptr(), y.data_ptr(),
+                                       mean.data_ptr() if want_stats else None, rstd.data_ptr() if want_stats else None,
+                                       rows, cols, eps, _dt(x), _stream(x)), "tf_add_layernorm_fwd")
+    return h, y, mean, rstd
+
+
+def tf_add_rmsnorm_fwd(x, r, weight, eps: float, h=None, y=None, want_rstd: bool = False):
+    """Fused residual add + RMSNorm: ``h = x + r`` (rounded to the storage type), ``y = rmsnorm(h)``.
+    Returns ``(h, y, rstd)``; pass ``h=r`` to update the residual stream in place."""
+    import torch
+    _check2d(x)
+    _check2d(r, "r")
+    rows, cols = x.shape
+    if r.shape != x.shape or r.dtype != x.dtype:
+        raise ValueError("r must match x")
+    h = torch.empty_like(x) if h is None else h
+    y = torch.empty_like(x) if y is None else y
+    rstd = torch.empty(rows, dtype=torch.float32, device=x.device) if want_rstd else None
+    with _on_device(x):
+        _ok(lib().tf_add_rmsnorm_fwd(x.data_ptr(), r.data_ptr(), weight.data_ptr(), h.data_ptr(), y.data_ptr(),
+                                     rstd.data_ptr() if want_rstd else None, rows, cols, eps, _dt(x), _stream(x)),
+            "tf_add_rmsnorm_fwd")
+    return h, y, rstd
+
+
 def tf_rmsnorm_fwd(x, weight, eps: float, y=None, rstd=None, want_rstd: bool = False):
     """RMSNorm forward; returns ``(y, rstd)`` (``rstd`` is None unless requested or passed in)."""
     import torch
@@ -241,6 +283,17 @@ def tf_tune(op, rows: int, cols: int, dt: int, like=None) -> dict:
     n, a, b = ctypes.c_int(), ctypes.c_float(), ctypes.c_float()
     lib().tf_tune_report(ctypes.byref(n), ctypes.byref(a), ctypes.byref(b))
     return {"timed": n.value, "heuristic_us": a.value, "best_us": b.value, "plan": tf_query_choice(code, rows, cols, dt)}
+
+
+def tf_tune_add(op, rows: int, cols: int, dt: int) -> dict:
+    """``tf_tune`` for the fused residual-add form of LayerNorm / RMSNorm (own cache entry).  Returns
+    ``{"timed": n, "heuristic_us": a, "best_us": b}``; raises TfError(TF_ERR_UNSUPPORTED) when only the two-kernel route
+    can serve the shape."""
+    code = OP_CODE[op] if isinstance(op, str) else int(op)
+    _ok(lib().tf_tune_add(code, rows, cols, dt), "tf_tune_add")
+    n, a, b = ctypes.c_int(), ctypes.c_float(), ctypes.c_float()
+    lib().tf_tune_report(ctypes.byref(n), ctypes.byref(a), ctypes.byref(b))
+    return {"timed": n.value, "heuristic_us": a.value, "best_us": b.value}
 
 
 def tf_force_plan(op, plan: str | None):

@@ -35,6 +35,7 @@ bool g_forced[OP_COUNT] = {false, false, false};
 Plan g_forced_plan[OP_COUNT];
 using Key = std::tuple<int, int, int, int64_t, int64_t>;      // device, op, dt, rows, cols
 std::map<Key, Plan> g_cache;
+constexpr int kAddKey = 16;              // cache key of a fused residual-add op = kAddKey + the op
 bool g_cache_file_loaded = false;
 
 tf_status cuda_fail(cudaError_t e) {
@@ -426,7 +427,7 @@ void load_cache_file_locked() {
         int dev, op, dt; long long rows, cols; char plan[256];
         if (sscanf(line, "%d %d %d %lld %lld %255s", &dev, &op, &dt, &rows, &cols, plan) != 6) continue;
         Plan p;
-        if (op < 0 || op >= OP_COUNT || (dt != DT_F32 && dt != DT_BF16) || !plan_from_string(plan, p)) continue;
+        if (op < 0 || (op >= OP_COUNT && (op < kAddKey + OP_LAYERNORM || op > kAddKey + OP_RMSNORM)) || (dt != DT_F32 && dt != DT_BF16) || !plan_from_string(plan, p)) continue;
         g_cache[Key(dev, op, dt, rows, cols)] = p;
     }
     fclose(f);
@@ -468,6 +469,35 @@ tf_status run(const Args& a0, void* stream) {
     if (!supports(p, a, ds->info)) return TF_ERR_UNSUPPORTED;
     cudaError_t e = launch(p, a, ds->info, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? TF_OK : cuda_fail(e);
+}
+
+// Fused residual add + norm.  A forced or tuned plan of the base op is reused when it is a register-resident one;
+// otherwise the register heuristic; otherwise an element-wise add followed by the ordinary op on h.
+tf_status run_add(const Args& a0, void* stream) {
+    if (a0.rows == 0) return TF_OK;
+    DevState* ds = nullptr;
+    tf_status s = device_state(&ds);
+    if (s != TF_OK) return s;
+    Args a = a0;
+    a.status = ds->status;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    bool forced = false;
+    Plan p = choose(a, ds->info, &forced);
+    if (!forced) {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_cache.find(Key(ds->info.ordinal, kAddKey + a.op, a.dt, a.rows, a.cols));
+        if (it != g_cache.end()) p = it->second;
+    }
+    if (!supports_addnorm(p, a, ds->info)) p = heuristic_addnorm(a, ds->info);
+    if (p.variant >= 0 && supports_addnorm(p, a, ds->info)) {
+        cudaError_t e = launch_addnorm(p, a, ds->info, st);
+        return e == cudaSuccess ? TF_OK : cuda_fail(e);
+    }
+    cudaError_t e = launch_add_elementwise(a.x, a.r, a.h, a.rows * a.cols, a.dt, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    Args b = a0;
+    b.x = a0.h; b.r = nullptr; b.h = nullptr;
+    return run(b, stream);
 }
 
 bool bad_shape(int64_t rows, int64_t cols, int dt) {  // dt arrives as an int so that out-of-range enum values are caught
@@ -551,9 +581,27 @@ tf_status tf_rmsnorm_fwd(const void* x, const void* weight, void* y, float* rstd
     return run(a, stream);
 }
 
+tf_status tf_add_layernorm_fwd(const void* x, const void* r, const void* gamma, const void* beta, void* h, void* y, float* mean,
+                               float* rstd, int64_t rows, int64_t cols, float eps, tf_dtype dt, void* stream) {
+    if (bad_shape(rows, cols, dt) || bad_eps(eps) || !gamma || !beta || (rows > 0 && (!x || !r || !h || !y))) return TF_ERR_INVALID_ARG;
+    if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
+    Args a{OP_LAYERNORM, dt, x, gamma, beta, y, mean, rstd, rows, cols, eps, nullptr, r, h};
+    return run_add(a, stream);
+}
+
+tf_status tf_add_rmsnorm_fwd(const void* x, const void* r, const void* weight, void* h, void* y, float* rstd, int64_t rows,
+                             int64_t cols, float eps, tf_dtype dt, void* stream) {
+    if (bad_shape(rows, cols, dt) || bad_eps(eps) || !weight || (rows > 0 && (!x || !r || !h || !y))) return TF_ERR_INVALID_ARG;
+    if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
+    Args a{OP_RMSNORM, dt, x, weight, nullptr, y, nullptr, rstd, rows, cols, eps, nullptr, r, h};
+    return run_add(a, stream);
+}
+
 // x_like / p0_like / p1_like: device tensors whose contents the timing input is copied from (NULL: synthetic).
-static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const void* x_like, const void* p0_like, const void* p1_like) {
-    if (op < 0 || op >= OP_COUNT || bad_shape(rows, cols, dt) || rows == 0) return TF_ERR_INVALID_ARG;
+// add: tune the fused residual-add form of the op (register-resident plans only) with its own cache entry.
+static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const void* x_like, const void* p0_like, const void* p1_like,
+                           bool add = false) {
+    if (op < 0 || op >= OP_COUNT || bad_shape(rows, cols, dt) || rows == 0 || (add && op == OP_SOFTMAX)) return TF_ERR_INVALID_ARG;
     if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
     DevState* ds = nullptr;
     tf_status s = device_state(&ds);
@@ -566,8 +614,10 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
     const int K = static_cast<int>(std::min<size_t>(64, std::max<size_t>(1, (want + 2 * tensor_bytes - 1) / (2 * tensor_bytes))));
 
     Scratch sc;
-    std::vector<void*> xs(K), ys(K);
+    std::vector<void*> xs(K), ys(K), rs(K, nullptr), hs(K, nullptr);
     for (int k = 0; k < K; ++k) { xs[k] = sc.get(tensor_bytes); ys[k] = sc.get(tensor_bytes); if (!xs[k] || !ys[k]) return TF_ERR_NOMEM; }
+    if (add)
+        for (int k = 0; k < K; ++k) { rs[k] = sc.get(tensor_bytes); hs[k] = sc.get(tensor_bytes); if (!rs[k] || !hs[k]) return TF_ERR_NOMEM; }
     void* yref = sc.get(tensor_bytes);
     void* p0 = sc.get(static_cast<size_t>(cols) * es);
     void* p1 = sc.get(static_cast<size_t>(cols) * es);
@@ -589,6 +639,10 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
         if (x_like) cudaMemcpyAsync(xs[k], x_like, tensor_bytes, cudaMemcpyDeviceToDevice, st);
         else if (dt == DT_F32) k_fill<DT_F32><<<fill_grid, 256, 0, st>>>(xs[k], n, -4.f, 4.f, 1000003ull * k);
         else k_fill<DT_BF16><<<fill_grid, 256, 0, st>>>(xs[k], n, -4.f, 4.f, 1000003ull * k);
+        if (add) {
+            if (dt == DT_F32) k_fill<DT_F32><<<fill_grid, 256, 0, st>>>(rs[k], n, -1.f, 1.f, 7000003ull * k + 5);
+            else k_fill<DT_BF16><<<fill_grid, 256, 0, st>>>(rs[k], n, -1.f, 1.f, 7000003ull * k + 5);
+        }
     }
     const int pgrid = static_cast<int>(std::min<int64_t>((cols + 255) / 256, 1024));
     if (dt == DT_F32) { k_fill<DT_F32><<<pgrid, 256, 0, st>>>(p0, cols, 0.5f, 1.5f, 7); k_fill<DT_F32><<<pgrid, 256, 0, st>>>(p1, cols, -0.5f, 0.5f, 11); }
@@ -600,12 +654,15 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
     auto args_for = [&](int k, void* y) {
         Args a{op, dt, xs[k], p0, p1, y, op == OP_LAYERNORM ? mean : nullptr, op == OP_LAYERNORM ? rstd : nullptr,
                rows, cols, op == OP_SOFTMAX ? 0.f : 1e-5f, ds->status};
+        if (add) { a.r = rs[k]; a.h = hs[k]; }
         return a;
     };
+    auto supports_it = [&](const Plan& p, const Args& a) { return add ? supports_addnorm(p, a, dev) : supports(p, a, dev); };
+    auto launch_it = [&](const Plan& p, const Args& a) { return add ? launch_addnorm(p, a, dev, st) : launch(p, a, dev, st); };
     // BuildRun: can it launch, and does it reproduce the incumbent's output?
     auto runs_and_matches = [&](const Plan& p, bool is_reference) -> bool {
         void* y = is_reference ? yref : ys[0];
-        if (launch(p, args_for(0, y), dev, st) != cudaSuccess) { cudaGetLastError(); return false; }
+        if (launch_it(p, args_for(0, y)) != cudaSuccess) { cudaGetLastError(); return false; }
         if (cudaStreamSynchronize(st) != cudaSuccess) return false;
         int flag = 0;                                        // a bounded wait gave up: the candidate is dropped
         if (cudaMemcpy(&flag, ds->status, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) return false;
@@ -625,7 +682,7 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
         for (int rep = 0; rep < 8; ++rep) {
             if (rep >= 3) cudaEventRecord(ev[0], st);
             for (int k = 0; k < K; ++k)
-                if (launch(p, args_for(k, ys[k]), dev, st) != cudaSuccess) { cudaGetLastError(); return false; }
+                if (launch_it(p, args_for(k, ys[k])) != cudaSuccess) { cudaGetLastError(); return false; }
             if (rep >= 3) {
                 cudaEventRecord(ev[1], st);
                 if (cudaEventSynchronize(ev[1]) != cudaSuccess) return false;
@@ -640,10 +697,11 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
     };
 
     const Args probe = args_for(0, ys[0]);
-    Plan best = heuristic(probe, dev);
+    Plan best = add ? heuristic_addnorm(probe, dev) : heuristic(probe, dev);
     float best_us = 0.f;
     int timed = 0;
-    if (!supports(best, probe, dev) || !runs_and_matches(best, true) || !profile(best, &best_us)) { cleanup(); return cuda_fail(cudaGetLastError()); }
+    if (add && best.variant < 0) { cleanup(); return TF_ERR_UNSUPPORTED; }            // no register-resident plan holds this row
+    if (!supports_it(best, probe) || !runs_and_matches(best, true) || !profile(best, &best_us)) { cleanup(); return cuda_fail(cudaGetLastError()); }
     ++timed;
     const float heur_us = best_us;
     const std::string best0 = plan_to_string(best);
@@ -657,7 +715,7 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
         if (std::find(seen.begin(), seen.end(), name) != seen.end()) return false;
         seen.push_back(name);
         float us = 0.f;
-        if (!supports(c, probe, dev) || !runs_and_matches(c, false)) return false;   // failed BuildRun: dropped, never cached
+        if (!supports_it(c, probe) || !runs_and_matches(c, false)) return false;   // failed BuildRun: dropped, never cached
         if (!profile(c, &us)) return false;
         ++timed;
         if (log) fprintf(stderr, "tf_tune: %8.2f us  %s\n", us, name.c_str());
@@ -679,7 +737,7 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
     {
         std::lock_guard<std::mutex> lk(g_mu);
         load_cache_file_locked();
-        g_cache[Key(dev.ordinal, op, dt, rows, cols)] = best;
+        g_cache[Key(dev.ordinal, (add ? kAddKey : 0) + op, dt, rows, cols)] = best;
         save_cache_file_locked();
     }
     return TF_OK;
@@ -692,6 +750,10 @@ tf_status tf_tune(tf_op op, int64_t rows, int64_t cols, tf_dtype dt) {
 tf_status tf_tune_like(tf_op op, const void* x, const void* p0, const void* p1, int64_t rows, int64_t cols, tf_dtype dt) {
     if (!x) return TF_ERR_INVALID_ARG;
     return tune_impl(op, rows, cols, dt, x, p0, p1);
+}
+
+tf_status tf_tune_add(tf_op op, int64_t rows, int64_t cols, tf_dtype dt) {
+    return tune_impl(op, rows, cols, dt, nullptr, nullptr, nullptr, true);
 }
 
 tf_status tf_tune_report(int* candidates_timed, float* heuristic_us, float* best_us) {

@@ -44,6 +44,8 @@ struct Args {
     int64_t rows, cols;
     float eps;
     int* status;         // device word that bounded waits set when they give up
+    const void* r = nullptr;   // fused residual add: second input ...
+    void* h = nullptr;         // ... and where x + r (rounded to the storage type) goes
 };
 
 struct DeviceInfo {
@@ -79,6 +81,13 @@ cudaError_t launch_twopass(const Plan&, const Args&, const DeviceInfo&, cudaStre
 cudaError_t launch_split(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 // The split plan with caller-provided scratch (split_scratch_bytes() of device memory).
 cudaError_t launch_split_with_scratch(const Plan&, const Args&, void* scratch, cudaStream_t);
+
+// Fused residual add + norm (Args::r, Args::h set): register-resident plans only; heuristic_addnorm returns variant -1
+// when none holds the row, and the caller then adds element-wise and runs the ordinary norm on h.
+bool supports_addnorm(const Plan&, const Args&, const DeviceInfo&);
+cudaError_t launch_addnorm(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+Plan heuristic_addnorm(const Args&, const DeviceInfo&);
+cudaError_t launch_add_elementwise(const void* x, const void* r, void* h, int64_t n, int dt, cudaStream_t);
 size_t split_scratch_bytes(const Plan&, const Args&);
 
 // Bookkeeping shared with the C ABI layer: count kernel launches; remember the CUDA error behind a TF_ERR_CUDA.

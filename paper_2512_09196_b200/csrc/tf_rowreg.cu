@@ -8,264 +8,52 @@
 //   V_CTA   a CTA of `threads` threads owns a row (vpt vectors per thread); with cluster > 1 the row is split
 //           over the CTAs of a thread-block cluster and the per-slice partials (max,sum | mean,M2 | sumsq) are
 //           exchanged through distributed shared memory with one cluster barrier per row.
-#include <cooperative_groups.h>
-
-#include <algorithm>
-
-#include "tf_rowmath.cuh"
-
-namespace cg = cooperative_groups;
+#include "tf_rowreg.cuh"
 
 namespace tf {
 namespace {
 
-struct KArgs {
-    const uint4* x;
-    const uint4* p0;
-    const uint4* p1;
-    uint4* y;
-    float* mean;
-    float* rstd;
-    int64_t rows;
-    int nvec;        // 16-byte vectors per row
-    float n;         // cols as float
-    float eps;
-};
-
-// Largest CTA each kernel is compiled for (bounds the registers a thread may use).
-constexpr int kWarpMaxThreads = 256;
-constexpr int cta_max_threads(int vpt) { return vpt <= 2 ? 1024 : 512; }
-
-// =====================================================================================================
-// V_WARP
-// =====================================================================================================
-template <int OP, int DT, int LANES, int VPT, int RPG>
-__global__ void __launch_bounds__(kWarpMaxThreads) k_warp(const KArgs a) {
-    pdl_wait();
-    pdl_trigger();
-    const int lane = threadIdx.x % LANES;
-    const int gpc = blockDim.x / LANES;                                   // groups per CTA
-    const int64_t g = static_cast<int64_t>(blockIdx.x) * gpc + threadIdx.x / LANES;
-    const int64_t G = static_cast<int64_t>(gridDim.x) * gpc;
-
-    bool valid[VPT];
-    HeldParams<VPT> par;
-#pragma unroll
-    for (int v = 0; v < VPT; ++v) {
-        const int idx = lane + v * LANES;
-        valid[v] = idx < a.nvec;
-        par.g[v] = make_uint4(0, 0, 0, 0); par.b[v] = make_uint4(0, 0, 0, 0);
-        if (OP != OP_SOFTMAX && valid[v]) par.g[v] = ld_param(a.p0 + idx);
-        if (OP == OP_LAYERNORM && valid[v]) par.b[v] = ld_param(a.p1 + idx);
-    }
-    const GroupRed<LANES> red;
-    const uint4 fill = fill_vec<DT>(OP);
-
-    for (int64_t base = 0; base < a.rows; base += G * RPG) {
-        uint4 raw[RPG][VPT];
-#pragma unroll
-        for (int rr = 0; rr < RPG; ++rr) {
-            const int64_t row = base + rr * G + g;                          // adjacent groups -> adjacent rows
-#pragma unroll
-            for (int v = 0; v < VPT; ++v)
-                raw[rr][v] = (row < a.rows && valid[v]) ? ld_stream(a.x + row * a.nvec + lane + v * LANES) : fill;
-        }
-#pragma unroll
-        for (int rr = 0; rr < RPG; ++rr) {
-            const int64_t row = base + rr * G + g;
-            uint4 out[VPT];
-            float st0 = 0.f, st1 = 0.f;
-            row_math<OP, DT, VPT>(raw[rr], valid, red, par, 0, a.n, a.eps, out, st0, st1);
-            if (row < a.rows) {
-#pragma unroll
-                for (int v = 0; v < VPT; ++v)
-                    if (valid[v]) st_stream(a.y + row * a.nvec + lane + v * LANES, out[v]);
-                if (lane == 0) {
-                    if (OP == OP_LAYERNORM && a.mean) a.mean[row] = st0;
-                    if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = st1;
-                }
-            }
-        }
-    }
-}
-
-// =====================================================================================================
-// V_CTA (optionally split over a cluster)
-// =====================================================================================================
-template <int OP, int DT, int VPT, bool CLUSTER>
-__global__ void __launch_bounds__(cta_max_threads(VPT)) k_cta(const KArgs a, const int cs) {
-    using E = Elem<DT>;
-    constexpr int NE = E::NE;
-    __shared__ float red_buf[4 * 32];
-    __shared__ float xch[2][kMaxCluster][2];          // partials pushed by the peers, double-buffered by row parity
-
-    pdl_wait();
-    pdl_trigger();
-    const int T = blockDim.x, t = threadIdx.x;
-    const int rank = CLUSTER ? static_cast<int>(blockIdx.x % cs) : 0;
-    const int64_t cluster_id = CLUSTER ? blockIdx.x / cs : blockIdx.x;
-    const int64_t num_clusters = CLUSTER ? gridDim.x / cs : gridDim.x;
-    const int per = CLUSTER ? (a.nvec + cs - 1) / cs : a.nvec;         // vectors per slice
-    const int first = rank * per;
-    const int len = max(0, min(per, a.nvec - first));                   // this CTA's slice length
-
-    bool valid[VPT];
-#pragma unroll
-    for (int v = 0; v < VPT; ++v) valid[v] = (t + v * T) < len;
-    const CtaRed red{red_buf};
-    const LazyParams par{a.p0, a.p1, first + t, T};
-    const uint4 fill = fill_vec<DT>(OP);
-
-    if constexpr (CLUSTER) cg::this_cluster().sync();      // every CTA of the cluster is resident before any remote write
-
-    int it = 0;
-    for (int64_t row = cluster_id; row < a.rows; row += num_clusters, ++it) {
-        const uint4* xr = a.x + row * a.nvec + first + t;
-        uint4* yr = a.y + row * a.nvec + first + t;
-        uint4 raw[VPT], out[VPT];
-#pragma unroll
-        for (int v = 0; v < VPT; ++v) raw[v] = valid[v] ? ld_stream(xr + v * T) : fill;
-        float st0 = 0.f, st1 = 0.f;
-        const int slot0 = (it & 1) * 2;
-
-        if constexpr (!CLUSTER) {
-            row_math<OP, DT, VPT>(raw, valid, red, par, slot0, a.n, a.eps, out, st0, st1);
-        } else {
-            cg::cluster_group cl = cg::this_cluster();
-            const int par_buf = it & 1;
-            F2 w[VPT][Pairs<DT>::NP];
-            const Part part = slice_stats<OP, DT, VPT>(raw, valid, red, slot0, static_cast<float>(len) * NE, w);
-            if (t < cs) {                                             // push my partial into every CTA of the cluster
-                float* dst = cl.map_shared_rank(&xch[par_buf][rank][0], t);
-                dst[0] = part.a; dst[1] = part.b;
-            }
-            cl.sync();                                                // release our writes, acquire the peers'
-            const Total tot = combine_parts<OP>(
-                cs, rank, [&](int k) { return Part{xch[par_buf][k][0], xch[par_buf][k][1]}; },
-                [&](int k) { return static_cast<float>(max(0, min(per, a.nvec - k * per))) * NE; }, a.n, a.eps);
-            st0 = tot.a; st1 = tot.b;
-            slice_finish<OP, DT, VPT, false>(valid, w, tot, par, out);
-        }
-#pragma unroll
-        for (int v = 0; v < VPT; ++v)
-            if (valid[v]) st_stream(yr + v * T, out[v]);
-        if (t == 0 && rank == 0) {
-            if (OP == OP_LAYERNORM && a.mean) a.mean[row] = st0;
-            if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = st1;
-        }
-    }
-}
-
-KArgs make_kargs(const Args& a) {
-    KArgs k;
-    k.x = static_cast<const uint4*>(a.x); k.p0 = static_cast<const uint4*>(a.p0); k.p1 = static_cast<const uint4*>(a.p1);
-    k.y = static_cast<uint4*>(a.y); k.mean = a.mean; k.rstd = a.rstd; k.rows = a.rows;
-    k.nvec = static_cast<int>(a.cols * elem_size(a.dt) / 16);
-    k.n = static_cast<float>(a.cols); k.eps = a.eps;
-    return k;
-}
-
-using WarpFn = void (*)(const KArgs);
-using CtaFn = void (*)(const KArgs, const int);
-
-template <int OP, int DT> WarpFn pick_warp(int lanes, int vpt, int rpg) {
-#define TF_W(L, V, R) if (lanes == L && vpt == V && rpg == R) return k_warp<OP, DT, L, V, R>;
-    TF_W(8, 1, 1) TF_W(8, 1, 2) TF_W(8, 1, 4) TF_W(8, 2, 1) TF_W(8, 2, 2)
-    TF_W(16, 1, 1) TF_W(16, 1, 2) TF_W(16, 1, 4) TF_W(16, 2, 1) TF_W(16, 2, 2)
-    TF_W(32, 1, 1) TF_W(32, 1, 2) TF_W(32, 1, 4) TF_W(32, 2, 1) TF_W(32, 2, 2) TF_W(32, 4, 1) TF_W(32, 4, 2) TF_W(32, 8, 1)
-#undef TF_W
-    return nullptr;
-}
-
-template <int OP, int DT> CtaFn pick_cta(int vpt, bool cluster) {
-#define TF_C(V) if (vpt == V) return cluster ? k_cta<OP, DT, V, true> : k_cta<OP, DT, V, false>;
-    TF_C(1) TF_C(2) TF_C(4) TF_C(8)
-#undef TF_C
-    return nullptr;
-}
+using namespace rowreg;
 
 WarpFn warp_fn(int op, int dt, int l, int v, int r) {
     switch (op * 2 + dt) {
-        case 0: return pick_warp<OP_SOFTMAX, DT_F32>(l, v, r);
-        case 1: return pick_warp<OP_SOFTMAX, DT_BF16>(l, v, r);
-        case 2: return pick_warp<OP_LAYERNORM, DT_F32>(l, v, r);
-        case 3: return pick_warp<OP_LAYERNORM, DT_BF16>(l, v, r);
-        case 4: return pick_warp<OP_RMSNORM, DT_F32>(l, v, r);
-        case 5: return pick_warp<OP_RMSNORM, DT_BF16>(l, v, r);
+        case 0: return pick_warp<OP_SOFTMAX, DT_F32, false>(l, v, r);
+        case 1: return pick_warp<OP_SOFTMAX, DT_BF16, false>(l, v, r);
+        case 2: return pick_warp<OP_LAYERNORM, DT_F32, false>(l, v, r);
+        case 3: return pick_warp<OP_LAYERNORM, DT_BF16, false>(l, v, r);
+        case 4: return pick_warp<OP_RMSNORM, DT_F32, false>(l, v, r);
+        case 5: return pick_warp<OP_RMSNORM, DT_BF16, false>(l, v, r);
     }
     return nullptr;
 }
 CtaFn cta_fn(int op, int dt, int v, bool c) {
     switch (op * 2 + dt) {
-        case 0: return pick_cta<OP_SOFTMAX, DT_F32>(v, c);
-        case 1: return pick_cta<OP_SOFTMAX, DT_BF16>(v, c);
-        case 2: return pick_cta<OP_LAYERNORM, DT_F32>(v, c);
-        case 3: return pick_cta<OP_LAYERNORM, DT_BF16>(v, c);
-        case 4: return pick_cta<OP_RMSNORM, DT_F32>(v, c);
-        case 5: return pick_cta<OP_RMSNORM, DT_BF16>(v, c);
+        case 0: return pick_cta<OP_SOFTMAX, DT_F32, false>(v, c);
+        case 1: return pick_cta<OP_SOFTMAX, DT_BF16, false>(v, c);
+        case 2: return pick_cta<OP_LAYERNORM, DT_F32, false>(v, c);
+        case 3: return pick_cta<OP_LAYERNORM, DT_BF16, false>(v, c);
+        case 4: return pick_cta<OP_RMSNORM, DT_F32, false>(v, c);
+        case 5: return pick_cta<OP_RMSNORM, DT_BF16, false>(v, c);
     }
     return nullptr;
 }
 
-bool threads_ok(int t) { return t >= 32 && t <= 1024 && t % 32 == 0; }
-
 }  // namespace
 
 bool supports_warp(const Plan& p, const Args& a, const DeviceInfo&) {
-    if (!vector_ok(a) || !threads_ok(p.threads) || p.threads > kWarpMaxThreads || p.lanes < 1 || p.threads % p.lanes) return false;
-    if (!warp_fn(a.op, a.dt, p.lanes, p.vpt, p.rpg)) return false;
-    const int64_t nvec = a.cols * elem_size(a.dt) / 16;
-    return nvec <= static_cast<int64_t>(p.lanes) * p.vpt;
+    return warp_geometry_ok(p, a) && warp_fn(a.op, a.dt, p.lanes, p.vpt, p.rpg) != nullptr;
 }
 
 cudaError_t launch_warp(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
-    WarpFn fn = warp_fn(a.op, a.dt, p.lanes, p.vpt, p.rpg);
-    if (!fn) return cudaErrorInvalidValue;
-    const int64_t rows_per_cta = static_cast<int64_t>(p.threads / p.lanes) * p.rpg;
-    int64_t grid = (a.rows + rows_per_cta - 1) / rows_per_cta;
-    if (p.persist > 0) grid = std::min<int64_t>(grid, static_cast<int64_t>(p.persist) * d.sms);
-    grid = std::min<int64_t>(grid, 0x7FFFFFFF);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(grid));
-    cfg.blockDim = dim3(p.threads);
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fn, make_kargs(a));
+    return launch_warp_fn(warp_fn(a.op, a.dt, p.lanes, p.vpt, p.rpg), p, a, d, st);
 }
 
 bool supports_cta(const Plan& p, const Args& a, const DeviceInfo& d) {
-    if (!vector_ok(a) || !threads_ok(p.threads)) return false;
-    if (p.cluster < 1 || p.cluster > kMaxCluster || p.cluster > d.max_cluster || (p.cluster & (p.cluster - 1))) return false;
-    if (!cta_fn(a.op, a.dt, p.vpt, p.cluster > 1) || p.threads > cta_max_threads(p.vpt)) return false;
-    const int64_t nvec = a.cols * elem_size(a.dt) / 16;
-    if (nvec > 0x7FFFFFFF) return false;
-    const int64_t per = (nvec + p.cluster - 1) / p.cluster;
-    return per <= static_cast<int64_t>(p.threads) * p.vpt;
+    return cta_geometry_ok(p, a, d) && cta_fn(a.op, a.dt, p.vpt, p.cluster > 1) != nullptr;
 }
 
 cudaError_t launch_cta(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
-    CtaFn fn = cta_fn(a.op, a.dt, p.vpt, p.cluster > 1);
-    if (!fn) return cudaErrorInvalidValue;
-    int64_t clusters = a.rows;
-    if (p.persist > 0) clusters = std::min<int64_t>(clusters, std::max<int64_t>(1, static_cast<int64_t>(p.persist) * d.sms / p.cluster));
-    clusters = std::min<int64_t>(clusters, 0x7FFFFFFF / p.cluster);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(clusters * p.cluster));
-    cfg.blockDim = dim3(p.threads);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = p.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = p.cluster > 1 ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, fn, make_kargs(a), p.cluster);
+    return launch_cta_fn(cta_fn(a.op, a.dt, p.vpt, p.cluster > 1), p, a, d, st);
 }
 
 }  // namespace tf
