@@ -61,6 +61,8 @@ def _load():
         lib.oracle_sin.restype = i32
         lib.oracle_bvecmat.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i32, i32]
         lib.oracle_bvecmat.restype = i32
+        lib.oracle_softmax_len.argtypes = [vp, vp, vp, vp, i64, i64, i32, i32]
+        lib.oracle_softmax_len.restype = i32
         lib.oracle_add.argtypes = [vp, vp, vp, vp, i64, i32]
         lib.oracle_add.restype = i32
         lib.oracle_bf16_from_double.argtypes = [vp, vp, i64]
@@ -90,6 +92,20 @@ def softmax(x: np.ndarray, dt: int, want64: bool = False, nthreads: int = 1):
     rc = _load().oracle_softmax(_p(x), _p(y), _p(y64), rows, cols, dt, nthreads)
     if rc:
         raise ValueError("oracle_softmax: bad argument")
+    return (y, y64) if want64 else y
+
+
+def softmax_len(x: np.ndarray, lengths: np.ndarray, dt: int, want64: bool = False, nthreads: int = 1):
+    """Row softmax over the first ``lengths[r]`` entries of row r; the rest of the output row is +0 and the rest of
+    the input row is not read.  ``lengths``: int32 [rows]."""
+    _check(x, dt, "x")
+    rows, cols = x.shape
+    if lengths.dtype != np.int32 or lengths.shape != (rows,) or not lengths.flags.c_contiguous:
+        raise TypeError("lengths: want C-contiguous int32 [rows]")
+    y = np.empty_like(x)
+    y64 = np.empty((rows, cols), np.float64) if want64 else None
+    if _load().oracle_softmax_len(_p(x), _p(lengths), _p(y), _p(y64), rows, cols, dt, nthreads):
+        raise ValueError("oracle_softmax_len: bad argument")
     return (y, y64) if want64 else y
 
 

@@ -28,6 +28,9 @@
 // linearity, and numpy's float64 einsum.  The residual add that precedes a fused add-and-normalise
 // (h = x + r, rounded once to the storage type; the norm is then the ordinary one applied to h) is
 // pinned by exact small sums, x + 0, x - x, commutativity, bf16 ties to even, and torch's CPU add.
+// Softmax with per-row valid lengths (row r is normalised over its first len[r] entries, the rest of the
+// output row is +0, the rest of the input row is never read) is pinned by equality with the plain softmax on
+// a copy whose tails hold -inf, by len = cols, len = 0, len = 1, and by NaN-filled tails leaving no trace.
 // tf_tune has
 // no oracle function here: which candidate wins is hardware-dependent ("parity unpinned" for the
 // winner's identity; its output is checked like any other launch).
@@ -219,6 +222,22 @@ int oracle_rmsnorm(const void* x, const void* w, void* y, double* y64, float* rs
     if (bad(rows, cols, dt) || !x || !w) return -1;
     const double e = static_cast<double>(eps);
     for_rows(rows, nthreads, [=](int64_t r) { rmsnorm_row(x, w, y, y64, rstd, stats64, cols, e, dt, r); });
+    return 0;
+}
+
+// Softmax over the first len[r] entries of row r (0 <= len[r] <= cols, values outside are clamped): the
+// definition above applied to x[r, 0:len[r]]; y[r, j] = +0 for j >= len[r]; x[r, j >= len[r]] is not read.
+// len[r] = 0 gives an all +0 row (the fully masked reading above).
+int oracle_softmax_len(const void* x, const int32_t* len, void* y, double* y64, int64_t rows, int64_t cols, int dt, int nthreads) {
+    if (bad(rows, cols, dt) || !x || !len) return -1;
+    for_rows(rows, nthreads, [=](int64_t r) {
+        const int64_t n = len[r] < 0 ? 0 : (len[r] > cols ? cols : len[r]);
+        if (n > 0) softmax_row(x, y, y64, n, dt, r * cols);
+        for (int64_t j = n; j < cols; ++j) {
+            if (y64) y64[r * cols + j] = 0.0;
+            if (y) store(y, r * cols + j, dt, 0.0);
+        }
+    });
     return 0;
 }
 

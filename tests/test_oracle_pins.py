@@ -393,3 +393,47 @@ def test_add_then_norm_is_the_composition():
             exact = oracle.bf16_to_double(x) + oracle.bf16_to_double(r)
             assert np.abs(mean.astype(np.float64) - oracle.bf16_to_double(h).mean(axis=1)).max() < 1e-6
             assert np.abs(oracle.bf16_to_double(h) - exact).max() > 0          # rounding did happen
+
+
+# ------------------------------------------------------------------ softmax with per-row valid lengths
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_softmax_len_equals_masked_softmax_and_never_reads_the_tail(dt):
+    rng = np.random.default_rng(31 + dt)
+    rows, cols = 23, 77
+    enc = f32 if dt == F32 else bf
+    xv = rng.standard_normal((rows, cols)) * 4
+    lens = rng.integers(0, cols + 1, rows).astype(np.int32)
+    lens[:4] = [0, 1, cols, cols - 1]
+    x = enc(xv)
+    y, y64 = oracle.softmax_len(x, lens, dt, want64=True)
+    # (1) the plain softmax on a copy whose tails hold -inf: bit for bit
+    masked = xv.copy()
+    for r in range(rows):
+        masked[r, lens[r]:] = -np.inf
+    ym, ym64 = oracle.softmax(enc(masked), dt, want64=True)
+    np.testing.assert_array_equal(y, ym)
+    np.testing.assert_array_equal(y64, ym64)
+    # (2) the tail of the input is never read: NaN and +inf there leave no trace
+    poisoned = xv.copy()
+    for r in range(rows):
+        poisoned[r, lens[r]:] = np.nan if r % 2 else np.inf
+    yp = oracle.softmax_len(enc(poisoned), lens, dt)
+    np.testing.assert_array_equal(yp, y)
+    # (3) special lengths: 0 -> all +0 bits; 1 -> a single 1; cols -> the plain softmax; sums are 1 over the live part
+    bits = y.view(np.uint32) if dt == F32 else y
+    assert not bits[0].any()
+    one = np.float32(1.0).view(np.uint32) if dt == F32 else 0x3F80
+    assert bits[1, 0] == one and not bits[1, 1:].any()
+    np.testing.assert_array_equal(y[2], oracle.softmax(x[2:3], dt)[0])
+    for r in range(rows):
+        assert not bits[r, lens[r]:].any()
+        if lens[r]:
+            assert abs(y64[r, :lens[r]].sum() - 1.0) < 1e-12
+    # (4) lengths outside [0, cols] are clamped; threads only spread rows
+    wild = lens.copy()
+    wild[5], wild[6] = -7, cols + 100
+    ref = lens.copy()
+    ref[5], ref[6] = 0, cols
+    np.testing.assert_array_equal(oracle.softmax_len(x, wild, dt), oracle.softmax_len(x, ref, dt))
+    np.testing.assert_array_equal(oracle.softmax_len(x, lens, dt, nthreads=4), y)
