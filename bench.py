@@ -573,6 +573,67 @@ def run_addnorm_table(args):
     (out_dir / "table_addnorm.json").write_text(json.dumps(rows_out, indent=1))
 
 
+def run_softmaxlen_table(args):
+    """Softmax with per-row valid lengths against the same rows with the mask stored in the data (-inf tails)."""
+    import numpy as np
+    import torch
+    import paper_2512_09196_b200 as tf
+    from paper_2512_09196_b200 import inputs
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak()
+    out_dir = ROOT / "gpurun_out"
+    out_dir.mkdir(exist_ok=True)
+    shapes = [("tail 32 r mod cols (the mask of the 2 GiB configuration)", inputs.BF16, 4096, 131072), ("uniform lengths", inputs.BF16, 16384, 8192),
+              ("uniform lengths", inputs.F32, 65536, 1024), ("uniform lengths", inputs.BF16, 262144, 256), ("full lengths", inputs.BF16, 16384, 8192)]
+    rows_out = []
+    for kind, dt, rows, cols in shapes:
+        es = inputs.ELEM_SIZE[dt]
+        r = np.arange(rows, dtype=np.int64)
+        if kind.startswith("tail"):
+            lens = (cols - (32 * r) % cols).astype(np.int32)
+        elif kind.startswith("full"):
+            lens = np.full(rows, cols, np.int32)
+        else:
+            lens = np.random.default_rng(cols).integers(1, cols + 1, rows).astype(np.int32)
+        conv = (lambda t: t.view(torch.bfloat16)) if dt == inputs.BF16 else (lambda t: t)
+        sets = max(1, min(8, int((1 << 30) // (2 * rows * cols * es))))
+        x = conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols, 0, 0.0, 3.0))).cuda()
+        ld = torch.from_numpy(lens).cuda()
+        xm = x.clone()
+        xm[torch.arange(cols, device="cuda")[None, :] >= ld[:, None]] = float("-inf")
+        xs = [x] + [x.clone() for _ in range(sets - 1)]
+        xms = [xm] + [xm.clone() for _ in range(sets - 1)]
+        ys = [torch.empty_like(x) for _ in range(sets)]
+        tf.tf_tune("softmax", rows, cols, dt, like=(xm, None, None))
+
+        def timed(fn, reps):
+            for k in range(3):
+                fn(k % sets)
+            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for k in range(reps):
+                fn(k % sets)
+            e.record()
+            torch.cuda.synchronize()
+            return 1e3 * a.elapsed_time(e) / reps
+
+        nbytes = int(lens.astype(np.int64).sum()) * es + rows * cols * es + 4 * rows
+        reps = max(10, min(200, int(0.05 / (2 * rows * cols * es / 5e12))))
+        us_len = timed(lambda k: tf.tf_softmax_len_fwd(xs[k], ld, ys[k]), reps)
+        us_data = timed(lambda k: tf.tf_softmax_fwd(xms[k], ys[k]), reps)
+        tf.tf_device_status()
+        row = {"workload": f"softmax_len_{'f32' if dt == inputs.F32 else 'bf16'}_{rows}x{cols}", "lengths": kind, "dtype": "f32" if dt == inputs.F32 else "bf16",
+               "rows": rows, "cols": cols, "live_fraction": float(lens.mean() / cols), "bytes": nbytes, "us": us_len, "gbs": nbytes / us_len / 1e3,
+               f"pct_of_{peak_kind}_{peak:.0f}": 100 * nbytes / us_len / 1e3 / peak, "mask_in_data_us": us_data,
+               "speedup_vs_mask_in_data": us_data / us_len, "plain_plan": tf.tf_query_choice("softmax", rows, cols, dt)}
+        rows_out.append(row)
+        print(json.dumps(row), flush=True)
+        del xs, xms, ys, x, xm
+        torch.cuda.empty_cache()
+    (out_dir / "table_softmaxlen.json").write_text(json.dumps(rows_out, indent=1))
+
+
 def run_case(args):
     """A few launches of one op/shape (for profiler captures): --case op:dtype:rows:cols or --case config:<i>[:rows]."""
     import torch
@@ -630,7 +691,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm"], default=None)
+    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm", "softmaxlen"], default=None)
     ap.add_argument("--filter", default=None)
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
@@ -651,6 +712,8 @@ def main():
         return run_vecmat_table(args)
     if args.table == "addnorm":
         return run_addnorm_table(args)
+    if args.table == "softmaxlen":
+        return run_softmaxlen_table(args)
     if args.table:
         return run_table(args)
     run_ours(args)

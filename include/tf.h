@@ -120,6 +120,17 @@ tf_status tf_copy(const void* x, void* y, int64_t bytes, void* cuda_stream);
  * fp32 arithmetic with full range reduction, one rounding to the storage type.  y == x is allowed. */
 tf_status tf_sin_fwd(const void* x, void* y, int64_t n, tf_dtype dt, int threads, int vectors_per_thread, void* cuda_stream);
 
+/* ---- softmax with per-row valid lengths ------------------------------------------------------------------ */
+
+/* Row r is normalised over its first len[r] entries: y[r, j] = softmax(x[r, 0:len[r]])_j for j < len[r] and +0 for
+ * j >= len[r]; the contents of x[r, j >= len[r]] are ignored (anything, NaN included; x must still be a whole
+ * [rows, cols] allocation) and for rows of 16 KiB and more they are not read at all; len[r] = 0 gives an all +0 row,
+ * values outside [0, cols] are clamped.  Equal, bit for bit where the same plan runs, to tf_softmax_fwd on an x whose
+ * tails hold -inf.  The paper has no counterpart (its kernels take their masks in the data).
+ * x, y: [rows, cols] row-major device memory (y may alias x); len: int32 [rows], device memory; cols <= 2^31 - 1.
+ * Errors and stream behaviour as tf_softmax_fwd, plus TF_ERR_INVALID_ARG for a null len.  Allocates nothing. */
+tf_status tf_softmax_len_fwd(const void* x, const int32_t* len, void* y, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
+
 /* ---- fused residual add + norm ------------------------------------------------------------------------ */
 
 /* h = x + r (fp32 add, ONE rounding to the storage type), then the LayerNorm / RMSNorm defined above applied to that

@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_status_string",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
 
@@ -56,6 +56,7 @@ def lib() -> ctypes.CDLL:
         L.tf_add_layernorm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_add_rmsnorm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_tune_add.argtypes = [i32, i64, i64, i32]
+        L.tf_softmax_len_fwd.argtypes = [vp, vp, vp, i64, i64, i32, vp]
         L.tf_bvecmat_fwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp]
         L.tf_sin_fwd.argtypes = [vp, vp, i64, i32, i32, i32, vp]
         L.tf_tune_like.argtypes = [i32, vp, vp, vp, i64, i64, i32]
@@ -72,7 +73,7 @@ def lib() -> ctypes.CDLL:
         L.tf_clear_cache.restype = None
         L.tf_launch_count.argtypes = []
         L.tf_launch_count.restype = i64
-        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add",
+        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd",
                      "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice",
                      "tf_candidate_count", "tf_candidate"):
             getattr(L, name).restype = i32
@@ -135,6 +136,22 @@ def tf_softmax_fwd(x, y=None):
     rows, cols = x.shape
     with _on_device(x):
         _ok(lib().tf_softmax_fwd(x.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)), "tf_softmax_fwd")
+    return y
+
+
+def tf_softmax_len_fwd(x, lengths, y=None):
+    """Softmax of row r over its first ``lengths[r]`` entries (int32 CUDA tensor [rows]); the rest of the output row is
+    +0 and the rest of the input row is never read.  ``y`` may alias ``x``."""
+    import torch
+    _check2d(x)
+    rows, cols = x.shape
+    if not lengths.is_cuda or lengths.dtype != torch.int32 or lengths.shape != (rows,) or not lengths.is_contiguous():
+        raise ValueError("lengths must be a contiguous int32 CUDA tensor of shape [rows]")
+    if y is None:
+        y = torch.empty_like(x)
+    with _on_device(x):
+        _ok(lib().tf_softmax_len_fwd(x.data_ptr(), lengths.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)),
+            "tf_softmax_len_fwd")
     return y
 
 

@@ -14,19 +14,19 @@ using namespace rowreg;
 
 WarpFn warp_fn_add(int op, int dt, int l, int v, int r) {
     switch (op * 2 + dt) {
-        case 2: return pick_warp<OP_LAYERNORM, DT_F32, true>(l, v, r);
-        case 3: return pick_warp<OP_LAYERNORM, DT_BF16, true>(l, v, r);
-        case 4: return pick_warp<OP_RMSNORM, DT_F32, true>(l, v, r);
-        case 5: return pick_warp<OP_RMSNORM, DT_BF16, true>(l, v, r);
+        case 2: return pick_warp<OP_LAYERNORM, DT_F32, kModeAdd>(l, v, r);
+        case 3: return pick_warp<OP_LAYERNORM, DT_BF16, kModeAdd>(l, v, r);
+        case 4: return pick_warp<OP_RMSNORM, DT_F32, kModeAdd>(l, v, r);
+        case 5: return pick_warp<OP_RMSNORM, DT_BF16, kModeAdd>(l, v, r);
     }
     return nullptr;
 }
 CtaFn cta_fn_add(int op, int dt, int v, bool c) {
     switch (op * 2 + dt) {
-        case 2: return pick_cta<OP_LAYERNORM, DT_F32, true>(v, c);
-        case 3: return pick_cta<OP_LAYERNORM, DT_BF16, true>(v, c);
-        case 4: return pick_cta<OP_RMSNORM, DT_F32, true>(v, c);
-        case 5: return pick_cta<OP_RMSNORM, DT_BF16, true>(v, c);
+        case 2: return pick_cta<OP_LAYERNORM, DT_F32, kModeAdd>(v, c);
+        case 3: return pick_cta<OP_LAYERNORM, DT_BF16, kModeAdd>(v, c);
+        case 4: return pick_cta<OP_RMSNORM, DT_F32, kModeAdd>(v, c);
+        case 5: return pick_cta<OP_RMSNORM, DT_BF16, kModeAdd>(v, c);
     }
     return nullptr;
 }

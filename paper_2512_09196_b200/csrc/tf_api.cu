@@ -226,6 +226,7 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
     if (a.op == OP_LAYERNORM || nvec > 8192) {
         Plan s;
         s.variant = V_TWOPASS; s.threads = 512; s.chunk = 49152;
+        if (a.op == OP_SOFTMAX) s.rpg = 2;           // the 40-register build: three CTAs per SM (measured faster on the 2 GiB softmax)
         return s;
     }
     {
@@ -500,6 +501,29 @@ tf_status run_add(const Args& a0, void* stream) {
     return run(b, stream);
 }
 
+// Softmax with per-row valid lengths: a forced plan when it is one of the kinds that have a length mode, else this
+// mode's own default (measured separately from the plain softmax).
+tf_status run_len(const Args& a0, void* stream) {
+    if (a0.rows == 0) return TF_OK;
+    DevState* ds = nullptr;
+    tf_status s = device_state(&ds);
+    if (s != TF_OK) return s;
+    Args a = a0;
+    a.status = ds->status;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (!vector_ok(a)) {
+        e = launch_softmax_len_scalar(a, st);
+        return e == cudaSuccess ? TF_OK : cuda_fail(e);
+    }
+    bool forced = false;
+    Plan p = choose(a, ds->info, &forced);
+    if (!forced || !supports_softmax_len(p, a, ds->info)) p = heuristic_softmax_len(a, ds->info);
+    if (!supports_softmax_len(p, a, ds->info)) return TF_ERR_UNSUPPORTED;
+    e = launch_softmax_len(p, a, ds->info, st);
+    return e == cudaSuccess ? TF_OK : cuda_fail(e);
+}
+
 bool bad_shape(int64_t rows, int64_t cols, int dt) {  // dt arrives as an int so that out-of-range enum values are caught
     return rows < 0 || cols <= 0 || (dt != DT_F32 && dt != DT_BF16); }
 bool too_big(int64_t rows, int64_t cols) { return rows > 0 && cols > (INT64_MAX / 8) / rows; }
@@ -563,6 +587,14 @@ tf_status tf_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols, tf_
     if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
     Args a{OP_SOFTMAX, dt, x, nullptr, nullptr, y, nullptr, nullptr, rows, cols, 0.f, nullptr};
     return run(a, stream);
+}
+
+tf_status tf_softmax_len_fwd(const void* x, const int32_t* len, void* y, int64_t rows, int64_t cols, tf_dtype dt, void* stream) {
+    if (bad_shape(rows, cols, dt) || cols > 0x7FFFFFFF || (rows > 0 && (!x || !y || !len))) return TF_ERR_INVALID_ARG;
+    if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
+    Args a{OP_SOFTMAX, dt, x, nullptr, nullptr, y, nullptr, nullptr, rows, cols, 0.f, nullptr};
+    a.len = len;
+    return run_len(a, stream);
 }
 
 tf_status tf_layernorm_fwd(const void* x, const void* gamma, const void* beta, void* y, float* mean, float* rstd,

@@ -46,6 +46,7 @@ struct Args {
     int* status;         // device word that bounded waits set when they give up
     const void* r = nullptr;   // fused residual add: second input ...
     void* h = nullptr;         // ... and where x + r (rounded to the storage type) goes
+    const int* len = nullptr;  // softmax with per-row valid lengths (elements), device memory
 };
 
 struct DeviceInfo {
@@ -88,6 +89,13 @@ bool supports_addnorm(const Plan&, const Args&, const DeviceInfo&);
 cudaError_t launch_addnorm(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 Plan heuristic_addnorm(const Args&, const DeviceInfo&);
 cudaError_t launch_add_elementwise(const void* x, const void* r, void* h, int64_t n, int dt, cudaStream_t);
+
+// Softmax with per-row valid lengths (Args::len set): register-resident plans and the two-pass plan; the scalar kernel
+// serves what they cannot (unaligned tensors, widths that are not whole 16-byte vectors).
+bool supports_softmax_len(const Plan&, const Args&, const DeviceInfo&);
+cudaError_t launch_softmax_len(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+cudaError_t launch_softmax_len_scalar(const Args&, cudaStream_t);
+Plan heuristic_softmax_len(const Args&, const DeviceInfo&);
 size_t split_scratch_bytes(const Plan&, const Args&);
 
 // Bookkeeping shared with the C ABI layer: count kernel launches; remember the CUDA error behind a TF_ERR_CUDA.

@@ -40,6 +40,22 @@ struct LazyParams {
     __device__ __forceinline__ uint4 beta(int v) const { return ld_param(p1 + first + v * stride); }
 };
 
+// Keeps the first `keep` (1 .. NE-1) elements of a vector and replaces the rest by -inf.
+template <int DT> __device__ __forceinline__ uint4 mask_tail(const uint4& v, int keep) {
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    if constexpr (DT == DT_F32) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) if (i >= keep) w[i] = 0xFF800000u;
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (2 * i >= keep) w[i] = (w[i] & 0xFFFF0000u) | 0x0000FF80u;
+            if (2 * i + 1 >= keep) w[i] = (w[i] & 0x0000FFFFu) | 0xFF800000u;
+        }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 // Parameters copied once into shared memory by the thread that will use them (a persistent CTA always owns the same
 // columns): no barrier is needed between the copy and the reads.
 struct OwnedSmemParams {

@@ -17,23 +17,23 @@ using namespace rowreg;
 
 WarpFn warp_fn(int op, int dt, int l, int v, int r) {
     switch (op * 2 + dt) {
-        case 0: return pick_warp<OP_SOFTMAX, DT_F32, false>(l, v, r);
-        case 1: return pick_warp<OP_SOFTMAX, DT_BF16, false>(l, v, r);
-        case 2: return pick_warp<OP_LAYERNORM, DT_F32, false>(l, v, r);
-        case 3: return pick_warp<OP_LAYERNORM, DT_BF16, false>(l, v, r);
-        case 4: return pick_warp<OP_RMSNORM, DT_F32, false>(l, v, r);
-        case 5: return pick_warp<OP_RMSNORM, DT_BF16, false>(l, v, r);
+        case 0: return pick_warp<OP_SOFTMAX, DT_F32, kModePlain>(l, v, r);
+        case 1: return pick_warp<OP_SOFTMAX, DT_BF16, kModePlain>(l, v, r);
+        case 2: return pick_warp<OP_LAYERNORM, DT_F32, kModePlain>(l, v, r);
+        case 3: return pick_warp<OP_LAYERNORM, DT_BF16, kModePlain>(l, v, r);
+        case 4: return pick_warp<OP_RMSNORM, DT_F32, kModePlain>(l, v, r);
+        case 5: return pick_warp<OP_RMSNORM, DT_BF16, kModePlain>(l, v, r);
     }
     return nullptr;
 }
 CtaFn cta_fn(int op, int dt, int v, bool c) {
     switch (op * 2 + dt) {
-        case 0: return pick_cta<OP_SOFTMAX, DT_F32, false>(v, c);
-        case 1: return pick_cta<OP_SOFTMAX, DT_BF16, false>(v, c);
-        case 2: return pick_cta<OP_LAYERNORM, DT_F32, false>(v, c);
-        case 3: return pick_cta<OP_LAYERNORM, DT_BF16, false>(v, c);
-        case 4: return pick_cta<OP_RMSNORM, DT_F32, false>(v, c);
-        case 5: return pick_cta<OP_RMSNORM, DT_BF16, false>(v, c);
+        case 0: return pick_cta<OP_SOFTMAX, DT_F32, kModePlain>(v, c);
+        case 1: return pick_cta<OP_SOFTMAX, DT_BF16, kModePlain>(v, c);
+        case 2: return pick_cta<OP_LAYERNORM, DT_F32, kModePlain>(v, c);
+        case 3: return pick_cta<OP_LAYERNORM, DT_BF16, kModePlain>(v, c);
+        case 4: return pick_cta<OP_RMSNORM, DT_F32, kModePlain>(v, c);
+        case 5: return pick_cta<OP_RMSNORM, DT_BF16, kModePlain>(v, c);
     }
     return nullptr;
 }

@@ -1,6 +1,8 @@
 // Kernel templates of the register-resident variants (V_WARP, V_CTA), shared by the plain row ops and by the fused
-// residual-add forms (ADD = true: h = x + r is formed in fp32, rounded to the storage type, written out, and the row
-// op then runs on the rounded h, exactly as if the two ops had been called one after the other).
+// residual-add forms (MODE = kModeAdd: h = x + r is formed in fp32, rounded to the storage type, written out, and the
+// row op then runs on the rounded h, exactly as if the two ops had been called one after the other) and by softmax with
+// per-row valid lengths (MODE = kModeLen: vectors past the row's length are not loaded, the vector that straddles it
+// has its tail replaced by -inf; the stores still cover the whole row, so the tail of y is +0).
 #pragma once
 
 #include <cooperative_groups.h>
@@ -19,8 +21,9 @@ struct KArgs {
     const uint4* p0;
     const uint4* p1;
     uint4* y;
-    const uint4* r;  // ADD: residual input
-    uint4* h;        // ADD: x + r, rounded to the storage type
+    const uint4* r;  // kModeAdd: residual input
+    uint4* h;        // kModeAdd: x + r, rounded to the storage type
+    const int* len;  // kModeLen: valid length of every row, in elements
     float* mean;
     float* rstd;
     int64_t rows;
@@ -28,6 +31,24 @@ struct KArgs {
     float n;         // cols as float
     float eps;
 };
+
+constexpr int kModePlain = 0, kModeAdd = 1, kModeLen = 2;
+
+// Row length in elements, clamped to [0, cols].
+__device__ __forceinline__ int row_len(const int* len, int64_t row, int cols) { return min(max(__ldg(len + row), 0), cols); }
+
+// What a loaded vector `vi` of a row is worth when only the row's first `len` elements count (NE per vector).
+template <int DT>
+__device__ __forceinline__ uint4 apply_len(const uint4& v, int vi, int len, const uint4& fill) {
+    constexpr int NE = Elem<DT>::NE;
+    const int keep = len - vi * NE;                                   // elements of this vector that count
+    if (keep <= 0) return fill;
+    return keep < NE ? mask_tail<DT>(v, keep) : v;                    // at most one vector of a row straddles the length
+}
+// Rows of at least this many vectors (16 KiB) do not read what lies behind their length: their loads wait for the row's
+// length to arrive first, which pays off from about this size on (measured at 16 KiB, half of every row live: 90 us
+// skipping, 96 us reading everything).  Shorter rows load the whole row at once, like the plain kernels, and discard.
+constexpr int kLenSkipVecs = 1024;
 
 template <int DT>
 __device__ __forceinline__ uint4 add_round(const uint4& a, const uint4& b) {
@@ -47,7 +68,7 @@ constexpr int cta_max_threads(int vpt) { return vpt <= 2 ? 1024 : 512; }
 // =====================================================================================================
 // V_WARP
 // =====================================================================================================
-template <int OP, int DT, int LANES, int VPT, int RPG, bool ADD>
+template <int OP, int DT, int LANES, int VPT, int RPG, int MODE>
 __global__ void __launch_bounds__(kWarpMaxThreads) k_warp(const KArgs a) {
     pdl_wait();
     pdl_trigger();
@@ -75,11 +96,14 @@ __global__ void __launch_bounds__(kWarpMaxThreads) k_warp(const KArgs a) {
         for (int rr = 0; rr < RPG; ++rr) {
             const int64_t row = base + rr * G + g;                          // adjacent groups -> adjacent rows
 #pragma unroll
+            const int len_row = (MODE == kModeLen && row < a.rows) ? row_len(a.len, row, a.nvec * Elem<DT>::NE) : 0;
+            (void)len_row;
             for (int v = 0; v < VPT; ++v) {
                 const bool ok = row < a.rows && valid[v];
                 const int64_t idx = row * a.nvec + lane + v * LANES;
                 raw[rr][v] = ok ? ld_stream(a.x + idx) : fill;
-                if constexpr (ADD) {
+                if constexpr (MODE == kModeLen) raw[rr][v] = apply_len<DT>(raw[rr][v], lane + v * LANES, len_row, fill);
+                if constexpr (MODE == kModeAdd) {
                     if (ok) {
                         raw[rr][v] = add_round<DT>(raw[rr][v], ld_stream(a.r + idx));
                         st_stream(a.h + idx, raw[rr][v]);
@@ -109,7 +133,7 @@ __global__ void __launch_bounds__(kWarpMaxThreads) k_warp(const KArgs a) {
 // =====================================================================================================
 // V_CTA (optionally split over a cluster)
 // =====================================================================================================
-template <int OP, int DT, int VPT, bool CLUSTER, bool ADD>
+template <int OP, int DT, int VPT, bool CLUSTER, int MODE>
 __global__ void __launch_bounds__(cta_max_threads(VPT)) k_cta(const KArgs a, const int cs) {
     using E = Elem<DT>;
     constexpr int NE = E::NE;
@@ -140,9 +164,20 @@ __global__ void __launch_bounds__(cta_max_threads(VPT)) k_cta(const KArgs a, con
         const uint4* xr = a.x + row * a.nvec + first + t;
         uint4* yr = a.y + row * a.nvec + first + t;
         uint4 raw[VPT], out[VPT];
+        const int len_row = MODE == kModeLen ? row_len(a.len, row, a.nvec * NE) : 0;
+        (void)len_row;
+        if (MODE == kModeLen && a.nvec >= kLenSkipVecs) {              // long rows: nothing behind the length is read
 #pragma unroll
-        for (int v = 0; v < VPT; ++v) raw[v] = valid[v] ? ld_stream(xr + v * T) : fill;
-        if constexpr (ADD) {
+            for (int v = 0; v < VPT; ++v) raw[v] = (valid[v] && (first + t + v * T) * NE < len_row) ? ld_stream(xr + v * T) : fill;
+        } else {
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) raw[v] = valid[v] ? ld_stream(xr + v * T) : fill;
+        }
+        if constexpr (MODE == kModeLen) {
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) raw[v] = apply_len<DT>(raw[v], first + t + v * T, len_row, fill);
+        }
+        if constexpr (MODE == kModeAdd) {
             const uint4* rr = a.r + row * a.nvec + first + t;
             uint4* hr = a.h + row * a.nvec + first + t;
 #pragma unroll
@@ -185,7 +220,7 @@ __global__ void __launch_bounds__(cta_max_threads(VPT)) k_cta(const KArgs a, con
 
 inline KArgs make_kargs(const Args& a) {
     KArgs k;
-    k.r = static_cast<const uint4*>(a.r); k.h = static_cast<uint4*>(a.h);
+    k.r = static_cast<const uint4*>(a.r); k.h = static_cast<uint4*>(a.h); k.len = a.len;
     k.x = static_cast<const uint4*>(a.x); k.p0 = static_cast<const uint4*>(a.p0); k.p1 = static_cast<const uint4*>(a.p1);
     k.y = static_cast<uint4*>(a.y); k.mean = a.mean; k.rstd = a.rstd; k.rows = a.rows;
     k.nvec = static_cast<int>(a.cols * elem_size(a.dt) / 16);
@@ -196,8 +231,8 @@ inline KArgs make_kargs(const Args& a) {
 using WarpFn = void (*)(const KArgs);
 using CtaFn = void (*)(const KArgs, const int);
 
-template <int OP, int DT, bool ADD> WarpFn pick_warp(int lanes, int vpt, int rpg) {
-#define TF_W(L, V, R) if (lanes == L && vpt == V && rpg == R) return k_warp<OP, DT, L, V, R, ADD>;
+template <int OP, int DT, int MODE> WarpFn pick_warp(int lanes, int vpt, int rpg) {
+#define TF_W(L, V, R) if (lanes == L && vpt == V && rpg == R) return k_warp<OP, DT, L, V, R, MODE>;
     TF_W(8, 1, 1) TF_W(8, 1, 2) TF_W(8, 1, 4) TF_W(8, 2, 1) TF_W(8, 2, 2)
     TF_W(16, 1, 1) TF_W(16, 1, 2) TF_W(16, 1, 4) TF_W(16, 2, 1) TF_W(16, 2, 2)
     TF_W(32, 1, 1) TF_W(32, 1, 2) TF_W(32, 1, 4) TF_W(32, 2, 1) TF_W(32, 2, 2) TF_W(32, 4, 1) TF_W(32, 4, 2) TF_W(32, 8, 1)
@@ -205,8 +240,8 @@ template <int OP, int DT, bool ADD> WarpFn pick_warp(int lanes, int vpt, int rpg
     return nullptr;
 }
 
-template <int OP, int DT, bool ADD> CtaFn pick_cta(int vpt, bool cluster) {
-#define TF_C(V) if (vpt == V) return cluster ? k_cta<OP, DT, V, true, ADD> : k_cta<OP, DT, V, false, ADD>;
+template <int OP, int DT, int MODE> CtaFn pick_cta(int vpt, bool cluster) {
+#define TF_C(V) if (vpt == V) return cluster ? k_cta<OP, DT, V, true, MODE> : k_cta<OP, DT, V, false, MODE>;
     TF_C(1) TF_C(2) TF_C(4) TF_C(8)
 #undef TF_C
     return nullptr;

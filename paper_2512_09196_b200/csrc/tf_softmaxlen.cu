@@ -1,0 +1,101 @@
+// Softmax with per-row valid lengths: row r is normalised over x[r, 0 : len[r]], y[r, len[r] :] = +0, and
+// x[r, len[r] :] is never read (it may hold anything).  Against a mask stored in the data this saves the reads of
+// the masked tails; the writes stay.
+//
+// Served by the register-resident kernels in their length mode (a lane group, a CTA or a cluster holds the row), by the
+// streamed two-pass kernel for rows beyond 128 KiB, and by a scalar CTA-per-row kernel for tensors that are not
+// 16-byte aligned or whose width is not a whole number of 16-byte vectors.
+#include "tf_rowreg.cuh"
+
+namespace tf {
+namespace {
+
+using namespace rowreg;
+
+WarpFn warp_fn_len(int dt, int l, int v, int r) {
+    return dt == DT_F32 ? pick_warp<OP_SOFTMAX, DT_F32, kModeLen>(l, v, r) : pick_warp<OP_SOFTMAX, DT_BF16, kModeLen>(l, v, r);
+}
+CtaFn cta_fn_len(int dt, int v, bool c) {
+    if (v > 4 && dt == DT_BF16) return nullptr;         // bf16 with eight vectors per thread needs 120 registers in this mode (92 plain)
+    return dt == DT_F32 ? pick_cta<OP_SOFTMAX, DT_F32, kModeLen>(v, c) : pick_cta<OP_SOFTMAX, DT_BF16, kModeLen>(v, c);
+}
+
+// Any alignment, any width: a CTA per row, three scalar passes over the live part (max, sum, write), zeros behind it.
+template <int DT>
+__global__ void __launch_bounds__(256) k_softmax_len_scalar(const typename Elem<DT>::scalar* x, const int* len, typename Elem<DT>::scalar* y,
+                                                            int64_t rows, int64_t cols) {
+    using E = Elem<DT>;
+    __shared__ float buf[2][32];
+    const int64_t row = blockIdx.x;
+    if (row >= rows) return;
+    const int64_t n = min(max(static_cast<int64_t>(len[row]), int64_t{0}), cols);
+    const typename E::scalar* xr = x + row * cols;
+    typename E::scalar* yr = y + row * cols;
+    float m = kNegInf;
+    for (int64_t j = threadIdx.x; j < n; j += blockDim.x) m = fmaxf(m, E::to_float(xr[j]));
+    m = cta_reduce<MaxOp>(m, buf[0]);
+    float s = 0.f;
+    if (m != kNegInf)
+        for (int64_t j = threadIdx.x; j < n; j += blockDim.x) s += expf(E::to_float(xr[j]) - m);
+    s = cta_reduce<SumOp>(s, buf[1]);
+    const float inv = s > 0.f ? 1.0f / s : 0.f;
+    for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) {
+        float v = 0.f;
+        if (j < n && m != kNegInf) v = expf(E::to_float(xr[j]) - m) * inv;
+        yr[j] = E::from_float(v);
+    }
+}
+
+}  // namespace
+
+bool supports_softmax_len(const Plan& p, const Args& a, const DeviceInfo& d) {
+    if (a.op != OP_SOFTMAX || !a.len) return false;
+    if (p.variant == V_WARP) return warp_geometry_ok(p, a) && warp_fn_len(a.dt, p.lanes, p.vpt, p.rpg) != nullptr;
+    if (p.variant == V_CTA) return cta_geometry_ok(p, a, d) && cta_fn_len(a.dt, p.vpt, p.cluster > 1) != nullptr;
+    if (p.variant == V_TWOPASS) return supports_twopass(p, a, d);
+    return false;
+}
+
+cudaError_t launch_softmax_len(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
+    count_launches(1);
+    if (p.variant == V_TWOPASS) return launch_twopass(p, a, d, st);
+    if (p.variant == V_WARP) return launch_warp_fn(warp_fn_len(a.dt, p.lanes, p.vpt, p.rpg), p, a, d, st);
+    return launch_cta_fn(cta_fn_len(a.dt, p.vpt, p.cluster > 1), p, a, d, st);
+}
+
+// Default plan, from measurements on rows of 512 B to 64 KiB: a lane group with one row in flight up to 1 KiB, a CTA
+// with four vectors per thread (eight for fp32 from 16 KiB on) up to 64 KiB, the streamed two-pass kernel from there.
+// (The plans that win for the plain softmax are not reused: more rows in flight per group or eight bf16 vectors per
+// thread cost this mode 30-80 %.)
+Plan heuristic_softmax_len(const Args& a, const DeviceInfo& d) {
+    const int64_t nvec = a.cols * elem_size(a.dt) / 16;
+    Plan q;
+    if (nvec <= 64) {
+        q.variant = V_WARP; q.threads = 128; q.rpg = 1;
+        if (nvec <= 8) { q.lanes = 8; q.vpt = 1; }
+        else if (nvec <= 16) { q.lanes = 8; q.vpt = 2; }
+        else if (nvec <= 32) { q.lanes = 16; q.vpt = 2; }
+        else { q.lanes = 32; q.vpt = 2; }
+        if (supports_softmax_len(q, a, d)) return q;
+    } else if (nvec < 4096) {
+        q.variant = V_CTA; q.cluster = 1;
+        q.vpt = (a.dt == DT_F32 && nvec >= 1024) ? 8 : 4;
+        q.threads = std::max(64, static_cast<int>((nvec + q.vpt - 1) / q.vpt + 31) / 32 * 32);
+        if (supports_softmax_len(q, a, d)) return q;
+    }
+    Plan t;
+    t.variant = V_TWOPASS; t.threads = 512; t.chunk = 49152; t.rpg = 2;
+    return t;
+}
+
+cudaError_t launch_softmax_len_scalar(const Args& a, cudaStream_t st) {
+    if (a.rows > 0x7FFFFFFF) return cudaErrorInvalidConfiguration;
+    count_launches(1);
+    if (a.dt == DT_F32)
+        k_softmax_len_scalar<DT_F32><<<static_cast<unsigned>(a.rows), 256, 0, st>>>(static_cast<const float*>(a.x), a.len, static_cast<float*>(a.y), a.rows, a.cols);
+    else
+        k_softmax_len_scalar<DT_BF16><<<static_cast<unsigned>(a.rows), 256, 0, st>>>(static_cast<const uint16_t*>(a.x), a.len, static_cast<uint16_t*>(a.y), a.rows, a.cols);
+    return cudaGetLastError();
+}
+
+}  // namespace tf

@@ -104,20 +104,26 @@ template <int OP, int DT> struct Running {
 // Pass A over `nvec` vectors starting at xs (all threads of the CTA take part).  The first `cache_vecs` vectors
 // are also parked in shared memory (`cache`), each by the thread that will want it back in pass B -- the same
 // thread meets the same vectors in both passes, so no barrier is needed between them.
+// len >= 0 (softmax with a valid length, in elements): only the first ceil(len / NE) vectors are read and the one that
+// straddles the length has its tail replaced by -inf.
 template <int OP, int DT>
 __device__ __forceinline__ Running<OP, DT> stream_stats(const uint4* xs, int64_t nvec, uint64_t policy, uint4* cache = nullptr,
-                                                        int64_t cache_vecs = 0) {
-    constexpr int U = kStreamU;
+                                                        int64_t cache_vecs = 0, int64_t len = -1) {
+    constexpr int U = kStreamU, NE = Elem<DT>::NE;
     const int T = blockDim.x, t = threadIdx.x;
     const uint4 fill = fill_vec<DT>(OP);
     Running<OP, DT> run;
+    if (len >= 0) nvec = (len + NE - 1) / NE;
+    const int64_t straddle = (len >= 0 && len % NE) ? nvec - 1 : -1;
     for (int64_t base = t; base < nvec; base += static_cast<int64_t>(T) * U) {
         uint4 raw[U];
         bool ok[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            ok[u] = base + static_cast<int64_t>(u) * T < nvec;
-            raw[u] = ok[u] ? ld_hint(xs + base + static_cast<int64_t>(u) * T, policy) : fill;
+            const int64_t idx = base + static_cast<int64_t>(u) * T;
+            ok[u] = idx < nvec;
+            raw[u] = ok[u] ? ld_hint(xs + idx, policy) : fill;
+            if (idx == straddle) raw[u] = mask_tail<DT>(raw[u], static_cast<int>(len % NE));
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -167,9 +173,10 @@ __device__ __forceinline__ RowScale scale_of_row(const Part& p, float n, float e
 template <int OP, int DT>
 __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const uint4* g, const uint4* b, int64_t nvec,
                                              const RowScale& sc, uint64_t policy, const uint4* cache = nullptr,
-                                             int64_t cache_vecs = 0, int64_t live_end = INT64_MAX) {
+                                             int64_t cache_vecs = 0, int64_t live_end = INT64_MAX, int64_t len = -1) {
     using P = Pairs<DT>;
-    constexpr int NP = P::NP, U = kStreamU;
+    constexpr int NP = P::NP, U = kStreamU, NE = Elem<DT>::NE;
+    const int64_t straddle = (len >= 0 && len % NE) ? len / NE : -1;      // live_end already ends at ceil(len / NE)
     const int T = blockDim.x, t = threadIdx.x;
     const uint4 fill = fill_vec<DT>(OP);
     const F2 ta2 = f2(sc.a), tb2 = f2(sc.b), l2e = f2(kLog2e);
@@ -183,6 +190,7 @@ __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const u
             const int64_t idx = base + static_cast<int64_t>(u) * T;
             ok[u] = idx < nvec;
             raw[u] = (!ok[u] || idx >= live_end) ? fill : (idx < cache_vecs ? cache[idx] : ld_hint(xs + idx, policy));
+            if (idx == straddle) raw[u] = mask_tail<DT>(raw[u], static_cast<int>(len % NE));
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {

@@ -26,6 +26,7 @@ struct WArgs {
     float* rstd;
     int64_t rows;
     int64_t nvec;
+    const int* len;       // softmax with per-row valid lengths (elements), or null
     int64_t cache_vecs;   // vectors at the head of a row parked in shared memory between the passes
     float n, eps;
 };
@@ -43,7 +44,9 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass(const WArgs a) {
     int it = 0;
     for (int64_t row = blockIdx.x; row < a.rows; row += gridDim.x, ++it) {
         const uint4* xr = a.x + row * a.nvec;
-        const Running<OP, DT> run = stream_stats<OP, DT>(xr, a.nvec, keep, cache, a.cache_vecs);
+        int64_t len = -1;
+        if (OP == OP_SOFTMAX && a.len) len = min(max(static_cast<int64_t>(__ldg(a.len + row)), int64_t{0}), a.nvec * Elem<DT>::NE);
+        const Running<OP, DT> run = stream_stats<OP, DT>(xr, a.nvec, keep, cache, a.cache_vecs, len);
         const Part part = merge_running<OP, DT>(run, a.n, red_buf + 64 * (it & 1));
         const RowScale sc = scale_of_row<OP>(part, a.n, a.eps);
         if (threadIdx.x == 0) {
@@ -51,7 +54,7 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass(const WArgs a) {
             if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = sc.b;
         }
         stream_apply<OP, DT>(xr, a.y + row * a.nvec, a.p0, a.p1, a.nvec, sc, last, cache, a.cache_vecs,
-                             OP == OP_SOFTMAX ? run.live_end : INT64_MAX);
+                             OP == OP_SOFTMAX ? run.live_end : INT64_MAX, len);
     }
 }
 
@@ -93,7 +96,7 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
     grid = std::min<int64_t>(grid, 0x7FFFFFFF);
     WArgs k;
     k.x = static_cast<const uint4*>(a.x); k.p0 = static_cast<const uint4*>(a.p0); k.p1 = static_cast<const uint4*>(a.p1);
-    k.y = static_cast<uint4*>(a.y); k.mean = a.mean; k.rstd = a.rstd; k.rows = a.rows;
+    k.y = static_cast<uint4*>(a.y); k.mean = a.mean; k.rstd = a.rstd; k.rows = a.rows; k.len = a.len;
     k.nvec = a.cols * elem_size(a.dt) / 16;
     k.n = static_cast<float>(a.cols); k.eps = a.eps;
     k.cache_vecs = std::min<int64_t>(k.nvec, p.chunk / 16);

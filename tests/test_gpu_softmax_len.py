@@ -1,0 +1,109 @@
+"""Softmax with per-row valid lengths through the C ABI against the CPU oracle.  The tails of x hold NaN in every
+test: a kernel that read them would poison its row."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import compare
+import oracle
+import paper_2512_09196_b200 as tf
+from paper_2512_09196_b200 import inputs
+import parity
+
+pytestmark = pytest.mark.gpu
+F32, BF16 = inputs.F32, inputs.BF16
+NAN = {F32: np.float32(np.nan), BF16: np.uint16(0x7FC0)}
+NINF = {F32: np.float32(-np.inf), BF16: np.uint16(0xFF80)}
+
+
+@pytest.fixture(autouse=True)
+def _auto_plans():
+    yield
+    tf.tf_force_plan("softmax", None)
+
+
+def lengths_for(rows, cols, seed):
+    rng = np.random.default_rng(seed)
+    ne = 8
+    lens = rng.integers(0, cols + 1, rows).astype(np.int32)
+    special = [0, 1, cols, max(0, cols - 1), min(cols, ne), min(cols, ne + 1), min(cols, max(0, ne - 1)), cols // 2]
+    lens[:min(rows, len(special))] = special[:min(rows, len(special))]
+    return lens
+
+
+def run_case(dt, rows, cols, seed=1, offset=0, inplace=False, x_std=3.0, compare_plain=False):
+    x = inputs.normal((rows, cols), dt, seed, 0, 0.0, x_std)
+    lens = lengths_for(rows, cols, seed)
+    poisoned, masked = x.copy(), x.copy()
+    for r in range(rows):
+        poisoned[r, lens[r]:] = NAN[dt]
+        masked[r, lens[r]:] = NINF[dt]
+    ref, ref64 = oracle.softmax_len(poisoned, lens, dt, want64=True, nthreads=8)
+    xd = parity.to_dev(poisoned, dt, offset)
+    ld = torch.from_numpy(lens).cuda()
+    y = tf.tf_softmax_len_fwd(xd, ld, xd if inplace else None)
+    torch.cuda.synchronize()
+    tf.tf_device_status()
+    got = parity.to_host(y, dt)
+    rep = compare.compare_softmax(got, ref, ref64, masked, dt)          # masked positions must hold the bits of +0
+    assert rep.ok, (dt, rows, cols, offset, inplace, str(rep))
+    if compare_plain:                                                   # same plan, mask in the data: the same bits
+        plain = parity.to_host(tf.tf_softmax_fwd(parity.to_dev(masked, dt, offset)), dt)
+        np.testing.assert_array_equal(got, plain)
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_automatic_plan_over_edge_widths(dt):
+    ne = 4 if dt == F32 else 8
+    for cols in (ne, 2 * ne, 3 * ne, 64, 256, 1000 // ne * ne, 1024, 4096, 5120, 12288, 32768, 65536, 200000 // ne * ne):
+        rows = max(9, min(200, (1 << 21) // cols))
+        run_case(dt, rows, cols, seed=cols)
+    run_case(dt, 0, 64)
+    run_case(dt, 1, 4096)
+    run_case(dt, 500, 2048, inplace=True)
+    run_case(dt, 9, 65536, inplace=True, x_std=20.0)
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_unaligned_and_odd_widths_take_the_scalar_kernel(dt):
+    run_case(dt, 9, 1001)
+    run_case(dt, 9, 7)
+    run_case(dt, 11, 1024, offset=1)
+    run_case(dt, 11, 4099, offset=3, inplace=True)
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_forced_plans_and_bitwise_equality_with_the_masked_plain_softmax(dt):
+    ne = 4 if dt == F32 else 8
+    for lanes, vpt, rpg in ((8, 1, 1), (8, 2, 2), (16, 1, 4), (32, 2, 2), (32, 4, 1), (32, 8, 1)):
+        cap = lanes * vpt
+        for nvec in (cap, max(1, cap - 1)):
+            tf.tf_force_plan("softmax", f"warp:threads=128,lanes={lanes},vpt={vpt},rpg={rpg},persist=0")
+            run_case(dt, 301, nvec * ne, seed=nvec, compare_plain=True)
+    for cluster in (1, 2, 8):
+        for vpt, threads in ((1, 64), (2, 1024), (4, 256), (8, 512)):
+            cap = threads * vpt * cluster
+            for nvec, persist in ((cap, 0), (max(1, cap - threads - 3), 1)):
+                tf.tf_force_plan("softmax", f"cta:threads={threads},vpt={vpt},cluster={cluster},persist={persist}")
+                run_case(dt, 9 if nvec >= 4096 else 170, nvec * ne, seed=nvec, compare_plain=vpt <= 4 or dt == F32)   # bf16 x 8 vectors: own choice
+    for threads, cache, regcap, persist in ((32, 0, 0, 0), (256, 4096, 1, 0), (512, 49152, 1, 0), (1024, 0, 0, 2)):
+        for nvec, rows in ((1, 9), (threads * 4 + 1, 9), (threads * 9 - 3, 60), (70001, 9)):
+            tf.tf_force_plan("softmax", f"twopass:threads={threads},cache={cache},persist={persist},regcap={regcap}")
+            run_case(dt, rows, nvec * ne, seed=nvec, compare_plain=True)
+    # a forced plan without a length mode (the pipeline) falls back to the length-aware choice
+    tf.tf_force_plan("softmax", "pipe:threads=512,lanes=64,vpt=8,rpg=1,stages=2,chunk=8192,persist=1")
+    run_case(dt, 100, 512 * ne)
+
+
+def test_bad_arguments():
+    L = tf.lib()
+    p = torch.zeros(64, device="cuda").data_ptr()
+    assert L.tf_softmax_len_fwd(p, None, p, 1, 8, 0, None) == 1
+    assert L.tf_softmax_len_fwd(None, p, p, 1, 8, 0, None) == 1
+    assert L.tf_softmax_len_fwd(p, p, p, 1, 0, 0, None) == 1
+    assert L.tf_softmax_len_fwd(p, p, p, 1, 8, 5, None) == 1
+    assert L.tf_softmax_len_fwd(p, p, p, 0, 8, 0, None) == 0
+    with pytest.raises(ValueError):
+        tf.tf_softmax_len_fwd(torch.zeros(4, 8, device="cuda"), torch.zeros(4, dtype=torch.int64, device="cuda"))
