@@ -119,3 +119,26 @@ def test_host_pipeline_matches_single_call():
     tf.tf_device_status()
     got = {"y": hy.view(torch.uint16).numpy(), "mean": hmean.numpy(), "rstd": hrstd.numpy()}
     assert not parity.check(w, data, got, parity.run_oracle(w, data))
+
+
+def test_host_pipeline_overlapped_calls_keep_their_results_apart():
+    """Consecutive calls without a join reuse the device staging buffers block by block: each call's host outputs must
+    still be exactly its own result."""
+    from paper_2512_09196_b200.host import HostPipeline
+    dev = torch.device("cuda", 0)
+    pin = lambda a: torch.from_numpy(a).view(torch.bfloat16).pin_memory()
+    cases = []
+    for seed in (11, 12, 13):
+        w = inputs.Workload(f"host_case_{seed}", "rmsnorm", inputs.BF16, 2051, 4096, seed=seed, x_std=float(seed - 9), eps=1e-6)
+        data = w.generate()
+        cases.append((w, data, pin(data["x"]), pin(data["w"]), torch.empty(w.rows, w.cols, dtype=torch.bfloat16).pin_memory()))
+    pipe = HostPipeline("rmsnorm", 2051, 4096, torch.bfloat16, dev, blocks=7)
+    dps = [{"w": torch.empty(4096, dtype=torch.bfloat16, device=dev)} for _ in cases]
+    for rep in range(2):
+        for (w, data, hx, hw, hy), dp in zip(cases, dps):
+            pipe.run(hx, hy, {"w": hw}, dp, w.eps, join=False)
+    pipe.finish()
+    torch.cuda.synchronize()
+    tf.tf_device_status()
+    for w, data, hx, hw, hy in cases:
+        assert not parity.check(w, data, {"y": hy.view(torch.uint16).numpy()}, parity.run_oracle(w, data)), w.name
