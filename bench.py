@@ -472,12 +472,14 @@ def run_vecmat_table(args):
         reps = max(20, min(200, int(0.05 / (nbytes / 5e12))))
         us_auto = timed(lambda: tf.tf_bvecmat_fwd(A, B, C), reps)
         grid, kvec = {}, w.K * w.elem_size // 16
+        ks_ok = lambda th: th >= 128
         if not args.no_tune:
             for threads in (128, 256, 512, 1024):
                 for lanes in (4, 8, 16, 32):
                     if w.dt == inputs.F32 and lanes <= kvec and (lanes == 32 or kvec <= 16 * lanes):
                         for rows in (1, 2, 4):
-                            grid[f"{threads},{lanes},{rows},0"] = timed(lambda: tf.tf_bvecmat_fwd(A, B, C, threads, lanes, rows), reps)
+                            for ks in ((1, 2, 4) if lanes == 32 and kvec >= 1024 and ks_ok(threads) else (1,)):
+                                grid[f"{threads},{lanes},{rows},{ks}"] = timed(lambda: tf.tf_bvecmat_fwd(A, B, C, threads, lanes, rows, ks), reps)
                 if w.dt == inputs.BF16 and threads < 1024:
                     for rows in (16, 32):
                         for ks in (1, 2, 4, 8):

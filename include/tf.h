@@ -161,7 +161,8 @@ tf_status tf_tune_add(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);
  *   lanes    per row group on the plain path (4, 8, 16 or 32); bf16 with lanes = 0 takes the tensor-core path;
  *   rows     consecutive n that share one load of the A[m,:] pieces: 1, 2 or 4 per lane group on the plain path,
  *            16 or 32 per warp on the tensor-core path;
- *   ksplit   warps of a CTA that share a row group along k on the tensor-core path (1, 2, 4 or 8).
+ *   ksplit   warps of a CTA that share a row group along k (1, 2, 4 or 8; on the plain path only with lanes = 32,
+ *            and never more than threads / 32).
  * 16-byte aligned A and B with K * sizeof(element) a multiple of 16 take a vector path, anything else a scalar one.
  * Errors: TF_ERR_INVALID_ARG for a null pointer with M*N > 0, K <= 0, an unknown element type or a knob outside its
  * set; TF_ERR_UNSUPPORTED when the grid would exceed 2^31 - 1 CTAs.  Asynchronous on cuda_stream; allocates nothing;

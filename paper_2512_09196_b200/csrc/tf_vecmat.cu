@@ -20,15 +20,22 @@ namespace tf {
 namespace {
 
 // Lane group of LANES lanes, R rows, U vectors per row and step.  All loops have warp-uniform trip counts.
-template <int DT, int LANES, int R, int U>
+// ksplit > 1 (LANES = 32 only): that many warps of the CTA share a row group, each taking every ksplit-th step, and
+// combine through shared memory -- for few, long rows, which would otherwise leave the SMs short of warps.
+// KS = false compiles the split away (constant strides matter for the short rows, which issue everything at once).
+template <int DT, int LANES, int R, int U, bool KS>
 __global__ void __launch_bounds__(1024) k_vecmat(const uint4* __restrict__ A, const uint4* __restrict__ B,
-                                                 typename Elem<DT>::scalar* __restrict__ C, int64_t N, int kvec, int tiles_per_m, int64_t tiles) {
+                                                 typename Elem<DT>::scalar* __restrict__ C, int64_t N, int kvec, int tiles_per_m, int64_t tiles,
+                                                 int ksplit_arg) {
     using P = Pairs<DT>;
     constexpr int NP = P::NP;
+    __shared__ float part[KS ? 32 : 1][R];
+    const int ksplit = KS ? ksplit_arg : 1;
     pdl_wait();
     pdl_trigger();
     const int lane = threadIdx.x % LANES;
-    const int64_t tile = static_cast<int64_t>(blockIdx.x) * (blockDim.x / LANES) + threadIdx.x / LANES;
+    const int group = threadIdx.x / LANES, kw = group % ksplit;
+    const int64_t tile = static_cast<int64_t>(blockIdx.x) * (blockDim.x / LANES / ksplit) + group / ksplit;
     const bool tile_live = tile < tiles;                          // every lane runs the loop: shuffles need the whole warp
     const int64_t m = tile_live ? tile / tiles_per_m : 0;
     const int64_t n0 = tile_live ? (tile - m * tiles_per_m) * R : 0;
@@ -43,7 +50,7 @@ __global__ void __launch_bounds__(1024) k_vecmat(const uint4* __restrict__ A, co
     for (int r = 0; r < R; ++r) acc[r] = f2(0.f);
     const uint4 zero = make_uint4(0, 0, 0, 0);
 #pragma unroll(R == 2 ? 2 : 1)                                  // measured: R = 2 gains from a second step in flight, R = 1 and 4 lose occupancy
-    for (int v0 = lane; v0 < kvec; v0 += LANES * U) {
+    for (int v0 = kw * LANES * U + lane; v0 < kvec; v0 += LANES * U * ksplit) {
         uint4 bv[R][U], av[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -66,10 +73,26 @@ __global__ void __launch_bounds__(1024) k_vecmat(const uint4* __restrict__ A, co
             }
         }
     }
+    float dot[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const float dot = group_reduce<SumOp, LANES>(hsum(acc[r]));
-        if (lane == 0 && r < n_left) C[out + r] = Elem<DT>::from_float(dot);
+    for (int r = 0; r < R; ++r) dot[r] = group_reduce<SumOp, LANES>(hsum(acc[r]));
+    if (!KS) {
+        if (lane == 0) {
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                if (r < n_left) C[out + r] = Elem<DT>::from_float(dot[r]);
+        }
+        return;
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) part[group][r] = dot[r];
+    }
+    __syncthreads();
+    if (kw == 0 && lane < n_left) {
+        float sum = 0.f;
+        for (int i = 0; i < ksplit; ++i) sum += part[group + i][lane];
+        C[out + lane] = Elem<DT>::from_float(sum);
     }
 }
 
@@ -215,38 +238,50 @@ int64_t warps_wanted(int sms) { return 4LL * 64 * sms; }
 
 
 template <int DT, int LANES, int R>
-cudaError_t launch_plain_lr(int threads, cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t kvec) {
+cudaError_t launch_plain_lr(int threads, int ksplit, cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t kvec) {
     constexpr int U = R == 1 ? 4 : R == 2 ? 2 : 1;
     using S = typename Elem<DT>::scalar;
     const int64_t tiles_per_m = (N + R - 1) / R, tiles = M * tiles_per_m;
     if (tiles_per_m > 0x7FFFFFFF || kvec > 0x7FFFFFF0) return cudaErrorInvalidConfiguration;
-    const int gpc = threads / LANES;
-    return launch_pdl(k_vecmat<DT, LANES, R, U>, (tiles + gpc - 1) / gpc, threads, st, static_cast<const uint4*>(A),
-                      static_cast<const uint4*>(B), static_cast<S*>(C), N, static_cast<int>(kvec), static_cast<int>(tiles_per_m), tiles);
+    if (LANES < 32) ksplit = 1;
+    while (ksplit > 1 && ksplit * 32 > threads) ksplit /= 2;
+    const int gpc = threads / LANES / ksplit;
+    if (LANES == 32 && ksplit > 1)
+        return launch_pdl(k_vecmat<DT, LANES, R, U, (LANES == 32)>, (tiles + gpc - 1) / gpc, threads, st, static_cast<const uint4*>(A),
+                          static_cast<const uint4*>(B), static_cast<S*>(C), N, static_cast<int>(kvec), static_cast<int>(tiles_per_m), tiles, ksplit);
+    return launch_pdl(k_vecmat<DT, LANES, R, U, false>, (tiles + gpc - 1) / gpc, threads, st, static_cast<const uint4*>(A),
+                      static_cast<const uint4*>(B), static_cast<S*>(C), N, static_cast<int>(kvec), static_cast<int>(tiles_per_m), tiles, 1);
 }
 
 template <int DT, int LANES>
-cudaError_t launch_plain_l(int rows, int threads, cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t kvec) {
+cudaError_t launch_plain_l(int rows, int threads, int ksplit, cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N,
+                           int64_t kvec) {
     switch (rows) {
-        case 1: return launch_plain_lr<DT, LANES, 1>(threads, st, A, B, C, M, N, kvec);
-        case 2: return launch_plain_lr<DT, LANES, 2>(threads, st, A, B, C, M, N, kvec);
-        default: return launch_plain_lr<DT, LANES, 4>(threads, st, A, B, C, M, N, kvec);
+        case 1: return launch_plain_lr<DT, LANES, 1>(threads, ksplit, st, A, B, C, M, N, kvec);
+        case 2: return launch_plain_lr<DT, LANES, 2>(threads, ksplit, st, A, B, C, M, N, kvec);
+        default: return launch_plain_lr<DT, LANES, 4>(threads, ksplit, st, A, B, C, M, N, kvec);
     }
 }
 
 template <int DT>
-cudaError_t launch_plain(int lanes, int rows, int threads, cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N,
-                         int64_t kvec) {
+cudaError_t launch_plain(int lanes, int rows, int ksplit, int threads, cudaStream_t st, const void* A, const void* B, void* C, int64_t M,
+                         int64_t N, int64_t kvec) {
     const int sms = sm_count();
     // Measured on the K sweep: rows of up to 4 KiB run best with two rows per group sharing each A load and two
     // vectors per lane and step; longer rows with one row per group and four vectors in flight per lane.
     if (lanes == 0) lanes = kvec <= 8 ? 4 : kvec <= 16 ? 8 : kvec <= 32 ? 16 : 32;
     if (rows == 0) rows = (kvec <= 256 && N >= 2 && M * ((N + 1) / 2) * lanes / 32 >= warps_wanted(sms) / 4) ? 2 : 1;
+    if (ksplit == 0) {                                            // few long rows: cut k until about one wave of warps exists
+        const int64_t groups = M * ((N + rows - 1) / rows);
+        const int64_t steps = kvec / (32 * (rows == 1 ? 4 : rows == 2 ? 2 : 1));
+        ksplit = 1;
+        while (lanes == 32 && ksplit < 8 && ksplit * 64 <= threads && groups * ksplit < 64LL * sms && steps >= 4 * ksplit) ksplit *= 2;
+    }
     switch (lanes) {
-        case 4: return launch_plain_l<DT, 4>(rows, threads, st, A, B, C, M, N, kvec);
-        case 8: return launch_plain_l<DT, 8>(rows, threads, st, A, B, C, M, N, kvec);
-        case 16: return launch_plain_l<DT, 16>(rows, threads, st, A, B, C, M, N, kvec);
-        default: return launch_plain_l<DT, 32>(rows, threads, st, A, B, C, M, N, kvec);
+        case 4: return launch_plain_l<DT, 4>(rows, threads, ksplit, st, A, B, C, M, N, kvec);
+        case 8: return launch_plain_l<DT, 8>(rows, threads, ksplit, st, A, B, C, M, N, kvec);
+        case 16: return launch_plain_l<DT, 16>(rows, threads, ksplit, st, A, B, C, M, N, kvec);
+        default: return launch_plain_l<DT, 32>(rows, threads, ksplit, st, A, B, C, M, N, kvec);
     }
 }
 
@@ -308,8 +343,8 @@ extern "C" tf_status tf_bvecmat_fwd(const void* A, const void* B, void* C, int64
     if (al16(A) && al16(B) && (K * es) % 16 == 0) {
         const int64_t kvec = K * es / 16;
         if (tensor) e = launch_mma(rows, ksplit, threads, st, A, B, C, M, N, kvec);
-        else if (dt == DT_F32) e = launch_plain<DT_F32>(lanes, rows, threads, st, A, B, C, M, N, kvec);
-        else e = launch_plain<DT_BF16>(lanes, rows, threads, st, A, B, C, M, N, kvec);
+        else if (dt == DT_F32) e = launch_plain<DT_F32>(lanes, rows, ksplit, threads, st, A, B, C, M, N, kvec);
+        else e = launch_plain<DT_BF16>(lanes, rows, ksplit, threads, st, A, B, C, M, N, kvec);
     } else {
         const int64_t grid = (nrows + threads / 32 - 1) / (threads / 32);
         if (grid > 0x7FFFFFFF) return TF_ERR_UNSUPPORTED;

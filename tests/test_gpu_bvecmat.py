@@ -50,6 +50,15 @@ def test_every_geometry(dt, lanes):
                 check(inputs.VecMat(f"t_{M}x{N}x{K}", dt, M, N, K, seed=K + lanes), threads, lanes, rows=rows)
 
 
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_every_k_split_of_the_plain_path(dt):
+    for ksplit in (1, 2, 4, 8):
+        for threads in (64, 256, 1024):
+            for rows in (1, 2, 4):
+                for M, N, K in ((3, 37, 8), (2, 65, 200), (5, 129, 1032), (1, 19, 8200), (1, 1, 32768)):
+                    check(inputs.VecMat(f"t_{M}x{N}x{K}", dt, M, N, K, seed=K + ksplit), threads, 32, ksplit=ksplit, rows=rows)
+
+
 def test_every_k_split_of_the_tensor_core_path():
     for ksplit in (1, 2, 4, 8):
         for threads in (128, 256, 512):
