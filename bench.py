@@ -668,6 +668,38 @@ def run_case(args):
         print(json.dumps({"case": w.name, "knobs": knobs, "launches": args.steps, "us_per_launch": us,
                           "gbs": w.algorithmic_bytes() / us / 1e3}))
         return
+    if parts[0] == "addnorm":                 # addnorm:op:dtype:rows:cols -- the fused residual add + norm, heuristic plan
+        op, dts, rows, cols = parts[1], parts[2], int(parts[3]), int(parts[4])
+        dt = inputs.F32 if dts == "f32" else inputs.BF16
+        w = inputs.Workload(f"case_add_{op}_{dts}_{rows}x{cols}", op, dt, rows, cols, seed=cols, eps=1e-5 if op == "layernorm" else 1e-6)
+        data = w.generate()
+        conv = (lambda t: t.view(torch.bfloat16)) if dt == inputs.BF16 else (lambda t: t)
+        x = conv(torch.from_numpy(data["x"])).cuda()
+        r = conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols + 1, 7, 0.0, 1.0))).cuda()
+        g = conv(torch.from_numpy(data["gamma"] if op == "layernorm" else data["w"])).cuda()
+        b = conv(torch.from_numpy(data["beta"])).cuda() if op == "layernorm" else None
+        h, y = torch.empty_like(x), torch.empty_like(x)
+        if not args.no_tune:
+            tf.tf_tune_add(op, rows, cols, dt)
+        a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def call():
+            if op == "layernorm":
+                tf.tf_add_layernorm_fwd(x, r, g, b, w.eps, h=h, y=y, want_stats=False)
+            else:
+                tf.tf_add_rmsnorm_fwd(x, r, g, w.eps, h=h, y=y)
+        for _ in range(max(1, args.warmup)):
+            call()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(args.steps):
+            call()
+        e.record()
+        torch.cuda.synchronize()
+        us = 1e3 * a.elapsed_time(e) / args.steps
+        nbytes = 4 * rows * cols * w.elem_size + (2 if op == "layernorm" else 1) * cols * w.elem_size
+        print(json.dumps({"case": w.name, "launches": args.steps, "us_per_launch": us, "gbs": nbytes / us / 1e3}))
+        return
     if parts[0] == "config":
         w = inputs.config(int(parts[1]))
         if len(parts) > 2:
@@ -700,7 +732,7 @@ def main():
     ap.add_argument("--filter", default=None)
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
-    ap.add_argument("--case", default=None, help="op:dtype:rows:cols or config:<i>[:rows] -- a few launches of one shape")
+    ap.add_argument("--case", default=None, help="op:dtype:rows:cols, config:<i>[:rows], vecmat:..., addnorm:op:dtype:rows:cols -- a few launches of one shape")
     ap.add_argument("--plan", default=None, help="with --case: force this launch plan")
     args = ap.parse_args()
     if args.impl == "reference":
