@@ -63,6 +63,10 @@ def _load():
         lib.oracle_bvecmat.restype = i32
         lib.oracle_softmax_len.argtypes = [vp, vp, vp, vp, i64, i64, i32, i32]
         lib.oracle_softmax_len.restype = i32
+        lib.oracle_log_softmax.argtypes = [vp, vp, vp, i64, i64, i32, i32]
+        lib.oracle_log_softmax.restype = i32
+        lib.oracle_softmax_bwd.argtypes = [vp, vp, vp, vp, vp, i64, i64, i32, i32]
+        lib.oracle_softmax_bwd.restype = i32
         lib.oracle_add.argtypes = [vp, vp, vp, vp, i64, i32]
         lib.oracle_add.restype = i32
         lib.oracle_bf16_from_double.argtypes = [vp, vp, i64]
@@ -107,6 +111,31 @@ def softmax_len(x: np.ndarray, lengths: np.ndarray, dt: int, want64: bool = Fals
     if _load().oracle_softmax_len(_p(x), _p(lengths), _p(y), _p(y64), rows, cols, dt, nthreads):
         raise ValueError("oracle_softmax_len: bad argument")
     return (y, y64) if want64 else y
+
+
+def log_softmax(x: np.ndarray, dt: int, want64: bool = False, nthreads: int = 1):
+    """Row log-softmax.  Returns ``y`` (and the unrounded float64 result if ``want64``)."""
+    _check(x, dt, "x")
+    rows, cols = x.shape
+    y = np.empty_like(x)
+    y64 = np.empty((rows, cols), np.float64) if want64 else None
+    if _load().oracle_log_softmax(_p(x), _p(y), _p(y64), rows, cols, dt, nthreads):
+        raise ValueError("oracle_log_softmax: bad argument")
+    return (y, y64) if want64 else y
+
+
+def softmax_bwd(y: np.ndarray, dy: np.ndarray, dt: int, want64: bool = False, nthreads: int = 1):
+    """Softmax backward ``dx = y * (dy - sum(y * dy))`` per row.  Returns ``dx`` plus ``(dx64, scale64)`` if ``want64``."""
+    _check(y, dt, "y"), _check(dy, dt, "dy")
+    if y.shape != dy.shape:
+        raise ValueError("y and dy must have the same shape")
+    rows, cols = y.shape
+    dx = np.empty_like(y)
+    dx64 = np.empty((rows, cols), np.float64) if want64 else None
+    sc = np.empty((rows, cols), np.float64) if want64 else None
+    if _load().oracle_softmax_bwd(_p(y), _p(dy), _p(dx), _p(dx64), _p(sc), rows, cols, dt, nthreads):
+        raise ValueError("oracle_softmax_bwd: bad argument")
+    return (dx, dx64, sc) if want64 else dx
 
 
 def layernorm(x, gamma, beta, eps: float, dt: int, want64: bool = False, nthreads: int = 1):

@@ -31,6 +31,11 @@
 // Softmax with per-row valid lengths (row r is normalised over its first len[r] entries, the rest of the
 // output row is +0, the rest of the input row is never read) is pinned by equality with the plain softmax on
 // a copy whose tails hold -inf, by len = cols, len = 0, len = 1, and by NaN-filled tails leaving no trace.
+// Log-softmax (y = (x - m) - ln sum exp(x - m)) is pinned by the logarithm of the pinned softmax, by
+// sum exp(y) = 1, exact shift invariance, the two-element closed form -log1p(e^(b-a)), uniform rows (-ln n),
+// masked entries (-inf) and torch's float64 routine.  The softmax backward pass (dx = y (dy - sum y dy)) is
+// pinned by the analytic Jacobian on one-hot dy, by central differences of the pinned softmax in double,
+// by dx = 0 for constant dy, by linearity in dy and by torch's float64 autograd.
 // tf_tune has
 // no oracle function here: which candidate wins is hardware-dependent ("parity unpinned" for the
 // winner's identity; its output is checked like any other launch).
@@ -236,6 +241,55 @@ int oracle_softmax_len(const void* x, const int32_t* len, void* y, double* y64, 
         for (int64_t j = n; j < cols; ++j) {
             if (y64) y64[r * cols + j] = 0.0;
             if (y) store(y, r * cols + j, dt, 0.0);
+        }
+    });
+    return 0;
+}
+
+// Log-softmax over the last axis:  y_j = (x_j - m) - ln sum_k exp(x_k - m), m = max x.  Entries with x_j = -inf
+// give y_j = -inf; a fully masked row gives -inf everywhere (the logarithm of the all-zero reading of softmax).
+int oracle_log_softmax(const void* x, void* y, double* y64, int64_t rows, int64_t cols, int dt, int nthreads) {
+    if (bad(rows, cols, dt) || !x) return -1;
+    for_rows(rows, nthreads, [=](int64_t r) {
+        const int64_t base = r * cols;
+        double m = -std::numeric_limits<double>::infinity();
+        for (int64_t j = 0; j < cols; ++j) {
+            const double v = load(x, base + j, dt);
+            if (v > m || std::isnan(v)) m = v;
+        }
+        double S = 0.0;
+        if (m != -std::numeric_limits<double>::infinity())
+            for (int64_t j = 0; j < cols; ++j) S += std::exp(load(x, base + j, dt) - m);
+        const double lnS = std::log(S);                      // S >= 1 for a live row
+        for (int64_t j = 0; j < cols; ++j) {
+            const double v = (m == -std::numeric_limits<double>::infinity()) ? m : (load(x, base + j, dt) - m) - lnS;
+            if (y64) y64[base + j] = v;
+            if (y) store(y, base + j, dt, v);
+        }
+    });
+    return 0;
+}
+
+// Softmax backward:  dx_j = y_j * (dy_j - sum_k y_k dy_k), y the forward output as stored, dy the incoming
+// gradient.  scale64 (nullable) receives |y_j| * (|dy_j| + sum_k |y_k dy_k|), the quantity an error bound for the
+// cancelling difference is stated against.
+int oracle_softmax_bwd(const void* y, const void* dy, void* dx, double* dx64, double* scale64, int64_t rows, int64_t cols,
+                       int dt, int nthreads) {
+    if (bad(rows, cols, dt) || !y || !dy) return -1;
+    for_rows(rows, nthreads, [=](int64_t r) {
+        const int64_t base = r * cols;
+        double s = 0.0, sa = 0.0;
+        for (int64_t j = 0; j < cols; ++j) {
+            const double p = load(y, base + j, dt) * load(dy, base + j, dt);
+            s += p;
+            sa += std::fabs(p);
+        }
+        for (int64_t j = 0; j < cols; ++j) {
+            const double yj = load(y, base + j, dt), gj = load(dy, base + j, dt);
+            const double v = yj * (gj - s);
+            if (dx64) dx64[base + j] = v;
+            if (scale64) scale64[base + j] = std::fabs(yj) * (std::fabs(gj) + sa);
+            if (dx) store(dx, base + j, dt, v);
         }
     });
     return 0;
