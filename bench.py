@@ -639,6 +639,57 @@ def run_softmaxlen_table(args):
     (out_dir / "table_softmaxlen.json").write_text(json.dumps(rows_out, indent=1))
 
 
+def run_softmax_variants_table(args):
+    """Log-softmax forward and softmax backward: achieved bandwidth of their algorithmic bytes, torch's routines as context."""
+    import torch
+    import paper_2512_09196_b200 as tf
+    from paper_2512_09196_b200 import inputs
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak()
+    out_dir = ROOT / "gpurun_out"
+    out_dir.mkdir(exist_ok=True)
+    shapes = [(inputs.BF16, 16384, 8192), (inputs.BF16, 32768, 4096), (inputs.F32, 65536, 1024), (inputs.BF16, 524288, 256),
+              (inputs.BF16, 8192, 32768), (inputs.F32, 4096, 32768), (inputs.F32, 2048, 131072)]
+    rows_out = []
+    for dt, rows, cols in shapes:
+        es = inputs.ELEM_SIZE[dt]
+        conv = (lambda t: t.view(torch.bfloat16)) if dt == inputs.BF16 else (lambda t: t)
+        sets = max(2, min(8, int((1 << 30) // (3 * rows * cols * es))))
+        xs = [conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols, 0, 0.0, 3.0))).cuda() for _ in range(sets)]
+        gs = [conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols + 1, 1, 0.0, 1.0))).cuda() for _ in range(sets)]
+        ys = [torch.softmax(x.float(), dim=1).to(x.dtype) for x in xs]
+        outs = [torch.empty_like(x) for x in xs]
+
+        def timed(fn, reps):
+            for k in range(3):
+                fn(k % sets)
+            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for k in range(reps):
+                fn(k % sets)
+            e.record()
+            torch.cuda.synchronize()
+            return 1e3 * a.elapsed_time(e) / reps
+
+        reps = max(10, min(200, int(0.05 / (3 * rows * cols * es / 5e12))))
+        for op, nbytes, ours, lib in (
+                ("log_softmax_fwd", 2 * rows * cols * es, lambda k: tf.tf_log_softmax_fwd(xs[k], outs[k]),
+                 lambda k: torch.log_softmax(xs[k], dim=1, out=outs[k]) if False else torch.log_softmax(xs[k], dim=1)),
+                ("softmax_bwd", 3 * rows * cols * es, lambda k: tf.tf_softmax_bwd(ys[k], gs[k], outs[k]),
+                 lambda k: torch._softmax_backward_data(gs[k], ys[k], 1, ys[k].dtype))):
+            us, us_lib = timed(ours, reps), timed(lib, max(5, reps // 2))
+            row = {"op": op, "dtype": "f32" if dt == inputs.F32 else "bf16", "rows": rows, "cols": cols, "bytes": nbytes, "us": us,
+                   "gbs": nbytes / us / 1e3, f"pct_of_{peak_kind}_{peak:.0f}": 100 * nbytes / us / 1e3 / peak, "torch_us": us_lib,
+                   "torch_gbs": nbytes / us_lib / 1e3}
+            rows_out.append(row)
+            print(json.dumps(row), flush=True)
+        tf.tf_device_status()
+        del xs, gs, ys, outs
+        torch.cuda.empty_cache()
+    (out_dir / "table_softmaxvariants.json").write_text(json.dumps(rows_out, indent=1))
+
+
 def run_case(args):
     """A few launches of one op/shape (for profiler captures): --case op:dtype:rows:cols or --case config:<i>[:rows]."""
     import torch
@@ -728,7 +779,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm", "softmaxlen"], default=None)
+    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm", "softmaxlen", "softmaxvariants"], default=None)
     ap.add_argument("--filter", default=None)
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
@@ -751,6 +802,8 @@ def main():
         return run_addnorm_table(args)
     if args.table == "softmaxlen":
         return run_softmaxlen_table(args)
+    if args.table == "softmaxvariants":
+        return run_softmax_variants_table(args)
     if args.table:
         return run_table(args)
     run_ours(args)

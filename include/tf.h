@@ -131,6 +131,20 @@ tf_status tf_sin_fwd(const void* x, void* y, int64_t n, tf_dtype dt, int threads
  * Errors and stream behaviour as tf_softmax_fwd, plus TF_ERR_INVALID_ARG for a null len.  Allocates nothing. */
 tf_status tf_softmax_len_fwd(const void* x, const int32_t* len, void* y, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
 
+/* ---- log-softmax forward, softmax backward ----------------------------------------------------------------- */
+
+/* y_j = (x_j - m) - ln sum_k exp(x_k - m), m = max_k x_k, over the last axis of x [rows, cols].  Entries with x_j = -inf
+ * give -inf; a row that is -inf throughout gives -inf throughout (the logarithm of the all-zero reading of softmax).
+ * fp32 arithmetic, one rounding to the storage type.  y may alias x.  The paper has no counterpart. */
+tf_status tf_log_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
+
+/* dx_j = y_j * (dy_j - sum_k y_k dy_k): the backward pass of softmax from its stored output y and the incoming
+ * gradient dy, all [rows, cols] of one element type; fp32 arithmetic, one rounding.  dx may alias y or dy.
+ * Both calls: device pointers, asynchronous on cuda_stream, allocate nothing; TF_ERR_INVALID_ARG for a null pointer
+ * with rows > 0, cols <= 0 or an unknown element type; rows = 0 is a no-op.  16-byte aligned tensors whose rows are
+ * whole 16-byte vectors of up to 32-128 KiB (by op and type) are held in registers; anything else runs scalar passes. */
+tf_status tf_softmax_bwd(const void* y, const void* dy, void* dx, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
+
 /* ---- fused residual add + norm ------------------------------------------------------------------------ */
 
 /* h = x + r (fp32 add, ONE rounding to the storage type), then the LayerNorm / RMSNorm defined above applied to that

@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_status_string",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
 
@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.tf_add_rmsnorm_fwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, f32, i32, vp]
         L.tf_tune_add.argtypes = [i32, i64, i64, i32]
         L.tf_softmax_len_fwd.argtypes = [vp, vp, vp, i64, i64, i32, vp]
+        L.tf_log_softmax_fwd.argtypes = [vp, vp, i64, i64, i32, vp]
+        L.tf_softmax_bwd.argtypes = [vp, vp, vp, i64, i64, i32, vp]
         L.tf_bvecmat_fwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp]
         L.tf_sin_fwd.argtypes = [vp, vp, i64, i32, i32, i32, vp]
         L.tf_tune_like.argtypes = [i32, vp, vp, vp, i64, i64, i32]
@@ -73,7 +75,7 @@ def lib() -> ctypes.CDLL:
         L.tf_clear_cache.restype = None
         L.tf_launch_count.argtypes = []
         L.tf_launch_count.restype = i64
-        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd",
+        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd",
                      "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice",
                      "tf_candidate_count", "tf_candidate"):
             getattr(L, name).restype = i32
@@ -153,6 +155,33 @@ def tf_softmax_len_fwd(x, lengths, y=None):
         _ok(lib().tf_softmax_len_fwd(x.data_ptr(), lengths.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)),
             "tf_softmax_len_fwd")
     return y
+
+
+def tf_log_softmax_fwd(x, y=None):
+    """Log-softmax over the last axis of a contiguous CUDA [rows, cols] tensor (fp32 or bf16); ``y`` may alias ``x``."""
+    import torch
+    _check2d(x)
+    if y is None:
+        y = torch.empty_like(x)
+    rows, cols = x.shape
+    with _on_device(x):
+        _ok(lib().tf_log_softmax_fwd(x.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)), "tf_log_softmax_fwd")
+    return y
+
+
+def tf_softmax_bwd(y, dy, dx=None):
+    """Softmax backward ``dx = y * (dy - sum(y * dy, -1))`` from the stored forward output ``y`` and the gradient ``dy``."""
+    import torch
+    _check2d(y, "y")
+    _check2d(dy, "dy")
+    if dy.shape != y.shape or dy.dtype != y.dtype:
+        raise ValueError("dy must match y")
+    if dx is None:
+        dx = torch.empty_like(y)
+    rows, cols = y.shape
+    with _on_device(y):
+        _ok(lib().tf_softmax_bwd(y.data_ptr(), dy.data_ptr(), dx.data_ptr(), rows, cols, _dt(y), _stream(y)), "tf_softmax_bwd")
+    return dx
 
 
 def tf_softmax_fwd_noalloc(x, y):

@@ -1,0 +1,413 @@
+// Two more row-wise reduce-then-normalise ops on the softmax family:
+//   log-softmax forward   y_j  = (x_j - m) - ln sum_k exp(x_k - m),  m = max_k x_k
+//   softmax backward      dx_j = y_j * (dy_j - sum_k y_k dy_k)
+// One kernel shape serves both: a CTA owns a row and holds it in registers (VPT 16-byte vectors per thread, loaded at
+// once), reduces across the CTA, finishes and stores -- one read of every input element, one write of every output
+// element.  Rows of up to 2 KiB are owned by lane groups instead (several rows per warp).  Rows beyond what 1024 threads
+// hold in 32 fp32 values each (32 KiB for the bf16 backward pass up to 128 KiB for the fp32 log-softmax) are streamed in
+// passes of 16-byte loads, the later passes from L2; unaligned tensors and odd widths take scalar passes.
+//
+// Log-softmax keeps x - m as a difference (exact for bf16 inputs, one rounding for fp32) and subtracts ln S computed
+// from S = sum 2^((x - m) log2 e) with the accurate logarithm; the term of the maximum is exactly 1, so S >= 1 and its
+// fp32 summation error is a few 2^-24 absolute, which is the absolute part of the tolerance the tests use.
+#include <algorithm>
+
+#include "../../include/tf.h"
+#include "tf_common.cuh"
+
+namespace tf {
+namespace {
+
+constexpr int kOpLogSoftmax = 0, kOpSoftmaxBwd = 1;
+
+// fp32 values a thread holds for its share of a row; up to 32 of them leave room for 1024 threads, up to 64 for 512.
+template <int WHICH, int DT, int VPT> constexpr int row2_floats() { return VPT * Elem<DT>::NE * (WHICH == kOpSoftmaxBwd ? 2 : 1); }
+template <int WHICH, int DT, int VPT> constexpr int row2_max_threads() { return row2_floats<WHICH, DT, VPT>() <= 32 ? 1024 : 512; }
+
+template <int WHICH, int DT, int VPT>
+__global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2(const uint4* __restrict__ in0, const uint4* __restrict__ in1, uint4* __restrict__ out,
+                                               int64_t rows, int nvec) {
+    using E = Elem<DT>;
+    constexpr int NE = E::NE;
+    __shared__ float buf[2][32];
+    pdl_wait();
+    pdl_trigger();
+    const int T = blockDim.x, t = threadIdx.x;
+    const int64_t row = blockIdx.x;
+    if (row >= rows) return;
+    const uint4* a = in0 + row * nvec + t;
+    uint4* o = out + row * nvec + t;
+    bool valid[VPT];
+    uint4 ra[VPT];
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+        valid[v] = t + v * T < nvec;
+        ra[v] = valid[v] ? ld_stream(a + v * T) : make_uint4(0, 0, 0, 0);
+    }
+    if constexpr (WHICH == kOpLogSoftmax) {
+        float m = kNegInf;
+#pragma unroll
+        for (int v = 0; v < VPT; ++v)
+            if (valid[v]) m = fmaxf(m, vec_max<DT>(ra[v]));
+        m = cta_reduce<MaxOp>(m, buf[0]);
+        float d[VPT][NE];
+        float s = 0.f;
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            float x[NE];
+            E::unpack(ra[v], x);
+#pragma unroll
+            for (int i = 0; i < NE; ++i) {
+                d[v][i] = x[i] - m;                                       // -inf for masked entries; NaN only if the whole row is masked
+                if (valid[v]) s += ex2_ftz(d[v][i] * kLog2e);             // 2^0 = 1 exactly for the maximum
+            }
+        }
+        s = cta_reduce<SumOp>(s, buf[1]);
+        const float lns = logf(s);
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            float y[NE];
+#pragma unroll
+            for (int i = 0; i < NE; ++i) y[i] = (m == kNegInf) ? kNegInf : d[v][i] - lns;
+            if (valid[v]) st_stream(o + v * T, E::pack(y));
+        }
+    } else {
+        const uint4* b = in1 + row * nvec + t;
+        float y[VPT][NE], g[VPT][NE];
+        float s = 0.f;
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            const uint4 rb = valid[v] ? ld_stream(b + v * T) : make_uint4(0, 0, 0, 0);
+            E::unpack(ra[v], y[v]);
+            E::unpack(rb, g[v]);
+#pragma unroll
+            for (int i = 0; i < NE; ++i) s = fmaf(y[v][i], g[v][i], s);    // absent vectors hold zeros
+        }
+        s = cta_reduce<SumOp>(s, buf[0]);
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            float dx[NE];
+#pragma unroll
+            for (int i = 0; i < NE; ++i) dx[i] = y[v][i] * (g[v][i] - s);
+            if (valid[v]) st_stream(o + v * T, E::pack(dx));
+        }
+    }
+}
+
+// Short rows (up to 2 KiB): a group of LANES lanes owns a row, a CTA of 128 threads covers 128 / LANES consecutive
+// rows, reductions are shuffles.  Every lane runs every step (the shuffles need the whole warp); rows past the end
+// are loaded as zeros and not stored.
+template <int WHICH, int DT, int LANES, int VPT>
+__global__ void __launch_bounds__(128) k_row2_group(const uint4* __restrict__ in0, const uint4* __restrict__ in1, uint4* __restrict__ out,
+                                                    int64_t rows, int nvec) {
+    using E = Elem<DT>;
+    constexpr int NE = E::NE;
+    pdl_wait();
+    pdl_trigger();
+    const int lane = threadIdx.x % LANES;
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x / LANES) + threadIdx.x / LANES;
+    const bool live = row < rows;
+    const int64_t base = (live ? row : 0) * nvec + lane;
+    bool valid[VPT];
+    uint4 ra[VPT];
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+        valid[v] = live && lane + v * LANES < nvec;
+        ra[v] = valid[v] ? ld_stream(in0 + base + v * LANES) : make_uint4(0, 0, 0, 0);
+    }
+    if constexpr (WHICH == kOpLogSoftmax) {
+        float m = kNegInf;
+#pragma unroll
+        for (int v = 0; v < VPT; ++v)
+            if (valid[v]) m = fmaxf(m, vec_max<DT>(ra[v]));
+        m = group_reduce<MaxOp, LANES>(m);
+        float d[VPT][NE];
+        float s = 0.f;
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            float x[NE];
+            E::unpack(ra[v], x);
+#pragma unroll
+            for (int i = 0; i < NE; ++i) {
+                d[v][i] = x[i] - m;
+                if (valid[v]) s += ex2_ftz(d[v][i] * kLog2e);
+            }
+        }
+        s = group_reduce<SumOp, LANES>(s);
+        const float lns = logf(s);
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            float y[NE];
+#pragma unroll
+            for (int i = 0; i < NE; ++i) y[i] = (m == kNegInf) ? kNegInf : d[v][i] - lns;
+            if (valid[v]) st_stream(out + base + v * LANES, E::pack(y));
+        }
+    } else {
+        float y[VPT][NE], g[VPT][NE];
+        float s = 0.f;
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            const uint4 rb = valid[v] ? ld_stream(in1 + base + v * LANES) : make_uint4(0, 0, 0, 0);
+            E::unpack(ra[v], y[v]);
+            E::unpack(rb, g[v]);
+#pragma unroll
+            for (int i = 0; i < NE; ++i) s = fmaf(y[v][i], g[v][i], s);
+        }
+        s = group_reduce<SumOp, LANES>(s);
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            float dx[NE];
+#pragma unroll
+            for (int i = 0; i < NE; ++i) dx[i] = y[v][i] * (g[v][i] - s);
+            if (valid[v]) st_stream(out + base + v * LANES, E::pack(dx));
+        }
+    }
+}
+
+// Rows too long for registers (aligned): a CTA per row, passes of four independent 16-byte loads per thread; the first
+// pass comes from HBM, the later ones find the row in L2 (a row is at most a few MiB).
+template <int WHICH, int DT>
+__global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ in0, const uint4* __restrict__ in1, uint4* __restrict__ out,
+                                                     int64_t rows, int64_t nvec) {
+    using E = Elem<DT>;
+    constexpr int NE = E::NE, U = 4;
+    __shared__ float buf[2][32];
+    pdl_wait();
+    pdl_trigger();
+    const int T = blockDim.x, t = threadIdx.x;
+    const int64_t row = blockIdx.x;
+    if (row >= rows) return;
+    const uint4* a = in0 + row * nvec;
+    uint4* o = out + row * nvec;
+    const int64_t step = static_cast<int64_t>(T) * U;
+    if constexpr (WHICH == kOpLogSoftmax) {
+        float m = kNegInf;
+        for (int64_t b0 = t; b0 < nvec; b0 += step) {
+            uint4 r[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) r[u] = b0 + u * T < nvec ? ld_param(a + b0 + u * T) : make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (b0 + u * T < nvec) m = fmaxf(m, vec_max<DT>(r[u]));
+        }
+        m = cta_reduce<MaxOp>(m, buf[0]);
+        float s = 0.f;
+        if (m != kNegInf)
+            for (int64_t b0 = t; b0 < nvec; b0 += step) {
+                uint4 r[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) r[u] = b0 + u * T < nvec ? ld_param(a + b0 + u * T) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    float x[NE];
+                    E::unpack(r[u], x);
+                    if (b0 + u * T < nvec) {
+#pragma unroll
+                        for (int i = 0; i < NE; ++i) s += ex2_ftz((x[i] - m) * kLog2e);
+                    }
+                }
+            }
+        s = cta_reduce<SumOp>(s, buf[1]);
+        const float lns = logf(s);
+        for (int64_t b0 = t; b0 < nvec; b0 += step) {
+            uint4 r[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) r[u] = b0 + u * T < nvec ? ld_stream(a + b0 + u * T) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float x[NE];
+                E::unpack(r[u], x);
+#pragma unroll
+                for (int i = 0; i < NE; ++i) x[i] = (m == kNegInf) ? kNegInf : (x[i] - m) - lns;
+                if (b0 + u * T < nvec) st_stream(o + b0 + u * T, E::pack(x));
+            }
+        }
+    } else {
+        const uint4* b = in1 + row * nvec;
+        float s = 0.f;
+        for (int64_t b0 = t; b0 < nvec; b0 += step) {
+            uint4 ry[U], rg[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const bool ok = b0 + u * T < nvec;
+                ry[u] = ok ? ld_param(a + b0 + u * T) : make_uint4(0, 0, 0, 0);
+                rg[u] = ok ? ld_param(b + b0 + u * T) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float y[NE], g[NE];
+                E::unpack(ry[u], y);
+                E::unpack(rg[u], g);
+#pragma unroll
+                for (int i = 0; i < NE; ++i) s = fmaf(y[i], g[i], s);
+            }
+        }
+        s = cta_reduce<SumOp>(s, buf[0]);
+        for (int64_t b0 = t; b0 < nvec; b0 += step) {
+            uint4 ry[U], rg[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const bool ok = b0 + u * T < nvec;
+                ry[u] = ok ? ld_stream(a + b0 + u * T) : make_uint4(0, 0, 0, 0);
+                rg[u] = ok ? ld_stream(b + b0 + u * T) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float y[NE], g[NE];
+                E::unpack(ry[u], y);
+                E::unpack(rg[u], g);
+#pragma unroll
+                for (int i = 0; i < NE; ++i) y[i] = y[i] * (g[i] - s);
+                if (b0 + u * T < nvec) st_stream(o + b0 + u * T, E::pack(y));
+            }
+        }
+    }
+}
+
+// Any alignment, any width, any length: a CTA per row, scalar passes.
+template <int WHICH, int DT>
+__global__ void __launch_bounds__(256) k_row2_scalar(const typename Elem<DT>::scalar* in0, const typename Elem<DT>::scalar* in1,
+                                                     typename Elem<DT>::scalar* out, int64_t rows, int64_t cols) {
+    using E = Elem<DT>;
+    __shared__ float buf[2][32];
+    const int64_t row = blockIdx.x;
+    if (row >= rows) return;
+    const typename E::scalar* a = in0 + row * cols;
+    typename E::scalar* o = out + row * cols;
+    if constexpr (WHICH == kOpLogSoftmax) {
+        float m = kNegInf;
+        for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) m = fmaxf(m, E::to_float(a[j]));
+        m = cta_reduce<MaxOp>(m, buf[0]);
+        float s = 0.f;
+        if (m != kNegInf)
+            for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) s += expf(E::to_float(a[j]) - m);
+        s = cta_reduce<SumOp>(s, buf[1]);
+        const float lns = logf(s);
+        for (int64_t j = threadIdx.x; j < cols; j += blockDim.x)
+            o[j] = E::from_float(m == kNegInf ? kNegInf : (E::to_float(a[j]) - m) - lns);
+    } else {
+        const typename E::scalar* b = in1 + row * cols;
+        float s = 0.f;
+        for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) s = fmaf(E::to_float(a[j]), E::to_float(b[j]), s);
+        s = cta_reduce<SumOp>(s, buf[0]);
+        for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) o[j] = E::from_float(E::to_float(a[j]) * (E::to_float(b[j]) - s));
+    }
+}
+
+bool al16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <int WHICH, int DT, int VPT>
+cudaError_t launch_vpt(int threads, cudaStream_t st, const void* in0, const void* in1, void* out, int64_t rows, int nvec) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(rows));
+    cfg.blockDim = dim3(threads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_row2<WHICH, DT, VPT>, static_cast<const uint4*>(in0), static_cast<const uint4*>(in1),
+                              static_cast<uint4*>(out), rows, nvec);
+}
+
+template <class... T>
+cudaError_t launch_pdl(void (*fn)(T...), int64_t grid, int threads, cudaStream_t st, T... args) {
+    if (grid > 0x7FFFFFFF) return cudaErrorInvalidConfiguration;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(threads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, args...);
+}
+
+template <int WHICH, int DT, int LANES, int VPT>
+cudaError_t launch_group(cudaStream_t st, const void* in0, const void* in1, void* out, int64_t rows, int nvec) {
+    const int rpc = 128 / LANES;
+    return launch_pdl(k_row2_group<WHICH, DT, LANES, VPT>, (rows + rpc - 1) / rpc, 128, st, static_cast<const uint4*>(in0),
+                      static_cast<const uint4*>(in1), static_cast<uint4*>(out), rows, nvec);
+}
+
+template <int WHICH, int DT>
+cudaError_t launch_dt(cudaStream_t st, const void* in0, const void* in1, void* out, int64_t rows, int64_t cols) {
+    using S = typename Elem<DT>::scalar;
+    if (rows > 0x7FFFFFFF) return cudaErrorInvalidConfiguration;
+    {
+        const int64_t b = cols * Elem<DT>::SIZE;
+        const bool al = al16(in0) && al16(out) && (WHICH == kOpLogSoftmax || al16(in1)) && b % 16 == 0;
+        if (al && b / 16 <= 128) {                                  // rows up to 2 KiB: lane groups
+            const int nv = static_cast<int>(b / 16);
+            if (nv <= 8) return launch_group<WHICH, DT, 8, 1>(st, in0, in1, out, rows, nv);
+            if (nv <= 16) return launch_group<WHICH, DT, 8, 2>(st, in0, in1, out, rows, nv);
+            if (nv <= 32) return launch_group<WHICH, DT, 16, 2>(st, in0, in1, out, rows, nv);
+            if (nv <= 64) return launch_group<WHICH, DT, 32, 2>(st, in0, in1, out, rows, nv);
+            return launch_group<WHICH, DT, 32, 4>(st, in0, in1, out, rows, nv);
+        }
+    }
+    const int64_t bytes = cols * Elem<DT>::SIZE;
+    const bool aligned = al16(in0) && al16(out) && (WHICH == kOpLogSoftmax || al16(in1)) && bytes % 16 == 0;
+    // the fewest vectors per thread that keep the CTA at 128 threads or fewer; else the most the register budget allows
+    int vpt = 0, threads = 0;
+    if (aligned && bytes / 16 <= 8192) {
+        const int nv = static_cast<int>(bytes / 16);
+        const int fl[4] = {row2_floats<WHICH, DT, 1>(), row2_floats<WHICH, DT, 2>(), row2_floats<WHICH, DT, 4>(), row2_floats<WHICH, DT, 8>()};
+        for (int k = 0; k < 4; ++k) {
+            const int v = 1 << k;
+            if (fl[k] > 64) break;
+            const int th = std::max(32, ((nv + v - 1) / v + 31) / 32 * 32);
+            if (th > (fl[k] <= 32 ? 1024 : 512)) continue;
+            vpt = v; threads = th;
+            if (th <= 128) break;
+        }
+    }
+    if (vpt == 0 && aligned)
+        return launch_pdl(k_row2_stream<WHICH, DT>, rows, 512, st, static_cast<const uint4*>(in0), static_cast<const uint4*>(in1),
+                          static_cast<uint4*>(out), rows, bytes / 16);
+    if (vpt == 0) {
+        k_row2_scalar<WHICH, DT><<<static_cast<unsigned>(rows), 256, 0, st>>>(static_cast<const S*>(in0), static_cast<const S*>(in1),
+                                                                             static_cast<S*>(out), rows, cols);
+        return cudaGetLastError();
+    }
+    const int nvec = static_cast<int>(bytes / 16);
+    switch (vpt) {
+        case 1: return launch_vpt<WHICH, DT, 1>(threads, st, in0, in1, out, rows, nvec);
+        case 2: return launch_vpt<WHICH, DT, 2>(threads, st, in0, in1, out, rows, nvec);
+        case 4: return launch_vpt<WHICH, DT, 4>(threads, st, in0, in1, out, rows, nvec);
+        default:
+            if constexpr (row2_floats<WHICH, DT, 8>() <= 64) return launch_vpt<WHICH, DT, 8>(threads, st, in0, in1, out, rows, nvec);
+            else return cudaErrorInvalidValue;
+    }
+}
+
+template <int WHICH>
+tf_status run2(const void* in0, const void* in1, void* out, int64_t rows, int64_t cols, int dt, void* stream) {
+    if (rows < 0 || cols <= 0 || (dt != DT_F32 && dt != DT_BF16)) return TF_ERR_INVALID_ARG;
+    if (rows > 0 && (!in0 || !out || (WHICH == kOpSoftmaxBwd && !in1))) return TF_ERR_INVALID_ARG;
+    if (rows == 0) return TF_OK;
+    if (cols > (INT64_MAX / 8) / rows) return TF_ERR_UNSUPPORTED;
+    count_launches(1);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const cudaError_t e = dt == DT_F32 ? launch_dt<WHICH, DT_F32>(st, in0, in1, out, rows, cols)
+                                       : launch_dt<WHICH, DT_BF16>(st, in0, in1, out, rows, cols);
+    if (e == cudaErrorInvalidConfiguration) return TF_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) { remember_cuda_error(e); return TF_ERR_CUDA; }
+    return TF_OK;
+}
+
+}  // namespace
+}  // namespace tf
+
+using namespace tf;
+
+extern "C" tf_status tf_log_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols, tf_dtype dt, void* stream) {
+    return run2<kOpLogSoftmax>(x, nullptr, y, rows, cols, dt, stream);
+}
+
+extern "C" tf_status tf_softmax_bwd(const void* y, const void* dy, void* dx, int64_t rows, int64_t cols, tf_dtype dt, void* stream) {
+    return run2<kOpSoftmaxBwd>(y, dy, dx, rows, cols, dt, stream);
+}
