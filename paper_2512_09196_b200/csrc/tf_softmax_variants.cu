@@ -181,32 +181,36 @@ __global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ i
     uint4* o = out + row * nvec;
     const int64_t step = static_cast<int64_t>(T) * U;
     if constexpr (WHICH == kOpLogSoftmax) {
-        float m = kNegInf;
+        // one pass for both statistics: every thread keeps (running max, sum relative to it) and rescales the sum when
+        // its maximum grows; exponents are formed from differences, never from a rounded offset
+        float mt = kNegInf, st = 0.f;
         for (int64_t b0 = t; b0 < nvec; b0 += step) {
             uint4 r[U];
+            float cm = kNegInf;
 #pragma unroll
-            for (int u = 0; u < U; ++u) r[u] = b0 + u * T < nvec ? ld_param(a + b0 + u * T) : make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-                if (b0 + u * T < nvec) m = fmaxf(m, vec_max<DT>(r[u]));
-        }
-        m = cta_reduce<MaxOp>(m, buf[0]);
-        float s = 0.f;
-        if (m != kNegInf)
-            for (int64_t b0 = t; b0 < nvec; b0 += step) {
-                uint4 r[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) r[u] = b0 + u * T < nvec ? ld_param(a + b0 + u * T) : make_uint4(0, 0, 0, 0);
+            for (int u = 0; u < U; ++u) {
+                const bool ok = b0 + u * T < nvec;
+                r[u] = ok ? ld_param(a + b0 + u * T) : make_uint4(0, 0, 0, 0);
+                if (ok) cm = fmaxf(cm, vec_max<DT>(r[u]));
+            }
+            if (cm > mt) {
+                st = (mt == kNegInf) ? 0.f : st * ex2_ftz((mt - cm) * kLog2e);
+                mt = cm;
+            }
+            if (mt != kNegInf) {
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     float x[NE];
                     E::unpack(r[u], x);
                     if (b0 + u * T < nvec) {
 #pragma unroll
-                        for (int i = 0; i < NE; ++i) s += ex2_ftz((x[i] - m) * kLog2e);
+                        for (int i = 0; i < NE; ++i) st += ex2_ftz((x[i] - mt) * kLog2e);
                     }
                 }
             }
+        }
+        const float m = cta_reduce<MaxOp>(mt, buf[0]);
+        float s = (mt == kNegInf) ? 0.f : st * ex2_ftz((mt - m) * kLog2e);          // 2^0 = 1 exactly for the thread that holds the maximum
         s = cta_reduce<SumOp>(s, buf[1]);
         const float lns = logf(s);
         for (int64_t b0 = t; b0 < nvec; b0 += step) {
