@@ -142,7 +142,8 @@ tf_status tf_log_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols,
  * gradient dy, all [rows, cols] of one element type; fp32 arithmetic, one rounding.  dx may alias y or dy.
  * Both calls: device pointers, asynchronous on cuda_stream, allocate nothing; TF_ERR_INVALID_ARG for a null pointer
  * with rows > 0, cols <= 0 or an unknown element type; rows = 0 is a no-op.  16-byte aligned tensors whose rows are
- * whole 16-byte vectors of up to 32-128 KiB (by op and type) are held in registers; anything else runs scalar passes. */
+ * whole 16-byte vectors are held in registers up to 32 KiB per row and streamed in two passes beyond; anything else
+ * runs scalar passes. */
 tf_status tf_softmax_bwd(const void* y, const void* dy, void* dx, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
 
 /* ---- fused residual add + norm ------------------------------------------------------------------------ */

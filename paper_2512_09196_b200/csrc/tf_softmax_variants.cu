@@ -3,9 +3,8 @@
 //   softmax backward      dx_j = y_j * (dy_j - sum_k y_k dy_k)
 // One kernel shape serves both: a CTA owns a row and holds it in registers (VPT 16-byte vectors per thread, loaded at
 // once), reduces across the CTA, finishes and stores -- one read of every input element, one write of every output
-// element.  Rows of up to 2 KiB are owned by lane groups instead (several rows per warp).  Rows beyond what 1024 threads
-// hold in 32 fp32 values each (32 KiB for the bf16 backward pass up to 128 KiB for the fp32 log-softmax) are streamed in
-// passes of 16-byte loads, the later passes from L2; unaligned tensors and odd widths take scalar passes.
+// element.  Rows of up to 2 KiB are owned by lane groups instead (several rows per warp).  Rows beyond 32 KiB are
+// streamed in two passes of 16-byte loads, the second from L2; unaligned tensors and odd widths take scalar passes.
 //
 // Log-softmax keeps x - m as a difference (exact for bf16 inputs, one rounding for fp32) and subtracts ln S computed
 // from S = sum 2^((x - m) log2 e) with the accurate logarithm; the term of the maximum is exactly 1, so S >= 1 and its
@@ -357,7 +356,9 @@ cudaError_t launch_dt(cudaStream_t st, const void* in0, const void* in1, void* o
     const bool aligned = al16(in0) && al16(out) && (WHICH == kOpLogSoftmax || al16(in1)) && bytes % 16 == 0;
     // the fewest vectors per thread that keep the CTA at 128 threads or fewer; else the most the register budget allows
     int vpt = 0, threads = 0;
-    if (aligned && bytes / 16 <= 8192) {
+    // beyond 32 KiB the streamed passes win: a CTA that holds such a row in registers is alone on its SM for too long
+    // (measured at 64 KiB: log-softmax 4.1 TB/s held, 5.4 streamed)
+    if (aligned && bytes / 16 <= 2048) {
         const int nv = static_cast<int>(bytes / 16);
         const int fl[4] = {row2_floats<WHICH, DT, 1>(), row2_floats<WHICH, DT, 2>(), row2_floats<WHICH, DT, 4>(), row2_floats<WHICH, DT, 8>()};
         for (int k = 0; k < 4; ++k) {
