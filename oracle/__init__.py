@@ -67,6 +67,8 @@ def _load():
         lib.oracle_log_softmax.restype = i32
         lib.oracle_softmax_bwd.argtypes = [vp, vp, vp, vp, vp, i64, i64, i32, i32]
         lib.oracle_softmax_bwd.restype = i32
+        lib.oracle_norm_bwd.argtypes = [vp] * 14 + [i64, i64, i32, i32, i32]
+        lib.oracle_norm_bwd.restype = i32
         lib.oracle_add.argtypes = [vp, vp, vp, vp, i64, i32]
         lib.oracle_add.restype = i32
         lib.oracle_bf16_from_double.argtypes = [vp, vp, i64]
@@ -220,6 +222,28 @@ def add_rmsnorm(x, r, w, eps: float, dt: int, want64: bool = False, nthreads: in
     """Fused residual add + RMSNorm: ``h = add(x, r)`` then ``rmsnorm(h)``.  Returns ``(h,) + rmsnorm(h, ...)``."""
     h = add(x, r, dt)
     return (h,) + tuple(rmsnorm(h, w, eps, dt, want64=want64, nthreads=nthreads))
+
+
+def norm_bwd(x, gamma, dy, mean, rstd, dt: int, rms: bool, nthreads: int = 1) -> dict:
+    """Backward pass of LayerNorm (``rms=False``) or RMSNorm (``rms=True``) from the forward pass's stored fp32
+    ``mean`` / ``rstd`` ([rows]; ``mean`` may be None for RMSNorm).  Returns a dict with ``dx, dgamma, dbeta`` in the
+    storage type (``dbeta`` None for RMSNorm), their unrounded float64 versions ``dx64, dg64, db64`` and the condition
+    scales ``dx_scale, dg_scale, db_scale``."""
+    _check(x, dt, "x"), _check(gamma, dt, "gamma"), _check(dy, dt, "dy")
+    rows, cols = x.shape
+    if dy.shape != x.shape or gamma.shape != (cols,):
+        raise ValueError("shape mismatch")
+    rstd = np.ascontiguousarray(rstd, np.float32)
+    mean = None if mean is None else np.ascontiguousarray(mean, np.float32)
+    out = {"dx": np.empty_like(x), "dgamma": np.empty_like(gamma), "dbeta": None if rms else np.empty_like(gamma),
+           "dx64": np.empty((rows, cols)), "dg64": np.empty(cols), "db64": np.empty(cols),
+           "dx_scale": np.empty((rows, cols)), "dg_scale": np.empty(cols), "db_scale": np.empty(cols)}
+    rc = _load().oracle_norm_bwd(_p(x), _p(gamma), _p(dy), _p(mean), _p(rstd), _p(out["dx"]), _p(out["dgamma"]), _p(out["dbeta"]),
+                                 _p(out["dx64"]), _p(out["dg64"]), _p(out["db64"]), _p(out["dx_scale"]), _p(out["dg_scale"]),
+                                 _p(out["db_scale"]), rows, cols, int(rms), dt, nthreads)
+    if rc:
+        raise ValueError("oracle_norm_bwd: bad argument")
+    return out
 
 
 def bf16_from_double(v: np.ndarray) -> np.ndarray:

@@ -36,6 +36,10 @@
 // masked entries (-inf) and torch's float64 routine.  The softmax backward pass (dx = y (dy - sum y dy)) is
 // pinned by the analytic Jacobian on one-hot dy, by central differences of the pinned softmax in double,
 // by dx = 0 for constant dy, by linearity in dy and by torch's float64 autograd.
+// The backward passes of LayerNorm and RMSNorm (dx per row from the stored statistics, parameter gradients
+// as column sums over the rows) are pinned by central differences of the pinned forward passes in double, by
+// the orthogonality invariants of dx (it sums to zero and is orthogonal to the normalised row for LayerNorm,
+// orthogonal to x for RMSNorm with unit weight), by plain column sums for dbeta, and by torch's float64 autograd.
 // tf_tune has
 // no oracle function here: which candidate wins is hardware-dependent ("parity unpinned" for the
 // winner's identity; its output is checked like any other launch).
@@ -291,6 +295,53 @@ int oracle_softmax_bwd(const void* y, const void* dy, void* dx, double* dx64, do
             if (scale64) scale64[base + j] = std::fabs(yj) * (std::fabs(gj) + sa);
             if (dx) store(dx, base + j, dt, v);
         }
+    });
+    return 0;
+}
+
+// Backward pass of LayerNorm (rms = 0) or RMSNorm (rms = 1) from the forward pass's stored fp32 statistics.
+//   xh_j = (x_j - mean) * rstd   (RMSNorm: x_j * rstd),   g_j = dy_j * gamma_j
+//   LayerNorm:  dx_j = rstd * (g_j - mean_k g_k - xh_j * mean_k (g_k xh_k))
+//   RMSNorm:    dx_j = rstd * (g_j - xh_j * mean_k (g_k xh_k))
+//   dgamma_j = sum_rows dy_j * xh_j,   dbeta_j = sum_rows dy_j   (LayerNorm only)
+// Everything in double, sums in increasing index, one rounding to the storage type.  dx_scale64 (nullable) receives
+// rstd * (|g_j| + mean|g| + |xh_j| mean|g xh|), dg_scale64 / db_scale64 the sums of absolute terms.
+int oracle_norm_bwd(const void* x, const void* gamma, const void* dy, const float* mean, const float* rstd, void* dx,
+                    void* dgamma, void* dbeta, double* dx64, double* dg64, double* db64, double* dx_scale64,
+                    double* dg_scale64, double* db_scale64, int64_t rows, int64_t cols, int rms, int dt, int nthreads) {
+    if (bad(rows, cols, dt) || !x || !gamma || !dy || !rstd || (!rms && !mean)) return -1;
+    const double n = static_cast<double>(cols);
+    for_rows(rows, nthreads, [=](int64_t r) {
+        const int64_t base = r * cols;
+        const double mu = rms ? 0.0 : static_cast<double>(mean[r]), rs = static_cast<double>(rstd[r]);
+        double sg = 0.0, sgx = 0.0, ag = 0.0, agx = 0.0;
+        for (int64_t j = 0; j < cols; ++j) {
+            const double xh = (load(x, base + j, dt) - mu) * rs, g = load(dy, base + j, dt) * load(gamma, j, dt);
+            sg += g; sgx += g * xh; ag += std::fabs(g); agx += std::fabs(g * xh);
+        }
+        const double mg = rms ? 0.0 : sg / n, mgx = sgx / n;
+        for (int64_t j = 0; j < cols; ++j) {
+            const double xh = (load(x, base + j, dt) - mu) * rs, g = load(dy, base + j, dt) * load(gamma, j, dt);
+            const double v = rs * (g - mg - xh * mgx);
+            if (dx64) dx64[base + j] = v;
+            if (dx_scale64) dx_scale64[base + j] = rs * (std::fabs(g) + (rms ? 0.0 : ag / n) + std::fabs(xh) * agx / n);
+            if (dx) store(dx, base + j, dt, v);
+        }
+    });
+    // parameter gradients: column sums over the rows (columns spread over the workers)
+    for_rows(cols, nthreads, [=](int64_t j) {
+        double sg = 0.0, sb = 0.0, ag = 0.0, ab = 0.0;
+        for (int64_t r = 0; r < rows; ++r) {
+            const double mu = rms ? 0.0 : static_cast<double>(mean[r]), rs = static_cast<double>(rstd[r]);
+            const double d = load(dy, r * cols + j, dt), t = d * ((load(x, r * cols + j, dt) - mu) * rs);
+            sg += t; sb += d; ag += std::fabs(t); ab += std::fabs(d);
+        }
+        if (dg64) dg64[j] = sg;
+        if (db64) db64[j] = sb;
+        if (dg_scale64) dg_scale64[j] = ag;
+        if (db_scale64) db_scale64[j] = ab;
+        if (dgamma) store(dgamma, j, dt, sg);
+        if (dbeta && !rms) store(dbeta, j, dt, sb);
     });
     return 0;
 }
