@@ -690,6 +690,77 @@ def run_softmax_variants_table(args):
     (out_dir / "table_softmaxvariants.json").write_text(json.dumps(rows_out, indent=1))
 
 
+def run_normbwd_table(args):
+    """LayerNorm / RMSNorm backward: achieved bandwidth of x, dy in and dx out; torch's native backward as context."""
+    import torch
+    import paper_2512_09196_b200 as tf
+    from paper_2512_09196_b200 import inputs
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak()
+    out_dir = ROOT / "gpurun_out"
+    out_dir.mkdir(exist_ok=True)
+    shapes = [("rmsnorm", inputs.BF16, 16384, 4096), ("rmsnorm", inputs.BF16, 16384, 8192), ("rmsnorm", inputs.F32, 16384, 4096),
+              ("layernorm", inputs.BF16, 16384, 4096), ("layernorm", inputs.BF16, 65536, 1024), ("layernorm", inputs.F32, 8192, 8192),
+              ("layernorm", inputs.BF16, 4096, 16384)]
+    rows_out = []
+    for op, dt, rows, cols in shapes:
+        es = inputs.ELEM_SIZE[dt]
+        tdt = torch.bfloat16 if dt == inputs.BF16 else torch.float32
+        conv = (lambda t: t.view(torch.bfloat16)) if dt == inputs.BF16 else (lambda t: t)
+        sets = max(2, min(8, int((1 << 30) // (3 * rows * cols * es))))
+        xs = [conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols, 0, 0.3, 2.0))).cuda() for _ in range(sets)]
+        dys = [conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols + 1, 3, 0.0, 1.0))).cuda() for _ in range(sets)]
+        dxs = [torch.empty_like(x) for x in xs]
+        g = (torch.rand(cols, device="cuda") + 0.5).to(tdt)
+        b = torch.zeros(cols, device="cuda", dtype=tdt)
+        if op == "layernorm":
+            stats = [tf.tf_layernorm_fwd(x, g, b, 1e-5)[1:] for x in xs]
+        else:
+            stats = [(None, tf.tf_rmsnorm_fwd(x, g, 1e-6, want_rstd=True)[1]) for x in xs]
+
+        def ours(k):
+            if op == "layernorm":
+                tf.tf_layernorm_bwd(xs[k], g, dys[k], stats[k][0], stats[k][1], dx=dxs[k])
+            else:
+                tf.tf_rmsnorm_bwd(xs[k], g, dys[k], stats[k][1], dx=dxs[k])
+
+        def lib(k):
+            if op == "layernorm":
+                torch.ops.aten.native_layer_norm_backward(dys[k], xs[k], [cols], stats[k][0].view(rows, 1), stats[k][1].view(rows, 1), g, b,
+                                                          [True, True, True])
+            else:
+                xf = xs[k].float()
+                xh = xf * stats[k][1][:, None]
+                gg = dys[k].float() * g.float()
+                (stats[k][1][:, None] * (gg - xh * (gg * xh).mean(dim=1, keepdim=True))).to(tdt)
+                (dys[k].float() * xh).sum(dim=0).to(tdt)
+
+        def timed(fn, reps):
+            for k in range(3):
+                fn(k % sets)
+            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for k in range(reps):
+                fn(k % sets)
+            e.record()
+            torch.cuda.synchronize()
+            return 1e3 * a.elapsed_time(e) / reps
+
+        nbytes = 3 * rows * cols * es + (3 if op == "layernorm" else 2) * cols * es + (8 if op == "layernorm" else 4) * rows
+        reps = max(10, min(200, int(0.05 / (nbytes / 5e12))))
+        us, us_lib = timed(ours, reps), timed(lib, max(5, reps // 4))
+        tf.tf_device_status()
+        row = {"op": op + "_bwd", "dtype": "f32" if dt == inputs.F32 else "bf16", "rows": rows, "cols": cols, "bytes": nbytes, "us": us,
+               "gbs": nbytes / us / 1e3, f"pct_of_{peak_kind}_{peak:.0f}": 100 * nbytes / us / 1e3 / peak, "torch_us": us_lib,
+               "torch_what": "aten native_layer_norm_backward" if op == "layernorm" else "eager fp32 expression (no fused kernel in torch)"}
+        rows_out.append(row)
+        print(json.dumps(row), flush=True)
+        del xs, dys, dxs
+        torch.cuda.empty_cache()
+    (out_dir / "table_normbwd.json").write_text(json.dumps(rows_out, indent=1))
+
+
 def run_case(args):
     """A few launches of one op/shape (for profiler captures): --case op:dtype:rows:cols or --case config:<i>[:rows]."""
     import torch
@@ -779,7 +850,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm", "softmaxlen", "softmaxvariants"], default=None)
+    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm", "softmaxlen", "softmaxvariants", "normbwd"], default=None)
     ap.add_argument("--filter", default=None)
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
@@ -804,6 +875,8 @@ def main():
         return run_softmaxlen_table(args)
     if args.table == "softmaxvariants":
         return run_softmax_variants_table(args)
+    if args.table == "normbwd":
+        return run_normbwd_table(args)
     if args.table:
         return run_table(args)
     run_ours(args)

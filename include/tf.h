@@ -146,6 +146,27 @@ tf_status tf_log_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols,
  * runs scalar passes. */
 tf_status tf_softmax_bwd(const void* y, const void* dy, void* dx, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
 
+/* ---- backward passes of the norms ------------------------------------------------------------------------- */
+
+/* From the forward pass's inputs and its stored fp32 statistics (mean, rstd: [rows]):
+ *     xh_j = (x_j - mean) rstd   (RMSNorm: x_j rstd),   g_j = dy_j gamma_j
+ *     dx_j = rstd (g_j - mean_k g_k - xh_j mean_k (g_k xh_k))          (RMSNorm: without the mean_k g_k term)
+ *     dgamma_j = sum over rows of dy_j xh_j,   dbeta_j = sum over rows of dy_j   (LayerNorm only)
+ * fp32 arithmetic; dx, dgamma, dbeta are rounded once to the storage type; the column sums are accumulated in fp32
+ * in a fixed order (deterministic).  x, dy, dx: [rows, cols]; gamma / weight, dgamma / dweight, dbeta: [cols]; dx may
+ * alias x or dy.  workspace: device memory of at least tf_norm_bwd_workspace_bytes(rows, cols) bytes, 4-byte aligned,
+ * used for partial column sums while the call runs (calls that may overlap on the GPU need separate workspaces); it
+ * is required when the tensors are 16-byte aligned with rows of whole 16-byte vectors and up to 25,600 (LayerNorm) /
+ * 51,200 (RMSNorm) columns, and ignored otherwise (such shapes run two plain kernels).  rows = 0 zeroes the parameter gradients.
+ * Errors: TF_ERR_INVALID_ARG for a null pointer, cols <= 0, an unknown element type or a missing / short workspace.
+ * Asynchronous on cuda_stream; allocates nothing.  The paper has no counterpart. */
+size_t tf_norm_bwd_workspace_bytes(int64_t rows, int64_t cols);
+tf_status tf_layernorm_bwd(const void* x, const void* gamma, const void* dy, const float* mean, const float* rstd, void* dx,
+                           void* dgamma, void* dbeta, void* workspace, size_t workspace_bytes, int64_t rows, int64_t cols,
+                           tf_dtype dt, void* cuda_stream);
+tf_status tf_rmsnorm_bwd(const void* x, const void* weight, const void* dy, const float* rstd, void* dx, void* dweight,
+                         void* workspace, size_t workspace_bytes, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
+
 /* ---- fused residual add + norm ------------------------------------------------------------------------ */
 
 /* h = x + r (fp32 add, ONE rounding to the storage type), then the LayerNorm / RMSNorm defined above applied to that

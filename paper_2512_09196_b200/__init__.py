@@ -20,7 +20,8 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_status_string",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_norm_bwd_workspace_bytes", "tf_layernorm_bwd", "tf_rmsnorm_bwd",
+           "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
 
@@ -59,6 +60,10 @@ def lib() -> ctypes.CDLL:
         L.tf_softmax_len_fwd.argtypes = [vp, vp, vp, i64, i64, i32, vp]
         L.tf_log_softmax_fwd.argtypes = [vp, vp, i64, i64, i32, vp]
         L.tf_softmax_bwd.argtypes = [vp, vp, vp, i64, i64, i32, vp]
+        L.tf_norm_bwd_workspace_bytes.argtypes = [i64, i64]
+        L.tf_norm_bwd_workspace_bytes.restype = ctypes.c_size_t
+        L.tf_layernorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i64, i64, i32, vp]
+        L.tf_rmsnorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i64, i64, i32, vp]
         L.tf_bvecmat_fwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp]
         L.tf_sin_fwd.argtypes = [vp, vp, i64, i32, i32, i32, vp]
         L.tf_tune_like.argtypes = [i32, vp, vp, vp, i64, i64, i32]
@@ -75,7 +80,7 @@ def lib() -> ctypes.CDLL:
         L.tf_clear_cache.restype = None
         L.tf_launch_count.argtypes = []
         L.tf_launch_count.restype = i64
-        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd",
+        for name in ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_layernorm_bwd", "tf_rmsnorm_bwd",
                      "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice",
                      "tf_candidate_count", "tf_candidate"):
             getattr(L, name).restype = i32
@@ -182,6 +187,44 @@ def tf_softmax_bwd(y, dy, dx=None):
     with _on_device(y):
         _ok(lib().tf_softmax_bwd(y.data_ptr(), dy.data_ptr(), dx.data_ptr(), rows, cols, _dt(y), _stream(y)), "tf_softmax_bwd")
     return dx
+
+
+def _norm_bwd_workspace(x):
+    import torch
+    rows, cols = x.shape
+    n = lib().tf_norm_bwd_workspace_bytes(rows, cols)
+    return torch.empty(max(1, n // 4), dtype=torch.float32, device=x.device), n
+
+
+def tf_layernorm_bwd(x, gamma, dy, mean, rstd, dx=None):
+    """LayerNorm backward from the forward pass's stored fp32 ``mean`` / ``rstd``.  Returns ``(dx, dgamma, dbeta)``."""
+    import torch
+    _check2d(x)
+    _check2d(dy, "dy")
+    rows, cols = x.shape
+    dx = torch.empty_like(x) if dx is None else dx
+    dgamma, dbeta = torch.empty_like(gamma), torch.empty_like(gamma)
+    ws, n = _norm_bwd_workspace(x)
+    with _on_device(x):
+        _ok(lib().tf_layernorm_bwd(x.data_ptr(), gamma.data_ptr(), dy.data_ptr(), mean.data_ptr(), rstd.data_ptr(), dx.data_ptr(),
+                                   dgamma.data_ptr(), dbeta.data_ptr(), ws.data_ptr(), n, rows, cols, _dt(x), _stream(x)),
+            "tf_layernorm_bwd")
+    return dx, dgamma, dbeta
+
+
+def tf_rmsnorm_bwd(x, weight, dy, rstd, dx=None):
+    """RMSNorm backward from the forward pass's stored fp32 ``rstd``.  Returns ``(dx, dweight)``."""
+    import torch
+    _check2d(x)
+    _check2d(dy, "dy")
+    rows, cols = x.shape
+    dx = torch.empty_like(x) if dx is None else dx
+    dweight = torch.empty_like(weight)
+    ws, n = _norm_bwd_workspace(x)
+    with _on_device(x):
+        _ok(lib().tf_rmsnorm_bwd(x.data_ptr(), weight.data_ptr(), dy.data_ptr(), rstd.data_ptr(), dx.data_ptr(), dweight.data_ptr(),
+                                 ws.data_ptr(), n, rows, cols, _dt(x), _stream(x)), "tf_rmsnorm_bwd")
+    return dx, dweight
 
 
 def tf_softmax_fwd_noalloc(x, y):
