@@ -790,6 +790,34 @@ def run_case(args):
         print(json.dumps({"case": w.name, "knobs": knobs, "launches": args.steps, "us_per_launch": us,
                           "gbs": w.algorithmic_bytes() / us / 1e3}))
         return
+    if parts[0] == "normbwd":                 # normbwd:op:dtype:rows:cols -- the backward pass of a norm
+        op, dts, rows, cols = parts[1], parts[2], int(parts[3]), int(parts[4])
+        dt = inputs.F32 if dts == "f32" else inputs.BF16
+        tdt = torch.float32 if dt == inputs.F32 else torch.bfloat16
+        conv = (lambda t: t.view(torch.bfloat16)) if dt == inputs.BF16 else (lambda t: t)
+        x = conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols, 0, 0.3, 2.0))).cuda()
+        dy = conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols + 1, 3, 0.0, 1.0))).cuda()
+        g = (torch.rand(cols, device="cuda") + 0.5).to(tdt)
+        dx = torch.empty_like(x)
+        if op == "layernorm":
+            _, mean, rstd = tf.tf_layernorm_fwd(x, g, torch.zeros_like(g), 1e-5)
+            call = lambda: tf.tf_layernorm_bwd(x, g, dy, mean, rstd, dx=dx)
+        else:
+            _, rstd = tf.tf_rmsnorm_fwd(x, g, 1e-6, want_rstd=True)
+            call = lambda: tf.tf_rmsnorm_bwd(x, g, dy, rstd, dx=dx)
+        a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(max(1, args.warmup)):
+            call()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(args.steps):
+            call()
+        e.record()
+        torch.cuda.synchronize()
+        us = 1e3 * a.elapsed_time(e) / args.steps
+        nbytes = 3 * rows * cols * inputs.ELEM_SIZE[dt]
+        print(json.dumps({"case": f"case_{op}_bwd_{dts}_{rows}x{cols}", "launches": args.steps, "us_per_launch": us, "gbs": nbytes / us / 1e3}))
+        return
     if parts[0] == "addnorm":                 # addnorm:op:dtype:rows:cols -- the fused residual add + norm, heuristic plan
         op, dts, rows, cols = parts[1], parts[2], int(parts[3]), int(parts[4])
         dt = inputs.F32 if dts == "f32" else inputs.BF16
