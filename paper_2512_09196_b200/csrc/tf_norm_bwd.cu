@@ -205,22 +205,34 @@ __global__ void __launch_bounds__(1024) k_norm_bwd_stream(const BArgs a) {
         }
 }
 
-// Adds the `nparts` partial column sums in index order and rounds once.
+// Adds the `nparts` partial column sums and rounds once.  A CTA of 32 x 8 threads owns 32 columns: thread (c, y) adds
+// parts y, y + 8, ... of column c, the eight slice sums meet in shared memory and are added in slice order -- a fixed
+// order of additions whatever the launch, hence deterministic -- and 128 CTAs instead of 16 share the reading.
 template <bool RMS, int DT>
-__global__ void __launch_bounds__(256) k_colsum_finish(const float* part, typename Elem<DT>::scalar* dgamma, typename Elem<DT>::scalar* dbeta,
-                                                       int nparts, int64_t cols) {
+__global__ void __launch_bounds__(256) k_colsum_finish(const float* __restrict__ part, typename Elem<DT>::scalar* dgamma,
+                                                       typename Elem<DT>::scalar* dbeta, int nparts, int64_t cols) {
     using E = Elem<DT>;
+    __shared__ float sm[2][8][32];
     pdl_wait();
-    const int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (j >= cols) return;
+    const int c = threadIdx.x & 31, y = threadIdx.x >> 5;
+    const int64_t j = static_cast<int64_t>(blockIdx.x) * 32 + c;
     const int64_t stride = (RMS ? 1 : 2) * cols;
     float sg = 0.f, sb = 0.f;
-    for (int p = 0; p < nparts; ++p) {
-        sg += part[p * stride + j];
-        if (!RMS) sb += part[p * stride + cols + j];
+    if (j < cols)
+        for (int p = y; p < nparts; p += 8) {
+            sg += part[p * stride + j];
+            if (!RMS) sb += part[p * stride + cols + j];
+        }
+    sm[0][y][c] = sg;
+    sm[1][y][c] = sb;
+    __syncthreads();
+    if (y == 0 && j < cols) {
+        float tg = 0.f, tb = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { tg += sm[0][k][c]; tb += sm[1][k][c]; }
+        dgamma[j] = E::from_float(tg);
+        if (!RMS) dbeta[j] = E::from_float(tb);
     }
-    dgamma[j] = E::from_float(sg);
-    if (!RMS) dbeta[j] = E::from_float(sb);
 }
 
 // ---- any shape, any alignment ------------------------------------------------------------------------------------
@@ -337,7 +349,7 @@ tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float*
         else if (p.vpt == 2) e = launch_pdl(k_norm_bwd<RMS, DT, 2>, p.grid, threads, st, a, p.gt);
         else e = launch_pdl(k_norm_bwd<RMS, DT, kMaxVpt>, p.grid, threads, st, a, p.gt);
         if (e == cudaSuccess)
-            e = launch_pdl(k_colsum_finish<RMS, DT>, (cols + 255) / 256, 256, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
+            e = launch_pdl(k_colsum_finish<RMS, DT>, (cols + 31) / 32, 256, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
                            static_cast<S*>(dbeta), parts, cols);
     } else if (aligned && cols <= 0x7FFFFFFF && static_cast<size_t>(RMS ? 1 : 2) * cols * 4 <= 200 * 1024) {
         const int nvec = static_cast<int>(bytes / 16);
@@ -357,7 +369,7 @@ tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float*
             cfg.stream = st;
             e = cudaLaunchKernelEx(&cfg, k_norm_bwd_stream<RMS, DT>, a);
             if (e == cudaSuccess)
-                e = launch_pdl(k_colsum_finish<RMS, DT>, (cols + 255) / 256, 256, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
+                e = launch_pdl(k_colsum_finish<RMS, DT>, (cols + 31) / 32, 256, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
                                static_cast<S*>(dbeta), grid, cols);
         }
     } else {
