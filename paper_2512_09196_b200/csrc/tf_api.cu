@@ -191,6 +191,41 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         s.cluster = static_cast<int>(std::max<int64_t>(2, std::min<int64_t>(nvec / 256, 2 * d.sms / a.rows)));
         if (supports_split(s, a, d)) return s;
     }
+    // Rules read off the plans that tf_tune ends up with on the 84-point shape sweep (rows of 128 B to 256 KiB, three ops,
+    // two types); what they do not cover falls through to the older defaults below.
+    {
+        Plan q;
+        const bool ln = a.op == OP_LAYERNORM;
+        if (nvec <= 256 && !(ln && a.dt == DT_BF16)) {
+            // rows up to 4 KiB: a lane group per row, every load issued at once, as many small CTAs as there are row blocks
+            q.variant = V_WARP; q.threads = 128; q.persist = 0; q.rpg = 1;
+            if (nvec <= 8) { q.lanes = 8; q.vpt = 1; q.rpg = a.op == OP_SOFTMAX ? 4 : 2; }
+            else if (nvec <= 16) { q.lanes = 8; q.vpt = 2; q.rpg = ln ? 2 : 1; }
+            else if (nvec <= 32) { q.lanes = 16; q.vpt = 2; q.rpg = ln ? 2 : 1; }
+            else if (nvec <= 64) { q.lanes = 32; q.vpt = 2; q.rpg = (a.dt == DT_F32 && a.op != OP_SOFTMAX) ? 2 : 1; }
+            else if (nvec <= 128) { q.lanes = 32; q.vpt = 4; }
+            else { q.lanes = 32; q.vpt = 8; }
+            if (supports_warp(q, a, d)) return q;
+        } else if (!ln && nvec <= (a.dt == DT_BF16 ? 1024 : (a.op == OP_SOFTMAX ? 4096 : 3072))) {
+            // softmax and RMSNorm from 4 KiB up to 16 KiB (bf16; eight bf16 vectors per thread cost too many registers) or
+            // 48-64 KiB (fp32): a CTA per row in registers, four vectors per thread up to 16 KiB, eight beyond
+            q.variant = V_CTA; q.cluster = 1; q.persist = 0;
+            q.vpt = nvec <= 1024 ? 4 : 8;
+            q.threads = std::max(64, round_up(static_cast<int>((nvec + q.vpt - 1) / q.vpt), 32));
+            if (supports_cta(q, a, d)) return q;
+        } else if (nvec <= 32768 && (nvec > 4096 || (a.op != OP_SOFTMAX && nvec >= 4096) || (ln && nvec >= 2048 && a.dt == DT_F32))) {
+            // long rows (and LayerNorm from 32-64 KiB on): persistent clusters with a prefetch ring; the norms keep their
+            // parameter slices in shared memory and need only one stage beside them
+            q.variant = V_RING; q.vpt = 8;
+            if (a.op == OP_SOFTMAX) { q.cluster = nvec <= 8192 ? 4 : 8; q.stages = 2; }
+            else { q.cluster = nvec <= 4096 ? (ln ? 2 : 1) : nvec <= 8192 ? 2 : 8; q.stages = 1; q.rpg = 2; }
+            const int64_t per = (nvec + q.cluster - 1) / q.cluster;
+            q.threads = std::max(64, round_up(static_cast<int>((per + 7) / 8), 32));
+            const int64_t smem = (q.stages + (q.rpg == 2 ? (ln ? 2 : 1) : 0)) * per * 16;
+            q.persist = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>({8, 200 * 1024 / std::max<int64_t>(1, smem), 2048 / q.threads})));
+            if (supports_ring(q, a, d)) return q;
+        }
+    }
     if (nvec <= 4096) {
         // rows up to 64 KiB: the persistent self-feeding pipeline, one CTA of 512 threads per SM, two stages per unit
         p.variant = V_PIPE;
