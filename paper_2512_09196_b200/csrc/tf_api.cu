@@ -244,6 +244,14 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         const int64_t pass_bytes = row_bytes * (ut / p.lanes);
         const int64_t param_bytes = a.op == OP_SOFTMAX ? 0 : row_bytes * (a.op == OP_LAYERNORM ? 2 : 1);
         const int64_t per_stage = (200 * 1024 - param_bytes) / (p.threads / ut) / p.stages;
+        int64_t target = 16384;
+        if (nvec <= 256) {                       // rows up to 4 KiB (what reaches here is LayerNorm bf16): the tuner's winners use
+            p.persist = 2; target = 4096;        // small stages and two CTAs per SM
+            if (nvec <= 16) p.rpg = 2;
+        }
+        p.chunk = static_cast<int>(std::max<int64_t>(pass_bytes, std::min<int64_t>(target, per_stage / p.persist) / pass_bytes * pass_bytes));
+        if (supports_pipe(p, a, d)) return p;
+        p.persist = 1; p.rpg = 1;
         p.chunk = static_cast<int>(std::max<int64_t>(pass_bytes, std::min<int64_t>(16384, per_stage) / pass_bytes * pass_bytes));
         if (supports_pipe(p, a, d)) return p;
         p = Plan();
