@@ -66,29 +66,38 @@ cudaError_t launch_addnorm(const Plan& p, const Args& a, const DeviceInfo& d, cu
     return launch_cta_fn(cta_fn_add(a.op, a.dt, p.vpt, p.cluster > 1), p, a, d, st);
 }
 
-// Default register-resident plan by row size; `variant` is -1 when no such plan holds the row.
+// Default register-resident plan by row size (read off what tf_tune_add ends up with: the add costs registers, so the
+// fused kernels like many threads with one or two vectors each); `variant` is -1 when no such plan holds the row.
 Plan heuristic_addnorm(const Args& a, const DeviceInfo& d) {
     Plan p;
     p.variant = -1;
     if (!vector_ok(a)) return p;
     const int64_t nvec = a.cols * elem_size(a.dt) / 16;
     Plan q;
-    if (nvec <= 128) {
-        q.variant = V_WARP; q.threads = 128;
-        if (nvec <= 8) { q.lanes = 8; q.vpt = 1; q.rpg = 2; }
-        else if (nvec <= 16) { q.lanes = 16; q.vpt = 1; q.rpg = 2; }
-        else if (nvec <= 32) { q.lanes = 32; q.vpt = 1; q.rpg = 2; }
-        else if (nvec <= 64) { q.lanes = 32; q.vpt = 2; q.rpg = 2; }
-        else { q.lanes = 32; q.vpt = 4; q.rpg = 1; }
+    if (nvec <= 32) {
+        q.variant = V_WARP; q.threads = 128; q.vpt = 1; q.rpg = 1;
+        q.lanes = nvec <= 8 ? 8 : nvec <= 16 ? 16 : 32;
     } else {
         q.variant = V_CTA;
         int cl = 1;
-        while (cl < kMaxCluster && nvec > 4096LL * cl) cl *= 2;          // up to 64 KiB of a row per CTA
+        while (cl < kMaxCluster && nvec > 2048LL * cl) cl *= 2;          // up to 32 KiB of a row per CTA
         const int64_t per = (nvec + cl - 1) / cl;
         q.cluster = cl;
-        q.vpt = per <= 1024 ? 2 : per <= 2048 ? 4 : 8;
-        q.threads = std::max(64, round_up32((per + q.vpt - 1) / q.vpt));
+        if (per < 256) { q.vpt = 2; q.threads = std::max(64, round_up32((per + 1) / 2)); }
+        else if (per <= 512) { q.threads = 256; q.vpt = per <= 256 ? 1 : 2; }
+        else if (per <= 2048 && cl == 1) { q.threads = 1024; q.vpt = per <= 1024 ? 1 : 2; }
+        else { q.threads = 512; q.vpt = 4; }
     }
+    if (supports_addnorm(q, a, d)) return q;
+    // anything the rules above do not hold: the widest register-resident geometry that does
+    q = Plan();
+    q.variant = V_CTA;
+    int cl = 1;
+    while (cl < kMaxCluster && nvec > 4096LL * cl) cl *= 2;
+    const int64_t per = (nvec + cl - 1) / cl;
+    q.cluster = cl;
+    q.vpt = per <= 1024 ? 2 : per <= 2048 ? 4 : 8;
+    q.threads = std::max(64, round_up32((per + q.vpt - 1) / q.vpt));
     if (supports_addnorm(q, a, d)) return q;
     return p;
 }
