@@ -38,20 +38,21 @@ struct BArgs {
 template <bool RMS, int DT, int VPT>
 __global__ void __launch_bounds__(512) k_norm_bwd(const BArgs a, const int gt) {
     using E = Elem<DT>;
-    constexpr int NE = E::NE;
+    using P = Pairs<DT>;
+    constexpr int NE = E::NE, NP = P::NP;                            // the arithmetic runs on packed fp32 pairs
     __shared__ float2 red[2][16];
     pdl_wait();
     pdl_trigger();
     const int t = threadIdx.x, gid = t / gt, lg = t % gt, R = blockDim.x / gt, wg = gt / 32;
     const int warp = t >> 5, lane = t & 31;
     bool valid[VPT];
-    float gam[VPT][NE], accg[VPT][NE], accb[RMS ? 1 : VPT][NE];
+    F2 gam[VPT][NP], accg[VPT][NP], accb[RMS ? 1 : VPT][NP];
 #pragma unroll
     for (int v = 0; v < VPT; ++v) {
         valid[v] = lg + v * gt < a.nvec;
-        E::unpack(valid[v] ? ld_param(a.gamma + lg + v * gt) : make_uint4(0, 0, 0, 0), gam[v]);
+        P::unpack(valid[v] ? ld_param(a.gamma + lg + v * gt) : make_uint4(0, 0, 0, 0), gam[v]);
 #pragma unroll
-        for (int i = 0; i < NE; ++i) { accg[v][i] = 0.f; if (!RMS) accb[v][i] = 0.f; }
+        for (int i = 0; i < NP; ++i) { accg[v][i] = f2(0.f); if (!RMS) accb[v][i] = f2(0.f); }
     }
     // the packed vectors of the NEXT row are requested before the current row is reduced, so that the reduction of a
     // row does not leave the memory pipe idle
@@ -71,45 +72,46 @@ __global__ void __launch_bounds__(512) k_norm_bwd(const BArgs a, const int gt) {
         const int64_t row = row0 + gid;
         const bool live = row < a.rows;
         const float mu = (RMS || !live) ? 0.f : __ldg(a.mean + row), rs = live ? __ldg(a.rstd + row) : 0.f;
-        float xh[VPT][NE], g[VPT][NE], dv[VPT][NE];
+        const F2 mu2 = f2(mu), rs2 = f2(rs);
+        F2 xh[VPT][NP], g[VPT][NP], dv[VPT][NP];
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
-            float xv[NE];
-            E::unpack(nx[v], xv);
-            E::unpack(nd[v], dv[v]);                                     // zeros for absent columns and rows
+            F2 xv[NP];
+            P::unpack(nx[v], xv);
+            P::unpack(nd[v], dv[v]);                                     // zeros for absent columns and rows
 #pragma unroll
-            for (int i = 0; i < NE; ++i) xh[v][i] = (valid[v] && live) ? (xv[i] - mu) * rs : 0.f;
+            for (int i = 0; i < NP; ++i) xh[v][i] = (valid[v] && live) ? mul2(sub2(xv[i], mu2), rs2) : f2(0.f);
         }
         request(row + stride);
-        float sgx = 0.f, sg = 0.f;
+        F2 sgx2 = f2(0.f), sg2 = f2(0.f);
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
 #pragma unroll
-            for (int i = 0; i < NE; ++i) {
-                g[v][i] = dv[v][i] * gam[v][i];
-                sgx = fmaf(g[v][i], xh[v][i], sgx);
-                sg += g[v][i];
-                accg[v][i] = fmaf(dv[v][i], xh[v][i], accg[v][i]);
-                if (!RMS) accb[v][i] += dv[v][i];
+            for (int i = 0; i < NP; ++i) {
+                g[v][i] = mul2(dv[v][i], gam[v][i]);
+                sgx2 = fma2(g[v][i], xh[v][i], sgx2);
+                sg2 = add2(sg2, g[v][i]);
+                accg[v][i] = fma2(dv[v][i], xh[v][i], accg[v][i]);
+                if (!RMS) accb[v][i] = add2(accb[v][i], dv[v][i]);
             }
         }
-        sgx = group_reduce<SumOp, 32>(sgx);
-        sg = group_reduce<SumOp, 32>(sg);
+        float sgx = group_reduce<SumOp, 32>(hsum(sgx2));
+        float sg = group_reduce<SumOp, 32>(hsum(sg2));
         if (wg > 1) {
             if (lane == 0) red[it & 1][warp] = make_float2(sgx, sg);
             __syncthreads();
             sgx = 0.f; sg = 0.f;
             for (int w = 0; w < wg; ++w) { const float2 p = red[it & 1][gid * wg + w]; sgx += p.x; sg += p.y; }
         }
-        const float mgx = sgx * a.inv_n, mg = RMS ? 0.f : sg * a.inv_n;
+        const F2 mgx2 = f2(sgx * a.inv_n), mg2 = f2(RMS ? 0.f : sg * a.inv_n);
         if (live) {
             uint4* o = a.dx + row * a.nvec + lg;
 #pragma unroll
             for (int v = 0; v < VPT; ++v) {
-                float d[NE];
+                F2 d[NP];
 #pragma unroll
-                for (int i = 0; i < NE; ++i) d[i] = rs * ((g[v][i] - mg) - xh[v][i] * mgx);
-                if (valid[v]) st_stream(o + v * gt, E::pack(d));
+                for (int i = 0; i < NP; ++i) d[i] = mul2(rs2, sub2(sub2(g[v][i], mg2), mul2(xh[v][i], mgx2)));
+                if (valid[v]) st_stream(o + v * gt, P::pack(d));
             }
         }
     }
@@ -120,9 +122,9 @@ __global__ void __launch_bounds__(512) k_norm_bwd(const BArgs a, const int gt) {
         if (!valid[v]) continue;
         const int64_t c0 = static_cast<int64_t>(lg + v * gt) * NE;
 #pragma unroll
-        for (int i = 0; i < NE; ++i) {
-            pg[c0 + i] = accg[v][i];
-            if (!RMS) pg[static_cast<int64_t>(a.nvec) * NE + c0 + i] = accb[v][i];
+        for (int i = 0; i < NP; ++i) {
+            split(accg[v][i], pg[c0 + 2 * i], pg[c0 + 2 * i + 1]);
+            if (!RMS) split(accb[v][i], pg[static_cast<int64_t>(a.nvec) * NE + c0 + 2 * i], pg[static_cast<int64_t>(a.nvec) * NE + c0 + 2 * i + 1]);
         }
     }
 }
