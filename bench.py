@@ -480,6 +480,8 @@ def run_vecmat_table(args):
                         for rows in (1, 2, 4):
                             for ks in ((1, 2, 4) if lanes == 32 and kvec >= 1024 and ks_ok(threads) else (1,)):
                                 grid[f"{threads},{lanes},{rows},{ks}"] = timed(lambda: tf.tf_bvecmat_fwd(A, B, C, threads, lanes, rows, ks), reps)
+                if threads == 128 and kvec >= 64:
+                    grid["staged"] = timed(lambda: tf.tf_bvecmat_fwd(A, B, C, 0, 1), reps)
                 if w.dt == inputs.BF16 and threads < 1024:
                     for rows in (16, 32):
                         for ks in (1, 2, 4, 8):

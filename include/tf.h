@@ -195,6 +195,7 @@ tf_status tf_tune_add(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);
  * the operation is bound by HBM bandwidth.  Launch geometry, every knob 0 = automatic:
  *   threads  per CTA, a multiple of 32, at most 1024;
  *   lanes    per row group on the plain path (4, 8, 16 or 32); bf16 with lanes = 0 takes the tensor-core path;
+ *            lanes = 1 selects the shared-memory staged path (bulk copies into a four-stage ring; rows, ksplit ignored);
  *   rows     consecutive n that share one load of the A[m,:] pieces: 1, 2 or 4 per lane group on the plain path,
  *            16 or 32 per warp on the tensor-core path;
  *   ksplit   warps of a CTA that share a row group along k (1, 2, 4 or 8; on the plain path only with lanes = 32,

@@ -154,6 +154,10 @@ int round_up(int v, int m) { return (v + m - 1) / m * m; }
 }  // namespace
 
 void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+int* device_status_word() {
+    DevState* ds = nullptr;
+    return device_state(&ds) == TF_OK ? ds->status : nullptr;
+}
 void remember_cuda_error(cudaError_t e) { cuda_fail(e); }
 
 cudaError_t ensure_max_smem(const void* fn, const DeviceInfo& d) {

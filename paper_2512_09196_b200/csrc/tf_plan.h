@@ -100,6 +100,7 @@ size_t split_scratch_bytes(const Plan&, const Args&);
 
 // Bookkeeping shared with the C ABI layer: count kernel launches; remember the CUDA error behind a TF_ERR_CUDA.
 void count_launches(int n);
+int* device_status_word();     // this device's status word (bounded waits set it when they give up), or null before first use fails
 void remember_cuda_error(cudaError_t e);
 
 // Raises a kernel's dynamic shared-memory limit to the device's opt-in maximum, once per kernel and device.

@@ -193,6 +193,129 @@ __global__ void __launch_bounds__(WARPS * 32) k_vecmat_mma(const uint4* __restri
     }
 }
 
+// Long rows, staged: the register paths above read a long row 128 B at a time per warp and step, from 16 rows that
+// lie kilobytes apart; here a producer lane copies 1 KiB of each of a tile's 16 rows (and of A[m,:]) per stage into a
+// four-stage shared-memory ring with bulk copies (no multicast), so that memory sees long contiguous reads and the
+// bytes in flight (three CTAs x 72 KiB per SM) cost no registers; four consumer warps take the stage apart.
+// bf16: every warp multiplies a quarter of the chunk for all 16 rows through m16n8k16 (fragments read from shared
+// memory; rows are padded by 64 B so that a quarter-warp's 16-byte reads hit distinct banks) and the four partial
+// sums meet in shared memory at the end.  fp32: every warp owns four rows.  Every wait is bounded: on expiry the CTA
+// sets the library's status word, stops waiting and finishes with uniform control flow.
+constexpr int kTmRows = 16, kTmChunk = 1024, kTmPad = 64, kTmStages = 4;
+constexpr int kTmRowStride = kTmChunk + kTmPad;
+constexpr int kTmStageBytes = kTmRows * kTmRowStride + kTmChunk;
+constexpr int kTmThreads = 160;                                   // four consumer warps and the producer's warp
+
+template <int DT>
+__global__ void __launch_bounds__(kTmThreads) k_vecmat_tma(const unsigned char* __restrict__ A, const unsigned char* __restrict__ B,
+                                                           typename Elem<DT>::scalar* __restrict__ C, int64_t N, int64_t row_bytes,
+                                                           int tiles_per_m, int* status) {
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) uint64_t full[kTmStages], empty[kTmStages];
+    __shared__ float part[4][kTmRows];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t tile = blockIdx.x;
+    const int64_t m = tile / tiles_per_m, n0 = (tile - m * tiles_per_m) * kTmRows;
+    const int n_left = static_cast<int>(N - n0 < kTmRows ? N - n0 : kTmRows);
+    const int steps = static_cast<int>((row_bytes + kTmChunk - 1) / kTmChunk);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTmStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 4); }
+        mbar_fence_init();
+    }
+    pdl_wait();
+    __syncthreads();
+    pdl_trigger();
+    float out0 = 0.f, out1 = 0.f;                                 // bf16: rows g and g + 8 of this warp's k quarter
+    F2 acc[4] = {f2(0.f), f2(0.f), f2(0.f), f2(0.f)};              // fp32: this warp's four rows
+    if (warp == 4) {
+        // the producer's warp: lane 0 waits for the stage to be free and announces the bytes, then lanes 0..n_left-1 each
+        // copy their row's piece and lane 16 the piece of A[m,:] (one lane issuing all 17 copies was the bottleneck)
+        const unsigned char* a = A + m * row_bytes;
+        const unsigned char* b = B + (m * N + n0) * row_bytes;
+        int issued = 0;
+        for (int s = 0; s < steps; ++s) {
+            const int st = s % kTmStages;
+            int ok = 1;
+            if (lane == 0 && s >= kTmStages && !mbar_wait(&empty[st], static_cast<uint32_t>(s / kTmStages - 1) & 1u)) { atomicExch(status, 4); ok = 0; }
+            ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+            if (!ok) break;                                           // uniform over the warp
+            const int64_t off = static_cast<int64_t>(s) * kTmChunk;
+            const uint32_t bytes = static_cast<uint32_t>(row_bytes - off < kTmChunk ? row_bytes - off : kTmChunk);
+            unsigned char* dst = ring + st * kTmStageBytes;
+            if (lane == 0) mbar_expect_tx(&full[st], bytes * static_cast<uint32_t>(n_left + 1));
+            __syncwarp();
+            if (lane < n_left) bulk_g2s(dst + lane * kTmRowStride, b + lane * row_bytes + off, bytes, &full[st]);
+            if (lane == 16) bulk_g2s(dst + kTmRows * kTmRowStride, a + off, bytes, &full[st]);
+            issued = s + 1;
+        }
+        // no copy may still be in flight when the CTA ends, even if the consumers gave up: poll (bounded) the barriers
+        // of the last stages that were fed
+        if (lane == 0)
+            for (int s = issued > kTmStages ? issued - kTmStages : 0; s < issued; ++s)
+                if (!mbar_wait(&full[s % kTmStages], static_cast<uint32_t>(s / kTmStages) & 1u)) { atomicExch(status, 4); break; }
+    } else {
+        bool failed = false;
+        const int g = lane >> 2, t = lane & 3;
+        for (int s = 0; s < steps; ++s) {
+            const int st = s % kTmStages;
+            if (!failed && !mbar_wait(&full[st], static_cast<uint32_t>(s / kTmStages) & 1u)) { failed = true; atomicExch(status, 4); }
+            const int64_t off = static_cast<int64_t>(s) * kTmChunk;
+            const int nv = static_cast<int>((row_bytes - off < kTmChunk ? row_bytes - off : kTmChunk) / 16);     // vectors of this chunk
+            const unsigned char* src = ring + st * kTmStageBytes;
+            const uint4 zero = make_uint4(0, 0, 0, 0);
+            if (!failed) {
+                if constexpr (DT == DT_BF16) {
+                    float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int vi = warp * 16 + j * 4 + t;                          // this warp's quarter of the chunk
+                        const bool ok = vi < nv;
+                        const uint4 r0 = ok && g < n_left ? *reinterpret_cast<const uint4*>(src + g * kTmRowStride + vi * 16) : zero;
+                        const uint4 r1 = ok && g + 8 < n_left ? *reinterpret_cast<const uint4*>(src + (g + 8) * kTmRowStride + vi * 16) : zero;
+                        const uint4 v = ok ? *reinterpret_cast<const uint4*>(src + kTmRows * kTmRowStride + vi * 16) : zero;
+                        mma_bf16_16816(c, r0.x, r1.x, r0.y, r1.y, v.x, v.y);
+                        mma_bf16_16816(c, r0.z, r1.z, r0.w, r1.w, v.z, v.w);
+                    }
+                    out0 += c[0];
+                    out1 += c[2];
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int vi = lane + 32 * u;
+                        if (vi < nv) {
+                            F2 y[2];
+                            Pairs<DT_F32>::unpack(*reinterpret_cast<const uint4*>(src + kTmRows * kTmRowStride + vi * 16), y);
+#pragma unroll
+                            for (int r = 0; r < 4; ++r) {
+                                if (warp * 4 + r < n_left) {
+                                    F2 x[2];
+                                    Pairs<DT_F32>::unpack(*reinterpret_cast<const uint4*>(src + (warp * 4 + r) * kTmRowStride + vi * 16), x);
+                                    acc[r] = fma2(x[0], y[0], acc[r]);
+                                    acc[r] = fma2(x[1], y[1], acc[r]);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[st]);               // also after a failure: the producer must not be left waiting
+        }
+        if constexpr (DT == DT_BF16) {
+            if (t == 0) { part[warp][g] = out0; part[warp][g + 8] = out1; }
+        } else {
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const float dot = group_reduce<SumOp, 32>(hsum(acc[r]));
+                if (lane == 0 && warp * 4 + r < n_left) C[m * N + n0 + warp * 4 + r] = Elem<DT>::from_float(dot);
+            }
+        }
+    }
+    __syncthreads();
+    if (DT == DT_BF16 && warp == 0 && lane < n_left)
+        C[m * N + n0 + lane] = Elem<DT>::from_float((part[0][lane] + part[1][lane]) + (part[2][lane] + part[3][lane]));
+}
+
 // Any alignment, any K: a warp per row, scalar accesses.
 template <int DT>
 __global__ void __launch_bounds__(1024) k_vecmat_scalar(const typename Elem<DT>::scalar* A, const typename Elem<DT>::scalar* B,
@@ -316,6 +439,30 @@ cudaError_t launch_mma(int rows, int ksplit, int threads, cudaStream_t st, const
                           : launch_mma_wr<16, 1>(st, A, B, C, M, N, kvec, ksplit);
 }
 
+template <int DT>
+cudaError_t launch_tma(cudaStream_t st, const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t row_bytes) {
+    using S = typename Elem<DT>::scalar;
+    const int64_t tiles_per_m = (N + kTmRows - 1) / kTmRows, tiles = M * tiles_per_m;
+    if (tiles_per_m > 0x7FFFFFFF || tiles > 0x7FFFFFFF || row_bytes / kTmChunk > 0x7FFFFF00) return cudaErrorInvalidConfiguration;
+    int* status = device_status_word();
+    if (!status) return cudaErrorInitializationError;
+    const int smem = kTmStages * kTmStageBytes;
+    cudaError_t e = cudaFuncSetAttribute(k_vecmat_tma<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(tiles));
+    cfg.blockDim = dim3(kTmThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_vecmat_tma<DT>, static_cast<const unsigned char*>(A), static_cast<const unsigned char*>(B),
+                              static_cast<S*>(C), N, row_bytes, static_cast<int>(tiles_per_m), status);
+}
+
 }  // namespace
 }  // namespace tf
 
@@ -327,7 +474,9 @@ extern "C" tf_status tf_bvecmat_fwd(const void* A, const void* B, void* C, int64
     if (M < 0 || N < 0 || K <= 0 || (dt != DT_F32 && dt != DT_BF16)) return TF_ERR_INVALID_ARG;
     if (M > 0 && N > 0 && (!A || !B || !C)) return TF_ERR_INVALID_ARG;
     if (threads == 0) threads = 128;
-    const bool tensor = dt == DT_BF16 && lanes == 0;              // a forced `lanes` selects the plain path
+    const bool staged = lanes == 1;                               // the shared-memory staged path
+    const bool tensor = dt == DT_BF16 && lanes == 0;              // any other forced `lanes` selects the plain path
+    if (staged) { lanes = 0; rows = 0; ksplit = 0; }
     if (threads < 32 || threads > 1024 || threads % 32 || (lanes != 0 && lanes != 4 && lanes != 8 && lanes != 16 && lanes != 32) ||
         (ksplit != 0 && ksplit != 1 && ksplit != 2 && ksplit != 4 && ksplit != 8))
         return TF_ERR_INVALID_ARG;
@@ -342,7 +491,8 @@ extern "C" tf_status tf_bvecmat_fwd(const void* A, const void* B, void* C, int64
     count_launches(1);
     if (al16(A) && al16(B) && (K * es) % 16 == 0) {
         const int64_t kvec = K * es / 16;
-        if (tensor) e = launch_mma(rows, ksplit, threads, st, A, B, C, M, N, kvec);
+        if (staged) e = dt == DT_F32 ? launch_tma<DT_F32>(st, A, B, C, M, N, K * es) : launch_tma<DT_BF16>(st, A, B, C, M, N, K * es);
+        else if (tensor) e = launch_mma(rows, ksplit, threads, st, A, B, C, M, N, kvec);
         else if (dt == DT_F32) e = launch_plain<DT_F32>(lanes, rows, ksplit, threads, st, A, B, C, M, N, kvec);
         else e = launch_plain<DT_BF16>(lanes, rows, ksplit, threads, st, A, B, C, M, N, kvec);
     } else {

@@ -59,6 +59,15 @@ def test_every_k_split_of_the_plain_path(dt):
                     check(inputs.VecMat(f"t_{M}x{N}x{K}", dt, M, N, K, seed=K + ksplit), threads, 32, ksplit=ksplit, rows=rows)
 
 
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_staged_path(dt):
+    # lanes = 1: the shared-memory staged kernel; row lengths around the 1 KiB stage, tiles with fewer than 16 rows
+    ne = 4 if dt == F32 else 8
+    for M, N, K in ((1, 1, ne), (3, 37, 2 * ne), (2, 16, 1024 // (16 // ne)), (2, 33, 1024 // (16 // ne) + ne), (5, 129, 1032), (1, 19, 8200),
+                    (2, 15, 640), (1, 1, 32768), (4, 64, 4096), (2, 100, 5000 // ne * ne)):
+        check(inputs.VecMat(f"t_{M}x{N}x{K}", dt, M, N, K, seed=K + 1), lanes=1)
+
+
 def test_every_k_split_of_the_tensor_core_path():
     for ksplit in (1, 2, 4, 8):
         for threads in (128, 256, 512):
