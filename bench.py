@@ -702,7 +702,8 @@ def run_normbwd_table(args):
     out_dir = ROOT / "gpurun_out"
     out_dir.mkdir(exist_ok=True)
     shapes = [("rmsnorm", inputs.BF16, 16384, 4096), ("rmsnorm", inputs.BF16, 16384, 8192), ("rmsnorm", inputs.F32, 16384, 4096),
-              ("layernorm", inputs.BF16, 16384, 4096), ("layernorm", inputs.BF16, 65536, 1024), ("layernorm", inputs.F32, 8192, 8192),
+              ("layernorm", inputs.BF16, 16384, 4096), ("layernorm", inputs.BF16, 16384, 8192), ("layernorm", inputs.BF16, 65536, 1024),
+              ("layernorm", inputs.F32, 8192, 8192),
               ("layernorm", inputs.BF16, 4096, 16384)]
     rows_out = []
     for op, dt, rows, cols in shapes:

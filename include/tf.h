@@ -232,6 +232,11 @@ tf_status tf_query_choice(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int
 int tf_candidate_count(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);
 tf_status tf_candidate(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int index, char* buf, size_t n);
 
+/* Which form of the norm backward passes runs on shapes that both serve: path 0 = automatic, 1 = rows requested into
+ * registers one row ahead, 2 = rows staged in a shared-memory ring by bulk copies (up to 512 threads per row), 3 = the
+ * same with up to 256 threads per row; stages = ring depth (0 = automatic, at most 8).  Ask tf_norm_bwd_workspace_bytes again after changing it.  TF_ERR_INVALID_ARG outside those ranges. */
+tf_status tf_norm_bwd_force(int path, int stages);
+
 /* Forgets every tuned plan (in memory only). */
 void tf_clear_cache(void);
 

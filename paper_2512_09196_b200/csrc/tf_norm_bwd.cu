@@ -8,6 +8,10 @@
 // widened in registers and accumulates its slice of dgamma / dbeta in fp32 across all the rows it meets.  At the end
 // every CTA writes its partial column sums to the caller's workspace and a second kernel adds the partials in a fixed
 // order (deterministic) and rounds once.  x and dy are read once, dx written once.
+// Two forms of that kernel: one requests the next row (and its statistics) into registers before it reduces the current
+// one; the other lets bulk copies bring the rows into a shared-memory ring, which keeps more bytes in flight than
+// registers can and is what 2-byte rows of 8 KiB and more take.  Both have a specialisation without predicates for
+// shapes in which no vector and no row slot is ever absent.
 // Rows beyond what 512 threads hold (16 KiB bf16, 32 KiB fp32) are streamed twice by one CTA per SM that keeps its
 // partial column sums in shared memory (up to 200 KiB of them); unaligned tensors, odd widths and wider rows still take
 // two plain kernels: scalar passes per row for dx, a thread per column for the parameter gradients.
@@ -32,10 +36,29 @@ struct BArgs {
     float inv_n;
 };
 
+// Sum of the wg per-warp partials of a row group, the same bits in every thread of the group.  A power-of-two count is
+// added as a butterfly (lane l starts from partial l mod wg; every lane walks the same tree, so all get the same bits):
+// one shared-memory read and log2(wg) shuffles instead of wg reads.
+__device__ __forceinline__ void group_total(const float2* part, int wg, int lane, float& a, float& b) {
+    if ((wg & (wg - 1)) == 0) {
+        const float2 p = part[lane & (wg - 1)];
+        a = p.x; b = p.y;
+        for (int o = wg >> 1; o > 0; o >>= 1) {
+            a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
+            b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
+        }
+    } else {
+        a = 0.f; b = 0.f;
+        for (int w = 0; w < wg; ++w) { const float2 p = part[w]; a += p.x; b += p.y; }
+    }
+}
+
 // A CTA is cut into row groups of `gt` threads (a multiple of 32); every group owns one row per iteration, so short rows
 // still fill a CTA and one barrier per iteration serves all of them.  Group-wide sums: warp shuffles, one float2 per warp
 // in shared memory, one barrier, then every thread adds the partials of its own group's warps.
-template <bool RMS, int DT, int VPT>
+// FULL: every thread's vectors exist and every row group meets a row in every iteration, so nothing needs a predicate
+// or a zero fill (selects and fills were a quarter of the instructions of the general form).
+template <bool RMS, int DT, int VPT, bool FULL>
 __global__ void __launch_bounds__(512) k_norm_bwd(const BArgs a, const int gt) {
     using E = Elem<DT>;
     using P = Pairs<DT>;
@@ -49,7 +72,7 @@ __global__ void __launch_bounds__(512) k_norm_bwd(const BArgs a, const int gt) {
     F2 gam[VPT][NP], accg[VPT][NP], accb[RMS ? 1 : VPT][NP];
 #pragma unroll
     for (int v = 0; v < VPT; ++v) {
-        valid[v] = lg + v * gt < a.nvec;
+        valid[v] = FULL || lg + v * gt < a.nvec;
         P::unpack(valid[v] ? ld_param(a.gamma + lg + v * gt) : make_uint4(0, 0, 0, 0), gam[v]);
 #pragma unroll
         for (int i = 0; i < NP; ++i) { accg[v][i] = f2(0.f); if (!RMS) accb[v][i] = f2(0.f); }
@@ -57,10 +80,26 @@ __global__ void __launch_bounds__(512) k_norm_bwd(const BArgs a, const int gt) {
     // the packed vectors of the NEXT row are requested before the current row is reduced, so that the reduction of a
     // row does not leave the memory pipe idle
     uint4 nx[VPT], nd[VPT];
+    float nmu = 0.f, nrs = 0.f;                                          // and its statistics: a load at the top of the iteration would stall it
     auto request = [&](int64_t row) {
+        const bool in = row < a.rows;
+        if (FULL) {                                                      // past the end: keep the stale registers, nobody reads them
+            if (in) {
+                nmu = RMS ? 0.f : __ldg(a.mean + row);
+                nrs = __ldg(a.rstd + row);
+#pragma unroll
+                for (int v = 0; v < VPT; ++v) {
+                    nx[v] = ld_stream(a.x + row * a.nvec + lg + v * gt);
+                    nd[v] = ld_stream(a.dy + row * a.nvec + lg + v * gt);
+                }
+            }
+            return;
+        }
+        nmu = (RMS || !in) ? 0.f : __ldg(a.mean + row);
+        nrs = in ? __ldg(a.rstd + row) : 0.f;
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
-            const bool ok = valid[v] && row < a.rows;
+            const bool ok = valid[v] && in;
             nx[v] = ok ? ld_stream(a.x + row * a.nvec + lg + v * gt) : make_uint4(0, 0, 0, 0);
             nd[v] = ok ? ld_stream(a.dy + row * a.nvec + lg + v * gt) : make_uint4(0, 0, 0, 0);
         }
@@ -70,9 +109,9 @@ __global__ void __launch_bounds__(512) k_norm_bwd(const BArgs a, const int gt) {
     int it = 0;
     for (int64_t row0 = static_cast<int64_t>(blockIdx.x) * R; row0 < a.rows; row0 += stride, ++it) {      // same trip count for the whole CTA
         const int64_t row = row0 + gid;
-        const bool live = row < a.rows;
-        const float mu = (RMS || !live) ? 0.f : __ldg(a.mean + row), rs = live ? __ldg(a.rstd + row) : 0.f;
-        const F2 mu2 = f2(mu), rs2 = f2(rs);
+        const bool live = FULL || row < a.rows;
+        const float rs = nrs;
+        const F2 mu2 = f2(nmu), rs2 = f2(rs);
         F2 xh[VPT][NP], g[VPT][NP], dv[VPT][NP];
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
@@ -100,22 +139,151 @@ __global__ void __launch_bounds__(512) k_norm_bwd(const BArgs a, const int gt) {
         if (wg > 1) {
             if (lane == 0) red[it & 1][warp] = make_float2(sgx, sg);
             __syncthreads();
-            sgx = 0.f; sg = 0.f;
-            for (int w = 0; w < wg; ++w) { const float2 p = red[it & 1][gid * wg + w]; sgx += p.x; sg += p.y; }
+            group_total(red[it & 1] + gid * wg, wg, lane, sgx, sg);
         }
-        const F2 mgx2 = f2(sgx * a.inv_n), mg2 = f2(RMS ? 0.f : sg * a.inv_n);
+        // dx = rstd g - rstd mean(g) - xh rstd mean(g xh): two fused multiply-adds per pair
+        const F2 c1 = f2(-rs * (sgx * a.inv_n)), c0 = f2(RMS ? 0.f : -rs * (sg * a.inv_n));
         if (live) {
             uint4* o = a.dx + row * a.nvec + lg;
 #pragma unroll
             for (int v = 0; v < VPT; ++v) {
                 F2 d[NP];
 #pragma unroll
-                for (int i = 0; i < NP; ++i) d[i] = mul2(rs2, sub2(sub2(g[v][i], mg2), mul2(xh[v][i], mgx2)));
+                for (int i = 0; i < NP; ++i) d[i] = fma2(xh[v][i], c1, fma2(g[v][i], rs2, c0));
                 if (valid[v]) st_stream(o + v * gt, P::pack(d));
             }
         }
     }
     // this row group's partial column sums (zeros if it met no row): part index = CTA * R + group
+    float* pg = a.part + (static_cast<int64_t>(blockIdx.x) * R + gid) * (RMS ? 1 : 2) * a.nvec * NE;
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+        if (!valid[v]) continue;
+        const int64_t c0 = static_cast<int64_t>(lg + v * gt) * NE;
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+            split(accg[v][i], pg[c0 + 2 * i], pg[c0 + 2 * i + 1]);
+            if (!RMS) split(accb[v][i], pg[static_cast<int64_t>(a.nvec) * NE + c0 + 2 * i], pg[static_cast<int64_t>(a.nvec) * NE + c0 + 2 * i + 1]);
+        }
+    }
+}
+
+// Staged form of the same kernel: the tile of R consecutive rows that the CTA's row groups take per iteration is one
+// contiguous range of x and one of dy, so it arrives in a shared-memory ring stage by two bulk copies (no multicast)
+// counted on the stage's mbarrier.  The bytes in flight are then the ring (64-128 KiB per CTA) and not the one row that
+// registers can request ahead, which is what held the register form of the 2-byte types below the copy rate.  The
+// barrier of the row reduction is also the point after which every thread has taken its vectors out of the stage, so
+// thread 0 refills that stage right behind it; no producer warp, no "empty" barrier.  Waits are bounded: a CTA that
+// gives up sets the status word, stops issuing copies and finishes its loop without waiting again.
+constexpr int kBwdMaxStages = 8;
+
+template <bool RMS, int DT, int VPT, bool FULL>
+__global__ void __launch_bounds__(512) k_norm_bwd_staged(const BArgs a, const int gt, const int S, int* status) {
+    using P = Pairs<DT>;
+    constexpr int NE = Elem<DT>::NE, NP = P::NP;
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    __shared__ __align__(8) uint64_t full[kBwdMaxStages];
+    __shared__ float2 red[2][16];
+    const int t = threadIdx.x, gid = t / gt, lg = t % gt, R = blockDim.x / gt, wg = gt / 32;
+    const int warp = t >> 5, lane = t & 31;
+    const size_t tile_vecs = static_cast<size_t>(R) * a.nvec;                 // vectors of x (and of dy) per stage
+    uint4* const ring = reinterpret_cast<uint4*>(dyn_smem);                    // [S][x | dy][R][nvec]
+    const int64_t num_tiles = (a.rows + R - 1) / R;
+    if (t == 0) {
+        for (int s = 0; s < S; ++s) mbar_init(&full[s], 1);
+        mbar_fence_init();
+    }
+    pdl_wait();
+    auto issue = [&](int64_t tile, int s) {                                    // thread 0 only
+        const int64_t row0 = tile * R;
+        const uint32_t bytes = static_cast<uint32_t>(min(static_cast<int64_t>(R), a.rows - row0)) * a.nvec * 16u;
+        mbar_expect_tx(&full[s], 2u * bytes);
+        bulk_g2s(ring + tile_vecs * (2 * s), a.x + row0 * a.nvec, bytes, &full[s]);
+        bulk_g2s(ring + tile_vecs * (2 * s + 1), a.dy + row0 * a.nvec, bytes, &full[s]);
+    };
+    if (t == 0)
+        for (int s = 0; s < S; ++s) {
+            const int64_t tile = blockIdx.x + static_cast<int64_t>(s) * gridDim.x;
+            if (tile < num_tiles) issue(tile, s);
+        }
+    bool valid[VPT];
+    F2 gam[VPT][NP], accg[VPT][NP], accb[RMS ? 1 : VPT][NP];
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+        valid[v] = FULL || lg + v * gt < a.nvec;
+        P::unpack(valid[v] ? ld_param(a.gamma + lg + v * gt) : make_uint4(0, 0, 0, 0), gam[v]);
+#pragma unroll
+        for (int i = 0; i < NP; ++i) { accg[v][i] = f2(0.f); if (!RMS) accb[v][i] = f2(0.f); }
+    }
+    __syncthreads();                                                           // barriers initialised
+    pdl_trigger();
+    bool failed = false;
+    int it = 0, s = 0;
+    uint32_t parity = 0;
+    float nmu = 0.f, nrs = 0.f;                                                // the statistics of a row are requested one tile ahead
+    auto request_stats = [&](int64_t tile) {
+        const int64_t row = tile * R + gid;
+        const bool in = tile < num_tiles && row < a.rows;
+        if (FULL) {
+            if (in) { nmu = RMS ? 0.f : __ldg(a.mean + row); nrs = __ldg(a.rstd + row); }
+            return;
+        }
+        nmu = (RMS || !in) ? 0.f : __ldg(a.mean + row);
+        nrs = in ? __ldg(a.rstd + row) : 0.f;
+    };
+    request_stats(blockIdx.x);
+    for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {       // same trip count for the whole CTA
+        if (!failed && !mbar_wait(&full[s], parity)) {
+            failed = true;
+            atomicExch(status, 4);
+            mbar_wait(&full[s], parity);                                       // one more bounded wait for the copies
+        }
+        const int64_t row = tile * R + gid;
+        const bool live = FULL || row < a.rows;
+        const float rs = nrs;
+        const F2 mu2 = f2(nmu), rs2 = f2(rs);
+        request_stats(tile + gridDim.x);
+        const uint4* sx = ring + tile_vecs * (2 * s) + static_cast<size_t>(gid) * a.nvec + lg;
+        const uint4* sd = sx + tile_vecs;
+        F2 xh[VPT][NP], g[VPT][NP], dv[VPT][NP];
+        F2 sgx2 = f2(0.f), sg2 = f2(0.f);
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            const bool ok = valid[v] && live;                                  // rows past the end were not copied
+            F2 xv[NP];
+            P::unpack(ok ? sx[v * gt] : make_uint4(0, 0, 0, 0), xv);
+            P::unpack(ok ? sd[v * gt] : make_uint4(0, 0, 0, 0), dv[v]);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                xh[v][i] = ok ? mul2(sub2(xv[i], mu2), rs2) : f2(0.f);
+                g[v][i] = mul2(dv[v][i], gam[v][i]);
+                sgx2 = fma2(g[v][i], xh[v][i], sgx2);
+                sg2 = add2(sg2, g[v][i]);
+                accg[v][i] = fma2(dv[v][i], xh[v][i], accg[v][i]);
+                if (!RMS) accb[v][i] = add2(accb[v][i], dv[v][i]);
+            }
+        }
+        float sgx = group_reduce<SumOp, 32>(hsum(sgx2));
+        float sg = group_reduce<SumOp, 32>(hsum(sg2));
+        if (lane == 0) red[it & 1][warp] = make_float2(sgx, sg);
+        __syncthreads();                                                       // also: every thread has left the stage
+        const int64_t next = tile + static_cast<int64_t>(S) * gridDim.x;
+        if (t == 0 && !failed && next < num_tiles) issue(next, s);
+        if (wg > 1) group_total(red[it & 1] + gid * wg, wg, lane, sgx, sg);
+        // dx = rstd g - rstd mean(g) - xh rstd mean(g xh): two fused multiply-adds per pair
+        const F2 c1 = f2(-rs * (sgx * a.inv_n)), c0 = f2(RMS ? 0.f : -rs * (sg * a.inv_n));
+        if (live) {
+            uint4* o = a.dx + row * a.nvec + lg;
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) {
+                F2 d[NP];
+#pragma unroll
+                for (int i = 0; i < NP; ++i) d[i] = fma2(xh[v][i], c1, fma2(g[v][i], rs2, c0));
+                if (valid[v]) st_stream(o + v * gt, P::pack(d));
+            }
+        }
+        if (++s == S) { s = 0; parity ^= 1u; }
+    }
     float* pg = a.part + (static_cast<int64_t>(blockIdx.x) * R + gid) * (RMS ? 1 : 2) * a.nvec * NE;
 #pragma unroll
     for (int v = 0; v < VPT; ++v) {
@@ -305,27 +473,79 @@ cudaError_t launch_pdl(void (*fn)(T...), int64_t grid, int threads, cudaStream_t
     return cudaLaunchKernelEx(&cfg, fn, args...);
 }
 
-// Launch geometry of the register-resident kernel: vectors per thread, threads per row group, row groups per CTA, CTAs.
-struct BwdPlan { int vpt, gt, groups, grid; };
+// Test and bench hook: 0 = automatic, 1 = the register form, 2 = the staged form with row groups of up to 512 threads,
+// 3 = the staged form with row groups of up to 256 threads; stages 0 = automatic.
+int g_force_path = 0, g_force_stages = 0;
+
+// Launch geometry of the row-group kernels: vectors per thread, threads per row group, row groups per CTA, CTAs; for
+// the staged form also the ring's stages and bytes (stages = 0: the register form).
+struct BwdPlan { int vpt, gt, groups, grid, stages; size_t smem; bool full; };
+
+template <bool RMS, int DT, int VPT> const void* bwd_fn(bool staged, bool full) {
+    return staged ? (full ? reinterpret_cast<const void*>(k_norm_bwd_staged<RMS, DT, VPT, true>) : reinterpret_cast<const void*>(k_norm_bwd_staged<RMS, DT, VPT, false>))
+           : full ? reinterpret_cast<const void*>(k_norm_bwd<RMS, DT, VPT, true>) : reinterpret_cast<const void*>(k_norm_bwd<RMS, DT, VPT, false>);
+}
 
 template <bool RMS, int DT>
-BwdPlan bwd_plan(int64_t rows, int nvec) {
+BwdPlan bwd_plan(int64_t rows, int nvec, bool staged, int stages, int gmax = 256) {
     constexpr int kMaxVpt = Elem<DT>::NE == 4 ? 4 : 2;            // 5 register arrays of VPT * NE fp32 values per thread
-    BwdPlan p;
+    BwdPlan p{};
     p.vpt = 1;
-    while (p.vpt < kMaxVpt && (nvec + p.vpt - 1) / p.vpt > 256) p.vpt *= 2;     // row groups of up to 256 threads while that holds the row
+    while (p.vpt < kMaxVpt && (nvec + p.vpt - 1) / p.vpt > gmax) p.vpt *= 2;    // row groups of up to gmax threads while that holds the row
     p.gt = std::max(32, ((nvec + p.vpt - 1) / p.vpt + 31) / 32 * 32);
     p.groups = std::max(1, std::min(8, 256 / p.gt));                            // short rows: several per CTA
     const int threads = p.gt * p.groups;
-    const void* fn = p.vpt == 1 ? reinterpret_cast<const void*>(k_norm_bwd<RMS, DT, 1>)
-                   : p.vpt == 2 ? reinterpret_cast<const void*>(k_norm_bwd<RMS, DT, 2>)
-                                : reinterpret_cast<const void*>(k_norm_bwd<RMS, DT, kMaxVpt>);
+    p.full = nvec == p.gt * p.vpt && rows % p.groups == 0;          // no vector and no row slot is ever absent
+    const void* fn = p.vpt == 1 ? bwd_fn<RMS, DT, 1>(staged, p.full) : p.vpt == 2 ? bwd_fn<RMS, DT, 2>(staged, p.full) : bwd_fn<RMS, DT, kMaxVpt>(staged, p.full);
+    if (staged) {
+        // ring: the shared memory of an SM divided among the CTAs its register file holds (at most three), up to eight stages
+        const size_t stage = static_cast<size_t>(2) * p.groups * nvec * 16;
+        int by_regs = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&by_regs, fn, threads, 0) != cudaSuccess || by_regs < 1) by_regs = 1;
+        by_regs = std::min(by_regs, 3);
+        while (by_regs > 1 && (216 * 1024 / by_regs) / stage < 2) --by_regs;
+        // three stages are enough (deeper rings measured a few percent slower)
+        p.stages = stages > 0 ? stages : static_cast<int>(std::min<size_t>(3, (216 * 1024 / by_regs) / stage));
+        p.stages = std::min(p.stages, kBwdMaxStages);
+        p.smem = stage * p.stages;
+        if (p.stages < 2 || p.smem > 216 * 1024 ||
+            cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024) != cudaSuccess) {      // the same limit for every shape
+            p.stages = 0; p.grid = 0; return p;                                         // does not fit: not available
+        }
+    }
     // as many CTAs as are resident at once: every further CTA would only add partial column sums to write and to add up
     int per_sm = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, p.smem) != cudaSuccess || per_sm < 1) per_sm = 1;
     const int64_t want = (rows + p.groups - 1) / p.groups;
     p.grid = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(want, static_cast<int64_t>(per_sm) * sm_count())));
     return p;
+}
+
+// Which form runs, unless the hook says otherwise: the staged one for 2-byte elements in rows of 8 KiB and more (measured
+// 9-15 % faster there: a row ahead in registers is half as many bytes in flight as with 4-byte elements), the register
+// form elsewhere (shorter rows and 4-byte elements: equal or faster).
+template <bool RMS, int DT>
+BwdPlan choose_bwd_plan_uncached(int64_t rows, int nvec) {
+    const bool want = g_force_path >= 2 || (g_force_path == 0 && DT == DT_BF16 && nvec >= 512);
+    if (want) {
+        const BwdPlan p = bwd_plan<RMS, DT>(rows, nvec, true, g_force_stages, g_force_path == 2 ? 512 : 256);
+        if (p.stages >= 2) return p;
+    }
+    return bwd_plan<RMS, DT>(rows, nvec, false, 0);
+}
+
+template <bool RMS, int DT>
+BwdPlan choose_bwd_plan(int64_t rows, int nvec) {
+    // the plan of the last shape is kept (per thread): the occupancy queries cost more host time than a launch
+    struct Key { int64_t rows; int nvec, path, stages, dev; };
+    thread_local Key last{-1, 0, 0, 0, -1};
+    thread_local BwdPlan kept{};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (last.rows == rows && last.nvec == nvec && last.path == g_force_path && last.stages == g_force_stages && last.dev == dev) return kept;
+    last = Key{rows, nvec, g_force_path, g_force_stages, dev};
+    kept = choose_bwd_plan_uncached<RMS, DT>(rows, nvec);
+    return kept;
 }
 
 template <bool RMS, int DT>
@@ -339,7 +559,7 @@ tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float*
     cudaError_t e;
     if (aligned && bytes / 16 <= 512 * kMaxVpt && cols <= 0x7FFFFFFF) {
         const int nvec = static_cast<int>(bytes / 16);
-        const BwdPlan p = bwd_plan<RMS, DT>(rows, nvec);
+        const BwdPlan p = choose_bwd_plan<RMS, DT>(rows, nvec);
         const int parts = p.grid * p.groups;
         const size_t need = static_cast<size_t>(parts) * (RMS ? 1 : 2) * cols * 4;
         if (!ws || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 3u)) return TF_ERR_INVALID_ARG;
@@ -347,9 +567,33 @@ tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float*
                 static_cast<uint4*>(dx), static_cast<float*>(ws), rows, nvec, 1.0f / static_cast<float>(cols)};
         count_launches(2);
         const int threads = p.gt * p.groups;
-        if (p.vpt == 1) e = launch_pdl(k_norm_bwd<RMS, DT, 1>, p.grid, threads, st, a, p.gt);
-        else if (p.vpt == 2) e = launch_pdl(k_norm_bwd<RMS, DT, 2>, p.grid, threads, st, a, p.gt);
-        else e = launch_pdl(k_norm_bwd<RMS, DT, kMaxVpt>, p.grid, threads, st, a, p.gt);
+        if (p.stages >= 2) {
+            int* status = device_status_word();
+            if (!status) return TF_ERR_CUDA;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(p.grid);
+            cfg.blockDim = dim3(threads);
+            cfg.dynamicSmemBytes = p.smem;
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (p.full) {
+                if (p.vpt == 1) e = cudaLaunchKernelEx(&cfg, k_norm_bwd_staged<RMS, DT, 1, true>, a, p.gt, p.stages, status);
+                else if (p.vpt == 2) e = cudaLaunchKernelEx(&cfg, k_norm_bwd_staged<RMS, DT, 2, true>, a, p.gt, p.stages, status);
+                else e = cudaLaunchKernelEx(&cfg, k_norm_bwd_staged<RMS, DT, kMaxVpt, true>, a, p.gt, p.stages, status);
+            } else if (p.vpt == 1) e = cudaLaunchKernelEx(&cfg, k_norm_bwd_staged<RMS, DT, 1, false>, a, p.gt, p.stages, status);
+            else if (p.vpt == 2) e = cudaLaunchKernelEx(&cfg, k_norm_bwd_staged<RMS, DT, 2, false>, a, p.gt, p.stages, status);
+            else e = cudaLaunchKernelEx(&cfg, k_norm_bwd_staged<RMS, DT, kMaxVpt, false>, a, p.gt, p.stages, status);
+        } else if (p.full) {
+            if (p.vpt == 1) e = launch_pdl(k_norm_bwd<RMS, DT, 1, true>, p.grid, threads, st, a, p.gt);
+            else if (p.vpt == 2) e = launch_pdl(k_norm_bwd<RMS, DT, 2, true>, p.grid, threads, st, a, p.gt);
+            else e = launch_pdl(k_norm_bwd<RMS, DT, kMaxVpt, true>, p.grid, threads, st, a, p.gt);
+        } else if (p.vpt == 1) e = launch_pdl(k_norm_bwd<RMS, DT, 1, false>, p.grid, threads, st, a, p.gt);
+        else if (p.vpt == 2) e = launch_pdl(k_norm_bwd<RMS, DT, 2, false>, p.grid, threads, st, a, p.gt);
+        else e = launch_pdl(k_norm_bwd<RMS, DT, kMaxVpt, false>, p.grid, threads, st, a, p.gt);
         if (e == cudaSuccess)
             e = launch_pdl(k_colsum_finish<RMS, DT>, (cols + 31) / 32, 256, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
                            static_cast<S*>(dbeta), parts, cols);
@@ -419,15 +663,30 @@ extern "C" size_t tf_norm_bwd_workspace_bytes(int64_t rows, int64_t cols) {
     if (rows <= 0 || cols <= 0 || cols > 0x7FFFFFFF) return 0;
     // the most partial column sums any of the paths may write for this shape, whatever the element type or the op
     int64_t parts = std::min<int64_t>(rows, sm_count());                          // the streamed kernel: one CTA per SM
+    auto widest = [&](auto plan) {                                                 // any form may be chosen (or forced)
+        for (int form = 0; form < 3; ++form) {
+            const BwdPlan p = plan(form != 0, form == 2 ? 512 : 256);
+            parts = std::max<int64_t>(parts, static_cast<int64_t>(p.grid) * p.groups);
+        }
+    };
     if (cols % 4 == 0 && cols / 4 <= 512 * 4) {
-        const BwdPlan p = bwd_plan<false, DT_F32>(rows, static_cast<int>(cols / 4)), q = bwd_plan<true, DT_F32>(rows, static_cast<int>(cols / 4));
-        parts = std::max<int64_t>(parts, std::max(p.grid * p.groups, q.grid * q.groups));
+        const int nvec = static_cast<int>(cols / 4);
+        widest([&](bool sg, int gmax) { return bwd_plan<false, DT_F32>(rows, nvec, sg, g_force_stages, gmax); });
+        widest([&](bool sg, int gmax) { return bwd_plan<true, DT_F32>(rows, nvec, sg, g_force_stages, gmax); });
     }
     if (cols % 8 == 0 && cols / 8 <= 512 * 2) {
-        const BwdPlan p = bwd_plan<false, DT_BF16>(rows, static_cast<int>(cols / 8)), q = bwd_plan<true, DT_BF16>(rows, static_cast<int>(cols / 8));
-        parts = std::max<int64_t>(parts, std::max(p.grid * p.groups, q.grid * q.groups));
+        const int nvec = static_cast<int>(cols / 8);
+        widest([&](bool sg, int gmax) { return bwd_plan<false, DT_BF16>(rows, nvec, sg, g_force_stages, gmax); });
+        widest([&](bool sg, int gmax) { return bwd_plan<true, DT_BF16>(rows, nvec, sg, g_force_stages, gmax); });
     }
     return static_cast<size_t>(parts) * 2 * static_cast<size_t>(cols) * 4;
+}
+
+extern "C" tf_status tf_norm_bwd_force(int path, int stages) {
+    if (path < 0 || path > 3 || stages < 0 || stages > kBwdMaxStages) return TF_ERR_INVALID_ARG;
+    g_force_path = path;
+    g_force_stages = stages;
+    return TF_OK;
 }
 
 extern "C" tf_status tf_layernorm_bwd(const void* x, const void* gamma, const void* dy, const float* mean, const float* rstd, void* dx,

@@ -78,6 +78,25 @@ def test_edge_shapes(rms, dt):
         run_case(rms, dt, 9, cols, offset=offset)
 
 
+@pytest.mark.parametrize("rms", [False, True])
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_every_form_on_shapes_both_serve(rms, dt):
+    """The register form and the staged form (both group widths, several ring depths) give the oracle's result."""
+    ne = 4 if dt == F32 else 8
+    try:
+        for path, stages in ((1, 0), (2, 0), (2, 2), (2, 3), (3, 0), (3, 8)):
+            tf.tf_norm_bwd_force(path, stages)
+            for rows, cols in ((1, ne), (5, 3 * ne), (77, 256), (1500, 512), (700, 1024), (333, 4096), (130, 5120), (64, 8192)):
+                run_case(rms, dt, rows, cols, seed=rows + cols + path)
+            run_case(rms, dt, 300, 2048, inplace=True)
+    finally:
+        tf.tf_norm_bwd_force(0, 0)
+    with pytest.raises(tf.TfError):
+        tf.tf_norm_bwd_force(4, 0)
+    with pytest.raises(tf.TfError):
+        tf.tf_norm_bwd_force(2, 9)
+
+
 def test_matches_torch_autograd_in_fp32():
     torch.manual_seed(0)
     x = torch.randn(257, 1024, device="cuda", requires_grad=True)
