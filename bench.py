@@ -704,7 +704,8 @@ def run_normbwd_table(args):
     shapes = [("rmsnorm", inputs.BF16, 16384, 4096), ("rmsnorm", inputs.BF16, 16384, 8192), ("rmsnorm", inputs.F32, 16384, 4096),
               ("layernorm", inputs.BF16, 16384, 4096), ("layernorm", inputs.BF16, 16384, 8192), ("layernorm", inputs.BF16, 65536, 1024),
               ("layernorm", inputs.F32, 8192, 8192),
-              ("layernorm", inputs.BF16, 4096, 16384)]
+              ("layernorm", inputs.BF16, 4096, 16384), ("rmsnorm", inputs.BF16, 4096, 16384), ("layernorm", inputs.F32, 4096, 16384),
+              ("layernorm", inputs.BF16, 2048, 32768)]
     rows_out = []
     for op, dt, rows, cols in shapes:
         es = inputs.ELEM_SIZE[dt]

@@ -156,8 +156,9 @@ tf_status tf_softmax_bwd(const void* y, const void* dy, void* dx, int64_t rows, 
  * in a fixed order (deterministic).  x, dy, dx: [rows, cols]; gamma / weight, dgamma / dweight, dbeta: [cols]; dx may
  * alias x or dy.  workspace: device memory of at least tf_norm_bwd_workspace_bytes(rows, cols) bytes, 4-byte aligned,
  * used for partial column sums while the call runs (calls that may overlap on the GPU need separate workspaces); it
- * is required when the tensors are 16-byte aligned with rows of whole 16-byte vectors and up to 25,600 (LayerNorm) /
- * 51,200 (RMSNorm) columns, and ignored otherwise (such shapes run two plain kernels).  rows = 0 zeroes the parameter gradients.
+ * is required when the tensors are 16-byte aligned with rows of whole 16-byte vectors and up to 65,536 columns, and
+ * ignored otherwise (such shapes run two plain kernels).  Rows one CTA cannot hold (more than 8,192 columns) are shared
+ * by the CTAs of a thread-block cluster.  rows = 0 zeroes the parameter gradients.
  * Errors: TF_ERR_INVALID_ARG for a null pointer, cols <= 0, an unknown element type or a missing / short workspace.
  * Asynchronous on cuda_stream; allocates nothing.  The paper has no counterpart. */
 size_t tf_norm_bwd_workspace_bytes(int64_t rows, int64_t cols);
@@ -232,10 +233,13 @@ tf_status tf_query_choice(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int
 int tf_candidate_count(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);
 tf_status tf_candidate(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int index, char* buf, size_t n);
 
-/* Which form of the norm backward passes runs on shapes that both serve: path 0 = automatic, 1 = rows requested into
- * registers one row ahead, 2 = rows staged in a shared-memory ring by bulk copies (up to 512 threads per row), 3 = the
- * same with up to 256 threads per row; stages = ring depth (0 = automatic, at most 8).  Ask tf_norm_bwd_workspace_bytes again after changing it.  TF_ERR_INVALID_ARG outside those ranges. */
-tf_status tf_norm_bwd_force(int path, int stages);
+/* Which form of the norm backward passes runs on shapes that several serve.  path: 0 = automatic, 1 = rows requested
+ * into registers one row ahead, 2 = rows staged in a shared-memory ring by bulk copies (up to 512 threads per row),
+ * 3 = the same with up to 256 threads per row.  stages = ring depth (0 = automatic, at most 8).  cluster: 0 = automatic
+ * (a thread-block cluster shares a row only when one CTA cannot hold it), 1 = never, 2 / 4 / 8 = that many CTAs per row
+ * wherever the slices fit.  Ask tf_norm_bwd_workspace_bytes again after changing it.  TF_ERR_INVALID_ARG outside those
+ * values. */
+tf_status tf_norm_bwd_force(int path, int stages, int cluster);
 
 /* Forgets every tuned plan (in memory only). */
 void tf_clear_cache(void);

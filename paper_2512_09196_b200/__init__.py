@@ -63,7 +63,7 @@ def lib() -> ctypes.CDLL:
         L.tf_norm_bwd_workspace_bytes.argtypes = [i64, i64]
         L.tf_norm_bwd_workspace_bytes.restype = ctypes.c_size_t
         L.tf_layernorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i64, i64, i32, vp]
-        L.tf_norm_bwd_force.argtypes = [i32, i32]
+        L.tf_norm_bwd_force.argtypes = [i32, i32, i32]
         L.tf_rmsnorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i64, i64, i32, vp]
         L.tf_bvecmat_fwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp]
         L.tf_sin_fwd.argtypes = [vp, vp, i64, i32, i32, i32, vp]
@@ -228,9 +228,9 @@ def tf_rmsnorm_bwd(x, weight, dy, rstd, dx=None):
     return dx, dweight
 
 
-def tf_norm_bwd_force(path=0, stages=0):
-    """Test and bench hook: 0 = automatic, 1 = the register form, 2 = the staged form of the norm backward passes."""
-    _ok(lib().tf_norm_bwd_force(int(path), int(stages)), "tf_norm_bwd_force")
+def tf_norm_bwd_force(path=0, stages=0, cluster=0):
+    """Test and bench hook: which form of the norm backward passes runs (0 = automatic everywhere); see ``tf.h``."""
+    _ok(lib().tf_norm_bwd_force(int(path), int(stages), int(cluster)), "tf_norm_bwd_force")
 
 
 def tf_softmax_fwd_noalloc(x, y):

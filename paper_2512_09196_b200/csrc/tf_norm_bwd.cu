@@ -12,13 +12,19 @@
 // one; the other lets bulk copies bring the rows into a shared-memory ring, which keeps more bytes in flight than
 // registers can and is what 2-byte rows of 8 KiB and more take.  Both have a specialisation without predicates for
 // shapes in which no vector and no row slot is ever absent.
-// Rows beyond what 512 threads hold (16 KiB bf16, 32 KiB fp32) are streamed twice by one CTA per SM that keeps its
-// partial column sums in shared memory (up to 200 KiB of them); unaligned tensors, odd widths and wider rows still take
-// two plain kernels: scalar passes per row for dx, a thread per column for the parameter gradients.
+// Rows beyond what 512 threads hold (16 KiB bf16, 32 KiB fp32) are shared by the 2-8 CTAs of a thread-block cluster, each
+// the staged form on its slice of the columns, which exchange only the two row sums (up to 65,536 columns).  Where the
+// clusters cannot be placed, rows are streamed twice by one CTA per SM that keeps its partial column sums in shared
+// memory (up to 200 KiB of them); unaligned tensors, odd widths and wider rows take two plain kernels: scalar passes per
+// row for dx, a thread per column for the parameter gradients.
+#include <cooperative_groups.h>
+
 #include <algorithm>
 
 #include "../../include/tf.h"
 #include "tf_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace tf {
 namespace {
@@ -297,9 +303,146 @@ __global__ void __launch_bounds__(512) k_norm_bwd_staged(const BArgs a, const in
     }
 }
 
-// Rows too long for registers: one CTA per SM keeps its partial column sums in shared memory (every thread owns the
-// same columns of every row, so it updates its own entries without synchronisation) and streams each of its rows
-// twice with 16-byte loads: once for the two row sums, once more (from L2) for dx and the column sums.
+// Rows too long for one CTA's registers: a thread-block cluster of `cs` CTAs shares each row.  Every CTA is the staged
+// kernel above on its own slice of the columns (its slice of gamma and of the parameter-gradient accumulators in
+// registers, its slice of the row in its own ring); the only thing the CTAs of a row owe each other is the pair of row
+// sums, which each pushes into every peer's shared memory with an asynchronous store counted on the receiver's mbarrier.
+// There is no cluster barrier inside the loop; a peer can be at most one row ahead (it needs this CTA's sums to finish
+// a row), so two slot buffers suffice, and every CTA has received all pushes of its last row before it leaves.
+__device__ __forceinline__ void push_sums(float* slot, uint64_t* bar, uint32_t rank, float a, float b) {
+    uint32_t rslot, rbar;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rslot) : "r"(smem_u32(slot)), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(smem_u32(bar)), "r"(rank));
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
+                 ::"r"(rslot), "f"(a), "f"(b), "r"(rbar) : "memory");
+}
+
+template <bool RMS, int DT, int VPT, bool FULL>
+__global__ void __launch_bounds__(512) k_norm_bwd_cluster(const BArgs a, const int cs, const int S, int* status) {
+    using P = Pairs<DT>;
+    constexpr int NE = Elem<DT>::NE, NP = P::NP;
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    __shared__ __align__(8) uint64_t full[kBwdMaxStages];
+    __shared__ __align__(8) uint64_t xbar[2];                     // the sums of a row have all arrived (by row parity)
+    __shared__ __align__(8) float xch[2][kMaxCluster][2];
+    __shared__ float2 red[2][16];
+    const int t = threadIdx.x, gt = blockDim.x, wg = gt / 32, warp = t >> 5, lane = t & 31;
+    const int rank = static_cast<int>(blockIdx.x % cs);
+    const int64_t cluster_id = blockIdx.x / cs, num_clusters = gridDim.x / cs;
+    const int per = (a.nvec + cs - 1) / cs;                        // vectors per slice
+    const int first = rank * per;
+    const int len = max(0, min(per, a.nvec - first));
+    uint4* const ring = reinterpret_cast<uint4*>(dyn_smem);        // [S][x | dy][per]
+    cg::cluster_group cl = cg::this_cluster();
+    if (t == 0) {
+        for (int s = 0; s < S; ++s) mbar_init(&full[s], 1);
+        mbar_init(&xbar[0], 1);
+        mbar_init(&xbar[1], 1);
+        mbar_fence_init();
+    }
+    pdl_wait();
+    auto issue = [&](int64_t row, int s) {                         // thread 0 only
+        if (len == 0) return;
+        const uint32_t bytes = static_cast<uint32_t>(len) * 16u;
+        mbar_expect_tx(&full[s], 2u * bytes);
+        bulk_g2s(ring + static_cast<size_t>(per) * (2 * s), a.x + row * a.nvec + first, bytes, &full[s]);
+        bulk_g2s(ring + static_cast<size_t>(per) * (2 * s + 1), a.dy + row * a.nvec + first, bytes, &full[s]);
+    };
+    if (t == 0)
+        for (int s = 0; s < S; ++s) {
+            const int64_t row = cluster_id + static_cast<int64_t>(s) * num_clusters;
+            if (row < a.rows) issue(row, s);
+        }
+    bool valid[VPT];
+    F2 gam[VPT][NP], accg[VPT][NP], accb[RMS ? 1 : VPT][NP];
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+        valid[v] = FULL || t + v * gt < len;
+        P::unpack(valid[v] ? ld_param(a.gamma + first + t + v * gt) : make_uint4(0, 0, 0, 0), gam[v]);
+#pragma unroll
+        for (int i = 0; i < NP; ++i) { accg[v][i] = f2(0.f); if (!RMS) accb[v][i] = f2(0.f); }
+    }
+    __syncthreads();
+    cl.sync();                     // every CTA of the cluster is resident, its barriers initialised, before any remote store
+    bool failed = false;
+    int it = 0, s = 0;
+    uint32_t parity = 0;
+    float nmu = 0.f, nrs = 0.f;
+    auto request_stats = [&](int64_t row) {
+        if (row < a.rows) { nmu = RMS ? 0.f : __ldg(a.mean + row); nrs = __ldg(a.rstd + row); }
+    };
+    request_stats(cluster_id);
+    for (int64_t row = cluster_id; row < a.rows; row += num_clusters, ++it) {          // same trip count for the whole cluster
+        if (len > 0 && !failed && !mbar_wait(&full[s], parity)) {
+            failed = true;
+            atomicExch(status, 4);
+            mbar_wait(&full[s], parity);                                       // one more bounded wait for the copies
+        }
+        const float rs = nrs;
+        const F2 mu2 = f2(nmu), rs2 = f2(rs);
+        request_stats(row + num_clusters);
+        const uint4* sx = ring + static_cast<size_t>(per) * (2 * s) + t;
+        const uint4* sd = sx + per;
+        F2 xh[VPT][NP], g[VPT][NP], dv[VPT][NP];
+        F2 sgx2 = f2(0.f), sg2 = f2(0.f);
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            F2 xv[NP];
+            P::unpack(valid[v] ? sx[v * gt] : make_uint4(0, 0, 0, 0), xv);
+            P::unpack(valid[v] ? sd[v * gt] : make_uint4(0, 0, 0, 0), dv[v]);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                xh[v][i] = valid[v] ? mul2(sub2(xv[i], mu2), rs2) : f2(0.f);
+                g[v][i] = mul2(dv[v][i], gam[v][i]);
+                sgx2 = fma2(g[v][i], xh[v][i], sgx2);
+                sg2 = add2(sg2, g[v][i]);
+                accg[v][i] = fma2(dv[v][i], xh[v][i], accg[v][i]);
+                if (!RMS) accb[v][i] = add2(accb[v][i], dv[v][i]);
+            }
+        }
+        float sgx = group_reduce<SumOp, 32>(hsum(sgx2));
+        float sg = group_reduce<SumOp, 32>(hsum(sg2));
+        const int xb = it & 1;
+        if (lane == 0) red[xb][warp] = make_float2(sgx, sg);
+        __syncthreads();                                                       // also: every thread has left the stage
+        const int64_t next = row + static_cast<int64_t>(S) * num_clusters;
+        if (t == 0 && !failed && next < a.rows) issue(next, s);
+        if (wg > 1) group_total(red[xb], wg, lane, sgx, sg);                   // this CTA's sums, the same bits in every thread
+        if (t == 0) mbar_expect_tx(&xbar[xb], static_cast<uint32_t>(cs) * 8u);
+        if (t < cs) push_sums(&xch[xb][rank][0], &xbar[xb], static_cast<uint32_t>(t), sgx, sg);
+        if (!failed && !mbar_wait(&xbar[xb], static_cast<uint32_t>(it >> 1) & 1u)) { failed = true; atomicExch(status, 4); }
+        sgx = 0.f; sg = 0.f;
+        for (int k = 0; k < cs; ++k) { sgx += xch[xb][k][0]; sg += xch[xb][k][1]; }     // rank order: the same bits in every CTA
+        const F2 c1 = f2(-rs * (sgx * a.inv_n)), c0 = f2(RMS ? 0.f : -rs * (sg * a.inv_n));
+        uint4* o = a.dx + row * a.nvec + first + t;
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            F2 d[NP];
+#pragma unroll
+            for (int i = 0; i < NP; ++i) d[i] = fma2(xh[v][i], c1, fma2(g[v][i], rs2, c0));
+            if (valid[v]) st_stream(o + v * gt, P::pack(d));
+        }
+        if (++s == S) { s = 0; parity ^= 1u; }
+    }
+    cl.sync();                     // nobody leaves while a peer (one that gave up waiting, say) may still push into its shared memory
+    // this cluster's partial column sums: CTA `rank` owns columns [first, first + len) of part `cluster_id`
+    float* pg = a.part + cluster_id * (RMS ? 1 : 2) * a.nvec * NE;
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+        if (!valid[v]) continue;
+        const int64_t c0 = static_cast<int64_t>(first + t + v * gt) * NE;
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+            split(accg[v][i], pg[c0 + 2 * i], pg[c0 + 2 * i + 1]);
+            if (!RMS) split(accb[v][i], pg[static_cast<int64_t>(a.nvec) * NE + c0 + 2 * i], pg[static_cast<int64_t>(a.nvec) * NE + c0 + 2 * i + 1]);
+        }
+    }
+}
+
+// Rows too long for that as well (or a device without room for the clusters): one CTA per SM keeps its partial column
+// sums in shared memory (every thread owns the same columns of every row, so it updates its own entries without
+// synchronisation) and streams each of its rows twice with 16-byte loads: once for the two row sums, once more (from
+// L2) for dx and the column sums.
 template <bool RMS, int DT>
 __global__ void __launch_bounds__(1024) k_norm_bwd_stream(const BArgs a) {
     using E = Elem<DT>;
@@ -475,7 +618,7 @@ cudaError_t launch_pdl(void (*fn)(T...), int64_t grid, int threads, cudaStream_t
 
 // Test and bench hook: 0 = automatic, 1 = the register form, 2 = the staged form with row groups of up to 512 threads,
 // 3 = the staged form with row groups of up to 256 threads; stages 0 = automatic.
-int g_force_path = 0, g_force_stages = 0;
+int g_force_path = 0, g_force_stages = 0, g_force_cluster = 0;      // cluster: 0 = automatic, 1 = never, 2/4/8 = that many CTAs per row
 
 // Launch geometry of the row-group kernels: vectors per thread, threads per row group, row groups per CTA, CTAs; for
 // the staged form also the ring's stages and bytes (stages = 0: the register form).
@@ -548,6 +691,80 @@ BwdPlan choose_bwd_plan(int64_t rows, int nvec) {
     return kept;
 }
 
+// Cluster split-row form: CTAs per row, threads, vectors per thread, ring stages, clusters resident at once.
+struct ClusterPlan { int cs, threads, vpt, stages, clusters; size_t smem; bool full; };
+
+template <bool RMS, int DT, int VPT> const void* cluster_fn(bool full) {
+    return full ? reinterpret_cast<const void*>(k_norm_bwd_cluster<RMS, DT, VPT, true>) : reinterpret_cast<const void*>(k_norm_bwd_cluster<RMS, DT, VPT, false>);
+}
+
+void cluster_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, const ClusterPlan& p, int clusters, cudaStream_t st) {
+    cfg = cudaLaunchConfig_t{};
+    cfg.gridDim = dim3(static_cast<unsigned>(clusters) * p.cs);
+    cfg.blockDim = dim3(p.threads);
+    cfg.dynamicSmemBytes = p.smem;
+    cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeClusterDimension;          // no programmatic early launch: persistent clusters must all be placed at once
+    attr[0].val.clusterDim.x = p.cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+}
+
+template <bool RMS, int DT>
+ClusterPlan cluster_plan(int64_t rows, int nvec, int cs_forced, int stages) {
+    constexpr int kMaxVpt = Elem<DT>::NE == 4 ? 4 : 2;
+    ClusterPlan p{};
+    int cs = cs_forced > 1 ? cs_forced : 2;
+    // the fewest CTAs whose slices are at most 16 KiB (measured: the exchange costs about as much per row whatever the
+    // slice, so large slices amortise it; beyond 16 KiB a CTA has too many registers for two of them to share an SM)
+    while (cs_forced <= 1 && cs < kMaxCluster && (nvec + cs - 1) / cs > 1024) cs *= 2;
+    const int per = (nvec + cs - 1) / cs;
+    if (per > 512 * kMaxVpt) return p;                                                                // clusters = 0: not available
+    p.cs = cs;
+    p.vpt = 1;
+    while (p.vpt < kMaxVpt && (per + p.vpt - 1) / p.vpt > 512) p.vpt *= 2;
+    p.threads = std::max(32, ((per + p.vpt - 1) / p.vpt + 31) / 32 * 32);
+    p.full = nvec % cs == 0 && per == p.threads * p.vpt;
+    const size_t stage = static_cast<size_t>(2) * per * 16;
+    p.stages = stages > 0 ? stages : static_cast<int>(std::min<size_t>(3, (216 * 1024) / stage));
+    p.smem = stage * p.stages;
+    if (p.stages < 2 || p.stages > kBwdMaxStages || p.smem > 216 * 1024) return p;
+    const void* fn = p.vpt == 1 ? cluster_fn<RMS, DT, 1>(p.full) : p.vpt == 2 ? cluster_fn<RMS, DT, 2>(p.full) : cluster_fn<RMS, DT, kMaxVpt>(p.full);
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024) != cudaSuccess) { cudaGetLastError(); return p; }
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    cluster_config(cfg, attr, p, sm_count(), nullptr);
+    int fit = 0;                                                   // clusters cannot straddle GPCs: ask how many are resident at once
+    if (cudaOccupancyMaxActiveClusters(&fit, fn, &cfg) != cudaSuccess) { cudaGetLastError(); return p; }
+    p.clusters = static_cast<int>(std::min<int64_t>(rows, std::min(fit, sm_count())));      // the workspace is sized for one part per SM
+    return p;
+}
+
+template <bool RMS, int DT>
+ClusterPlan choose_cluster_plan(int64_t rows, int nvec) {          // the last shape's plan is kept, like the row-group plan
+    struct Key { int64_t rows; int nvec, cs, stages, dev; };
+    thread_local Key last{-1, 0, 0, 0, -1};
+    thread_local ClusterPlan kept{};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (last.rows == rows && last.nvec == nvec && last.cs == g_force_cluster && last.stages == g_force_stages && last.dev == dev) return kept;
+    last = Key{rows, nvec, g_force_cluster, g_force_stages, dev};
+    kept = cluster_plan<RMS, DT>(rows, nvec, g_force_cluster, g_force_stages);
+    return kept;
+}
+
+template <bool RMS, int DT>
+cudaError_t launch_cluster(const ClusterPlan& p, const BArgs& a, int* status, cudaStream_t st) {
+    constexpr int kMaxVpt = Elem<DT>::NE == 4 ? 4 : 2;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    cluster_config(cfg, attr, p, p.clusters, st);
+#define TF_CL(V, F) cudaLaunchKernelEx(&cfg, k_norm_bwd_cluster<RMS, DT, V, F>, a, p.cs, p.stages, status)
+    if (p.full) return p.vpt == 1 ? TF_CL(1, true) : p.vpt == 2 ? TF_CL(2, true) : TF_CL(kMaxVpt, true);
+    return p.vpt == 1 ? TF_CL(1, false) : p.vpt == 2 ? TF_CL(2, false) : TF_CL(kMaxVpt, false);
+#undef TF_CL
+}
+
 template <bool RMS, int DT>
 tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float* mean, const float* rstd, void* dx, void* dgamma,
                   void* dbeta, void* ws, size_t ws_bytes, int64_t rows, int64_t cols, cudaStream_t st) {
@@ -557,7 +774,25 @@ tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float*
     const bool aligned = al16(x) && al16(gamma) && al16(dy) && al16(dx) && bytes % 16 == 0;
     constexpr int kMaxVpt = NE == 4 ? 4 : 2;
     cudaError_t e;
-    if (aligned && bytes / 16 <= 512 * kMaxVpt && cols <= 0x7FFFFFFF) {
+    // a cluster per row: rows beyond one CTA's registers (or wherever the hook asks for it)
+    ClusterPlan cp{};
+    if (aligned && cols <= 0x7FFFFFFF && g_force_cluster != 1 && (g_force_cluster > 1 || bytes / 16 > 512 * kMaxVpt) &&
+        bytes / 16 <= static_cast<int64_t>(kMaxCluster) * 512 * kMaxVpt)
+        cp = choose_cluster_plan<RMS, DT>(rows, static_cast<int>(bytes / 16));
+    if (cp.clusters > 0) {
+        const int nvec = static_cast<int>(bytes / 16);
+        const size_t need = static_cast<size_t>(cp.clusters) * (RMS ? 1 : 2) * cols * 4;
+        if (!ws || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 3u)) return TF_ERR_INVALID_ARG;
+        int* status = device_status_word();
+        if (!status) return TF_ERR_CUDA;
+        BArgs a{static_cast<const uint4*>(x), static_cast<const uint4*>(gamma), static_cast<const uint4*>(dy), mean, rstd,
+                static_cast<uint4*>(dx), static_cast<float*>(ws), rows, nvec, 1.0f / static_cast<float>(cols)};
+        count_launches(2);
+        e = launch_cluster<RMS, DT>(cp, a, status, st);
+        if (e == cudaSuccess)
+            e = launch_pdl(k_colsum_finish<RMS, DT>, (cols + 31) / 32, 256, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
+                           static_cast<S*>(dbeta), cp.clusters, cols);
+    } else if (aligned && bytes / 16 <= 512 * kMaxVpt && cols <= 0x7FFFFFFF) {
         const int nvec = static_cast<int>(bytes / 16);
         const BwdPlan p = choose_bwd_plan<RMS, DT>(rows, nvec);
         const int parts = p.grid * p.groups;
@@ -682,10 +917,12 @@ extern "C" size_t tf_norm_bwd_workspace_bytes(int64_t rows, int64_t cols) {
     return static_cast<size_t>(parts) * 2 * static_cast<size_t>(cols) * 4;
 }
 
-extern "C" tf_status tf_norm_bwd_force(int path, int stages) {
+extern "C" tf_status tf_norm_bwd_force(int path, int stages, int cluster) {
     if (path < 0 || path > 3 || stages < 0 || stages > kBwdMaxStages) return TF_ERR_INVALID_ARG;
+    if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8) return TF_ERR_INVALID_ARG;
     g_force_path = path;
     g_force_stages = stages;
+    g_force_cluster = cluster;
     return TF_OK;
 }
 

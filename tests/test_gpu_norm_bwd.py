@@ -90,11 +90,36 @@ def test_every_form_on_shapes_both_serve(rms, dt):
                 run_case(rms, dt, rows, cols, seed=rows + cols + path)
             run_case(rms, dt, 300, 2048, inplace=True)
     finally:
-        tf.tf_norm_bwd_force(0, 0)
+        tf.tf_norm_bwd_force(0, 0, 0)
     with pytest.raises(tf.TfError):
         tf.tf_norm_bwd_force(4, 0)
     with pytest.raises(tf.TfError):
         tf.tf_norm_bwd_force(2, 9)
+    with pytest.raises(tf.TfError):
+        tf.tf_norm_bwd_force(0, 0, 3)
+
+
+@pytest.mark.parametrize("rms", [False, True])
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_cluster_per_row(rms, dt):
+    """A thread-block cluster shares each row: forced on short rows (ragged slices, an empty slice, one row, fewer rows
+    than clusters, many rows per cluster) and chosen by itself beyond what one CTA holds."""
+    ne = 4 if dt == F32 else 8
+    try:
+        for cluster, stages in ((2, 0), (4, 2), (8, 0)):
+            tf.tf_norm_bwd_force(0, stages, cluster)
+            for rows, cols in ((1, ne), (3, 5 * ne), (40, 256), (2000, 512), (300, 1024 + ne), (100, 4096), (37, 8192)):
+                run_case(rms, dt, rows, cols, seed=rows + cols + cluster)
+            run_case(rms, dt, 64, 2048, inplace=True)
+    finally:
+        tf.tf_norm_bwd_force(0, 0, 0)
+    for rows, cols in ((200, 16384), (31, 16384 + ne), (20, 32768), (9, 65536)):
+        run_case(rms, dt, rows, cols, seed=cols)
+    try:                                                           # the same long rows without clusters: the streamed form
+        tf.tf_norm_bwd_force(0, 0, 1)
+        run_case(rms, dt, 50, 16384, seed=5)
+    finally:
+        tf.tf_norm_bwd_force(0, 0, 0)
 
 
 def test_matches_torch_autograd_in_fp32():
