@@ -130,3 +130,10 @@ def test_bad_arguments():
     assert L.tf_add_layernorm_fwd(p, p, p, None, p, p, None, None, 1, 8, 1e-5, 0, None) == 1  # beta missing
     assert L.tf_add_layernorm_fwd(p, p, p, p, p, p, None, None, 1, 8, -1.0, 0, None) == 1
     assert L.tf_add_layernorm_fwd(p, p, p, p, p, p, None, None, 0, 8, 1e-5, 0, None) == 0
+
+
+@pytest.mark.parametrize("op,dt,rows,cols", [("rmsnorm", BF16, 16384, 4096), ("layernorm", BF16, 16384, 4096), ("rmsnorm", BF16, 4096, 16384),
+                                              ("layernorm", F32, 16384, 4096), ("rmsnorm", BF16, 256, 8192)])
+def test_shapes_of_the_bench_table_every_element(op, dt, rows, cols):
+    """The shapes `bench.py --table addnorm` times, in the plan it times (automatic), every element against the oracle."""
+    run_case(op, dt, rows, cols, seed=cols)

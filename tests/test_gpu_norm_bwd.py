@@ -153,3 +153,12 @@ def test_deterministic_and_bad_arguments():
     assert L.tf_layernorm_bwd(p, p, p, None, p, p, p, p, p, 1 << 20, 4, 64, 0, None) == 1   # mean missing
     assert L.tf_layernorm_bwd(p, p, p, p, p, p, p, None, p, 1 << 20, 4, 64, 0, None) == 1   # dbeta missing
     assert L.tf_rmsnorm_bwd(p, p, p, p, p, p, p, 1 << 20, 4, 0, 0, None) == 1
+
+
+@pytest.mark.parametrize("rms,dt,rows,cols", [(True, BF16, 16384, 4096), (True, BF16, 16384, 8192), (True, F32, 16384, 4096), (False, BF16, 16384, 4096),
+                                              (False, BF16, 65536, 1024), (False, F32, 8192, 8192), (False, BF16, 4096, 16384), (False, F32, 4096, 16384),
+                                              (False, BF16, 2048, 32768)])
+def test_shapes_of_the_bench_table_every_element(rms, dt, rows, cols):
+    """The shapes `bench.py --table normbwd` times, in the form it times (automatic): dx element by element, the parameter
+    gradients summed over all rows."""
+    run_case(rms, dt, rows, cols, seed=cols)

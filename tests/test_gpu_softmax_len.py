@@ -107,3 +107,9 @@ def test_bad_arguments():
     assert L.tf_softmax_len_fwd(p, p, p, 0, 8, 0, None) == 0
     with pytest.raises(ValueError):
         tf.tf_softmax_len_fwd(torch.zeros(4, 8, device="cuda"), torch.zeros(4, dtype=torch.int64, device="cuda"))
+
+
+@pytest.mark.parametrize("dt,rows,cols", [(BF16, 16384, 8192), (F32, 65536, 1024), (BF16, 262144, 256), (BF16, 1024, 131072)])
+def test_shapes_of_the_bench_table_every_element(dt, rows, cols):
+    """The shapes `bench.py --table softmaxlen` times (the 128 Ki-column one on a quarter of its rows), every element."""
+    run_case(dt, rows, cols, seed=cols)

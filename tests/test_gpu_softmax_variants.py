@@ -129,3 +129,12 @@ def test_bad_arguments():
     assert L.tf_softmax_bwd(p, None, p, 1, 8, 0, None) == 1
     assert L.tf_softmax_bwd(p, p, None, 1, 8, 0, None) == 1
     assert L.tf_softmax_bwd(p, p, p, 0, 8, 1, None) == 0
+
+
+@pytest.mark.parametrize("dt,rows,cols", [(BF16, 16384, 8192), (BF16, 32768, 4096), (F32, 65536, 1024), (BF16, 524288, 256), (BF16, 2048, 32768),
+                                          (F32, 1024, 131072)])
+def test_shapes_of_the_bench_table_every_element(dt, rows, cols):
+    """The shapes `bench.py --table softmaxvariants` times (the two widest on a quarter / half of their rows), both ops,
+    every element against the oracle."""
+    run_log_softmax(dt, rows, cols, seed=cols)
+    run_softmax_bwd(dt, rows, cols, seed=cols)
