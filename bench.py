@@ -692,6 +692,80 @@ def run_softmax_variants_table(args):
     (out_dir / "table_softmaxvariants.json").write_text(json.dumps(rows_out, indent=1))
 
 
+def run_launch_table(args):
+    """Launch-bound shapes: time per call made eagerly through the Python binding and as one CUDA graph of 32 captured calls."""
+    import torch
+    import paper_2512_09196_b200 as tf
+    from paper_2512_09196_b200 import inputs
+    torch.cuda.set_device(0)
+    out_dir = ROOT / "gpurun_out"
+    out_dir.mkdir(exist_ok=True)
+    sets, per_graph = 8, 32
+    bf = torch.bfloat16
+    rows_out = []
+
+    def softmax_case():
+        w = inputs.config(0)
+        xs = [torch.from_numpy(inputs.normal((w.rows, w.cols), w.dt, k, 0, 0.0, 1.0)).cuda() for k in range(sets)]
+        ys = [torch.empty_like(x) for x in xs]
+        return "softmax f32 [1024, 1024] (configuration 0)", 2 * w.rows * w.cols * 4, lambda k: tf.tf_softmax_fwd(xs[k], ys[k])
+
+    def add_case():
+        rows, cols = 256, 8192
+        xs = [torch.randn(rows, cols, device="cuda").to(bf) for _ in range(sets)]
+        rs = [torch.randn(rows, cols, device="cuda").to(bf) for _ in range(sets)]
+        hs, ys = [torch.empty_like(x) for x in xs], [torch.empty_like(x) for x in xs]
+        wt = (torch.rand(cols, device="cuda") + 0.5).to(bf)
+        return "add + rmsnorm bf16 [256, 8192] (a decode batch)", 4 * rows * cols * 2, lambda k: tf.tf_add_rmsnorm_fwd(xs[k], rs[k], wt, 1e-6, h=hs[k], y=ys[k])
+
+    def lsm_case(rows, cols, dt, label):
+        def make():
+            xs = [torch.randn(rows, cols, device="cuda").to(dt) for _ in range(sets)]
+            ys = [torch.empty_like(x) for x in xs]
+            return label, 2 * rows * cols * xs[0].element_size(), lambda k: tf.tf_log_softmax_fwd(xs[k], ys[k])
+        return make
+
+    for make in (softmax_case, add_case, lsm_case(64, 32768, bf, "log-softmax bf16 [64, 32768] (logits of a decode batch)"),
+                 lsm_case(8, 131072, torch.float32, "log-softmax f32 [8, 131072] (fp32 logits, 128 Ki vocabulary)"),
+                 lsm_case(1, 262144, bf, "log-softmax bf16 [1, 262144] (one sequence, 256 Ki vocabulary)")):
+        name, nbytes, call = make()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):                         # first use outside the capture
+            for k in range(sets):
+                call(k)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for k in range(per_graph):
+                call(k % sets)
+
+        def timed(fn, reps):
+            for _ in range(3):
+                fn()
+            a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for _ in range(reps):
+                fn()
+            e.record()
+            torch.cuda.synchronize()
+            return 1e3 * a.elapsed_time(e) / reps
+
+        def eager():
+            for k in range(per_graph):
+                call(k % sets)
+        us_eager = min(timed(eager, 20) for _ in range(3)) / per_graph
+        us_graph = min(timed(graph.replay, 20) for _ in range(3)) / per_graph
+        tf.tf_device_status()
+        row = {"case": name, "bytes": nbytes, "eager_us_per_call": us_eager, "graph_us_per_call": us_graph,
+               "graph_gbs": nbytes / us_graph / 1e3, "calls_per_graph": per_graph}
+        rows_out.append(row)
+        print(json.dumps(row), flush=True)
+    (out_dir / "table_launch.json").write_text(json.dumps(rows_out, indent=1))
+
+
 def run_normbwd_table(args):
     """LayerNorm / RMSNorm backward: achieved bandwidth of x, dy in and dx out; torch's native backward as context."""
     import torch
@@ -882,7 +956,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm", "softmaxlen", "softmaxvariants", "normbwd"], default=None)
+    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm", "softmaxlen", "softmaxvariants", "normbwd", "launch"], default=None)
     ap.add_argument("--filter", default=None)
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
@@ -909,6 +983,8 @@ def main():
         return run_softmax_variants_table(args)
     if args.table == "normbwd":
         return run_normbwd_table(args)
+    if args.table == "launch":
+        return run_launch_table(args)
     if args.table:
         return run_table(args)
     run_ours(args)

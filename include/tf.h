@@ -142,7 +142,8 @@ tf_status tf_log_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols,
  * gradient dy, all [rows, cols] of one element type; fp32 arithmetic, one rounding.  dx may alias y or dy.
  * Both calls: device pointers, asynchronous on cuda_stream, allocate nothing; TF_ERR_INVALID_ARG for a null pointer
  * with rows > 0, cols <= 0 or an unknown element type; rows = 0 is a no-op.  16-byte aligned tensors whose rows are
- * whole 16-byte vectors are held in registers up to 32 KiB per row and streamed in two passes beyond; anything else
+ * whole 16-byte vectors are held in registers up to 32 KiB per row and streamed in two passes beyond; when such long rows
+ * are too few to fill the device with one CTA each, the 2-8 CTAs of a thread-block cluster share a row.  Anything else
  * runs scalar passes. */
 tf_status tf_softmax_bwd(const void* y, const void* dy, void* dx, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
 
@@ -232,6 +233,10 @@ tf_status tf_query_choice(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int
 /* Number of candidate plans tf_tune would consider for this problem, and the index-th of them as text. */
 int tf_candidate_count(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);
 tf_status tf_candidate(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int index, char* buf, size_t n);
+
+/* Whether tf_log_softmax_fwd / tf_softmax_bwd share a row among the CTAs of a thread-block cluster: 0 = automatic (rows
+ * beyond 32 KiB), 1 = never, 2 / 4 / 8 = that many CTAs per row wherever the slices fit.  TF_ERR_INVALID_ARG otherwise. */
+tf_status tf_softmax_variants_force(int cluster);
 
 /* Which form of the norm backward passes runs on shapes that several serve.  path: 0 = automatic, 1 = rows requested
  * into registers one row ahead, 2 = rows staged in a shared-memory ring by bulk copies (up to 512 threads per row),

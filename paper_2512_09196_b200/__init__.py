@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_norm_bwd_workspace_bytes", "tf_layernorm_bwd", "tf_rmsnorm_bwd", "tf_norm_bwd_force",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_norm_bwd_workspace_bytes", "tf_layernorm_bwd", "tf_rmsnorm_bwd", "tf_norm_bwd_force", "tf_softmax_variants_force",
            "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
@@ -64,6 +64,7 @@ def lib() -> ctypes.CDLL:
         L.tf_norm_bwd_workspace_bytes.restype = ctypes.c_size_t
         L.tf_layernorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i64, i64, i32, vp]
         L.tf_norm_bwd_force.argtypes = [i32, i32, i32]
+        L.tf_softmax_variants_force.argtypes = [i32]
         L.tf_rmsnorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i64, i64, i32, vp]
         L.tf_bvecmat_fwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp]
         L.tf_sin_fwd.argtypes = [vp, vp, i64, i32, i32, i32, vp]
@@ -226,6 +227,11 @@ def tf_rmsnorm_bwd(x, weight, dy, rstd, dx=None):
         _ok(lib().tf_rmsnorm_bwd(x.data_ptr(), weight.data_ptr(), dy.data_ptr(), rstd.data_ptr(), dx.data_ptr(), dweight.data_ptr(),
                                  ws.data_ptr(), n, rows, cols, _dt(x), _stream(x)), "tf_rmsnorm_bwd")
     return dx, dweight
+
+
+def tf_softmax_variants_force(cluster=0):
+    """Test and bench hook: CTAs per row of ``tf_log_softmax_fwd`` / ``tf_softmax_bwd`` (0 = automatic, 1 = never a cluster)."""
+    _ok(lib().tf_softmax_variants_force(int(cluster)), "tf_softmax_variants_force")
 
 
 def tf_norm_bwd_force(path=0, stages=0, cluster=0):

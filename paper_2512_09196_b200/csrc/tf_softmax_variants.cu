@@ -4,15 +4,22 @@
 // One kernel shape serves both: a CTA owns a row and holds it in registers (VPT 16-byte vectors per thread, loaded at
 // once), reduces across the CTA, finishes and stores -- one read of every input element, one write of every output
 // element.  Rows of up to 2 KiB are owned by lane groups instead (several rows per warp).  Rows beyond 32 KiB are
-// streamed in two passes of 16-byte loads, the second from L2; unaligned tensors and odd widths take scalar passes.
+// streamed in two passes of 16-byte loads, the second from L2; when such rows are too few to give every SM a CTA (logits
+// of a decode batch), the CTAs of a thread-block cluster share each row, slices in registers where they fit and streamed
+// where not, with one exchange of partials through distributed shared memory.  Unaligned tensors and odd widths take
+// scalar passes.
 //
 // Log-softmax keeps x - m as a difference (exact for bf16 inputs, one rounding for fp32) and subtracts ln S computed
 // from S = sum 2^((x - m) log2 e) with the accurate logarithm; the term of the maximum is exactly 1, so S >= 1 and its
 // fp32 summation error is a few 2^-24 absolute, which is the absolute part of the tolerance the tests use.
+#include <cooperative_groups.h>
+
 #include <algorithm>
 
 #include "../../include/tf.h"
 #include "tf_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace tf {
 namespace {
@@ -93,6 +100,103 @@ __global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2(con
     }
 }
 
+// Rows beyond what one CTA should hold in registers: a thread-block cluster of `cs` CTAs owns a row, each CTA a slice of
+// it in registers (the same VPT vectors per thread, loaded at once).  One exchange: every CTA writes its partial --
+// (slice maximum, sum of 2^((x - slice maximum) log2 e)) for log-softmax, sum y dy for the backward pass -- into every
+// peer's shared memory, one cluster barrier, and every CTA combines the partials in rank order (the same bits in all of
+// them): M = max m_k, S = sum_k s_k 2^((m_k - M) log2 e).  Still one read of every input element and one write of every
+// output element, and small slices keep several CTAs on an SM, which is what the long rows lacked.
+template <int WHICH, int DT, int VPT>
+__global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2_cluster(const uint4* __restrict__ in0, const uint4* __restrict__ in1,
+                                                                                     uint4* __restrict__ out, int64_t rows, int nvec, int cs) {
+    using E = Elem<DT>;
+    constexpr int NE = E::NE;
+    __shared__ float buf[2][32];
+    __shared__ float xch[kMaxCluster][2];
+    pdl_wait();
+    pdl_trigger();
+    cg::cluster_group cl = cg::this_cluster();
+    const int T = blockDim.x, t = threadIdx.x;
+    const int rank = static_cast<int>(blockIdx.x % cs);
+    const int64_t row = blockIdx.x / cs;                          // the grid is rows x cs CTAs
+    const int per = (nvec + cs - 1) / cs;
+    const int first = rank * per;
+    const int len = max(0, min(per, nvec - first));
+    const uint4* a = in0 + row * nvec + first + t;
+    uint4* o = out + row * nvec + first + t;
+    bool valid[VPT];
+    uint4 ra[VPT], rb[VPT];
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+        valid[v] = t + v * T < len;
+        ra[v] = valid[v] ? ld_stream(a + v * T) : make_uint4(0, 0, 0, 0);
+        if (WHICH == kOpSoftmaxBwd) rb[v] = valid[v] ? ld_stream(in1 + row * nvec + first + t + v * T) : make_uint4(0, 0, 0, 0);
+    }
+    cl.sync();                     // every CTA of the cluster is resident before any remote write (the loads are already under way)
+    if constexpr (WHICH == kOpLogSoftmax) {
+        float m = kNegInf;
+#pragma unroll
+        for (int v = 0; v < VPT; ++v)
+            if (valid[v]) m = fmaxf(m, vec_max<DT>(ra[v]));
+        m = cta_reduce<MaxOp>(m, buf[0]);
+        float s = 0.f;
+        if (m != kNegInf) {
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) {
+                float x[NE];
+                E::unpack(ra[v], x);
+#pragma unroll
+                for (int i = 0; i < NE; ++i)
+                    if (valid[v]) s += ex2_ftz((x[i] - m) * kLog2e);
+            }
+        }
+        s = cta_reduce<SumOp>(s, buf[1]);
+        if (t < cs) {
+            float* dst = cl.map_shared_rank(&xch[rank][0], t);
+            dst[0] = m; dst[1] = s;
+        }
+        cl.sync();                                                 // release our writes, acquire the peers'
+        float M = kNegInf, S = 0.f;
+        for (int k = 0; k < cs; ++k) M = fmaxf(M, xch[k][0]);
+        for (int k = 0; k < cs; ++k)
+            if (xch[k][0] != kNegInf) S += xch[k][1] * ex2_ftz((xch[k][0] - M) * kLog2e);      // the slice of the maximum contributes exactly s_k
+        const float lns = logf(S);
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            float x[NE], y[NE];
+            E::unpack(ra[v], x);
+#pragma unroll
+            for (int i = 0; i < NE; ++i) y[i] = (M == kNegInf) ? kNegInf : (x[i] - M) - lns;
+            if (valid[v]) st_stream(o + v * T, E::pack(y));
+        }
+    } else {
+        float y[VPT][NE], g[VPT][NE];
+        float s = 0.f;
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            E::unpack(ra[v], y[v]);
+            E::unpack(rb[v], g[v]);
+#pragma unroll
+            for (int i = 0; i < NE; ++i) s = fmaf(y[v][i], g[v][i], s);    // absent vectors hold zeros
+        }
+        s = cta_reduce<SumOp>(s, buf[0]);
+        if (t < cs) {
+            float* dst = cl.map_shared_rank(&xch[rank][0], t);
+            dst[0] = s; dst[1] = 0.f;
+        }
+        cl.sync();
+        float total = 0.f;
+        for (int k = 0; k < cs; ++k) total += xch[k][0];
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) {
+            float dx[NE];
+#pragma unroll
+            for (int i = 0; i < NE; ++i) dx[i] = y[v][i] * (g[v][i] - total);
+            if (valid[v]) st_stream(o + v * T, E::pack(dx));
+        }
+    }
+}
+
 // Short rows (up to 2 KiB): a group of LANES lanes owns a row, a CTA of 128 threads covers 128 / LANES consecutive
 // rows, reductions are shuffles.  Every lane runs every step (the shuffles need the whole warp); rows past the end
 // are loaded as zeros and not stored.
@@ -165,19 +269,26 @@ __global__ void __launch_bounds__(128) k_row2_group(const uint4* __restrict__ in
 
 // Rows too long for registers (aligned): a CTA per row, passes of four independent 16-byte loads per thread; the first
 // pass comes from HBM, the later ones find the row in L2 (a row is at most a few MiB).
-template <int WHICH, int DT>
+// CL: the row is shared by the `cs` CTAs of a thread-block cluster (few rows of many columns: one CTA per row would leave
+// most of the device idle); each streams its own slice and the partials meet as in k_row2_cluster, between the passes.
+template <int WHICH, int DT, bool CL>
 __global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ in0, const uint4* __restrict__ in1, uint4* __restrict__ out,
-                                                     int64_t rows, int64_t nvec) {
+                                                     int64_t rows, int64_t row_vecs, int cs) {
     using E = Elem<DT>;
     constexpr int NE = E::NE, U = 4;
     __shared__ float buf[2][32];
+    __shared__ float xch[kMaxCluster][2];
     pdl_wait();
     pdl_trigger();
     const int T = blockDim.x, t = threadIdx.x;
-    const int64_t row = blockIdx.x;
-    if (row >= rows) return;
-    const uint4* a = in0 + row * nvec;
-    uint4* o = out + row * nvec;
+    const int rank = CL ? static_cast<int>(blockIdx.x % cs) : 0;
+    const int64_t row = CL ? blockIdx.x / cs : blockIdx.x;
+    if (!CL && row >= rows) return;
+    const int64_t per = CL ? (row_vecs + cs - 1) / cs : row_vecs, first = rank * per;
+    const int64_t nvec = per < row_vecs - first ? per : (row_vecs - first > 0 ? row_vecs - first : 0);      // this CTA's slice
+    const uint4* a = in0 + row * row_vecs + first;
+    uint4* o = out + row * row_vecs + first;
+    if constexpr (CL) cg::this_cluster().sync();                  // every CTA of the cluster is resident before any remote write
     const int64_t step = static_cast<int64_t>(T) * U;
     if constexpr (WHICH == kOpLogSoftmax) {
         // one pass for both statistics: every thread keeps (running max, sum relative to it) and rescales the sum when
@@ -208,9 +319,21 @@ __global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ i
                 }
             }
         }
-        const float m = cta_reduce<MaxOp>(mt, buf[0]);
+        float m = cta_reduce<MaxOp>(mt, buf[0]);
         float s = (mt == kNegInf) ? 0.f : st * ex2_ftz((mt - m) * kLog2e);          // 2^0 = 1 exactly for the thread that holds the maximum
         s = cta_reduce<SumOp>(s, buf[1]);
+        if constexpr (CL) {
+            cg::cluster_group cl = cg::this_cluster();
+            if (t < cs) {
+                float* dst = cl.map_shared_rank(&xch[rank][0], t);
+                dst[0] = m; dst[1] = s;
+            }
+            cl.sync();
+            m = kNegInf; s = 0.f;
+            for (int k = 0; k < cs; ++k) m = fmaxf(m, xch[k][0]);
+            for (int k = 0; k < cs; ++k)
+                if (xch[k][0] != kNegInf) s += xch[k][1] * ex2_ftz((xch[k][0] - m) * kLog2e);
+        }
         const float lns = logf(s);
         for (int64_t b0 = t; b0 < nvec; b0 += step) {
             uint4 r[U];
@@ -226,7 +349,7 @@ __global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ i
             }
         }
     } else {
-        const uint4* b = in1 + row * nvec;
+        const uint4* b = in1 + row * row_vecs + first;
         float s = 0.f;
         for (int64_t b0 = t; b0 < nvec; b0 += step) {
             uint4 ry[U], rg[U];
@@ -246,6 +369,16 @@ __global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ i
             }
         }
         s = cta_reduce<SumOp>(s, buf[0]);
+        if constexpr (CL) {
+            cg::cluster_group cl = cg::this_cluster();
+            if (t < cs) {
+                float* dst = cl.map_shared_rank(&xch[rank][0], t);
+                dst[0] = s; dst[1] = 0.f;
+            }
+            cl.sync();
+            s = 0.f;
+            for (int k = 0; k < cs; ++k) s += xch[k][0];
+        }
         for (int64_t b0 = t; b0 < nvec; b0 += step) {
             uint4 ry[U], rg[U];
 #pragma unroll
@@ -299,6 +432,13 @@ __global__ void __launch_bounds__(256) k_row2_scalar(const typename Elem<DT>::sc
 
 bool al16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+int sm_count() {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms;
+}
+
 template <int WHICH, int DT, int VPT>
 cudaError_t launch_vpt(int threads, cudaStream_t st, const void* in0, const void* in1, void* out, int64_t rows, int nvec) {
     cudaLaunchConfig_t cfg = {};
@@ -336,6 +476,42 @@ cudaError_t launch_group(cudaStream_t st, const void* in0, const void* in1, void
                       static_cast<const uint4*>(in1), static_cast<uint4*>(out), rows, nvec);
 }
 
+// Test and bench hook: 0 = automatic, 1 = never a cluster per row, 2 / 4 / 8 = that many CTAs per row wherever the slices fit.
+int g_force_cluster = 0;
+
+template <int WHICH, int DT, int VPT>
+cudaError_t launch_cluster_vpt(int threads, int cs, cudaStream_t st, const void* in0, const void* in1, void* out, int64_t rows, int nvec) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(rows * cs));
+    cfg.blockDim = dim3(threads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, k_row2_cluster<WHICH, DT, VPT>, static_cast<const uint4*>(in0), static_cast<const uint4*>(in1),
+                              static_cast<uint4*>(out), rows, nvec, cs);
+}
+
+// Geometry of a register-resident slice of `nv` vectors: the fewest vectors per thread that keep the CTA at 128 threads
+// or fewer; else the most the register budget allows.  vpt = 0: does not fit.
+template <int WHICH, int DT>
+void slice_geometry(int nv, int& vpt, int& threads) {
+    vpt = 0; threads = 0;
+    const int fl[4] = {row2_floats<WHICH, DT, 1>(), row2_floats<WHICH, DT, 2>(), row2_floats<WHICH, DT, 4>(), row2_floats<WHICH, DT, 8>()};
+    for (int k = 0; k < 4; ++k) {
+        const int v = 1 << k;
+        if (fl[k] > 64) break;
+        const int th = std::max(32, ((nv + v - 1) / v + 31) / 32 * 32);
+        if (th > (fl[k] <= 32 ? 1024 : 512)) continue;
+        vpt = v; threads = th;
+        if (th <= 128) break;
+    }
+}
+
 template <int WHICH, int DT>
 cudaError_t launch_dt(cudaStream_t st, const void* in0, const void* in1, void* out, int64_t rows, int64_t cols) {
     using S = typename Elem<DT>::scalar;
@@ -343,7 +519,7 @@ cudaError_t launch_dt(cudaStream_t st, const void* in0, const void* in1, void* o
     {
         const int64_t b = cols * Elem<DT>::SIZE;
         const bool al = al16(in0) && al16(out) && (WHICH == kOpLogSoftmax || al16(in1)) && b % 16 == 0;
-        if (al && b / 16 <= 128) {                                  // rows up to 2 KiB: lane groups
+        if (al && b / 16 <= 128 && g_force_cluster <= 1) {          // rows up to 2 KiB: lane groups
             const int nv = static_cast<int>(b / 16);
             if (nv <= 8) return launch_group<WHICH, DT, 8, 1>(st, in0, in1, out, rows, nv);
             if (nv <= 16) return launch_group<WHICH, DT, 8, 2>(st, in0, in1, out, rows, nv);
@@ -354,25 +530,58 @@ cudaError_t launch_dt(cudaStream_t st, const void* in0, const void* in1, void* o
     }
     const int64_t bytes = cols * Elem<DT>::SIZE;
     const bool aligned = al16(in0) && al16(out) && (WHICH == kOpLogSoftmax || al16(in1)) && bytes % 16 == 0;
-    // the fewest vectors per thread that keep the CTA at 128 threads or fewer; else the most the register budget allows
     int vpt = 0, threads = 0;
-    // beyond 32 KiB the streamed passes win: a CTA that holds such a row in registers is alone on its SM for too long
-    // (measured at 64 KiB: log-softmax 4.1 TB/s held, 5.4 streamed)
-    if (aligned && bytes / 16 <= 2048) {
-        const int nv = static_cast<int>(bytes / 16);
-        const int fl[4] = {row2_floats<WHICH, DT, 1>(), row2_floats<WHICH, DT, 2>(), row2_floats<WHICH, DT, 4>(), row2_floats<WHICH, DT, 8>()};
-        for (int k = 0; k < 4; ++k) {
-            const int v = 1 << k;
-            if (fl[k] > 64) break;
-            const int th = std::max(32, ((nv + v - 1) / v + 31) / 32 * 32);
-            if (th > (fl[k] <= 32 ? 1024 : 512)) continue;
-            vpt = v; threads = th;
-            if (th <= 128) break;
+    // a cluster per row: rows beyond 32 KiB when there are too few of them to fill the device with one CTA each -- as many
+    // CTAs per row (2, 4 or 8) as keep the launch within about two CTAs per SM.  With more rows the streamed passes are
+    // faster (bf16 [8192, 32768]: 5.4 TB/s streamed, 3.6 with clusters).  Or where the hook asks.
+    int cs = g_force_cluster > 1 ? g_force_cluster : 0;
+    if (g_force_cluster == 0 && bytes / 16 > 2048) {
+        const int64_t room = 2 * static_cast<int64_t>(sm_count()) / rows;
+        cs = room >= 8 ? 8 : room >= 4 ? 4 : room >= 2 ? 2 : 0;
+    }
+    if (aligned && cs >= 2 && rows * kMaxCluster <= 0x7FFFFFFF) {
+        const int64_t nv = bytes / 16;
+        int64_t per = (nv + cs - 1) / cs;
+        if (per > 2048) {                                           // slices too long for registers: every CTA streams its own
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(static_cast<unsigned>(rows * cs));
+            cfg.blockDim = dim3(512);
+            cfg.stream = st;
+            cudaLaunchAttribute attr[2];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[1].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 2;
+            const cudaError_t e = cudaLaunchKernelEx(&cfg, k_row2_stream<WHICH, DT, true>, static_cast<const uint4*>(in0), static_cast<const uint4*>(in1),
+                                                     static_cast<uint4*>(out), rows, nv, cs);
+            if (e == cudaSuccess) return e;
+            cudaGetLastError();
+        } else {
+            slice_geometry<WHICH, DT>(static_cast<int>(per), vpt, threads);
+            if (vpt) {
+                const int nvec = static_cast<int>(nv);
+                cudaError_t e = cudaErrorInvalidValue;
+                switch (vpt) {
+                    case 1: e = launch_cluster_vpt<WHICH, DT, 1>(threads, cs, st, in0, in1, out, rows, nvec); break;
+                    case 2: e = launch_cluster_vpt<WHICH, DT, 2>(threads, cs, st, in0, in1, out, rows, nvec); break;
+                    case 4: e = launch_cluster_vpt<WHICH, DT, 4>(threads, cs, st, in0, in1, out, rows, nvec); break;
+                    default:
+                        if constexpr (row2_floats<WHICH, DT, 8>() <= 64) e = launch_cluster_vpt<WHICH, DT, 8>(threads, cs, st, in0, in1, out, rows, nvec);
+                }
+                if (e == cudaSuccess) return e;
+                cudaGetLastError();                                 // the cluster could not be launched here: the forms below serve the shape
+                vpt = 0;
+            }
         }
     }
+    // beyond 32 KiB a single CTA that holds the row in registers is alone on its SM for too long (measured at 64 KiB:
+    // log-softmax 4.1 TB/s held, 5.4 streamed), so such rows are streamed when no cluster took them
+    if (aligned && bytes / 16 <= 2048) slice_geometry<WHICH, DT>(static_cast<int>(bytes / 16), vpt, threads);
     if (vpt == 0 && aligned)
-        return launch_pdl(k_row2_stream<WHICH, DT>, rows, 512, st, static_cast<const uint4*>(in0), static_cast<const uint4*>(in1),
-                          static_cast<uint4*>(out), rows, bytes / 16);
+        return launch_pdl(k_row2_stream<WHICH, DT, false>, rows, 512, st, static_cast<const uint4*>(in0), static_cast<const uint4*>(in1),
+                          static_cast<uint4*>(out), rows, bytes / 16, 1);
     if (vpt == 0) {
         k_row2_scalar<WHICH, DT><<<static_cast<unsigned>(rows), 256, 0, st>>>(static_cast<const S*>(in0), static_cast<const S*>(in1),
                                                                              static_cast<S*>(out), rows, cols);
@@ -408,6 +617,12 @@ tf_status run2(const void* in0, const void* in1, void* out, int64_t rows, int64_
 }  // namespace tf
 
 using namespace tf;
+
+extern "C" tf_status tf_softmax_variants_force(int cluster) {
+    if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8) return TF_ERR_INVALID_ARG;
+    g_force_cluster = cluster;
+    return TF_OK;
+}
 
 extern "C" tf_status tf_log_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols, tf_dtype dt, void* stream) {
     return run2<kOpLogSoftmax>(x, nullptr, y, rows, cols, dt, stream);

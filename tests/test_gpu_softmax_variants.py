@@ -96,6 +96,32 @@ def test_softmax_bwd_over_edge_widths(dt):
         run_softmax_bwd(dt, 9, cols, offset=offset)
 
 
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_cluster_per_row_and_streamed_forms(dt):
+    """A thread-block cluster shares a row: forced on short rows (ragged slices, empty slices, masked slices) and chosen by
+    itself beyond 32 KiB; with clusters switched off the same long rows take the streamed passes."""
+    ne = 4 if dt == F32 else 8
+    try:
+        for cluster in (2, 4, 8):
+            tf.tf_softmax_variants_force(cluster)
+            for rows, cols in ((1, ne), (5, 3 * ne), (33, 256), (700, 1000 // ne * ne), (64, 4096), (9, 40000 // ne * ne)):
+                run_log_softmax(dt, rows, cols, seed=cols + cluster, mask=True)
+                run_softmax_bwd(dt, rows, cols, seed=cols + cluster)
+            run_log_softmax(dt, 40, 2048, seed=3, inplace=True)
+            run_softmax_bwd(dt, 40, 2048, seed=3, inplace=True)
+        tf.tf_softmax_variants_force(1)
+        for rows, cols in ((6, 32768), (3, 200000 // ne * ne)):
+            run_log_softmax(dt, rows, cols, seed=cols, mask=True)
+            run_softmax_bwd(dt, rows, cols, seed=cols)
+    finally:
+        tf.tf_softmax_variants_force(0)
+    for rows, cols in ((70, 16384), (6, 32768), (5, 65536 + ne), (3, 131072)):      # automatic: clusters where the slices fit
+        run_log_softmax(dt, rows, cols, seed=cols, mask=True)
+        run_softmax_bwd(dt, rows, cols, seed=cols)
+    with pytest.raises(tf.TfError):
+        tf.tf_softmax_variants_force(3)
+
+
 def test_peaked_rows_and_closed_forms():
     # one dominant entry: y_max = -ln S is tiny and must still be right to the absolute part of the tolerance
     x = torch.full((4, 1024), -20.0, device="cuda")
