@@ -80,7 +80,7 @@ std::string plan_to_string(const Plan& p) {
         case V_TMA: snprintf(b, sizeof b, "tma:threads=%d,cluster=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.cluster, p.stages, p.chunk, p.persist); break;
         case V_PIPE: snprintf(b, sizeof b, "pipe:threads=%d,lanes=%d,vpt=%d,rpg=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.lanes, p.vpt, p.rpg, p.stages, p.chunk, p.persist); break;
         case V_RING: snprintf(b, sizeof b, "ring:threads=%d,vpt=%d,cluster=%d,stages=%d,persist=%d,psmem=%d", p.threads, p.vpt, p.cluster, p.stages, p.persist, p.rpg == 2 ? 1 : 0); break;
-        case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,cache=%d,persist=%d,regcap=%d", p.threads, p.chunk, p.persist, p.rpg == 2 ? 1 : 0); break;
+        case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,cache=%d,persist=%d,regcap=%d,cluster=%d", p.threads, p.chunk, p.persist, p.rpg == 2 ? 1 : 0, p.cluster); break;
         case V_SPLIT: snprintf(b, sizeof b, "split:threads=%d,splits=%d", p.threads, p.cluster); break;
         default: snprintf(b, sizeof b, "stream:threads=%d,lanes=%d,persist=%d", p.threads, p.lanes, p.persist); break;
     }
@@ -392,6 +392,10 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
                     p.chunk = cache ? static_cast<int>(std::min<int64_t>(nvec * 16, (200 * 1024 / (2048 / th)) / 16 * 16)) : 0;
                     add(p);
                     if (th <= 768 && persist == 0) { p.rpg = 2; add(p); }      // 40-register form: 1536 resident threads per SM
+                    // a cluster per row where rows are very long or few
+                    if (persist == 0 && th >= 512 && (nvec >= 16384 || a.rows < 2 * d.sms))
+                        for (int cl : {2, 4, 8})
+                            if (nvec / cl >= 2048) { Plan q = p; q.cluster = cl; q.chunk = std::min(q.chunk, static_cast<int>(nvec / cl * 16)); add(q); }
                 }
     // persistent cluster ring for long rows
     if (nvec >= 2048)
@@ -454,7 +458,7 @@ std::vector<Plan> neighbours(const Plan& b) {
     if (b.variant == V_SPLIT)
         for (int sp : {b.cluster / 2, b.cluster * 3 / 4, b.cluster * 3 / 2, b.cluster * 2})
             if (sp >= 1 && sp != b.cluster) with([&](Plan& p) { p.cluster = sp; });
-    if (b.variant == V_CTA || b.variant == V_RING || b.variant == V_TMA)
+    if (b.variant == V_CTA || b.variant == V_RING || b.variant == V_TMA || b.variant == V_TWOPASS)
         for (int cl : {b.cluster / 2, b.cluster * 2})
             if (cl >= 1 && cl <= kMaxCluster && cl != b.cluster) with([&](Plan& p) { p.cluster = cl; });
     return out;

@@ -532,12 +532,17 @@ cudaError_t launch_dt(cudaStream_t st, const void* in0, const void* in1, void* o
     const bool aligned = al16(in0) && al16(out) && (WHICH == kOpLogSoftmax || al16(in1)) && bytes % 16 == 0;
     int vpt = 0, threads = 0;
     // a cluster per row: rows beyond 32 KiB when there are too few of them to fill the device with one CTA each -- as many
-    // CTAs per row (2, 4 or 8) as keep the launch within about two CTAs per SM.  With more rows the streamed passes are
-    // faster (bf16 [8192, 32768]: 5.4 TB/s streamed, 3.6 with clusters).  Or where the hook asks.
+    // CTAs per row (2, 4 or 8) as keep the launch within about two CTAs per SM.  With more rows of up to 128 KiB the
+    // streamed passes of one CTA are faster (bf16 [8192, 32768]: 5.4 TB/s streamed, 3.6 with clusters).  Or where the hook asks.
+    // Rows of 256 KiB and more are shared whatever their number, in streamed slices of about 128 KiB: one CTA per row in
+    // flight on every SM is more than L2 holds of such rows, so the second pass went back to HBM (fp32 [2048, 131072]:
+    // 4.4 -> 6.0 TB/s with four CTAs per row).
     int cs = g_force_cluster > 1 ? g_force_cluster : 0;
     if (g_force_cluster == 0 && bytes / 16 > 2048) {
         const int64_t room = 2 * static_cast<int64_t>(sm_count()) / rows;
         cs = room >= 8 ? 8 : room >= 4 ? 4 : room >= 2 ? 2 : 0;
+        const int64_t pieces = bytes / (128 * 1024);
+        cs = std::max(cs, pieces >= 8 ? 8 : pieces >= 4 ? 4 : pieces >= 2 ? 2 : 0);
     }
     if (aligned && cs >= 2 && rows * kMaxCluster <= 0x7FFFFFFF) {
         const int64_t nv = bytes / 16;

@@ -257,7 +257,22 @@ def test_forced_twopass_variants(op, dt):
             tf.tf_force_plan(op, f"twopass:threads={threads},persist={persist},regcap={regcap}")
             fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec))
             assert not fails, (threads, persist, regcap, nvec, rows, fails)
+    # a thread-block cluster per row: ragged and empty slices, one row, rows left over after the last full pass, heads in shared memory
+    for cluster, threads, persist, regcap, cache in ((2, 256, 0, 0, 0), (4, 512, 0, 1, 4096), (8, 128, 1, 0, 0), (8, 1024, 2, 0, 16384), (2, 768, 0, 1, 49152)):
+        for nvec, rows in ((cluster, 5), (cluster + 1, 3), (threads * 4 * cluster + 1, 9), (threads * 9 - 3, 150), (70001, 3), (9, 1)):
+            tf.tf_force_plan(op, f"twopass:threads={threads},cache={cache},persist={persist},regcap={regcap},cluster={cluster}")
+            fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec + cluster))
+            assert not fails, (cluster, threads, persist, regcap, cache, nvec, rows, fails)
     if op == "softmax":                                    # masks, a fully masked row and outputs in the subnormal range
+        for plan in ("twopass:threads=256,persist=0,cluster=4", "twopass:threads=512,cache=8192,persist=0,regcap=1,cluster=8"):
+            tf.tf_force_plan(op, plan)
+            w = Workload("m", "softmax", dt, 12, 40000, seed=5, x_std=10.0, mask_step=3001)
+            data = w.generate()
+            ninf = np.float32(-np.inf) if dt == F32 else np.uint16(0xFF80)
+            data["x"][3, :] = ninf                                   # fully masked row
+            data["x"][5, :20000] = ninf                              # whole slices masked
+            data["x"][7, 0] = np.float32(75.0) if dt == F32 else np.uint16(0x4296)
+            assert not parity.check(w, data, parity.run_gpu(w, data), parity.run_oracle(w, data)), plan
         tf.tf_force_plan(op, "twopass:threads=256,persist=0")
         w = Workload("m", "softmax", dt, 12, 40000, seed=5, x_std=10.0, mask_step=3001)
         data = w.generate()

@@ -92,6 +92,10 @@ def test_forced_plans_and_bitwise_equality_with_the_masked_plain_softmax(dt):
         for nvec, rows in ((1, 9), (threads * 4 + 1, 9), (threads * 9 - 3, 60), (70001, 9)):
             tf.tf_force_plan("softmax", f"twopass:threads={threads},cache={cache},persist={persist},regcap={regcap}")
             run_case(dt, rows, nvec * ne, seed=nvec, compare_plain=True)
+    for cluster, threads, cache in ((2, 256, 0), (4, 512, 8192), (8, 128, 0)):           # lengths that end inside any slice, or before the first
+        for nvec, rows in ((cluster + 1, 9), (threads * 4 * cluster + 1, 9), (70001, 9)):
+            tf.tf_force_plan("softmax", f"twopass:threads={threads},cache={cache},persist=0,regcap=0,cluster={cluster}")
+            run_case(dt, rows, nvec * ne, seed=nvec + cluster)
     # a forced plan without a length mode (the pipeline) falls back to the length-aware choice
     tf.tf_force_plan("softmax", "pipe:threads=512,lanes=64,vpt=8,rpg=1,stages=2,chunk=8192,persist=1")
     run_case(dt, 100, 512 * ne)
