@@ -636,7 +636,7 @@ BwdPlan bwd_plan(int64_t rows, int nvec, bool staged, int stages, int gmax = 256
     p.vpt = 1;
     while (p.vpt < kMaxVpt && (nvec + p.vpt - 1) / p.vpt > gmax) p.vpt *= 2;    // row groups of up to gmax threads while that holds the row
     p.gt = std::max(32, ((nvec + p.vpt - 1) / p.vpt + 31) / 32 * 32);
-    p.groups = std::max(1, std::min(8, 256 / p.gt));                            // short rows: several per CTA
+    p.groups = std::max(1, std::min(8, 128 / p.gt));                            // short rows: several per CTA (CTAs of 128 threads measured best)
     const int threads = p.gt * p.groups;
     p.full = nvec == p.gt * p.vpt && rows % p.groups == 0;          // no vector and no row slot is ever absent
     const void* fn = p.vpt == 1 ? bwd_fn<RMS, DT, 1>(staged, p.full) : p.vpt == 2 ? bwd_fn<RMS, DT, 2>(staged, p.full) : bwd_fn<RMS, DT, kMaxVpt>(staged, p.full);
@@ -664,14 +664,14 @@ BwdPlan bwd_plan(int64_t rows, int nvec, bool staged, int stages, int gmax = 256
     return p;
 }
 
-// Which form runs, unless the hook says otherwise: the staged one for 2-byte elements in rows of 8 KiB and more (measured
-// 9-15 % faster there: a row ahead in registers is half as many bytes in flight as with 4-byte elements), the register
-// form elsewhere (shorter rows and 4-byte elements: equal or faster).
+// Which form runs, unless the hook says otherwise: the staged one for 2-byte elements in rows of 2 KiB and more, two
+// vectors per thread (measured 7-15 % faster there: a row ahead in registers is half as many bytes in flight as with
+// 4-byte elements), the register form elsewhere (shorter rows and 4-byte elements: equal or faster).
 template <bool RMS, int DT>
 BwdPlan choose_bwd_plan_uncached(int64_t rows, int nvec) {
-    const bool want = g_force_path >= 2 || (g_force_path == 0 && DT == DT_BF16 && nvec >= 512);
+    const bool want = g_force_path >= 2 || (g_force_path == 0 && DT == DT_BF16 && nvec >= 128);
     if (want) {
-        const BwdPlan p = bwd_plan<RMS, DT>(rows, nvec, true, g_force_stages, g_force_path == 2 ? 512 : 256);
+        const BwdPlan p = bwd_plan<RMS, DT>(rows, nvec, true, g_force_stages, g_force_path == 2 ? 512 : g_force_path == 3 ? 256 : 64);
         if (p.stages >= 2) return p;
     }
     return bwd_plan<RMS, DT>(rows, nvec, false, 0);
@@ -899,8 +899,8 @@ extern "C" size_t tf_norm_bwd_workspace_bytes(int64_t rows, int64_t cols) {
     // the most partial column sums any of the paths may write for this shape, whatever the element type or the op
     int64_t parts = std::min<int64_t>(rows, sm_count());                          // the streamed kernel: one CTA per SM
     auto widest = [&](auto plan) {                                                 // any form may be chosen (or forced)
-        for (int form = 0; form < 3; ++form) {
-            const BwdPlan p = plan(form != 0, form == 2 ? 512 : 256);
+        for (int form = 0; form < 4; ++form) {
+            const BwdPlan p = plan(form != 0, form == 2 ? 512 : form == 3 ? 64 : 256);
             parts = std::max<int64_t>(parts, static_cast<int64_t>(p.grid) * p.groups);
         }
     };
