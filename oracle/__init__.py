@@ -67,6 +67,8 @@ def _load():
         lib.oracle_log_softmax.restype = i32
         lib.oracle_softmax_bwd.argtypes = [vp, vp, vp, vp, vp, i64, i64, i32, i32]
         lib.oracle_softmax_bwd.restype = i32
+        lib.oracle_log_softmax_bwd.argtypes = [vp, vp, vp, vp, vp, i64, i64, i32, i32]
+        lib.oracle_log_softmax_bwd.restype = i32
         lib.oracle_norm_bwd.argtypes = [vp] * 14 + [i64, i64, i32, i32, i32]
         lib.oracle_norm_bwd.restype = i32
         lib.oracle_add.argtypes = [vp, vp, vp, vp, i64, i32]
@@ -137,6 +139,20 @@ def softmax_bwd(y: np.ndarray, dy: np.ndarray, dt: int, want64: bool = False, nt
     sc = np.empty((rows, cols), np.float64) if want64 else None
     if _load().oracle_softmax_bwd(_p(y), _p(dy), _p(dx), _p(dx64), _p(sc), rows, cols, dt, nthreads):
         raise ValueError("oracle_softmax_bwd: bad argument")
+    return (dx, dx64, sc) if want64 else dx
+
+
+def log_softmax_bwd(y: np.ndarray, dy: np.ndarray, dt: int, want64: bool = False, nthreads: int = 1):
+    """Log-softmax backward ``dx = dy - exp(y) * sum(dy)`` per row.  Returns ``dx`` plus ``(dx64, scale64)`` if ``want64``."""
+    _check(y, dt, "y"), _check(dy, dt, "dy")
+    if y.shape != dy.shape:
+        raise ValueError("y and dy must have the same shape")
+    rows, cols = y.shape
+    dx = np.empty_like(y)
+    dx64 = np.empty((rows, cols), np.float64) if want64 else None
+    sc = np.empty((rows, cols), np.float64) if want64 else None
+    if _load().oracle_log_softmax_bwd(_p(y), _p(dy), _p(dx), _p(dx64), _p(sc), rows, cols, dt, nthreads):
+        raise ValueError("oracle_log_softmax_bwd: bad argument")
     return (dx, dx64, sc) if want64 else dx
 
 

@@ -299,6 +299,31 @@ int oracle_softmax_bwd(const void* y, const void* dy, void* dx, double* dx64, do
     return 0;
 }
 
+// Log-softmax backward:  dx_j = dy_j - exp(y_j) * sum_k dy_k, y the forward output (log-probabilities) as stored, dy the
+// incoming gradient; exp(-inf) = 0, so masked entries pass their gradient through.  scale64 (nullable) receives
+// |dy_j| + exp(y_j) * sum_k |dy_k|, the quantity an error bound for the difference is stated against.
+int oracle_log_softmax_bwd(const void* y, const void* dy, void* dx, double* dx64, double* scale64, int64_t rows, int64_t cols,
+                           int dt, int nthreads) {
+    if (bad(rows, cols, dt) || !y || !dy) return -1;
+    for_rows(rows, nthreads, [=](int64_t r) {
+        const int64_t base = r * cols;
+        double s = 0.0, sa = 0.0;
+        for (int64_t j = 0; j < cols; ++j) {
+            const double g = load(dy, base + j, dt);
+            s += g;
+            sa += std::fabs(g);
+        }
+        for (int64_t j = 0; j < cols; ++j) {
+            const double p = std::exp(load(y, base + j, dt)), gj = load(dy, base + j, dt);
+            const double v = gj - p * s;
+            if (dx64) dx64[base + j] = v;
+            if (scale64) scale64[base + j] = std::fabs(gj) + p * sa;
+            if (dx) store(dx, base + j, dt, v);
+        }
+    });
+    return 0;
+}
+
 // Backward pass of LayerNorm (rms = 0) or RMSNorm (rms = 1) from the forward pass's stored fp32 statistics.
 //   xh_j = (x_j - mean) * rstd   (RMSNorm: x_j * rstd),   g_j = dy_j * gamma_j
 //   LayerNorm:  dx_j = rstd * (g_j - mean_k g_k - xh_j * mean_k (g_k xh_k))

@@ -1,4 +1,4 @@
-"""Pins for the oracle's log-softmax and softmax backward pass.  CPU only."""
+"""Pins for the oracle's log-softmax, softmax backward and log-softmax backward passes.  CPU only."""
 from __future__ import annotations
 
 import math
@@ -124,3 +124,65 @@ def test_softmax_bwd_jacobian_finite_differences_and_library():
     np.testing.assert_array_equal(dxb, oracle.bf16_from_double(dxb64))
     ybd, gbd = oracle.bf16_to_double(yb), oracle.bf16_to_double(gb)
     np.testing.assert_allclose(dxb64, ybd * (gbd - (ybd * gbd).sum(axis=1, keepdims=True)), rtol=1e-13, atol=1e-17)
+
+
+def test_log_softmax_bwd_jacobian_finite_differences_and_library():
+    rng = np.random.default_rng(47)
+    rows, n = 4, 9
+    x = f32(rng.standard_normal((rows, n)) * 2)
+    _, y64 = oracle.log_softmax(x, F32, want64=True)
+    y = f32(y64)                                                                # the stored log-probabilities
+    yd = y.astype(np.float64)
+    p = np.exp(yd)
+    # (1) one-hot dy = e_i gives row i of the Jacobian of log-softmax: dx_j = delta_ij - p_j
+    for i in (0, 4, n - 1):
+        dy = np.zeros((rows, n)); dy[:, i] = 1.0
+        _, dx64, _ = oracle.log_softmax_bwd(y, f32(dy), F32, want64=True)
+        np.testing.assert_allclose(dx64, (np.arange(n)[None, :] == i) - p, rtol=1e-14, atol=1e-17)
+    # (2) the loss -y_t of a cross entropy: dy = -e_t gives p - e_t, whose entries sum to zero as far as p sums to one
+    dy = np.zeros((rows, n)); dy[np.arange(rows), [1, 0, 8, 3]] = -1.0
+    _, dx64, _ = oracle.log_softmax_bwd(y, f32(dy), F32, want64=True)
+    np.testing.assert_allclose(dx64, p + dy, rtol=1e-14, atol=1e-17)
+    np.testing.assert_allclose(dx64.sum(axis=1), p.sum(axis=1) - 1.0, rtol=0, atol=1e-15)
+    assert np.abs(dx64.sum(axis=1)).max() < 1e-6
+    # (3) a gradient that sums to zero passes through unchanged, exactly
+    z = rng.standard_normal((rows, n)); z[:, -1] = 0; z = f32(z)
+    z[:, -1] = 0
+    zs = z.astype(np.float64); zs[:, -1] = -zs[:, :-1].sum(axis=1)
+    if np.array_equal(f32(zs).astype(np.float64), zs) and (f32(zs).astype(np.float64).sum(axis=1) == 0).all():
+        np.testing.assert_array_equal(oracle.log_softmax_bwd(y, f32(zs), F32, want64=True)[1], zs)
+    # (4) central differences of the pinned forward pass in double
+    dyv = f32(rng.standard_normal((rows, n)))
+    xd = x.astype(np.float64)
+    def fwd(zz):
+        m = zz.max(axis=1, keepdims=True); return (zz - m) - np.log(np.exp(zz - m).sum(axis=1, keepdims=True))
+    num = np.zeros((rows, n))
+    h = 1e-6
+    for j in range(n):
+        zp, zm = xd.copy(), xd.copy()
+        zp[:, j] += h; zm[:, j] -= h
+        num[:, j] = ((fwd(zp) - fwd(zm)) / (2 * h) * dyv.astype(np.float64)).sum(axis=1)
+    _, exact, _ = oracle.log_softmax_bwd(f32(fwd(xd)), dyv, F32, want64=True)   # y rounded to fp32: error ~1e-6
+    np.testing.assert_allclose(exact, num, rtol=0, atol=5e-6)
+    # (5) torch autograd in float64, the formula re-evaluated on the stored y, linearity in dy, the condition scale
+    gt = torch.from_numpy(dyv.astype(np.float64))
+    xt = torch.from_numpy(xd).requires_grad_(True)
+    torch.log_softmax(xt, dim=1).backward(gt)
+    _, dx64, sc = oracle.log_softmax_bwd(y, dyv, F32, want64=True, nthreads=2)
+    gd = dyv.astype(np.float64)
+    np.testing.assert_allclose(dx64, gd - p * gd.sum(axis=1, keepdims=True), rtol=1e-13, atol=1e-16)
+    np.testing.assert_allclose(dx64, xt.grad.numpy(), rtol=0, atol=3e-6)         # autograd uses the unrounded y
+    np.testing.assert_allclose(sc, np.abs(gd) + p * np.abs(gd).sum(axis=1, keepdims=True), rtol=1e-13)
+    _, dx2, _ = oracle.log_softmax_bwd(y, f32(2.0 * gd), F32, want64=True)
+    np.testing.assert_array_equal(dx2, 2.0 * dx64)
+    # (6) masked entries (y = -inf) pass their gradient through; a fully masked row passes dy through entirely
+    ym = y.copy(); ym[1, 3:] = -np.inf; ym[2, :] = -np.inf
+    _, dxm, _ = oracle.log_softmax_bwd(ym, dyv, F32, want64=True)
+    np.testing.assert_array_equal(dxm[1, 3:], gd[1, 3:])
+    np.testing.assert_array_equal(dxm[2], gd[2])
+    # (7) bf16: stored result is the single rounding of the double
+    yb, gb = bf(yd), bf(dyv)
+    dxb, dxb64, _ = oracle.log_softmax_bwd(yb, gb, BF16, want64=True)
+    np.testing.assert_array_equal(dxb, oracle.bf16_from_double(dxb64))
+    ybd, gbd = oracle.bf16_to_double(yb), oracle.bf16_to_double(gb)
+    np.testing.assert_allclose(dxb64, gbd - np.exp(ybd) * gbd.sum(axis=1, keepdims=True), rtol=1e-13, atol=1e-17)
