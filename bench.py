@@ -660,6 +660,7 @@ def run_softmax_variants_table(args):
         xs = [conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols, 0, 0.0, 3.0))).cuda() for _ in range(sets)]
         gs = [conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols + 1, 1, 0.0, 1.0))).cuda() for _ in range(sets)]
         ys = [torch.softmax(x.float(), dim=1).to(x.dtype) for x in xs]
+        lys = [torch.log_softmax(x.float(), dim=1).to(x.dtype) for x in xs]
         outs = [torch.empty_like(x) for x in xs]
 
         def timed(fn, reps):
@@ -679,7 +680,9 @@ def run_softmax_variants_table(args):
                 ("log_softmax_fwd", 2 * rows * cols * es, lambda k: tf.tf_log_softmax_fwd(xs[k], outs[k]),
                  lambda k: torch.log_softmax(xs[k], dim=1, out=outs[k]) if False else torch.log_softmax(xs[k], dim=1)),
                 ("softmax_bwd", 3 * rows * cols * es, lambda k: tf.tf_softmax_bwd(ys[k], gs[k], outs[k]),
-                 lambda k: torch._softmax_backward_data(gs[k], ys[k], 1, ys[k].dtype))):
+                 lambda k: torch._softmax_backward_data(gs[k], ys[k], 1, ys[k].dtype)),
+                ("log_softmax_bwd", 3 * rows * cols * es, lambda k: tf.tf_log_softmax_bwd(lys[k], gs[k], outs[k]),
+                 lambda k: torch._log_softmax_backward_data(gs[k], lys[k], 1, lys[k].dtype))):
             us, us_lib = timed(ours, reps), timed(lib, max(5, reps // 2))
             row = {"op": op, "dtype": "f32" if dt == inputs.F32 else "bf16", "rows": rows, "cols": cols, "bytes": nbytes, "us": us,
                    "gbs": nbytes / us / 1e3, f"pct_of_{peak_kind}_{peak:.0f}": 100 * nbytes / us / 1e3 / peak, "torch_us": us_lib,
@@ -687,7 +690,7 @@ def run_softmax_variants_table(args):
             rows_out.append(row)
             print(json.dumps(row), flush=True)
         tf.tf_device_status()
-        del xs, gs, ys, outs
+        del xs, gs, ys, lys, outs
         torch.cuda.empty_cache()
     (out_dir / "table_softmaxvariants.json").write_text(json.dumps(rows_out, indent=1))
 

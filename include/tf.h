@@ -147,6 +147,12 @@ tf_status tf_log_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols,
  * runs scalar passes. */
 tf_status tf_softmax_bwd(const void* y, const void* dy, void* dx, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
 
+/* dx_j = dy_j - exp(y_j) * sum_k dy_k: the backward pass of log-softmax from its stored output y (log-probabilities) and
+ * the incoming gradient dy; with dy = -e_t it is the gradient of a cross-entropy loss, softmax(x) - e_t.  exp(-inf) = 0:
+ * masked entries pass their gradient through.  fp32 arithmetic, one rounding; probabilities in the subnormal range are
+ * not flushed.  Same layouts, aliasing, forms and errors as tf_softmax_bwd.  The paper has no counterpart. */
+tf_status tf_log_softmax_bwd(const void* y, const void* dy, void* dx, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
+
 /* ---- backward passes of the norms ------------------------------------------------------------------------- */
 
 /* From the forward pass's inputs and its stored fp32 statistics (mean, rstd: [rows]):

@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_norm_bwd_workspace_bytes", "tf_layernorm_bwd", "tf_rmsnorm_bwd", "tf_norm_bwd_force", "tf_softmax_variants_force",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_log_softmax_bwd", "tf_norm_bwd_workspace_bytes", "tf_layernorm_bwd", "tf_rmsnorm_bwd", "tf_norm_bwd_force", "tf_softmax_variants_force",
            "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
@@ -60,6 +60,7 @@ def lib() -> ctypes.CDLL:
         L.tf_softmax_len_fwd.argtypes = [vp, vp, vp, i64, i64, i32, vp]
         L.tf_log_softmax_fwd.argtypes = [vp, vp, i64, i64, i32, vp]
         L.tf_softmax_bwd.argtypes = [vp, vp, vp, i64, i64, i32, vp]
+        L.tf_log_softmax_bwd.argtypes = [vp, vp, vp, i64, i64, i32, vp]
         L.tf_norm_bwd_workspace_bytes.argtypes = [i64, i64]
         L.tf_norm_bwd_workspace_bytes.restype = ctypes.c_size_t
         L.tf_layernorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i64, i64, i32, vp]
@@ -188,6 +189,21 @@ def tf_softmax_bwd(y, dy, dx=None):
     rows, cols = y.shape
     with _on_device(y):
         _ok(lib().tf_softmax_bwd(y.data_ptr(), dy.data_ptr(), dx.data_ptr(), rows, cols, _dt(y), _stream(y)), "tf_softmax_bwd")
+    return dx
+
+
+def tf_log_softmax_bwd(y, dy, dx=None):
+    """Log-softmax backward ``dx = dy - exp(y) * sum(dy, -1)`` from the stored log-probabilities ``y`` and the gradient ``dy``."""
+    import torch
+    _check2d(y, "y")
+    _check2d(dy, "dy")
+    if dy.shape != y.shape or dy.dtype != y.dtype:
+        raise ValueError("dy must match y")
+    if dx is None:
+        dx = torch.empty_like(y)
+    rows, cols = y.shape
+    with _on_device(y):
+        _ok(lib().tf_log_softmax_bwd(y.data_ptr(), dy.data_ptr(), dx.data_ptr(), rows, cols, _dt(y), _stream(y)), "tf_log_softmax_bwd")
     return dx
 
 

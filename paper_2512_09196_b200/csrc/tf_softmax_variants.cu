@@ -1,7 +1,8 @@
-// Two more row-wise reduce-then-normalise ops on the softmax family:
-//   log-softmax forward   y_j  = (x_j - m) - ln sum_k exp(x_k - m),  m = max_k x_k
-//   softmax backward      dx_j = y_j * (dy_j - sum_k y_k dy_k)
-// One kernel shape serves both: a CTA owns a row and holds it in registers (VPT 16-byte vectors per thread, loaded at
+// Three more row-wise reduce-then-normalise ops on the softmax family:
+//   log-softmax forward    y_j  = (x_j - m) - ln sum_k exp(x_k - m),  m = max_k x_k
+//   softmax backward       dx_j = y_j * (dy_j - sum_k y_k dy_k)
+//   log-softmax backward   dx_j = dy_j - exp(y_j) * sum_k dy_k
+// One kernel shape serves all of them: a CTA owns a row and holds it in registers (VPT 16-byte vectors per thread, loaded at
 // once), reduces across the CTA, finishes and stores -- one read of every input element, one write of every output
 // element.  Rows of up to 2 KiB are owned by lane groups instead (several rows per warp).  Rows beyond 32 KiB are
 // streamed in two passes of 16-byte loads, the second from L2; when such rows are too few to give every SM a CTA (logits
@@ -24,10 +25,24 @@ namespace cg = cooperative_groups;
 namespace tf {
 namespace {
 
-constexpr int kOpLogSoftmax = 0, kOpSoftmaxBwd = 1;
+constexpr int kOpLogSoftmax = 0, kOpSoftmaxBwd = 1, kOpLogSoftmaxBwd = 2;
+
+// The two backward passes share every kernel: both reduce one number per row from (y, dy) and finish element-wise.
+//   softmax backward       term y dy,  dx = y (dy - sum)
+//   log-softmax backward   term dy,    dx = dy - exp(y) sum
+// exp(y) is one MUFU op on a biased exponent (2^(y log2 e + 64), flushing only below a true value of 2^-190) scaled back
+// by an exact, non-flushing 2^-64: probabilities in the subnormal range stay exact to rounding; exp(-inf) = 0.
+template <int WHICH> __device__ __forceinline__ float bwd_accumulate(float y, float g, float s) {
+    return WHICH == kOpSoftmaxBwd ? fmaf(y, g, s) : s + g;
+}
+template <int WHICH> __device__ __forceinline__ float bwd_finish(float y, float g, float s) {
+    if (WHICH == kOpSoftmaxBwd) return y * (g - s);
+    const float p = ex2_ftz(fmaf(y, kLog2e, 64.f)) * 0x1p-64f;
+    return fmaf(-p, s, g);
+}
 
 // fp32 values a thread holds for its share of a row; up to 32 of them leave room for 1024 threads, up to 64 for 512.
-template <int WHICH, int DT, int VPT> constexpr int row2_floats() { return VPT * Elem<DT>::NE * (WHICH == kOpSoftmaxBwd ? 2 : 1); }
+template <int WHICH, int DT, int VPT> constexpr int row2_floats() { return VPT * Elem<DT>::NE * (WHICH != kOpLogSoftmax ? 2 : 1); }
 template <int WHICH, int DT, int VPT> constexpr int row2_max_threads() { return row2_floats<WHICH, DT, VPT>() <= 32 ? 1024 : 512; }
 
 template <int WHICH, int DT, int VPT>
@@ -87,14 +102,14 @@ __global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2(con
             E::unpack(ra[v], y[v]);
             E::unpack(rb, g[v]);
 #pragma unroll
-            for (int i = 0; i < NE; ++i) s = fmaf(y[v][i], g[v][i], s);    // absent vectors hold zeros
+            for (int i = 0; i < NE; ++i) s = bwd_accumulate<WHICH>(y[v][i], g[v][i], s);    // absent vectors hold zeros
         }
         s = cta_reduce<SumOp>(s, buf[0]);
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
             float dx[NE];
 #pragma unroll
-            for (int i = 0; i < NE; ++i) dx[i] = y[v][i] * (g[v][i] - s);
+            for (int i = 0; i < NE; ++i) dx[i] = bwd_finish<WHICH>(y[v][i], g[v][i], s);
             if (valid[v]) st_stream(o + v * T, E::pack(dx));
         }
     }
@@ -130,7 +145,7 @@ __global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2_clu
     for (int v = 0; v < VPT; ++v) {
         valid[v] = t + v * T < len;
         ra[v] = valid[v] ? ld_stream(a + v * T) : make_uint4(0, 0, 0, 0);
-        if (WHICH == kOpSoftmaxBwd) rb[v] = valid[v] ? ld_stream(in1 + row * nvec + first + t + v * T) : make_uint4(0, 0, 0, 0);
+        if (WHICH != kOpLogSoftmax) rb[v] = valid[v] ? ld_stream(in1 + row * nvec + first + t + v * T) : make_uint4(0, 0, 0, 0);
     }
     cl.sync();                     // every CTA of the cluster is resident before any remote write (the loads are already under way)
     if constexpr (WHICH == kOpLogSoftmax) {
@@ -177,7 +192,7 @@ __global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2_clu
             E::unpack(ra[v], y[v]);
             E::unpack(rb[v], g[v]);
 #pragma unroll
-            for (int i = 0; i < NE; ++i) s = fmaf(y[v][i], g[v][i], s);    // absent vectors hold zeros
+            for (int i = 0; i < NE; ++i) s = bwd_accumulate<WHICH>(y[v][i], g[v][i], s);    // absent vectors hold zeros
         }
         s = cta_reduce<SumOp>(s, buf[0]);
         if (t < cs) {
@@ -191,7 +206,7 @@ __global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2_clu
         for (int v = 0; v < VPT; ++v) {
             float dx[NE];
 #pragma unroll
-            for (int i = 0; i < NE; ++i) dx[i] = y[v][i] * (g[v][i] - total);
+            for (int i = 0; i < NE; ++i) dx[i] = bwd_finish<WHICH>(y[v][i], g[v][i], total);
             if (valid[v]) st_stream(o + v * T, E::pack(dx));
         }
     }
@@ -254,14 +269,14 @@ __global__ void __launch_bounds__(128) k_row2_group(const uint4* __restrict__ in
             E::unpack(ra[v], y[v]);
             E::unpack(rb, g[v]);
 #pragma unroll
-            for (int i = 0; i < NE; ++i) s = fmaf(y[v][i], g[v][i], s);
+            for (int i = 0; i < NE; ++i) s = bwd_accumulate<WHICH>(y[v][i], g[v][i], s);
         }
         s = group_reduce<SumOp, LANES>(s);
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
             float dx[NE];
 #pragma unroll
-            for (int i = 0; i < NE; ++i) dx[i] = y[v][i] * (g[v][i] - s);
+            for (int i = 0; i < NE; ++i) dx[i] = bwd_finish<WHICH>(y[v][i], g[v][i], s);
             if (valid[v]) st_stream(out + base + v * LANES, E::pack(dx));
         }
     }
@@ -365,7 +380,7 @@ __global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ i
                 E::unpack(ry[u], y);
                 E::unpack(rg[u], g);
 #pragma unroll
-                for (int i = 0; i < NE; ++i) s = fmaf(y[i], g[i], s);
+                for (int i = 0; i < NE; ++i) s = bwd_accumulate<WHICH>(y[i], g[i], s);
             }
         }
         s = cta_reduce<SumOp>(s, buf[0]);
@@ -393,7 +408,7 @@ __global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ i
                 E::unpack(ry[u], y);
                 E::unpack(rg[u], g);
 #pragma unroll
-                for (int i = 0; i < NE; ++i) y[i] = y[i] * (g[i] - s);
+                for (int i = 0; i < NE; ++i) y[i] = bwd_finish<WHICH>(y[i], g[i], s);
                 if (b0 + u * T < nvec) st_stream(o + b0 + u * T, E::pack(y));
             }
         }
@@ -424,9 +439,9 @@ __global__ void __launch_bounds__(256) k_row2_scalar(const typename Elem<DT>::sc
     } else {
         const typename E::scalar* b = in1 + row * cols;
         float s = 0.f;
-        for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) s = fmaf(E::to_float(a[j]), E::to_float(b[j]), s);
+        for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) s = bwd_accumulate<WHICH>(E::to_float(a[j]), E::to_float(b[j]), s);
         s = cta_reduce<SumOp>(s, buf[0]);
-        for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) o[j] = E::from_float(E::to_float(a[j]) * (E::to_float(b[j]) - s));
+        for (int64_t j = threadIdx.x; j < cols; j += blockDim.x) o[j] = E::from_float(bwd_finish<WHICH>(E::to_float(a[j]), E::to_float(b[j]), s));
     }
 }
 
@@ -606,7 +621,7 @@ cudaError_t launch_dt(cudaStream_t st, const void* in0, const void* in1, void* o
 template <int WHICH>
 tf_status run2(const void* in0, const void* in1, void* out, int64_t rows, int64_t cols, int dt, void* stream) {
     if (rows < 0 || cols <= 0 || (dt != DT_F32 && dt != DT_BF16)) return TF_ERR_INVALID_ARG;
-    if (rows > 0 && (!in0 || !out || (WHICH == kOpSoftmaxBwd && !in1))) return TF_ERR_INVALID_ARG;
+    if (rows > 0 && (!in0 || !out || (WHICH != kOpLogSoftmax && !in1))) return TF_ERR_INVALID_ARG;
     if (rows == 0) return TF_OK;
     if (cols > (INT64_MAX / 8) / rows) return TF_ERR_UNSUPPORTED;
     count_launches(1);
@@ -631,6 +646,10 @@ extern "C" tf_status tf_softmax_variants_force(int cluster) {
 
 extern "C" tf_status tf_log_softmax_fwd(const void* x, void* y, int64_t rows, int64_t cols, tf_dtype dt, void* stream) {
     return run2<kOpLogSoftmax>(x, nullptr, y, rows, cols, dt, stream);
+}
+
+extern "C" tf_status tf_log_softmax_bwd(const void* y, const void* dy, void* dx, int64_t rows, int64_t cols, tf_dtype dt, void* stream) {
+    return run2<kOpLogSoftmaxBwd>(y, dy, dx, rows, cols, dt, stream);
 }
 
 extern "C" tf_status tf_softmax_bwd(const void* y, const void* dy, void* dx, int64_t rows, int64_t cols, tf_dtype dt, void* stream) {

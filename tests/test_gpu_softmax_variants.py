@@ -6,7 +6,9 @@ Tolerances (derived from the arithmetic, fp32 throughout):
   2^17 terms (a few 2^-24 of absolute error however small ln S itself is).  bf16 outputs add half a bf16 ulp.
   Where x_j = -inf the output must be -inf.
 * softmax backward: |g - o| <= 1e-5 * |y_j| (|dy_j| + sum_k |y_k dy_k|) -- dy_j - sum y dy cancels, so the bound is
-  stated against what is subtracted -- plus one fp32 subnormal quantum; bf16 outputs add half a bf16 ulp."""
+  stated against what is subtracted -- plus one fp32 subnormal quantum; bf16 outputs add half a bf16 ulp.
+* log-softmax backward: |g - o| <= 1e-5 * (|dy_j| + exp(y_j) sum_k |dy_k|), the same rule on dy_j - exp(y_j) sum dy (the
+  exponential is one rounding of y log2 e + 64 and one MUFU op: at most 6e-6 relative at |y| ~ 100, 1e-6 at |y| ~ 20)."""
 from __future__ import annotations
 
 import numpy as np
@@ -72,6 +74,49 @@ def run_softmax_bwd(dt, rows, cols, seed=1, offset=0, inplace=False):
     check_close(parity.to_host(dx, dt), ref, ref64, sc, dt, 0.0, ("softmax_bwd", dt, rows, cols, offset))
 
 
+def run_log_softmax_bwd(dt, rows, cols, seed=1, offset=0, inplace=False, mask=False, std=2.0):
+    x = inputs.normal((rows, cols), dt, seed, 0, 0.0, std)
+    if mask:
+        ninf = np.float32(-np.inf) if dt == F32 else np.uint16(0xFF80)
+        x[::3, cols // 2:] = ninf
+        if rows > 1:
+            x[1, :] = ninf                                        # a fully masked row: y = -inf, dx = dy
+    y = oracle.log_softmax(x, dt, nthreads=8)                     # real stored log-probabilities
+    dy = inputs.normal((rows, cols), dt, seed + 7, 1, 0.1, 1.5)
+    ref, ref64, sc = oracle.log_softmax_bwd(y, dy, dt, want64=True, nthreads=8)
+    yd, gd = parity.to_dev(y, dt, offset), parity.to_dev(dy, dt, offset)
+    dx = tf.tf_log_softmax_bwd(yd, gd, gd if inplace else None)
+    torch.cuda.synchronize()
+    check_close(parity.to_host(dx, dt), ref, ref64, sc, dt, 0.0, ("log_softmax_bwd", dt, rows, cols, offset))
+
+
+@pytest.mark.parametrize("dt", [F32, BF16])
+def test_log_softmax_bwd_over_edge_widths(dt):
+    ne = 4 if dt == F32 else 8
+    for cols in (ne, 3 * ne, 64, 256, 1000 // ne * ne, 1024, 2048 + ne, 4096, 5120, 16384, 32768 + ne, 65536, 200000 // ne * ne):
+        for rows in (1, 9, 300):
+            if rows * cols > (1 << 22):
+                rows = max(3, (1 << 22) // cols)
+            run_log_softmax_bwd(dt, rows, cols, seed=cols + rows, mask=cols >= 64)
+    run_log_softmax_bwd(dt, 2000, 512)
+    run_log_softmax_bwd(dt, 40, 2048, inplace=True)
+    run_log_softmax_bwd(dt, 20, 4096, std=30.0)                   # log-probabilities down to -100 and below: tiny and zero exp(y)
+    for cols, offset in ((1001, 0), (7, 0), (1024, 1), (4099, 3)):
+        run_log_softmax_bwd(dt, 9, cols, offset=offset)
+    assert tf.tf_log_softmax_bwd(torch.empty(0, 64, device="cuda"), torch.empty(0, 64, device="cuda")).shape == (0, 64)
+
+
+def test_log_softmax_bwd_is_the_cross_entropy_gradient():
+    torch.manual_seed(0)
+    x = torch.randn(300, 5000, device="cuda", requires_grad=True)
+    t = torch.randint(0, 5000, (300,), device="cuda")
+    torch.nn.functional.cross_entropy(x, t, reduction="sum").backward()
+    y = tf.tf_log_softmax_fwd(x.detach())
+    dy = torch.zeros_like(y); dy[torch.arange(300), t] = -1.0
+    dx = tf.tf_log_softmax_bwd(y, dy)
+    assert (dx - x.grad).abs().max().item() < 2e-6
+
+
 @pytest.mark.parametrize("dt", [F32, BF16])
 def test_log_softmax_over_edge_widths(dt):
     ne = 4 if dt == F32 else 8
@@ -107,17 +152,20 @@ def test_cluster_per_row_and_streamed_forms(dt):
             for rows, cols in ((1, ne), (5, 3 * ne), (33, 256), (700, 1000 // ne * ne), (64, 4096), (9, 40000 // ne * ne)):
                 run_log_softmax(dt, rows, cols, seed=cols + cluster, mask=True)
                 run_softmax_bwd(dt, rows, cols, seed=cols + cluster)
+                run_log_softmax_bwd(dt, rows, cols, seed=cols + cluster, mask=True)
             run_log_softmax(dt, 40, 2048, seed=3, inplace=True)
             run_softmax_bwd(dt, 40, 2048, seed=3, inplace=True)
         tf.tf_softmax_variants_force(1)
         for rows, cols in ((6, 32768), (3, 200000 // ne * ne)):
             run_log_softmax(dt, rows, cols, seed=cols, mask=True)
             run_softmax_bwd(dt, rows, cols, seed=cols)
+            run_log_softmax_bwd(dt, rows, cols, seed=cols, mask=True)
     finally:
         tf.tf_softmax_variants_force(0)
     for rows, cols in ((70, 16384), (6, 32768), (5, 65536 + ne), (3, 131072)):      # automatic: clusters where the slices fit
         run_log_softmax(dt, rows, cols, seed=cols, mask=True)
         run_softmax_bwd(dt, rows, cols, seed=cols)
+        run_log_softmax_bwd(dt, rows, cols, seed=cols, mask=True)
     with pytest.raises(tf.TfError):
         tf.tf_softmax_variants_force(3)
 
@@ -164,3 +212,4 @@ def test_shapes_of_the_bench_table_every_element(dt, rows, cols):
     every element against the oracle."""
     run_log_softmax(dt, rows, cols, seed=cols)
     run_softmax_bwd(dt, rows, cols, seed=cols)
+    run_log_softmax_bwd(dt, rows, cols, seed=cols)
