@@ -37,13 +37,23 @@ constexpr int kModePlain = 0, kModeAdd = 1, kModeLen = 2;
 // Row length in elements, clamped to [0, cols].
 __device__ __forceinline__ int row_len(const int* len, int64_t row, int cols) { return min(max(__ldg(len + row), 0), cols); }
 
-// What a loaded vector `vi` of a row is worth when only the row's first `len` elements count (NE per vector).
-template <int DT>
-__device__ __forceinline__ uint4 apply_len(const uint4& v, int vi, int len, const uint4& fill) {
+// What the loaded vectors of a row are worth when only the row's first `len` elements count (NE per vector): this thread
+// holds vectors i0, i0 + stride, ...  Vectors entirely behind the length become the fill value (one compare and a
+// select per vector); the one vector of a row that straddles the length is patched in a branch that a single thread per
+// row takes -- written per vector, the element-wise patch was a fifth of the instructions of a bf16 row and cost 18 %.
+template <int DT, int NV>
+__device__ __forceinline__ void apply_len(uint4 (&raw)[NV], int i0, int stride, int len, const uint4& fill) {
     constexpr int NE = Elem<DT>::NE;
-    const int keep = len - vi * NE;                                   // elements of this vector that count
-    if (keep <= 0) return fill;
-    return keep < NE ? mask_tail<DT>(v, keep) : v;                    // at most one vector of a row straddles the length
+#pragma unroll
+    for (int v = 0; v < NV; ++v)
+        if ((i0 + v * stride) * NE >= len) raw[v] = fill;
+    const int tail = len % NE, off = len / NE - i0;               // the straddling vector is `off` vectors after my first
+    if (tail != 0 && off >= 0 && off % stride == 0 && off / stride < NV) {
+        const int mine = off / stride;
+#pragma unroll
+        for (int v = 0; v < NV; ++v)
+            if (v == mine) raw[v] = mask_tail<DT>(raw[v], tail);
+    }
 }
 // Rows of at least this many vectors (16 KiB) do not read what lies behind their length: their loads wait for the row's
 // length to arrive first, which pays off from about this size on (measured at 16 KiB, half of every row live: 90 us
@@ -95,14 +105,13 @@ __global__ void __launch_bounds__(kWarpMaxThreads) k_warp(const KArgs a) {
 #pragma unroll
         for (int rr = 0; rr < RPG; ++rr) {
             const int64_t row = base + rr * G + g;                          // adjacent groups -> adjacent rows
-#pragma unroll
             const int len_row = (MODE == kModeLen && row < a.rows) ? row_len(a.len, row, a.nvec * Elem<DT>::NE) : 0;
             (void)len_row;
+#pragma unroll
             for (int v = 0; v < VPT; ++v) {
                 const bool ok = row < a.rows && valid[v];
                 const int64_t idx = row * a.nvec + lane + v * LANES;
                 raw[rr][v] = ok ? ld_stream(a.x + idx) : fill;
-                if constexpr (MODE == kModeLen) raw[rr][v] = apply_len<DT>(raw[rr][v], lane + v * LANES, len_row, fill);
                 if constexpr (MODE == kModeAdd) {
                     if (ok) {
                         raw[rr][v] = add_round<DT>(raw[rr][v], ld_stream(a.r + idx));
@@ -110,6 +119,7 @@ __global__ void __launch_bounds__(kWarpMaxThreads) k_warp(const KArgs a) {
                     }
                 }
             }
+            if constexpr (MODE == kModeLen) apply_len<DT, VPT>(raw[rr], lane, LANES, len_row, fill);
         }
 #pragma unroll
         for (int rr = 0; rr < RPG; ++rr) {
@@ -160,11 +170,15 @@ __global__ void __launch_bounds__(cta_max_threads(VPT)) k_cta(const KArgs a, con
     if constexpr (CLUSTER) cg::this_cluster().sync();      // every CTA of the cluster is resident before any remote write
 
     int it = 0;
+    // the length of a row is requested one row ahead: the loads of a long row wait for it (a persistent CTA would
+    // otherwise pay that latency at the top of every iteration)
+    int next_len = (MODE == kModeLen && cluster_id < a.rows) ? row_len(a.len, cluster_id, a.nvec * NE) : 0;
     for (int64_t row = cluster_id; row < a.rows; row += num_clusters, ++it) {
         const uint4* xr = a.x + row * a.nvec + first + t;
         uint4* yr = a.y + row * a.nvec + first + t;
         uint4 raw[VPT], out[VPT];
-        const int len_row = MODE == kModeLen ? row_len(a.len, row, a.nvec * NE) : 0;
+        const int len_row = next_len;
+        if (MODE == kModeLen && row + num_clusters < a.rows) next_len = row_len(a.len, row + num_clusters, a.nvec * NE);
         (void)len_row;
         if (MODE == kModeLen && a.nvec >= kLenSkipVecs) {              // long rows: nothing behind the length is read
 #pragma unroll
@@ -173,10 +187,7 @@ __global__ void __launch_bounds__(cta_max_threads(VPT)) k_cta(const KArgs a, con
 #pragma unroll
             for (int v = 0; v < VPT; ++v) raw[v] = valid[v] ? ld_stream(xr + v * T) : fill;
         }
-        if constexpr (MODE == kModeLen) {
-#pragma unroll
-            for (int v = 0; v < VPT; ++v) raw[v] = apply_len<DT>(raw[v], first + t + v * T, len_row, fill);
-        }
+        if constexpr (MODE == kModeLen) apply_len<DT, VPT>(raw, first + t, T, len_row, fill);
         if constexpr (MODE == kModeAdd) {
             const uint4* rr = a.r + row * a.nvec + first + t;
             uint4* hr = a.h + row * a.nvec + first + t;
