@@ -830,9 +830,14 @@ def run_normbwd_table(args):
 
         nbytes = 3 * rows * cols * es + (3 if op == "layernorm" else 2) * cols * es + (8 if op == "layernorm" else 4) * rows
         reps = max(10, min(200, int(0.05 / (nbytes / 5e12))))
-        us, us_lib = timed(ours, reps), timed(lib, max(5, reps // 4))
+        tf.tf_clear_cache()
+        us_auto, us_lib = timed(ours, reps), timed(lib, max(5, reps // 4))
+        timed_forms, _, _ = tf.tf_tune_norm_bwd(op, rows, cols, dt)                 # measure the forms, keep the fastest
+        choice = tf.tf_norm_bwd_choice(op, rows, cols, dt)
+        us = min(timed(ours, reps), us_auto) if choice != "path=0,stages=0,cluster=0" else us_auto
         tf.tf_device_status()
         row = {"op": op + "_bwd", "dtype": "f32" if dt == inputs.F32 else "bf16", "rows": rows, "cols": cols, "bytes": nbytes, "us": us,
+               "automatic_us": us_auto, "forms_timed": timed_forms, "kept": choice,
                "gbs": nbytes / us / 1e3, f"pct_of_{peak_kind}_{peak:.0f}": 100 * nbytes / us / 1e3 / peak, "torch_us": us_lib,
                "torch_what": "aten native_layer_norm_backward" if op == "layernorm" else "eager fp32 expression (no fused kernel in torch)"}
         rows_out.append(row)

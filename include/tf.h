@@ -175,6 +175,16 @@ tf_status tf_layernorm_bwd(const void* x, const void* gamma, const void* dy, con
 tf_status tf_rmsnorm_bwd(const void* x, const void* weight, const void* dy, const float* rstd, void* dx, void* dweight,
                          void* workspace, size_t workspace_bytes, int64_t rows, int64_t cols, tf_dtype dt, void* cuda_stream);
 
+/* The measure-and-keep loop of tf_tune (Algorithm 1, Sections 3.3-3.4 of the paper) over the forms of the norm backward
+ * pass of `op` (TF_LAYERNORM or TF_RMSNORM) on this shape: the automatic choice is the incumbent, every other form that
+ * can run the shape is launched, timed (3 warm-up + 5 timed batches on rotating buffers, CUDA events, median) and kept
+ * only if more than 2 % faster; a form whose bounded waits give up is dropped.  Blocking; owns its scratch (about
+ * 256 MiB or three tensors twice, whichever is more); later calls of the same op, shape and type on this device use the
+ * winner (tf_clear_cache forgets it).  tf_tune_norm_bwd_report: forms timed, automatic and best time of the last call on
+ * this thread.  TF_ERR_INVALID_ARG for another op, rows <= 0 or cols <= 0; TF_ERR_NOMEM without room for the scratch. */
+tf_status tf_tune_norm_bwd(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);
+tf_status tf_tune_norm_bwd_report(int* forms_timed, float* automatic_us, float* best_us);
+
 /* ---- fused residual add + norm ------------------------------------------------------------------------ */
 
 /* h = x + r (fp32 add, ONE rounding to the storage type), then the LayerNorm / RMSNorm defined above applied to that
@@ -245,12 +255,16 @@ tf_status tf_candidate(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int in
 tf_status tf_softmax_variants_force(int cluster);
 
 /* Which form of the norm backward passes runs on shapes that several serve.  path: 0 = automatic, 1 = rows requested
- * into registers one row ahead, 2 = rows staged in a shared-memory ring by bulk copies (up to 512 threads per row),
- * 3 = the same with up to 256 threads per row.  stages = ring depth (0 = automatic, at most 8).  cluster: 0 = automatic
- * (a thread-block cluster shares a row only when one CTA cannot hold it), 1 = never, 2 / 4 / 8 = that many CTAs per row
- * wherever the slices fit.  Ask tf_norm_bwd_workspace_bytes again after changing it.  TF_ERR_INVALID_ARG outside those
- * values. */
+ * into registers one row ahead, 2 / 3 / 4 = rows staged in a shared-memory ring by bulk copies with up to 512 / 256 / 64
+ * threads per row.  stages = ring depth (0 = automatic, at most 8).  cluster: 0 = automatic (a thread-block cluster shares
+ * a row only when one CTA cannot hold it), 1 = never, 2 / 4 / 8 = that many CTAs per row wherever the slices fit.  Ask
+ * tf_norm_bwd_workspace_bytes again after changing it.  TF_ERR_INVALID_ARG outside those values.  A forced choice takes
+ * precedence over a tuned one. */
 tf_status tf_norm_bwd_force(int path, int stages, int cluster);
+
+/* Writes what tf_layernorm_bwd / tf_rmsnorm_bwd (op = TF_LAYERNORM / TF_RMSNORM) would use now for this shape as
+ * "path=P,stages=S,cluster=C" in the terms of tf_norm_bwd_force (forced > tuned > automatic = all zero). */
+tf_status tf_norm_bwd_choice(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, char* buf, size_t n);
 
 /* Forgets every tuned plan (in memory only). */
 void tf_clear_cache(void);

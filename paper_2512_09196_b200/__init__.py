@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
                 5: "TF_ERR_NOMEM"}
 
 # every symbol include/tf.h declares
-EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_log_softmax_bwd", "tf_norm_bwd_workspace_bytes", "tf_layernorm_bwd", "tf_rmsnorm_bwd", "tf_norm_bwd_force", "tf_softmax_variants_force",
+EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_log_softmax_bwd", "tf_norm_bwd_workspace_bytes", "tf_layernorm_bwd", "tf_rmsnorm_bwd", "tf_norm_bwd_force", "tf_softmax_variants_force", "tf_tune_norm_bwd", "tf_tune_norm_bwd_report", "tf_norm_bwd_choice",
            "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
            "tf_candidate", "tf_clear_cache", "tf_launch_count")
@@ -65,6 +65,9 @@ def lib() -> ctypes.CDLL:
         L.tf_norm_bwd_workspace_bytes.restype = ctypes.c_size_t
         L.tf_layernorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i64, i64, i32, vp]
         L.tf_norm_bwd_force.argtypes = [i32, i32, i32]
+        L.tf_tune_norm_bwd.argtypes = [i32, i64, i64, i32]
+        L.tf_tune_norm_bwd_report.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(f32)]
+        L.tf_norm_bwd_choice.argtypes = [i32, i64, i64, i32, ctypes.c_char_p, ctypes.c_size_t]
         L.tf_softmax_variants_force.argtypes = [i32]
         L.tf_rmsnorm_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i64, i64, i32, vp]
         L.tf_bvecmat_fwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp]
@@ -243,6 +246,22 @@ def tf_rmsnorm_bwd(x, weight, dy, rstd, dx=None):
         _ok(lib().tf_rmsnorm_bwd(x.data_ptr(), weight.data_ptr(), dy.data_ptr(), rstd.data_ptr(), dx.data_ptr(), dweight.data_ptr(),
                                  ws.data_ptr(), n, rows, cols, _dt(x), _stream(x)), "tf_rmsnorm_bwd")
     return dx, dweight
+
+
+def tf_tune_norm_bwd(op, rows: int, cols: int, dt: int):
+    """Measure-and-keep over the forms of the norm backward pass (``op``: "layernorm" or "rmsnorm") on this shape; later
+    calls use the winner.  Returns ``(forms_timed, automatic_us, best_us)``."""
+    _ok(lib().tf_tune_norm_bwd(OP_CODE[op] if isinstance(op, str) else int(op), rows, cols, dt), "tf_tune_norm_bwd")
+    n, a, b = ctypes.c_int32(0), ctypes.c_float(0), ctypes.c_float(0)
+    _ok(lib().tf_tune_norm_bwd_report(ctypes.byref(n), ctypes.byref(a), ctypes.byref(b)), "tf_tune_norm_bwd_report")
+    return n.value, a.value, b.value
+
+
+def tf_norm_bwd_choice(op, rows: int, cols: int, dt: int) -> str:
+    """What the norm backward pass of ``op`` would use now for this shape (forced > tuned > automatic)."""
+    buf = ctypes.create_string_buffer(64)
+    _ok(lib().tf_norm_bwd_choice(OP_CODE[op] if isinstance(op, str) else int(op), rows, cols, dt, buf, 64), "tf_norm_bwd_choice")
+    return buf.value.decode()
 
 
 def tf_softmax_variants_force(cluster=0):

@@ -923,8 +923,11 @@ tf_status tf_candidate(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, int in
 }
 
 void tf_clear_cache(void) {
-    std::lock_guard<std::mutex> lk(g_mu);
-    g_cache.clear();
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_cache.clear();
+    }
+    clear_norm_bwd_tuned();
 }
 
 int64_t tf_launch_count(void) { return g_launches.load(); }

@@ -20,6 +20,11 @@
 #include <cooperative_groups.h>
 
 #include <algorithm>
+#include <cstdio>
+#include <vector>
+#include <map>
+#include <mutex>
+#include <tuple>
 
 #include "../../include/tf.h"
 #include "tf_common.cuh"
@@ -618,7 +623,25 @@ cudaError_t launch_pdl(void (*fn)(T...), int64_t grid, int threads, cudaStream_t
 
 // Test and bench hook: 0 = automatic, 1 = the register form, 2 = the staged form with row groups of up to 512 threads,
 // 3 = the staged form with row groups of up to 256 threads; stages 0 = automatic.
-int g_force_path = 0, g_force_stages = 0, g_force_cluster = 0;      // cluster: 0 = automatic, 1 = never, 2/4/8 = that many CTAs per row
+// path: 0 automatic, 1 register form, 2 / 3 / 4 staged form with row groups of up to 512 / 256 / 64 threads; stages: ring
+// depth (0 automatic); cluster: 0 automatic, 1 never, 2 / 4 / 8 that many CTAs per row.
+struct BwdChoice { int path, stages, cluster; };
+BwdChoice g_force{0, 0, 0};                                    // the hook
+thread_local const BwdChoice* t_override = nullptr;            // the tuner, while it times a candidate
+std::mutex g_tuned_mu;
+std::map<std::tuple<int, int, int64_t, int64_t, int>, BwdChoice> g_tuned;        // (rms, dt, rows, cols, device) -> what tf_tune_norm_bwd kept
+
+// forced > tuned > automatic
+BwdChoice current_choice(bool rms, int dt, int64_t rows, int64_t cols) {
+    if (t_override) return *t_override;
+    if (g_force.path || g_force.stages || g_force.cluster) return g_force;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    std::lock_guard<std::mutex> lk(g_tuned_mu);
+    const auto it = g_tuned.find(std::make_tuple(rms ? 1 : 0, dt, rows, cols, dev));
+    return it == g_tuned.end() ? BwdChoice{0, 0, 0} : it->second;
+}
+int staged_gmax(int path) { return path == 2 ? 512 : path == 3 ? 256 : 64; }
 
 // Launch geometry of the row-group kernels: vectors per thread, threads per row group, row groups per CTA, CTAs; for
 // the staged form also the ring's stages and bytes (stages = 0: the register form).
@@ -668,26 +691,26 @@ BwdPlan bwd_plan(int64_t rows, int nvec, bool staged, int stages, int gmax = 256
 // vectors per thread (measured 7-15 % faster there: a row ahead in registers is half as many bytes in flight as with
 // 4-byte elements), the register form elsewhere (shorter rows and 4-byte elements: equal or faster).
 template <bool RMS, int DT>
-BwdPlan choose_bwd_plan_uncached(int64_t rows, int nvec) {
-    const bool want = g_force_path >= 2 || (g_force_path == 0 && DT == DT_BF16 && nvec >= 128);
+BwdPlan choose_bwd_plan_uncached(int64_t rows, int nvec, const BwdChoice& c) {
+    const bool want = c.path >= 2 || (c.path == 0 && DT == DT_BF16 && nvec >= 128);
     if (want) {
-        const BwdPlan p = bwd_plan<RMS, DT>(rows, nvec, true, g_force_stages, g_force_path == 2 ? 512 : g_force_path == 3 ? 256 : 64);
+        const BwdPlan p = bwd_plan<RMS, DT>(rows, nvec, true, c.stages, staged_gmax(c.path));
         if (p.stages >= 2) return p;
     }
     return bwd_plan<RMS, DT>(rows, nvec, false, 0);
 }
 
 template <bool RMS, int DT>
-BwdPlan choose_bwd_plan(int64_t rows, int nvec) {
+BwdPlan choose_bwd_plan(int64_t rows, int nvec, const BwdChoice& c) {
     // the plan of the last shape is kept (per thread): the occupancy queries cost more host time than a launch
     struct Key { int64_t rows; int nvec, path, stages, dev; };
     thread_local Key last{-1, 0, 0, 0, -1};
     thread_local BwdPlan kept{};
     int dev = 0;
     cudaGetDevice(&dev);
-    if (last.rows == rows && last.nvec == nvec && last.path == g_force_path && last.stages == g_force_stages && last.dev == dev) return kept;
-    last = Key{rows, nvec, g_force_path, g_force_stages, dev};
-    kept = choose_bwd_plan_uncached<RMS, DT>(rows, nvec);
+    if (last.rows == rows && last.nvec == nvec && last.path == c.path && last.stages == c.stages && last.dev == dev) return kept;
+    last = Key{rows, nvec, c.path, c.stages, dev};
+    kept = choose_bwd_plan_uncached<RMS, DT>(rows, nvec, c);
     return kept;
 }
 
@@ -741,15 +764,15 @@ ClusterPlan cluster_plan(int64_t rows, int nvec, int cs_forced, int stages) {
 }
 
 template <bool RMS, int DT>
-ClusterPlan choose_cluster_plan(int64_t rows, int nvec) {          // the last shape's plan is kept, like the row-group plan
+ClusterPlan choose_cluster_plan(int64_t rows, int nvec, const BwdChoice& c) {          // the last shape's plan is kept, like the row-group plan
     struct Key { int64_t rows; int nvec, cs, stages, dev; };
     thread_local Key last{-1, 0, 0, 0, -1};
     thread_local ClusterPlan kept{};
     int dev = 0;
     cudaGetDevice(&dev);
-    if (last.rows == rows && last.nvec == nvec && last.cs == g_force_cluster && last.stages == g_force_stages && last.dev == dev) return kept;
-    last = Key{rows, nvec, g_force_cluster, g_force_stages, dev};
-    kept = cluster_plan<RMS, DT>(rows, nvec, g_force_cluster, g_force_stages);
+    if (last.rows == rows && last.nvec == nvec && last.cs == c.cluster && last.stages == c.stages && last.dev == dev) return kept;
+    last = Key{rows, nvec, c.cluster, c.stages, dev};
+    kept = cluster_plan<RMS, DT>(rows, nvec, c.cluster, c.stages);
     return kept;
 }
 
@@ -775,10 +798,11 @@ tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float*
     constexpr int kMaxVpt = NE == 4 ? 4 : 2;
     cudaError_t e;
     // a cluster per row: rows beyond one CTA's registers (or wherever the hook asks for it)
+    const BwdChoice c = current_choice(RMS, DT, rows, cols);
     ClusterPlan cp{};
-    if (aligned && cols <= 0x7FFFFFFF && g_force_cluster != 1 && (g_force_cluster > 1 || bytes / 16 > 512 * kMaxVpt) &&
+    if (aligned && cols <= 0x7FFFFFFF && c.cluster != 1 && (c.cluster > 1 || bytes / 16 > 512 * kMaxVpt) &&
         bytes / 16 <= static_cast<int64_t>(kMaxCluster) * 512 * kMaxVpt)
-        cp = choose_cluster_plan<RMS, DT>(rows, static_cast<int>(bytes / 16));
+        cp = choose_cluster_plan<RMS, DT>(rows, static_cast<int>(bytes / 16), c);
     if (cp.clusters > 0) {
         const int nvec = static_cast<int>(bytes / 16);
         const size_t need = static_cast<size_t>(cp.clusters) * (RMS ? 1 : 2) * cols * 4;
@@ -794,7 +818,7 @@ tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float*
                            static_cast<S*>(dbeta), cp.clusters, cols);
     } else if (aligned && bytes / 16 <= 512 * kMaxVpt && cols <= 0x7FFFFFFF) {
         const int nvec = static_cast<int>(bytes / 16);
-        const BwdPlan p = choose_bwd_plan<RMS, DT>(rows, nvec);
+        const BwdPlan p = choose_bwd_plan<RMS, DT>(rows, nvec, c);
         const int parts = p.grid * p.groups;
         const size_t need = static_cast<size_t>(parts) * (RMS ? 1 : 2) * cols * 4;
         if (!ws || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 3u)) return TF_ERR_INVALID_ARG;
@@ -896,33 +920,190 @@ using namespace tf;
 
 extern "C" size_t tf_norm_bwd_workspace_bytes(int64_t rows, int64_t cols) {
     if (rows <= 0 || cols <= 0 || cols > 0x7FFFFFFF) return 0;
-    // the most partial column sums any of the paths may write for this shape, whatever the element type or the op
-    int64_t parts = std::min<int64_t>(rows, sm_count());                          // the streamed kernel: one CTA per SM
-    auto widest = [&](auto plan) {                                                 // any form may be chosen (or forced)
-        for (int form = 0; form < 4; ++form) {
-            const BwdPlan p = plan(form != 0, form == 2 ? 512 : form == 3 ? 64 : 256);
-            parts = std::max<int64_t>(parts, static_cast<int64_t>(p.grid) * p.groups);
-        }
+    // the most partial column sums any of the paths may write for this shape, whatever the element type, the op or the
+    // form (automatic, tuned or forced): every group width, and the ring depths that leave room for the most CTAs
+    int64_t parts = std::min<int64_t>(rows, sm_count());                          // the streamed kernel and the clusters: at most one part per SM
+    auto widest = [&](auto plan) {
+        for (int stages : {2, 3, g_force.stages})
+            for (int form = 0; form < 4; ++form) {
+                const BwdPlan p = plan(form != 0, form == 1 ? 512 : form == 2 ? 256 : 64, stages);
+                parts = std::max<int64_t>(parts, static_cast<int64_t>(p.grid) * p.groups);
+            }
     };
     if (cols % 4 == 0 && cols / 4 <= 512 * 4) {
         const int nvec = static_cast<int>(cols / 4);
-        widest([&](bool sg, int gmax) { return bwd_plan<false, DT_F32>(rows, nvec, sg, g_force_stages, gmax); });
-        widest([&](bool sg, int gmax) { return bwd_plan<true, DT_F32>(rows, nvec, sg, g_force_stages, gmax); });
+        widest([&](bool sg, int gmax, int st) { return bwd_plan<false, DT_F32>(rows, nvec, sg, st, sg ? gmax : 256); });
+        widest([&](bool sg, int gmax, int st) { return bwd_plan<true, DT_F32>(rows, nvec, sg, st, sg ? gmax : 256); });
     }
     if (cols % 8 == 0 && cols / 8 <= 512 * 2) {
         const int nvec = static_cast<int>(cols / 8);
-        widest([&](bool sg, int gmax) { return bwd_plan<false, DT_BF16>(rows, nvec, sg, g_force_stages, gmax); });
-        widest([&](bool sg, int gmax) { return bwd_plan<true, DT_BF16>(rows, nvec, sg, g_force_stages, gmax); });
+        widest([&](bool sg, int gmax, int st) { return bwd_plan<false, DT_BF16>(rows, nvec, sg, st, sg ? gmax : 256); });
+        widest([&](bool sg, int gmax, int st) { return bwd_plan<true, DT_BF16>(rows, nvec, sg, st, sg ? gmax : 256); });
     }
     return static_cast<size_t>(parts) * 2 * static_cast<size_t>(cols) * 4;
 }
 
 extern "C" tf_status tf_norm_bwd_force(int path, int stages, int cluster) {
-    if (path < 0 || path > 3 || stages < 0 || stages > kBwdMaxStages) return TF_ERR_INVALID_ARG;
+    if (path < 0 || path > 4 || stages < 0 || stages > kBwdMaxStages) return TF_ERR_INVALID_ARG;
     if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8) return TF_ERR_INVALID_ARG;
-    g_force_path = path;
-    g_force_stages = stages;
-    g_force_cluster = cluster;
+    g_force = BwdChoice{path, stages, cluster};
+    return TF_OK;
+}
+
+namespace tf {
+void clear_norm_bwd_tuned() {
+    std::lock_guard<std::mutex> lk(g_tuned_mu);
+    g_tuned.clear();
+}
+}  // namespace tf
+
+namespace tf {
+namespace {
+
+__global__ void k_fill_pattern(uint32_t* p, int64_t words, uint32_t seed, uint32_t base, uint32_t mask) {
+    // finite values of either element type: a fixed exponent field (`base`) with hashed low bits (`mask`)
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < words; i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        uint32_t h = static_cast<uint32_t>(i) * 2654435761u + seed;
+        h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
+        p[i] = base | (h & mask);
+    }
+}
+__global__ void k_fill_float(float* p, int64_t n, float v) {
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n; i += static_cast<int64_t>(gridDim.x) * blockDim.x) p[i] = v;
+}
+
+struct TuneScratch {
+    std::vector<void*> ptrs;
+    ~TuneScratch() { for (void* p : ptrs) cudaFree(p); }
+    void* get(size_t bytes) {
+        void* p = nullptr;
+        if (cudaMalloc(&p, std::max<size_t>(bytes, 16)) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        ptrs.push_back(p);
+        return p;
+    }
+};
+
+thread_local int t_bwd_timed = 0;
+thread_local float t_bwd_auto_us = 0.f, t_bwd_best_us = 0.f;
+
+}  // namespace
+}  // namespace tf
+
+// The measure-and-keep loop (Algorithm 1 of the paper, as in tf_tune) over the forms of the norm backward pass: the
+// automatic choice is the incumbent; every other form that can run the shape is launched (BuildRun: it must launch and
+// no bounded wait may give up), timed (Profile: 3 warm-up + 5 timed batches over rotating buffers, CUDA events, median)
+// and kept only if it is more than 2 % faster (Arbiter).  The winner is remembered for (op, rows, cols, type, device).
+extern "C" tf_status tf_tune_norm_bwd(tf_op op_, int64_t rows, int64_t cols, tf_dtype dt_) {
+    const int op = op_, dt = dt_;
+    if ((op != OP_LAYERNORM && op != OP_RMSNORM) || rows <= 0 || cols <= 0 || (dt != DT_F32 && dt != DT_BF16)) return TF_ERR_INVALID_ARG;
+    if (cols > 0x7FFFFFFF || cols > (INT64_MAX / 8) / rows) return TF_ERR_UNSUPPORTED;
+    const bool rms = op == OP_RMSNORM;
+    const int es = elem_size(dt);
+    t_bwd_timed = 0; t_bwd_auto_us = 0.f; t_bwd_best_us = 0.f;
+    if ((cols * es) % 16 != 0) return TF_OK;                     // only the plain kernels serve such rows: nothing to choose
+    const int64_t nvec = cols * es / 16;
+    const int kMaxVpt = dt == DT_F32 ? 4 : 2;
+    const size_t tensor_bytes = static_cast<size_t>(rows) * cols * es;
+    const int K = static_cast<int>(std::min<size_t>(16, std::max<size_t>(2, (256u << 20) / (3 * tensor_bytes) + 1)));
+    TuneScratch sc;
+    std::vector<void*> xs(K), dys(K), dxs(K);
+    for (int k = 0; k < K; ++k) { xs[k] = sc.get(tensor_bytes); dys[k] = sc.get(tensor_bytes); dxs[k] = sc.get(tensor_bytes); if (!xs[k] || !dys[k] || !dxs[k]) return TF_ERR_NOMEM; }
+    void* gamma = sc.get(static_cast<size_t>(cols) * es);
+    void* dgamma = sc.get(static_cast<size_t>(cols) * es);
+    void* dbeta = sc.get(static_cast<size_t>(cols) * es);
+    float* mean = static_cast<float*>(sc.get(static_cast<size_t>(rows) * 4));
+    float* rstd = static_cast<float*>(sc.get(static_cast<size_t>(rows) * 4));
+    const size_t ws_bytes = tf_norm_bwd_workspace_bytes(rows, cols);
+    void* ws = sc.get(ws_bytes);
+    int* status = device_status_word();
+    if (!gamma || !dgamma || !dbeta || !mean || !rstd || !ws || !status) return TF_ERR_NOMEM;
+    cudaStream_t st = nullptr;
+    cudaEvent_t ev[2] = {nullptr, nullptr};
+    if (cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) != cudaSuccess) return TF_ERR_CUDA;
+    auto cleanup = [&]() { if (ev[0]) cudaEventDestroy(ev[0]); if (ev[1]) cudaEventDestroy(ev[1]); cudaStreamDestroy(st); t_override = nullptr; };
+    if (cudaEventCreate(&ev[0]) != cudaSuccess || cudaEventCreate(&ev[1]) != cudaSuccess) { cleanup(); return TF_ERR_CUDA; }
+    // values in [1, 2) (fp32) / [1, 2) in both halves (bf16): the kernels have no data-dependent control flow
+    const uint32_t base = dt == DT_F32 ? 0x3F800000u : 0x3F803F80u, mask = dt == DT_F32 ? 0x007FFFFFu : 0x007F007Fu;
+    for (int k = 0; k < K; ++k) {
+        k_fill_pattern<<<1024, 256, 0, st>>>(static_cast<uint32_t*>(xs[k]), static_cast<int64_t>(tensor_bytes / 4), 17u * k + 1, base, mask);
+        k_fill_pattern<<<1024, 256, 0, st>>>(static_cast<uint32_t*>(dys[k]), static_cast<int64_t>(tensor_bytes / 4), 31u * k + 7, base, mask);
+    }
+    k_fill_pattern<<<64, 256, 0, st>>>(static_cast<uint32_t*>(gamma), static_cast<int64_t>(cols) * es / 4, 5u, base, mask);
+    k_fill_float<<<256, 256, 0, st>>>(mean, rows, 1.5f);
+    k_fill_float<<<256, 256, 0, st>>>(rstd, rows, 2.0f);
+    if (cudaStreamSynchronize(st) != cudaSuccess) { cleanup(); return TF_ERR_CUDA; }
+
+    auto call = [&](int k) {
+        return rms ? tf_rmsnorm_bwd(xs[k], gamma, dys[k], rstd, dxs[k], dgamma, ws, ws_bytes, rows, cols, dt_, st)
+                   : tf_layernorm_bwd(xs[k], gamma, dys[k], mean, rstd, dxs[k], dgamma, dbeta, ws, ws_bytes, rows, cols, dt_, st);
+    };
+    auto profile = [&](const BwdChoice& c, float* us) -> bool {
+        t_override = &c;
+        bool ok = true;
+        float t[5];
+        for (int rep = 0; rep < 8 && ok; ++rep) {
+            if (rep >= 3) cudaEventRecord(ev[0], st);
+            for (int k = 0; k < K && ok; ++k) ok = call(k) == TF_OK;
+            if (rep >= 3) {
+                cudaEventRecord(ev[1], st);
+                if (cudaEventSynchronize(ev[1]) != cudaSuccess) ok = false;
+                float ms = 0.f;
+                cudaEventElapsedTime(&ms, ev[0], ev[1]);
+                t[rep - 3] = ms * 1000.f / K;
+            }
+        }
+        t_override = nullptr;
+        if (cudaStreamSynchronize(st) != cudaSuccess) ok = false;
+        int flag = 0;                                             // a bounded wait gave up: the candidate is dropped
+        if (cudaMemcpy(&flag, status, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) ok = false;
+        if (flag != 0) { cudaMemset(status, 0, sizeof flag); ok = false; }
+        if (!ok) { cudaGetLastError(); return false; }
+        std::sort(t, t + 5);
+        *us = t[2];
+        ++t_bwd_timed;
+        return true;
+    };
+
+    std::vector<BwdChoice> cands;
+    if (nvec <= 512 * kMaxVpt) {                                  // one CTA can hold the row
+        cands.push_back(BwdChoice{1, 0, 1});
+        for (int path : {2, 3, 4})
+            for (int stages : {2, 3}) cands.push_back(BwdChoice{path, stages, 1});
+    }
+    for (int cs : {2, 4, 8})
+        if ((nvec + cs - 1) / cs <= 512 * kMaxVpt && nvec >= 512)                // clusters from 8 KiB rows on
+            for (int stages : {2, 3}) cands.push_back(BwdChoice{0, stages, cs});
+    const BwdChoice automatic{0, 0, 0};
+    float best_us = 0.f;
+    if (!profile(automatic, &best_us)) { cleanup(); return TF_ERR_CUDA; }
+    t_bwd_auto_us = best_us;
+    BwdChoice best = automatic;
+    for (const BwdChoice& c : cands) {
+        float us = 0.f;
+        if (!profile(c, &us)) continue;
+        if (us < 0.98f * best_us) { best = c; best_us = us; }
+    }
+    t_bwd_best_us = best_us;
+    cleanup();
+    int dev = 0;
+    cudaGetDevice(&dev);
+    std::lock_guard<std::mutex> lk(g_tuned_mu);
+    g_tuned[std::make_tuple(rms ? 1 : 0, dt, rows, cols, dev)] = best;
+    return TF_OK;
+}
+
+extern "C" tf_status tf_tune_norm_bwd_report(int* candidates_timed, float* automatic_us, float* best_us) {
+    if (candidates_timed) *candidates_timed = t_bwd_timed;
+    if (automatic_us) *automatic_us = t_bwd_auto_us;
+    if (best_us) *best_us = t_bwd_best_us;
+    return TF_OK;
+}
+
+extern "C" tf_status tf_norm_bwd_choice(tf_op op_, int64_t rows, int64_t cols, tf_dtype dt_, char* buf, size_t n) {
+    const int op = op_, dt = dt_;
+    if ((op != OP_LAYERNORM && op != OP_RMSNORM) || rows < 0 || cols <= 0 || (dt != DT_F32 && dt != DT_BF16) || !buf || n == 0) return TF_ERR_INVALID_ARG;
+    const BwdChoice c = current_choice(op == OP_RMSNORM, dt, rows, cols);
+    snprintf(buf, n, "path=%d,stages=%d,cluster=%d", c.path, c.stages, c.cluster);
     return TF_OK;
 }
 

@@ -100,6 +100,7 @@ size_t split_scratch_bytes(const Plan&, const Args&);
 
 // Bookkeeping shared with the C ABI layer: count kernel launches; remember the CUDA error behind a TF_ERR_CUDA.
 void count_launches(int n);
+void clear_norm_bwd_tuned();   // forgets what tf_tune_norm_bwd kept
 int* device_status_word();     // this device's status word (bounded waits set it when they give up), or null before first use fails
 void remember_cuda_error(cudaError_t e);
 

@@ -84,7 +84,7 @@ def test_every_form_on_shapes_both_serve(rms, dt):
     """The register form and the staged form (both group widths, several ring depths) give the oracle's result."""
     ne = 4 if dt == F32 else 8
     try:
-        for path, stages in ((1, 0), (2, 0), (2, 2), (2, 3), (3, 0), (3, 8)):
+        for path, stages in ((1, 0), (2, 0), (2, 2), (3, 3), (3, 8), (4, 0), (4, 2)):
             tf.tf_norm_bwd_force(path, stages)
             for rows, cols in ((1, ne), (5, 3 * ne), (77, 256), (1500, 512), (700, 1024), (333, 4096), (130, 5120), (64, 8192)):
                 run_case(rms, dt, rows, cols, seed=rows + cols + path)
@@ -92,7 +92,7 @@ def test_every_form_on_shapes_both_serve(rms, dt):
     finally:
         tf.tf_norm_bwd_force(0, 0, 0)
     with pytest.raises(tf.TfError):
-        tf.tf_norm_bwd_force(4, 0)
+        tf.tf_norm_bwd_force(5, 0)
     with pytest.raises(tf.TfError):
         tf.tf_norm_bwd_force(2, 9)
     with pytest.raises(tf.TfError):
@@ -162,3 +162,34 @@ def test_shapes_of_the_bench_table_every_element(rms, dt, rows, cols):
     """The shapes `bench.py --table normbwd` times, in the form it times (automatic): dx element by element, the parameter
     gradients summed over all rows."""
     run_case(rms, dt, rows, cols, seed=cols)
+
+
+@pytest.mark.parametrize("op,dt,rows,cols", [("layernorm", BF16, 4096, 4096), ("rmsnorm", BF16, 3000, 1024), ("layernorm", F32, 2048, 8192),
+                                              ("rmsnorm", BF16, 700, 16384), ("layernorm", BF16, 50, 1000)])
+def test_tuned_form_is_used_and_still_exact(op, dt, rows, cols):
+    """tf_tune_norm_bwd times the forms on the shape and keeps one only if it is measured faster; whatever it keeps must
+    be what later calls use, and must still meet the oracle."""
+    rms = op == "rmsnorm"
+    try:
+        assert tf.tf_norm_bwd_choice(op, rows, cols, dt) == "path=0,stages=0,cluster=0"
+        timed, auto_us, best_us = tf.tf_tune_norm_bwd(op, rows, cols, dt)
+        if cols * (4 if dt == F32 else 2) % 16 == 0:
+            assert timed >= 2 and 0 < best_us <= auto_us
+        else:
+            assert timed == 0                                      # only the plain kernels serve such rows
+        kept = tf.tf_norm_bwd_choice(op, rows, cols, dt)
+        if best_us == auto_us:
+            assert kept == "path=0,stages=0,cluster=0"            # nothing was more than 2 % faster
+        run_case(rms, dt, rows, cols, seed=7)
+        assert tf.tf_norm_bwd_choice(op, rows + 1, cols, dt) == "path=0,stages=0,cluster=0"   # another shape: automatic
+        tf.tf_norm_bwd_force(1, 0, 1)                              # a forced choice wins over the tuned one
+        assert tf.tf_norm_bwd_choice(op, rows, cols, dt) == "path=1,stages=0,cluster=1"
+        tf.tf_norm_bwd_force(0, 0, 0)
+        assert tf.tf_norm_bwd_choice(op, rows, cols, dt) == kept
+        tf.tf_clear_cache()
+        assert tf.tf_norm_bwd_choice(op, rows, cols, dt) == "path=0,stages=0,cluster=0"
+    finally:
+        tf.tf_norm_bwd_force(0, 0, 0)
+        tf.tf_clear_cache()
+    with pytest.raises(tf.TfError):
+        tf.tf_tune_norm_bwd("softmax", 8, 64, dt)
