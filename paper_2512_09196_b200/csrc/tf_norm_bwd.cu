@@ -738,9 +738,13 @@ ClusterPlan cluster_plan(int64_t rows, int nvec, int cs_forced, int stages) {
     constexpr int kMaxVpt = Elem<DT>::NE == 4 ? 4 : 2;
     ClusterPlan p{};
     int cs = cs_forced > 1 ? cs_forced : 2;
-    // the fewest CTAs whose slices are at most 16 KiB (measured: the exchange costs about as much per row whatever the
-    // slice, so large slices amortise it; beyond 16 KiB a CTA has too many registers for two of them to share an SM)
-    while (cs_forced <= 1 && cs < kMaxCluster && (nvec + cs - 1) / cs > 1024) cs *= 2;
+    // the fewest CTAs whose slices are at most 1024 vectors (2-byte elements) or 1536 (4-byte): the exchange costs about
+    // as much per row whatever the slice, so large slices amortise it, up to what leaves a CTA enough registers; and
+    // rather four CTAs with the largest slices than eight (clusters of eight leave SMs of a GPC unused).  Read off what
+    // tf_tune_norm_bwd keeps on rows of 12-64 Ki columns.
+    const int slice_cap = Elem<DT>::NE == 4 ? 1536 : 1024;
+    while (cs_forced <= 1 && cs < kMaxCluster && (nvec + cs - 1) / cs > slice_cap) cs *= 2;
+    if (cs_forced <= 1 && cs == 8 && (nvec + 3) / 4 <= 512 * kMaxVpt) cs = 4;
     const int per = (nvec + cs - 1) / cs;
     if (per > 512 * kMaxVpt) return p;                                                                // clusters = 0: not available
     p.cs = cs;
@@ -749,7 +753,7 @@ ClusterPlan cluster_plan(int64_t rows, int nvec, int cs_forced, int stages) {
     p.threads = std::max(32, ((per + p.vpt - 1) / p.vpt + 31) / 32 * 32);
     p.full = nvec % cs == 0 && per == p.threads * p.vpt;
     const size_t stage = static_cast<size_t>(2) * per * 16;
-    p.stages = stages > 0 ? stages : static_cast<int>(std::min<size_t>(3, (216 * 1024) / stage));
+    p.stages = stages > 0 ? stages : 2;                           // two stages: what the tuner keeps for every cluster shape
     p.smem = stage * p.stages;
     if (p.stages < 2 || p.stages > kBwdMaxStages || p.smem > 216 * 1024) return p;
     const void* fn = p.vpt == 1 ? cluster_fn<RMS, DT, 1>(p.full) : p.vpt == 2 ? cluster_fn<RMS, DT, 2>(p.full) : cluster_fn<RMS, DT, kMaxVpt>(p.full);
