@@ -124,7 +124,8 @@ tf_status tf_sin_fwd(const void* x, void* y, int64_t n, tf_dtype dt, int threads
 
 /* Row r is normalised over its first len[r] entries: y[r, j] = softmax(x[r, 0:len[r]])_j for j < len[r] and +0 for
  * j >= len[r]; the contents of x[r, j >= len[r]] are ignored (anything, NaN included; x must still be a whole
- * [rows, cols] allocation) and for rows of 16 KiB and more they are not read at all; len[r] = 0 gives an all +0 row,
+ * [rows, cols] allocation) and for 2-byte rows of 4 KiB and more and any rows of 16 KiB and more they are not read at
+ * all; len[r] = 0 gives an all +0 row,
  * values outside [0, cols] are clamped.  Equal, bit for bit where the same plan runs, to tf_softmax_fwd on an x whose
  * tails hold -inf.  The paper has no counterpart (its kernels take their masks in the data).
  * x, y: [rows, cols] row-major device memory (y may alias x); len: int32 [rows], device memory; cols <= 2^31 - 1.

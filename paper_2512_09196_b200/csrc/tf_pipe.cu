@@ -32,6 +32,7 @@ bool pipe_geometry(const Plan& p, const Args& a, const DeviceInfo& d, PipeGeomet
     const int rpp = ut / p.lanes * std::max(1, p.rpg);       // rows a unit takes per pass
     const int units = p.threads / ut;
     int64_t rows = std::max<int64_t>(rpp, p.chunk / row_bytes / rpp * rpp);
+    if (a.len) rows = rpp;                                    // length-aware: one row per tile
     const int64_t rows_per_unit = (a.rows + static_cast<int64_t>(units) * d.sms - 1) / (static_cast<int64_t>(units) * d.sms);
     rows = std::min<int64_t>(rows, std::max<int64_t>(rpp, (rows_per_unit + rpp - 1) / rpp * rpp));   // small problems: spread over all SMs
     const size_t param_bytes = a.op == OP_SOFTMAX ? 0 : static_cast<size_t>(row_bytes) * (a.op == OP_LAYERNORM ? 2 : 1);
@@ -47,7 +48,9 @@ bool pipe_geometry(const Plan& p, const Args& a, const DeviceInfo& d, PipeGeomet
 bool supports_pipe(const Plan& p, const Args& a, const DeviceInfo& d) {
     if (!vector_ok(a) || p.lanes < 8 || p.threads < 32 || p.threads > kPipeMaxThreads || p.threads % 32) return false;
     const int ut = p.lanes < 32 ? 32 : p.lanes;
-    if (p.threads % ut || p.rpg < 1 || !pipe_fn(a.op, a.dt, p.lanes, p.vpt, p.rpg, row_fills(p, a))) return false;
+    if (a.len) {                                              // softmax with lengths: a row per tile, a row per pass
+        if (a.op != OP_SOFTMAX || p.lanes < 32 || p.rpg != 1 || p.threads % ut || !pipe::pipe_fn_softmax_len(a.dt, p.lanes, p.vpt)) return false;
+    } else if (p.threads % ut || p.rpg < 1 || !pipe_fn(a.op, a.dt, p.lanes, p.vpt, p.rpg, row_fills(p, a))) return false;
     const int units = p.threads / ut;
     if (p.stages < 1 || units * p.stages > kPipeMaxBarriers || p.persist < 0 || p.persist > 8 || p.chunk < 16) return false;
     if (ut > 32 && units > 15) return false;                  // one named barrier per multi-warp unit
@@ -58,7 +61,7 @@ bool supports_pipe(const Plan& p, const Args& a, const DeviceInfo& d) {
 }
 
 cudaError_t launch_pipe(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
-    PipeFn fn = pipe_fn(a.op, a.dt, p.lanes, p.vpt, p.rpg, row_fills(p, a));
+    PipeFn fn = a.len ? pipe::pipe_fn_softmax_len(a.dt, p.lanes, p.vpt) : pipe_fn(a.op, a.dt, p.lanes, p.vpt, p.rpg, row_fills(p, a));
     PipeGeometry g;
     if (!fn || !pipe_geometry(p, a, d, g)) return cudaErrorInvalidValue;
     cudaError_t e = ensure_max_smem(reinterpret_cast<const void*>(fn), d);
@@ -76,7 +79,7 @@ cudaError_t launch_pipe(const Plan& p, const Args& a, const DeviceInfo& d, cudaS
     k.y = static_cast<uint4*>(a.y); k.mean = a.mean; k.rstd = a.rstd; k.rows = a.rows;
     k.nvec = static_cast<int>(a.cols * elem_size(a.dt) / 16);
     k.n = static_cast<float>(a.cols); k.eps = a.eps;
-    k.tile_rows = g.tile_rows; k.nstage = p.stages; k.status = a.status;
+    k.tile_rows = g.tile_rows; k.nstage = p.stages; k.status = a.status; k.len = a.len;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid));
     cfg.blockDim = dim3(p.threads);

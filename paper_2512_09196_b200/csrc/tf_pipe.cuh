@@ -40,6 +40,7 @@ struct PArgs {
     int tile_rows;     // rows per stage of a unit
     int nstage;        // stages per unit
     int* status;
+    const int* len;    // LEN builds: valid elements per row (softmax over x[r, 0:len[r]], zeros behind)
 };
 
 constexpr int kPipeMaxBarriers = 128;                    // units x stages per CTA
@@ -55,7 +56,11 @@ constexpr int kPipeMaxThreads = 512;
 
 // RPG: rows of the same columns a thread carries through one pass (parameters, barriers and shuffle latency are
 // shared by them).  FULL: the row fills LANES x VPL vectors exactly, so no vector needs a predicate.
-template <int OP, int DT, int LANES, int VPL, int RPG, bool FULL>
+// LEN (softmax, one row per tile): only the live part of a row is copied -- the bulk copy of a tile is as long as its
+// row's length says, so bytes behind the length never leave HBM and the bytes in flight are all live; the length of a
+// tile travels with its stage (written by the issuing lane before it arms the barrier) and the issuing lane requests
+// the length of the tile after next an iteration early, so that no copy waits for a length.
+template <int OP, int DT, int LANES, int VPL, int RPG, bool FULL, bool LEN = false>
 __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     using E = Elem<DT>;
     constexpr int NE = E::NE;
@@ -66,6 +71,7 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ __align__(8) uint64_t full_bar[kPipeMaxBarriers];
     __shared__ float xch[W > 1 ? (kPipeMaxThreads / UT) * 2 * RPG * W * 2 : 1];     // [unit][parity][row][warp][2]
+    __shared__ int tile_len[LEN ? kPipeMaxBarriers : 1];                            // LEN: the length of the row in each stage
 
     const int t = threadIdx.x;
     const int units = blockDim.x / UT;
@@ -86,18 +92,33 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     }
     pdl_wait();   // everything below may read what the previous kernel wrote
 
-    auto issue = [&](int64_t tile, int s) {              // first thread of the unit only
+    auto len_of = [&](int64_t tile) {                    // LEN: a tile is a row
+        return tile < num_tiles ? min(max(__ldg(a.len + tile), 0), a.nvec * NE) : 0;
+    };
+    auto issue = [&](int64_t tile, int s, int len) {     // first thread of the unit only
         const int64_t row0 = tile * a.tile_rows;
         const int rows_here = static_cast<int>(min(static_cast<int64_t>(a.tile_rows), a.rows - row0));
-        const uint32_t bytes = static_cast<uint32_t>(rows_here) * a.nvec * 16u;
-        mbar_expect_tx(&bars[s], bytes);
-        bulk_g2s(ring + tile_vecs * s, a.x + row0 * a.nvec, bytes, &bars[s]);
+        uint32_t bytes = static_cast<uint32_t>(rows_here) * a.nvec * 16u;
+        if constexpr (LEN) {
+            tile_len[unit * S + s] = len;
+            bytes = static_cast<uint32_t>((len + NE - 1) / NE) * 16u;              // the live vectors only
+        }
+        mbar_expect_tx(&bars[s], bytes);                 // also publishes tile_len to the threads that wait on the barrier
+        if (bytes) bulk_g2s(ring + tile_vecs * s, a.x + row0 * a.nvec, bytes, &bars[s]);
     };
-    if (ut == 0)
+    int pref_len = 0;                                    // LEN, issuing lane: the length of the tile it will issue next
+    if (ut == 0) {
+        int first_len[kPipeMaxBarriers > 8 ? 8 : kPipeMaxBarriers];
+        if constexpr (LEN) {
+#pragma unroll
+            for (int s = 0; s < 8; ++s) first_len[s] = s < S ? len_of(gu + s * GU) : 0;     // all requested before any is used
+            pref_len = len_of(gu + static_cast<int64_t>(S) * GU);
+        }
         for (int s = 0; s < S; ++s) {
             const int64_t tile = gu + s * GU;
-            if (tile < num_tiles) issue(tile, s);
+            if (tile < num_tiles) issue(tile, s, LEN ? first_len[s & 7] : 0);
         }
+    }
     if (OP != OP_SOFTMAX) {
         for (int i = t; i < a.nvec; i += blockDim.x) {
             params[i] = ld_param(a.p0 + i);
@@ -147,13 +168,29 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
                 r[q] = r0 + q * RPP + sub;
                 live[q] = (RPU == 1) || r[q] < rows_here;
                 const uint4* xr = stage + static_cast<size_t>(live[q] ? r[q] : 0) * a.nvec + lane;
+                if constexpr (LEN) {
+                    const int len = tile_len[unit * S + s];
 #pragma unroll
-                for (int v = 0; v < VPL; ++v) raw[q][v] = (live[q] && valid[v]) ? xr[v * LANES] : fill;
+                    for (int v = 0; v < VPL; ++v) raw[q][v] = (live[q] && valid[v] && (lane + v * LANES) * NE < len) ? xr[v * LANES] : fill;
+                    const int tail = len % NE, off = len / NE - lane;            // the vector that straddles the length: one thread's
+                    if (tail != 0 && off >= 0 && off % LANES == 0 && off / LANES < VPL) {
+                        const int mine = off / LANES;
+#pragma unroll
+                        for (int v = 0; v < VPL; ++v)
+                            if (v == mine) raw[q][v] = mask_tail<DT>(raw[q][v], tail);
+                    }
+                } else {
+#pragma unroll
+                    for (int v = 0; v < VPL; ++v) raw[q][v] = (live[q] && valid[v]) ? xr[v * LANES] : fill;
+                }
             }
             F2 w[RPG][VPL][Pairs<DT>::NP];
             Part part[RPG];
+            bool livev[VPL];                                      // LEN: vectors with at least one element in front of the length
 #pragma unroll
-            for (int q = 0; q < RPG; ++q) part[q] = slice_stats<OP, DT, VPL, decltype(red), FULL>(raw[q], valid, red, 0, my_count, w[q]);
+            for (int v = 0; v < VPL; ++v) livev[v] = LEN ? (valid[v] && (lane + v * LANES) * NE < tile_len[unit * S + s]) : valid[v];
+#pragma unroll
+            for (int q = 0; q < RPG; ++q) part[q] = slice_stats<OP, DT, VPL, decltype(red), FULL>(raw[q], livev, red, 0, my_count, w[q]);
             Total tot[RPG];
             if constexpr (W > 1) {
                 float* slot = xch + ((unit * 2 + xpar) * RPG) * W * 2;
@@ -173,8 +210,11 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
             }
             // The reductions above consumed every value this unit read from the stage (shuffle results and the
             // named barrier both depend on all of its loads): after the tile's last pass the stage is refilled.
-            if (r0 + RPU >= rows_here && ut == 0 && !failed && next < num_tiles) issue(next, s);
-            slice_finish_rows<OP, DT, VPL, RPG, (W == 1), FULL>(valid, w, tot, par, out);
+            if (r0 + RPU >= rows_here && ut == 0 && !failed && next < num_tiles) {
+                issue(next, s, pref_len);
+                if constexpr (LEN) pref_len = len_of(next + GU);
+            }
+            slice_finish_rows<OP, DT, VPL, RPG, (W == 1), FULL>(livev, w, tot, par, out);
 #pragma unroll
             for (int q = 0; q < RPG; ++q) {
                 if (live[q]) {
@@ -215,10 +255,20 @@ template <int OP> PipeFn pipe_fn_op(int dt, int lanes, int vpl, int rpg, bool fu
     return dt == DT_F32 ? pick_pipe<OP, DT_F32>(lanes, vpl, rpg, full) : pick_pipe<OP, DT_BF16>(lanes, vpl, rpg, full);
 }
 
+// The length-aware builds: softmax, one row per tile (units of at least a warp per row), one row per pass.
+template <int DT> PipeFn pick_pipe_len(int lanes, int vpl) {
+#define TF_PL(L, V) if (lanes == L && vpl == V) return k_pipe<OP_SOFTMAX, DT, L, V, 1, false, true>;
+    TF_PL(32, 2) TF_PL(32, 4) TF_PL(32, 8) TF_PL(64, 2) TF_PL(64, 4) TF_PL(64, 8) TF_PL(128, 2) TF_PL(128, 4) TF_PL(128, 8)
+    TF_PL(256, 2) TF_PL(256, 4) TF_PL(256, 8) TF_PL(512, 4) TF_PL(512, 8)
+#undef TF_PL
+    return nullptr;
+}
+
 // one translation unit per op instantiates the kernels
 PipeFn pipe_fn_softmax(int dt, int lanes, int vpl, int rpg, bool full);
 PipeFn pipe_fn_layernorm(int dt, int lanes, int vpl, int rpg, bool full);
 PipeFn pipe_fn_rmsnorm(int dt, int lanes, int vpl, int rpg, bool full);
+PipeFn pipe_fn_softmax_len(int dt, int lanes, int vpl);
 
 }  // namespace pipe
 }  // namespace tf

@@ -84,17 +84,25 @@ __device__ __forceinline__ Part slice_stats(const uint4 (&raw)[NV], const bool (
     using P = Pairs<DT>;
     constexpr int NP = P::NP;
     if constexpr (OP == OP_SOFTMAX) {
+        // vectors that are absent (or, with a row length, entirely behind it) hold -inf and contribute exact zeros: their
+        // exponentials are not evaluated
         float m = kNegInf;
 #pragma unroll
-        for (int v = 0; v < NV; ++v) m = fmaxf(m, vec_max<DT>(raw[v]));
+        for (int v = 0; v < NV; ++v)
+            if (ALLV || valid[v]) m = fmaxf(m, vec_max<DT>(raw[v]));
         m = red.max(m, slot0);
         const F2 off = f2(exp_offset(m)), l2e = f2(kLog2e);
         F2 s = f2(0.f);
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
-            P::unpack(raw[v], w[v]);
+            if (ALLV || valid[v]) {
+                P::unpack(raw[v], w[v]);
 #pragma unroll
-            for (int i = 0; i < NP; ++i) { w[v][i] = ex2_ftz2(fma2(w[v][i], l2e, off)); s = add2(s, w[v][i]); }
+                for (int i = 0; i < NP; ++i) { w[v][i] = ex2_ftz2(fma2(w[v][i], l2e, off)); s = add2(s, w[v][i]); }
+            } else {
+#pragma unroll
+                for (int i = 0; i < NP; ++i) w[v][i] = f2(0.f);
+            }
         }
         return Part{(m == kNegInf) ? -kNegInf : exp_offset(m), red.sum(hsum(s), slot0 + 1)};
     } else if constexpr (OP == OP_LAYERNORM) {
@@ -176,9 +184,13 @@ __device__ __forceinline__ void slice_finish_rows(const bool (&valid)[NV], F2 (&
             // maximum) while 1/S carries 2^-bias; their product could lose the subnormal bits.
 #pragma unroll
             for (int r = 0; r < R; ++r) {
+                if (ALLV || valid[v]) {
 #pragma unroll
-                for (int i = 0; i < NP; ++i) w[r][v][i] = SINGLE ? mul2(w[r][v][i], tb[r]) : mul2(mul2(w[r][v][i], ta[r]), tb[r]);
-                out[r][v] = P::pack(w[r][v]);
+                    for (int i = 0; i < NP; ++i) w[r][v][i] = SINGLE ? mul2(w[r][v][i], tb[r]) : mul2(mul2(w[r][v][i], ta[r]), tb[r]);
+                    out[r][v] = P::pack(w[r][v]);
+                } else {
+                    out[r][v] = make_uint4(0, 0, 0, 0);               // +0 in either element type
+                }
             }
         } else if constexpr (OP == OP_LAYERNORM) {
             if (ALLV || valid[v]) {

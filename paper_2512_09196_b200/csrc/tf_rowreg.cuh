@@ -126,7 +126,12 @@ __global__ void __launch_bounds__(kWarpMaxThreads) k_warp(const KArgs a) {
             const int64_t row = base + rr * G + g;
             uint4 out[VPT];
             float st0 = 0.f, st1 = 0.f;
-            row_math<OP, DT, VPT>(raw[rr], valid, red, par, 0, a.n, a.eps, out, st0, st1);
+            // which vectors the arithmetic visits: for softmax all of them (absent or masked ones hold -inf and give exact
+            // zeros; a test per vector cost these latency-bound kernels 4-10 %), for the norms the ones that exist
+            bool visit[VPT];
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) visit[v] = OP == OP_SOFTMAX || valid[v];
+            row_math<OP, DT, VPT>(raw[rr], visit, red, par, 0, a.n, a.eps, out, st0, st1);
             if (row < a.rows) {
 #pragma unroll
                 for (int v = 0; v < VPT; ++v)
@@ -200,14 +205,17 @@ __global__ void __launch_bounds__(cta_max_threads(VPT)) k_cta(const KArgs a, con
         }
         float st0 = 0.f, st1 = 0.f;
         const int slot0 = (it & 1) * 2;
+        bool livev[VPT];                                          // softmax visits every vector (see k_warp); the norms the ones that exist
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) livev[v] = (OP == OP_SOFTMAX && MODE != kModeAdd) || valid[v];
 
         if constexpr (!CLUSTER) {
-            row_math<OP, DT, VPT>(raw, valid, red, par, slot0, a.n, a.eps, out, st0, st1);
+            row_math<OP, DT, VPT>(raw, livev, red, par, slot0, a.n, a.eps, out, st0, st1);
         } else {
             cg::cluster_group cl = cg::this_cluster();
             const int par_buf = it & 1;
             F2 w[VPT][Pairs<DT>::NP];
-            const Part part = slice_stats<OP, DT, VPT>(raw, valid, red, slot0, static_cast<float>(len) * NE, w);
+            const Part part = slice_stats<OP, DT, VPT>(raw, livev, red, slot0, static_cast<float>(len) * NE, w);
             if (t < cs) {                                             // push my partial into every CTA of the cluster
                 float* dst = cl.map_shared_rank(&xch[par_buf][rank][0], t);
                 dst[0] = part.a; dst[1] = part.b;
@@ -217,7 +225,7 @@ __global__ void __launch_bounds__(cta_max_threads(VPT)) k_cta(const KArgs a, con
                 cs, rank, [&](int k) { return Part{xch[par_buf][k][0], xch[par_buf][k][1]}; },
                 [&](int k) { return static_cast<float>(max(0, min(per, a.nvec - k * per))) * NE; }, a.n, a.eps);
             st0 = tot.a; st1 = tot.b;
-            slice_finish<OP, DT, VPT, false>(valid, w, tot, par, out);
+            slice_finish<OP, DT, VPT, false>(livev, w, tot, par, out);
         }
 #pragma unroll
         for (int v = 0; v < VPT; ++v)

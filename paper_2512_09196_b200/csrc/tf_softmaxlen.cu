@@ -53,18 +53,21 @@ bool supports_softmax_len(const Plan& p, const Args& a, const DeviceInfo& d) {
     if (p.variant == V_WARP) return warp_geometry_ok(p, a) && warp_fn_len(a.dt, p.lanes, p.vpt, p.rpg) != nullptr;
     if (p.variant == V_CTA) return cta_geometry_ok(p, a, d) && cta_fn_len(a.dt, p.vpt, p.cluster > 1) != nullptr;
     if (p.variant == V_TWOPASS) return supports_twopass(p, a, d);
+    if (p.variant == V_PIPE) return supports_pipe(p, a, d) && p.stages <= 8;
     return false;
 }
 
 cudaError_t launch_softmax_len(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
     count_launches(1);
     if (p.variant == V_TWOPASS) return launch_twopass(p, a, d, st);
+    if (p.variant == V_PIPE) return launch_pipe(p, a, d, st);
     if (p.variant == V_WARP) return launch_warp_fn(warp_fn_len(a.dt, p.lanes, p.vpt, p.rpg), p, a, d, st);
     return launch_cta_fn(cta_fn_len(a.dt, p.vpt, p.cluster > 1), p, a, d, st);
 }
 
-// Default plan, from measurements on rows of 512 B to 64 KiB: a lane group with one row in flight up to 1 KiB, a CTA
-// with four vectors per thread (eight for fp32 from 16 KiB on) up to 64 KiB, the streamed two-pass kernel from there.
+// Default plan, from measurements on rows of 512 B to 64 KiB: a lane group with one row in flight up to 1 KiB, the
+// length-aware pipeline for 2-byte rows of 4-64 KiB, a CTA with four vectors per thread (eight for fp32 from 16 KiB on)
+// for the rest up to 64 KiB, the streamed two-pass kernel from there.
 // (The plans that win for the plain softmax are not reused: more rows in flight per group or eight bf16 vectors per
 // thread cost this mode 30-80 %.)
 Plan heuristic_softmax_len(const Args& a, const DeviceInfo& d) {
@@ -76,6 +79,21 @@ Plan heuristic_softmax_len(const Args& a, const DeviceInfo& d) {
         else if (nvec <= 16) { q.lanes = 8; q.vpt = 2; }
         else if (nvec <= 32) { q.lanes = 16; q.vpt = 2; }
         else { q.lanes = 32; q.vpt = 2; }
+        if (supports_softmax_len(q, a, d)) return q;
+    } else if (a.dt == DT_BF16 && nvec >= 256 && nvec <= 4096) {
+        // 2-byte rows of 4-64 KiB: the pipeline copies only the live part of each row and its units skip the vectors
+        // behind the length (measured 7-16 % faster than the masked plain softmax at half-live rows, where the register
+        // plans below are slower than it)
+        q.variant = V_PIPE; q.vpt = 8; q.rpg = 1; q.stages = 2; q.chunk = 16;
+        q.lanes = 32;
+        while (q.lanes < 512 && static_cast<int64_t>(q.lanes) * 8 < nvec) q.lanes *= 2;
+        q.threads = std::max(256, q.lanes);
+        q.persist = q.threads == 256 ? 2 : 1;
+        if (supports_softmax_len(q, a, d)) return q;
+        q = Plan{};
+        q.variant = V_CTA; q.cluster = 1;
+        q.vpt = 4;
+        q.threads = std::max(64, static_cast<int>((nvec + q.vpt - 1) / q.vpt + 31) / 32 * 32);
         if (supports_softmax_len(q, a, d)) return q;
     } else if (nvec < 4096) {
         q.variant = V_CTA; q.cluster = 1;

@@ -96,9 +96,17 @@ def test_forced_plans_and_bitwise_equality_with_the_masked_plain_softmax(dt):
         for nvec, rows in ((cluster + 1, 9), (threads * 4 * cluster + 1, 9), (70001, 9)):
             tf.tf_force_plan("softmax", f"twopass:threads={threads},cache={cache},persist=0,regcap=0,cluster={cluster}")
             run_case(dt, rows, nvec * ne, seed=nvec + cluster)
-    # a forced plan without a length mode (the pipeline) falls back to the length-aware choice
-    tf.tf_force_plan("softmax", "pipe:threads=512,lanes=64,vpt=8,rpg=1,stages=2,chunk=8192,persist=1")
-    run_case(dt, 100, 512 * ne)
+    # the pipeline: only the live part of a row is copied; exact and ragged fits, few and many rows per unit, every ring depth
+    for lanes, vpt, threads, stages, persist in ((32, 2, 128, 2, 1), (32, 8, 512, 4, 2), (64, 8, 512, 2, 1), (128, 4, 256, 3, 0), (256, 8, 512, 1, 1),
+                                                 (512, 4, 512, 8, 1)):
+        cap = lanes * vpt
+        for nvec, rows in ((cap, 9), (cap - 1, 700), (max(1, cap // 2 + 1), 3000)):
+            rows = min(rows, max(3, (1 << 22) // (nvec * ne)))
+            tf.tf_force_plan("softmax", f"pipe:threads={threads},lanes={lanes},vpt={vpt},rpg=1,stages={stages},chunk=16,persist={persist}")
+            run_case(dt, rows, nvec * ne, seed=nvec + lanes, compare_plain=False)
+    # a forced plan without a length mode (the cluster ring) falls back to the length-aware choice
+    tf.tf_force_plan("softmax", "ring:threads=256,vpt=4,cluster=2,stages=2,persist=1")
+    run_case(dt, 100, 2048 * ne)
 
 
 def test_bad_arguments():
