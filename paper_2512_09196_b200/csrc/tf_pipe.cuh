@@ -186,9 +186,9 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
             }
             F2 w[RPG][VPL][Pairs<DT>::NP];
             Part part[RPG];
-            bool livev[VPL];                                      // LEN: vectors with at least one element in front of the length
+            bool livev[VPL];      // vectors the arithmetic visits: LEN: those in front of the length; plain softmax: all (absent ones hold -inf)
 #pragma unroll
-            for (int v = 0; v < VPL; ++v) livev[v] = LEN ? (valid[v] && (lane + v * LANES) * NE < tile_len[unit * S + s]) : valid[v];
+            for (int v = 0; v < VPL; ++v) livev[v] = LEN ? (valid[v] && (lane + v * LANES) * NE < tile_len[unit * S + s]) : (OP == OP_SOFTMAX || valid[v]);
 #pragma unroll
             for (int q = 0; q < RPG; ++q) part[q] = slice_stats<OP, DT, VPL, decltype(red), FULL>(raw[q], livev, red, 0, my_count, w[q]);
             Total tot[RPG];

@@ -146,7 +146,10 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
         for (int v = 0; v < VPT; ++v) raw[v] = valid[v] ? buf[v * T] : fill;
         const int xb = it & 1;
         F2 w[VPT][Pairs<DT>::NP];
-        const Part part = slice_stats<OP, DT, VPT>(raw, valid, red, xb * 2, slice_count(rank), w);
+        bool visit[VPT];                                          // softmax visits every vector (absent ones hold -inf), the norms the ones that exist
+#pragma unroll
+        for (int v = 0; v < VPT; ++v) visit[v] = OP == OP_SOFTMAX || valid[v];
+        const Part part = slice_stats<OP, DT, VPT>(raw, visit, red, xb * 2, slice_count(rank), w);
         // every thread passed the CTA barrier inside the reduction after its shared-memory reads: refill the stage
         const int64_t next = row + static_cast<int64_t>(S) * num_clusters;
         if (t == 0 && !failed && next < a.rows) issue(next, s);
@@ -161,9 +164,9 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
             __syncthreads();
         }
         const Total tot = combine_parts<OP>(cs, rank, [&](int k) { return Part{xch[xb][k][0], xch[xb][k][1]}; }, slice_count, a.n, a.eps);
-        if constexpr (kHeld) slice_finish<OP, DT, VPT, false>(valid, w, tot, held, out);
-        else if constexpr (PSMEM) slice_finish<OP, DT, VPT, false>(valid, w, tot, inshared, out);
-        else slice_finish<OP, DT, VPT, false>(valid, w, tot, lazy, out);
+        if constexpr (kHeld) slice_finish<OP, DT, VPT, false>(visit, w, tot, held, out);
+        else if constexpr (PSMEM) slice_finish<OP, DT, VPT, false>(visit, w, tot, inshared, out);
+        else slice_finish<OP, DT, VPT, false>(visit, w, tot, lazy, out);
         uint4* yr = a.y + row * a.nvec + first + t;
 #pragma unroll
         for (int v = 0; v < VPT; ++v)
