@@ -876,6 +876,28 @@ def run_case(args):
         print(json.dumps({"case": w.name, "knobs": knobs, "launches": args.steps, "us_per_launch": us,
                           "gbs": w.algorithmic_bytes() / us / 1e3}))
         return
+    if parts[0] == "softmaxlen":              # softmaxlen:dtype:rows:cols -- softmax with uniform per-row lengths
+        import numpy as np
+        dts, rows, cols = parts[1], int(parts[2]), int(parts[3])
+        dt = inputs.F32 if dts == "f32" else inputs.BF16
+        conv = (lambda t: t.view(torch.bfloat16)) if dt == inputs.BF16 else (lambda t: t)
+        x = conv(torch.from_numpy(inputs.normal((rows, cols), dt, cols, 0, 0.0, 3.0))).cuda()
+        lens = torch.from_numpy(np.random.default_rng(cols).integers(0, cols + 1, rows).astype(np.int32)).cuda()
+        y = torch.empty_like(x)
+        a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(max(1, args.warmup)):
+            tf.tf_softmax_len_fwd(x, lens, y)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(args.steps):
+            tf.tf_softmax_len_fwd(x, lens, y)
+        e.record()
+        torch.cuda.synchronize()
+        us = 1e3 * a.elapsed_time(e) / args.steps
+        live = int(lens.sum().item()) * inputs.ELEM_SIZE[dt]
+        nbytes = live + rows * cols * inputs.ELEM_SIZE[dt] + 4 * rows
+        print(json.dumps({"case": f"case_softmax_len_{dts}_{rows}x{cols}", "launches": args.steps, "us_per_launch": us, "gbs": nbytes / us / 1e3}))
+        return
     if parts[0] == "normbwd":                 # normbwd:op:dtype:rows:cols -- the backward pass of a norm
         op, dts, rows, cols = parts[1], parts[2], int(parts[3]), int(parts[4])
         dt = inputs.F32 if dts == "f32" else inputs.BF16
@@ -968,7 +990,7 @@ def main():
     ap.add_argument("--filter", default=None)
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
-    ap.add_argument("--case", default=None, help="op:dtype:rows:cols, config:<i>[:rows], vecmat:..., addnorm:op:dtype:rows:cols -- a few launches of one shape")
+    ap.add_argument("--case", default=None, help="op:dtype:rows:cols, config:<i>[:rows], vecmat:..., addnorm:op:dtype:rows:cols, normbwd:op:dtype:rows:cols, softmaxlen:dtype:rows:cols -- a few launches of one shape")
     ap.add_argument("--plan", default=None, help="with --case: force this launch plan")
     args = ap.parse_args()
     if args.impl == "reference":
