@@ -108,15 +108,19 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     };
     int pref_len = 0;                                    // LEN, issuing lane: the length of the tile it will issue next
     if (ut == 0) {
-        int first_len[kPipeMaxBarriers > 8 ? 8 : kPipeMaxBarriers];
-        if constexpr (LEN) {
+        if constexpr (LEN) {                             // at most eight stages: the lengths are all requested before any is used
+            int first_len[8];
 #pragma unroll
-            for (int s = 0; s < 8; ++s) first_len[s] = s < S ? len_of(gu + s * GU) : 0;     // all requested before any is used
+            for (int s = 0; s < 8; ++s) first_len[s] = s < S ? len_of(gu + s * GU) : 0;
             pref_len = len_of(gu + static_cast<int64_t>(S) * GU);
-        }
-        for (int s = 0; s < S; ++s) {
-            const int64_t tile = gu + s * GU;
-            if (tile < num_tiles) issue(tile, s, LEN ? first_len[s & 7] : 0);
+#pragma unroll
+            for (int s = 0; s < 8; ++s)
+                if (s < S && gu + s * GU < num_tiles) issue(gu + s * GU, s, first_len[s]);
+        } else {
+            for (int s = 0; s < S; ++s) {
+                const int64_t tile = gu + s * GU;
+                if (tile < num_tiles) issue(tile, s, 0);
+            }
         }
     }
     if (OP != OP_SOFTMAX) {
