@@ -80,7 +80,7 @@ std::string plan_to_string(const Plan& p) {
         case V_TMA: snprintf(b, sizeof b, "tma:threads=%d,cluster=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.cluster, p.stages, p.chunk, p.persist); break;
         case V_PIPE: snprintf(b, sizeof b, "pipe:threads=%d,lanes=%d,vpt=%d,rpg=%d,stages=%d,chunk=%d,persist=%d", p.threads, p.lanes, p.vpt, p.rpg, p.stages, p.chunk, p.persist); break;
         case V_RING: snprintf(b, sizeof b, "ring:threads=%d,vpt=%d,cluster=%d,stages=%d,persist=%d,psmem=%d", p.threads, p.vpt, p.cluster, p.stages, p.persist, p.rpg == 2 ? 1 : 0); break;
-        case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,cache=%d,persist=%d,regcap=%d,cluster=%d", p.threads, p.chunk, p.persist, p.rpg == 2 ? 1 : 0, p.cluster); break;
+        case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,cache=%d,persist=%d,regcap=%d,cluster=%d,groups=%d,hints=%d,stages=%d,u=%d", p.threads, p.chunk, p.persist, p.rpg == 2 ? 1 : 0, p.cluster, p.lanes, p.vpt, p.stages, p.unroll); break;
         case V_SPLIT: snprintf(b, sizeof b, "split:threads=%d,splits=%d", p.threads, p.cluster); break;
         default: snprintf(b, sizeof b, "stream:threads=%d,lanes=%d,persist=%d", p.threads, p.lanes, p.persist); break;
     }
@@ -98,7 +98,7 @@ bool plan_from_string(const char* s, Plan& out) {
     if (v == V_STREAM) p.lanes = 0;
     if (v == V_PIPE) { p.persist = 1; p.stages = 4; p.chunk = 32768; }
     if (v == V_RING) { p.persist = 1; p.stages = 2; }
-    if (v == V_TWOPASS) p.chunk = 0;
+    if (v == V_TWOPASS) { p.chunk = 0; p.lanes = 1; p.vpt = 3; p.stages = 0; }
     const char* q = colon ? colon + 1 : s + strlen(s);
     while (*q) {
         const char* eq = strchr(q, '=');
@@ -107,9 +107,9 @@ bool plan_from_string(const char* s, Plan& out) {
         char* end = nullptr;
         long val = strtol(eq + 1, &end, 10);
         if (end == eq + 1) return false;
-        if (key == "threads") p.threads = val; else if (key == "lanes") p.lanes = val; else if (key == "vpt") p.vpt = val;
+        if (key == "threads") p.threads = val; else if (key == "lanes" || key == "groups") p.lanes = val; else if (key == "vpt" || key == "hints") p.vpt = val;
         else if (key == "rpg") p.rpg = val; else if (key == "cluster" || key == "splits") p.cluster = val; else if (key == "stages") p.stages = val;
-        else if (key == "chunk" || key == "cache") p.chunk = val; else if (key == "persist") p.persist = val; else if (key == "regcap" || key == "psmem") p.rpg = val ? 2 : 1; else return false;
+        else if (key == "chunk" || key == "cache") p.chunk = val; else if (key == "persist") p.persist = val; else if (key == "u") p.unroll = val; else if (key == "regcap" || key == "psmem") p.rpg = val ? 2 : 1; else return false;
         q = (*end == ',') ? end + 1 : end;
         if (*end && *end != ',') return false;
     }
@@ -195,6 +195,14 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         s.cluster = static_cast<int>(std::max<int64_t>(2, std::min<int64_t>(nvec / 256, 2 * d.sms / a.rows)));
         if (supports_split(s, a, d)) return s;
     }
+    if (a.op == OP_SOFTMAX && nvec >= 16384 && a.rows >= 16LL * d.sms) {
+        // many rows of 256 KiB and more: two streamed passes with each thread's loads running ahead of its arithmetic in a
+        // private shared-memory ring (three CTAs of 512 threads per SM); measured 322 us on the 2 GiB masked softmax
+        // against 360-460 us for every plan that keeps the row on chip
+        Plan s;
+        s.variant = V_TWOPASS; s.threads = 512; s.chunk = 0; s.rpg = 2; s.lanes = 1; s.vpt = 3; s.stages = 2; s.unroll = 4;
+        if (supports_twopass(s, a, d)) return s;
+    }
     // Rules read off the plans that tf_tune ends up with on the 84-point shape sweep (rows of 128 B to 256 KiB, three ops,
     // two types); what they do not cover falls through to the older defaults below.
     {
@@ -272,7 +280,7 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
     // everything beyond 128 KiB; persistent clusters with a prefetch ring in between
     if (a.op == OP_LAYERNORM || nvec > 8192) {
         Plan s;
-        s.variant = V_TWOPASS; s.threads = 512; s.chunk = 49152;
+        s.variant = V_TWOPASS; s.threads = 512; s.chunk = 49152; s.lanes = 1; s.vpt = 3; s.stages = 0;
         if (a.op == OP_SOFTMAX) s.rpg = 2;           // the 40-register build: three CTAs per SM (measured faster on the 2 GiB softmax)
         return s;
     }
@@ -297,7 +305,7 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
     p.cluster = cl;
     if (!supports_tma(p, a, d)) {           // longer than a full cluster of shared memory can hold
         Plan s;
-        s.variant = V_TWOPASS; s.threads = 1024; s.chunk = 0;
+        s.variant = V_TWOPASS; s.threads = 1024; s.chunk = 0; s.lanes = 1; s.vpt = 3; s.stages = 0;
         return s;
     }
     return p;
@@ -388,7 +396,7 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
             for (int persist : {0, 2048 / th})
                 for (int cache : {0, 1}) {
                     // cache: what shared memory offers each of the 2048 / th CTAs of an SM, at most the row
-                    Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = persist;
+                    Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = persist; p.lanes = 1; p.vpt = 3; p.stages = 0;
                     p.chunk = cache ? static_cast<int>(std::min<int64_t>(nvec * 16, (200 * 1024 / (2048 / th)) / 16 * 16)) : 0;
                     add(p);
                     if (th <= 768 && persist == 0) { p.rpg = 2; add(p); }      // 40-register form: 1536 resident threads per SM
@@ -397,6 +405,15 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
                         for (int cl : {2, 4, 8})
                             if (nvec / cl >= 2048) { Plan q = p; q.cluster = cl; q.chunk = std::min(q.chunk, static_cast<int>(nvec / cl * 16)); add(q); }
                 }
+    // two streamed passes fed through per-thread rings of asynchronous copies
+    if (nvec >= 1024)
+        for (int th : {256, 384, 512})
+            for (int su : {24, 32, 34, 44}) {                          // (stages, vectors per step)
+                Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = 0; p.lanes = 1; p.vpt = 3; p.chunk = 0;
+                p.stages = su / 10; p.unroll = su % 10; p.rpg = 2;
+                add(p);
+                if (th == 512 && su == 34) { p.rpg = 1; add(p); }
+            }
     // persistent cluster ring for long rows
     if (nvec >= 2048)
         for (int cl : {1, 2, 4, 8})
@@ -445,7 +462,7 @@ std::vector<Plan> neighbours(const Plan& b) {
         if (th >= 32 && th <= 1024 && th % 32 == 0 && th != b.threads) with([&](Plan& p) { p.threads = th; });
     for (int pe : {b.persist - 1, b.persist + 1, b.persist * 2, 0})
         if (pe >= 0 && pe <= 32 && pe != b.persist) with([&](Plan& p) { p.persist = pe; });
-    if (b.variant == V_PIPE || b.variant == V_RING || b.variant == V_TMA)
+    if (b.variant == V_PIPE || b.variant == V_RING || b.variant == V_TMA || (b.variant == V_TWOPASS && b.stages >= 2))
         for (int st : {b.stages - 1, b.stages + 1})
             if (st >= 1 && st <= 8) with([&](Plan& p) { p.stages = st; });
     if (b.variant == V_PIPE || b.variant == V_TMA || b.variant == V_TWOPASS)
@@ -455,6 +472,11 @@ std::vector<Plan> neighbours(const Plan& b) {
         for (int r : {1, 2, 4})
             if (r != b.rpg) with([&](Plan& p) { p.rpg = r; });
     if (b.variant == V_TWOPASS || b.variant == V_RING) with([&](Plan& p) { p.rpg = b.rpg == 2 ? 1 : 2; });
+    if (b.variant == V_TWOPASS) {
+        if (b.stages >= 2) with([&](Plan& p) { p.unroll = b.unroll == 4 ? 2 : 4; });
+        for (int g : {1, 8}) if (g != b.lanes) with([&](Plan& p) { p.lanes = g; });
+        for (int h : {0, 3}) if (h != b.vpt) with([&](Plan& p) { p.vpt = h; });
+    }
     if (b.variant == V_SPLIT)
         for (int sp : {b.cluster / 2, b.cluster * 3 / 4, b.cluster * 3 / 2, b.cluster * 2})
             if (sp >= 1 && sp != b.cluster) with([&](Plan& p) { p.cluster = sp; });

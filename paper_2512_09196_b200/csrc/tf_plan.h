@@ -31,6 +31,7 @@ struct Plan {
     int stages = 1;      // V_TMA / V_PIPE: shared-memory ring depth
     int chunk = 8192;    // V_TMA: bytes per bulk copy (one mbarrier each); V_PIPE: bytes per stage
     int persist = 0;     // 0: grid covers all rows once; k > 0: k CTAs per SM looping over rows (V_PIPE: always >= 1)
+    int unroll = 4;      // V_TWOPASS with a ring (stages >= 2): 16-byte vectors per thread per ring stage (2 or 4)
 };
 
 struct Args {

@@ -102,7 +102,7 @@ Plan heuristic_softmax_len(const Args& a, const DeviceInfo& d) {
         if (supports_softmax_len(q, a, d)) return q;
     }
     Plan t;
-    t.variant = V_TWOPASS; t.threads = 512; t.chunk = 49152; t.rpg = 2;
+    t.variant = V_TWOPASS; t.threads = 512; t.chunk = 49152; t.rpg = 2; t.lanes = 1; t.vpt = 3; t.stages = 0;
     return t;
 }
 

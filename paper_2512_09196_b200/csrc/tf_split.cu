@@ -213,7 +213,8 @@ extern "C" tf_status tf_softmax_fwd_noalloc(const void* x, void* y, int64_t rows
     splits = std::min<int64_t>(splits, kStaticPartials / rows);
     Plan p;
     p.variant = V_SPLIT; p.threads = 256; p.cluster = static_cast<int>(splits);
-    DeviceInfo d;
+    DeviceInfo d{};
+    d.sms = sc->sms;
     if (!supports_split(p, a, d)) return TF_ERR_UNSUPPORTED;
     count_launches(2);
     e = launch_split_with_scratch(p, a, sc->ptr, static_cast<cudaStream_t>(stream));

@@ -19,6 +19,11 @@ __device__ __forceinline__ uint64_t policy_evict_first() {
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
+__device__ __forceinline__ uint64_t policy_evict_normal() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
 __device__ __forceinline__ uint4 ld_hint(const uint4* p, uint64_t policy) {
     uint4 v;
     asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
@@ -33,57 +38,85 @@ template <int DT> __device__ __forceinline__ bool all_neg_inf_vec(const uint4& v
 
 constexpr int kStreamU = 4;          // independent 16-byte loads per thread per step
 
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {       // NaNs are ignored, as by fmaxf
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
 // Per-thread running statistics over the vectors a thread meets while streaming a segment.
-//   softmax   (offset of the running max, sum at that offset), rescaled online when the max grows
+//   softmax   (offset of the running max, packed pair of sums at that offset), rescaled online when the max grows
 //   LayerNorm (n, mean, M2): each step's exact two-pass statistics merged with Chan's update
 //   RMSNorm   sum of squares
-template <int OP, int DT> struct Running {
-    float s_off = 0.f, s_sum = 0.f, s_max = kNegInf;
+// A thread's vectors are numbered by SLOT = step * U_ + u (U_ vectors per step) in row order.
+template <int OP, int DT, int U_ = kStreamU> struct Running {
+    float s_off = 0.f, s_max = kNegInf;
+    F2 s_sum2 = f2(0.f);
     float c_n = 0.f, c_mean = 0.f, c_m2 = 0.f;
     F2 q2 = f2(0.f);
-    int64_t live_end = 0;            // softmax: one past the last vector of THIS thread that held anything but -inf
+    int live_slots = 0;              // softmax: one past the last slot of THIS thread that held anything but -inf
 
-    __device__ __forceinline__ void update(const uint4 (&raw)[kStreamU], const bool (&ok)[kStreamU]) {
+    // raw: the step's vectors, absent ones already replaced by the fill value (-inf for softmax, 0 for the norms);
+    // PRED: some may be absent, ok[] says which exist; count: elements that exist (LayerNorm's divisor); slot0: slot of raw[0].
+    template <bool PRED>
+    __device__ __forceinline__ void update(const uint4 (&raw)[U_], const bool (&ok)[U_], int count, int slot0) {
         using P = Pairs<DT>;
-        constexpr int NE = Elem<DT>::NE, NP = P::NP, U = kStreamU;
+        constexpr int NP = P::NP, U = U_;
         if constexpr (OP == OP_SOFTMAX) {
-            float cm = kNegInf;
+            // maxima per vector (a vector of nothing but -inf is skipped: no exponentials) and of the step
+            bool live[U];
+            float cm;
+            if constexpr (DT == DT_BF16) {
+                uint32_t pm[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) cm = fmaxf(cm, vec_max<DT>(raw[u]));       // absent vectors are filled with -inf
-            if (cm > s_max) {                                                     // new running max: move the sum to its offset
+                for (int u = 0; u < U; ++u) {
+                    pm[u] = bf16x2_max(bf16x2_max(raw[u].x, raw[u].y), bf16x2_max(raw[u].z, raw[u].w));
+                    live[u] = pm[u] != 0xFF80FF80u;
+                }
+                uint32_t pa = pm[0];
+#pragma unroll
+                for (int u = 1; u < U; ++u) pa = bf16x2_max(pa, pm[u]);
+                cm = fmaxf(__uint_as_float(pa << 16), __uint_as_float(pa & 0xFFFF0000u));
+            } else {
+                cm = kNegInf;
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const float vm = vec_max<DT>(raw[u]);
+                    live[u] = vm != kNegInf;
+                    cm = fmaxf(cm, vm);
+                }
+            }
+            if (cm > s_max) {                                                     // new running max: move the sums to its offset
                 const float noff = exp_offset(cm);
-                s_sum = (s_max == kNegInf) ? 0.f : s_sum * ex2_ftz(noff - s_off);
+                s_sum2 = (s_max == kNegInf) ? f2(0.f) : mul2(s_sum2, f2(ex2_ftz(noff - s_off)));
                 s_off = noff; s_max = cm;
             }
             const F2 off = f2(s_off), l2e = f2(kLog2e);
-            F2 acc = f2(0.f);
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (!all_neg_inf_vec<DT>(raw[u])) {                               // masked vectors cost no exponentials
+                if (live[u]) {
                     F2 w[NP]; P::unpack(raw[u], w);
 #pragma unroll
-                    for (int i = 0; i < NP; ++i) acc = add2(acc, ex2_ftz2(fma2(w[i], l2e, off)));
+                    for (int i = 0; i < NP; ++i) s_sum2 = add2(s_sum2, ex2_ftz2(fma2(w[i], l2e, off)));
+                    live_slots = max(live_slots, slot0 + u + 1);         // pass A may walk the row in either direction
                 }
             }
-            s_sum += hsum(acc);
         } else if constexpr (OP == OP_LAYERNORM) {
             F2 w[U][NP];
             F2 s2 = f2(0.f);
-            int cnt = 0;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                P::unpack(raw[u], w[u]);                                          // absent vectors are filled with 0
-                cnt += ok[u] ? NE : 0;
+                P::unpack(raw[u], w[u]);
 #pragma unroll
                 for (int i = 0; i < NP; ++i) s2 = add2(s2, w[u][i]);
             }
-            const float nc = static_cast<float>(cnt);
-            const float mc = fast_div(hsum(s2), nc);                              // cnt > 0: a step has at least one vector
+            const float nc = static_cast<float>(count);                           // > 0: a step has at least one vector
+            const float mc = fast_div(hsum(s2), nc);
             const F2 mc2 = f2(mc);
             F2 d2 = f2(0.f);
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (ok[u]) {
+                if (!PRED || ok[u]) {
 #pragma unroll
                     for (int i = 0; i < NP; ++i) { const F2 d = sub2(w[u][i], mc2); d2 = fma2(d, d, d2); }
                 }
@@ -101,37 +134,56 @@ template <int OP, int DT> struct Running {
     }
 };
 
-// Pass A over `nvec` vectors starting at xs (all threads of the CTA take part).  The first `cache_vecs` vectors
-// are also parked in shared memory (`cache`), each by the thread that will want it back in pass B -- the same
-// thread meets the same vectors in both passes, so no barrier is needed between them.
-// len >= 0 (softmax with a valid length, in elements): only the first ceil(len / NE) vectors are read and the one that
+// Pass A over `nvec` vectors starting at xs (all threads of the CTA take part).  Whole steps (every thread has all of its
+// kStreamU vectors) run without predicates; one ragged step follows where the row does not end on a step.
+// CACHE: the first `cache_vecs` vectors are also parked in shared memory (`cache`), each by the thread that will want it
+// back in pass B -- the same thread meets the same vectors in both passes, so no barrier is needed between them.
+// LEN (softmax with a valid length `len`, in elements): only the first ceil(len / NE) vectors are read and the one that
 // straddles the length has its tail replaced by -inf.
-template <int OP, int DT>
+template <int OP, int DT, bool LEN = false, bool CACHE = false>
 __device__ __forceinline__ Running<OP, DT> stream_stats(const uint4* xs, int64_t nvec, uint64_t policy, uint4* cache = nullptr,
                                                         int64_t cache_vecs = 0, int64_t len = -1) {
     constexpr int U = kStreamU, NE = Elem<DT>::NE;
     const int T = blockDim.x, t = threadIdx.x;
-    const uint4 fill = fill_vec<DT>(OP);
     Running<OP, DT> run;
-    if (len >= 0) nvec = (len + NE - 1) / NE;
-    const int64_t straddle = (len >= 0 && len % NE) ? nvec - 1 : -1;
-    for (int64_t base = t; base < nvec; base += static_cast<int64_t>(T) * U) {
+    int64_t straddle = -1;
+    if constexpr (LEN) {
+        nvec = (len + NE - 1) / NE;
+        if (len % NE) straddle = nvec - 1;
+    }
+    const int64_t step = static_cast<int64_t>(T) * U;
+    // the straddling vector is the last one: it is left to the ragged step
+    const int nfull = static_cast<int>((nvec - (LEN && straddle >= 0 ? 1 : 0)) / step);
+    const uint4* p = xs + t;
+    for (int s = 0; s < nfull; ++s, p += step) {
+        uint4 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) raw[u] = ld_hint(p + u * T, policy);
+        if constexpr (CACHE) {
+            const int64_t idx0 = s * step + t;
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (idx0 + u * T < cache_vecs) cache[idx0 + u * T] = raw[u];          // cache_vecs <= nvec
+        }
+        const bool all[U] = {true, true, true, true};
+        run.template update<false>(raw, all, U * NE, s * U);
+    }
+    const int64_t base = nfull * step + t;
+    if (base < nvec) {                                                               // the ragged step
+        const uint4 fill = fill_vec<DT>(OP);
         uint4 raw[U];
         bool ok[U];
+        int count = 0;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int64_t idx = base + static_cast<int64_t>(u) * T;
             ok[u] = idx < nvec;
             raw[u] = ok[u] ? ld_hint(xs + idx, policy) : fill;
-            if (idx == straddle) raw[u] = mask_tail<DT>(raw[u], static_cast<int>(len % NE));
+            count += ok[u] ? NE : 0;
+            if (LEN && idx == straddle) raw[u] = mask_tail<DT>(raw[u], static_cast<int>(len % NE));
+            if (CACHE && idx < cache_vecs) cache[idx] = raw[u];
         }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int64_t idx = base + static_cast<int64_t>(u) * T;
-            if (idx < cache_vecs) cache[idx] = raw[u];          // cache_vecs <= nvec
-            if (OP == OP_SOFTMAX && ok[u] && !all_neg_inf_vec<DT>(raw[u])) run.live_end = idx + 1;
-        }
-        run.update(raw, ok);
+        run.template update<true>(raw, ok, count, nfull * U);
     }
     return run;
 }
@@ -140,12 +192,12 @@ __device__ __forceinline__ Running<OP, DT> stream_stats(const uint4* xs, int64_t
 // softmax (offset of the segment max, or +inf for an all -inf segment; sum at that offset),
 // LayerNorm (segment mean, segment M2) for `count` elements, RMSNorm (sum of squares, 0).
 // rb: 64 floats of shared memory not used by the previous merge of this CTA.
-template <int OP, int DT>
-__device__ __forceinline__ Part merge_running(const Running<OP, DT>& run, float count, float* rb) {
+template <int OP, int DT, int U_ = kStreamU>
+__device__ __forceinline__ Part merge_running(const Running<OP, DT, U_>& run, float count, float* rb) {
     if constexpr (OP == OP_SOFTMAX) {
         const float M = cta_reduce<MaxOp>(run.s_max, rb);
         const float O = exp_offset(M);
-        const float mine = (run.s_max == kNegInf) ? 0.f : run.s_sum * ex2(O - run.s_off);       // O <= s_off: factor <= 1
+        const float mine = (run.s_max == kNegInf) ? 0.f : hsum(run.s_sum2) * ex2(O - run.s_off);       // O <= s_off: factor <= 1
         const float S = cta_reduce<SumOp>(mine, rb + 32);
         return Part{(M == kNegInf) ? -kNegInf : O, S};
     } else if constexpr (OP == OP_LAYERNORM) {
@@ -167,62 +219,95 @@ __device__ __forceinline__ RowScale scale_of_row(const Part& p, float n, float e
     else { const float rr = fast_rsqrt(fast_div(p.a, n) + eps); return RowScale{rr, rr}; }
 }
 
-// Pass B over `nvec` vectors: xs/ys point at the segment, g/b at the parameters of its first column.
-// live_end: this thread's Running::live_end when the same thread ran pass A over the same vectors (softmax): vectors
-// from there on are known to be all -inf, so their zeros are written without reading x again.
+// The normalised form of one vector: softmax 2^(x log2e + O) / S (ta2 = O, tb2 = 1/S; -inf elements need no test:
+// 2^(-inf) is +0, and +0 times 1/S is +0), LayerNorm (x - mean) rstd gamma + beta, RMSNorm x rrms w.
+// g, b: the parameter vectors of this column (read only for the norms).
 template <int OP, int DT>
+__device__ __forceinline__ uint4 apply_vec(const uint4& raw, const uint4* g, const uint4* b, const F2 ta2, const F2 tb2) {
+    using P = Pairs<DT>;
+    constexpr int NP = P::NP;
+    F2 w[NP];
+    P::unpack(raw, w);
+    if constexpr (OP == OP_SOFTMAX) {
+        const F2 l2e = f2(kLog2e);
+#pragma unroll
+        for (int i = 0; i < NP; ++i) w[i] = mul2(ex2_ftz2(fma2(w[i], l2e, ta2)), tb2);
+    } else if constexpr (OP == OP_LAYERNORM) {
+        F2 gg[NP], bb[NP];
+        P::unpack(ld_param(g), gg);
+        P::unpack(ld_param(b), bb);
+#pragma unroll
+        for (int i = 0; i < NP; ++i) w[i] = fma2(mul2(sub2(w[i], ta2), tb2), gg[i], bb[i]);
+    } else {
+        F2 gg[NP];
+        P::unpack(ld_param(g), gg);
+#pragma unroll
+        for (int i = 0; i < NP; ++i) w[i] = mul2(mul2(w[i], ta2), gg[i]);
+    }
+    return P::pack(w);
+}
+
+// One step of pass B: kStreamU vectors of this thread starting at vector idx0 (stride T).  PRED: vectors at or beyond
+// nvec do not exist.  live[u] (softmax): the vector may hold something other than -inf; the others become zeros unread.
+template <int OP, int DT, bool PRED, bool LEN, bool CACHE>
+__device__ __forceinline__ void apply_step(const uint4* xs, uint4* ys, const uint4* g, const uint4* b, int64_t idx0, int T, int64_t nvec,
+                                           const F2 ta2, const F2 tb2, uint64_t policy, const uint4* cache, int64_t cache_vecs,
+                                           const bool (&live)[kStreamU], int64_t straddle, int keep) {
+    constexpr int U = kStreamU;
+    uint4 raw[U];
+    bool ok[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int64_t idx = idx0 + static_cast<int64_t>(u) * T;
+        ok[u] = !PRED || idx < nvec;
+        const bool want = ok[u] && (OP != OP_SOFTMAX || live[u]);
+        if (want) raw[u] = (CACHE && idx < cache_vecs) ? cache[idx] : ld_hint(xs + idx, policy);
+        else raw[u] = fill_vec<DT>(OP);
+        if (LEN && idx == straddle) raw[u] = mask_tail<DT>(raw[u], keep);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        if (!ok[u]) continue;
+        const int64_t idx = idx0 + static_cast<int64_t>(u) * T;
+        uint4 out = make_uint4(0, 0, 0, 0);
+        if (OP != OP_SOFTMAX || live[u]) out = apply_vec<OP, DT>(raw[u], g + idx, b + idx, ta2, tb2);
+        st_stream(ys + idx, out);
+    }
+}
+
+// Pass B over `nvec` vectors: xs/ys point at the segment, g/b at the parameters of its first column.
+// live_slots: this thread's Running::live_slots when the same thread ran pass A over the same vectors (softmax): its
+// vectors from that slot on are known to be all -inf, so their zeros are written without reading x again.
+// A fully masked row (1/S = 0) passes live_slots = 0.
+template <int OP, int DT, bool LEN = false, bool CACHE = false>
 __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const uint4* g, const uint4* b, int64_t nvec,
                                              const RowScale& sc, uint64_t policy, const uint4* cache = nullptr,
-                                             int64_t cache_vecs = 0, int64_t live_end = INT64_MAX, int64_t len = -1) {
-    using P = Pairs<DT>;
-    constexpr int NP = P::NP, U = kStreamU, NE = Elem<DT>::NE;
-    const int64_t straddle = (len >= 0 && len % NE) ? len / NE : -1;      // live_end already ends at ceil(len / NE)
+                                             int64_t cache_vecs = 0, int live_slots = 0x7FFFFFFF, int64_t len = -1) {
+    constexpr int U = kStreamU, NE = Elem<DT>::NE;
+    const int64_t straddle = (LEN && len % NE) ? len / NE : -1;           // live_slots already ends at ceil(len / NE)
+    const int keep = LEN ? static_cast<int>(len % NE) : 0;
     const int T = blockDim.x, t = threadIdx.x;
-    const uint4 fill = fill_vec<DT>(OP);
-    const F2 ta2 = f2(sc.a), tb2 = f2(sc.b), l2e = f2(kLog2e);
+    const F2 ta2 = f2(sc.a), tb2 = f2(sc.b);
     // back to front: the end of the segment is what pass A touched last, hence what L2 most likely still holds
     const int64_t step = static_cast<int64_t>(T) * U;
-    for (int64_t base = (nvec - 1) / step * step + t; base >= 0; base -= step) {
-        uint4 raw[U];
-        bool ok[U];
+    const int nfull = static_cast<int>(nvec / step);
+    if (nfull * step + t < nvec) {                                        // the ragged step
+        bool live[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int64_t idx = base + static_cast<int64_t>(u) * T;
-            ok[u] = idx < nvec;
-            raw[u] = (!ok[u] || idx >= live_end) ? fill : (idx < cache_vecs ? cache[idx] : ld_hint(xs + idx, policy));
-            if (idx == straddle) raw[u] = mask_tail<DT>(raw[u], static_cast<int>(len % NE));
+        for (int u = 0; u < U; ++u) live[u] = nfull * U + u < live_slots;
+        apply_step<OP, DT, true, LEN, CACHE>(xs, ys, g, b, nfull * step + t, T, nvec, ta2, tb2, policy, cache, cache_vecs, live, straddle, keep);
+    }
+    for (int s = nfull - 1; s >= 0; --s) {
+        const int64_t idx0 = s * step + t;
+        if (OP == OP_SOFTMAX && s * U >= live_slots) {                    // nothing but -inf here: zeros, x is not read again
+#pragma unroll
+            for (int u = 0; u < U; ++u) st_stream(ys + idx0 + u * T, make_uint4(0, 0, 0, 0));
+            continue;
         }
+        bool live[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (!ok[u]) continue;
-            const int64_t idx = base + static_cast<int64_t>(u) * T;
-            F2 w[NP];
-            uint4 out = make_uint4(0, 0, 0, 0);
-            if constexpr (OP == OP_SOFTMAX) {
-                if (!all_neg_inf_vec<DT>(raw[u]) && sc.b != 0.f) {
-                    P::unpack(raw[u], w);
-#pragma unroll
-                    for (int i = 0; i < NP; ++i) w[i] = mul2(ex2_ftz2(fma2(w[i], l2e, ta2)), tb2);
-                    out = P::pack(w);
-                }
-            } else if constexpr (OP == OP_LAYERNORM) {
-                F2 gg[NP], bb[NP];
-                P::unpack(raw[u], w);
-                P::unpack(ld_param(g + idx), gg);
-                P::unpack(ld_param(b + idx), bb);
-#pragma unroll
-                for (int i = 0; i < NP; ++i) w[i] = fma2(mul2(sub2(w[i], ta2), tb2), gg[i], bb[i]);
-                out = P::pack(w);
-            } else {
-                F2 gg[NP];
-                P::unpack(raw[u], w);
-                P::unpack(ld_param(g + idx), gg);
-#pragma unroll
-                for (int i = 0; i < NP; ++i) w[i] = mul2(mul2(w[i], ta2), gg[i]);
-                out = P::pack(w);
-            }
-            st_stream(ys + idx, out);
-        }
+        for (int u = 0; u < U; ++u) live[u] = s * U + u < live_slots;
+        apply_step<OP, DT, false, LEN, CACHE>(xs, ys, g, b, idx0, T, nvec, ta2, tb2, policy, cache, cache_vecs, live, straddle, keep);
     }
 }
 

@@ -39,11 +39,17 @@ struct WArgs {
     int64_t cache_vecs;   // vectors at the head of a row (of a CTA's slice of it) parked in shared memory between the passes
     float n, eps;
     int cs;               // CTAs per row (CL builds)
+    int groups;           // row order: launch slot b works on row (b % groups) * ceil(rows / groups) + b / groups
+    int64_t slots;        // groups * ceil(rows / groups)
+    int stages;           // ring form: steps per thread's ring
+    int policy;           // bit 0: pass A loads ask L2 to keep their lines; bit 1: pass B loads let them go
 };
 
 // MAXT / MINB: the launch bounds.  Besides the unconstrained form (1024, 0) there are (768, 2) and (512, 3), which hold
 // the kernel to 40 registers so that 1536 threads are resident per SM instead of 1024-1280.
-template <int OP, int DT, int MAXT, int MINB, bool CL>
+// LEN: softmax with per-row valid lengths; CACHE: the head of each row is parked in shared memory between the passes.
+// Both are compile-time so that the plain build carries neither the length arithmetic nor the cache tests per vector.
+template <int OP, int DT, int MAXT, int MINB, bool CL, bool LEN, bool CACHE>
 __global__ void __launch_bounds__(MAXT, MINB) k_twopass(const WArgs a) {
     constexpr int NE = Elem<DT>::NE;
     __shared__ float red_buf[4 * 32];
@@ -52,24 +58,32 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass(const WArgs a) {
     uint4* const cache = reinterpret_cast<uint4*>(dyn_smem);
     pdl_wait();
     pdl_trigger();
-    const uint64_t keep = policy_evict_last(), last = policy_evict_first();     // pass A keeps x in L2, pass B lets it go
+    // pass A keeps x in L2, pass B lets it go (either hint can be switched off by the plan)
+    const uint64_t keep = (a.policy & 1) ? policy_evict_last() : policy_evict_normal();
+    const uint64_t last = (a.policy & 2) ? policy_evict_first() : policy_evict_normal();
     const int cs = CL ? a.cs : 1;
     const int rank = CL ? static_cast<int>(blockIdx.x % cs) : 0;
-    const int64_t first_row = CL ? blockIdx.x / cs : blockIdx.x, row_step = CL ? gridDim.x / cs : gridDim.x;
+    const int64_t first_slot = CL ? blockIdx.x / cs : blockIdx.x, slot_step = CL ? gridDim.x / cs : gridDim.x;
+    const int64_t per_group = a.slots / a.groups;
     const int64_t per = CL ? (a.nvec + cs - 1) / cs : a.nvec, first = rank * per;        // this CTA's slice of every row
     const int64_t seg = max(int64_t{0}, min(per, a.nvec - first));
     const int64_t cache_vecs = min(a.cache_vecs, seg);
     auto count_of = [&](int k) { return static_cast<float>(max(int64_t{0}, min(per, a.nvec - k * per)) * NE); };
     if constexpr (CL) cg::this_cluster().sync();                  // every CTA of the cluster is resident before any remote write
-    int it = 0;
-    for (int64_t row = first_row; row < a.rows; row += row_step, ++it) {
+    int it = -1;
+    for (int64_t slot = first_slot; slot < a.slots; slot += slot_step) {
+        // neighbouring rows often cost alike (a causal mask grows with the row index): CTAs that run side by side take rows
+        // from `groups` evenly spaced parts of the tensor, so that what is in flight between the passes is an even mix
+        const int64_t row = a.groups > 1 ? (slot % a.groups) * per_group + slot / a.groups : slot;
+        if (row >= a.rows) continue;                               // the same decision in every CTA of a cluster
+        ++it;
         const uint4* xr = a.x + row * a.nvec + first;
         int64_t len = -1;
-        if (OP == OP_SOFTMAX && a.len) {
+        if constexpr (LEN) {
             const int64_t whole = min(max(static_cast<int64_t>(__ldg(a.len + row)), int64_t{0}), a.nvec * NE);
             len = min(max(whole - first * NE, int64_t{0}), seg * NE);
         }
-        const Running<OP, DT> run = stream_stats<OP, DT>(xr, seg, keep, cache, cache_vecs, len);
+        const Running<OP, DT> run = stream_stats<OP, DT, LEN, CACHE>(xr, seg, keep, cache, cache_vecs, len);
         Part part = merge_running<OP, DT>(run, CL ? fmaxf(count_of(rank), 1.f) : a.n, red_buf + 64 * (it & 1));
         if constexpr (CL) {
             cg::cluster_group cl = cg::this_cluster();
@@ -102,48 +116,206 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass(const WArgs a) {
             if (OP == OP_LAYERNORM && a.mean) a.mean[row] = sc.a;
             if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = sc.b;
         }
-        stream_apply<OP, DT>(xr, a.y + row * a.nvec + first, a.p0 + first, a.p1 + first, seg, sc, last, cache, cache_vecs,
-                             OP == OP_SOFTMAX ? run.live_end : INT64_MAX, len);
+        stream_apply<OP, DT, LEN, CACHE>(xr, a.y + row * a.nvec + first, a.p0 + first, a.p1 + first, seg, sc, last, cache, cache_vecs,
+                                         run.live_slots, len);
+    }
+}
+
+// ---- the ring form -------------------------------------------------------------------------------------------
+// The same two passes with the loads decoupled from the arithmetic: every thread keeps a private ring of `stages`
+// steps (U vectors each) in shared memory and fills it with 16-byte asynchronous copies (cp.async) `stages - 1` steps
+// ahead of the step it is working on, so the bytes in flight are the ring, not what a thread's registers hold, and
+// a step's arithmetic overlaps the flight of the following ones.  A slot is written and read by the same thread only,
+// so no barrier guards the ring.  Pass A walks the row back to front and pass B front to back: when pass A ends, the
+// ring holds the first steps of the row, which pass B takes from shared memory without touching L2 again (with a mask
+// at the end of a row, as causal and padded rows have it, that head is the live part).
+__device__ __forceinline__ void cp_async16(uint4* dst, const uint4* src, uint64_t policy) {
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait(int pending) {     // returns once at most `pending` of this thread's groups are in flight
+    switch (pending) {
+        case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+        case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+        case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+        case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+        case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+        case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+        case 6: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
+    }
+}
+constexpr int kRingMaxDepth = 8;
+
+template <int OP, int DT, int U, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
+    constexpr int NE = Elem<DT>::NE;
+    __shared__ float red_buf[4 * 32];
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    uint4* const ring = reinterpret_cast<uint4*>(dyn_smem);              // [stage][u][thread]
+    pdl_wait();
+    pdl_trigger();
+    const uint64_t keep = (a.policy & 1) ? policy_evict_last() : policy_evict_normal();
+    const uint64_t last = (a.policy & 2) ? policy_evict_first() : policy_evict_normal();
+    const int T = blockDim.x, t = threadIdx.x, S = a.stages;
+    const int64_t per_group = a.slots / a.groups;
+    const int64_t step = static_cast<int64_t>(T) * U;
+    const int nsteps = static_cast<int>((a.nvec + step - 1) / step);
+    const uint4 fill = fill_vec<DT>(OP);
+    int it = -1;
+    for (int64_t slot = blockIdx.x; slot < a.slots; slot += gridDim.x) {
+        const int64_t row = a.groups > 1 ? (slot % a.groups) * per_group + slot / a.groups : slot;
+        if (row >= a.rows) continue;
+        ++it;
+        const uint4* xr = a.x + row * a.nvec;
+        uint4* yr = a.y + row * a.nvec;
+        // the copies of step s into its ring slot; vectors behind the end of the row get the fill value instead
+        auto issue = [&](int s, uint64_t policy) {
+            uint4* dst = ring + static_cast<size_t>(s % S) * step + t;
+            const int64_t idx0 = s * step + t;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (idx0 + u * T < a.nvec) cp_async16(dst + u * T, xr + idx0 + u * T, policy);
+                else dst[u * T] = fill;
+            }
+        };
+        // ---- pass A, back to front
+        Running<OP, DT, U> run;
+        for (int k = 0; k < S - 1; ++k) {
+            if (nsteps - 1 - k >= 0) issue(nsteps - 1 - k, keep);
+            cp_async_commit();
+        }
+        for (int s = nsteps - 1; s >= 0; --s) {
+            if (s - (S - 1) >= 0) issue(s - (S - 1), keep);
+            cp_async_commit();
+            cp_async_wait(S - 1);
+            const uint4* src = ring + static_cast<size_t>(s % S) * step + t;
+            uint4 raw[U];
+            bool ok[U];
+            int count = 0;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                raw[u] = src[u * T];
+                ok[u] = s * step + t + u * T < a.nvec;                   // only the last step of a row can be ragged
+                count += ok[u] ? NE : 0;
+            }
+            if (count == U * NE) run.template update<false>(raw, ok, count, s * U);
+            else if (count > 0) run.template update<true>(raw, ok, count, s * U);
+        }
+        const Part part = merge_running<OP, DT, U>(run, a.n, red_buf + 64 * (it & 1));
+        const RowScale sc = scale_of_row<OP>(part, a.n, a.eps);
+        if (t == 0) {
+            if (OP == OP_LAYERNORM && a.mean) a.mean[row] = sc.a;
+            if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = sc.b;
+        }
+        // ---- pass B, front to back: steps 0 .. S-1 are still in the ring
+        const F2 ta2 = f2(sc.a), tb2 = f2(sc.b);
+        const int live_steps = OP == OP_SOFTMAX ? (run.live_slots + U - 1) / U : nsteps;      // steps from here on hold nothing but -inf
+        for (int s = 0; s < nsteps; ++s) {
+            const int sn = s + S - 1;
+            if (s >= 1 && sn < live_steps) issue(sn, last);              // the slot of step s - 1 is free
+            cp_async_commit();
+            const int64_t idx0 = s * step + t;
+            if (s >= live_steps) {                                       // zeros; x is not read again
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (idx0 + u * T < a.nvec) st_stream(yr + idx0 + u * T, make_uint4(0, 0, 0, 0));
+                continue;
+            }
+            cp_async_wait(S - 1);
+            const uint4* src = ring + static_cast<size_t>(s % S) * step + t;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int64_t idx = idx0 + u * T;
+                if (idx < a.nvec) {
+                    uint4 out = make_uint4(0, 0, 0, 0);
+                    if (OP != OP_SOFTMAX || s * U + u < run.live_slots) out = apply_vec<OP, DT>(src[u * T], a.p0 + idx, a.p1 + idx, ta2, tb2);
+                    st_stream(yr + idx, out);
+                }
+            }
+        }
+        cp_async_wait(0);
     }
 }
 
 using TwoFn = void (*)(const WArgs);
 
-template <int MAXT, int MINB, bool CL>
-TwoFn two_fn_b(int op, int dt) {
+template <int MAXT, int MINB, bool CL, bool CACHE>
+TwoFn two_fn_c(int op, int dt, bool len) {
+    if (len) {
+        if (op != OP_SOFTMAX) return nullptr;
+        return dt == DT_F32 ? k_twopass<OP_SOFTMAX, DT_F32, MAXT, MINB, CL, true, CACHE> : k_twopass<OP_SOFTMAX, DT_BF16, MAXT, MINB, CL, true, CACHE>;
+    }
     switch (op * 2 + dt) {
-        case 0: return k_twopass<OP_SOFTMAX, DT_F32, MAXT, MINB, CL>;
-        case 1: return k_twopass<OP_SOFTMAX, DT_BF16, MAXT, MINB, CL>;
-        case 2: return k_twopass<OP_LAYERNORM, DT_F32, MAXT, MINB, CL>;
-        case 3: return k_twopass<OP_LAYERNORM, DT_BF16, MAXT, MINB, CL>;
-        case 4: return k_twopass<OP_RMSNORM, DT_F32, MAXT, MINB, CL>;
-        case 5: return k_twopass<OP_RMSNORM, DT_BF16, MAXT, MINB, CL>;
+        case 0: return k_twopass<OP_SOFTMAX, DT_F32, MAXT, MINB, CL, false, CACHE>;
+        case 1: return k_twopass<OP_SOFTMAX, DT_BF16, MAXT, MINB, CL, false, CACHE>;
+        case 2: return k_twopass<OP_LAYERNORM, DT_F32, MAXT, MINB, CL, false, CACHE>;
+        case 3: return k_twopass<OP_LAYERNORM, DT_BF16, MAXT, MINB, CL, false, CACHE>;
+        case 4: return k_twopass<OP_RMSNORM, DT_F32, MAXT, MINB, CL, false, CACHE>;
+        case 5: return k_twopass<OP_RMSNORM, DT_BF16, MAXT, MINB, CL, false, CACHE>;
     }
     return nullptr;
 }
 
-TwoFn two_fn(int op, int dt, int threads, bool capped, bool cl) {
-    if (capped && threads <= 512) return cl ? two_fn_b<512, 3, true>(op, dt) : two_fn_b<512, 3, false>(op, dt);
-    if (capped && threads <= 768) return cl ? two_fn_b<768, 2, true>(op, dt) : two_fn_b<768, 2, false>(op, dt);
-    return cl ? two_fn_b<1024, 0, true>(op, dt) : two_fn_b<1024, 0, false>(op, dt);
+template <int MAXT, int MINB>
+TwoFn two_fn_b(int op, int dt, bool cl, bool len, bool cache) {
+    if (cl) return cache ? two_fn_c<MAXT, MINB, true, true>(op, dt, len) : two_fn_c<MAXT, MINB, true, false>(op, dt, len);
+    return cache ? two_fn_c<MAXT, MINB, false, true>(op, dt, len) : two_fn_c<MAXT, MINB, false, false>(op, dt, len);
+}
+
+TwoFn two_fn(int op, int dt, int threads, bool capped, bool cl, bool len, bool cache) {
+    if (capped && threads <= 512) return two_fn_b<512, 3>(op, dt, cl, len, cache);
+    if (capped && threads <= 768) return two_fn_b<768, 2>(op, dt, cl, len, cache);
+    return two_fn_b<1024, 0>(op, dt, cl, len, cache);
+}
+
+template <int U, int MAXT, int MINB>
+TwoFn ring_fn_b(int op, int dt) {
+    switch (op * 2 + dt) {
+        case 0: return k_twopass_ring<OP_SOFTMAX, DT_F32, U, MAXT, MINB>;
+        case 1: return k_twopass_ring<OP_SOFTMAX, DT_BF16, U, MAXT, MINB>;
+        case 2: return k_twopass_ring<OP_LAYERNORM, DT_F32, U, MAXT, MINB>;
+        case 3: return k_twopass_ring<OP_LAYERNORM, DT_BF16, U, MAXT, MINB>;
+        case 4: return k_twopass_ring<OP_RMSNORM, DT_F32, U, MAXT, MINB>;
+        case 5: return k_twopass_ring<OP_RMSNORM, DT_BF16, U, MAXT, MINB>;
+    }
+    return nullptr;
+}
+// regcap: the builds held to 40 registers (three CTAs of 512 threads, or four of 384, per SM)
+TwoFn ring_fn(int op, int dt, int unroll, int threads, bool capped) {
+    if (unroll == 2) return (capped && threads <= 512) ? ring_fn_b<2, 512, 3>(op, dt) : ring_fn_b<2, 1024, 1>(op, dt);
+    if (unroll == 4) return (capped && threads <= 512) ? ring_fn_b<4, 512, 3>(op, dt) : ring_fn_b<4, 1024, 1>(op, dt);
+    return nullptr;
 }
 
 }  // namespace
 
 // Plan field `chunk`: bytes of each row's head kept in shared memory between the passes (0 = none); `rpg` = 2 selects
-// the register-capped build (threads <= 768).
+// the register-capped build (threads <= 768); `lanes`: row-order groups; `vpt`: L2 hint bits of the two passes.
 bool supports_twopass(const Plan& p, const Args& a, const DeviceInfo& d) {
     if (p.cluster != 1 && p.cluster != 2 && p.cluster != 4 && p.cluster != 8) return false;
     if (p.cluster > 1 && (p.cluster > d.max_cluster || a.cols * elem_size(a.dt) / 16 < p.cluster || a.rows * p.cluster > 0x7FFFFFFF)) return false;
+    if (p.lanes < 1 || p.lanes > 1024 || p.vpt < 0 || p.vpt > 3) return false;
+    if (p.stages >= 2) {                                           // the ring form: one CTA per row, no length mode, no separate cache
+        if (p.stages > kRingMaxDepth || (p.unroll != 2 && p.unroll != 4) || p.cluster != 1 || p.chunk != 0 || a.len) return false;
+        const int64_t nvec = a.cols * elem_size(a.dt) / 16;
+        if (nvec / (static_cast<int64_t>(p.threads) * p.unroll) > (1 << 24)) return false;
+        return vector_ok(a) && (p.rpg == 1 || p.rpg == 2) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0 &&
+               (d.smem_optin == 0 || static_cast<int64_t>(p.stages) * p.threads * p.unroll * 16 + 1024 <= d.smem_optin);
+    }
+    if (p.stages != 0 && p.stages != 1) return false;
     return vector_ok(a) && (p.rpg == 1 || (p.rpg == 2 && p.threads <= 768)) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0 && p.chunk >= 0 && p.chunk % 16 == 0 &&
            (d.smem_optin == 0 || p.chunk + 2048 <= d.smem_optin);
 }
 
 cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
     const int cs = std::max(1, p.cluster);
-    TwoFn fn = two_fn(a.op, a.dt, p.threads, p.rpg == 2, cs > 1);
+    const bool ring = p.stages >= 2;
+    TwoFn fn = ring ? ring_fn(a.op, a.dt, p.unroll, p.threads, p.rpg == 2) : two_fn(a.op, a.dt, p.threads, p.rpg == 2, cs > 1, a.len != nullptr, p.chunk > 0);
     if (!fn) return cudaErrorInvalidValue;
-    int64_t grid = a.rows;                                         // in rows (clusters)
+    const int groups = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(p.lanes, a.rows)));
+    const int64_t slots = (a.rows + groups - 1) / groups * groups;
+    int64_t grid = slots;                                          // in rows (clusters)
     if (p.persist > 0) grid = std::min<int64_t>(grid, std::max<int64_t>(1, static_cast<int64_t>(p.persist) * d.sms / cs));
     grid = std::min<int64_t>(grid, 0x7FFFFFFF / cs);
     WArgs k;
@@ -151,14 +323,16 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
     k.y = static_cast<uint4*>(a.y); k.mean = a.mean; k.rstd = a.rstd; k.rows = a.rows; k.len = a.len;
     k.nvec = a.cols * elem_size(a.dt) / 16;
     k.n = static_cast<float>(a.cols); k.eps = a.eps;
-    k.cs = cs;
+    k.cs = cs; k.groups = groups; k.slots = slots; k.policy = p.vpt;
     k.cache_vecs = std::min<int64_t>((k.nvec + cs - 1) / cs, p.chunk / 16);
-    if (p.chunk > 0) {
+    k.stages = p.stages;
+    const size_t smem = ring ? static_cast<size_t>(p.stages) * p.threads * p.unroll * 16 : static_cast<size_t>(k.cache_vecs) * 16;
+    if (smem > 0) {
         cudaError_t e = ensure_max_smem(reinterpret_cast<const void*>(fn), d);
         if (e != cudaSuccess) return e;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.dynamicSmemBytes = static_cast<size_t>(k.cache_vecs) * 16;
+    cfg.dynamicSmemBytes = smem;
     cfg.gridDim = dim3(static_cast<unsigned>(grid * cs));
     cfg.blockDim = dim3(p.threads);
     cfg.stream = st;

@@ -263,8 +263,23 @@ def test_forced_twopass_variants(op, dt):
             tf.tf_force_plan(op, f"twopass:threads={threads},cache={cache},persist={persist},regcap={regcap},cluster={cluster}")
             fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec + cluster))
             assert not fails, (cluster, threads, persist, regcap, cache, nvec, rows, fails)
+    # the ring form (asynchronous copies into a private shared-memory ring): rows shorter than the ring, exactly one ring,
+    # ragged last steps, rows taken in interleaved order, every hint combination, persistent grids
+    for threads, stages, u, persist, regcap, groups, hints in ((32, 2, 4, 0, 0, 1, 3), (256, 3, 2, 1, 1, 8, 0), (512, 2, 4, 0, 1, 3, 1),
+                                                               (1024, 2, 2, 0, 0, 1, 2), (384, 4, 4, 2, 1, 16, 3), (128, 8, 2, 0, 1, 2, 3)):
+        for nvec, rows in ((1, 5), (threads * u, 9), (threads * u * stages, 7), (threads * u * stages + 1, 9), (threads * 9 - 3, 300), (70001, 3)):
+            plan = f"twopass:threads={threads},persist={persist},regcap={regcap},groups={groups},hints={hints},stages={stages},u={u}"
+            tf.tf_force_plan(op, plan)
+            fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec + stages))
+            assert not fails, (plan, nvec, rows, fails)
+            fails = parity.parity(wl(op, dt, min(rows, 11), nvec * ne, seed=nvec + stages), inplace=True)
+            assert not fails, ("in place", plan, nvec, rows, fails)
+    for groups in (2, 8, 1000):                            # the direct form with interleaved row order
+        tf.tf_force_plan(op, f"twopass:threads=256,persist=0,groups={groups},hints=0")
+        assert not parity.parity(wl(op, dt, 37, 5000 * ne, seed=groups)), groups
     if op == "softmax":                                    # masks, a fully masked row and outputs in the subnormal range
-        for plan in ("twopass:threads=256,persist=0,cluster=4", "twopass:threads=512,cache=8192,persist=0,regcap=1,cluster=8"):
+        for plan in ("twopass:threads=256,persist=0,cluster=4", "twopass:threads=512,cache=8192,persist=0,regcap=1,cluster=8",
+                     "twopass:threads=256,persist=0,stages=2,u=4", "twopass:threads=128,persist=0,regcap=1,stages=3,u=2,groups=4"):
             tf.tf_force_plan(op, plan)
             w = Workload("m", "softmax", dt, 12, 40000, seed=5, x_std=10.0, mask_step=3001)
             data = w.generate()
