@@ -2,13 +2,16 @@
 """Benchmark of the row-wise reduce-then-normalise library on B200.
 
 Default run (``python bench.py [--gpus N --steps K --warmup W]``): one step = one pass of the hot path
-(``tf_layernorm_fwd`` through the C ABI) over one bf16 [8192, 4096] batch that is already resident in HBM.
-Prints ONE JSON line: achieved HBM GB/s (algorithmic bytes / device time), the roofline fraction against the
-measured copy bandwidth of this machine, the end-to-end figure with host<->device copies inside the timed region, and
-the CPU oracle timed on this machine's host cores as a reported baseline.
+(``tf_softmax_fwd`` through the C ABI) over the largest fixed configuration, the tail-masked bf16 softmax
+[4096, 131072] (2 GiB of algorithmic bytes per step), already resident in HBM.  The timed span is R back-to-back
+regions of K steps each with an event between regions and no synchronisation inside; the line reports the median
+region and the spread.  Prints ONE JSON line: achieved HBM GB/s (algorithmic bytes / device time), the roofline
+fraction against the measured copy bandwidth of this machine, the end-to-end figure with host<->device copies inside the
+timed region, the CPU oracle timed on this machine's host cores as a reported baseline, and (one GPU only) a record per
+fixed configuration (``per_config``) and a summary of the 84-point shape sweep (``sweep_summary``).
 
 ``--impl reference`` times the CPU oracle alone (the reference arm).
-``--table configs|sweep`` measures the other configurations / the shape sweep and writes a table (not a bench line).
+``--table configs|sweep|...`` measure tables (not bench lines) and write them under ``--out``.
 """
 from __future__ import annotations
 
@@ -27,14 +30,20 @@ sys.path.insert(0, str(ROOT))
 NOMINAL_HBM_GBS = 8000.0          # the "~8 TB/s" the 80% bar is quoted against
 FALLBACK_HBM_GBS = 6650.0         # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
 L2_BYTES = 126 << 20
+HEADLINE_CONFIG = 3               # the largest fixed configuration that fits one GPU: masked softmax bf16 [4096, 131072]
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
-# profiles/; None until a capture of that kernel exists.
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel of each fixed
+# configuration, from profiler captures of cases too large for the 126 MB L2 to hide the writes; None where no capture
+# exists.  Value = (bytes of the captured case, factor to a full launch of the configuration).
 NCU_TRAFFIC_BYTES = {
-    # profiles/k_pipe_layernorm_bf16_8192x4096.md: 67.16 MB read (= the algorithmic reads) + 9.48 MB written inside the
-    # kernel; the other 57.7 MB of y are still dirty in the 126 MB L2 when an isolated launch ends
-    "layernorm_bf16_8192x4096": 67157760 + 9477888,
+    # LayerNorm bf16 [32768, 4096] (four times the rows of the configuration): 268.5 MB read + 210.8 MB written
+    "layernorm_bf16_8192x4096": (268_497_408 + 210_806_400, 0.25),
 }
+
+
+def traffic_of(name):
+    t = NCU_TRAFFIC_BYTES.get(name)
+    return None if t is None else int(t[0] * t[1])
 
 
 def measured_peak():
@@ -153,6 +162,30 @@ class DeviceCase:
         else:
             tf.tf_rmsnorm_fwd(self.x[k], self.params["w"], w.eps, self.y[k])
 
+    def time_regions(self, steps: int, regions: int, warmup: int, step=None):
+        """`regions` back-to-back regions of `steps` launches each, an event between regions, no synchronisation inside.
+        Returns the region times in milliseconds."""
+        torch = self.torch
+        step = step or self.step
+        for _ in range(warmup):
+            step()
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(regions + 1)]
+        torch.cuda.synchronize()
+        evs[0].record()
+        for r in range(regions):
+            for _ in range(steps):
+                step()
+            evs[r + 1].record()
+        torch.cuda.synchronize()
+        return [evs[r].elapsed_time(evs[r + 1]) for r in range(regions)]
+
+    def copy_step(self):
+        """The library's own streaming copy of the same tensors (x -> y): the practical ceiling at this size."""
+        import paper_2512_09196_b200 as tf
+        k = self.i % self.sets
+        self.i += 1
+        tf.tf_copy(self.x[k], self.y[k])
+
     def time_steps(self, steps: int, warmup: int) -> float:
         """Milliseconds for `steps` back-to-back launches (CUDA events on the launching stream)."""
         torch = self.torch
@@ -168,10 +201,19 @@ class DeviceCase:
         return a.elapsed_time(b)
 
 
-def time_oracle(w, data, rows: int, reps: int = 1) -> float:
-    """Seconds (best of reps) for the single-threaded oracle on the first `rows` rows."""
+def sample_rows(w, n: int):
+    """n row indices spread evenly over the workload (the tail mask of the 2 GiB softmax grows with the row index, so
+    the first rows alone would not be a fair sample)."""
+    import numpy as np
+    n = max(1, min(n, w.rows))
+    return np.unique((np.arange(n, dtype=np.int64) * w.rows) // n)
+
+
+def time_oracle(w, data, rows, reps: int = 1) -> float:
+    """Seconds (best of reps) for the single-threaded oracle on the given rows (a count = the first rows, or indices)."""
+    import numpy as np
     import oracle
-    x = data["x"][:rows]
+    x = data["x"][:rows] if isinstance(rows, (int, np.integer)) else np.ascontiguousarray(data["x"][rows])
     best = float("inf")
     for _ in range(reps):
         t0 = time.perf_counter()
@@ -185,16 +227,17 @@ def time_oracle(w, data, rows: int, reps: int = 1) -> float:
     return best
 
 
-def cpu_baseline(w, data, budget_s: float = 15.0) -> dict:
-    """The oracle as it stands, one thread, on a bounded sample of the workload."""
-    probe_rows = max(1, min(w.rows, 64))
-    t_probe = max(time_oracle(w, data, probe_rows), 1e-6)
-    rows = int(max(1, min(w.rows, probe_rows * budget_s / 3 / t_probe)))
-    reps = 3 if rows == w.rows else 1
+def cpu_baseline(w, data, budget_s: float = 12.0) -> dict:
+    """The oracle as it stands, one thread, on a bounded sample of the workload: rows spread evenly over it."""
+    probe = sample_rows(w, 16)
+    t_probe = max(time_oracle(w, data, probe), 1e-6) / len(probe)
+    n = int(max(1, min(w.rows, budget_s / 2 / t_probe)))
+    rows = sample_rows(w, n)
+    reps = 3 if len(rows) == w.rows and t_probe * w.rows * 3 < budget_s else 1
     t = time_oracle(w, data, rows, reps)
-    gbs = w.algorithmic_bytes(rows) / t / 1e9
-    sample = (f"full batch [{rows}, {w.cols}], best of {reps}" if rows == w.rows
-              else f"first {rows} of {w.rows} rows, one pass, scaled per byte")
+    gbs = w.algorithmic_bytes(len(rows)) / t / 1e9
+    sample = (f"full batch [{w.rows}, {w.cols}], best of {reps}" if len(rows) == w.rows
+              else f"{len(rows)} of {w.rows} rows spread evenly over the batch, one pass, GB/s of those rows' bytes")
     return {"value": gbs, "unit": "GB/s", "cores": 1, "cores_available": os.cpu_count(), "kind": "oracle", "sample": sample,
             "seconds": t}
 
@@ -249,6 +292,72 @@ def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
 
+def _spread(ms_regions, steps):
+    """Median / min / max time per step over the timed regions."""
+    per = sorted(m / steps for m in ms_regions)
+    return per[len(per) // 2], per[0], per[-1]
+
+
+def _tune_or_query(tf, w, case, no_tune):
+    like = (case.x[0], case.params.get("gamma", case.params.get("w")), case.params.get("beta"))
+    if no_tune:
+        return {"plan": tf.tf_query_choice(w.op, w.rows, w.cols, w.dt), "timed": 0}
+    return tf.tf_tune(w.op, w.rows, w.cols, w.dt, like=like)
+
+
+def measure_config(tf, w, data, device, peak, no_tune, regions=25):
+    """One fixed configuration: tuned plan, `regions` regions sized to a few milliseconds each, and the library's own
+    streaming copy of the same tensors as the ceiling at that size."""
+    case = DeviceCase(w, data, device)
+    tuned = _tune_or_query(tf, w, case, no_tune)
+    est = max(case.bytes_per_step / 6e12, 2e-6)
+    steps = int(max(4, min(2000, 3e-3 / est)))
+    med, lo, hi = _spread(case.time_regions(steps, regions, 5), steps)
+    cmed, _, _ = _spread(case.time_regions(steps, 7, 3, step=case.copy_step), steps)
+    gbs = case.bytes_per_step / (med * 1e-3) / 1e9
+    copy_bytes = 2 * case.x[0].numel() * case.x[0].element_size()
+    rec = {"workload": w.name, "op": w.op, "storage": w.dtype_name, "rows": w.rows, "cols": w.cols,
+           "algorithmic_bytes": case.bytes_per_step, "plan": tuned["plan"], "us_per_launch": 1e3 * med,
+           "us_min": 1e3 * lo, "us_max": 1e3 * hi, "launches_per_region": steps, "regions": regions, "gbs": gbs,
+           "frac": gbs / peak, "pct_of_nominal_8000": 100 * gbs / NOMINAL_HBM_GBS,
+           "tf_copy_gbs": copy_bytes / (cmed * 1e-3) / 1e9, "traffic": traffic_of(w.name),
+           "tune": {k: tuned[k] for k in tuned if k != "plan"},
+           "l2": f"rotating {case.sets} buffer sets ({case.sets * case.footprint / 1e9:.2f} GB)"}
+    if case.footprint <= L2_BYTES // 4:
+        rec["note"] = "latency-bound: the whole problem is a fraction of L2 and takes a few microseconds"
+    return rec, case
+
+
+def sweep_summary(tf, device, peak, tune: bool):
+    """The 84-point shape sweep (256 MiB of input per point) in one pass: GB/s per point, how many reach 80 % of the
+    nominal 8 TB/s, and the worst point.  x depends on (type, width) only, so it is generated once per pair."""
+    import torch
+    from paper_2512_09196_b200 import inputs
+    pts, cache = [], {}
+    for w in inputs.sweep():
+        key = (w.dt, w.cols)
+        if key not in cache:
+            cache.clear()
+            cache[key] = w.generate()["x"]
+        data = dict(w.generate(0, 0), x=cache[key])
+        case = DeviceCase(w, data, device)
+        tf.tf_clear_cache()
+        plan = _tune_or_query(tf, w, case, not tune)["plan"]
+        steps = 20
+        med, lo, hi = _spread(case.time_regions(steps, 5, 4), steps)
+        gbs = case.bytes_per_step / (med * 1e-3) / 1e9
+        pts.append({"workload": w.name, "us": 1e3 * med, "gbs": gbs, "plan": plan})
+        del case
+        torch.cuda.empty_cache()
+    tf.tf_clear_cache()
+    worst = min(pts, key=lambda r: r["gbs"])
+    srt = sorted(r["gbs"] for r in pts)
+    return {"points": len(pts), "input_bytes_per_point": inputs.SWEEP_BYTES, "plans": "tf_tune per point" if tune else "untuned defaults",
+            "reach_6400": sum(r["gbs"] >= 0.8 * NOMINAL_HBM_GBS for r in pts), "reach_90pct_of_peak": sum(r["gbs"] >= 0.9 * peak for r in pts),
+            "median_gbs": srt[len(srt) // 2], "worst": worst,
+            "below_6400": [{"workload": r["workload"], "gbs": round(r["gbs"], 1)} for r in sorted(pts, key=lambda r: r["gbs"]) if r["gbs"] < 0.8 * NOMINAL_HBM_GBS]}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -263,43 +372,48 @@ def run_ours(args):
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=device)
+    peak, peak_kind = measured_peak()
 
     # weak scaling: every rank owns one full batch (rows are independent; there is no exchange step)
-    base = inputs.config(1)
+    base = inputs.config(HEADLINE_CONFIG)
     w = inputs.Workload(base.name, base.op, base.dt, base.rows, base.cols, seed=base.seed + 1000 * rank, x_mean=base.x_mean,
-                        x_std=base.x_std, eps=base.eps, scale=base.scale, shift=base.shift)
+                        x_std=base.x_std, eps=base.eps, outlier_p=base.outlier_p, outlier_factor=base.outlier_factor,
+                        mask_step=base.mask_step, scale=base.scale, shift=base.shift)
     data = w.generate()
     case = DeviceCase(w, data, device)
-    like = (case.x[0], case.params.get("gamma", case.params.get("w")), case.params.get("beta"))
-    tuned = tf.tf_tune(w.op, w.rows, w.cols, w.dt, like=like) if not args.no_tune else {"plan": tf.tf_query_choice(w.op, w.rows, w.cols, w.dt)}
+    tuned = _tune_or_query(tf, w, case, args.no_tune)
 
     steps, warmup = args.steps, max(args.warmup, 3)
+    # R regions of `steps` launches each: at least 25, and enough of them for about 100 ms of device time
+    est_ms = 1e3 * case.bytes_per_step / 6e12
+    regions = int(max(25, min(400, 100.0 / max(steps * est_ms, 1e-3))))
     for _ in range(warmup):
         case.step()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(regions + 1)]
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     launches0 = tf.tf_launch_count()
     with ClockSampler(local_rank) as clk:
         torch.cuda.nvtx.range_push("BIG_OP")         # the label the paper's profiling step filters on (Section 3.3)
-        start.record()
-        for _ in range(steps):
-            case.step()
-        end.record()
+        evs[0].record()
+        for r in range(regions):
+            for _ in range(steps):
+                case.step()
+            evs[r + 1].record()
         torch.cuda.synchronize()
         torch.cuda.nvtx.range_pop()
     launches = tf.tf_launch_count() - launches0
-    ms = start.elapsed_time(end)
+    med, lo, hi = _spread([evs[r].elapsed_time(evs[r + 1]) for r in range(regions)], steps)
     if world > 1:
-        t = torch.tensor([ms], device=device, dtype=torch.float64)
+        t = torch.tensor([med, lo, hi], device=device, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.barrier()
-        ms = float(t.item())
+        med, lo, hi = (float(v) for v in t.tolist())
     tf.tf_device_status()
 
-    e2e_steps = max(3, min(steps, 20))
-    blocks = 2              # per-block enqueue cost outweighs finer overlap once consecutive steps overlap (measured 1-32)
+    e2e_steps = max(3, min(steps, 6))
+    blocks = 4
     e2e_ms, h2d, d2h = time_e2e(w, data, device, e2e_steps, 3, blocks)
     if world > 1:
         t = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
@@ -307,22 +421,22 @@ def run_ours(args):
         e2e_ms = float(t.item())
 
     if rank == 0:
-        peak, peak_kind = measured_peak()
         bytes_step = case.bytes_per_step
-        value = world * bytes_step * steps / (ms * 1e-3) / 1e9
-        per_launch_gbs = bytes_step / (ms * 1e-3 / steps) / 1e9
+        per_launch_gbs = bytes_step / (med * 1e-3) / 1e9
         line = {
-            "metric": "achieved HBM GB/s (algorithmic bytes / device time)", "value": value, "unit": "GB/s",
-            "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms / steps, "higher_is_better": True,
+            "metric": "achieved HBM GB/s (algorithmic bytes / device time)", "value": world * per_launch_gbs, "unit": "GB/s",
+            "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": med, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "op": w.op, "storage": w.dtype_name, "rows_per_gpu": w.rows, "cols": w.cols,
                        "algorithmic_bytes_per_step": bytes_step, "plan": tuned["plan"],
                        "l2": f"rotating {case.sets} buffer sets ({case.sets * case.footprint / 1e9:.2f} GB) > 126 MB L2",
                        "sharding": "independent row batches per GPU, no collective"},
+            "timing": {"regions": regions, "steps_per_region": steps, "statistic": "median region / steps",
+                       "ms_per_step_min": lo, "ms_per_step_max": hi, "spread_pct": 100 * (hi - lo) / med},
             "pct_of_nominal_8000": 100 * per_launch_gbs / NOMINAL_HBM_GBS,
             "pct_of_measured_peak": 100 * per_launch_gbs / peak,
             "roofline": {"bound": "hbm", "achieved": per_launch_gbs, "peak": peak, "peak_kind": f"of {peak_kind}",
-                         "unit": "GB/s", "frac": per_launch_gbs / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+                         "unit": "GB/s", "frac": per_launch_gbs / peak, "traffic": traffic_of(w.name)},
             "e2e": {"value": world * bytes_step * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                     "ms_per_step": e2e_ms / e2e_steps,
@@ -332,36 +446,67 @@ def run_ours(args):
             "tune": {k: tuned[k] for k in tuned if k != "plan"},
         }
         line["cpu_baseline"] = cpu_baseline(w, data) if world == 1 else None
+        if world == 1 and not args.no_extras:
+            del case
+            torch.cuda.empty_cache()
+            per = []
+            for i in range(4):
+                if i == HEADLINE_CONFIG:
+                    per.append({"workload": w.name, "op": w.op, "storage": w.dtype_name, "rows": w.rows, "cols": w.cols,
+                                "algorithmic_bytes": bytes_step, "plan": tuned["plan"], "us_per_launch": 1e3 * med, "us_min": 1e3 * lo,
+                                "us_max": 1e3 * hi, "launches_per_region": steps, "regions": regions, "gbs": per_launch_gbs,
+                                "frac": per_launch_gbs / peak, "pct_of_nominal_8000": 100 * per_launch_gbs / NOMINAL_HBM_GBS,
+                                "tf_copy_gbs": None, "traffic": traffic_of(w.name), "note": "the headline measurement above"})
+                    continue
+                wi = inputs.config(i)
+                rec, c = measure_config(tf, wi, wi.generate(), device, peak, args.no_tune)
+                per.append(rec)
+                del c
+                torch.cuda.empty_cache()
+            # the copy ceiling of the headline configuration, on fresh buffers
+            hc = DeviceCase(w, data, device)
+            cm, _, _ = _spread(hc.time_regions(10, 7, 3, step=hc.copy_step), 10)
+            per[HEADLINE_CONFIG]["tf_copy_gbs"] = 2 * hc.x[0].numel() * hc.x[0].element_size() / (cm * 1e-3) / 1e9
+            del hc
+            torch.cuda.empty_cache()
+            line["per_config"] = per
+            line["sweep_summary"] = sweep_summary(tf, device, peak, args.sweep_tune)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
 def run_reference(args):
-    """The reference arm: the CPU oracle, as it stands, on this machine's host cores."""
+    """The reference arm: the CPU oracle, as it stands, on this machine's host cores, on the headline workload; every step is a
+    bounded sample of it (rows spread evenly over the batch)."""
     rank, _, world = dist_env()
     if rank != 0:
         return
+    import numpy as np
     from paper_2512_09196_b200 import inputs
-    w = inputs.config(1)
-    data = w.generate()
+    w = inputs.config(HEADLINE_CONFIG)
     steps, warmup = args.steps, args.warmup
-    probe = max(time_oracle(w, data, 64), 1e-6) / 64                      # seconds per row
+    # a quarter of a second per step, found on a few rows first; only the sampled rows are generated
+    probe_rows = sample_rows(w, 4)
+    probe = {"x": np.concatenate([w.generate(int(r), 1)["x"] for r in probe_rows])}
+    per_row = max(time_oracle(w, probe, len(probe_rows)), 1e-6) / len(probe_rows)
     budget = 120.0 / max(1, steps + warmup)
-    rows = int(max(1, min(w.rows, min(0.25, budget) / probe)))
+    rows = sample_rows(w, int(max(1, min(w.rows, min(0.25, budget) / per_row))))
+    data = {"x": np.concatenate([w.generate(int(r), 1)["x"] for r in rows])}
+    n = len(rows)
     for _ in range(warmup):
-        time_oracle(w, data, rows)
+        time_oracle(w, data, n)
     t0 = time.perf_counter()
     for _ in range(steps):
-        time_oracle(w, data, rows)
+        time_oracle(w, data, n)
     sec = time.perf_counter() - t0
-    value = w.algorithmic_bytes(rows) * steps / sec / 1e9
-    sample = f"first {rows} of {w.rows} rows per step"
+    value = w.algorithmic_bytes(n) * steps / sec / 1e9
+    sample = f"{n} of {w.rows} rows spread evenly over the batch per step"
     print(json.dumps({
         "impl": "reference", "metric": "achieved HBM GB/s (algorithmic bytes / device time)", "value": value, "unit": "GB/s",
         "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": 1e3 * sec / steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "op": w.op, "storage": w.dtype_name, "rows_per_step": rows, "cols": w.cols},
+        "config": {"workload": w.name, "op": w.op, "storage": w.dtype_name, "rows_per_step": n, "cols": w.cols},
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -384,7 +529,7 @@ def run_table(args):
         points = inputs.sweep()
         if args.filter:
             points = [p for p in points if args.filter in p.name]
-    out_dir = ROOT / "gpurun_out"
+    out_dir = Path(args.out)
     out_dir.mkdir(exist_ok=True)
     rows_out = []
     for w in points:
@@ -447,7 +592,7 @@ def run_vecmat_table(args):
     points = inputs.vecmat_sweep()
     if args.filter:
         points = [p for p in points if args.filter in p.name]
-    out_dir = ROOT / "gpurun_out"
+    out_dir = Path(args.out)
     out_dir.mkdir(exist_ok=True)
 
     def timed(fn, reps):
@@ -519,7 +664,7 @@ def run_addnorm_table(args):
     from paper_2512_09196_b200 import inputs
     torch.cuda.set_device(0)
     peak, peak_kind = measured_peak()
-    out_dir = ROOT / "gpurun_out"
+    out_dir = Path(args.out)
     out_dir.mkdir(exist_ok=True)
     shapes = [("rmsnorm", inputs.BF16, 16384, 4096), ("rmsnorm", inputs.BF16, 16384, 8192), ("rmsnorm", inputs.BF16, 4096, 16384),
               ("rmsnorm", inputs.F32, 8192, 8192), ("layernorm", inputs.BF16, 16384, 4096), ("layernorm", inputs.BF16, 65536, 1024),
@@ -588,7 +733,7 @@ def run_softmaxlen_table(args):
     from paper_2512_09196_b200 import inputs
     torch.cuda.set_device(0)
     peak, peak_kind = measured_peak()
-    out_dir = ROOT / "gpurun_out"
+    out_dir = Path(args.out)
     out_dir.mkdir(exist_ok=True)
     shapes = [("tail 32 r mod cols (the mask of the 2 GiB configuration)", inputs.BF16, 4096, 131072), ("uniform lengths", inputs.BF16, 16384, 8192),
               ("uniform lengths", inputs.F32, 65536, 1024), ("uniform lengths", inputs.BF16, 262144, 256), ("full lengths", inputs.BF16, 16384, 8192)]
@@ -648,7 +793,7 @@ def run_softmax_variants_table(args):
     from paper_2512_09196_b200 import inputs
     torch.cuda.set_device(0)
     peak, peak_kind = measured_peak()
-    out_dir = ROOT / "gpurun_out"
+    out_dir = Path(args.out)
     out_dir.mkdir(exist_ok=True)
     shapes = [(inputs.BF16, 16384, 8192), (inputs.BF16, 32768, 4096), (inputs.F32, 65536, 1024), (inputs.BF16, 524288, 256),
               (inputs.BF16, 8192, 32768), (inputs.F32, 4096, 32768), (inputs.F32, 2048, 131072)]
@@ -701,7 +846,7 @@ def run_launch_table(args):
     import paper_2512_09196_b200 as tf
     from paper_2512_09196_b200 import inputs
     torch.cuda.set_device(0)
-    out_dir = ROOT / "gpurun_out"
+    out_dir = Path(args.out)
     out_dir.mkdir(exist_ok=True)
     sets, per_graph = 8, 32
     bf = torch.bfloat16
@@ -776,7 +921,7 @@ def run_normbwd_table(args):
     from paper_2512_09196_b200 import inputs
     torch.cuda.set_device(0)
     peak, peak_kind = measured_peak()
-    out_dir = ROOT / "gpurun_out"
+    out_dir = Path(args.out)
     out_dir.mkdir(exist_ok=True)
     shapes = [("rmsnorm", inputs.BF16, 16384, 4096), ("rmsnorm", inputs.BF16, 16384, 8192), ("rmsnorm", inputs.F32, 16384, 4096),
               ("layernorm", inputs.BF16, 16384, 4096), ("layernorm", inputs.BF16, 16384, 8192), ("layernorm", inputs.BF16, 65536, 1024),
@@ -848,7 +993,9 @@ def run_normbwd_table(args):
 
 
 def run_case(args):
-    """A few launches of one op/shape (for profiler captures): --case op:dtype:rows:cols or --case config:<i>[:rows]."""
+    """A few launches of one op/shape (for profiler captures): --case op:dtype:rows:cols or --case config:<i>[:rows[:mask_step]]
+    (fewer rows of a fixed configuration; mask_step 128 on 1024 rows of the masked softmax spreads the tail mask over the
+    whole range of lengths, like the full 4096 rows with their step of 32)."""
     import torch
     import paper_2512_09196_b200 as tf
     from paper_2512_09196_b200 import inputs
@@ -962,8 +1109,8 @@ def run_case(args):
         w = inputs.config(int(parts[1]))
         if len(parts) > 2:
             w = inputs.Workload(w.name, w.op, w.dt, int(parts[2]), w.cols, seed=w.seed, x_mean=w.x_mean, x_std=w.x_std, eps=w.eps,
-                                outlier_p=w.outlier_p, outlier_factor=w.outlier_factor, mask_step=w.mask_step, scale=w.scale,
-                                shift=w.shift)
+                                outlier_p=w.outlier_p, outlier_factor=w.outlier_factor,
+                                mask_step=int(parts[3]) if len(parts) > 3 else w.mask_step, scale=w.scale, shift=w.shift)
     else:
         op, dt, rows, cols = parts
         eps = {"softmax": 0.0, "layernorm": 1e-5, "rmsnorm": 1e-6}[op]
@@ -988,6 +1135,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm", "softmaxlen", "softmaxvariants", "normbwd", "launch"], default=None)
     ap.add_argument("--filter", default=None)
+    ap.add_argument("--out", default=str(ROOT / "bench_out"), help="folder for the JSON files the --table modes write")
+    ap.add_argument("--no-extras", action="store_true", help="default run: skip per_config and sweep_summary")
+    ap.add_argument("--sweep-tune", action="store_true", help="default run: tune every sweep point before timing it")
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
     ap.add_argument("--case", default=None, help="op:dtype:rows:cols, config:<i>[:rows], vecmat:..., addnorm:op:dtype:rows:cols, normbwd:op:dtype:rows:cols, softmaxlen:dtype:rows:cols -- a few launches of one shape")
@@ -997,8 +1147,8 @@ def main():
         args.steps = 10 if args.steps is None else args.steps
         args.warmup = 3 if args.warmup is None else args.warmup
         return run_reference(args)
-    args.steps = 5000 if args.steps is None else args.steps
-    args.warmup = 50 if args.warmup is None else args.warmup
+    args.steps = 20 if args.steps is None else args.steps
+    args.warmup = 5 if args.warmup is None else args.warmup
     import __graft_entry__
     __graft_entry__.build()
     if args.case:

@@ -267,8 +267,23 @@ tf_status tf_norm_bwd_force(int path, int stages, int cluster);
  * "path=P,stages=S,cluster=C" in the terms of tf_norm_bwd_force (forced > tuned > automatic = all zero). */
 tf_status tf_norm_bwd_choice(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, char* buf, size_t n);
 
-/* Forgets every tuned plan (in memory only). */
+/* Forgets every tuned plan in memory; if the environment variable TF_TUNE_CACHE names a file, the next call reads the
+ * plans stored there again. */
 void tf_clear_cache(void);
+
+/* The bounded wait that every staged kernel of this library uses, on its own: launches one small kernel on `cuda_stream`
+ * that brings 16 bytes from src16 (device memory, 16-byte aligned) into shared memory with a bulk copy but arms the
+ * barrier for 32, so its wait can only end by running out of `budget_cycles` SM clock cycles (1 .. 2e9; a millisecond is
+ * about 2e6).  The kernel then records the timeout like any other kernel (tf_device_status() returns TF_ERR_TIMEOUT
+ * once), writes 1 to *gave_up (device memory; 0 if the wait was satisfied) and returns; nothing traps or spins without a
+ * bound, and the device stays usable.  The paper has no counterpart: it exercises the remediation branch of its loop,
+ * where a candidate whose run fails is dropped (Algorithm 1), from the device side. */
+tf_status tf_debug_wait_probe(const void* src16, int64_t budget_cycles, int* gave_up, void* cuda_stream);
+
+/* Host-side fault injection for tf_tune: while plan_prefix is non-empty, every candidate whose plan text starts with it
+ * is treated as if one of its bounded waits had given up (the status word is set from the host after its run), so the
+ * tuner must drop it: never time it, never cache it.  NULL or "" switches the injection off. */
+tf_status tf_debug_tune_inject_timeout(const char* plan_prefix);
 
 /* Number of kernels this library has launched since it was loaded (all threads). */
 int64_t tf_launch_count(void);

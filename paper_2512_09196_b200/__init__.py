@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
 EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_log_softmax_bwd", "tf_norm_bwd_workspace_bytes", "tf_layernorm_bwd", "tf_rmsnorm_bwd", "tf_norm_bwd_force", "tf_softmax_variants_force", "tf_tune_norm_bwd", "tf_tune_norm_bwd_report", "tf_norm_bwd_choice",
            "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
-           "tf_candidate", "tf_clear_cache", "tf_launch_count")
+           "tf_candidate", "tf_clear_cache", "tf_launch_count", "tf_debug_wait_probe", "tf_debug_tune_inject_timeout")
 
 
 class TfError(RuntimeError):
@@ -82,6 +82,10 @@ def lib() -> ctypes.CDLL:
         L.tf_query_choice.argtypes = [i32, i64, i64, i32, i32, ctypes.c_char_p, sz]
         L.tf_candidate_count.argtypes = [i32, i64, i64, i32]
         L.tf_candidate.argtypes = [i32, i64, i64, i32, i32, ctypes.c_char_p, sz]
+        L.tf_debug_wait_probe.argtypes = [vp, i64, vp, vp]
+        L.tf_debug_wait_probe.restype = i32
+        L.tf_debug_tune_inject_timeout.argtypes = [cp]
+        L.tf_debug_tune_inject_timeout.restype = i32
         L.tf_clear_cache.argtypes = []
         L.tf_clear_cache.restype = None
         L.tf_launch_count.argtypes = []
@@ -108,6 +112,34 @@ def _check2d(x, name="x"):
         raise ValueError(f"{name} must be a CUDA tensor")
     if x.dim() != 2 or not x.is_contiguous():
         raise ValueError(f"{name} must be a contiguous [rows, cols] tensor")
+
+
+def _like(x, t, name, shape=None, dtype=None):
+    """``t`` must be a contiguous tensor on ``x``'s device with this shape and dtype (default: ``x``'s own).  The C ABI sees
+    only pointers, so a tensor that is too small, of another type or on another GPU would make a kernel read or write out
+    of bounds: it is refused here, before the call."""
+    shape = tuple(x.shape) if shape is None else tuple(shape)
+    dtype = x.dtype if dtype is None else dtype
+    if not t.is_cuda or t.device != x.device:
+        raise ValueError(f"{name} must be on the same CUDA device as x ({x.device}), got {t.device}")
+    if t.dtype != dtype:
+        raise ValueError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    if tuple(t.shape) != shape:
+        raise ValueError(f"{name} must have shape {shape}, got {tuple(t.shape)}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t
+
+
+def _param(x, t, name):
+    """An affine parameter vector: [cols], x's dtype and device."""
+    return _like(x, t, name, shape=(x.shape[1],))
+
+
+def _stat(x, t, name):
+    """A per-row statistic: fp32 [rows] on x's device."""
+    import torch
+    return _like(x, t, name, shape=(x.shape[0],), dtype=torch.float32)
 
 
 def _stream(x) -> int:
@@ -144,8 +176,7 @@ def tf_softmax_fwd(x, y=None):
     """Softmax over the last axis of a contiguous CUDA [rows, cols] tensor (fp32 or bf16); ``y`` may alias ``x``."""
     import torch
     _check2d(x)
-    if y is None:
-        y = torch.empty_like(x)
+    y = torch.empty_like(x) if y is None else _like(x, y, "y")
     rows, cols = x.shape
     with _on_device(x):
         _ok(lib().tf_softmax_fwd(x.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)), "tf_softmax_fwd")
@@ -160,8 +191,9 @@ def tf_softmax_len_fwd(x, lengths, y=None):
     rows, cols = x.shape
     if not lengths.is_cuda or lengths.dtype != torch.int32 or lengths.shape != (rows,) or not lengths.is_contiguous():
         raise ValueError("lengths must be a contiguous int32 CUDA tensor of shape [rows]")
-    if y is None:
-        y = torch.empty_like(x)
+    if lengths.device != x.device:
+        raise ValueError("lengths must be on x's device")
+    y = torch.empty_like(x) if y is None else _like(x, y, "y")
     with _on_device(x):
         _ok(lib().tf_softmax_len_fwd(x.data_ptr(), lengths.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)),
             "tf_softmax_len_fwd")
@@ -172,8 +204,7 @@ def tf_log_softmax_fwd(x, y=None):
     """Log-softmax over the last axis of a contiguous CUDA [rows, cols] tensor (fp32 or bf16); ``y`` may alias ``x``."""
     import torch
     _check2d(x)
-    if y is None:
-        y = torch.empty_like(x)
+    y = torch.empty_like(x) if y is None else _like(x, y, "y")
     rows, cols = x.shape
     with _on_device(x):
         _ok(lib().tf_log_softmax_fwd(x.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)), "tf_log_softmax_fwd")
@@ -185,10 +216,8 @@ def tf_softmax_bwd(y, dy, dx=None):
     import torch
     _check2d(y, "y")
     _check2d(dy, "dy")
-    if dy.shape != y.shape or dy.dtype != y.dtype:
-        raise ValueError("dy must match y")
-    if dx is None:
-        dx = torch.empty_like(y)
+    _like(y, dy, "dy")
+    dx = torch.empty_like(y) if dx is None else _like(y, dx, "dx")
     rows, cols = y.shape
     with _on_device(y):
         _ok(lib().tf_softmax_bwd(y.data_ptr(), dy.data_ptr(), dx.data_ptr(), rows, cols, _dt(y), _stream(y)), "tf_softmax_bwd")
@@ -200,10 +229,8 @@ def tf_log_softmax_bwd(y, dy, dx=None):
     import torch
     _check2d(y, "y")
     _check2d(dy, "dy")
-    if dy.shape != y.shape or dy.dtype != y.dtype:
-        raise ValueError("dy must match y")
-    if dx is None:
-        dx = torch.empty_like(y)
+    _like(y, dy, "dy")
+    dx = torch.empty_like(y) if dx is None else _like(y, dx, "dx")
     rows, cols = y.shape
     with _on_device(y):
         _ok(lib().tf_log_softmax_bwd(y.data_ptr(), dy.data_ptr(), dx.data_ptr(), rows, cols, _dt(y), _stream(y)), "tf_log_softmax_bwd")
@@ -217,14 +244,18 @@ def _norm_bwd_workspace(x):
     return torch.empty(max(1, n // 4), dtype=torch.float32, device=x.device), n
 
 
-def tf_layernorm_bwd(x, gamma, dy, mean, rstd, dx=None):
+def tf_layernorm_bwd(x, gamma, dy, mean, rstd, dx=None, dgamma=None, dbeta=None):
     """LayerNorm backward from the forward pass's stored fp32 ``mean`` / ``rstd``.  Returns ``(dx, dgamma, dbeta)``."""
     import torch
     _check2d(x)
-    _check2d(dy, "dy")
+    _like(x, dy, "dy")
+    _param(x, gamma, "gamma")
+    _stat(x, mean, "mean")
+    _stat(x, rstd, "rstd")
     rows, cols = x.shape
-    dx = torch.empty_like(x) if dx is None else dx
-    dgamma, dbeta = torch.empty_like(gamma), torch.empty_like(gamma)
+    dx = torch.empty_like(x) if dx is None else _like(x, dx, "dx")
+    dgamma = torch.empty_like(gamma) if dgamma is None else _param(x, dgamma, "dgamma")
+    dbeta = torch.empty_like(gamma) if dbeta is None else _param(x, dbeta, "dbeta")
     ws, n = _norm_bwd_workspace(x)
     with _on_device(x):
         _ok(lib().tf_layernorm_bwd(x.data_ptr(), gamma.data_ptr(), dy.data_ptr(), mean.data_ptr(), rstd.data_ptr(), dx.data_ptr(),
@@ -233,14 +264,16 @@ def tf_layernorm_bwd(x, gamma, dy, mean, rstd, dx=None):
     return dx, dgamma, dbeta
 
 
-def tf_rmsnorm_bwd(x, weight, dy, rstd, dx=None):
+def tf_rmsnorm_bwd(x, weight, dy, rstd, dx=None, dweight=None):
     """RMSNorm backward from the forward pass's stored fp32 ``rstd``.  Returns ``(dx, dweight)``."""
     import torch
     _check2d(x)
-    _check2d(dy, "dy")
+    _like(x, dy, "dy")
+    _param(x, weight, "weight")
+    _stat(x, rstd, "rstd")
     rows, cols = x.shape
-    dx = torch.empty_like(x) if dx is None else dx
-    dweight = torch.empty_like(weight)
+    dx = torch.empty_like(x) if dx is None else _like(x, dx, "dx")
+    dweight = torch.empty_like(weight) if dweight is None else _param(x, dweight, "dweight")
     ws, n = _norm_bwd_workspace(x)
     with _on_device(x):
         _ok(lib().tf_rmsnorm_bwd(x.data_ptr(), weight.data_ptr(), dy.data_ptr(), rstd.data_ptr(), dx.data_ptr(), dweight.data_ptr(),
@@ -280,7 +313,7 @@ def tf_softmax_fwd_noalloc(x, y):
     ``y`` must be preallocated (it may alias ``x``); rows <= 8192, 16-byte aligned tensors.  Calls that may overlap on
     the GPU share one fixed scratch array inside the library and must be ordered by the caller."""
     _check2d(x)
-    _check2d(y, "y")
+    _like(x, y, "y")
     rows, cols = x.shape
     with _on_device(x):
         _ok(lib().tf_softmax_fwd_noalloc(x.data_ptr(), y.data_ptr(), rows, cols, _dt(x), _stream(x)), "tf_softmax_fwd_noalloc")
@@ -292,8 +325,7 @@ def tf_copy(x, y=None):
     import torch
     if not x.is_cuda or not x.is_contiguous():
         raise ValueError("x must be a contiguous CUDA tensor")
-    if y is None:
-        y = torch.empty_like(x)
+    y = torch.empty_like(x) if y is None else _like(x, y, "y")
     with _on_device(x):
         _ok(lib().tf_copy(x.data_ptr(), y.data_ptr(), x.numel() * x.element_size(), _stream(x)), "tf_copy")
     return y
@@ -305,8 +337,7 @@ def tf_sin_fwd(x, y=None, threads: int = 0, vectors_per_thread: int = 0):
     import torch
     if not x.is_cuda or not x.is_contiguous():
         raise ValueError("x must be a contiguous CUDA tensor")
-    if y is None:
-        y = torch.empty_like(x)
+    y = torch.empty_like(x) if y is None else _like(x, y, "y")
     with _on_device(x):
         _ok(lib().tf_sin_fwd(x.data_ptr(), y.data_ptr(), x.numel(), _dt(x), threads, vectors_per_thread, _stream(x)), "tf_sin_fwd")
     return y
@@ -321,8 +352,9 @@ def tf_bvecmat_fwd(a, b, c=None, threads: int = 0, lanes: int = 0, rows: int = 0
     if b.shape[0] != M or b.shape[2] != K or b.dtype != a.dtype:
         raise ValueError("shape or dtype mismatch between a and b")
     N = b.shape[1]
-    if c is None:
-        c = torch.empty((M, N), dtype=a.dtype, device=a.device)
+    if b.device != a.device:
+        raise ValueError("a and b must be on the same device")
+    c = torch.empty((M, N), dtype=a.dtype, device=a.device) if c is None else _like(a, c, "c", shape=(M, N))
     with _on_device(a):
         _ok(lib().tf_bvecmat_fwd(a.data_ptr(), b.data_ptr(), c.data_ptr(), M, N, K, _dt(a), threads, lanes, rows, ksplit,
                                  _stream(a)),
@@ -336,11 +368,16 @@ def tf_layernorm_fwd(x, gamma, beta, eps: float, y=None, mean=None, rstd=None, w
     import torch
     _check2d(x)
     rows, cols = x.shape
-    if y is None:
-        y = torch.empty_like(x)
-    if want_stats and mean is None:
+    _param(x, gamma, "gamma")
+    _param(x, beta, "beta")
+    y = torch.empty_like(x) if y is None else _like(x, y, "y")
+    if mean is not None:
+        _stat(x, mean, "mean")
+    elif want_stats:
         mean = torch.empty(rows, dtype=torch.float32, device=x.device)
-    if want_stats and rstd is None:
+    if rstd is not None:
+        _stat(x, rstd, "rstd")
+    elif want_stats:
         rstd = torch.empty(rows, dtype=torch.float32, device=x.device)
     with _on_device(x):
         _ok(lib().tf_layernorm_fwd(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(),
@@ -350,41 +387,49 @@ def tf_layernorm_fwd(x, gamma, beta, eps: float, y=None, mean=None, rstd=None, w
     return y, mean, rstd
 
 
-def tf_add_layernorm_fwd(x, r, gamma, beta, eps: float, h=None, y=None, want_stats: bool = True):
+def tf_add_layernorm_fwd(x, r, gamma, beta, eps: float, h=None, y=None, want_stats: bool = True, mean=None, rstd=None):
     """Fused residual add + LayerNorm: ``h = x + r`` (rounded to the storage type), ``y = layernorm(h)``.
     Returns ``(h, y, mean, rstd)``; pass ``h=r`` to update the residual stream in place."""
     import torch
     _check2d(x)
-    _check2d(r, "r")
+    _like(x, r, "r")
+    _param(x, gamma, "gamma")
+    _param(x, beta, "beta")
     rows, cols = x.shape
-    if r.shape != x.shape or r.dtype != x.dtype:
-        raise ValueError("r must match x")
-    h = torch.empty_like(x) if h is None else h
-    y = torch.empty_like(x) if y is None else y
-    mean = torch.empty(rows, dtype=torch.float32, device=x.device) if want_stats else None
-    rstd = torch.empty(rows, dtype=torch.float32, device=x.device) if want_stats else None
+    h = torch.empty_like(x) if h is None else _like(x, h, "h")
+    y = torch.empty_like(x) if y is None else _like(x, y, "y")
+    if mean is not None:
+        _stat(x, mean, "mean")
+    elif want_stats:
+        mean = torch.empty(rows, dtype=torch.float32, device=x.device)
+    if rstd is not None:
+        _stat(x, rstd, "rstd")
+    elif want_stats:
+        rstd = torch.empty(rows, dtype=torch.float32, device=x.device)
     with _on_device(x):
         _ok(lib().tf_add_layernorm_fwd(x.data_ptr(), r.data_ptr(), gamma.data_ptr(), beta.data_ptr(), h.data_ptr(), y.data_ptr(),
-                                       mean.data_ptr() if want_stats else None, rstd.data_ptr() if want_stats else None,
+                                       mean.data_ptr() if mean is not None else None, rstd.data_ptr() if rstd is not None else None,
                                        rows, cols, eps, _dt(x), _stream(x)), "tf_add_layernorm_fwd")
     return h, y, mean, rstd
 
 
-def tf_add_rmsnorm_fwd(x, r, weight, eps: float, h=None, y=None, want_rstd: bool = False):
+def tf_add_rmsnorm_fwd(x, r, weight, eps: float, h=None, y=None, want_rstd: bool = False, rstd=None):
     """Fused residual add + RMSNorm: ``h = x + r`` (rounded to the storage type), ``y = rmsnorm(h)``.
     Returns ``(h, y, rstd)``; pass ``h=r`` to update the residual stream in place."""
     import torch
     _check2d(x)
-    _check2d(r, "r")
+    _like(x, r, "r")
+    _param(x, weight, "weight")
     rows, cols = x.shape
-    if r.shape != x.shape or r.dtype != x.dtype:
-        raise ValueError("r must match x")
-    h = torch.empty_like(x) if h is None else h
-    y = torch.empty_like(x) if y is None else y
-    rstd = torch.empty(rows, dtype=torch.float32, device=x.device) if want_rstd else None
+    h = torch.empty_like(x) if h is None else _like(x, h, "h")
+    y = torch.empty_like(x) if y is None else _like(x, y, "y")
+    if rstd is not None:
+        _stat(x, rstd, "rstd")
+    elif want_rstd:
+        rstd = torch.empty(rows, dtype=torch.float32, device=x.device)
     with _on_device(x):
         _ok(lib().tf_add_rmsnorm_fwd(x.data_ptr(), r.data_ptr(), weight.data_ptr(), h.data_ptr(), y.data_ptr(),
-                                     rstd.data_ptr() if want_rstd else None, rows, cols, eps, _dt(x), _stream(x)),
+                                     rstd.data_ptr() if rstd is not None else None, rows, cols, eps, _dt(x), _stream(x)),
             "tf_add_rmsnorm_fwd")
     return h, y, rstd
 
@@ -394,9 +439,11 @@ def tf_rmsnorm_fwd(x, weight, eps: float, y=None, rstd=None, want_rstd: bool = F
     import torch
     _check2d(x)
     rows, cols = x.shape
-    if y is None:
-        y = torch.empty_like(x)
-    if want_rstd and rstd is None:
+    _param(x, weight, "weight")
+    y = torch.empty_like(x) if y is None else _like(x, y, "y")
+    if rstd is not None:
+        _stat(x, rstd, "rstd")
+    elif want_rstd:
         rstd = torch.empty(rows, dtype=torch.float32, device=x.device)
     with _on_device(x):
         _ok(lib().tf_rmsnorm_fwd(x.data_ptr(), weight.data_ptr(), y.data_ptr(),
@@ -414,6 +461,12 @@ def tf_tune(op, rows: int, cols: int, dt: int, like=None) -> dict:
         _ok(lib().tf_tune(code, rows, cols, dt), "tf_tune")
     else:
         x, p0, p1 = like
+        _check2d(x)
+        if tuple(x.shape) != (rows, cols) or _dt(x) != dt:
+            raise ValueError("like[0] must be the [rows, cols] tensor of this dtype")
+        for q, nm in ((p0, "like[1]"), (p1, "like[2]")):
+            if q is not None:
+                _param(x, q, nm)
         _ok(lib().tf_tune_like(code, x.data_ptr(), p0.data_ptr() if p0 is not None else None,
                                p1.data_ptr() if p1 is not None else None, rows, cols, dt), "tf_tune_like")
     n, a, b = ctypes.c_int(), ctypes.c_float(), ctypes.c_float()
@@ -459,6 +512,24 @@ def tf_candidates(op, rows: int, cols: int, dt: int) -> list[str]:
 
 def tf_device_status():
     _ok(lib().tf_device_status(), "tf_device_status")
+
+
+def tf_debug_wait_probe(src, budget_cycles: int = 2_000_000) -> bool:
+    """Test hook: runs the library's bounded wait on a barrier that cannot complete; returns True if the wait gave up
+    (the status word is then set: ``tf_device_status()`` raises TF_ERR_TIMEOUT once).  ``src``: any CUDA tensor of at
+    least 16 bytes."""
+    import torch
+    if not src.is_cuda or src.numel() * src.element_size() < 16:
+        raise ValueError("src must be a CUDA tensor of at least 16 bytes")
+    flag = torch.zeros(1, dtype=torch.int32, device=src.device)
+    with _on_device(src):
+        _ok(lib().tf_debug_wait_probe(src.data_ptr(), int(budget_cycles), flag.data_ptr(), _stream(src)), "tf_debug_wait_probe")
+    return bool(flag.item())
+
+
+def tf_debug_tune_inject_timeout(plan_prefix: str | None):
+    """Test hook: ``tf_tune`` treats candidates whose plan starts with ``plan_prefix`` as timed out (None switches it off)."""
+    _ok(lib().tf_debug_tune_inject_timeout(plan_prefix.encode() if plan_prefix else None), "tf_debug_tune_inject_timeout")
 
 
 def tf_clear_cache():

@@ -15,6 +15,8 @@
 //
 // Bounded waits: an mbarrier wait that runs out of its clock budget sets TF_ERR_TIMEOUT in the status word; the
 // CTA stops issuing copies and waiting but keeps taking part in every CTA and cluster barrier, so no peer hangs.
+// The kernel ends with a cluster barrier (no CTA exits while a peer may still write a partial into its shared memory)
+// and, after a failed wait, with one more bounded wait for each of its own copies still in flight.
 #include <cooperative_groups.h>
 
 #include <algorithm>
@@ -84,8 +86,10 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
         mbar_fence_init();
     }
     pdl_wait();             // global reads below follow the previous kernel
+    uint32_t pending = 0, phase = 0;       // thread 0: stages with a copy in flight; parity of each stage's next completion
     auto issue = [&](int64_t row, int s) {                           // thread 0 only; a slice may need several copies
         if (len == 0) return;
+        pending |= 1u << s;
         const char* src = reinterpret_cast<const char*>(a.x + row * a.nvec + first);
         char* dst = reinterpret_cast<char*>(ring + static_cast<size_t>(s) * per);
         const uint32_t bytes = static_cast<uint32_t>(len) * 16u;
@@ -135,10 +139,14 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
     int it = 0;
     for (int64_t row = cluster_id; row < a.rows; row += num_clusters, ++it) {
         const int s = it % S;
-        if (len > 0 && !failed && !mbar_wait(&full_bar[s], static_cast<uint32_t>(it / S) & 1u)) {
-            failed = true;
-            atomicExch(a.status, 4);
-            mbar_wait(&full_bar[s], static_cast<uint32_t>(it / S) & 1u);      // one more bounded wait for the copy in flight
+        if (len > 0 && !failed) {
+            bool landed = mbar_wait(&full_bar[s], static_cast<uint32_t>(it / S) & 1u);
+            if (!landed) {
+                failed = true;
+                atomicExch(a.status, 4);
+                landed = mbar_wait(&full_bar[s], static_cast<uint32_t>(it / S) & 1u);      // one more bounded wait for the copy in flight
+            }
+            if (landed) { pending &= ~(1u << s); phase ^= 1u << s; }
         }
         const uint4* buf = ring + static_cast<size_t>(s) * per + t;
         uint4 raw[VPT], out[VPT];
@@ -176,6 +184,14 @@ __global__ void __launch_bounds__(ring_max_threads(VPT)) k_ring(const RArgs a) {
             if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = tot.b;
         }
     }
+    // Nobody leaves while a peer may still push a partial into its shared memory.  Every CTA of the cluster gets here:
+    // all waits above are bounded and the CTAs of a cluster walk the same rows.
+    if (cs > 1) cl.sync();
+    // After a wait has given up this CTA stopped consuming its ring: copies issued before that may still be in flight and
+    // get one more bounded wait each before the shared memory they target is released.
+    if (failed && t == 0)
+        for (int s = 0; s < S; ++s)
+            if (pending & (1u << s)) mbar_wait(&full_bar[s], (phase >> s) & 1u);
 }
 
 using RingFn = void (*)(const RArgs);

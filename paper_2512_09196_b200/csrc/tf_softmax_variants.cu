@@ -18,7 +18,7 @@
 #include <algorithm>
 
 #include "../../include/tf.h"
-#include "tf_common.cuh"
+#include "tf_streamrow.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -46,7 +46,7 @@ template <int WHICH, int DT, int VPT> constexpr int row2_floats() { return VPT *
 template <int WHICH, int DT, int VPT> constexpr int row2_max_threads() { return row2_floats<WHICH, DT, VPT>() <= 32 ? 1024 : 512; }
 
 template <int WHICH, int DT, int VPT>
-__global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2(const uint4* __restrict__ in0, const uint4* __restrict__ in1, uint4* __restrict__ out,
+__global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2(const uint4* in0, const uint4* in1, uint4* out,
                                                int64_t rows, int nvec) {
     using E = Elem<DT>;
     constexpr int NE = E::NE;
@@ -122,8 +122,8 @@ __global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2(con
 // them): M = max m_k, S = sum_k s_k 2^((m_k - M) log2 e).  Still one read of every input element and one write of every
 // output element, and small slices keep several CTAs on an SM, which is what the long rows lacked.
 template <int WHICH, int DT, int VPT>
-__global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2_cluster(const uint4* __restrict__ in0, const uint4* __restrict__ in1,
-                                                                                     uint4* __restrict__ out, int64_t rows, int nvec, int cs) {
+__global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2_cluster(const uint4* in0, const uint4* in1,
+                                                                                     uint4* out, int64_t rows, int nvec, int cs) {
     using E = Elem<DT>;
     constexpr int NE = E::NE;
     __shared__ float buf[2][32];
@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(row2_max_threads<WHICH, DT, VPT>()) k_row2_clu
 // rows, reductions are shuffles.  Every lane runs every step (the shuffles need the whole warp); rows past the end
 // are loaded as zeros and not stored.
 template <int WHICH, int DT, int LANES, int VPT>
-__global__ void __launch_bounds__(128) k_row2_group(const uint4* __restrict__ in0, const uint4* __restrict__ in1, uint4* __restrict__ out,
+__global__ void __launch_bounds__(128) k_row2_group(const uint4* in0, const uint4* in1, uint4* out,
                                                     int64_t rows, int nvec) {
     using E = Elem<DT>;
     constexpr int NE = E::NE;
@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(128) k_row2_group(const uint4* __restrict__ in
 // CL: the row is shared by the `cs` CTAs of a thread-block cluster (few rows of many columns: one CTA per row would leave
 // most of the device idle); each streams its own slice and the partials meet as in k_row2_cluster, between the passes.
 template <int WHICH, int DT, bool CL>
-__global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ in0, const uint4* __restrict__ in1, uint4* __restrict__ out,
+__global__ void __launch_bounds__(512) k_row2_stream(const uint4* in0, const uint4* in1, uint4* out,
                                                      int64_t rows, int64_t row_vecs, int cs) {
     using E = Elem<DT>;
     constexpr int NE = E::NE, U = 4;
@@ -299,6 +299,9 @@ __global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ i
     const int rank = CL ? static_cast<int>(blockIdx.x % cs) : 0;
     const int64_t row = CL ? blockIdx.x / cs : blockIdx.x;
     if (!CL && row >= rows) return;
+    // the output may alias an input (in-place calls), so the first pass reads with ordinary coherent loads (not the
+    // read-only path) and asks L2 to keep the lines for the passes that follow
+    const uint64_t keep = policy_evict_last();
     const int64_t per = CL ? (row_vecs + cs - 1) / cs : row_vecs, first = rank * per;
     const int64_t nvec = per < row_vecs - first ? per : (row_vecs - first > 0 ? row_vecs - first : 0);      // this CTA's slice
     const uint4* a = in0 + row * row_vecs + first;
@@ -315,7 +318,7 @@ __global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ i
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const bool ok = b0 + u * T < nvec;
-                r[u] = ok ? ld_param(a + b0 + u * T) : make_uint4(0, 0, 0, 0);
+                r[u] = ok ? ld_hint(a + b0 + u * T, keep) : make_uint4(0, 0, 0, 0);
                 if (ok) cm = fmaxf(cm, vec_max<DT>(r[u]));
             }
             if (cm > mt) {
@@ -371,8 +374,8 @@ __global__ void __launch_bounds__(512) k_row2_stream(const uint4* __restrict__ i
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const bool ok = b0 + u * T < nvec;
-                ry[u] = ok ? ld_param(a + b0 + u * T) : make_uint4(0, 0, 0, 0);
-                rg[u] = ok ? ld_param(b + b0 + u * T) : make_uint4(0, 0, 0, 0);
+                ry[u] = ok ? ld_hint(a + b0 + u * T, keep) : make_uint4(0, 0, 0, 0);
+                rg[u] = ok ? ld_hint(b + b0 + u * T, keep) : make_uint4(0, 0, 0, 0);
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {

@@ -26,3 +26,14 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _guard_bands(request):
+    """After every GPU test: no kernel wrote outside the tensors the drivers allocated (see parity.guarded)."""
+    yield
+    if "gpu" in request.keywords:
+        import parity
+        import torch
+        torch.cuda.synchronize()
+        parity.check_guards()

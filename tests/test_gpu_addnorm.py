@@ -32,14 +32,17 @@ def run_case(op, dt, rows, cols, seed=3, offset=0, inplace=False, r_scale=1.0):
     r_host = inputs.normal((rows, cols), dt, seed + 1000, 7, -0.2, r_scale)
     h_ref = oracle.add(data["x"], r_host, dt)
     x, r = parity.to_dev(data["x"], dt, offset), parity.to_dev(r_host, dt, offset)
-    h = r if inplace else None                       # the usual use: the residual stream is updated in place
+    # the usual use: the residual stream is updated in place; every output sits between guard bands
+    h = r if inplace else parity.guarded(tuple(x.shape), x.dtype, offset, name="h")
+    yg = parity.guarded(tuple(x.shape), x.dtype, offset, name="y")
+    st = lambda name: parity.guarded((rows,), torch.float32, name=name)
     got = {}
     if op == "layernorm":
         hh, y, mean, rstd = tf.tf_add_layernorm_fwd(x, r, parity.to_dev(data["gamma"], dt, offset), parity.to_dev(data["beta"], dt, offset),
-                                                    w.eps, h=h)
+                                                    w.eps, h=h, y=yg, mean=st("mean"), rstd=st("rstd"))
         got["mean"], got["rstd"] = mean.cpu().numpy(), rstd.cpu().numpy()
     else:
-        hh, y, rstd = tf.tf_add_rmsnorm_fwd(x, r, parity.to_dev(data["w"], dt, offset), w.eps, h=h, want_rstd=True)
+        hh, y, rstd = tf.tf_add_rmsnorm_fwd(x, r, parity.to_dev(data["w"], dt, offset), w.eps, h=h, y=yg, rstd=st("rstd"))
         got["rstd"] = rstd.cpu().numpy()
     torch.cuda.synchronize()
     tf.tf_device_status()

@@ -24,7 +24,7 @@ def check(w: inputs.VecMat, threads=0, lanes=0, offset=0, data=None, ksplit=0, r
     data = data or w.generate()
     c, c64, sc = oracle.bvecmat(data["a"], data["b"], w.dt, want64=True, nthreads=8)
     a, b = parity.to_dev(data["a"], w.dt, offset), parity.to_dev(data["b"], w.dt, offset)
-    g = tf.tf_bvecmat_fwd(a, b, None, threads, lanes, rows, ksplit)
+    g = tf.tf_bvecmat_fwd(a, b, parity.guarded((w.M, w.N), a.dtype, offset, name="c"), threads, lanes, rows, ksplit)
     torch.cuda.synchronize()
     r = compare.compare_values(parity.to_host(g, w.dt), c, c64, w.dt, cond=sc)
     assert r.ok, (w.name, threads, lanes, rows, ksplit, offset, str(r))

@@ -34,7 +34,7 @@ def test_sin_matches_the_oracle_for_every_geometry(dt):
         ref, ref64 = oracle.sin(x, dt, want64=True)
         for threads, per_sm, offset in ((0, 0, 0), (32, 1, 0), (1024, 2, 0), (128, 8, 1)):
             xd = parity.to_dev(x, dt, offset)
-            y = tf.tf_sin_fwd(xd, None, threads, per_sm)
+            y = tf.tf_sin_fwd(xd, parity.guarded(tuple(xd.shape), xd.dtype, offset, name="y"), threads, per_sm)
             torch.cuda.synchronize()
             r = compare.compare_values(parity.to_host(y, dt), ref, ref64, dt)
             assert r.ok, (n, std, threads, per_sm, offset, str(r))

@@ -47,11 +47,13 @@ def run_case(rms, dt, rows, cols, seed=1, offset=0, inplace=False):
     ref = oracle.norm_bwd(data["x"], gamma, dy, mean, rstd, dt, rms, nthreads=8)
     xd, gd, dyd = parity.to_dev(data["x"], dt, offset), parity.to_dev(gamma, dt, offset), parity.to_dev(dy, dt, offset)
     rs = torch.from_numpy(rstd).cuda()
+    dxg = dyd if inplace else parity.guarded(tuple(xd.shape), xd.dtype, offset, name="dx")      # every output between guard bands
+    pg = lambda name: parity.guarded(tuple(gd.shape), gd.dtype, offset, name=name)
     if rms:
-        dx, dg = tf.tf_rmsnorm_bwd(xd, gd, dyd, rs, dx=dyd if inplace else None)
+        dx, dg = tf.tf_rmsnorm_bwd(xd, gd, dyd, rs, dx=dxg, dweight=pg("dweight"))
         db = None
     else:
-        dx, dg, db = tf.tf_layernorm_bwd(xd, gd, dyd, torch.from_numpy(mean).cuda(), rs, dx=dyd if inplace else None)
+        dx, dg, db = tf.tf_layernorm_bwd(xd, gd, dyd, torch.from_numpy(mean).cuda(), rs, dx=dxg, dgamma=pg("dgamma"), dbeta=pg("dbeta"))
     torch.cuda.synchronize()
     tf.tf_device_status()
     what = (op, dt, rows, cols, offset)

@@ -43,7 +43,7 @@ def run_case(dt, rows, cols, seed=1, offset=0, inplace=False, x_std=3.0, compare
     ref, ref64 = oracle.softmax_len(poisoned, lens, dt, want64=True, nthreads=8)
     xd = parity.to_dev(poisoned, dt, offset)
     ld = torch.from_numpy(lens).cuda()
-    y = tf.tf_softmax_len_fwd(xd, ld, xd if inplace else None)
+    y = tf.tf_softmax_len_fwd(xd, ld, xd if inplace else parity.guarded(tuple(xd.shape), xd.dtype, offset, name="y"))
     torch.cuda.synchronize()
     tf.tf_device_status()
     got = parity.to_host(y, dt)

@@ -50,7 +50,7 @@ def run_log_softmax(dt, rows, cols, seed=1, offset=0, std=3.0, mask=False, inpla
             x[1, :] = ninf                                        # a fully masked row
     ref, ref64 = oracle.log_softmax(x, dt, want64=True, nthreads=8)
     xd = parity.to_dev(x, dt, offset)
-    y = tf.tf_log_softmax_fwd(xd, xd if inplace else None)
+    y = tf.tf_log_softmax_fwd(xd, xd if inplace else parity.guarded(tuple(xd.shape), xd.dtype, offset, name="y"))
     torch.cuda.synchronize()
     x64 = compare.to_f64(x, dt)
     with np.errstate(invalid="ignore"):
@@ -69,7 +69,7 @@ def run_softmax_bwd(dt, rows, cols, seed=1, offset=0, inplace=False):
     dy = inputs.normal((rows, cols), dt, seed + 7, 1, 0.1, 1.5)
     ref, ref64, sc = oracle.softmax_bwd(y, dy, dt, want64=True, nthreads=8)
     yd, gd = parity.to_dev(y, dt, offset), parity.to_dev(dy, dt, offset)
-    dx = tf.tf_softmax_bwd(yd, gd, gd if inplace else None)
+    dx = tf.tf_softmax_bwd(yd, gd, gd if inplace else parity.guarded(tuple(yd.shape), yd.dtype, offset, name="dx"))
     torch.cuda.synchronize()
     check_close(parity.to_host(dx, dt), ref, ref64, sc, dt, 0.0, ("softmax_bwd", dt, rows, cols, offset))
 
@@ -85,7 +85,7 @@ def run_log_softmax_bwd(dt, rows, cols, seed=1, offset=0, inplace=False, mask=Fa
     dy = inputs.normal((rows, cols), dt, seed + 7, 1, 0.1, 1.5)
     ref, ref64, sc = oracle.log_softmax_bwd(y, dy, dt, want64=True, nthreads=8)
     yd, gd = parity.to_dev(y, dt, offset), parity.to_dev(dy, dt, offset)
-    dx = tf.tf_log_softmax_bwd(yd, gd, gd if inplace else None)
+    dx = tf.tf_log_softmax_bwd(yd, gd, gd if inplace else parity.guarded(tuple(yd.shape), yd.dtype, offset, name="dx"))
     torch.cuda.synchronize()
     check_close(parity.to_host(dx, dt), ref, ref64, sc, dt, 0.0, ("log_softmax_bwd", dt, rows, cols, offset))
 
