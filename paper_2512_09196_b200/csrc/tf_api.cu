@@ -198,10 +198,10 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
     }
     if (a.op == OP_SOFTMAX && nvec >= 16384 && a.rows >= 16LL * d.sms) {
         // many rows of 256 KiB and more: two streamed passes with each thread's loads running ahead of its arithmetic in a
-        // private shared-memory ring (three CTAs of 512 threads per SM); measured 322 us on the 2 GiB masked softmax
-        // against 360-460 us for every plan that keeps the row on chip
+        // private shared-memory ring, a pair of CTAs per row (three CTAs of 384 threads per SM); measured 328 us on the
+        // 2 GiB masked softmax against 360-460 us for every plan that keeps the row on chip
         Plan s;
-        s.variant = V_TWOPASS; s.threads = 512; s.chunk = 0; s.rpg = 2; s.lanes = 1; s.vpt = 3; s.stages = 2; s.unroll = 4;
+        s.variant = V_TWOPASS; s.threads = 384; s.chunk = 0; s.rpg = 2; s.lanes = 1; s.vpt = 3; s.stages = 3; s.unroll = 4; s.cluster = 2;
         if (supports_twopass(s, a, d)) return s;
     }
     // Rules read off the plans that tf_tune ends up with on the 84-point shape sweep (rows of 128 B to 256 KiB, three ops,
@@ -408,13 +408,15 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
                 }
     // two streamed passes fed through per-thread rings of asynchronous copies
     if (nvec >= 1024)
-        for (int th : {256, 384, 512})
-            for (int su : {24, 32, 34, 44}) {                          // (stages, vectors per step)
-                Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = 0; p.lanes = 1; p.vpt = 3; p.chunk = 0;
-                p.stages = su / 10; p.unroll = su % 10; p.rpg = 2;
-                add(p);
-                if (th == 512 && su == 34) { p.rpg = 1; add(p); }
-            }
+        for (int cl : {1, 2})
+            for (int th : {256, 384, 512})
+                for (int su : {24, 34, 44}) {                          // (stages, vectors per step)
+                    if (cl > 1 && nvec < 4096) continue;
+                    Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = 0; p.lanes = 1; p.vpt = 3; p.chunk = 0; p.cluster = cl;
+                    p.stages = su / 10; p.unroll = su % 10; p.rpg = 2;
+                    add(p);
+                    if (th == 512 && su == 34) { p.rpg = 1; add(p); }
+                }
     // persistent cluster ring for long rows
     if (nvec >= 2048)
         for (int cl : {1, 2, 4, 8})

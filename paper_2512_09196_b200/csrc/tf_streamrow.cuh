@@ -54,7 +54,7 @@ template <int OP, int DT, int U_ = kStreamU> struct Running {
     F2 s_sum2 = f2(0.f);
     float c_n = 0.f, c_mean = 0.f, c_m2 = 0.f;
     F2 q2 = f2(0.f);
-    int live_slots = 0;              // softmax: one past the last slot of THIS thread that held anything but -inf
+    int live_slots = 0;              // softmax: one past the last slot of the last STEP of this thread that held anything but -inf
 
     // raw: the step's vectors, absent ones already replaced by the fill value (-inf for softmax, 0 for the norms);
     // PRED: some may be absent, ok[] says which exist; count: elements that exist (LayerNorm's divisor); slot0: slot of raw[0].
@@ -63,43 +63,38 @@ template <int OP, int DT, int U_ = kStreamU> struct Running {
         using P = Pairs<DT>;
         constexpr int NP = P::NP, U = U_;
         if constexpr (OP == OP_SOFTMAX) {
-            // maxima per vector (a vector of nothing but -inf is skipped: no exponentials) and of the step
-            bool live[U];
+            // maximum of the step, on the packed values; a step of nothing but -inf is skipped as a whole (no exponentials,
+            // one test per step instead of one per vector: masks are runs, so mixed steps are rare, and the -inf elements
+            // of a mixed step contribute exact zeros)
             float cm;
             if constexpr (DT == DT_BF16) {
-                uint32_t pm[U];
+                uint32_t pa = bf16x2_max(bf16x2_max(raw[0].x, raw[0].y), bf16x2_max(raw[0].z, raw[0].w));
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    pm[u] = bf16x2_max(bf16x2_max(raw[u].x, raw[u].y), bf16x2_max(raw[u].z, raw[u].w));
-                    live[u] = pm[u] != 0xFF80FF80u;
-                }
-                uint32_t pa = pm[0];
-#pragma unroll
-                for (int u = 1; u < U; ++u) pa = bf16x2_max(pa, pm[u]);
+                for (int u = 1; u < U; ++u) pa = bf16x2_max(pa, bf16x2_max(bf16x2_max(raw[u].x, raw[u].y), bf16x2_max(raw[u].z, raw[u].w)));
                 cm = fmaxf(__uint_as_float(pa << 16), __uint_as_float(pa & 0xFFFF0000u));
             } else {
-                cm = kNegInf;
+                cm = vec_max<DT>(raw[0]);
+#pragma unroll
+                for (int u = 1; u < U; ++u) cm = fmaxf(cm, vec_max<DT>(raw[u]));
+            }
+            if (cm != kNegInf) {
+                if (cm > s_max) {                                                 // new running max: move the sums to its offset
+                    const float noff = exp_offset(cm);
+                    s_sum2 = (s_max == kNegInf) ? f2(0.f) : mul2(s_sum2, f2(ex2_ftz(noff - s_off)));
+                    s_off = noff; s_max = cm;
+                }
+                const F2 off = f2(s_off), l2e = f2(kLog2e);
+                F2 acc[U];                                                        // independent chains: the exponentials overlap
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    const float vm = vec_max<DT>(raw[u]);
-                    live[u] = vm != kNegInf;
-                    cm = fmaxf(cm, vm);
-                }
-            }
-            if (cm > s_max) {                                                     // new running max: move the sums to its offset
-                const float noff = exp_offset(cm);
-                s_sum2 = (s_max == kNegInf) ? f2(0.f) : mul2(s_sum2, f2(ex2_ftz(noff - s_off)));
-                s_off = noff; s_max = cm;
-            }
-            const F2 off = f2(s_off), l2e = f2(kLog2e);
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (live[u]) {
                     F2 w[NP]; P::unpack(raw[u], w);
+                    acc[u] = ex2_ftz2(fma2(w[0], l2e, off));
 #pragma unroll
-                    for (int i = 0; i < NP; ++i) s_sum2 = add2(s_sum2, ex2_ftz2(fma2(w[i], l2e, off)));
-                    live_slots = max(live_slots, slot0 + u + 1);         // pass A may walk the row in either direction
+                    for (int i = 1; i < NP; ++i) acc[u] = add2(acc[u], ex2_ftz2(fma2(w[i], l2e, off)));
                 }
+#pragma unroll
+                for (int u = 0; u < U; ++u) s_sum2 = add2(s_sum2, acc[u]);
+                live_slots = max(live_slots, slot0 + U);                          // pass A may walk the row in either direction
             }
         } else if constexpr (OP == OP_LAYERNORM) {
             F2 w[U][NP];
@@ -249,10 +244,11 @@ __device__ __forceinline__ uint4 apply_vec(const uint4& raw, const uint4* g, con
 
 // One step of pass B: kStreamU vectors of this thread starting at vector idx0 (stride T).  PRED: vectors at or beyond
 // nvec do not exist.  live[u] (softmax): the vector may hold something other than -inf; the others become zeros unread.
+// nlive (LEN): vectors from there on lie behind the row's length: never read, always zeros.
 template <int OP, int DT, bool PRED, bool LEN, bool CACHE>
 __device__ __forceinline__ void apply_step(const uint4* xs, uint4* ys, const uint4* g, const uint4* b, int64_t idx0, int T, int64_t nvec,
                                            const F2 ta2, const F2 tb2, uint64_t policy, const uint4* cache, int64_t cache_vecs,
-                                           const bool (&live)[kStreamU], int64_t straddle, int keep) {
+                                           const bool (&live)[kStreamU], int64_t straddle, int keep, int64_t nlive) {
     constexpr int U = kStreamU;
     uint4 raw[U];
     bool ok[U];
@@ -260,7 +256,7 @@ __device__ __forceinline__ void apply_step(const uint4* xs, uint4* ys, const uin
     for (int u = 0; u < U; ++u) {
         const int64_t idx = idx0 + static_cast<int64_t>(u) * T;
         ok[u] = !PRED || idx < nvec;
-        const bool want = ok[u] && (OP != OP_SOFTMAX || live[u]);
+        const bool want = ok[u] && (OP != OP_SOFTMAX || (live[u] && (!LEN || idx < nlive)));
         if (want) raw[u] = (CACHE && idx < cache_vecs) ? cache[idx] : ld_hint(xs + idx, policy);
         else raw[u] = fill_vec<DT>(OP);
         if (LEN && idx == straddle) raw[u] = mask_tail<DT>(raw[u], keep);
@@ -270,7 +266,7 @@ __device__ __forceinline__ void apply_step(const uint4* xs, uint4* ys, const uin
         if (!ok[u]) continue;
         const int64_t idx = idx0 + static_cast<int64_t>(u) * T;
         uint4 out = make_uint4(0, 0, 0, 0);
-        if (OP != OP_SOFTMAX || live[u]) out = apply_vec<OP, DT>(raw[u], g + idx, b + idx, ta2, tb2);
+        if (OP != OP_SOFTMAX || (live[u] && (!LEN || idx < nlive))) out = apply_vec<OP, DT>(raw[u], g + idx, b + idx, ta2, tb2);
         st_stream(ys + idx, out);
     }
 }
@@ -286,6 +282,7 @@ __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const u
     constexpr int U = kStreamU, NE = Elem<DT>::NE;
     const int64_t straddle = (LEN && len % NE) ? len / NE : -1;           // live_slots already ends at ceil(len / NE)
     const int keep = LEN ? static_cast<int>(len % NE) : 0;
+    const int64_t nlive = LEN ? (len + NE - 1) / NE : nvec;
     const int T = blockDim.x, t = threadIdx.x;
     const F2 ta2 = f2(sc.a), tb2 = f2(sc.b);
     // back to front: the end of the segment is what pass A touched last, hence what L2 most likely still holds
@@ -295,7 +292,7 @@ __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const u
         bool live[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) live[u] = nfull * U + u < live_slots;
-        apply_step<OP, DT, true, LEN, CACHE>(xs, ys, g, b, nfull * step + t, T, nvec, ta2, tb2, policy, cache, cache_vecs, live, straddle, keep);
+        apply_step<OP, DT, true, LEN, CACHE>(xs, ys, g, b, nfull * step + t, T, nvec, ta2, tb2, policy, cache, cache_vecs, live, straddle, keep, nlive);
     }
     for (int s = nfull - 1; s >= 0; --s) {
         const int64_t idx0 = s * step + t;
@@ -307,7 +304,7 @@ __device__ __forceinline__ void stream_apply(const uint4* xs, uint4* ys, const u
         bool live[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) live[u] = s * U + u < live_slots;
-        apply_step<OP, DT, false, LEN, CACHE>(xs, ys, g, b, idx0, T, nvec, ta2, tb2, policy, cache, cache_vecs, live, straddle, keep);
+        apply_step<OP, DT, false, LEN, CACHE>(xs, ys, g, b, idx0, T, nvec, ta2, tb2, policy, cache, cache_vecs, live, straddle, keep, nlive);
     }
 }
 

@@ -147,92 +147,183 @@ __device__ __forceinline__ void cp_async_wait(int pending) {     // returns once
 }
 constexpr int kRingMaxDepth = 8;
 
-template <int OP, int DT, int U, int MAXT, int MINB>
+// Work is laid out by warps: in one step a warp takes U x 32 consecutive vectors (lane l the vectors l, l + 32, ... of that
+// run), so a thread's U copies, loads and stores of a step sit at fixed offsets from one pointer that advances by a
+// step's worth per iteration; all counters are 32-bit.  Only the last step of a row can be ragged, and it has its own
+// code: the loops over whole steps carry no predicates.
+// CL: the `cs` CTAs of a thread-block cluster share a row, CTA `rank` taking the steps rank, rank + cs, ... of it (so a mask
+// at the end of the row costs every CTA of the cluster the same); the partials meet between the passes through
+// distributed shared memory and one cluster barrier.  A row is then in flight for 1 / cs of the time, which keeps what lies
+// between the passes within L2, and each CTA's ring holds cs times as large a share of the row.
+template <int OP, int DT, int U, int MAXT, int MINB, bool CL>
 __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
-    constexpr int NE = Elem<DT>::NE;
+    constexpr int NE = Elem<DT>::NE, CH = U * 32;                        // vectors a warp takes per step
     __shared__ float red_buf[4 * 32];
+    __shared__ float xch[CL ? 2 : 1][CL ? kMaxCluster : 1][2];           // partials of the CTAs of the cluster, by row parity
     extern __shared__ __align__(16) unsigned char dyn_smem[];
-    uint4* const ring = reinterpret_cast<uint4*>(dyn_smem);              // [stage][u][thread]
     pdl_wait();
     pdl_trigger();
     const uint64_t keep = (a.policy & 1) ? policy_evict_last() : policy_evict_normal();
     const uint64_t last = (a.policy & 2) ? policy_evict_first() : policy_evict_normal();
-    const int T = blockDim.x, t = threadIdx.x, S = a.stages;
+    const int t = threadIdx.x, S = a.stages;
+    const int cs = CL ? a.cs : 1;
+    const int rank = CL ? static_cast<int>(blockIdx.x % cs) : 0;
+    const int nvec = static_cast<int>(a.nvec);
+    const int step = (blockDim.x >> 5) * CH;                             // vectors the CTA takes per step
+    const int gstep = cs * step;                                         // distance in the row between two steps of this CTA
+    const int nfull = nvec / step;                                       // whole steps of the row
+    const int rag = nvec - nfull * step;                                 // vectors of the row's ragged last step (0: there is none)
+    // the steps of CTA k: k, k + cs, ...; its last one is the ragged step iff that falls to it
+    auto steps_of = [&](int k) { const int n = nfull + (rag ? 1 : 0); return n > k ? (n - k - 1) / cs + 1 : 0; };
+    auto ragged_of = [&](int k) { return rag != 0 && nfull % cs == k; };
+    auto count_of = [&](int k) { return static_cast<float>(((steps_of(k) - (ragged_of(k) ? 1 : 0)) * step + (ragged_of(k) ? rag : 0)) * NE); };
+    const int nsteps = steps_of(rank);                                   // this CTA's steps, numbered 0 .. nsteps-1 from here on
+    const bool has_rag = ragged_of(rank);
+    const int nwhole = nsteps - (has_rag ? 1 : 0);
+    const int toff = (t >> 5) * CH + (t & 31);                           // this thread's first vector within a step
+    uint4* const myring = reinterpret_cast<uint4*>(dyn_smem) + toff;     // slot k of the ring: myring + k * step (+ u * 32)
+    uint4* const ring_end = myring + S * step;
     const int64_t per_group = a.slots / a.groups;
-    const int64_t step = static_cast<int64_t>(T) * U;
-    const int nsteps = static_cast<int>((a.nvec + step - 1) / step);
     const uint4 fill = fill_vec<DT>(OP);
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    const int slot_of_step0 = nsteps > 0 ? (nsteps - 1) % S : 0;         // pass A visits step s as its (nsteps-1-s)-th: slot = that mod S
+    if constexpr (CL) cg::this_cluster().sync();                         // every CTA of the cluster is resident before any remote write
+    const int64_t first_slot = CL ? blockIdx.x / cs : blockIdx.x, slot_step = CL ? gridDim.x / cs : gridDim.x;
     int it = -1;
-    for (int64_t slot = blockIdx.x; slot < a.slots; slot += gridDim.x) {
+    for (int64_t slot = first_slot; slot < a.slots; slot += slot_step) {
         const int64_t row = a.groups > 1 ? (slot % a.groups) * per_group + slot / a.groups : slot;
-        if (row >= a.rows) continue;
+        if (row >= a.rows) continue;                                     // the same decision in every CTA of a cluster
         ++it;
-        const uint4* xr = a.x + row * a.nvec;
-        uint4* yr = a.y + row * a.nvec;
-        // the copies of step s into its ring slot; vectors behind the end of the row get the fill value instead
-        auto issue = [&](int s, uint64_t policy) {
-            uint4* dst = ring + static_cast<size_t>(s % S) * step + t;
-            const int64_t idx0 = s * step + t;
+        const int64_t base = row * nvec + rank * step + toff;            // this thread's vectors of step s: base + s * gstep (+ u * 32)
+        const uint4* const xr = a.x + base;
+        uint4* const yr = a.y + base;
+        auto issue_full = [&](const uint4* src, uint4* dst, uint64_t policy) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) cp_async16(dst + u * 32, src + u * 32, policy);
+        };
+        auto issue_ragged = [&](uint4* dst, uint64_t policy) {           // vectors behind the end of the row get the fill value
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (idx0 + u * T < a.nvec) cp_async16(dst + u * T, xr + idx0 + u * T, policy);
-                else dst[u * T] = fill;
+                if (toff + u * 32 < rag) cp_async16(dst + u * 32, xr + nwhole * gstep + u * 32, policy);
+                else dst[u * 32] = fill;
             }
         };
-        // ---- pass A, back to front
+        // ---- pass A, back to front: the k-th step visited is s = nsteps - 1 - k and lives in slot k mod S
         Running<OP, DT, U> run;
-        for (int k = 0; k < S - 1; ++k) {
-            if (nsteps - 1 - k >= 0) issue(nsteps - 1 - k, keep);
-            cp_async_commit();
-        }
-        for (int s = nsteps - 1; s >= 0; --s) {
-            if (s - (S - 1) >= 0) issue(s - (S - 1), keep);
-            cp_async_commit();
-            cp_async_wait(S - 1);
-            const uint4* src = ring + static_cast<size_t>(s % S) * step + t;
-            uint4 raw[U];
-            bool ok[U];
-            int count = 0;
+        {
+            int k_issue = 0;
+            uint4* dst_i = myring;                                       // ring slot of the step issued next
+            const uint4* src_i = xr + (nsteps - 1) * gstep;
+            auto issue_next = [&]() {
+                if (k_issue < nsteps) {
+                    if (has_rag && k_issue == 0) issue_ragged(dst_i, keep);
+                    else issue_full(src_i, dst_i, keep);
+                }
+                cp_async_commit();
+                ++k_issue; src_i -= gstep; dst_i += step;
+                if (dst_i == ring_end) dst_i = myring;
+            };
+            for (int j = 0; j < S - 1; ++j) issue_next();
+            const uint4* cur = myring;                                   // ring slot of the step worked on
+            for (int k = 0; k < nsteps; ++k) {
+                issue_next();
+                cp_async_wait(S - 1);
+                uint4 raw[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                raw[u] = src[u * T];
-                ok[u] = s * step + t + u * T < a.nvec;                   // only the last step of a row can be ragged
-                count += ok[u] ? NE : 0;
+                for (int u = 0; u < U; ++u) raw[u] = cur[u * 32];
+                cur += step;
+                if (cur == ring_end) cur = myring;
+                const int s = nsteps - 1 - k;
+                if (has_rag && k == 0) {
+                    bool ok[U];
+                    int count = 0;
+#pragma unroll
+                    for (int u = 0; u < U; ++u) { ok[u] = toff + u * 32 < rag; count += ok[u] ? NE : 0; }
+                    if (count > 0) run.template update<true>(raw, ok, count, s * U);
+                } else {
+                    const bool all[U] = {};
+                    run.template update<false>(raw, all, U * NE, s * U);
+                }
             }
-            if (count == U * NE) run.template update<false>(raw, ok, count, s * U);
-            else if (count > 0) run.template update<true>(raw, ok, count, s * U);
         }
-        const Part part = merge_running<OP, DT, U>(run, a.n, red_buf + 64 * (it & 1));
+        Part part = merge_running<OP, DT, U>(run, CL ? fmaxf(count_of(rank), 1.f) : a.n, red_buf + 64 * (it & 1));
+        if constexpr (CL) {
+            cg::cluster_group cl = cg::this_cluster();
+            const int xb = it & 1;
+            if (t < cs) {                                                 // my partial into every CTA of the cluster
+                float* dstp = cl.map_shared_rank(&xch[xb][rank][0], t);
+                dstp[0] = part.a; dstp[1] = part.b;
+            }
+            cl.sync();                                                    // release our writes, acquire the peers'
+            // the row's partial from the CTAs', in rank order (the same bits in every CTA)
+            if constexpr (OP == OP_SOFTMAX) {
+                float O = -kNegInf, Ssum = 0.f;
+                for (int k = 0; k < cs; ++k) O = fminf(O, xch[xb][k][0]);
+                for (int k = 0; k < cs; ++k) Ssum = fmaf(xch[xb][k][1], softmax_rescale(O, xch[xb][k][0]), Ssum);
+                part = Part{O, Ssum};
+            } else if constexpr (OP == OP_LAYERNORM) {
+                float sum = 0.f, m2 = 0.f;
+                for (int k = 0; k < cs; ++k) sum = fmaf(count_of(k), xch[xb][k][0], sum);
+                const float mean = fast_div(sum, a.n);
+                for (int k = 0; k < cs; ++k) { const float d = xch[xb][k][0] - mean; m2 += fmaf(count_of(k) * d, d, xch[xb][k][1]); }
+                part = Part{mean, m2};
+            } else {
+                float q = 0.f;
+                for (int k = 0; k < cs; ++k) q += xch[xb][k][0];
+                part = Part{q, 0.f};
+            }
+        }
         const RowScale sc = scale_of_row<OP>(part, a.n, a.eps);
-        if (t == 0) {
+        if (t == 0 && rank == 0) {
             if (OP == OP_LAYERNORM && a.mean) a.mean[row] = sc.a;
             if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = sc.b;
         }
-        // ---- pass B, front to back: steps 0 .. S-1 are still in the ring
+        // ---- pass B, front to back: steps 0 .. S-1 are still in the ring; step s + S - 1 is requested while step s is
+        // worked on, into the slot that step s - 1 has just left.  Softmax: from this thread's first step that holds
+        // nothing but -inf on, zeros are written and x is not read again.
         const F2 ta2 = f2(sc.a), tb2 = f2(sc.b);
-        const int live_steps = OP == OP_SOFTMAX ? (run.live_slots + U - 1) / U : nsteps;      // steps from here on hold nothing but -inf
-        for (int s = 0; s < nsteps; ++s) {
+        const int live_steps = OP == OP_SOFTMAX ? (run.live_slots + U - 1) / U : nsteps;
+        const int live_whole = min(live_steps, nwhole);
+        const uint4* cur = myring + slot_of_step0 * step;                // ring slot of step s: one slot down per step
+        const uint4* src_n = xr + S * gstep;                             // step s + S - 1 of x (s = 1 first)
+        const uint4* gp = a.p0 + rank * step + toff;
+        const uint4* bp = a.p1 + rank * step + toff;
+        uint4* dst = yr;
+        int s = 0;
+        for (; s < live_whole; ++s) {
             const int sn = s + S - 1;
-            if (s >= 1 && sn < live_steps) issue(sn, last);              // the slot of step s - 1 is free
-            cp_async_commit();
-            const int64_t idx0 = s * step + t;
-            if (s >= live_steps) {                                       // zeros; x is not read again
-#pragma unroll
-                for (int u = 0; u < U; ++u)
-                    if (idx0 + u * T < a.nvec) st_stream(yr + idx0 + u * T, make_uint4(0, 0, 0, 0));
-                continue;
-            }
-            cp_async_wait(S - 1);
-            const uint4* src = ring + static_cast<size_t>(s % S) * step + t;
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int64_t idx = idx0 + u * T;
-                if (idx < a.nvec) {
-                    uint4 out = make_uint4(0, 0, 0, 0);
-                    if (OP != OP_SOFTMAX || s * U + u < run.live_slots) out = apply_vec<OP, DT>(src[u * T], a.p0 + idx, a.p1 + idx, ta2, tb2);
-                    st_stream(yr + idx, out);
+            if (s >= 1) {
+                uint4* freed = const_cast<uint4*>(cur) + step;           // the slot step s - 1 has just left
+                if (freed == ring_end) freed = myring;
+                if (sn < live_steps) {
+                    if (sn < nwhole) issue_full(src_n, freed, last);
+                    else issue_ragged(freed, last);
                 }
+                src_n += gstep;
             }
+            cp_async_commit();
+            cp_async_wait(S - 1);
+#pragma unroll
+            for (int u = 0; u < U; ++u) st_stream(dst + u * 32, apply_vec<OP, DT>(cur[u * 32], gp + u * 32, bp + u * 32, ta2, tb2));
+            cur = (cur == myring ? ring_end : cur) - step;
+            dst += gstep; gp += gstep; bp += gstep;
+        }
+        if (has_rag && s == nwhole && s < live_steps) {                  // the ragged step is live
+            cp_async_commit();
+            cp_async_wait(0);
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (toff + u * 32 < rag) st_stream(dst + u * 32, apply_vec<OP, DT>(cur[u * 32], gp + u * 32, bp + u * 32, ta2, tb2));
+            ++s;
+        }
+        for (; s < nwhole; ++s) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) st_stream(yr + s * gstep + u * 32, zero);
+        }
+        if (has_rag && s == nwhole) {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (toff + u * 32 < rag) st_stream(yr + s * gstep + u * 32, zero);
         }
         cp_async_wait(0);
     }
@@ -269,22 +360,24 @@ TwoFn two_fn(int op, int dt, int threads, bool capped, bool cl, bool len, bool c
     return two_fn_b<1024, 0>(op, dt, cl, len, cache);
 }
 
-template <int U, int MAXT, int MINB>
-TwoFn ring_fn_b(int op, int dt) {
+template <int U, int MAXT, int MINB, bool CL>
+TwoFn ring_fn_c(int op, int dt) {
     switch (op * 2 + dt) {
-        case 0: return k_twopass_ring<OP_SOFTMAX, DT_F32, U, MAXT, MINB>;
-        case 1: return k_twopass_ring<OP_SOFTMAX, DT_BF16, U, MAXT, MINB>;
-        case 2: return k_twopass_ring<OP_LAYERNORM, DT_F32, U, MAXT, MINB>;
-        case 3: return k_twopass_ring<OP_LAYERNORM, DT_BF16, U, MAXT, MINB>;
-        case 4: return k_twopass_ring<OP_RMSNORM, DT_F32, U, MAXT, MINB>;
-        case 5: return k_twopass_ring<OP_RMSNORM, DT_BF16, U, MAXT, MINB>;
+        case 0: return k_twopass_ring<OP_SOFTMAX, DT_F32, U, MAXT, MINB, CL>;
+        case 1: return k_twopass_ring<OP_SOFTMAX, DT_BF16, U, MAXT, MINB, CL>;
+        case 2: return k_twopass_ring<OP_LAYERNORM, DT_F32, U, MAXT, MINB, CL>;
+        case 3: return k_twopass_ring<OP_LAYERNORM, DT_BF16, U, MAXT, MINB, CL>;
+        case 4: return k_twopass_ring<OP_RMSNORM, DT_F32, U, MAXT, MINB, CL>;
+        case 5: return k_twopass_ring<OP_RMSNORM, DT_BF16, U, MAXT, MINB, CL>;
     }
     return nullptr;
 }
+template <int U, int MAXT, int MINB>
+TwoFn ring_fn_b(int op, int dt, bool cl) { return cl ? ring_fn_c<U, MAXT, MINB, true>(op, dt) : ring_fn_c<U, MAXT, MINB, false>(op, dt); }
 // regcap: the builds held to 40 registers (three CTAs of 512 threads, or four of 384, per SM)
-TwoFn ring_fn(int op, int dt, int unroll, int threads, bool capped) {
-    if (unroll == 2) return (capped && threads <= 512) ? ring_fn_b<2, 512, 3>(op, dt) : ring_fn_b<2, 1024, 1>(op, dt);
-    if (unroll == 4) return (capped && threads <= 512) ? ring_fn_b<4, 512, 3>(op, dt) : ring_fn_b<4, 1024, 1>(op, dt);
+TwoFn ring_fn(int op, int dt, int unroll, int threads, bool capped, bool cl) {
+    if (unroll == 2) return (capped && threads <= 512) ? ring_fn_b<2, 512, 3>(op, dt, cl) : ring_fn_b<2, 1024, 1>(op, dt, cl);
+    if (unroll == 4) return (capped && threads <= 512) ? ring_fn_b<4, 512, 3>(op, dt, cl) : ring_fn_b<4, 1024, 1>(op, dt, cl);
     return nullptr;
 }
 
@@ -294,16 +387,16 @@ TwoFn ring_fn(int op, int dt, int unroll, int threads, bool capped) {
 // the register-capped build (threads <= 768); `lanes`: row-order groups; `vpt`: L2 hint bits of the two passes.
 bool supports_twopass(const Plan& p, const Args& a, const DeviceInfo& d) {
     if (p.cluster != 1 && p.cluster != 2 && p.cluster != 4 && p.cluster != 8) return false;
-    if (p.cluster > 1 && (p.cluster > d.max_cluster || a.cols * elem_size(a.dt) / 16 < p.cluster || a.rows * p.cluster > 0x7FFFFFFF)) return false;
+    if (p.cluster > 1 && (p.cluster > d.max_cluster || a.rows * p.cluster > 0x7FFFFFFF)) return false;
     if (p.lanes < 1 || p.lanes > 1024 || p.vpt < 0 || p.vpt > 3) return false;
-    if (p.stages >= 2) {                                           // the ring form: one CTA per row, no length mode, no separate cache
-        if (p.stages > kRingMaxDepth || (p.unroll != 2 && p.unroll != 4) || p.cluster != 1 || p.chunk != 0 || a.len) return false;
+    if (p.stages >= 2) {                                           // the ring form: no length mode, no separate cache
+        if (p.stages > kRingMaxDepth || (p.unroll != 2 && p.unroll != 4) || p.chunk != 0 || a.len) return false;
         const int64_t nvec = a.cols * elem_size(a.dt) / 16;
-        if (nvec / (static_cast<int64_t>(p.threads) * p.unroll) > (1 << 24)) return false;
+        if (nvec > 0x7FFFFFFF - 65536) return false;              // 32-bit vector indices inside the kernel
         return vector_ok(a) && (p.rpg == 1 || p.rpg == 2) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0 &&
                (d.smem_optin == 0 || static_cast<int64_t>(p.stages) * p.threads * p.unroll * 16 + 1024 <= d.smem_optin);
     }
-    if (p.stages != 0 && p.stages != 1) return false;
+    if ((p.stages != 0 && p.stages != 1) || a.cols * elem_size(a.dt) / 16 < p.cluster) return false;
     return vector_ok(a) && (p.rpg == 1 || (p.rpg == 2 && p.threads <= 768)) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0 && p.chunk >= 0 && p.chunk % 16 == 0 &&
            (d.smem_optin == 0 || p.chunk + 2048 <= d.smem_optin);
 }
@@ -311,7 +404,7 @@ bool supports_twopass(const Plan& p, const Args& a, const DeviceInfo& d) {
 cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream_t st) {
     const int cs = std::max(1, p.cluster);
     const bool ring = p.stages >= 2;
-    TwoFn fn = ring ? ring_fn(a.op, a.dt, p.unroll, p.threads, p.rpg == 2) : two_fn(a.op, a.dt, p.threads, p.rpg == 2, cs > 1, a.len != nullptr, p.chunk > 0);
+    TwoFn fn = ring ? ring_fn(a.op, a.dt, p.unroll, p.threads, p.rpg == 2, cs > 1) : two_fn(a.op, a.dt, p.threads, p.rpg == 2, cs > 1, a.len != nullptr, p.chunk > 0);
     if (!fn) return cudaErrorInvalidValue;
     const int groups = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(p.lanes, a.rows)));
     const int64_t slots = (a.rows + groups - 1) / groups * groups;

@@ -274,12 +274,22 @@ def test_forced_twopass_variants(op, dt):
             assert not fails, (plan, nvec, rows, fails)
             fails = parity.parity(wl(op, dt, min(rows, 11), nvec * ne, seed=nvec + stages), inplace=True)
             assert not fails, ("in place", plan, nvec, rows, fails)
+    # the ring form with the CTAs of a cluster sharing a row step by step: rows shorter than one CTA's step (CTAs without
+    # work), ragged steps falling to every rank, persistent clusters, one row
+    for cluster, threads, stages, u, persist, regcap in ((2, 128, 2, 4, 0, 1), (4, 256, 3, 2, 0, 0), (8, 64, 2, 4, 1, 1), (2, 512, 3, 4, 0, 0)):
+        st = threads * u
+        for nvec, rows in ((1, 3), (st, 5), (st + 1, 5), (st * cluster - 1, 9), (st * cluster * stages + 5, 9), (st * (cluster + 1) + 7, 150), (70001, 3), (st * 3, 1)):
+            plan = f"twopass:threads={threads},persist={persist},regcap={regcap},cluster={cluster},stages={stages},u={u}"
+            tf.tf_force_plan(op, plan)
+            fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec + cluster))
+            assert not fails, (plan, nvec, rows, fails)
     for groups in (2, 8, 1000):                            # the direct form with interleaved row order
         tf.tf_force_plan(op, f"twopass:threads=256,persist=0,groups={groups},hints=0")
         assert not parity.parity(wl(op, dt, 37, 5000 * ne, seed=groups)), groups
     if op == "softmax":                                    # masks, a fully masked row and outputs in the subnormal range
         for plan in ("twopass:threads=256,persist=0,cluster=4", "twopass:threads=512,cache=8192,persist=0,regcap=1,cluster=8",
-                     "twopass:threads=256,persist=0,stages=2,u=4", "twopass:threads=128,persist=0,regcap=1,stages=3,u=2,groups=4"):
+                     "twopass:threads=256,persist=0,stages=2,u=4", "twopass:threads=128,persist=0,regcap=1,stages=3,u=2,groups=4",
+                     "twopass:threads=128,persist=0,regcap=1,stages=2,u=4,cluster=2", "twopass:threads=64,persist=0,stages=3,u=2,cluster=8"):
             tf.tf_force_plan(op, plan)
             w = Workload("m", "softmax", dt, 12, 40000, seed=5, x_std=10.0, mask_step=3001)
             data = w.generate()
