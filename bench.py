@@ -36,8 +36,11 @@ HEADLINE_CONFIG = 3               # the largest fixed configuration that fits on
 # configuration, from profiler captures of cases too large for the 126 MB L2 to hide the writes; None where no capture
 # exists.  Value = (bytes of the captured case, factor to a full launch of the configuration).
 NCU_TRAFFIC_BYTES = {
-    # LayerNorm bf16 [32768, 4096] (four times the rows of the configuration): 268.5 MB read + 210.8 MB written
-    "layernorm_bf16_8192x4096": (268_497_408 + 210_806_400, 0.25),
+    # LayerNorm bf16 [32768, 4096] (four times the rows of the configuration): 268.5 MB read + 215.3 MB written
+    "layernorm_bf16_8192x4096": (268_493_568 + 215_280_128, 0.25),
+    # the 2 GiB masked softmax itself, a one-pass capture of the two DRAM counters on the full 4096 rows (untuned plan):
+    # 1080.3 MB read (the algorithmic reads are 1073.7 MB) + 1029.6 MB written inside the kernel
+    "masked_softmax_bf16_4096x131072": (1_080_327_168 + 1_029_625_088, 1.0),
 }
 
 

@@ -267,6 +267,20 @@ tf_status tf_norm_bwd_force(int path, int stages, int cluster);
  * "path=P,stages=S,cluster=C" in the terms of tf_norm_bwd_force (forced > tuned > automatic = all zero). */
 tf_status tf_norm_bwd_choice(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, char* buf, size_t n);
 
+/* The refinement hint of tf_tune (Algorithm 1's Targeted-Refinement-Hint step, rule-based here): what the library reads
+ * about a plan's launch without a profiler -- registers and resident CTAs of its kernel, waves of its grid and the empty
+ * share of the last one, bytes in flight per SM -- and the rule that fires on it:
+ *   occupancy  (<= 25 % resident threads and > 96 registers)  try fewer vectors or rows per thread, smaller CTAs first
+ *   tail       (more than 15 % of the last wave empty)        try persistent CTAs or finer units of work first
+ *   inflight   (less than 40 KB in flight per SM)             try deeper rings, larger stages, more resident threads first
+ *   ceiling    (within 2 % of the library's own copy of the same tensors; tf_tune only)   finish
+ * tf_refine_hint launches `plan` once on zero-filled scratch tensors of this shape and writes
+ * "rule=... regs=... ctas_per_sm=... occupancy=... waves=... tail=... inflight_kb=... vs_copy=... first=<plan>;<plan>;<plan>"
+ * (the first neighbours the refinement would try).  tf_tune_last_hint writes the hint tf_tune computed for the heuristic
+ * plan in its last run on the calling thread. */
+tf_status tf_refine_hint(tf_op op, int64_t rows, int64_t cols, tf_dtype dt, const char* plan, char* buf, size_t n);
+tf_status tf_tune_last_hint(char* buf, size_t n);
+
 /* Forgets every tuned plan in memory; if the environment variable TF_TUNE_CACHE names a file, the next call reads the
  * plans stored there again. */
 void tf_clear_cache(void);

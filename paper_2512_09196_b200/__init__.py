@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "TF_OK", 1: "TF_ERR_INVALID_ARG", 2: "TF_ERR_UNSUPPORTED", 3:
 EXPORTS = ("tf_softmax_fwd", "tf_softmax_fwd_noalloc", "tf_layernorm_fwd", "tf_rmsnorm_fwd", "tf_tune", "tf_tune_like", "tf_tune_report", "tf_copy", "tf_sin_fwd", "tf_bvecmat_fwd", "tf_add_layernorm_fwd", "tf_add_rmsnorm_fwd", "tf_tune_add", "tf_softmax_len_fwd", "tf_log_softmax_fwd", "tf_softmax_bwd", "tf_log_softmax_bwd", "tf_norm_bwd_workspace_bytes", "tf_layernorm_bwd", "tf_rmsnorm_bwd", "tf_norm_bwd_force", "tf_softmax_variants_force", "tf_tune_norm_bwd", "tf_tune_norm_bwd_report", "tf_norm_bwd_choice",
            "tf_status_string",
            "tf_last_cuda_error", "tf_device_status", "tf_force_plan", "tf_query_choice", "tf_candidate_count",
-           "tf_candidate", "tf_clear_cache", "tf_launch_count", "tf_debug_wait_probe", "tf_debug_tune_inject_timeout")
+           "tf_candidate", "tf_clear_cache", "tf_launch_count", "tf_debug_wait_probe", "tf_debug_tune_inject_timeout", "tf_refine_hint", "tf_tune_last_hint")
 
 
 class TfError(RuntimeError):
@@ -86,6 +86,10 @@ def lib() -> ctypes.CDLL:
         L.tf_debug_wait_probe.restype = i32
         L.tf_debug_tune_inject_timeout.argtypes = [cp]
         L.tf_debug_tune_inject_timeout.restype = i32
+        L.tf_refine_hint.argtypes = [i32, i64, i64, i32, cp, ctypes.c_char_p, sz]
+        L.tf_refine_hint.restype = i32
+        L.tf_tune_last_hint.argtypes = [ctypes.c_char_p, sz]
+        L.tf_tune_last_hint.restype = i32
         L.tf_clear_cache.argtypes = []
         L.tf_clear_cache.restype = None
         L.tf_launch_count.argtypes = []
@@ -512,6 +516,36 @@ def tf_candidates(op, rows: int, cols: int, dt: int) -> list[str]:
 
 def tf_device_status():
     _ok(lib().tf_device_status(), "tf_device_status")
+
+
+def _parse_hint(text: str) -> dict:
+    out = {}
+    for part in text.split(" "):
+        if "=" in part:
+            k, v = part.split("=", 1)
+            if k == "first":
+                out[k] = [q for q in v.split(";") if q]
+            elif k == "rule":
+                out[k] = v
+            else:
+                out[k] = float(v)
+    return out
+
+
+def tf_refine_hint(op, rows: int, cols: int, dt: int, plan: str) -> dict:
+    """The refinement hint for ``plan`` on this shape: ``{"rule": ..., "regs": ..., "ctas_per_sm": ..., "occupancy": ...,
+    "waves": ..., "tail": ..., "inflight_kb": ..., "vs_copy": ..., "first": [plans the refinement would try first]}``."""
+    code = OP_CODE[op] if isinstance(op, str) else int(op)
+    buf = ctypes.create_string_buffer(1024)
+    _ok(lib().tf_refine_hint(code, rows, cols, dt, plan.encode(), buf, 1024), "tf_refine_hint")
+    return _parse_hint(buf.value.decode())
+
+
+def tf_tune_last_hint() -> dict:
+    """The hint ``tf_tune`` computed for the heuristic plan in its last run on this thread."""
+    buf = ctypes.create_string_buffer(256)
+    _ok(lib().tf_tune_last_hint(buf, 256), "tf_tune_last_hint")
+    return _parse_hint(buf.value.decode())
 
 
 def tf_debug_wait_probe(src, budget_cycles: int = 2_000_000) -> bool:

@@ -155,6 +155,9 @@ int round_up(int v, int m) { return (v + m - 1) / m * m; }
 }  // namespace
 
 void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+namespace { thread_local LaunchFacts t_facts; thread_local char t_last_hint[256] = ""; }
+void note_launch(const void* fn, int64_t grid, int threads, size_t dyn_smem, int cluster) { t_facts = LaunchFacts{fn, grid, threads, dyn_smem, cluster}; }
+LaunchFacts last_launch() { return t_facts; }
 int* device_status_word() {
     DevState* ds = nullptr;
     return device_state(&ds) == TF_OK ? ds->status : nullptr;
@@ -474,6 +477,12 @@ std::vector<Plan> neighbours(const Plan& b) {
     if (b.variant == V_PIPE || b.variant == V_WARP)
         for (int r : {1, 2, 4})
             if (r != b.rpg) with([&](Plan& p) { p.rpg = r; });
+    // the same row on fewer registers per thread: half the vectors per thread on twice the threads (or lanes)
+    if (b.variant == V_PIPE && b.vpt >= 2 && b.lanes * 2 <= 512)
+        with([&](Plan& p) { p.vpt = b.vpt / 2; p.lanes = b.lanes * 2; p.threads = std::max(b.threads, p.lanes) / p.lanes * p.lanes; });
+    if ((b.variant == V_CTA || b.variant == V_RING) && b.vpt >= 2 && b.threads * 2 <= 1024)
+        with([&](Plan& p) { p.vpt = b.vpt / 2; p.threads = b.threads * 2; });
+    if (b.variant == V_WARP && b.vpt >= 2 && b.lanes * 2 <= 32) with([&](Plan& p) { p.vpt = b.vpt / 2; p.lanes = b.lanes * 2; });
     if (b.variant == V_TWOPASS || b.variant == V_RING) with([&](Plan& p) { p.rpg = b.rpg == 2 ? 1 : 2; });
     if (b.variant == V_TWOPASS) {
         if (b.stages >= 2) with([&](Plan& p) { p.unroll = b.unroll == 4 ? 2 : 4; });
@@ -487,6 +496,73 @@ std::vector<Plan> neighbours(const Plan& b) {
         for (int cl : {b.cluster / 2, b.cluster * 2})
             if (cl >= 1 && cl <= kMaxCluster && cl != b.cluster) with([&](Plan& p) { p.cluster = cl; });
     return out;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Targeted refinement hint (Algorithm 1's RefineHint step; the paper's is an LLM reading profiler deltas, Section 3.3).
+// Here the signal is what the library can read about its own launch without a profiler: registers and resident CTAs of
+// the kernel (function attributes, the occupancy calculator), the waves of the grid and the empty share of the last one,
+// the bytes a plan keeps in flight per SM, and the distance to the library's own streaming copy of the same tensors.  A
+// rule table turns the signal into WHICH knobs to try first; a round stops at the first accepted candidate.
+// ------------------------------------------------------------------------------------------------
+struct RefineHint {
+    int regs = 0, ctas_per_sm = 0;
+    float occupancy = 0.f;        // resident threads / 2048
+    float waves = 0.f, tail = 0.f; // grid / resident CTAs; empty share of the last wave
+    float inflight_kb = 0.f;      // bytes of loads or copies a plan keeps in flight per SM
+    float vs_copy = 0.f;          // time / time of the streaming copy of the same tensors (0: not measured)
+    const char* rule = "none";    // occupancy | tail | inflight | ceiling | none
+};
+
+RefineHint make_hint(const Plan& p, const DeviceInfo& d, float plan_us, float copy_us, bool small_problem) {
+    RefineHint h;
+    const LaunchFacts f = last_launch();
+    if (!f.fn) return h;
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, f.fn) != cudaSuccess) { cudaGetLastError(); return h; }
+    h.regs = fa.numRegs;
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, f.fn, f.threads, f.dyn_smem) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    h.ctas_per_sm = n;
+    h.occupancy = static_cast<float>(n) * f.threads / 2048.f;
+    const float resident = std::max(1.f, static_cast<float>(n) * d.sms);
+    h.waves = static_cast<float>(f.grid) / resident;
+    h.tail = h.waves > 1.f ? (std::ceil(h.waves) - h.waves) / std::ceil(h.waves) : 0.f;
+    const float ctas = static_cast<float>(std::max<int64_t>(1, std::min<int64_t>(n, (f.grid + d.sms - 1) / d.sms)));
+    switch (p.variant) {
+        case V_WARP: h.inflight_kb = ctas * f.threads * p.vpt * p.rpg * 16 / 1024.f; break;
+        case V_CTA: h.inflight_kb = ctas * f.threads * p.vpt * 16 / 1024.f; break;
+        case V_TWOPASS: h.inflight_kb = p.stages >= 2 ? ctas * f.dyn_smem * (p.stages - 1) / p.stages / 1024.f : ctas * f.threads * 4 * 16 / 1024.f; break;
+        case V_STREAM: h.inflight_kb = ctas * f.threads * 4 / 1024.f; break;
+        default: h.inflight_kb = ctas * f.dyn_smem / 1024.f; break;           // the staged variants: their rings are what is in flight
+    }
+    h.vs_copy = copy_us > 0.f ? plan_us / copy_us : 0.f;
+    if (!small_problem && h.vs_copy > 0.f && h.vs_copy <= 1.02f) h.rule = "ceiling";
+    else if (h.occupancy <= 0.25f && h.regs > 96) h.rule = "occupancy";
+    else if (h.tail > 0.15f) h.rule = "tail";
+    else if (h.inflight_kb < 40.f) h.rule = "inflight";
+    return h;
+}
+
+// Does candidate c turn, relative to the incumbent b, a knob that the fired rule names?
+bool hinted(const RefineHint& h, const Plan& b, const Plan& c) {
+    const std::string r = h.rule;
+    if (r == "occupancy")       // fewer registers per thread or smaller CTAs: fewer vectors or rows per thread, a capped build, fewer threads
+        return c.vpt < b.vpt || (c.threads < b.threads && c.vpt == b.vpt) || (b.variant != V_TWOPASS && b.variant != V_RING && c.rpg < b.rpg) ||
+               (b.variant == V_TWOPASS && c.rpg == 2 && b.rpg != 2) || c.unroll < b.unroll;
+    if (r == "tail")            // a grid that does not end in a part-empty wave: persistent CTAs, finer units of work
+        return (b.persist == 0 && c.persist > 0) || c.cluster > b.cluster || c.threads < b.threads;
+    if (r == "inflight")        // more bytes in flight: deeper rings, larger stages, more resident CTAs or threads
+        return c.stages > b.stages || c.chunk > b.chunk || c.persist > b.persist || c.threads > b.threads || c.unroll > b.unroll ||
+               (b.variant == V_WARP && c.rpg > b.rpg);
+    return false;
+}
+
+std::string hint_to_string(const RefineHint& h) {
+    char b[200];
+    snprintf(b, sizeof b, "rule=%s regs=%d ctas_per_sm=%d occupancy=%.2f waves=%.2f tail=%.2f inflight_kb=%.0f vs_copy=%.3f", h.rule, h.regs,
+             h.ctas_per_sm, h.occupancy, h.waves, h.tail, h.inflight_kb, h.vs_copy);
+    return b;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -851,12 +927,7 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
     // Profile: 3 warm-up batches, then 5 timed regions, CUDA events, median per launch.  A batch is one launch per
     // buffer set; a region repeats the batch until it lasts about 2 ms (the last warm-up batch is timed to size it), so
     // that an event pair never brackets just a launch or two.
-    auto profile = [&](const Plan& p, float* us) -> bool {
-        auto batch = [&]() -> bool {
-            for (int k = 0; k < K; ++k)
-                if (launch_it(p, args_for(k, ys[k])) != cudaSuccess) { cudaGetLastError(); return false; }
-            return true;
-        };
+    auto profile_batch = [&](auto&& batch, float* us) -> bool {
         float ms = 0.f;
         for (int rep = 0; rep < 3; ++rep) {
             if (rep == 2) cudaEventRecord(ev[0], st);
@@ -879,6 +950,13 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
         std::sort(t, t + 5);
         *us = t[2];
         return true;
+    };
+    auto profile = [&](const Plan& p, float* us) -> bool {
+        return profile_batch([&]() -> bool {
+            for (int k = 0; k < K; ++k)
+                if (launch_it(p, args_for(k, ys[k])) != cudaSuccess) { cudaGetLastError(); return false; }
+            return true;
+        }, us);
     };
 
     const Args probe = args_for(0, ys[0]);
@@ -907,13 +985,43 @@ static tf_status tune_impl(int op, int64_t rows, int64_t cols, int dt, const voi
         if (us < 0.98f * best_us) { best = c; best_us = us; return true; }             // Arbiter: accept only a measured improvement
         return false;
     };
-    // Proposals: the fixed list of launch geometries around the row size.
-    for (const Plan& c : candidates(probe, dev)) consider(c);
-    // Targeted refinement (Algorithm 1's RefineHint, rule-based): one-parameter neighbours of the best plan so far,
-    // repeated while a round still brings a measured improvement, at most 8 rounds (the paper's iteration cap).
-    for (int round = 0; round < 8; ++round) {
+    // The ceiling this shape has on this device: the library's own streaming copy of the same tensors, timed like a plan.
+    float copy_us = 0.f;
+    if (!profile_batch([&]() -> bool {
+            for (int k = 0; k < K; ++k)
+                if (tf_copy(xs[k], ys[k], static_cast<int64_t>(tensor_bytes), st) != TF_OK) return false;
+            return true;
+        }, &copy_us)) copy_us = 0.f;
+    const bool small_problem = 2 * tensor_bytes < static_cast<size_t>(dev.l2_bytes) / 4;      // L2-resident: the copy is no ceiling there
+    auto hint_for_best = [&]() -> RefineHint {
+        launch_it(best, args_for(0, ys[0]));                     // refresh the launch facts of the incumbent
+        cudaStreamSynchronize(st);
+        return make_hint(best, dev, best_us, copy_us, small_problem);
+    };
+    RefineHint hint = hint_for_best();
+    snprintf(t_last_hint, sizeof t_last_hint, "%s", hint_to_string(hint).c_str());
+    if (log) fprintf(stderr, "tf_tune: copy %8.2f us; heuristic: %s\n", copy_us, t_last_hint);
+    // Proposals: the fixed list of launch geometries around the row size; skipped when the incumbent already runs at the
+    // copy ceiling, cut short as soon as a proposal gets there ("accept ... finish", Algorithm 1).
+    const bool at_ceiling0 = std::string(hint.rule) == "ceiling";
+    if (!at_ceiling0)
+        for (const Plan& c : candidates(probe, dev)) {
+            consider(c);
+            if (!small_problem && copy_us > 0.f && best_us <= 1.02f * copy_us) break;
+        }
+    // Targeted refinement: one-parameter neighbours of the best plan so far, the knobs the hint names first; a round ends
+    // at the first accepted candidate ("continue") and refinement ends after a round without one or at the ceiling
+    // ("finish"), at most 8 rounds (the paper's iteration cap).
+    for (int round = 0; round < 8 && !at_ceiling0; ++round) {
+        hint = hint_for_best();
+        if (log) fprintf(stderr, "tf_tune: refinement round %d: %s\n", round + 1, hint_to_string(hint).c_str());
+        if (std::string(hint.rule) == "ceiling") break;
+        std::vector<Plan> nb = neighbours(best);
+        const Plan incumbent = best;
+        std::stable_partition(nb.begin(), nb.end(), [&](const Plan& c) { return hinted(hint, incumbent, c); });
         bool improved = false;
-        for (const Plan& c : neighbours(best)) improved |= consider(c);
+        for (const Plan& c : nb)
+            if (consider(c)) { improved = true; break; }
         if (log) fprintf(stderr, "tf_tune: refinement round %d: %s\n", round + 1, improved ? "continue" : "finish");
         if (!improved) break;                                                            // diminishing returns: finish
     }
@@ -1033,6 +1141,44 @@ tf_status tf_debug_wait_probe(const void* src16, int64_t budget_cycles, int* gav
     k_wait_probe<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint4*>(src16), budget_cycles, ds->status, gave_up);
     const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? TF_OK : cuda_fail(e);
+}
+
+tf_status tf_tune_last_hint(char* buf, size_t n) {
+    if (!buf || n == 0) return TF_ERR_INVALID_ARG;
+    snprintf(buf, n, "%s", t_last_hint);
+    return TF_OK;
+}
+
+tf_status tf_refine_hint(tf_op op_, int64_t rows, int64_t cols, tf_dtype dt_, const char* plan, char* buf, size_t n) {
+    const int op = op_, dt = dt_;
+    Plan p;
+    if (!buf || n == 0 || !plan || op < 0 || op >= OP_COUNT || bad_shape(rows, cols, dt) || rows == 0 || !plan_from_string(plan, p)) return TF_ERR_INVALID_ARG;
+    if (too_big(rows, cols)) return TF_ERR_UNSUPPORTED;
+    DevState* ds = nullptr;
+    tf_status s = device_state(&ds);
+    if (s != TF_OK) return s;
+    Scratch sc;
+    const size_t bytes = static_cast<size_t>(rows) * cols * elem_size(dt);
+    void* x = sc.get(bytes);
+    void* y = sc.get(bytes);
+    void* p0 = sc.get(static_cast<size_t>(cols) * 4);
+    void* p1 = sc.get(static_cast<size_t>(cols) * 4);
+    if (!x || !y || !p0 || !p1) return TF_ERR_NOMEM;
+    cudaMemset(x, 0, bytes); cudaMemset(p0, 0, static_cast<size_t>(cols) * 4); cudaMemset(p1, 0, static_cast<size_t>(cols) * 4);
+    Args a{op, dt, x, p0, p1, y, nullptr, nullptr, rows, cols, op == OP_SOFTMAX ? 0.f : 1e-5f, ds->status};
+    if (!supports(p, a, ds->info)) return TF_ERR_UNSUPPORTED;
+    cudaError_t e = launch(p, a, ds->info, nullptr);
+    if (e != cudaSuccess || (e = cudaDeviceSynchronize()) != cudaSuccess) return cuda_fail(e);
+    const RefineHint h = make_hint(p, ds->info, 0.f, 0.f, false);
+    std::vector<Plan> nb = neighbours(p);
+    std::stable_partition(nb.begin(), nb.end(), [&](const Plan& c) { return hinted(h, p, c); });
+    std::string out = hint_to_string(h) + " first=";
+    int shown = 0;
+    for (int pass = 0; pass < 2 && shown == 0; ++pass)          // the neighbours the rule names; the plain order if it names none
+        for (const Plan& c : nb)
+            if ((pass == 1 || hinted(h, p, c)) && supports(c, a, ds->info) && shown < 3) { out += (shown ? ";" : "") + plan_to_string(c); ++shown; }
+    snprintf(buf, n, "%s", out.c_str());
+    return TF_OK;
 }
 
 tf_status tf_debug_tune_inject_timeout(const char* plan_prefix) {

@@ -90,6 +90,7 @@ cudaError_t launch_pipe(const Plan& p, const Args& a, const DeviceInfo& d, cudaS
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    note_launch(reinterpret_cast<const void*>(fn), grid, p.threads, g.smem, 1);
     return cudaLaunchKernelEx(&cfg, fn, k);
 }
 

@@ -99,6 +99,12 @@ cudaError_t launch_softmax_len_scalar(const Args&, cudaStream_t);
 Plan heuristic_softmax_len(const Args&, const DeviceInfo&);
 size_t split_scratch_bytes(const Plan&, const Args&);
 
+// What the launcher of a forward plan last launched on this host thread (kernel, grid, CTA size, dynamic shared memory,
+// CTAs per cluster): the tuner's refinement hint reads the kernel's registers and its occupancy from these.
+struct LaunchFacts { const void* fn = nullptr; int64_t grid = 0; int threads = 0; size_t dyn_smem = 0; int cluster = 1; };
+void note_launch(const void* fn, int64_t grid, int threads, size_t dyn_smem, int cluster);
+LaunchFacts last_launch();
+
 // Bookkeeping shared with the C ABI layer: count kernel launches; remember the CUDA error behind a TF_ERR_CUDA.
 void count_launches(int n);
 void clear_norm_bwd_tuned();   // forgets what tf_tune_norm_bwd kept

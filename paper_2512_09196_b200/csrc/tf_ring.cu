@@ -289,6 +289,7 @@ cudaError_t launch_ring(const Plan& p, const Args& a, const DeviceInfo& d, cudaS
     }
     clusters = std::min<int64_t>(clusters, a.rows);
     cfg.gridDim = dim3(static_cast<unsigned>(clusters * p.cluster));
+    note_launch(reinterpret_cast<const void*>(fn), clusters * p.cluster, p.threads, cfg.dynamicSmemBytes, p.cluster);
     return cudaLaunchKernelEx(&cfg, fn, k);
 }
 

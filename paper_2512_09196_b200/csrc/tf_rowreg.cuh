@@ -299,6 +299,7 @@ inline cudaError_t launch_warp_fn(WarpFn fn, const Plan& p, const Args& a, const
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    note_launch(reinterpret_cast<const void*>(fn), grid, p.threads, 0, 1);
     return cudaLaunchKernelEx(&cfg, fn, make_kargs(a));
 }
 
@@ -319,6 +320,7 @@ inline cudaError_t launch_cta_fn(CtaFn fn, const Plan& p, const Args& a, const D
     attr[1].val.clusterDim.x = p.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = p.cluster > 1 ? 2 : 1;
+    note_launch(reinterpret_cast<const void*>(fn), clusters * p.cluster, p.threads, 0, p.cluster);
     return cudaLaunchKernelEx(&cfg, fn, make_kargs(a), p.cluster);
 }
 

@@ -111,6 +111,7 @@ cudaError_t launch_one(SplitFn fn, const SplitArgs& k, dim3 grid, int threads, c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    note_launch(reinterpret_cast<const void*>(fn), static_cast<int64_t>(grid.x) * grid.y, threads, 0, 1);
     return cudaLaunchKernelEx(&cfg, fn, k);
 }
 

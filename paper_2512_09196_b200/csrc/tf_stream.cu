@@ -112,6 +112,7 @@ cudaError_t launch_stream(const Plan& p, const Args& a, const DeviceInfo& d, cud
     if (p.persist > 0) grid = std::min<int64_t>(grid, static_cast<int64_t>(p.persist) * d.sms);
     grid = std::min<int64_t>(grid, 0x7FFFFFFF);
     SArgs k{a.x, a.p0, a.p1, a.y, a.mean, a.rstd, a.rows, a.cols, a.eps};
+    note_launch(reinterpret_cast<const void*>(fn), grid, p.threads, 0, 1);
     fn<<<static_cast<unsigned>(grid), p.threads, 0, st>>>(k);
     return cudaGetLastError();
 }

@@ -306,6 +306,7 @@ cudaError_t launch_tma(const Plan& p, const Args& a, const DeviceInfo& d, cudaSt
     attr[1].val.clusterDim.x = p.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = p.cluster > 1 ? 2 : 1;
+    note_launch(reinterpret_cast<const void*>(fn), clusters * p.cluster, p.threads, g.smem, p.cluster);
     return cudaLaunchKernelEx(&cfg, fn, k);
 }
 

@@ -374,11 +374,13 @@ TwoFn ring_fn_c(int op, int dt) {
 }
 template <int U, int MAXT, int MINB>
 TwoFn ring_fn_b(int op, int dt, bool cl) { return cl ? ring_fn_c<U, MAXT, MINB, true>(op, dt) : ring_fn_c<U, MAXT, MINB, false>(op, dt); }
-// regcap: the builds held to 40 registers (three CTAs of 512 threads, or four of 384, per SM)
+// regcap: the builds whose registers are held to what three CTAs per SM leave each thread: 56 for CTAs of up to 384
+// threads, 40 for CTAs of up to 512
 TwoFn ring_fn(int op, int dt, int unroll, int threads, bool capped, bool cl) {
     if (unroll == 2) return (capped && threads <= 512) ? ring_fn_b<2, 512, 3>(op, dt, cl) : ring_fn_b<2, 1024, 1>(op, dt, cl);
-    if (unroll == 4) return (capped && threads <= 512) ? ring_fn_b<4, 512, 3>(op, dt, cl) : ring_fn_b<4, 1024, 1>(op, dt, cl);
-    return nullptr;
+    if (unroll != 4) return nullptr;
+    if (capped && threads <= 384) return ring_fn_b<4, 384, 3>(op, dt, cl);
+    return (capped && threads <= 512) ? ring_fn_b<4, 512, 3>(op, dt, cl) : ring_fn_b<4, 1024, 1>(op, dt, cl);
 }
 
 }  // namespace
@@ -440,6 +442,7 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
+    note_launch(reinterpret_cast<const void*>(fn), grid * cs, p.threads, smem, cs);
     return cudaLaunchKernelEx(&cfg, fn, k);
 }
 
