@@ -12,7 +12,9 @@
  *              The library keeps no reference after the call returns.  It allocates nothing, with one
  *              exception: for a handful of very long rows (rows <= 4, >= 256 KiB each) the split-row plan takes
  *              8 bytes per row segment from the stream-ordered allocator (cudaMallocAsync / cudaFreeAsync on the
- *              caller's stream) for the duration of the call.
+ *              caller's stream) for the duration of the call, so that calls on different streams cannot race on
+ *              shared scratch.  Callers that must never allocate use tf_softmax_fwd_noalloc, or force another
+ *              plan for such shapes (tf_force_plan).
  *   Layout     x and y are dense row-major [rows, cols] (row stride = cols); gamma/beta/weight are [cols];
  *              mean/rstd are [rows], always fp32.  x, y and the parameters share one element type `dt`.
  *   Alignment  Any.  A 16-byte aligned x, y and parameters with cols * sizeof(element) a multiple of 16
@@ -74,8 +76,12 @@ tf_status tf_rmsnorm_fwd(const void* x, const void* weight, void* y, float* rstd
  *   Limits   rows <= 8192; x and y 16-byte aligned and cols * sizeof(element) a multiple of 16.  Anything else
  *            returns TF_ERR_UNSUPPORTED and launches nothing.  Long rows are its purpose; short ones work
  *            but are served better by tf_softmax_fwd.
- *   Set-up   The first call on a device looks up the array's device address (with that device current).  Make
- *            that first call before any stream capture begins.
+ *   Set-up   The first call on a device looks up the array's device address (with that device current).  That
+ *            first use of the library on a device is also when the CUDA runtime loads the library's module
+ *            onto it -- the kernels' code and this 64 KiB array occupy device memory from then on, and the
+ *            runtime takes that memory itself.  So make the first call on each device early: before the
+ *            process hands the remaining free memory to its pool, and before any stream capture begins.
+ *            Later calls touch no allocator at all.
  *   Sharing  Every call on a device uses the same array, which keeps the previous call's partials.  Nothing in
  *            it needs clearing (each call overwrites every partial it later reads), but two calls whose
  *            kernels can overlap on the GPU (different streams without an ordering between them) race on it:
@@ -85,11 +91,17 @@ tf_status tf_softmax_fwd_noalloc(const void* x, void* y, int64_t rows, int64_t c
 /* Measure-and-keep tuning for one (op, rows, cols, dt) on the current device (Algorithm 1 of the paper,
  * with the hand-written launch plans as proposals): starting from the heuristic plan as incumbent, every
  * candidate plan that can launch is run on library-owned scratch tensors, its output is checked against
- * the incumbent's, it is timed with CUDA events (3 warm-up + 5 timed launches, median; the paper's
- * Section 3.4 protocol) on rotating buffers larger than L2, and it replaces the incumbent only if it is
- * at least 2% faster.  After the fixed proposal list, one-parameter neighbours of the best plan are tried in
- * rounds (the rule-based stand-in for Algorithm 1's refinement hint) until a round brings no improvement, at
- * most 8 rounds (the paper's iteration cap).  The winner is cached in memory (and in the file named by the TF_TUNE_CACHE
+ * the incumbent's at the level of the parity tolerances (two results that both meet them: 2 bf16 ulps, 2e-5 of the
+ * condition scale in fp32), it is timed with CUDA events (3 warm-up batches + 5 timed regions of at least 2 ms each,
+ * median; the paper's Section 3.4 protocol of 3 + 5 runs, with each run made long enough to time) on at least two
+ * rotating buffer sets larger than L2, and it replaces the incumbent only if it is at least 2% faster.  A candidate
+ * that cannot launch, fails that check, or whose bounded device-side wait gives up is dropped and never cached (the
+ * remediation branch of Algorithm 1).  The library's own streaming copy of the same tensors is timed the same way as
+ * the ceiling of the shape: tuning ends at once when the incumbent is within 2% of it, and the proposal list is cut
+ * short when a proposal gets there.  After the proposals come refinement rounds: the one-parameter neighbours of the
+ * best plan, the knobs named by the refinement hint first (see tf_refine_hint), a round ending at the first accepted
+ * candidate ("continue") and refinement ending after a round without one ("finish"), at most 8 rounds (the paper's
+ * iteration cap).  The winner is cached in memory (and in the file named by the TF_TUNE_CACHE
  * environment variable, if set) and used by later *_fwd calls with the same key.  Blocking; allocates and
  * frees its own scratch; assumes 16-byte aligned tensors. */
 tf_status tf_tune(tf_op op, int64_t rows, int64_t cols, tf_dtype dt);

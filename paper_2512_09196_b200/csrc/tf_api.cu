@@ -199,19 +199,69 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         s.cluster = static_cast<int>(std::max<int64_t>(2, std::min<int64_t>(nvec / 256, 2 * d.sms / a.rows)));
         if (supports_split(s, a, d)) return s;
     }
-    if (a.op == OP_SOFTMAX && nvec >= 16384 && a.rows >= 16LL * d.sms) {
-        // many rows of 256 KiB and more: two streamed passes with each thread's loads running ahead of its arithmetic in a
-        // private shared-memory ring, a pair of CTAs per row (three CTAs of 384 threads per SM); measured 328 us on the
-        // 2 GiB masked softmax against 360-460 us for every plan that keeps the row on chip
+    // Long rows, read off the tuner's winners on the sweep and the 2 GiB softmax: two streamed passes.  The ring form
+    // (each thread's loads run ahead of its arithmetic in a private shared-memory ring) for softmax from 64-128 KiB rows
+    // on, with a pair of CTAs per row from 256 KiB (2 GiB masked softmax: 325-329 us against 360-460 us for every plan
+    // that keeps the row on chip); the direct form for fp32 LayerNorm from 32 KiB and bf16 RMSNorm of 32-64 KiB.
+    {
         Plan s;
-        s.variant = V_TWOPASS; s.threads = 384; s.chunk = 0; s.rpg = 2; s.lanes = 1; s.vpt = 3; s.stages = 3; s.unroll = 4; s.cluster = 2;
-        if (supports_twopass(s, a, d)) return s;
+        s.variant = V_TWOPASS; s.chunk = 0; s.rpg = 2; s.lanes = 1; s.vpt = 3; s.stages = 0; s.unroll = 4; s.cluster = 1; s.persist = 0;
+        auto ring = [&](int threads, int stages, int cluster, bool capped) { s.threads = threads; s.stages = stages; s.cluster = cluster; s.rpg = capped ? 2 : 1; };
+        auto direct = [&](int threads, int cluster) { s.threads = threads; s.stages = 0; s.cluster = cluster; s.rpg = 2; };
+        bool take = false;
+        const bool f32 = a.dt == DT_F32;
+        if (a.op == OP_SOFTMAX) {
+            if (nvec >= 16384) { ring(256, 4, 2, true); take = true; }
+            else if (nvec >= 8192) { ring(384, f32 ? 4 : 2, 1, true); take = true; }
+            else if (nvec >= 4096 && !f32) { ring(256, 2, 1, true); take = true; }
+        } else if (a.op == OP_LAYERNORM) {
+            if (f32 && nvec >= 2048) { direct(nvec < 4096 ? 256 : 512, nvec >= 16384 ? 2 : 1); if (nvec == 8192) s.rpg = 1; take = true; }
+            else if (!f32 && nvec >= 8192) { ring(512, 3, 1, false); take = true; }
+            else if (!f32 && nvec >= 4096) { ring(256, 2, 1, true); take = true; }
+        } else {
+            if (f32 && nvec >= 8192 && nvec < 16384) { ring(512, 3, 1, false); take = true; }
+            else if (f32 && nvec >= 4096 && nvec < 8192) { ring(256, 4, 1, true); take = true; }
+            else if (!f32 && nvec >= 8192) { ring(512, 3, 1, false); take = true; }
+            else if (!f32 && nvec >= 2048) { direct(nvec < 4096 ? 256 : 512, 1); take = true; }
+        }
+        if (take && a.rows >= 2LL * d.sms && supports_twopass(s, a, d)) return s;
     }
     // Rules read off the plans that tf_tune ends up with on the 84-point shape sweep (rows of 128 B to 256 KiB, three ops,
     // two types); what they do not cover falls through to the older defaults below.
     {
         Plan q;
         const bool ln = a.op == OP_LAYERNORM;
+        // widths that are not powers of two (5120 and 12288 columns): the winners are the plans whose geometry the row fills
+        // exactly -- a pipeline unit of 192 threads x 8 vectors for 24 KiB bf16 rows, a CTA of 160 threads x 4 vectors for
+        // 10 KiB ones -- or, where no unit fits, the shared-memory staged CTA per row
+        if (nvec == 1536 && a.dt == DT_BF16 && a.op != OP_RMSNORM) {
+            q.variant = V_PIPE; q.threads = 192; q.lanes = 192; q.vpt = 8; q.rpg = 1; q.stages = 2; q.chunk = 24576; q.persist = 2;
+            if (supports_pipe(q, a, d)) return q;
+        }
+        if ((nvec == 1536 && a.dt == DT_BF16 && a.op == OP_RMSNORM) || (nvec == 1280 && ln && a.dt == DT_F32)) {
+            q = Plan(); q.variant = V_TMA; q.cluster = 1; q.stages = 1; q.persist = 0;
+            q.threads = ln ? 256 : 128; q.chunk = ln ? 32768 : 8192;
+            if (supports_tma(q, a, d)) return q;
+        }
+        if (nvec == 640 && ln && a.dt == DT_BF16) {
+            q = Plan(); q.variant = V_CTA; q.cluster = 1; q.persist = 0; q.vpt = 4; q.threads = 160;
+            if (supports_cta(q, a, d)) return q;
+        }
+        if (nvec == 1024 && ln) {                      // LayerNorm rows of 16 KiB: four warps per row, two units per CTA
+            q = Plan(); q.variant = V_PIPE; q.threads = 256; q.lanes = 128; q.vpt = 8; q.rpg = 1; q.persist = 1;
+            q.stages = a.dt == DT_F32 ? 3 : 2; q.chunk = a.dt == DT_F32 ? 16384 : 32768;
+            if (supports_pipe(q, a, d)) return q;
+        }
+        q = Plan();
+        if (nvec == 256 && !ln && a.dt == DT_BF16) {
+            // bf16 rows of 4 KiB (softmax, RMSNorm): two warps per row with four vectors per thread beat a lane group with eight
+            q.variant = V_CTA; q.cluster = 1; q.persist = 0; q.vpt = 4; q.threads = 64;
+            if (supports_cta(q, a, d)) return q;
+        }
+        if (nvec == 512 && ln && a.dt == DT_F32) {
+            q.variant = V_CTA; q.cluster = 1; q.persist = 0; q.vpt = 4; q.threads = 128;
+            if (supports_cta(q, a, d)) return q;
+        }
         if (nvec <= 256 && !(ln && a.dt == DT_BF16)) {
             // rows up to 4 KiB: a lane group per row, every load issued at once, as many small CTAs as there are row blocks
             q.variant = V_WARP; q.threads = 128; q.persist = 0; q.rpg = 1;
@@ -219,14 +269,14 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
             else if (nvec <= 16) { q.lanes = 8; q.vpt = 2; q.rpg = ln ? 2 : 1; }
             else if (nvec <= 32) { q.lanes = 16; q.vpt = 2; q.rpg = ln ? 2 : 1; }
             else if (nvec <= 64) { q.lanes = 32; q.vpt = 2; q.rpg = (a.dt == DT_F32 && a.op != OP_SOFTMAX) ? 2 : 1; }
-            else if (nvec <= 128) { q.lanes = 32; q.vpt = 4; }
+            else if (nvec <= 128) { q.lanes = 32; q.vpt = 4; q.rpg = (a.op == OP_RMSNORM && a.dt == DT_BF16) ? 2 : 1; }
             else { q.lanes = 32; q.vpt = 8; }
             if (supports_warp(q, a, d)) return q;
         } else if (!ln && nvec <= (a.dt == DT_BF16 ? 1024 : (a.op == OP_SOFTMAX ? 4096 : 3072))) {
             // softmax and RMSNorm from 4 KiB up to 16 KiB (bf16; eight bf16 vectors per thread cost too many registers) or
             // 48-64 KiB (fp32): a CTA per row in registers, four vectors per thread up to 16 KiB, eight beyond
             q.variant = V_CTA; q.cluster = 1; q.persist = 0;
-            q.vpt = nvec <= 1024 ? 4 : 8;
+            q.vpt = (nvec < 1024 || (nvec == 1024 && !(a.op == OP_SOFTMAX && a.dt == DT_BF16))) ? 4 : 8;
             q.threads = std::max(64, round_up(static_cast<int>((nvec + q.vpt - 1) / q.vpt), 32));
             if (supports_cta(q, a, d)) return q;
         } else if (nvec <= 32768 && (nvec > 4096 || (a.op != OP_SOFTMAX && nvec >= 4096) || (ln && nvec >= 2048 && a.dt == DT_F32))) {
@@ -256,16 +306,21 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         else if (nvec <= 1024) { p.lanes = 128; p.vpt = 8; }
         else if (nvec <= 2048) { p.lanes = 256; p.vpt = 8; }
         else { p.lanes = 512; p.vpt = 8; }
-        const int ut = p.lanes < 32 ? 32 : p.lanes;
-        const int64_t pass_bytes = row_bytes * (ut / p.lanes);
-        const int64_t param_bytes = a.op == OP_SOFTMAX ? 0 : row_bytes * (a.op == OP_LAYERNORM ? 2 : 1);
-        const int64_t per_stage = (200 * 1024 - param_bytes) / (p.threads / ut) / p.stages;
         int64_t target = 16384;
         if (nvec <= 256) {                       // rows up to 4 KiB (what reaches here is LayerNorm bf16): the tuner's winners use
             p.persist = 2; target = 4096;        // small stages and two CTAs per SM
             if (nvec <= 16) p.rpg = 2;
+            if (nvec == 64) { p.threads = 256; target = 6144; }
+            if (nvec == 128) { p.threads = 128; p.rpg = 2; p.persist = 0; }
+            if (nvec == 256) { p.threads = 256; p.persist = 0; }
         }
-        p.chunk = static_cast<int>(std::max<int64_t>(pass_bytes, std::min<int64_t>(target, per_stage / p.persist) / pass_bytes * pass_bytes));
+        if (nvec == 512 && a.op == OP_LAYERNORM && a.dt == DT_BF16) { p.lanes = 128; p.vpt = 4; }
+        const int ut = p.lanes < 32 ? 32 : p.lanes;
+        const int64_t pass_bytes = row_bytes * (ut / p.lanes) * p.rpg;
+        const int64_t param_bytes = a.op == OP_SOFTMAX ? 0 : row_bytes * (a.op == OP_LAYERNORM ? 2 : 1);
+        const int64_t per_stage = (200 * 1024 - param_bytes) / (p.threads / ut) / p.stages;
+        const int share = p.persist > 0 ? p.persist : 3;          // non-persistent grids: rings sized for three CTAs per SM
+        p.chunk = static_cast<int>(std::max<int64_t>(pass_bytes, std::min<int64_t>(target, per_stage / share) / pass_bytes * pass_bytes));
         if (supports_pipe(p, a, d)) return p;
         p.persist = 1; p.rpg = 1;
         p.chunk = static_cast<int>(std::max<int64_t>(pass_bytes, std::min<int64_t>(16384, per_stage) / pass_bytes * pass_bytes));
