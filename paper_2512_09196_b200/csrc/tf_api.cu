@@ -210,14 +210,20 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         auto direct = [&](int threads, int cluster) { s.threads = threads; s.stages = 0; s.cluster = cluster; s.rpg = 2; };
         bool take = false;
         const bool f32 = a.dt == DT_F32;
+        // rows of 16-32 KiB: the ring form with CTAs of 128 threads holds the whole row in its two stages, so nothing is
+        // read twice, and a dozen such CTAs fit an SM (RMSNorm bf16 [16384, 8192]: 81 us against 86 us for the pipeline)
+        const bool mid = nvec >= 1024 && nvec <= 2048;
         if (a.op == OP_SOFTMAX) {
             if (nvec >= 16384) { ring(256, 4, 2, true); take = true; }
             else if (nvec >= 8192) { ring(384, f32 ? 4 : 2, 1, true); take = true; }
             else if (nvec >= 4096 && !f32) { ring(256, 2, 1, true); take = true; }
+            else if (nvec == 2048 && !f32) { ring(128, 2, 1, true); take = true; }
         } else if (a.op == OP_LAYERNORM) {
             if (f32 && nvec >= 2048) { direct(nvec < 4096 ? 256 : 512, nvec >= 16384 ? 2 : 1); if (nvec == 8192) s.rpg = 1; take = true; }
             else if (!f32 && nvec >= 8192) { ring(512, 3, 1, false); take = true; }
             else if (!f32 && nvec >= 4096) { ring(256, 2, 1, true); take = true; }
+            else if (mid) { ring(128, 2, 1, true); take = true; }
+        } else if (!f32 && nvec == 1024) { ring(128, 2, 1, true); take = true;
         } else {
             if (f32 && nvec >= 8192 && nvec < 16384) { ring(512, 3, 1, false); take = true; }
             else if (f32 && nvec >= 4096 && nvec < 8192) { ring(256, 4, 1, true); take = true; }
@@ -314,7 +320,7 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
             if (nvec == 128) { p.threads = 128; p.rpg = 2; p.persist = 0; }
             if (nvec == 256) { p.threads = 256; p.persist = 0; }
         }
-        if (nvec == 512 && a.op == OP_LAYERNORM && a.dt == DT_BF16) { p.lanes = 128; p.vpt = 4; }
+        if (nvec == 512 && a.op == OP_LAYERNORM && a.dt == DT_BF16 && a.rows >= 24576) { p.lanes = 128; p.vpt = 4; }
         const int ut = p.lanes < 32 ? 32 : p.lanes;
         const int64_t pass_bytes = row_bytes * (ut / p.lanes) * p.rpg;
         const int64_t param_bytes = a.op == OP_SOFTMAX ? 0 : row_bytes * (a.op == OP_LAYERNORM ? 2 : 1);
@@ -467,9 +473,9 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
     // two streamed passes fed through per-thread rings of asynchronous copies
     if (nvec >= 1024)
         for (int cl : {1, 2})
-            for (int th : {256, 384, 512})
+            for (int th : {64, 128, 256, 384, 512})
                 for (int su : {24, 34, 44}) {                          // (stages, vectors per step)
-                    if (cl > 1 && nvec < 4096) continue;
+                    if ((cl > 1 && nvec < 4096) || (th < 256 && (nvec > 4096 || cl > 1))) continue;
                     Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = 0; p.lanes = 1; p.vpt = 3; p.chunk = 0; p.cluster = cl;
                     p.stages = su / 10; p.unroll = su % 10; p.rpg = 2;
                     add(p);

@@ -137,6 +137,17 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     for (int v = 0; v < VPL; ++v) valid[v] = FULL || (lane + v * LANES) < a.nvec;
     const GroupRed<(LANES < 32 ? LANES : 32)> red;
     const SmemParams par{params, a.nvec, lane, LANES};
+    // a thread that owns one or two vectors per row (lane groups of narrow rows) keeps its parameters widened in registers
+    constexpr bool kHeldWide = OP != OP_SOFTMAX && VPL <= 2 && LANES <= 32;
+    HeldWideParams<DT, kHeldWide ? VPL : 1> wide;
+    if constexpr (kHeldWide) {
+#pragma unroll
+        for (int v = 0; v < VPL; ++v) {
+            const bool have = valid[v];
+            Pairs<DT>::unpack(have ? par.gamma(v) : make_uint4(0, 0, 0, 0), wide.g[v]);
+            Pairs<DT>::unpack((have && OP == OP_LAYERNORM) ? par.beta(v) : make_uint4(0, 0, 0, 0), wide.b[v]);
+        }
+    }
     const uint4 fill = fill_vec<DT>(OP);
     // element count of warp w's slice of a row (multi-warp units): lanes 32w .. 32w+31 own vectors l + v*LANES
     auto slice_count = [&](int w) {
@@ -218,7 +229,8 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
                 issue(next, s, pref_len);
                 if constexpr (LEN) pref_len = len_of(next + GU);
             }
-            slice_finish_rows<OP, DT, VPL, RPG, (W == 1), FULL>(livev, w, tot, par, out);
+            if constexpr (kHeldWide) slice_finish_rows<OP, DT, VPL, RPG, (W == 1), FULL>(livev, w, tot, wide, out);
+            else slice_finish_rows<OP, DT, VPL, RPG, (W == 1), FULL>(livev, w, tot, par, out);
 #pragma unroll
             for (int q = 0; q < RPG; ++q) {
                 if (live[q]) {

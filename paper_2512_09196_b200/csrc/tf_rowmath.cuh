@@ -40,6 +40,28 @@ struct LazyParams {
     __device__ __forceinline__ uint4 beta(int v) const { return ld_param(p1 + first + v * stride); }
 };
 
+// Parameters of a persistent thread's own columns, widened to fp32 pairs once and kept in registers (worth it where a
+// thread owns one or two vectors per row: a 2-byte gamma / beta then costs neither a load nor a widening per row).
+template <int DT, int NV> struct HeldWideParams {
+    F2 g[NV][Pairs<DT>::NP], b[NV][Pairs<DT>::NP];
+};
+
+// gamma / beta of vector v as fp32 pairs, whatever the provider keeps them as.
+template <int DT, class Par>
+__device__ __forceinline__ void load_gamma(const Par& par, int v, F2 (&g)[Pairs<DT>::NP]) { Pairs<DT>::unpack(par.gamma(v), g); }
+template <int DT, class Par>
+__device__ __forceinline__ void load_beta(const Par& par, int v, F2 (&b)[Pairs<DT>::NP]) { Pairs<DT>::unpack(par.beta(v), b); }
+template <int DT, int NV>
+__device__ __forceinline__ void load_gamma(const HeldWideParams<DT, NV>& par, int v, F2 (&g)[Pairs<DT>::NP]) {
+#pragma unroll
+    for (int i = 0; i < Pairs<DT>::NP; ++i) g[i] = par.g[v][i];
+}
+template <int DT, int NV>
+__device__ __forceinline__ void load_beta(const HeldWideParams<DT, NV>& par, int v, F2 (&b)[Pairs<DT>::NP]) {
+#pragma unroll
+    for (int i = 0; i < Pairs<DT>::NP; ++i) b[i] = par.b[v][i];
+}
+
 // Keeps the first `keep` (1 .. NE-1) elements of a vector and replaces the rest by -inf.
 template <int DT> __device__ __forceinline__ uint4 mask_tail(const uint4& v, int keep) {
     uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -176,7 +198,11 @@ __device__ __forceinline__ void slice_finish_rows(const bool (&valid)[NV], F2 (&
     constexpr int NP = P::NP;
     F2 ta[R], tb[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) { ta[r] = f2(t[r].a); tb[r] = f2(t[r].b); }
+    for (int r = 0; r < R; ++r) {
+        // LayerNorm: (x - mean) rstd gamma + beta as two fused multiply-adds, x rstd + (-mean rstd) first: ta holds -mean rstd
+        ta[r] = f2(OP == OP_LAYERNORM ? -t[r].a * t[r].b : t[r].a);
+        tb[r] = f2(t[r].b);
+    }
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
         if constexpr (OP == OP_SOFTMAX) {
@@ -195,19 +221,19 @@ __device__ __forceinline__ void slice_finish_rows(const bool (&valid)[NV], F2 (&
         } else if constexpr (OP == OP_LAYERNORM) {
             if (ALLV || valid[v]) {
                 F2 g[NP], b[NP];
-                P::unpack(par.gamma(v), g);
-                P::unpack(par.beta(v), b);
+                load_gamma<DT>(par, v, g);
+                load_beta<DT>(par, v, b);
 #pragma unroll
                 for (int r = 0; r < R; ++r)
 #pragma unroll
-                    for (int i = 0; i < NP; ++i) w[r][v][i] = fma2(mul2(sub2(w[r][v][i], ta[r]), tb[r]), g[i], b[i]);
+                    for (int i = 0; i < NP; ++i) w[r][v][i] = fma2(fma2(w[r][v][i], tb[r], ta[r]), g[i], b[i]);
             }
 #pragma unroll
             for (int r = 0; r < R; ++r) out[r][v] = P::pack(w[r][v]);
         } else {
             if (ALLV || valid[v]) {
                 F2 g[NP];
-                P::unpack(par.gamma(v), g);
+                load_gamma<DT>(par, v, g);
 #pragma unroll
                 for (int r = 0; r < R; ++r)
 #pragma unroll

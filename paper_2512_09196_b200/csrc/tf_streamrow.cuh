@@ -214,10 +214,13 @@ __device__ __forceinline__ RowScale scale_of_row(const Part& p, float n, float e
     else { const float rr = fast_rsqrt(fast_div(p.a, n) + eps); return RowScale{rr, rr}; }
 }
 
+__device__ __forceinline__ float ta2_lo(F2 a) { float lo, hi; split(a, lo, hi); return lo; }
+
 // The normalised form of one vector: softmax 2^(x log2e + O) / S (ta2 = O, tb2 = 1/S; -inf elements need no test:
 // 2^(-inf) is +0, and +0 times 1/S is +0), LayerNorm (x - mean) rstd gamma + beta, RMSNorm x rrms w.
 // g, b: the parameter vectors of this column (read only for the norms).
-template <int OP, int DT>
+// SMEM: g and b point into shared memory (parameters staged there by the caller), else into global memory.
+template <int OP, int DT, bool SMEM = false>
 __device__ __forceinline__ uint4 apply_vec(const uint4& raw, const uint4* g, const uint4* b, const F2 ta2, const F2 tb2) {
     using P = Pairs<DT>;
     constexpr int NP = P::NP;
@@ -228,14 +231,16 @@ __device__ __forceinline__ uint4 apply_vec(const uint4& raw, const uint4* g, con
 #pragma unroll
         for (int i = 0; i < NP; ++i) w[i] = mul2(ex2_ftz2(fma2(w[i], l2e, ta2)), tb2);
     } else if constexpr (OP == OP_LAYERNORM) {
+        // (x - mean) rstd gamma + beta as two fused multiply-adds: x rstd + (-mean rstd), then times gamma plus beta
         F2 gg[NP], bb[NP];
-        P::unpack(ld_param(g), gg);
-        P::unpack(ld_param(b), bb);
+        P::unpack(SMEM ? *g : ld_param(g), gg);
+        P::unpack(SMEM ? *b : ld_param(b), bb);
+        const F2 nmr2 = f2(-ta2_lo(ta2) * ta2_lo(tb2));
 #pragma unroll
-        for (int i = 0; i < NP; ++i) w[i] = fma2(mul2(sub2(w[i], ta2), tb2), gg[i], bb[i]);
+        for (int i = 0; i < NP; ++i) w[i] = fma2(fma2(w[i], tb2, nmr2), gg[i], bb[i]);
     } else {
         F2 gg[NP];
-        P::unpack(ld_param(g), gg);
+        P::unpack(SMEM ? *g : ld_param(g), gg);
 #pragma unroll
         for (int i = 0; i < NP; ++i) w[i] = mul2(mul2(w[i], ta2), gg[i]);
     }
