@@ -216,19 +216,20 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         if (a.op == OP_SOFTMAX) {
             if (nvec >= 16384) { ring(256, 4, 2, true); take = true; }
             else if (nvec >= 8192) { ring(384, f32 ? 4 : 2, 1, true); take = true; }
-            else if (nvec >= 4096 && !f32) { ring(256, 2, 1, true); take = true; }
-            else if (nvec == 2048 && !f32) { ring(128, 2, 1, true); take = true; }
+            else if (nvec >= 4096 && !f32) { ring(256, 2, 1, false); take = true; }
+            else if (nvec == 2048 && !f32) { ring(128, 2, 1, false); take = true; }
         } else if (a.op == OP_LAYERNORM) {
             if (f32 && nvec >= 2048) { direct(nvec < 4096 ? 256 : 512, nvec >= 16384 ? 2 : 1); if (nvec == 8192) s.rpg = 1; take = true; }
-            else if (!f32 && nvec >= 8192) { ring(512, 3, 1, false); take = true; }
-            else if (!f32 && nvec >= 4096) { ring(256, 2, 1, true); take = true; }
-            else if (mid) { ring(128, 2, 1, true); take = true; }
-        } else if (!f32 && nvec == 1024) { ring(128, 2, 1, true); take = true;
+            else if (!f32 && nvec >= 8192) { ring(512, nvec >= 16384 ? 3 : 2, 1, false); take = true; }
+            else if (!f32 && nvec >= 4096) { ring(256, 2, 1, false); take = true; }
+            else if (mid) { ring(128, 2, 1, false); take = true; }
+        } else if (!f32 && nvec == 1024) { ring(128, 2, 1, false); take = true;
         } else {
             if (f32 && nvec >= 8192 && nvec < 16384) { ring(512, 3, 1, false); take = true; }
             else if (f32 && nvec >= 4096 && nvec < 8192) { ring(256, 4, 1, true); take = true; }
             else if (!f32 && nvec >= 8192) { ring(512, 3, 1, false); take = true; }
-            else if (!f32 && nvec >= 2048) { direct(nvec < 4096 ? 256 : 512, 1); take = true; }
+            else if (!f32 && nvec >= 4096) { ring(256, 4, 1, false); take = true; }
+            else if (!f32 && nvec >= 2048) { direct(256, 1); take = true; }
         }
         if (take && a.rows >= 2LL * d.sms && supports_twopass(s, a, d)) return s;
     }
@@ -477,9 +478,10 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
                 for (int su : {24, 34, 44}) {                          // (stages, vectors per step)
                     if ((cl > 1 && nvec < 4096) || (th < 256 && (nvec > 4096 || cl > 1))) continue;
                     Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = 0; p.lanes = 1; p.vpt = 3; p.chunk = 0; p.cluster = cl;
-                    p.stages = su / 10; p.unroll = su % 10; p.rpg = 2;
-                    add(p);
-                    if (th == 512 && su == 34) { p.rpg = 1; add(p); }
+                    p.stages = su / 10; p.unroll = su % 10;
+                    // up to 256 threads the 64-register build holds as many CTAs per SM as the capped one; above, try both
+                    p.rpg = 1; add(p);
+                    if (th > 256) { p.rpg = 2; add(p); }
                 }
     // persistent cluster ring for long rows
     if (nvec >= 2048)

@@ -42,6 +42,8 @@ struct WArgs {
     int groups;           // row order: launch slot b works on row (b % groups) * ceil(rows / groups) + b / groups
     int64_t slots;        // groups * ceil(rows / groups)
     int stages;           // ring form: steps per thread's ring
+    int64_t per_group;    // slots / groups
+    int step, nfull, rag; // ring form: vectors a CTA takes per step; whole steps of a row; vectors of its ragged last step
     int policy;           // bit 0: pass A loads ask L2 to keep their lines; bit 1: pass B loads let them go
 };
 
@@ -64,7 +66,7 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass(const WArgs a) {
     const int cs = CL ? a.cs : 1;
     const int rank = CL ? static_cast<int>(blockIdx.x % cs) : 0;
     const int64_t first_slot = CL ? blockIdx.x / cs : blockIdx.x, slot_step = CL ? gridDim.x / cs : gridDim.x;
-    const int64_t per_group = a.slots / a.groups;
+    const int64_t per_group = a.per_group;
     const int64_t per = CL ? (a.nvec + cs - 1) / cs : a.nvec, first = rank * per;        // this CTA's slice of every row
     const int64_t seg = max(int64_t{0}, min(per, a.nvec - first));
     const int64_t cache_vecs = min(a.cache_vecs, seg);
@@ -134,6 +136,7 @@ __device__ __forceinline__ void cp_async16(uint4* dst, const uint4* src, uint64_
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait(int pending) {     // returns once at most `pending` of this thread's groups are in flight
+    if (pending == 1) { asm volatile("cp.async.wait_group 1;" ::: "memory"); return; }      // two stages: the common case
     switch (pending) {
         case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
         case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
@@ -169,13 +172,13 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
     const int cs = CL ? a.cs : 1;
     const int rank = CL ? static_cast<int>(blockIdx.x % cs) : 0;
     const int nvec = static_cast<int>(a.nvec);
-    const int step = (blockDim.x >> 5) * CH;                             // vectors the CTA takes per step
+    const int step = a.step;                                             // vectors the CTA takes per step: warps x CH
     const int gstep = cs * step;                                         // distance in the row between two steps of this CTA
-    const int nfull = nvec / step;                                       // whole steps of the row
-    const int rag = nvec - nfull * step;                                 // vectors of the row's ragged last step (0: there is none)
+    const int nfull = a.nfull;                                           // whole steps of the row
+    const int rag = a.rag;                                               // vectors of the row's ragged last step (0: there is none)
     // the steps of CTA k: k, k + cs, ...; its last one is the ragged step iff that falls to it
-    auto steps_of = [&](int k) { const int n = nfull + (rag ? 1 : 0); return n > k ? (n - k - 1) / cs + 1 : 0; };
-    auto ragged_of = [&](int k) { return rag != 0 && nfull % cs == k; };
+    auto steps_of = [&](int k) { const int n = nfull + (rag ? 1 : 0); return CL ? (n > k ? (n - k - 1) / cs + 1 : 0) : n; };
+    auto ragged_of = [&](int k) { return rag != 0 && (!CL || nfull % cs == k); };
     auto count_of = [&](int k) { return static_cast<float>(((steps_of(k) - (ragged_of(k) ? 1 : 0)) * step + (ragged_of(k) ? rag : 0)) * NE); };
     const int nsteps = steps_of(rank);                                   // this CTA's steps, numbered 0 .. nsteps-1 from here on
     const bool has_rag = ragged_of(rank);
@@ -183,10 +186,11 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
     const int toff = (t >> 5) * CH + (t & 31);                           // this thread's first vector within a step
     uint4* const myring = reinterpret_cast<uint4*>(dyn_smem) + toff;     // slot k of the ring: myring + k * step (+ u * 32)
     uint4* const ring_end = myring + S * step;
-    const int64_t per_group = a.slots / a.groups;
+    const int64_t per_group = a.per_group;
     const uint4 fill = fill_vec<DT>(OP);
     const uint4 zero = make_uint4(0, 0, 0, 0);
-    const int slot_of_step0 = nsteps > 0 ? (nsteps - 1) % S : 0;         // pass A visits step s as its (nsteps-1-s)-th: slot = that mod S
+    // pass A visits step s as its (nsteps-1-s)-th: slot = that mod S (two stages, the common case, without a division)
+    const int slot_of_step0 = nsteps > 0 ? (S == 2 ? ((nsteps - 1) & 1) : (nsteps - 1) % S) : 0;
     if constexpr (CL) cg::this_cluster().sync();                         // every CTA of the cluster is resident before any remote write
     const int64_t first_slot = CL ? blockIdx.x / cs : blockIdx.x, slot_step = CL ? gridDim.x / cs : gridDim.x;
     int it = -1;
@@ -418,7 +422,10 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
     k.y = static_cast<uint4*>(a.y); k.mean = a.mean; k.rstd = a.rstd; k.rows = a.rows; k.len = a.len;
     k.nvec = a.cols * elem_size(a.dt) / 16;
     k.n = static_cast<float>(a.cols); k.eps = a.eps;
-    k.cs = cs; k.groups = groups; k.slots = slots; k.policy = p.vpt;
+    k.cs = cs; k.groups = groups; k.slots = slots; k.policy = p.vpt; k.per_group = slots / groups;
+    k.step = (p.threads / 32) * p.unroll * 32;
+    k.nfull = static_cast<int>(k.nvec / k.step);
+    k.rag = static_cast<int>(k.nvec - static_cast<int64_t>(k.nfull) * k.step);
     k.cache_vecs = std::min<int64_t>((k.nvec + cs - 1) / cs, p.chunk / 16);
     k.stages = p.stages;
     const size_t smem = ring ? static_cast<size_t>(p.stages) * p.threads * p.unroll * 16 : static_cast<size_t>(k.cache_vecs) * 16;
