@@ -202,7 +202,8 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
     // Long rows, read off the tuner's winners on the sweep and the 2 GiB softmax: two streamed passes.  The ring form
     // (each thread's loads run ahead of its arithmetic in a private shared-memory ring) for softmax from 64-128 KiB rows
     // on, with a pair of CTAs per row from 256 KiB (2 GiB masked softmax: 325-329 us against 360-460 us for every plan
-    // that keeps the row on chip); the direct form for fp32 LayerNorm from 32 KiB and bf16 RMSNorm of 32-64 KiB.
+    // that keeps the row on chip), and for LayerNorm and bf16 RMSNorm rows from 16-64 KiB on with the 64-register build
+    // (fp32 LayerNorm [4096, 16384]: 88 us against 100 us for the direct form); the direct form where it still wins.
     {
         Plan s;
         s.variant = V_TWOPASS; s.chunk = 0; s.rpg = 2; s.lanes = 1; s.vpt = 3; s.stages = 0; s.unroll = 4; s.cluster = 1; s.persist = 0;
@@ -215,17 +216,19 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         const bool mid = nvec >= 1024 && nvec <= 2048;
         if (a.op == OP_SOFTMAX) {
             if (nvec >= 16384) { ring(256, 4, 2, true); take = true; }
-            else if (nvec >= 8192) { ring(384, f32 ? 4 : 2, 1, true); take = true; }
+            else if (nvec >= 8192) { if (f32) ring(384, 4, 1, true); else ring(512, 2, 1, false); take = true; }
             else if (nvec >= 4096 && !f32) { ring(256, 2, 1, false); take = true; }
             else if (nvec == 2048 && !f32) { ring(128, 2, 1, false); take = true; }
+            else if (nvec == 1536 && !f32) { ring(128, 3, 1, false); take = true; }
         } else if (a.op == OP_LAYERNORM) {
-            if (f32 && nvec >= 2048) { direct(nvec < 4096 ? 256 : 512, nvec >= 16384 ? 2 : 1); if (nvec == 8192) s.rpg = 1; take = true; }
-            else if (!f32 && nvec >= 8192) { ring(512, nvec >= 16384 ? 3 : 2, 1, false); take = true; }
-            else if (!f32 && nvec >= 4096) { ring(256, 2, 1, false); take = true; }
-            else if (mid) { ring(128, 2, 1, false); take = true; }
+            if (f32 && nvec >= 16384) { direct(512, 2); take = true; }
+            else if (nvec >= 8192) { ring(512, (!f32 && nvec >= 16384) ? 3 : 2, 1, false); take = true; }
+            else if (nvec > 2048) { ring(256, 2, 1, false); take = true; }
+            else if (mid) { ring(nvec == 1280 ? 160 : 128, 2, 1, false); take = true; }      // 1280 vectors: two steps of five warps
         } else if (!f32 && nvec == 1024) { ring(128, 2, 1, false); take = true;
         } else {
             if (f32 && nvec >= 8192 && nvec < 16384) { ring(512, 3, 1, false); take = true; }
+            else if (f32 && nvec == 3072) { ring(384, 2, 1, true); take = true; }
             else if (f32 && nvec >= 4096 && nvec < 8192) { ring(256, 4, 1, true); take = true; }
             else if (!f32 && nvec >= 8192) { ring(512, 3, 1, false); take = true; }
             else if (!f32 && nvec >= 4096) { ring(256, 4, 1, false); take = true; }
@@ -266,8 +269,17 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
             if (supports_cta(q, a, d)) return q;
         }
         if (nvec == 512 && ln && a.dt == DT_F32) {
-            q.variant = V_CTA; q.cluster = 1; q.persist = 0; q.vpt = 4; q.threads = 128;
+            q.variant = V_CTA; q.cluster = 1; q.persist = 0; q.vpt = 8; q.threads = 64;
             if (supports_cta(q, a, d)) return q;
+        }
+        if (nvec <= 64 && a.op == OP_RMSNORM && a.dt == DT_BF16) {
+            // bf16 RMSNorm rows up to 1 KiB: small non-persistent pipeline CTAs (3-5 % ahead of the lane-group form)
+            q.variant = V_PIPE; q.threads = 256; q.stages = 2; q.chunk = 3072; q.persist = 0;
+            q.lanes = nvec <= 8 ? 8 : nvec <= 16 ? 16 : 32;
+            q.vpt = nvec <= 32 ? 1 : 2;
+            q.rpg = (nvec <= 8 || (nvec > 16 && nvec <= 32)) ? 2 : 1;
+            if (supports_pipe(q, a, d)) return q;
+            q = Plan();
         }
         if (nvec <= 256 && !(ln && a.dt == DT_BF16)) {
             // rows up to 4 KiB: a lane group per row, every load issued at once, as many small CTAs as there are row blocks
@@ -276,7 +288,7 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
             else if (nvec <= 16) { q.lanes = 8; q.vpt = 2; q.rpg = ln ? 2 : 1; }
             else if (nvec <= 32) { q.lanes = 16; q.vpt = 2; q.rpg = ln ? 2 : 1; }
             else if (nvec <= 64) { q.lanes = 32; q.vpt = 2; q.rpg = (a.dt == DT_F32 && a.op != OP_SOFTMAX) ? 2 : 1; }
-            else if (nvec <= 128) { q.lanes = 32; q.vpt = 4; q.rpg = (a.op == OP_RMSNORM && a.dt == DT_BF16) ? 2 : 1; }
+            else if (nvec <= 128) { q.lanes = 32; q.vpt = 4; q.rpg = ((a.op == OP_RMSNORM && a.dt == DT_BF16) || (ln && a.dt == DT_F32)) ? 2 : 1; }
             else { q.lanes = 32; q.vpt = 8; }
             if (supports_warp(q, a, d)) return q;
         } else if (!ln && nvec <= (a.dt == DT_BF16 ? 1024 : (a.op == OP_SOFTMAX ? 4096 : 3072))) {
@@ -316,8 +328,8 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         int64_t target = 16384;
         if (nvec <= 256) {                       // rows up to 4 KiB (what reaches here is LayerNorm bf16): the tuner's winners use
             p.persist = 2; target = 4096;        // small stages and two CTAs per SM
-            if (nvec <= 16) p.rpg = 2;
-            if (nvec == 64) { p.threads = 256; target = 6144; }
+            if (nvec <= 8) p.rpg = 2;
+            if (nvec == 64) { p.threads = 256; p.rpg = 2; p.persist = 0; target = 6144; }
             if (nvec == 128) { p.threads = 128; p.rpg = 2; p.persist = 0; }
             if (nvec == 256) { p.threads = 256; p.persist = 0; }
         }

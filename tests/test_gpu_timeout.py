@@ -47,7 +47,8 @@ def test_probe_rejects_bad_arguments():
 
 
 def test_tuner_drops_candidates_whose_wait_gave_up():
-    op, rows, cols, dt = "rmsnorm", 4000, 4096, inputs.F32
+    # an L2-resident shape: the tuner has no copy ceiling to finish early at, so the free run times its whole list
+    op, rows, cols, dt = "rmsnorm", 512, 4096, inputs.F32
     tf.tf_clear_cache()
     heur = tf.tf_query_choice(op, rows, cols, dt)
     free = tf.tf_tune(op, rows, cols, dt)
