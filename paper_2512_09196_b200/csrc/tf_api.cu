@@ -211,28 +211,33 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         auto direct = [&](int threads, int cluster) { s.threads = threads; s.stages = 0; s.cluster = cluster; s.rpg = 2; };
         bool take = false;
         const bool f32 = a.dt == DT_F32;
-        // rows of 16-32 KiB: the ring form with CTAs of 128 threads holds the whole row in its two stages, so nothing is
-        // read twice, and a dozen such CTAs fit an SM (RMSNorm bf16 [16384, 8192]: 81 us against 86 us for the pipeline)
-        const bool mid = nvec >= 1024 && nvec <= 2048;
-        if (a.op == OP_SOFTMAX) {
+        // Rows of 4-64 KiB: the ring form with the whole row in the ring (every copy of the row requested at once, the
+        // second pass out of shared memory, straight-line code): CTAs of an eighth of the row's vectors, up to 256
+        // threads, so a row takes two to four steps.  LayerNorm bf16 [16384, 8192]: 80 us against 88 us for the general
+        // ring form and 89 us for the pipeline; [8192, 4096]: 22.5 us against 24.0 us.  The lighter ops take 8 KiB rows
+        // in one step.
+        auto fit = [&](bool one_step) {
+            const int t = std::min(256, std::max(32, round_up(static_cast<int>((nvec + (one_step ? 3 : 7)) / (one_step ? 4 : 8)), 32)));
+            const int steps = static_cast<int>((nvec + 4 * t - 1) / (4 * t));
+            ring(t, std::max(2, steps), 1, false);
+        };
+        const bool ln_bf16 = a.op == OP_LAYERNORM && !f32;
+        const bool fits = nvec <= 4096 &&
+                          ((ln_bf16 && nvec >= 256) || (a.op == OP_LAYERNORM && f32 && nvec >= 512) ||
+                           (a.op == OP_RMSNORM && !f32 && nvec >= 512) || (a.op == OP_SOFTMAX && !f32 && nvec >= 512 && nvec <= 2048));
+        if (fits) { fit(nvec == 512 && !ln_bf16); take = true; }
+        else if (a.op == OP_SOFTMAX) {
             if (nvec >= 16384) { ring(256, 4, 2, true); take = true; }
             else if (nvec >= 8192) { if (f32) ring(384, 4, 1, true); else ring(512, 2, 1, false); take = true; }
             else if (nvec >= 4096 && !f32) { ring(256, 2, 1, false); take = true; }
-            else if (nvec == 2048 && !f32) { ring(128, 2, 1, false); take = true; }
-            else if (nvec == 1536 && !f32) { ring(128, 3, 1, false); take = true; }
         } else if (a.op == OP_LAYERNORM) {
             if (f32 && nvec >= 16384) { direct(512, 2); take = true; }
             else if (nvec >= 8192) { ring(512, (!f32 && nvec >= 16384) ? 3 : 2, 1, false); take = true; }
-            else if (nvec > 2048) { ring(256, 2, 1, false); take = true; }
-            else if (mid) { ring(nvec == 1280 ? 160 : 128, 2, 1, false); take = true; }      // 1280 vectors: two steps of five warps
-        } else if (!f32 && nvec == 1024) { ring(128, 2, 1, false); take = true;
         } else {
             if (f32 && nvec >= 8192 && nvec < 16384) { ring(512, 3, 1, false); take = true; }
             else if (f32 && nvec == 3072) { ring(384, 2, 1, true); take = true; }
             else if (f32 && nvec >= 4096 && nvec < 8192) { ring(256, 4, 1, true); take = true; }
             else if (!f32 && nvec >= 8192) { ring(512, 3, 1, false); take = true; }
-            else if (!f32 && nvec >= 4096) { ring(256, 4, 1, false); take = true; }
-            else if (!f32 && nvec >= 2048) { direct(256, 1); take = true; }
         }
         if (take && a.rows >= 2LL * d.sms && supports_twopass(s, a, d)) return s;
     }
@@ -495,6 +500,17 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
                     p.rpg = 1; add(p);
                     if (th > 256) { p.rpg = 2; add(p); }
                 }
+    // the ring form where the whole row fits the ring (straight-line build, one row per CTA): every CTA size whose
+    // steps the row fills to at least three quarters
+    if (nvec >= 128 && nvec <= 8192)
+        for (int th : {32, 64, 96, 128, 160, 192, 256, 320, 384, 512}) {
+            const int64_t step = static_cast<int64_t>(th) * 4;
+            const int64_t steps = (nvec + step - 1) / step;
+            if (steps > 4 || nvec * 4 < steps * step * 3) continue;
+            Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = 0; p.lanes = 1; p.vpt = 3; p.chunk = 0; p.cluster = 1;
+            p.stages = static_cast<int>(std::max<int64_t>(2, steps)); p.unroll = 4; p.rpg = 1;
+            add(p);
+        }
     // persistent cluster ring for long rows
     if (nvec >= 2048)
         for (int cl : {1, 2, 4, 8})

@@ -333,7 +333,100 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
     }
 }
 
+// ---- the ring form for rows that fit the ring ---------------------------------------------------------------------
+// When a row takes no more steps than the ring has stages (rows of 8-64 KiB with CTAs of 64-512 threads), every copy
+// of the row is requested in the prologue, nothing is refilled and the second pass finds the whole row in shared
+// memory: x crosses L2 once.  One row per CTA, NS steps known at compile time, so both passes are straight-line code;
+// FULL: the row fills the NS steps exactly and no access carries a predicate.
+template <int OP, int DT, int U, int NS, bool FULL>
+__global__ void __launch_bounds__(1024, 1) k_twopass_fit(const WArgs a) {
+    constexpr int NE = Elem<DT>::NE, CH = U * 32;
+    __shared__ float red_buf[2 * 32];
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    pdl_wait();
+    pdl_trigger();
+    const uint64_t once = (a.policy & 2) ? policy_evict_first() : policy_evict_normal();     // x is read once
+    const int t = threadIdx.x;
+    const int nvec = static_cast<int>(a.nvec), step = a.step;
+    const int toff = (t >> 5) * CH + (t & 31);                           // this thread's first vector within a step
+    const int64_t row = blockIdx.x;
+    const uint4* const xr = a.x + row * nvec + toff;
+    uint4* const yr = a.y + row * nvec + toff;
+    uint4* const myring = reinterpret_cast<uint4*>(dyn_smem) + toff;
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (FULL || s * step + toff + u * 32 < nvec) cp_async16(myring + s * step + u * 32, xr + s * step + u * 32, once);
+        cp_async_commit();
+    }
+    Running<OP, DT, U> run;
+    const uint4 fill = fill_vec<DT>(OP);
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+        cp_async_wait(NS - 1 - s);
+        const int first = s * step + toff;
+        uint4 raw[U];
+        if (FULL || first + (U - 1) * 32 < nvec) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) raw[u] = myring[s * step + u * 32];
+            const bool all[U] = {};
+            run.template update<false>(raw, all, U * NE, s * U);
+        } else if (first < nvec) {
+            bool ok[U];
+            int count = 0;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                ok[u] = first + u * 32 < nvec;
+                raw[u] = ok[u] ? myring[s * step + u * 32] : fill;
+                count += ok[u] ? NE : 0;
+            }
+            run.template update<true>(raw, ok, count, s * U);
+        }
+    }
+    const Part part = merge_running<OP, DT, U>(run, a.n, red_buf);
+    const RowScale sc = scale_of_row<OP>(part, a.n, a.eps);
+    if (t == 0) {
+        if (OP == OP_LAYERNORM && a.mean) a.mean[row] = sc.a;
+        if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = sc.b;
+    }
+    const F2 ta2 = f2(sc.a), tb2 = f2(sc.b);
+    const uint4* const gp = a.p0 + toff;
+    const uint4* const bp = a.p1 + toff;
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int o = s * step + u * 32;
+            if (FULL || o + toff < nvec) st_stream(yr + o, apply_vec<OP, DT>(myring[o], gp + o, bp + o, ta2, tb2));
+        }
+    }
+}
+
 using TwoFn = void (*)(const WArgs);
+
+template <int NS, bool FULL>
+TwoFn fit_fn_c(int op, int dt) {
+    switch (op * 2 + dt) {
+        case 0: return k_twopass_fit<OP_SOFTMAX, DT_F32, 4, NS, FULL>;
+        case 1: return k_twopass_fit<OP_SOFTMAX, DT_BF16, 4, NS, FULL>;
+        case 2: return k_twopass_fit<OP_LAYERNORM, DT_F32, 4, NS, FULL>;
+        case 3: return k_twopass_fit<OP_LAYERNORM, DT_BF16, 4, NS, FULL>;
+        case 4: return k_twopass_fit<OP_RMSNORM, DT_F32, 4, NS, FULL>;
+        case 5: return k_twopass_fit<OP_RMSNORM, DT_BF16, 4, NS, FULL>;
+    }
+    return nullptr;
+}
+// steps: what the row takes (1 .. 4)
+TwoFn fit_fn(int op, int dt, int steps, bool full) {
+    switch (steps) {
+        case 1: return full ? fit_fn_c<1, true>(op, dt) : fit_fn_c<1, false>(op, dt);
+        case 2: return full ? fit_fn_c<2, true>(op, dt) : fit_fn_c<2, false>(op, dt);
+        case 3: return full ? fit_fn_c<3, true>(op, dt) : fit_fn_c<3, false>(op, dt);
+        case 4: return full ? fit_fn_c<4, true>(op, dt) : fit_fn_c<4, false>(op, dt);
+    }
+    return nullptr;
+}
 
 template <int MAXT, int MINB, bool CL, bool CACHE>
 TwoFn two_fn_c(int op, int dt, bool len) {
@@ -413,6 +506,16 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
     TwoFn fn = ring ? ring_fn(a.op, a.dt, p.unroll, p.threads, p.rpg == 2, cs > 1) : two_fn(a.op, a.dt, p.threads, p.rpg == 2, cs > 1, a.len != nullptr, p.chunk > 0);
     if (!fn) return cudaErrorInvalidValue;
     const int groups = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(p.lanes, a.rows)));
+    // a row that takes no more steps than the ring has stages: the straight-line build, one row per CTA
+    int fit_steps = 0;
+    if (ring && cs == 1 && groups == 1 && p.persist == 0 && p.unroll == 4 && p.rpg == 1 && a.rows <= 0x7FFFFFFF) {
+        const int64_t step = static_cast<int64_t>(p.threads / 32) * p.unroll * 32;
+        const int64_t steps = (a.cols * elem_size(a.dt) / 16 + step - 1) / step;
+        if (steps <= std::min(p.stages, 4)) {
+            fit_steps = static_cast<int>(steps);
+            fn = fit_fn(a.op, a.dt, fit_steps, steps * step == a.cols * elem_size(a.dt) / 16);
+        }
+    }
     const int64_t slots = (a.rows + groups - 1) / groups * groups;
     int64_t grid = slots;                                          // in rows (clusters)
     if (p.persist > 0) grid = std::min<int64_t>(grid, std::max<int64_t>(1, static_cast<int64_t>(p.persist) * d.sms / cs));
@@ -428,7 +531,7 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
     k.rag = static_cast<int>(k.nvec - static_cast<int64_t>(k.nfull) * k.step);
     k.cache_vecs = std::min<int64_t>((k.nvec + cs - 1) / cs, p.chunk / 16);
     k.stages = p.stages;
-    const size_t smem = ring ? static_cast<size_t>(p.stages) * p.threads * p.unroll * 16 : static_cast<size_t>(k.cache_vecs) * 16;
+    const size_t smem = ring ? static_cast<size_t>(fit_steps ? fit_steps : p.stages) * p.threads * p.unroll * 16 : static_cast<size_t>(k.cache_vecs) * 16;
     if (smem > 0) {
         cudaError_t e = ensure_max_smem(reinterpret_cast<const void*>(fn), d);
         if (e != cudaSuccess) return e;
