@@ -227,7 +227,8 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
                            (a.op == OP_RMSNORM && !f32 && nvec >= 512) || (a.op == OP_SOFTMAX && !f32 && nvec >= 512 && nvec <= 2048));
         if (fits) { fit(nvec == 512 && !ln_bf16); take = true; }
         else if (a.op == OP_SOFTMAX) {
-            if (nvec >= 16384) { ring(256, 4, 2, true); take = true; }
+            if (nvec == 16384 && f32) { ring(128, 4, 8, false); take = true; }          // the row in the rings of a cluster of 8 (87 us against 90 us)
+            else if (nvec >= 16384) { ring(256, 4, 2, true); take = true; }
             else if (nvec >= 8192) { if (f32) ring(384, 4, 1, true); else ring(512, 2, 1, false); take = true; }
             else if (nvec >= 4096 && !f32) { ring(256, 2, 1, false); take = true; }
         } else if (a.op == OP_LAYERNORM) {
@@ -511,6 +512,17 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
             p.stages = static_cast<int>(std::max<int64_t>(2, steps)); p.unroll = 4; p.rpg = 1;
             add(p);
         }
+    // ... and with the CTAs of a cluster sharing the row (rows of 64 KiB to 1 MiB)
+    if (nvec >= 4096 && nvec <= 65536)
+        for (int cl : {2, 4, 8})
+            for (int th : {128, 256, 384, 512}) {
+                const int64_t step = static_cast<int64_t>(th) * 4 * cl;
+                const int64_t steps = (nvec + step - 1) / step;
+                if (steps > 4 || nvec * 4 < steps * step * 3 || cl > d.max_cluster) continue;
+                Plan p; p.variant = V_TWOPASS; p.threads = th; p.persist = 0; p.lanes = 1; p.vpt = 3; p.chunk = 0; p.cluster = cl;
+                p.stages = static_cast<int>(std::max<int64_t>(2, steps)); p.unroll = 4; p.rpg = 1;
+                add(p);
+            }
     // persistent cluster ring for long rows
     if (nvec >= 2048)
         for (int cl : {1, 2, 4, 8})

@@ -15,6 +15,9 @@
 // barrier.  With rows of 256 KiB and more this keeps what is in flight between the passes within L2 (one CTA per row
 // on every SM is more than L2 holds of such rows, and the second pass then goes back to HBM), and with few rows it
 // gives every SM a share.
+// Three kernels implement the plan: k_twopass (loads straight into registers), k_twopass_ring (plan field `stages` >= 2:
+// asynchronous copies through per-thread rings in shared memory) and k_twopass_fit, which the launcher picks by itself
+// when the ring of the plan holds the whole row (rows of 4-64 KiB per CTA): the second pass then never leaves the SM.
 #include <cooperative_groups.h>
 
 #include <algorithm>
@@ -334,30 +337,42 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
 }
 
 // ---- the ring form for rows that fit the ring ---------------------------------------------------------------------
-// When a row takes no more steps than the ring has stages (rows of 8-64 KiB with CTAs of 64-512 threads), every copy
+// When a row takes no more steps than the ring has stages (rows of 4-64 KiB with CTAs of 32-512 threads), every copy
 // of the row is requested in the prologue, nothing is refilled and the second pass finds the whole row in shared
 // memory: x crosses L2 once.  One row per CTA, NS steps known at compile time, so both passes are straight-line code;
-// FULL: the row fills the NS steps exactly and no access carries a predicate.
-template <int OP, int DT, int U, int NS, bool FULL>
+// FULL: the row fills the steps exactly and no access carries a predicate.
+// CL: the `cs` CTAs of a cluster share a row of up to cs x 64 KiB, CTA `rank` taking the steps rank, rank + cs, ...;
+// their partials meet once, through distributed shared memory.  A CTA writes into its peers only after a cluster
+// barrier that every CTA arrives at when it starts (so the peers are running), and reads what it received after a second one.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+template <int OP, int DT, int U, int NS, bool FULL, bool CL>
 __global__ void __launch_bounds__(1024, 1) k_twopass_fit(const WArgs a) {
     constexpr int NE = Elem<DT>::NE, CH = U * 32;
     __shared__ float red_buf[2 * 32];
+    __shared__ float xch[CL ? kMaxCluster : 1][2];                       // partials of the CTAs of the cluster
     extern __shared__ __align__(16) unsigned char dyn_smem[];
+    if constexpr (CL) cluster_arrive();
     pdl_wait();
     pdl_trigger();
     const uint64_t once = (a.policy & 2) ? policy_evict_first() : policy_evict_normal();     // x is read once
     const int t = threadIdx.x;
     const int nvec = static_cast<int>(a.nvec), step = a.step;
+    const int cs = CL ? a.cs : 1;
+    const int rank = CL ? static_cast<int>(blockIdx.x % cs) : 0;
+    const int gstep = cs * step;                                         // distance in the row between two steps of this CTA
     const int toff = (t >> 5) * CH + (t & 31);                           // this thread's first vector within a step
-    const int64_t row = blockIdx.x;
-    const uint4* const xr = a.x + row * nvec + toff;
-    uint4* const yr = a.y + row * nvec + toff;
+    const int mine = rank * step + toff;                                 // ... within the row
+    const int64_t row = CL ? blockIdx.x / cs : blockIdx.x;
+    const uint4* const xr = a.x + row * nvec + mine;
+    uint4* const yr = a.y + row * nvec + mine;
     uint4* const myring = reinterpret_cast<uint4*>(dyn_smem) + toff;
 #pragma unroll
     for (int s = 0; s < NS; ++s) {
 #pragma unroll
         for (int u = 0; u < U; ++u)
-            if (FULL || s * step + toff + u * 32 < nvec) cp_async16(myring + s * step + u * 32, xr + s * step + u * 32, once);
+            if (FULL || s * gstep + mine + u * 32 < nvec) cp_async16(myring + s * step + u * 32, xr + s * gstep + u * 32, once);
         cp_async_commit();
     }
     Running<OP, DT, U> run;
@@ -365,7 +380,7 @@ __global__ void __launch_bounds__(1024, 1) k_twopass_fit(const WArgs a) {
 #pragma unroll
     for (int s = 0; s < NS; ++s) {
         cp_async_wait(NS - 1 - s);
-        const int first = s * step + toff;
+        const int first = s * gstep + mine;
         uint4 raw[U];
         if (FULL || first + (U - 1) * 32 < nvec) {
 #pragma unroll
@@ -384,46 +399,85 @@ __global__ void __launch_bounds__(1024, 1) k_twopass_fit(const WArgs a) {
             run.template update<true>(raw, ok, count, s * U);
         }
     }
-    const Part part = merge_running<OP, DT, U>(run, a.n, red_buf);
+    // elements CTA k holds: its steps k, k + cs, ... clipped to the row
+    auto count_of = [&](int k) {
+        int c = 0;
+#pragma unroll
+        for (int s = 0; s < NS; ++s) c += max(0, min(step, nvec - (s * cs + k) * step));
+        return static_cast<float>(c * NE);
+    };
+    Part part = merge_running<OP, DT, U>(run, CL ? fmaxf(count_of(rank), 1.f) : a.n, red_buf);
+    if constexpr (CL) {
+        cg::cluster_group cl = cg::this_cluster();
+        cluster_wait();                                                   // every CTA of the cluster has started
+        if (t < cs) {                                                     // my partial into every CTA of the cluster
+            float* dstp = cl.map_shared_rank(&xch[rank][0], t);
+            dstp[0] = part.a; dstp[1] = part.b;
+        }
+        cluster_arrive();
+        cluster_wait();                                                   // release our writes, acquire the peers'
+        // the row's partial from the CTAs', in rank order (the same bits in every CTA)
+        if constexpr (OP == OP_SOFTMAX) {
+            float O = -kNegInf, Ssum = 0.f;
+            for (int k = 0; k < cs; ++k) O = fminf(O, xch[k][0]);
+            for (int k = 0; k < cs; ++k) Ssum = fmaf(xch[k][1], softmax_rescale(O, xch[k][0]), Ssum);
+            part = Part{O, Ssum};
+        } else if constexpr (OP == OP_LAYERNORM) {
+            float sum = 0.f, m2 = 0.f;
+            for (int k = 0; k < cs; ++k) sum = fmaf(count_of(k), xch[k][0], sum);
+            const float mean = fast_div(sum, a.n);
+            for (int k = 0; k < cs; ++k) { const float d = xch[k][0] - mean; m2 += fmaf(count_of(k) * d, d, xch[k][1]); }
+            part = Part{mean, m2};
+        } else {
+            float q = 0.f;
+            for (int k = 0; k < cs; ++k) q += xch[k][0];
+            part = Part{q, 0.f};
+        }
+    }
     const RowScale sc = scale_of_row<OP>(part, a.n, a.eps);
-    if (t == 0) {
+    if (t == 0 && rank == 0) {
         if (OP == OP_LAYERNORM && a.mean) a.mean[row] = sc.a;
         if (OP != OP_SOFTMAX && a.rstd) a.rstd[row] = sc.b;
     }
     const F2 ta2 = f2(sc.a), tb2 = f2(sc.b);
-    const uint4* const gp = a.p0 + toff;
-    const uint4* const bp = a.p1 + toff;
+    const uint4* const gp = a.p0 + mine;
+    const uint4* const bp = a.p1 + mine;
 #pragma unroll
     for (int s = 0; s < NS; ++s) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int o = s * step + u * 32;
-            if (FULL || o + toff < nvec) st_stream(yr + o, apply_vec<OP, DT>(myring[o], gp + o, bp + o, ta2, tb2));
+            const int o = s * gstep + u * 32;
+            if (FULL || o + mine < nvec) st_stream(yr + o, apply_vec<OP, DT>(myring[s * step + u * 32], gp + o, bp + o, ta2, tb2));
         }
     }
 }
 
 using TwoFn = void (*)(const WArgs);
 
-template <int NS, bool FULL>
+template <int NS, bool FULL, bool CL>
 TwoFn fit_fn_c(int op, int dt) {
     switch (op * 2 + dt) {
-        case 0: return k_twopass_fit<OP_SOFTMAX, DT_F32, 4, NS, FULL>;
-        case 1: return k_twopass_fit<OP_SOFTMAX, DT_BF16, 4, NS, FULL>;
-        case 2: return k_twopass_fit<OP_LAYERNORM, DT_F32, 4, NS, FULL>;
-        case 3: return k_twopass_fit<OP_LAYERNORM, DT_BF16, 4, NS, FULL>;
-        case 4: return k_twopass_fit<OP_RMSNORM, DT_F32, 4, NS, FULL>;
-        case 5: return k_twopass_fit<OP_RMSNORM, DT_BF16, 4, NS, FULL>;
+        case 0: return k_twopass_fit<OP_SOFTMAX, DT_F32, 4, NS, FULL, CL>;
+        case 1: return k_twopass_fit<OP_SOFTMAX, DT_BF16, 4, NS, FULL, CL>;
+        case 2: return k_twopass_fit<OP_LAYERNORM, DT_F32, 4, NS, FULL, CL>;
+        case 3: return k_twopass_fit<OP_LAYERNORM, DT_BF16, 4, NS, FULL, CL>;
+        case 4: return k_twopass_fit<OP_RMSNORM, DT_F32, 4, NS, FULL, CL>;
+        case 5: return k_twopass_fit<OP_RMSNORM, DT_BF16, 4, NS, FULL, CL>;
     }
     return nullptr;
 }
-// steps: what the row takes (1 .. 4)
-TwoFn fit_fn(int op, int dt, int steps, bool full) {
+template <int NS>
+TwoFn fit_fn_b(int op, int dt, bool full, bool cl) {
+    if (cl) return full ? fit_fn_c<NS, true, true>(op, dt) : fit_fn_c<NS, false, true>(op, dt);
+    return full ? fit_fn_c<NS, true, false>(op, dt) : fit_fn_c<NS, false, false>(op, dt);
+}
+// steps: what a CTA takes of the row (1 .. 4)
+TwoFn fit_fn(int op, int dt, int steps, bool full, bool cl) {
     switch (steps) {
-        case 1: return full ? fit_fn_c<1, true>(op, dt) : fit_fn_c<1, false>(op, dt);
-        case 2: return full ? fit_fn_c<2, true>(op, dt) : fit_fn_c<2, false>(op, dt);
-        case 3: return full ? fit_fn_c<3, true>(op, dt) : fit_fn_c<3, false>(op, dt);
-        case 4: return full ? fit_fn_c<4, true>(op, dt) : fit_fn_c<4, false>(op, dt);
+        case 1: return fit_fn_b<1>(op, dt, full, cl);
+        case 2: return fit_fn_b<2>(op, dt, full, cl);
+        case 3: return fit_fn_b<3>(op, dt, full, cl);
+        case 4: return fit_fn_b<4>(op, dt, full, cl);
     }
     return nullptr;
 }
@@ -506,14 +560,15 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
     TwoFn fn = ring ? ring_fn(a.op, a.dt, p.unroll, p.threads, p.rpg == 2, cs > 1) : two_fn(a.op, a.dt, p.threads, p.rpg == 2, cs > 1, a.len != nullptr, p.chunk > 0);
     if (!fn) return cudaErrorInvalidValue;
     const int groups = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(p.lanes, a.rows)));
-    // a row that takes no more steps than the ring has stages: the straight-line build, one row per CTA
+    // a row that takes no more steps (per CTA of its cluster) than the ring has stages: the straight-line build
     int fit_steps = 0;
-    if (ring && cs == 1 && groups == 1 && p.persist == 0 && p.unroll == 4 && p.rpg == 1 && a.rows <= 0x7FFFFFFF) {
+    if (ring && groups == 1 && p.persist == 0 && p.unroll == 4 && p.rpg == 1 && a.rows * cs <= 0x7FFFFFFF) {
+        const int64_t nvec = a.cols * elem_size(a.dt) / 16;
         const int64_t step = static_cast<int64_t>(p.threads / 32) * p.unroll * 32;
-        const int64_t steps = (a.cols * elem_size(a.dt) / 16 + step - 1) / step;
+        const int64_t steps = ((nvec + step - 1) / step + cs - 1) / cs;
         if (steps <= std::min(p.stages, 4)) {
             fit_steps = static_cast<int>(steps);
-            fn = fit_fn(a.op, a.dt, fit_steps, steps * step == a.cols * elem_size(a.dt) / 16);
+            fn = fit_fn(a.op, a.dt, fit_steps, steps * step * cs == nvec, cs > 1);
         }
     }
     const int64_t slots = (a.rows + groups - 1) / groups * groups;

@@ -283,13 +283,27 @@ def test_forced_twopass_variants(op, dt):
             tf.tf_force_plan(op, plan)
             fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec + cluster))
             assert not fails, (plan, nvec, rows, fails)
+    # rows that fit the ring (straight-line build, one row per CTA or per cluster): a single vector, steps without work,
+    # rows that fill the steps exactly and by one vector less, a last CTA that falls short, one row; one vector more than
+    # fits goes to the general ring form
+    for cluster, threads, stages in ((1, 64, 2), (1, 96, 3), (1, 256, 4), (1, 128, 2), (2, 128, 2), (4, 64, 4), (8, 32, 3), (2, 512, 2)):
+        st, cap = threads * 4, threads * 4 * cluster * stages
+        for nvec, rows in ((1, 3), (st - 1, 5), (st, 150), (st * cluster, 9), (cap, 9), (cap - 1, 300), (cap - st - 3, 9),
+                           (cap - st * cluster + 5, 1), (cap + 1, 5)):
+            plan = f"twopass:threads={threads},persist=0,regcap=0,cluster={cluster},stages={stages},u=4"
+            tf.tf_force_plan(op, plan)
+            fails = parity.parity(wl(op, dt, rows, nvec * ne, seed=nvec + cluster))
+            assert not fails, (plan, nvec, rows, fails)
+            fails = parity.parity(wl(op, dt, min(rows, 7), nvec * ne, seed=nvec + stages), inplace=True)
+            assert not fails, ("in place", plan, nvec, rows, fails)
     for groups in (2, 8, 1000):                            # the direct form with interleaved row order
         tf.tf_force_plan(op, f"twopass:threads=256,persist=0,groups={groups},hints=0")
         assert not parity.parity(wl(op, dt, 37, 5000 * ne, seed=groups)), groups
     if op == "softmax":                                    # masks, a fully masked row and outputs in the subnormal range
         for plan in ("twopass:threads=256,persist=0,cluster=4", "twopass:threads=512,cache=8192,persist=0,regcap=1,cluster=8",
                      "twopass:threads=256,persist=0,stages=2,u=4", "twopass:threads=128,persist=0,regcap=1,stages=3,u=2,groups=4",
-                     "twopass:threads=128,persist=0,regcap=1,stages=2,u=4,cluster=2", "twopass:threads=64,persist=0,stages=3,u=2,cluster=8"):
+                     "twopass:threads=128,persist=0,regcap=1,stages=2,u=4,cluster=2", "twopass:threads=64,persist=0,stages=3,u=2,cluster=8",
+                     "twopass:threads=512,persist=0,stages=4,u=4", "twopass:threads=256,persist=0,stages=3,u=4,cluster=4"):
             tf.tf_force_plan(op, plan)
             w = Workload("m", "softmax", dt, 12, 40000, seed=5, x_std=10.0, mask_step=3001)
             data = w.generate()
