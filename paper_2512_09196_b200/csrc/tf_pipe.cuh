@@ -74,11 +74,12 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     __shared__ int tile_len[LEN ? kPipeMaxBarriers : 1];                            // LEN: the length of the row in each stage
 
     const int t = threadIdx.x;
+    const int nvec = FULL ? LANES * VPL : a.nvec;        // FULL builds: the row fills the unit, so its length is a constant
     const int units = blockDim.x / UT;
     const int unit = t / UT, ut = t % UT;               // unit index, thread index within the unit
     const int sub = ut / LANES, lane = ut % LANES;      // row slot within a pass, lane within the row
     const int S = a.nstage;
-    const size_t tile_vecs = static_cast<size_t>(a.tile_rows) * a.nvec;
+    const size_t tile_vecs = static_cast<size_t>(a.tile_rows) * nvec;
     uint4* const ring = reinterpret_cast<uint4*>(dyn_smem) + tile_vecs * S * unit;
     uint4* const params = reinterpret_cast<uint4*>(dyn_smem) + tile_vecs * S * units;
     uint64_t* const bars = full_bar + unit * S;
@@ -93,18 +94,18 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     pdl_wait();   // everything below may read what the previous kernel wrote
 
     auto len_of = [&](int64_t tile) {                    // LEN: a tile is a row
-        return tile < num_tiles ? min(max(__ldg(a.len + tile), 0), a.nvec * NE) : 0;
+        return tile < num_tiles ? min(max(__ldg(a.len + tile), 0), nvec * NE) : 0;
     };
     auto issue = [&](int64_t tile, int s, int len) {     // first thread of the unit only
         const int64_t row0 = tile * a.tile_rows;
         const int rows_here = static_cast<int>(min(static_cast<int64_t>(a.tile_rows), a.rows - row0));
-        uint32_t bytes = static_cast<uint32_t>(rows_here) * a.nvec * 16u;
+        uint32_t bytes = static_cast<uint32_t>(rows_here) * nvec * 16u;
         if constexpr (LEN) {
             tile_len[unit * S + s] = len;
             bytes = static_cast<uint32_t>((len + NE - 1) / NE) * 16u;              // the live vectors only
         }
         mbar_expect_tx(&bars[s], bytes);                 // also publishes tile_len to the threads that wait on the barrier
-        if (bytes) bulk_g2s(ring + tile_vecs * s, a.x + row0 * a.nvec, bytes, &bars[s]);
+        if (bytes) bulk_g2s(ring + tile_vecs * s, a.x + row0 * nvec, bytes, &bars[s]);
     };
     int pref_len = 0;                                    // LEN, issuing lane: the length of the tile it will issue next
     if (ut == 0) {
@@ -124,9 +125,9 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
         }
     }
     if (OP != OP_SOFTMAX) {
-        for (int i = t; i < a.nvec; i += blockDim.x) {
+        for (int i = t; i < nvec; i += blockDim.x) {
             params[i] = ld_param(a.p0 + i);
-            if (OP == OP_LAYERNORM) params[a.nvec + i] = ld_param(a.p1 + i);
+            if (OP == OP_LAYERNORM) params[nvec + i] = ld_param(a.p1 + i);
         }
     }
     __syncthreads();                                      // barriers initialised, parameters staged
@@ -134,9 +135,9 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
 
     bool valid[VPL];
 #pragma unroll
-    for (int v = 0; v < VPL; ++v) valid[v] = FULL || (lane + v * LANES) < a.nvec;
+    for (int v = 0; v < VPL; ++v) valid[v] = FULL || (lane + v * LANES) < nvec;
     const GroupRed<(LANES < 32 ? LANES : 32)> red;
-    const SmemParams par{params, a.nvec, lane, LANES};
+    const SmemParams par{params, nvec, lane, LANES};
     // a thread that owns one or two vectors per row (lane groups of narrow rows) keeps its parameters widened in registers
     constexpr bool kHeldWide = OP != OP_SOFTMAX && VPL <= 2 && LANES <= 32;
     HeldWideParams<DT, kHeldWide ? VPL : 1> wide;
@@ -153,7 +154,7 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     auto slice_count = [&](int w) {
         int c = 0;
 #pragma unroll
-        for (int v = 0; v < VPL; ++v) c += max(0, min(32, a.nvec - (w * 32 + v * LANES)));
+        for (int v = 0; v < VPL; ++v) c += max(0, min(32, nvec - (w * 32 + v * LANES)));
         return static_cast<float>(c * NE);
     };
     const int my_warp = ut >> 5;
@@ -161,17 +162,18 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
     (void)my_warp;
 
     bool failed = false;
-    int i = 0, xpar = 0;
-    for (int64_t tile = gu; tile < num_tiles; tile += GU, ++i) {
-        const int s = i % S;
-        if (!failed && !mbar_wait(&bars[s], static_cast<uint32_t>(i / S) & 1u)) {
+    int s = 0, xpar = 0;                                  // stage of the current tile; its barrier's phase parity
+    uint32_t phase = 0;
+    for (int64_t tile = gu; tile < num_tiles; tile += GU, s = (s + 1 == S ? 0 : s + 1), phase ^= (s == 0)) {
+        if (!failed && !mbar_wait(&bars[s], phase)) {
             failed = true;
             atomicExch(a.status, 4);
-            mbar_wait(&bars[s], static_cast<uint32_t>(i / S) & 1u);    // one more bounded wait for the copy
+            mbar_wait(&bars[s], phase);                    // one more bounded wait for the copy
         }
         const int64_t row0 = tile * a.tile_rows;
         const int rows_here = static_cast<int>(min(static_cast<int64_t>(a.tile_rows), a.rows - row0));
-        const uint4* stage = ring + tile_vecs * s;
+        const uint4* const stage = ring + tile_vecs * s + lane;          // this lane's column of the stage's first row
+        uint4* const ytile = a.y + row0 * nvec + lane;                  // ... and of the tile's first row of y (offsets inside a tile fit 32 bits)
         const int64_t next = tile + static_cast<int64_t>(S) * GU;
         // same trip count for every thread of the unit; slots past the tile compute on fill values and store nothing
         for (int r0 = 0; r0 < rows_here; r0 += RPU) {
@@ -182,7 +184,7 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
             for (int q = 0; q < RPG; ++q) {
                 r[q] = r0 + q * RPP + sub;
                 live[q] = (RPU == 1) || r[q] < rows_here;
-                const uint4* xr = stage + static_cast<size_t>(live[q] ? r[q] : 0) * a.nvec + lane;
+                const uint4* xr = stage + (live[q] ? r[q] : 0) * nvec;
                 if constexpr (LEN) {
                     const int len = tile_len[unit * S + s];
 #pragma unroll
@@ -235,7 +237,7 @@ __global__ void __launch_bounds__(kPipeMaxThreads) k_pipe(const PArgs a) {
             for (int q = 0; q < RPG; ++q) {
                 if (live[q]) {
                     const int64_t row = row0 + r[q];
-                    uint4* yr = a.y + row * a.nvec + lane;
+                    uint4* yr = ytile + r[q] * nvec;
 #pragma unroll
                     for (int v = 0; v < VPL; ++v)
                         if (valid[v]) st_stream(yr + v * LANES, out[q][v]);
