@@ -36,11 +36,15 @@ HEADLINE_CONFIG = 3               # the largest fixed configuration that fits on
 # configuration, from profiler captures of cases too large for the 126 MB L2 to hide the writes; None where no capture
 # exists.  Value = (bytes of the captured case, factor to a full launch of the configuration).
 NCU_TRAFFIC_BYTES = {
-    # LayerNorm bf16 [32768, 4096] (four times the rows of the configuration): 268.5 MB read + 215.3 MB written
-    "layernorm_bf16_8192x4096": (268_493_568 + 215_280_128, 0.25),
+    # LayerNorm bf16 [8192, 4096] itself (k_twopass_fit, untuned plan): 67.2 MB read (= the algorithmic reads) + 15.7 MB
+    # written inside an isolated launch; the rest of y is still dirty in L2 when the kernel ends (the problem is the size of L2)
+    "layernorm_bf16_8192x4096": (67_156_224 + 15_669_760, 1.0),
+    # RMSNorm bf16 [16384, 8192] itself (k_twopass_fit, untuned plan), a one-pass capture of the two DRAM counters:
+    # 268.5 MB read (= the algorithmic reads) + 212.1 MB written inside the kernel
+    "rmsnorm_bf16_16384x8192_outliers": (268_470_528 + 212_073_472, 1.0),
     # the 2 GiB masked softmax itself, a one-pass capture of the two DRAM counters on the full 4096 rows (untuned plan):
-    # 1080.3 MB read (the algorithmic reads are 1073.7 MB) + 1029.6 MB written inside the kernel
-    "masked_softmax_bf16_4096x131072": (1_080_327_168 + 1_029_625_088, 1.0),
+    # 1084.8 MB read (the algorithmic reads are 1073.7 MB) + 1015.9 MB written inside the kernel
+    "masked_softmax_bf16_4096x131072": (1_084_780_032 + 1_015_859_712, 1.0),
 }
 
 
