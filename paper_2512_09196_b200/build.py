@@ -13,7 +13,7 @@ HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 INCLUDE = HERE.parent / "include"
 LIB = HERE / "libtf.so"
-SOURCES = ["tf_api.cu", "tf_rowreg.cu", "tf_tma.cu", "tf_stream.cu", "tf_pipe.cu", "tf_ring.cu", "tf_twopass.cu", "tf_split.cu", "tf_elementwise.cu", "tf_vecmat.cu", "tf_addnorm.cu", "tf_softmaxlen.cu", "tf_softmax_variants.cu", "tf_norm_bwd.cu", "tf_pipe_softmax.cu", "tf_pipe_layernorm.cu", "tf_pipe_rmsnorm.cu"]
+SOURCES = ["tf_api.cu", "tf_rowreg.cu", "tf_tma.cu", "tf_stream.cu", "tf_pipe.cu", "tf_ring.cu", "tf_twopass.cu", "tf_split.cu", "tf_srows.cu", "tf_elementwise.cu", "tf_vecmat.cu", "tf_addnorm.cu", "tf_softmaxlen.cu", "tf_softmax_variants.cu", "tf_norm_bwd.cu", "tf_pipe_softmax.cu", "tf_pipe_layernorm.cu", "tf_pipe_rmsnorm.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-Xcompiler", "-fPIC"]
 
 

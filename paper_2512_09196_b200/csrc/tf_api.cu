@@ -71,7 +71,7 @@ tf_status device_state(DevState** out) {
 // ------------------------------------------------------------------------------------------------
 // plans as text
 // ------------------------------------------------------------------------------------------------
-const char* kVariantName[V_COUNT] = {"warp", "cta", "tma", "stream", "pipe", "ring", "twopass", "split"};
+const char* kVariantName[V_COUNT] = {"warp", "cta", "tma", "stream", "pipe", "ring", "twopass", "split", "srows"};
 
 std::string plan_to_string(const Plan& p) {
     char b[160];
@@ -83,6 +83,7 @@ std::string plan_to_string(const Plan& p) {
         case V_RING: snprintf(b, sizeof b, "ring:threads=%d,vpt=%d,cluster=%d,stages=%d,persist=%d,psmem=%d", p.threads, p.vpt, p.cluster, p.stages, p.persist, p.rpg == 2 ? 1 : 0); break;
         case V_TWOPASS: snprintf(b, sizeof b, "twopass:threads=%d,cache=%d,persist=%d,regcap=%d,cluster=%d,groups=%d,hints=%d,stages=%d,u=%d", p.threads, p.chunk, p.persist, p.rpg == 2 ? 1 : 0, p.cluster, p.lanes, p.vpt, p.stages, p.unroll); break;
         case V_SPLIT: snprintf(b, sizeof b, "split:threads=%d,splits=%d", p.threads, p.cluster); break;
+        case V_SROWS: snprintf(b, sizeof b, "srows:threads=%d,lanes=%d,vpt=%d", p.threads, p.lanes, p.vpt); break;
         default: snprintf(b, sizeof b, "stream:threads=%d,lanes=%d,persist=%d", p.threads, p.lanes, p.persist); break;
     }
     return b;
@@ -132,6 +133,7 @@ bool supports(const Plan& p, const Args& a, const DeviceInfo& d) {
         case V_RING: return supports_ring(p, a, d);
         case V_TWOPASS: return supports_twopass(p, a, d);
         case V_SPLIT: return supports_split(p, a, d);
+        case V_SROWS: return supports_srows(p, a, d);
     }
     return false;
 }
@@ -146,6 +148,7 @@ cudaError_t launch(const Plan& p, const Args& a, const DeviceInfo& d, cudaStream
         case V_RING: return launch_ring(p, a, d, st);
         case V_TWOPASS: return launch_twopass(p, a, d, st);
         case V_SPLIT: return launch_split(p, a, d, st);
+        case V_SROWS: return launch_srows(p, a, d, st);
         default: return launch_stream(p, a, d, st);
     }
 }
@@ -277,6 +280,17 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
         if (nvec == 512 && ln && a.dt == DT_F32) {
             q.variant = V_CTA; q.cluster = 1; q.persist = 0; q.vpt = 8; q.threads = 64;
             if (supports_cta(q, a, d)) return q;
+        }
+        if (nvec <= 128 && a.dt == DT_BF16 && a.op != OP_SOFTMAX && !(a.op == OP_RMSNORM && nvec > 64) && a.rows >= 64LL * d.sms) {
+            // bf16 LayerNorm rows up to 2 KiB and bf16 RMSNorm rows up to 1 KiB: blocks of rows resident in shared memory, a
+            // few lanes per row walking 4-16 vectors each (no or few shuffles per row), y leaving as one bulk copy per
+            // block.  LayerNorm bf16 rows of 64-512 columns: 81-82 us against 90-95 us for the pipeline (issue-bound there).
+            q.variant = V_SROWS; q.threads = (nvec > 8 && nvec <= 16) ? 64 : 128;
+            q.lanes = nvec <= 8 ? 2 : nvec <= 32 ? 4 : 8;
+            const int64_t need = (nvec + q.lanes - 1) / q.lanes;
+            q.vpt = need <= 4 ? 4 : need <= 8 ? 8 : 16;
+            if (supports_srows(q, a, d)) return q;
+            q = Plan();
         }
         if (nvec <= 64 && a.op == OP_RMSNORM && a.dt == DT_BF16) {
             // bf16 RMSNorm rows up to 1 KiB: small non-persistent pipeline CTAs (3-5 % ahead of the lane-group form)
@@ -501,6 +515,16 @@ std::vector<Plan> candidates(const Args& a, const DeviceInfo& d) {
                     p.rpg = 1; add(p);
                     if (th > 256) { p.rpg = 2; add(p); }
                 }
+    // narrow LayerNorm / RMSNorm rows resident in shared memory: every split of the row into 1-8 lanes x 4-16 vectors
+    if (nvec <= 128 && (a.op == OP_LAYERNORM || a.op == OP_RMSNORM))
+        for (int th : {64, 128, 256})
+            for (int lanes : {1, 2, 4, 8}) {
+                const int64_t need = (nvec + lanes - 1) / lanes;
+                const int vpt = need <= 4 ? 4 : need <= 8 ? 8 : 16;
+                if (need > 16) continue;
+                Plan p; p.variant = V_SROWS; p.threads = th; p.lanes = lanes; p.vpt = vpt;
+                add(p);
+            }
     // the ring form where the whole row fits the ring (straight-line build, one row per CTA): every CTA size whose
     // steps the row fills to at least three quarters
     if (nvec >= 128 && nvec <= 8192)
@@ -591,6 +615,10 @@ std::vector<Plan> neighbours(const Plan& b) {
         if (b.stages >= 2) with([&](Plan& p) { p.unroll = b.unroll == 4 ? 2 : 4; });
         for (int g : {1, 8}) if (g != b.lanes) with([&](Plan& p) { p.lanes = g; });
         for (int h : {0, 3}) if (h != b.vpt) with([&](Plan& p) { p.vpt = h; });
+    }
+    if (b.variant == V_SROWS) {                            // the same row on more lanes with fewer vectors each, and the other way round
+        if (b.vpt >= 8 && b.lanes * 2 <= 8) with([&](Plan& p) { p.vpt = b.vpt / 2; p.lanes = b.lanes * 2; });
+        if (b.lanes >= 2 && b.vpt * 2 <= 16) with([&](Plan& p) { p.vpt = b.vpt * 2; p.lanes = b.lanes / 2; });
     }
     if (b.variant == V_SPLIT)
         for (int sp : {b.cluster / 2, b.cluster * 3 / 4, b.cluster * 3 / 2, b.cluster * 2})

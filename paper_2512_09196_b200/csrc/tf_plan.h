@@ -18,7 +18,8 @@ enum Variant : int {
     V_RING = 5,     // persistent clusters: each CTA prefetches its slice of a long row into a shared-memory ring, registers hold it
     V_TWOPASS = 6,  // CTA per row, the row streamed twice with vector loads (second time from L2); any row length
     V_SPLIT = 7,    // few very long rows: a row cut into segments over many CTAs, partials merged through global scratch
-    V_COUNT = 8
+    V_SROWS = 8,    // narrow LayerNorm / RMSNorm rows resident in shared memory, 1-8 lanes per row, y leaves as one bulk copy
+    V_COUNT = 9
 };
 
 struct Plan {
@@ -73,6 +74,7 @@ bool supports_pipe(const Plan&, const Args&, const DeviceInfo&);
 bool supports_ring(const Plan&, const Args&, const DeviceInfo&);
 bool supports_twopass(const Plan&, const Args&, const DeviceInfo&);
 bool supports_split(const Plan&, const Args&, const DeviceInfo&);
+bool supports_srows(const Plan&, const Args&, const DeviceInfo&);
 cudaError_t launch_warp(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_cta(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_tma(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
@@ -81,6 +83,7 @@ cudaError_t launch_pipe(const Plan&, const Args&, const DeviceInfo&, cudaStream_
 cudaError_t launch_ring(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_twopass(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 cudaError_t launch_split(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
+cudaError_t launch_srows(const Plan&, const Args&, const DeviceInfo&, cudaStream_t);
 // The split plan with caller-provided scratch (split_scratch_bytes() of device memory).
 cudaError_t launch_split_with_scratch(const Plan&, const Args&, void* scratch, cudaStream_t);
 
