@@ -250,7 +250,9 @@ tf_status tf_device_status(void);
 /* ---- test and bench hooks ------------------------------------------------------------------------- */
 
 /* Plans are written as "variant:key=value,..." e.g. "cta:threads=256,vpt=2", "warp:lanes=8,vpt=1,rpg=4",
- * "tma:threads=512,cluster=4,stages=1", "stream:threads=256".  tf_force_plan makes every later call of `op`
+ * "tma:threads=512,cluster=4,stages=1", "srows:threads=128,lanes=4,vpt=8" (LayerNorm / RMSNorm rows of up to
+ * lanes x vpt 16-byte vectors, resident in shared memory), "twopass:threads=256,stages=2,u=4", "stream:threads=256".
+ * tf_force_plan makes every later call of `op`
  * use that plan (NULL or "" returns to automatic choice); a forced plan that cannot run a given shape
  * makes the call return TF_ERR_UNSUPPORTED. */
 tf_status tf_force_plan(tf_op op, const char* plan);
