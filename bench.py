@@ -847,6 +847,60 @@ def run_softmax_variants_table(args):
     (out_dir / "table_softmaxvariants.json").write_text(json.dumps(rows_out, indent=1))
 
 
+def run_sine_table(args):
+    """The element-wise sine (the paper's Case Study 1): time over its one tuning knob, the launch geometry
+    (threads per CTA x 16-byte vectors per thread = the "block size"), on 256 MiB of input per storage type."""
+    import torch
+    import paper_2512_09196_b200 as tf
+    torch.cuda.set_device(0)
+    out_dir = Path(args.out)
+    out_dir.mkdir(exist_ok=True)
+    rows_out = []
+    for dt, name in ((torch.float32, "f32"), (torch.bfloat16, "bf16")):
+        n = (256 << 20) // torch.empty(0, dtype=dt).element_size()
+        sets = 2                                              # 1 GiB of x and y in rotation: no launch finds its lines in L2
+        gen = torch.Generator(device="cuda").manual_seed(7)
+        xs = [(torch.rand(n, device="cuda", generator=gen) * 200.0 - 100.0).to(dt) for _ in range(sets)]
+        ys = [torch.empty_like(x) for x in xs]
+        nbytes = 2 * n * xs[0].element_size()
+
+        def timed(fn, reps=20):
+            for k in range(3):
+                fn(k % sets)
+            best = None
+            for _ in range(3):
+                a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                a.record()
+                for k in range(reps):
+                    fn(k % sets)
+                e.record()
+                torch.cuda.synchronize()
+                us = 1e3 * a.elapsed_time(e) / reps
+                best = us if best is None else min(best, us)
+            return best
+
+        grid = {}
+        for threads in (32, 64, 128, 256, 512, 1024):
+            for vpt in (1, 2, 4, 8):
+                grid[(threads, vpt)] = timed(lambda k: tf.tf_sin_fwd(xs[k], ys[k], threads, vpt))
+        us_default = timed(lambda k: tf.tf_sin_fwd(xs[k], ys[k]))
+        us_torch = timed(lambda k: torch.sin(xs[k], out=ys[k]))
+        us_copy = timed(lambda k: tf.tf_copy(xs[k], ys[k]))
+        tf.tf_device_status()
+        best, worst = min(grid, key=grid.get), max(grid, key=grid.get)
+        row = {"dtype": name, "elements": n, "bytes": nbytes, "default_us": us_default, "default_gbs": nbytes / us_default / 1e3,
+               "best_geometry": list(best), "best_us": grid[best], "best_gbs": nbytes / grid[best] / 1e3,
+               "worst_geometry": list(worst), "worst_us": grid[worst], "worst_over_best": grid[worst] / grid[best],
+               "torch_sin_us": us_torch, "tf_copy_us": us_copy,
+               "grid_us": {f"{t}x{v}": grid[(t, v)] for (t, v) in sorted(grid)}}
+        rows_out.append(row)
+        print(json.dumps(row), flush=True)
+        del xs, ys
+        torch.cuda.empty_cache()
+    (out_dir / "table_sine.json").write_text(json.dumps(rows_out, indent=1))
+
+
 def run_launch_table(args):
     """Launch-bound shapes: time per call made eagerly through the Python binding and as one CUDA graph of 32 captured calls."""
     import torch
@@ -1140,7 +1194,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm", "softmaxlen", "softmaxvariants", "normbwd", "launch"], default=None)
+    ap.add_argument("--table", choices=["configs", "sweep", "vecmat", "addnorm", "softmaxlen", "softmaxvariants", "normbwd", "launch", "sine"], default=None)
     ap.add_argument("--filter", default=None)
     ap.add_argument("--out", default=str(ROOT / "bench_out"), help="folder for the JSON files the --table modes write")
     ap.add_argument("--no-extras", action="store_true", help="default run: skip per_config and sweep_summary")
@@ -1172,6 +1226,8 @@ def main():
         return run_normbwd_table(args)
     if args.table == "launch":
         return run_launch_table(args)
+    if args.table == "sine":
+        return run_sine_table(args)
     if args.table:
         return run_table(args)
     run_ours(args)
