@@ -1,4 +1,5 @@
-// V_SROWS: narrow rows (128 B ... 2 KiB) of LayerNorm and RMSNorm, resident in shared memory, G lanes per row.
+// V_SROWS: narrow rows (128 B ... 2 KiB) of LayerNorm and RMSNorm (softmax: up to 512 B), resident in shared memory,
+// G lanes per row.
 //
 // The register-resident forms give a thread one or two vectors of such a row, so the per-row work -- two reductions
 // over 8-32 lanes, the row scalars, the statistics stores -- is paid once per vector or two, and bf16 LayerNorm rows
@@ -72,9 +73,11 @@ __global__ void __launch_bounds__(256, 4) k_srows(const SArgs a) {       // 64 r
     pdl_trigger();
     const uint4* const src = a.x + row0 * nvec;
     for (int i = t; i < tile_vecs; i += T) cp_async16_plain(tile + i, src + i);
-    for (int i = t; i < nvec; i += T) {
-        params[i] = ld_param(a.p0 + i);
-        if (OP == OP_LAYERNORM) params[nvec + i] = ld_param(a.p1 + i);
+    if (OP != OP_SOFTMAX) {
+        for (int i = t; i < nvec; i += T) {
+            params[i] = ld_param(a.p0 + i);
+            if (OP == OP_LAYERNORM) params[nvec + i] = ld_param(a.p1 + i);
+        }
     }
     cp_async_wait_all_plain();
     __syncthreads();
@@ -88,8 +91,44 @@ __global__ void __launch_bounds__(256, 4) k_srows(const SArgs a) {       // 64 r
         // (the walks are unrolled four vectors at a time: fully unrolled, the compiler hoists all of a pass's reads and spills)
         auto vec_of = [&](int k) { return g + G * ((k + rot) & (VPT - 1)); };
         const GroupRed<G> red;
-        float mean = 0.f, scale;
-        if constexpr (OP == OP_LAYERNORM) {
+        float mean = 0.f, scale = 0.f;
+        if constexpr (OP == OP_SOFTMAX) {
+            // softmax (VPT <= 4 only): the exponentials stay in registers between the sum and the normalisation, one MUFU
+            // per element; vectors behind the end of a ragged row contribute nothing
+            float m = kNegInf;
+#pragma unroll
+            for (int k = 0; k < VPT; ++k) {
+                const int j = vec_of(k);
+                if (FULL || j < nvec) m = fmaxf(m, vec_max<DT>(lds_again(rowp + j)));
+            }
+            m = red.max(m, 0);
+            const F2 off = f2(exp_offset(m)), l2e = f2(kLog2e);
+            F2 e[VPT][NP];
+            F2 s0 = f2(0.f);
+#pragma unroll
+            for (int k = 0; k < VPT; ++k) {
+                const int j = vec_of(k);
+                if (FULL || j < nvec) {
+                    P::unpack(lds_again(rowp + j), e[k]);
+#pragma unroll
+                    for (int i = 0; i < NP; ++i) { e[k][i] = ex2_ftz2(fma2(e[k][i], l2e, off)); s0 = add2(s0, e[k][i]); }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < NP; ++i) e[k][i] = f2(0.f);
+                }
+            }
+            const float sum = red.sum(hsum(s0), 0);
+            const F2 inv = f2(sum == 0.f ? 0.f : fast_rcp(sum));
+#pragma unroll
+            for (int k = 0; k < VPT; ++k) {
+                const int j = vec_of(k);
+                if (live && (FULL || j < nvec)) {
+#pragma unroll
+                    for (int i = 0; i < NP; ++i) e[k][i] = mul2(e[k][i], inv);
+                    rowp[j] = P::pack(e[k]);
+                }
+            }
+        } else if constexpr (OP == OP_LAYERNORM) {
             F2 s0 = f2(0.f), s1 = f2(0.f);
 #pragma unroll 4
             for (int k = 0; k < VPT; ++k) {
@@ -132,17 +171,19 @@ __global__ void __launch_bounds__(256, 4) k_srows(const SArgs a) {       // 64 r
             }
             scale = fast_rsqrt(fast_div(red.sum(hsum(add2(q0, q1)), 0), a.n) + a.eps);
         }
-        if (g == 0 && live) {
-            const int64_t row = row0 + r;
-            if (OP == OP_LAYERNORM && a.mean) a.mean[row] = mean;
-            if (a.rstd) a.rstd[row] = scale;
-        }
-        // LayerNorm: (mean, rstd); RMSNorm: (rrms, rrms)
-        const F2 ta2 = f2(OP == OP_LAYERNORM ? mean : scale), tb2 = f2(scale);
+        if constexpr (OP != OP_SOFTMAX) {
+            if (g == 0 && live) {
+                const int64_t row = row0 + r;
+                if (OP == OP_LAYERNORM && a.mean) a.mean[row] = mean;
+                if (a.rstd) a.rstd[row] = scale;
+            }
+            // LayerNorm: (mean, rstd); RMSNorm: (rrms, rrms)
+            const F2 ta2 = f2(OP == OP_LAYERNORM ? mean : scale), tb2 = f2(scale);
 #pragma unroll 4
-        for (int k = 0; k < VPT; ++k) {
-            const int j = vec_of(k);
-            if (live && (FULL || j < nvec)) rowp[j] = apply_vec<OP, DT, true>(lds_again(rowp + j), params + j, params + nvec + j, ta2, tb2);
+            for (int k = 0; k < VPT; ++k) {
+                const int j = vec_of(k);
+                if (live && (FULL || j < nvec)) rowp[j] = apply_vec<OP, DT, true>(lds_again(rowp + j), params + j, params + nvec + j, ta2, tb2);
+            }
         }
     }
     fence_async_proxy();
@@ -156,6 +197,9 @@ template <int G, int VPT, bool FULL>
 SFn srows_fn_c(int op, int dt) {
     if (op == OP_LAYERNORM) return dt == DT_F32 ? k_srows<OP_LAYERNORM, DT_F32, G, VPT, FULL> : k_srows<OP_LAYERNORM, DT_BF16, G, VPT, FULL>;
     if (op == OP_RMSNORM) return dt == DT_F32 ? k_srows<OP_RMSNORM, DT_F32, G, VPT, FULL> : k_srows<OP_RMSNORM, DT_BF16, G, VPT, FULL>;
+    if constexpr (VPT <= 4) {
+        if (op == OP_SOFTMAX) return dt == DT_F32 ? k_srows<OP_SOFTMAX, DT_F32, G, VPT, FULL> : k_srows<OP_SOFTMAX, DT_BF16, G, VPT, FULL>;
+    }
     return nullptr;
 }
 SFn srows_fn(int op, int dt, int g, int vpt, bool full) {
@@ -167,14 +211,14 @@ SFn srows_fn(int op, int dt, int g, int vpt, bool full) {
 
 size_t srows_smem(const Plan& p, const Args& a) {
     const int64_t nvec = a.cols * elem_size(a.dt) / 16;
-    return static_cast<size_t>((p.threads / p.lanes) * nvec + nvec * (a.op == OP_LAYERNORM ? 2 : 1)) * 16;
+    return static_cast<size_t>((p.threads / p.lanes) * nvec + nvec * (a.op == OP_LAYERNORM ? 2 : a.op == OP_RMSNORM ? 1 : 0)) * 16;
 }
 
 }  // namespace
 
 // Plan fields: `threads` (64, 128 or 256), `lanes` = lanes per row (1, 2, 4, 8), `vpt` = vectors per lane (4, 8, 16).
 bool supports_srows(const Plan& p, const Args& a, const DeviceInfo& d) {
-    if (!vector_ok(a) || a.len || a.r || (a.op != OP_LAYERNORM && a.op != OP_RMSNORM)) return false;
+    if (!vector_ok(a) || a.len || a.r) return false;                  // (softmax: rows of up to lanes x 4 vectors)
     if (p.threads != 64 && p.threads != 128 && p.threads != 256) return false;
     const int64_t nvec = a.cols * elem_size(a.dt) / 16;
     if (p.lanes < 1 || p.vpt < 1 || nvec < 1 || nvec > static_cast<int64_t>(p.lanes) * p.vpt) return false;
