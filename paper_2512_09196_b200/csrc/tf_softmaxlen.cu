@@ -3,8 +3,11 @@
 // the masked tails; the writes stay.
 //
 // Served by the register-resident kernels in their length mode (a lane group, a CTA or a cluster holds the row), by the
-// streamed two-pass kernel for rows beyond 128 KiB, and by a scalar CTA-per-row kernel for tensors that are not
+// pipeline and by the two-pass kernel's ring form for rows that fit the ring (only the live part of a row is copied), by
+// the streamed two-pass kernel for rows beyond 64 KiB, and by a scalar CTA-per-row kernel for tensors that are not
 // 16-byte aligned or whose width is not a whole number of 16-byte vectors.
+#include <algorithm>
+
 #include "tf_rowreg.cuh"
 
 namespace tf {
@@ -65,9 +68,10 @@ cudaError_t launch_softmax_len(const Plan& p, const Args& a, const DeviceInfo& d
     return launch_cta_fn(cta_fn_len(a.dt, p.vpt, p.cluster > 1), p, a, d, st);
 }
 
-// Default plan, from measurements on rows of 512 B to 64 KiB: a lane group with one row in flight up to 1 KiB, the
-// length-aware pipeline for 2-byte rows of 4-64 KiB, a CTA with four vectors per thread (eight for fp32 from 16 KiB on)
-// for the rest up to 64 KiB, the streamed two-pass kernel from there.
+// Default plan, from measurements on rows of 512 B to 64 KiB: a lane group with one row in flight up to 1 KiB, the ring
+// form of the two-pass kernel with the whole row in the ring for rows of 4-64 KiB (behind it, for what that form
+// refuses: the length-aware pipeline for 2-byte rows, a CTA with four vectors per thread, eight for fp32 from 16 KiB
+// on), the streamed two-pass kernel from there.
 // (The plans that win for the plain softmax are not reused: more rows in flight per group or eight bf16 vectors per
 // thread cost this mode 30-80 %.)
 Plan heuristic_softmax_len(const Args& a, const DeviceInfo& d) {
@@ -80,6 +84,23 @@ Plan heuristic_softmax_len(const Args& a, const DeviceInfo& d) {
         else if (nvec <= 32) { q.lanes = 16; q.vpt = 2; }
         else { q.lanes = 32; q.vpt = 2; }
         if (supports_softmax_len(q, a, d)) return q;
+    }
+    if (nvec >= 256 && nvec <= 4096) {
+        // rows of 4-64 KiB: the two-pass ring form with the whole row in the ring of one CTA copies only the live vectors of a
+        // row and finds them in shared memory for the second pass.  Half-live bf16 rows of 8-64 KiB: 64 us against 73-94 us
+        // for the pipeline and the two-pass direct form (and 79-85 us for the plain softmax on the same rows with the mask in
+        // the data); full-length rows 82-84 us against 89-110 us.  CTAs of a sixteenth of the row's vectors for 2-byte rows
+        // (four steps), an eighth for 4-byte ones.
+        const int64_t per = (nvec + (a.dt == DT_BF16 ? 15 : 7)) / (a.dt == DT_BF16 ? 16 : 8);
+        q = Plan{};
+        q.variant = V_TWOPASS; q.chunk = 0; q.lanes = 1; q.vpt = 3; q.persist = 0; q.rpg = 1; q.cluster = 1; q.unroll = 4;
+        q.threads = static_cast<int>(std::min<int64_t>(256, std::max<int64_t>(32, (per + 31) / 32 * 32)));
+        const int64_t steps = (nvec + 4 * q.threads - 1) / (4 * q.threads);
+        q.stages = static_cast<int>(std::max<int64_t>(2, steps));
+        if (steps <= 4 && supports_softmax_len(q, a, d)) return q;
+        q = Plan{};
+    }
+    if (nvec <= 64) {
     } else if (a.dt == DT_BF16 && nvec >= 256 && nvec <= 4096) {
         // 2-byte rows of 4-64 KiB: the pipeline copies only the live part of each row and its units skip the vectors
         // behind the length (measured 7-16 % faster than the masked plain softmax at half-live rows, where the register

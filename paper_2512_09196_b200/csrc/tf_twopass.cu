@@ -347,7 +347,9 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
-template <int OP, int DT, int U, int NS, bool FULL, bool CL>
+// LEN (softmax, one CTA per row): the row is normalised over its first len[row] elements; only the live vectors are
+// copied, the vector the length ends in is masked where it is used, and zeros are written behind it.
+template <int OP, int DT, int U, int NS, bool FULL, bool CL, bool LEN = false>
 __global__ void __launch_bounds__(1024, 1) k_twopass_fit(const WArgs a) {
     constexpr int NE = Elem<DT>::NE, CH = U * 32;
     __shared__ float red_buf[2 * 32];
@@ -368,11 +370,18 @@ __global__ void __launch_bounds__(1024, 1) k_twopass_fit(const WArgs a) {
     const uint4* const xr = a.x + row * nvec + mine;
     uint4* const yr = a.y + row * nvec + mine;
     uint4* const myring = reinterpret_cast<uint4*>(dyn_smem) + toff;
+    int lim = nvec, straddle = -1, keep = 0;                             // LEN: live vectors; the vector the length ends in and how much of it is live
+    if constexpr (LEN) {
+        const int len = min(max(__ldg(a.len + row), 0), nvec * NE);
+        lim = (len + NE - 1) / NE;
+        keep = len % NE;
+        straddle = keep ? len / NE : -1;
+    }
 #pragma unroll
     for (int s = 0; s < NS; ++s) {
 #pragma unroll
         for (int u = 0; u < U; ++u)
-            if (FULL || s * gstep + mine + u * 32 < nvec) cp_async16(myring + s * step + u * 32, xr + s * gstep + u * 32, once);
+            if (FULL || s * gstep + mine + u * 32 < lim) cp_async16(myring + s * step + u * 32, xr + s * gstep + u * 32, once);
         cp_async_commit();
     }
     Running<OP, DT, U> run;
@@ -382,18 +391,19 @@ __global__ void __launch_bounds__(1024, 1) k_twopass_fit(const WArgs a) {
         cp_async_wait(NS - 1 - s);
         const int first = s * gstep + mine;
         uint4 raw[U];
-        if (FULL || first + (U - 1) * 32 < nvec) {
+        if (FULL || (!LEN && first + (U - 1) * 32 < nvec)) {
 #pragma unroll
             for (int u = 0; u < U; ++u) raw[u] = myring[s * step + u * 32];
             const bool all[U] = {};
             run.template update<false>(raw, all, U * NE, s * U);
-        } else if (first < nvec) {
+        } else if (first < lim) {
             bool ok[U];
             int count = 0;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                ok[u] = first + u * 32 < nvec;
+                ok[u] = first + u * 32 < lim;
                 raw[u] = ok[u] ? myring[s * step + u * 32] : fill;
+                if (LEN && first + u * 32 == straddle) raw[u] = mask_tail<DT>(raw[u], keep);
                 count += ok[u] ? NE : 0;
             }
             run.template update<true>(raw, ok, count, s * U);
@@ -447,7 +457,17 @@ __global__ void __launch_bounds__(1024, 1) k_twopass_fit(const WArgs a) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int o = s * gstep + u * 32;
-            if (FULL || o + mine < nvec) st_stream(yr + o, apply_vec<OP, DT>(myring[s * step + u * 32], gp + o, bp + o, ta2, tb2));
+            if constexpr (LEN) {
+                if (o + mine < lim) {
+                    uint4 raw = myring[s * step + u * 32];
+                    if (o + mine == straddle) raw = mask_tail<DT>(raw, keep);
+                    st_stream(yr + o, apply_vec<OP, DT>(raw, gp + o, bp + o, ta2, tb2));
+                } else if (o + mine < nvec) {
+                    st_stream(yr + o, make_uint4(0, 0, 0, 0));
+                }
+            } else if (FULL || o + mine < nvec) {
+                st_stream(yr + o, apply_vec<OP, DT>(myring[s * step + u * 32], gp + o, bp + o, ta2, tb2));
+            }
         }
     }
 }
@@ -470,6 +490,13 @@ template <int NS>
 TwoFn fit_fn_b(int op, int dt, bool full, bool cl) {
     if (cl) return full ? fit_fn_c<NS, true, true>(op, dt) : fit_fn_c<NS, false, true>(op, dt);
     return full ? fit_fn_c<NS, true, false>(op, dt) : fit_fn_c<NS, false, false>(op, dt);
+}
+// softmax with per-row lengths
+TwoFn fit_len_fn(int dt, int steps) {
+#define TF_FL(NS) if (steps == NS) return dt == DT_F32 ? k_twopass_fit<OP_SOFTMAX, DT_F32, 4, NS, false, false, true> : k_twopass_fit<OP_SOFTMAX, DT_BF16, 4, NS, false, false, true>;
+    TF_FL(1) TF_FL(2) TF_FL(3) TF_FL(4)
+#undef TF_FL
+    return nullptr;
 }
 // steps: what a CTA takes of the row (1 .. 4)
 TwoFn fit_fn(int op, int dt, int steps, bool full, bool cl) {
@@ -543,8 +570,13 @@ bool supports_twopass(const Plan& p, const Args& a, const DeviceInfo& d) {
     if (p.cluster > 1 && (p.cluster > d.max_cluster || a.rows * p.cluster > 0x7FFFFFFF)) return false;
     if (p.lanes < 1 || p.lanes > 1024 || p.vpt < 0 || p.vpt > 3) return false;
     if (p.stages >= 2) {                                           // the ring form: no length mode, no separate cache
-        if (p.stages > kRingMaxDepth || (p.unroll != 2 && p.unroll != 4) || p.chunk != 0 || a.len) return false;
+        if (p.stages > kRingMaxDepth || (p.unroll != 2 && p.unroll != 4) || p.chunk != 0) return false;
         const int64_t nvec = a.cols * elem_size(a.dt) / 16;
+        if (a.len) {                                               // lengths: softmax rows that fit the ring of one CTA
+            const int64_t step = static_cast<int64_t>(p.threads / 32) * p.unroll * 32;
+            if (a.op != OP_SOFTMAX || p.cluster != 1 || p.lanes != 1 || p.persist != 0 || p.unroll != 4 || p.rpg != 1 ||
+                (nvec + step - 1) / step > std::min(p.stages, 4) || a.rows > 0x7FFFFFFF) return false;
+        }
         if (nvec > 0x7FFFFFFF - 65536) return false;              // 32-bit vector indices inside the kernel
         return vector_ok(a) && (p.rpg == 1 || p.rpg == 2) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0 &&
                (d.smem_optin == 0 || static_cast<int64_t>(p.stages) * p.threads * p.unroll * 16 + 1024 <= d.smem_optin);
@@ -568,9 +600,11 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
         const int64_t steps = ((nvec + step - 1) / step + cs - 1) / cs;
         if (steps <= std::min(p.stages, 4)) {
             fit_steps = static_cast<int>(steps);
-            fn = fit_fn(a.op, a.dt, fit_steps, steps * step * cs == nvec, cs > 1);
+            fn = a.len ? (cs == 1 && a.op == OP_SOFTMAX ? fit_len_fn(a.dt, fit_steps) : nullptr) : fit_fn(a.op, a.dt, fit_steps, steps * step * cs == nvec, cs > 1);
         }
     }
+    if (ring && a.len && !fit_steps) fn = nullptr;                 // the ring form knows lengths only where the row fits the ring
+    if (!fn) return cudaErrorInvalidValue;
     const int64_t slots = (a.rows + groups - 1) / groups * groups;
     int64_t grid = slots;                                          // in rows (clusters)
     if (p.persist > 0) grid = std::min<int64_t>(grid, std::max<int64_t>(1, static_cast<int64_t>(p.persist) * d.sms / cs));

@@ -104,6 +104,14 @@ def test_forced_plans_and_bitwise_equality_with_the_masked_plain_softmax(dt):
             rows = min(rows, max(3, (1 << 22) // (nvec * ne)))
             tf.tf_force_plan("softmax", f"pipe:threads={threads},lanes={lanes},vpt={vpt},rpg=1,stages={stages},chunk=16,persist={persist}")
             run_case(dt, rows, nvec * ne, seed=nvec + lanes, compare_plain=False)
+    # rows that fit the ring of one CTA: only the live vectors are copied; exact and ragged fits, one to four steps
+    for threads, stages in ((32, 3), (64, 2), (128, 4), (256, 2), (512, 1 + 1)):
+        st = threads * 4
+        for nvec, rows in ((st * stages, 9), (st * stages - 1, 170), (st + 1, 170), (1, 9), (max(1, st // 2), 301)):
+            rows = min(rows, max(3, (1 << 22) // (nvec * ne)))
+            tf.tf_force_plan("softmax", f"twopass:threads={threads},persist=0,regcap=0,stages={stages},u=4")
+            run_case(dt, rows, nvec * ne, seed=nvec + threads)
+        run_case(dt, 23, st * ne, seed=st, inplace=True)
     # a forced plan without a length mode (the cluster ring) falls back to the length-aware choice
     tf.tf_force_plan("softmax", "ring:threads=256,vpt=4,cluster=2,stages=2,persist=1")
     run_case(dt, 100, 2048 * ne)
