@@ -450,6 +450,117 @@ __global__ void __launch_bounds__(256) k_row2_scalar(const typename Elem<DT>::sc
 
 bool al16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Log-softmax forward on rows of 8-64 KiB: the row is copied into shared memory by 16-byte asynchronous copies that are
+// all requested at once (NS steps of four vectors per thread, a warp taking 128 consecutive vectors per step), then swept
+// three times out of shared memory -- maximum, sum of exponentials, result -- with the arithmetic of the register forms
+// above ((x - m) first, then minus ln S).  The row costs no registers, so a dozen small CTAs are resident per SM and
+// the copies of the next rows are in flight while this one is worked on.  FULL: the row fills the steps exactly.
+__device__ __forceinline__ void lsm_cp_async16(uint4* dst, const uint4* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+template <int N> __device__ __forceinline__ void lsm_cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <int DT, int NS, bool FULL>
+__global__ void __launch_bounds__(256, 4) k_logsoftmax_smem(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t rows, int nvec) {
+    using E = Elem<DT>;
+    constexpr int NE = E::NE, U = 4;
+    __shared__ float buf[2][32];
+    extern __shared__ __align__(16) unsigned char lsm_smem[];
+    pdl_wait();
+    pdl_trigger();
+    const int t = threadIdx.x;
+    const int step = (blockDim.x >> 5) * U * 32;
+    const int toff = (t >> 5) * U * 32 + (t & 31);
+    const int64_t row = blockIdx.x;
+    const uint4* const xr = x + row * nvec + toff;
+    uint4* const yr = y + row * nvec + toff;
+    const uint4* const ring = reinterpret_cast<const uint4*>(lsm_smem) + toff;
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (FULL || s * step + toff + u * 32 < nvec) lsm_cp_async16(const_cast<uint4*>(ring) + s * step + u * 32, xr + s * step + u * 32);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    float m = kNegInf;
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+        if (s == 0) lsm_cp_async_wait<NS - 1>();
+        else if (s == 1) lsm_cp_async_wait<(NS > 2 ? NS - 2 : 0)>();
+        else if (s == 2) lsm_cp_async_wait<(NS > 3 ? NS - 3 : 0)>();
+        else lsm_cp_async_wait<0>();
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (FULL || s * step + toff + u * 32 < nvec) m = fmaxf(m, vec_max<DT>(ring[s * step + u * 32]));
+    }
+    m = cta_reduce<MaxOp>(m, buf[0]);
+    float acc[U] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (FULL || s * step + toff + u * 32 < nvec) {
+                float v[NE];
+                E::unpack(ring[s * step + u * 32], v);
+#pragma unroll
+                for (int i = 0; i < NE; ++i) acc[u] += ex2_ftz((v[i] - m) * kLog2e);     // 2^0 = 1 exactly for the maximum
+            }
+        }
+    }
+    const float sum = cta_reduce<SumOp>((acc[0] + acc[1]) + (acc[2] + acc[3]), buf[1]);
+    const float lns = logf(sum);
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (FULL || s * step + toff + u * 32 < nvec) {
+                float v[NE];
+                E::unpack(ring[s * step + u * 32], v);
+#pragma unroll
+                for (int i = 0; i < NE; ++i) v[i] = (m == kNegInf) ? kNegInf : (v[i] - m) - lns;
+                st_stream(yr + s * step + u * 32, E::pack(v));
+            }
+        }
+    }
+}
+
+template <int DT, int NS, bool FULL>
+cudaError_t launch_logsoftmax_smem(int threads, cudaStream_t st, const void* in0, void* out, int64_t rows, int nvec) {
+    auto fn = k_logsoftmax_smem<DT, NS, FULL>;
+    const size_t smem = static_cast<size_t>(NS) * threads * 4 * 16;
+    static bool raised = false;                                  // per instantiation; the limit is a property of the function
+    if (smem > 40 * 1024 && !raised) {                           // the default limit counts the static buffers as well
+        const cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+        if (e != cudaSuccess) return e;
+        raised = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(rows));
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, static_cast<const uint4*>(in0), static_cast<uint4*>(out), rows, nvec);
+}
+
+template <int DT>
+cudaError_t launch_logsoftmax_smem_dt(cudaStream_t st, const void* in0, void* out, int64_t rows, int nvec) {
+    const int threads = std::min(256, std::max(32, ((nvec + 7) / 8 + 31) / 32 * 32));
+    const int steps = (nvec + threads * 4 - 1) / (threads * 4);
+    const bool full = steps * threads * 4 == nvec;
+    switch (steps) {
+        case 1: return full ? launch_logsoftmax_smem<DT, 1, true>(threads, st, in0, out, rows, nvec) : launch_logsoftmax_smem<DT, 1, false>(threads, st, in0, out, rows, nvec);
+        case 2: return full ? launch_logsoftmax_smem<DT, 2, true>(threads, st, in0, out, rows, nvec) : launch_logsoftmax_smem<DT, 2, false>(threads, st, in0, out, rows, nvec);
+        case 3: return full ? launch_logsoftmax_smem<DT, 3, true>(threads, st, in0, out, rows, nvec) : launch_logsoftmax_smem<DT, 3, false>(threads, st, in0, out, rows, nvec);
+        case 4: return full ? launch_logsoftmax_smem<DT, 4, true>(threads, st, in0, out, rows, nvec) : launch_logsoftmax_smem<DT, 4, false>(threads, st, in0, out, rows, nvec);
+    }
+    return cudaErrorInvalidValue;
+}
+
 int sm_count() {
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
@@ -548,6 +659,11 @@ cudaError_t launch_dt(cudaStream_t st, const void* in0, const void* in1, void* o
     }
     const int64_t bytes = cols * Elem<DT>::SIZE;
     const bool aligned = al16(in0) && al16(out) && (WHICH == kOpLogSoftmax || al16(in1)) && bytes % 16 == 0;
+    if constexpr (WHICH == kOpLogSoftmax) {
+        // the forward pass on many rows of 8-64 KiB: the row staged in shared memory by asynchronous copies
+        if (aligned && g_force_cluster == 0 && bytes >= 8 * 1024 && bytes <= 64 * 1024 && rows >= 2LL * sm_count())
+            return launch_logsoftmax_smem_dt<DT>(st, in0, out, rows, static_cast<int>(bytes / 16));
+    }
     int vpt = 0, threads = 0;
     // a cluster per row: rows beyond 32 KiB when there are too few of them to fill the device with one CTA each -- as many
     // CTAs per row (2, 4 or 8) as keep the launch within about two CTAs per SM.  With more rows of up to 128 KiB the

@@ -123,6 +123,15 @@ def test_log_softmax_over_edge_widths(dt):
     for cols in (ne, 2 * ne, 64, 256, 1000 // ne * ne, 1024, 2048, 4096, 5120, 8192, 16384, 32768, 65536, 131072, 200000 // ne * ne):
         run_log_softmax(dt, max(3, min(200, (1 << 21) // cols)), cols, seed=cols)
     run_log_softmax(dt, 0, 64)
+    # many rows of 8-64 KiB (the form that stages the row in shared memory): rows that fill one to four steps exactly, ragged
+    # ones, masks and a fully masked row, in place; 295 rows of the same width take the register forms
+    es = 4 if dt == F32 else 2
+    for kib, rows in ((8, 320), (12, 300), (16, 333), (24, 296), (32, 300), (48, 297), (64, 296)):
+        cols = kib * 1024 // es
+        run_log_softmax(dt, rows, cols, seed=kib, mask=True)
+        run_log_softmax(dt, rows, cols - ne, seed=kib + 1, mask=kib % 16 == 0, std=12.0)
+    run_log_softmax(dt, 310, 10240 // es + 3 * ne, seed=5, inplace=True)
+    run_log_softmax(dt, 295, 16384 // es, seed=6, mask=True)
     run_log_softmax(dt, 301, 1024, mask=True)
     run_log_softmax(dt, 9, 40000, mask=True, std=20.0)
     run_log_softmax(dt, 50, 2048, inplace=True)
