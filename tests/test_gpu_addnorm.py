@@ -92,6 +92,18 @@ def test_forced_register_plans(op, dt):
                 tf.tf_force_plan(op, f"cta:threads={threads},vpt={vpt},cluster={cluster},persist={persist}")
                 run_case(op, dt, 9 if nvec >= 4096 else 170, nvec * ne, seed=nvec)
     # a forced plan that the fused kernels do not have (the pipeline) falls back to their own choice: still exact
+    # x and r staged in shared memory: rows of one to four steps, exact and ragged, in place, one row
+    for threads, stages in ((32, 2), (64, 4), (128, 2), (256, 3)):
+        st = threads * 4
+        for nvec, rows in ((st * stages, 9), (st * stages - 1, 170), (st + 1, 301), (1, 5), (st, 1)):
+            tf.tf_force_plan(op, f"twopass:threads={threads},persist=0,regcap=0,stages={stages},u=4")
+            run_case(op, dt, min(rows, max(3, (1 << 21) // (nvec * ne))), nvec * ne, seed=nvec + threads)
+        run_case(op, dt, 23, st * 2 * ne, seed=st, inplace=True)
+    tf.tf_force_plan(op, None)
+    es = 4 if dt == F32 else 2
+    for kib in (8, 16, 24, 32):                          # the default for many rows of 8-32 KiB
+        run_case(op, dt, 300, kib * 1024 // es, seed=kib)
+        run_case(op, dt, 297, kib * 1024 // es - ne, seed=kib + 1, inplace=True)
     tf.tf_force_plan(op, "pipe:threads=512,lanes=64,vpt=8,rpg=1,stages=2,chunk=8192,persist=1")
     run_case(op, dt, 100, 512 * ne)
 
