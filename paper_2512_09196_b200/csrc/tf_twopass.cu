@@ -347,7 +347,7 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
-// LEN (softmax, one CTA per row): the row is normalised over its first len[row] elements; only the live vectors are
+// LEN (softmax): the row is normalised over its first len[row] elements; only the live vectors are
 // copied, the vector the length ends in is masked where it is used, and zeros are written behind it.
 template <int OP, int DT, int U, int NS, bool FULL, bool CL, bool LEN = false>
 __global__ void __launch_bounds__(1024, 1) k_twopass_fit(const WArgs a) {
@@ -491,9 +491,13 @@ TwoFn fit_fn_b(int op, int dt, bool full, bool cl) {
     if (cl) return full ? fit_fn_c<NS, true, true>(op, dt) : fit_fn_c<NS, false, true>(op, dt);
     return full ? fit_fn_c<NS, true, false>(op, dt) : fit_fn_c<NS, false, false>(op, dt);
 }
-// softmax with per-row lengths
-TwoFn fit_len_fn(int dt, int steps) {
-#define TF_FL(NS) if (steps == NS) return dt == DT_F32 ? k_twopass_fit<OP_SOFTMAX, DT_F32, 4, NS, false, false, true> : k_twopass_fit<OP_SOFTMAX, DT_BF16, 4, NS, false, false, true>;
+// softmax with per-row lengths (one CTA per row, or the CTAs of a cluster)
+TwoFn fit_len_fn(int dt, int steps, bool cl) {
+#define TF_FL(NS)                                                                                                                  \
+    if (steps == NS) {                                                                                                             \
+        if (cl) return dt == DT_F32 ? k_twopass_fit<OP_SOFTMAX, DT_F32, 4, NS, false, true, true> : k_twopass_fit<OP_SOFTMAX, DT_BF16, 4, NS, false, true, true>; \
+        return dt == DT_F32 ? k_twopass_fit<OP_SOFTMAX, DT_F32, 4, NS, false, false, true> : k_twopass_fit<OP_SOFTMAX, DT_BF16, 4, NS, false, false, true>; \
+    }
     TF_FL(1) TF_FL(2) TF_FL(3) TF_FL(4)
 #undef TF_FL
     return nullptr;
@@ -574,8 +578,8 @@ bool supports_twopass(const Plan& p, const Args& a, const DeviceInfo& d) {
         const int64_t nvec = a.cols * elem_size(a.dt) / 16;
         if (a.len) {                                               // lengths: softmax rows that fit the ring of one CTA
             const int64_t step = static_cast<int64_t>(p.threads / 32) * p.unroll * 32;
-            if (a.op != OP_SOFTMAX || p.cluster != 1 || p.lanes != 1 || p.persist != 0 || p.unroll != 4 || p.rpg != 1 ||
-                (nvec + step - 1) / step > std::min(p.stages, 4) || a.rows > 0x7FFFFFFF) return false;
+            if (a.op != OP_SOFTMAX || p.lanes != 1 || p.persist != 0 || p.unroll != 4 || p.rpg != 1 ||
+                ((nvec + step - 1) / step + p.cluster - 1) / p.cluster > std::min(p.stages, 4) || a.rows * p.cluster > 0x7FFFFFFF) return false;
         }
         if (nvec > 0x7FFFFFFF - 65536) return false;              // 32-bit vector indices inside the kernel
         return vector_ok(a) && (p.rpg == 1 || p.rpg == 2) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0 &&
@@ -600,7 +604,7 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
         const int64_t steps = ((nvec + step - 1) / step + cs - 1) / cs;
         if (steps <= std::min(p.stages, 4)) {
             fit_steps = static_cast<int>(steps);
-            fn = a.len ? (cs == 1 && a.op == OP_SOFTMAX ? fit_len_fn(a.dt, fit_steps) : nullptr) : fit_fn(a.op, a.dt, fit_steps, steps * step * cs == nvec, cs > 1);
+            fn = a.len ? (a.op == OP_SOFTMAX ? fit_len_fn(a.dt, fit_steps, cs > 1) : nullptr) : fit_fn(a.op, a.dt, fit_steps, steps * step * cs == nvec, cs > 1);
         }
     }
     if (ring && a.len && !fit_steps) fn = nullptr;                 // the ring form knows lengths only where the row fits the ring

@@ -112,6 +112,13 @@ def test_forced_plans_and_bitwise_equality_with_the_masked_plain_softmax(dt):
             tf.tf_force_plan("softmax", f"twopass:threads={threads},persist=0,regcap=0,stages={stages},u=4")
             run_case(dt, rows, nvec * ne, seed=nvec + threads)
         run_case(dt, 23, st * ne, seed=st, inplace=True)
+    # ... and the rings of the CTAs of a cluster: lengths that end in any CTA's steps, or before the first
+    for cluster, threads, stages in ((2, 128, 2), (4, 64, 4), (8, 32, 3), (2, 256, 1 + 1)):
+        cap = threads * 4 * cluster * stages
+        for nvec, rows in ((cap, 9), (cap - 1, 60), (threads * 4 * cluster + 1, 60), (cluster + 1, 9)):
+            rows = min(rows, max(3, (1 << 22) // (nvec * ne)))
+            tf.tf_force_plan("softmax", f"twopass:threads={threads},persist=0,regcap=0,cluster={cluster},stages={stages},u=4")
+            run_case(dt, rows, nvec * ne, seed=nvec + cluster)
     # a forced plan without a length mode (the cluster ring) falls back to the length-aware choice
     tf.tf_force_plan("softmax", "ring:threads=256,vpt=4,cluster=2,stages=2,persist=1")
     run_case(dt, 100, 2048 * ne)
