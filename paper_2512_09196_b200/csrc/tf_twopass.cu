@@ -161,7 +161,7 @@ constexpr int kRingMaxDepth = 8;
 // at the end of the row costs every CTA of the cluster the same); the partials meet between the passes through
 // distributed shared memory and one cluster barrier.  A row is then in flight for 1 / cs of the time, which keeps what lies
 // between the passes within L2, and each CTA's ring holds cs times as large a share of the row.
-template <int OP, int DT, int U, int MAXT, int MINB, bool CL>
+template <int OP, int DT, int U, int MAXT, int MINB, bool CL, bool LEN = false>
 __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
     constexpr int NE = Elem<DT>::NE, CH = U * 32;                        // vectors a warp takes per step
     __shared__ float red_buf[4 * 32];
@@ -177,23 +177,35 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
     const int nvec = static_cast<int>(a.nvec);
     const int step = a.step;                                             // vectors the CTA takes per step: warps x CH
     const int gstep = cs * step;                                         // distance in the row between two steps of this CTA
-    const int nfull = a.nfull;                                           // whole steps of the row
-    const int rag = a.rag;                                               // vectors of the row's ragged last step (0: there is none)
-    // the steps of CTA k: k, k + cs, ...; its last one is the ragged step iff that falls to it
-    auto steps_of = [&](int k) { const int n = nfull + (rag ? 1 : 0); return CL ? (n > k ? (n - k - 1) / cs + 1 : 0) : n; };
-    auto ragged_of = [&](int k) { return rag != 0 && (!CL || nfull % cs == k); };
-    auto count_of = [&](int k) { return static_cast<float>(((steps_of(k) - (ragged_of(k) ? 1 : 0)) * step + (ragged_of(k) ? rag : 0)) * NE); };
-    const int nsteps = steps_of(rank);                                   // this CTA's steps, numbered 0 .. nsteps-1 from here on
-    const bool has_rag = ragged_of(rank);
-    const int nwhole = nsteps - (has_rag ? 1 : 0);
+    // What a CTA needs to know about a row of `lv` vectors: whole steps of the row and vectors of its ragged last step; this
+    // CTA's steps (CTA k takes the steps k, k + cs, ...; its last one is the ragged step iff that falls to it), numbered
+    // 0 .. nsteps-1 from here on; pass A visits step s as its (nsteps-1-s)-th, so step 0 lives in ring slot (nsteps-1) mod S
+    // (two stages, the common case, without a division).  LEN: a row is as long as its length says.
+    struct Geo { int nfull, rag, nsteps, nwhole, slot0; bool has_rag; };
+    auto geo_of = [&](int nfull, int rag) {
+        Geo g;
+        g.nfull = nfull; g.rag = rag;
+        const int n = nfull + (rag ? 1 : 0);
+        g.nsteps = CL ? (n > rank ? (n - rank - 1) / cs + 1 : 0) : n;
+        g.has_rag = rag != 0 && (!CL || nfull % cs == rank);
+        g.nwhole = g.nsteps - (g.has_rag ? 1 : 0);
+        g.slot0 = g.nsteps > 0 ? (S == 2 ? ((g.nsteps - 1) & 1) : (g.nsteps - 1) % S) : 0;
+        return g;
+    };
+    const Geo g0 = geo_of(a.nfull, a.rag);
+    // elements CTA k holds of a full row (LayerNorm's merge of the CTAs' partial means)
+    auto count_of = [&](int k) {
+        const int n = a.nfull + (a.rag ? 1 : 0);
+        const int st = CL ? (n > k ? (n - k - 1) / cs + 1 : 0) : n;
+        const bool rg = a.rag != 0 && (!CL || a.nfull % cs == k);
+        return static_cast<float>(((st - (rg ? 1 : 0)) * step + (rg ? a.rag : 0)) * NE);
+    };
     const int toff = (t >> 5) * CH + (t & 31);                           // this thread's first vector within a step
     uint4* const myring = reinterpret_cast<uint4*>(dyn_smem) + toff;     // slot k of the ring: myring + k * step (+ u * 32)
     uint4* const ring_end = myring + S * step;
     const int64_t per_group = a.per_group;
     const uint4 fill = fill_vec<DT>(OP);
     const uint4 zero = make_uint4(0, 0, 0, 0);
-    // pass A visits step s as its (nsteps-1-s)-th: slot = that mod S (two stages, the common case, without a division)
-    const int slot_of_step0 = nsteps > 0 ? (S == 2 ? ((nsteps - 1) & 1) : (nsteps - 1) % S) : 0;
     if constexpr (CL) cg::this_cluster().sync();                         // every CTA of the cluster is resident before any remote write
     const int64_t first_slot = CL ? blockIdx.x / cs : blockIdx.x, slot_step = CL ? gridDim.x / cs : gridDim.x;
     int it = -1;
@@ -201,6 +213,15 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
         const int64_t row = a.groups > 1 ? (slot % a.groups) * per_group + slot / a.groups : slot;
         if (row >= a.rows) continue;                                     // the same decision in every CTA of a cluster
         ++it;
+        int straddle = -1, keep_el = 0;                                  // LEN: the vector the length ends in, and how much of it is live
+        int lv = nvec;                                                   // LEN: live vectors of this row
+        if constexpr (LEN) {
+            const int len = min(max(__ldg(a.len + row), 0), nvec * NE);
+            lv = (len + NE - 1) / NE;
+            keep_el = len % NE;
+            straddle = keep_el ? len / NE : -1;
+        }
+        const Geo g = LEN ? geo_of(lv / step, lv % step) : g0;
         const int64_t base = row * nvec + rank * step + toff;            // this thread's vectors of step s: base + s * gstep (+ u * 32)
         const uint4* const xr = a.x + base;
         uint4* const yr = a.y + base;
@@ -211,19 +232,19 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
         auto issue_ragged = [&](uint4* dst, uint64_t policy) {           // vectors behind the end of the row get the fill value
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (toff + u * 32 < rag) cp_async16(dst + u * 32, xr + nwhole * gstep + u * 32, policy);
+                if (toff + u * 32 < g.rag) cp_async16(dst + u * 32, xr + g.nwhole * gstep + u * 32, policy);
                 else dst[u * 32] = fill;
             }
         };
-        // ---- pass A, back to front: the k-th step visited is s = nsteps - 1 - k and lives in slot k mod S
+        // ---- pass A, back to front: the k-th step visited is s = g.nsteps - 1 - k and lives in slot k mod S
         Running<OP, DT, U> run;
         {
             int k_issue = 0;
             uint4* dst_i = myring;                                       // ring slot of the step issued next
-            const uint4* src_i = xr + (nsteps - 1) * gstep;
+            const uint4* src_i = xr + (g.nsteps - 1) * gstep;
             auto issue_next = [&]() {
-                if (k_issue < nsteps) {
-                    if (has_rag && k_issue == 0) issue_ragged(dst_i, keep);
+                if (k_issue < g.nsteps) {
+                    if (g.has_rag && k_issue == 0) issue_ragged(dst_i, keep);
                     else issue_full(src_i, dst_i, keep);
                 }
                 cp_async_commit();
@@ -232,7 +253,7 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
             };
             for (int j = 0; j < S - 1; ++j) issue_next();
             const uint4* cur = myring;                                   // ring slot of the step worked on
-            for (int k = 0; k < nsteps; ++k) {
+            for (int k = 0; k < g.nsteps; ++k) {
                 issue_next();
                 cp_async_wait(S - 1);
                 uint4 raw[U];
@@ -240,12 +261,18 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
                 for (int u = 0; u < U; ++u) raw[u] = cur[u * 32];
                 cur += step;
                 if (cur == ring_end) cur = myring;
-                const int s = nsteps - 1 - k;
-                if (has_rag && k == 0) {
+                const int s = g.nsteps - 1 - k;
+                if constexpr (LEN) {                                     // the vector the length ends in: its dead elements count as -inf
+                    const int v0 = (rank + s * cs) * step + toff;
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+                        if (v0 + u * 32 == straddle) raw[u] = mask_tail<DT>(raw[u], keep_el);
+                }
+                if (g.has_rag && k == 0) {
                     bool ok[U];
                     int count = 0;
 #pragma unroll
-                    for (int u = 0; u < U; ++u) { ok[u] = toff + u * 32 < rag; count += ok[u] ? NE : 0; }
+                    for (int u = 0; u < U; ++u) { ok[u] = toff + u * 32 < g.rag; count += ok[u] ? NE : 0; }
                     if (count > 0) run.template update<true>(raw, ok, count, s * U);
                 } else {
                     const bool all[U] = {};
@@ -289,9 +316,9 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
         // worked on, into the slot that step s - 1 has just left.  Softmax: from this thread's first step that holds
         // nothing but -inf on, zeros are written and x is not read again.
         const F2 ta2 = f2(sc.a), tb2 = f2(sc.b);
-        const int live_steps = OP == OP_SOFTMAX ? (run.live_slots + U - 1) / U : nsteps;
-        const int live_whole = min(live_steps, nwhole);
-        const uint4* cur = myring + slot_of_step0 * step;                // ring slot of step s: one slot down per step
+        const int live_steps = OP == OP_SOFTMAX ? (run.live_slots + U - 1) / U : g.nsteps;
+        const int live_whole = min(live_steps, g.nwhole);
+        const uint4* cur = myring + g.slot0 * step;                // ring slot of step s: one slot down per step
         const uint4* src_n = xr + S * gstep;                             // step s + S - 1 of x (s = 1 first)
         const uint4* gp = a.p0 + rank * step + toff;
         const uint4* bp = a.p1 + rank * step + toff;
@@ -303,7 +330,7 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
                 uint4* freed = const_cast<uint4*>(cur) + step;           // the slot step s - 1 has just left
                 if (freed == ring_end) freed = myring;
                 if (sn < live_steps) {
-                    if (sn < nwhole) issue_full(src_n, freed, last);
+                    if (sn < g.nwhole) issue_full(src_n, freed, last);
                     else issue_ragged(freed, last);
                 }
                 src_n += gstep;
@@ -311,28 +338,41 @@ __global__ void __launch_bounds__(MAXT, MINB) k_twopass_ring(const WArgs a) {
             cp_async_commit();
             cp_async_wait(S - 1);
 #pragma unroll
-            for (int u = 0; u < U; ++u) st_stream(dst + u * 32, apply_vec<OP, DT>(cur[u * 32], gp + u * 32, bp + u * 32, ta2, tb2));
+            for (int u = 0; u < U; ++u) {
+                uint4 raw = cur[u * 32];
+                if (LEN && (rank + s * cs) * step + toff + u * 32 == straddle) raw = mask_tail<DT>(raw, keep_el);
+                st_stream(dst + u * 32, apply_vec<OP, DT>(raw, gp + u * 32, bp + u * 32, ta2, tb2));
+            }
             cur = (cur == myring ? ring_end : cur) - step;
             dst += gstep; gp += gstep; bp += gstep;
         }
-        if (has_rag && s == nwhole && s < live_steps) {                  // the ragged step is live
+        if (g.has_rag && s == g.nwhole && s < live_steps) {                  // the ragged step is live
             cp_async_commit();
             cp_async_wait(0);
 #pragma unroll
-            for (int u = 0; u < U; ++u)
-                if (toff + u * 32 < rag) st_stream(dst + u * 32, apply_vec<OP, DT>(cur[u * 32], gp + u * 32, bp + u * 32, ta2, tb2));
+            for (int u = 0; u < U; ++u) {
+                if (toff + u * 32 < g.rag) {
+                    uint4 raw = cur[u * 32];
+                    if (LEN && (rank + s * cs) * step + toff + u * 32 == straddle) raw = mask_tail<DT>(raw, keep_el);
+                    st_stream(dst + u * 32, apply_vec<OP, DT>(raw, gp + u * 32, bp + u * 32, ta2, tb2));
+                }
+            }
             ++s;
         }
-        for (; s < nwhole; ++s) {
+        for (; s < g.nwhole; ++s) {
 #pragma unroll
             for (int u = 0; u < U; ++u) st_stream(yr + s * gstep + u * 32, zero);
         }
-        if (has_rag && s == nwhole) {
+        if (g.has_rag && s == g.nwhole) {
 #pragma unroll
             for (int u = 0; u < U; ++u)
-                if (toff + u * 32 < rag) st_stream(yr + s * gstep + u * 32, zero);
+                if (toff + u * 32 < g.rag) st_stream(yr + s * gstep + u * 32, zero);
         }
         cp_async_wait(0);
+        if constexpr (LEN) {                                             // +0 behind the length, shared by the CTAs of the row
+            uint4* const y_row = a.y + row * nvec;
+            for (int i = lv + rank * static_cast<int>(blockDim.x) + t; i < nvec; i += cs * static_cast<int>(blockDim.x)) st_stream(y_row + i, zero);
+        }
     }
 }
 
@@ -556,6 +596,15 @@ TwoFn ring_fn_c(int op, int dt) {
 }
 template <int U, int MAXT, int MINB>
 TwoFn ring_fn_b(int op, int dt, bool cl) { return cl ? ring_fn_c<U, MAXT, MINB, true>(op, dt) : ring_fn_c<U, MAXT, MINB, false>(op, dt); }
+// softmax with per-row lengths in the general ring form
+TwoFn ring_len_fn(int dt, int threads, bool capped, bool cl) {
+    if (capped && threads <= 384) {
+        if (cl) return dt == DT_F32 ? k_twopass_ring<OP_SOFTMAX, DT_F32, 4, 384, 3, true, true> : k_twopass_ring<OP_SOFTMAX, DT_BF16, 4, 384, 3, true, true>;
+        return dt == DT_F32 ? k_twopass_ring<OP_SOFTMAX, DT_F32, 4, 384, 3, false, true> : k_twopass_ring<OP_SOFTMAX, DT_BF16, 4, 384, 3, false, true>;
+    }
+    if (cl) return dt == DT_F32 ? k_twopass_ring<OP_SOFTMAX, DT_F32, 4, 1024, 1, true, true> : k_twopass_ring<OP_SOFTMAX, DT_BF16, 4, 1024, 1, true, true>;
+    return dt == DT_F32 ? k_twopass_ring<OP_SOFTMAX, DT_F32, 4, 1024, 1, false, true> : k_twopass_ring<OP_SOFTMAX, DT_BF16, 4, 1024, 1, false, true>;
+}
 // regcap: the builds whose registers are held to what three CTAs per SM leave each thread: 56 for CTAs of up to 384
 // threads, 40 for CTAs of up to 512
 TwoFn ring_fn(int op, int dt, int unroll, int threads, bool capped, bool cl) {
@@ -578,8 +627,9 @@ bool supports_twopass(const Plan& p, const Args& a, const DeviceInfo& d) {
         const int64_t nvec = a.cols * elem_size(a.dt) / 16;
         if (a.len) {                                               // lengths: softmax rows that fit the ring of one CTA
             const int64_t step = static_cast<int64_t>(p.threads / 32) * p.unroll * 32;
-            if (a.op != OP_SOFTMAX || p.lanes != 1 || p.persist != 0 || p.unroll != 4 || p.rpg != 1 ||
-                ((nvec + step - 1) / step + p.cluster - 1) / p.cluster > std::min(p.stages, 4) || a.rows * p.cluster > 0x7FFFFFFF) return false;
+            const bool fits = p.persist == 0 && p.rpg == 1 && ((nvec + step - 1) / step + p.cluster - 1) / p.cluster <= std::min(p.stages, 4);
+            if (a.op != OP_SOFTMAX || p.lanes != 1 || p.unroll != 4 || a.rows * p.cluster > 0x7FFFFFFF) return false;
+            if (!fits && p.rpg == 2 && p.threads > 384) return false;      // the general ring form: its 56-register build ends at 384 threads
         }
         if (nvec > 0x7FFFFFFF - 65536) return false;              // 32-bit vector indices inside the kernel
         return vector_ok(a) && (p.rpg == 1 || p.rpg == 2) && p.threads >= 32 && p.threads <= 1024 && p.threads % 32 == 0 &&
@@ -607,7 +657,8 @@ cudaError_t launch_twopass(const Plan& p, const Args& a, const DeviceInfo& d, cu
             fn = a.len ? (a.op == OP_SOFTMAX ? fit_len_fn(a.dt, fit_steps, cs > 1) : nullptr) : fit_fn(a.op, a.dt, fit_steps, steps * step * cs == nvec, cs > 1);
         }
     }
-    if (ring && a.len && !fit_steps) fn = nullptr;                 // the ring form knows lengths only where the row fits the ring
+    if (ring && a.len && !fit_steps)                               // lengths in the general ring form: softmax, four vectors per step
+        fn = (a.op == OP_SOFTMAX && p.unroll == 4 && groups == 1) ? ring_len_fn(a.dt, p.threads, p.rpg == 2, cs > 1) : nullptr;
     if (!fn) return cudaErrorInvalidValue;
     const int64_t slots = (a.rows + groups - 1) / groups * groups;
     int64_t grid = slots;                                          // in rows (clusters)

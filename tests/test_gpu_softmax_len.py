@@ -119,6 +119,15 @@ def test_forced_plans_and_bitwise_equality_with_the_masked_plain_softmax(dt):
             rows = min(rows, max(3, (1 << 22) // (nvec * ne)))
             tf.tf_force_plan("softmax", f"twopass:threads={threads},persist=0,regcap=0,cluster={cluster},stages={stages},u=4")
             run_case(dt, rows, nvec * ne, seed=nvec + cluster)
+    # the general ring form (rows longer than the ring): lengths that end in a whole step, a ragged one, the first step, nowhere
+    # (length 0), with and without a cluster, persistent grids, both register builds
+    for cluster, threads, stages, persist, regcap in ((1, 64, 2, 0, 0), (1, 256, 3, 0, 1), (2, 128, 2, 0, 1), (4, 64, 4, 0, 0), (8, 32, 2, 1, 0), (2, 384, 3, 2, 1)):
+        st = threads * 4
+        for nvec, rows in ((st * cluster * stages + 1, 60), (st * (cluster * stages + 3) + 5, 60), (st * cluster * 9, 33), (70001, 9)):
+            rows = min(rows, max(3, (1 << 22) // (nvec * ne)))
+            tf.tf_force_plan("softmax", f"twopass:threads={threads},persist={persist},regcap={regcap},cluster={cluster},stages={stages},u=4")
+            run_case(dt, rows, nvec * ne, seed=nvec + cluster)
+        run_case(dt, 11, (st * cluster * stages * 2 + 7) * ne, seed=st, inplace=True, x_std=20.0)
     # a forced plan without a length mode (the cluster ring) falls back to the length-aware choice
     tf.tf_force_plan("softmax", "ring:threads=256,vpt=4,cluster=2,stages=2,persist=1")
     run_case(dt, 100, 2048 * ne)
