@@ -188,35 +188,81 @@ __global__ void __launch_bounds__(512) k_norm_bwd(const BArgs a, const int gt) {
 // gives up sets the status word, stops issuing copies and finishes its loop without waiting again.
 constexpr int kBwdMaxStages = 8;
 
+// The two row sums of a group of wg warps with half the shuffles of two separate reductions: after the first exchange
+// the even lanes carry the first sum and the odd lanes the second, each over its lane pair, and the remaining steps keep
+// that parity.  Per-warp partials meet in `red` (2 * warps floats: first and second sum of warp w at 2w and 2w + 1;
+// RMSNorm has one sum, at w); after a barrier the partials of a power-of-two number of warps are added as a butterfly, so
+// every thread of the group gets the same bits.
+template <bool RMS>
+__device__ __forceinline__ void warp_sums_store(float sgx, float sg, float* red, int warp, int lane) {
+    constexpr unsigned kAll = 0xFFFFFFFFu;
+    if constexpr (RMS) {
+        sgx = group_reduce<SumOp, 32>(sgx);
+        if (lane == 0) red[warp] = sgx;
+    } else {
+        const bool odd = lane & 1;
+        float v = (odd ? sg : sgx) + __shfl_xor_sync(kAll, odd ? sgx : sg, 1);
+#pragma unroll
+        for (int o = 2; o < 32; o <<= 1) v += __shfl_xor_sync(kAll, v, o);
+        if (lane < 2) red[2 * warp + lane] = v;
+    }
+}
+template <bool RMS>
+__device__ __forceinline__ void group_sums_load(float& sgx, float& sg, const float* red, int wg, int gid, int lane) {
+    constexpr unsigned kAll = 0xFFFFFFFFu;
+    if constexpr (RMS) {
+        if ((wg & (wg - 1)) == 0) {
+            sgx = red[gid * wg + (lane & (wg - 1))];
+            for (int o = wg >> 1; o > 0; o >>= 1) sgx += __shfl_xor_sync(kAll, sgx, o);
+        } else {
+            sgx = 0.f;
+            for (int w = 0; w < wg; ++w) sgx += red[gid * wg + w];
+        }
+        sg = 0.f;
+    } else {
+        const bool odd = lane & 1;
+        float v;
+        if ((wg & (wg - 1)) == 0) {
+            v = red[2 * gid * wg + (lane & (2 * wg - 1))];
+            for (int o = wg; o > 1; o >>= 1) v += __shfl_xor_sync(kAll, v, o);
+        } else {
+            v = 0.f;
+            for (int w = 0; w < wg; ++w) v += red[2 * (gid * wg + w) + (odd ? 1 : 0)];
+        }
+        const float u = __shfl_xor_sync(kAll, v, 1);
+        sgx = odd ? u : v;
+        sg = odd ? v : u;
+    }
+}
+
 template <bool RMS, int DT, int VPT, bool FULL>
 __global__ void __launch_bounds__(512) k_norm_bwd_staged(const BArgs a, const int gt, const int S, int* status) {
     using P = Pairs<DT>;
     constexpr int NE = Elem<DT>::NE, NP = P::NP;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ __align__(8) uint64_t full[kBwdMaxStages];
-    __shared__ float2 red[2][16];
-    const int t = threadIdx.x, gid = t / gt, lg = t % gt, R = blockDim.x / gt, wg = gt / 32;
+    __shared__ float red[2][32];
+    const int t = threadIdx.x, gid = t / gt, lg = t - gid * gt, R = blockDim.x / gt, wg = gt >> 5;
     const int warp = t >> 5, lane = t & 31;
-    const size_t tile_vecs = static_cast<size_t>(R) * a.nvec;                 // vectors of x (and of dy) per stage
+    const uint32_t tile_vecs = static_cast<uint32_t>(R) * a.nvec;             // vectors of x (and of dy) per stage
     uint4* const ring = reinterpret_cast<uint4*>(dyn_smem);                    // [S][x | dy][R][nvec]
     const int64_t num_tiles = (a.rows + R - 1) / R;
+    // this CTA's tiles: blockIdx.x, + gridDim.x, ...; the loop below counts them instead of comparing 64-bit row numbers
+    const int n_iters = blockIdx.x < num_tiles ? static_cast<int>((num_tiles - 1 - blockIdx.x) / gridDim.x) + 1 : 0;
     if (t == 0) {
         for (int s = 0; s < S; ++s) mbar_init(&full[s], 1);
         mbar_fence_init();
     }
     pdl_wait();
-    auto issue = [&](int64_t tile, int s) {                                    // thread 0 only
-        const int64_t row0 = tile * R;
+    auto issue = [&](int k, int s) {                                           // thread 0 only: this CTA's k-th tile into stage s
+        const int64_t row0 = (blockIdx.x + static_cast<int64_t>(k) * gridDim.x) * R;
         const uint32_t bytes = static_cast<uint32_t>(min(static_cast<int64_t>(R), a.rows - row0)) * a.nvec * 16u;
         mbar_expect_tx(&full[s], 2u * bytes);
         bulk_g2s(ring + tile_vecs * (2 * s), a.x + row0 * a.nvec, bytes, &full[s]);
         bulk_g2s(ring + tile_vecs * (2 * s + 1), a.dy + row0 * a.nvec, bytes, &full[s]);
     };
     if (t == 0)
-        for (int s = 0; s < S; ++s) {
-            const int64_t tile = blockIdx.x + static_cast<int64_t>(s) * gridDim.x;
-            if (tile < num_tiles) issue(tile, s);
-        }
+        for (int s = 0; s < S && s < n_iters; ++s) issue(s, s);
     bool valid[VPT];
     F2 gam[VPT][NP], accg[VPT][NP], accb[RMS ? 1 : VPT][NP];
 #pragma unroll
@@ -229,32 +275,31 @@ __global__ void __launch_bounds__(512) k_norm_bwd_staged(const BArgs a, const in
     __syncthreads();                                                           // barriers initialised
     pdl_trigger();
     bool failed = false;
-    int it = 0, s = 0;
-    uint32_t parity = 0;
+    int s = 0;
+    uint32_t parity = 0, stage_vecs = 0;                                       // stage s starts at vector 2 s tile_vecs of the ring
+    // everything that moves with the row advances by one stride per iteration: the row number, the statistics, dx
+    int64_t row = static_cast<int64_t>(blockIdx.x) * R + gid;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * R;
+    const float* pmean = RMS ? nullptr : a.mean + row;
+    const float* prstd = a.rstd + row;
+    uint4* o = a.dx + row * a.nvec + lg;
+    const int64_t ostride = stride * a.nvec;
+    const uint32_t mine = static_cast<uint32_t>(gid) * a.nvec + lg;
     float nmu = 0.f, nrs = 0.f;                                                // the statistics of a row are requested one tile ahead
-    auto request_stats = [&](int64_t tile) {
-        const int64_t row = tile * R + gid;
-        const bool in = tile < num_tiles && row < a.rows;
-        if (FULL) {
-            if (in) { nmu = RMS ? 0.f : __ldg(a.mean + row); nrs = __ldg(a.rstd + row); }
-            return;
-        }
-        nmu = (RMS || !in) ? 0.f : __ldg(a.mean + row);
-        nrs = in ? __ldg(a.rstd + row) : 0.f;
-    };
-    request_stats(blockIdx.x);
-    for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {       // same trip count for the whole CTA
+    if (n_iters > 0 && (FULL || row < a.rows)) { nmu = RMS ? 0.f : __ldg(pmean); nrs = __ldg(prstd); }
+    for (int it = 0; it < n_iters; ++it) {                                     // same trip count for the whole CTA
         if (!failed && !mbar_wait(&full[s], parity)) {
             failed = true;
             atomicExch(status, 4);
             mbar_wait(&full[s], parity);                                       // one more bounded wait for the copies
         }
-        const int64_t row = tile * R + gid;
         const bool live = FULL || row < a.rows;
         const float rs = nrs;
         const F2 mu2 = f2(nmu), rs2 = f2(rs);
-        request_stats(tile + gridDim.x);
-        const uint4* sx = ring + tile_vecs * (2 * s) + static_cast<size_t>(gid) * a.nvec + lg;
+        prstd += stride;
+        if (!RMS) pmean += stride;
+        if (it + 1 < n_iters && (FULL || row + stride < a.rows)) { nmu = RMS ? 0.f : __ldg(pmean); nrs = __ldg(prstd); }
+        const uint4* sx = ring + stage_vecs + mine;
         const uint4* sd = sx + tile_vecs;
         F2 xh[VPT][NP], g[VPT][NP], dv[VPT][NP];
         F2 sgx2 = f2(0.f), sg2 = f2(0.f);
@@ -269,22 +314,19 @@ __global__ void __launch_bounds__(512) k_norm_bwd_staged(const BArgs a, const in
                 xh[v][i] = ok ? mul2(sub2(xv[i], mu2), rs2) : f2(0.f);
                 g[v][i] = mul2(dv[v][i], gam[v][i]);
                 sgx2 = fma2(g[v][i], xh[v][i], sgx2);
-                sg2 = add2(sg2, g[v][i]);
+                if (!RMS) sg2 = add2(sg2, g[v][i]);
                 accg[v][i] = fma2(dv[v][i], xh[v][i], accg[v][i]);
                 if (!RMS) accb[v][i] = add2(accb[v][i], dv[v][i]);
             }
         }
-        float sgx = group_reduce<SumOp, 32>(hsum(sgx2));
-        float sg = group_reduce<SumOp, 32>(hsum(sg2));
-        if (lane == 0) red[it & 1][warp] = make_float2(sgx, sg);
+        float sgx = hsum(sgx2), sg = RMS ? 0.f : hsum(sg2);
+        warp_sums_store<RMS>(sgx, sg, red[it & 1], warp, lane);
         __syncthreads();                                                       // also: every thread has left the stage
-        const int64_t next = tile + static_cast<int64_t>(S) * gridDim.x;
-        if (t == 0 && !failed && next < num_tiles) issue(next, s);
-        if (wg > 1) group_total(red[it & 1] + gid * wg, wg, lane, sgx, sg);
+        if (t == 0 && !failed && it + S < n_iters) issue(it + S, s);
+        group_sums_load<RMS>(sgx, sg, red[it & 1], wg, gid, lane);
         // dx = rstd g - rstd mean(g) - xh rstd mean(g xh): two fused multiply-adds per pair
         const F2 c1 = f2(-rs * (sgx * a.inv_n)), c0 = f2(RMS ? 0.f : -rs * (sg * a.inv_n));
         if (live) {
-            uint4* o = a.dx + row * a.nvec + lg;
 #pragma unroll
             for (int v = 0; v < VPT; ++v) {
                 F2 d[NP];
@@ -293,7 +335,10 @@ __global__ void __launch_bounds__(512) k_norm_bwd_staged(const BArgs a, const in
                 if (valid[v]) st_stream(o + v * gt, P::pack(d));
             }
         }
-        if (++s == S) { s = 0; parity ^= 1u; }
+        row += stride;
+        o += ostride;
+        stage_vecs += 2 * tile_vecs;
+        if (++s == S) { s = 0; parity ^= 1u; stage_vecs = 0; }
     }
     float* pg = a.part + (static_cast<int64_t>(blockIdx.x) * R + gid) * (RMS ? 1 : 2) * a.nvec * NE;
 #pragma unroll
@@ -523,37 +568,64 @@ __global__ void __launch_bounds__(1024) k_norm_bwd_stream(const BArgs a) {
         }
 }
 
-// Adds the `nparts` partial column sums and rounds once.  A CTA of 32 x 8 threads owns 32 columns: thread (c, y) adds
-// parts y, y + 8, ... of column c, the eight slice sums meet in shared memory and are added in slice order -- a fixed
-// order of additions whatever the launch, hence deterministic -- and 128 CTAs instead of 16 share the reading.
-template <bool RMS, int DT>
-__global__ void __launch_bounds__(256) k_colsum_finish(const float* __restrict__ part, typename Elem<DT>::scalar* dgamma,
-                                                       typename Elem<DT>::scalar* dbeta, int nparts, int64_t cols) {
+// Adds the `nparts` partial column sums and rounds once.  A part is one row of [dgamma | dbeta] partials (RMSNorm: the
+// first alone), `width` floats; a CTA of 32 x ny threads owns 32 V consecutive positions: thread (c, y) adds parts y,
+// y + ny, ... of its V positions on four independent accumulators (four reads in flight per thread: the reads, from L2,
+// are what the kernel waits for -- a thread per column that walked its parts one after the other took 11-33 us on the
+// training shapes, a sixth to a third of the whole call), the ny slice sums meet in shared memory and are added in slice
+// order.  The order of the additions is fixed whatever the launch, hence deterministic.  V = 4 (16-byte reads; width a
+// multiple of 4, so a thread's positions never straddle the two halves) is for parts wide enough to fill the GPU that
+// way; ny (8, 16 or 32) follows the number of parts.
+template <int V> struct FinishVec;
+template <> struct FinishVec<1> {
+    static __device__ __forceinline__ void add(float (&a)[1], const float* p) { a[0] += *p; }
+};
+template <> struct FinishVec<4> {
+    static __device__ __forceinline__ void add(float (&a)[4], const float* p) {
+        const float4 v = *reinterpret_cast<const float4*>(p);
+        a[0] += v.x; a[1] += v.y; a[2] += v.z; a[3] += v.w;
+    }
+};
+template <bool RMS, int DT, int V>
+__global__ void __launch_bounds__(1024) k_colsum_finish(const float* __restrict__ part, typename Elem<DT>::scalar* dgamma,
+                                                        typename Elem<DT>::scalar* dbeta, int nparts, int64_t cols) {
     using E = Elem<DT>;
-    __shared__ float sm[2][8][32];
+    __shared__ float sm[32][32 * V + 1];
     pdl_wait();
-    const int c = threadIdx.x & 31, y = threadIdx.x >> 5;
-    const int64_t j = static_cast<int64_t>(blockIdx.x) * 32 + c;
-    const int64_t stride = (RMS ? 1 : 2) * cols;
-    float sg = 0.f, sb = 0.f;
-    if (j < cols)
-        for (int p = y; p < nparts; p += 8) {
-            sg += part[p * stride + j];
-            if (!RMS) sb += part[p * stride + cols + j];
-        }
-    sm[0][y][c] = sg;
-    sm[1][y][c] = sb;
-    __syncthreads();
-    if (y == 0 && j < cols) {
-        float tg = 0.f, tb = 0.f;
+    const int c = threadIdx.x & 31, y = threadIdx.x >> 5, ny = blockDim.x >> 5;
+    const int64_t width = (RMS ? 1 : 2) * cols;
+    const int64_t j0 = (static_cast<int64_t>(blockIdx.x) * 32 + c) * V;
+    float acc[4][V];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { tg += sm[0][k][c]; tb += sm[1][k][c]; }
-        dgamma[j] = E::from_float(tg);
-        if (!RMS) dbeta[j] = E::from_float(tb);
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < V; ++v) acc[u][v] = 0.f;
+    if (j0 < width) {
+        const int64_t step = ny * width;
+        const float* p = part + y * width + j0;
+        int k = y;
+        for (; k + 3 * ny < nparts; k += 4 * ny, p += 4 * step) {
+            FinishVec<V>::add(acc[0], p);
+            FinishVec<V>::add(acc[1], p + step);
+            FinishVec<V>::add(acc[2], p + 2 * step);
+            FinishVec<V>::add(acc[3], p + 3 * step);
+        }
+        if (k < nparts) FinishVec<V>::add(acc[0], p);
+        if (k + ny < nparts) FinishVec<V>::add(acc[1], p + step);
+        if (k + 2 * ny < nparts) FinishVec<V>::add(acc[2], p + 2 * step);
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) sm[y][c * V + v] = (acc[0][v] + acc[1][v]) + (acc[2][v] + acc[3][v]);
+    __syncthreads();
+    const int64_t j = static_cast<int64_t>(blockIdx.x) * 32 * V + threadIdx.x;          // one position per thread of the first 32 V
+    if (threadIdx.x < 32 * V && j < width) {
+        float t = 0.f;
+        for (int k = 0; k < ny; ++k) t += sm[k][threadIdx.x];
+        if (j < cols) dgamma[j] = E::from_float(t);
+        else dbeta[j - cols] = E::from_float(t);
     }
 }
 
-// ---- any shape, any alignment ------------------------------------------------------------------------------------
 template <bool RMS, int DT>
 __global__ void __launch_bounds__(256) k_norm_bwd_dx_scalar(const typename Elem<DT>::scalar* x, const typename Elem<DT>::scalar* gamma,
                                                             const typename Elem<DT>::scalar* dy, const float* mean, const float* rstd,
@@ -619,6 +691,19 @@ cudaError_t launch_pdl(void (*fn)(T...), int64_t grid, int threads, cudaStream_t
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, fn, args...);
+}
+
+template <bool RMS, int DT>
+cudaError_t launch_finish(const void* ws, void* dgamma, void* dbeta, int nparts, int64_t cols, cudaStream_t st) {
+    using S = typename Elem<DT>::scalar;
+    const int64_t width = (RMS ? 1 : 2) * cols;
+    const int ny = nparts >= 256 ? 32 : nparts >= 128 ? 16 : 8;
+    const bool wide = width % 4 == 0 && width >= static_cast<int64_t>(256) * sm_count();       // two CTAs of 128 positions per SM and more
+    if (wide)
+        return launch_pdl(k_colsum_finish<RMS, DT, 4>, (width + 127) / 128, 32 * ny, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
+                          static_cast<S*>(dbeta), nparts, cols);
+    return launch_pdl(k_colsum_finish<RMS, DT, 1>, (width + 31) / 32, 32 * ny, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
+                      static_cast<S*>(dbeta), nparts, cols);
 }
 
 // Test and bench hook: 0 = automatic, 1 = the register form, 2 = the staged form with row groups of up to 512 threads,
@@ -818,8 +903,7 @@ tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float*
         count_launches(2);
         e = launch_cluster<RMS, DT>(cp, a, status, st);
         if (e == cudaSuccess)
-            e = launch_pdl(k_colsum_finish<RMS, DT>, (cols + 31) / 32, 256, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
-                           static_cast<S*>(dbeta), cp.clusters, cols);
+            e = launch_finish<RMS, DT>(ws, dgamma, dbeta, cp.clusters, cols, st);
     } else if (aligned && bytes / 16 <= 512 * kMaxVpt && cols <= 0x7FFFFFFF) {
         const int nvec = static_cast<int>(bytes / 16);
         const BwdPlan p = choose_bwd_plan<RMS, DT>(rows, nvec, c);
@@ -858,8 +942,7 @@ tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float*
         else if (p.vpt == 2) e = launch_pdl(k_norm_bwd<RMS, DT, 2, false>, p.grid, threads, st, a, p.gt);
         else e = launch_pdl(k_norm_bwd<RMS, DT, kMaxVpt, false>, p.grid, threads, st, a, p.gt);
         if (e == cudaSuccess)
-            e = launch_pdl(k_colsum_finish<RMS, DT>, (cols + 31) / 32, 256, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
-                           static_cast<S*>(dbeta), parts, cols);
+            e = launch_finish<RMS, DT>(ws, dgamma, dbeta, parts, cols, st);
     } else if (aligned && cols <= 0x7FFFFFFF && static_cast<size_t>(RMS ? 1 : 2) * cols * 4 <= 200 * 1024) {
         const int nvec = static_cast<int>(bytes / 16);
         const int grid = static_cast<int>(std::min<int64_t>(rows, sm_count()));          // one CTA per SM: the accumulators fill shared memory
@@ -878,8 +961,7 @@ tf_status run_bwd(const void* x, const void* gamma, const void* dy, const float*
             cfg.stream = st;
             e = cudaLaunchKernelEx(&cfg, k_norm_bwd_stream<RMS, DT>, a);
             if (e == cudaSuccess)
-                e = launch_pdl(k_colsum_finish<RMS, DT>, (cols + 31) / 32, 256, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
-                               static_cast<S*>(dbeta), grid, cols);
+                e = launch_finish<RMS, DT>(ws, dgamma, dbeta, grid, cols, st);
         }
     } else {
         if (rows > 0x7FFFFFFF) return TF_ERR_UNSUPPORTED;
