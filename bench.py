@@ -1134,6 +1134,25 @@ def run_case(args):
         nbytes = 3 * rows * cols * inputs.ELEM_SIZE[dt]
         print(json.dumps({"case": f"case_{op}_bwd_{dts}_{rows}x{cols}", "launches": args.steps, "us_per_launch": us, "gbs": nbytes / us / 1e3}))
         return
+    if parts[0] == "sine":                    # sine:dtype:elements[:threads:vectors] -- the element-wise sine, inputs as in the sine table
+        dts, n = parts[1], int(parts[2])
+        threads, vectors = (int(parts[3]), int(parts[4])) if len(parts) > 4 else (0, 0)
+        tdt = torch.float32 if dts == "f32" else torch.bfloat16
+        gen = torch.Generator(device="cuda").manual_seed(n)
+        x = (torch.rand(n, device="cuda", generator=gen) * 200.0 - 100.0).to(tdt)
+        y = torch.empty_like(x)
+        a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(max(1, args.warmup)):
+            tf.tf_sin_fwd(x, y, threads, vectors)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(args.steps):
+            tf.tf_sin_fwd(x, y, threads, vectors)
+        e.record()
+        torch.cuda.synchronize()
+        us = 1e3 * a.elapsed_time(e) / args.steps
+        print(json.dumps({"case": f"case_sin_{dts}_{n}", "launches": args.steps, "us_per_launch": us, "gbs": 2 * n * x.element_size() / us / 1e3}))
+        return
     if parts[0] == "addnorm":                 # addnorm:op:dtype:rows:cols -- the fused residual add + norm, heuristic plan
         op, dts, rows, cols = parts[1], parts[2], int(parts[3]), int(parts[4])
         dt = inputs.F32 if dts == "f32" else inputs.BF16
@@ -1201,7 +1220,7 @@ def main():
     ap.add_argument("--sweep-tune", action="store_true", help="default run: tune every sweep point before timing it")
     ap.add_argument("--no-tune", action="store_true")
     ap.add_argument("--cpu", action="store_true", help="with --table: also time the oracle")
-    ap.add_argument("--case", default=None, help="op:dtype:rows:cols, config:<i>[:rows], vecmat:..., addnorm:op:dtype:rows:cols, normbwd:op:dtype:rows:cols, softmaxlen:dtype:rows:cols -- a few launches of one shape")
+    ap.add_argument("--case", default=None, help="op:dtype:rows:cols, config:<i>[:rows], vecmat:..., addnorm:op:dtype:rows:cols, normbwd:op:dtype:rows:cols, softmaxlen:dtype:rows:cols, sine:dtype:elements[:threads:vectors] -- a few launches of one shape")
     ap.add_argument("--plan", default=None, help="with --case: force this launch plan")
     args = ap.parse_args()
     if args.impl == "reference":
