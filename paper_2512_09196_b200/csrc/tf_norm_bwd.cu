@@ -698,7 +698,8 @@ cudaError_t launch_finish(const void* ws, void* dgamma, void* dbeta, int nparts,
     using S = typename Elem<DT>::scalar;
     const int64_t width = (RMS ? 1 : 2) * cols;
     const int ny = nparts >= 256 ? 32 : nparts >= 128 ? 16 : 8;
-    const bool wide = width % 4 == 0 && width >= static_cast<int64_t>(256) * sm_count();       // two CTAs of 128 positions per SM and more
+    // 16-byte reads: a workspace aligned for them, parts that keep the alignment, and two CTAs of 128 positions per SM and more
+    const bool wide = (reinterpret_cast<uintptr_t>(ws) & 15u) == 0 && width % 4 == 0 && width >= static_cast<int64_t>(256) * sm_count();
     if (wide)
         return launch_pdl(k_colsum_finish<RMS, DT, 4>, (width + 127) / 128, 32 * ny, st, static_cast<const float*>(ws), static_cast<S*>(dgamma),
                           static_cast<S*>(dbeta), nparts, cols);

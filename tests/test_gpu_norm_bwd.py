@@ -157,6 +157,28 @@ def test_deterministic_and_bad_arguments():
     assert L.tf_rmsnorm_bwd(p, p, p, p, p, p, p, 1 << 20, 4, 0, 0, None) == 1
 
 
+def test_workspace_needs_only_4_byte_alignment():
+    """Wide parts are added with 16-byte reads when the workspace allows them: a workspace that is only 4-byte aligned gives
+    the same bits (same order of additions) through the 4-byte reads."""
+    rows, cols = 40, 32768
+    x = torch.randn(rows, cols, device="cuda", dtype=torch.bfloat16)
+    dy = torch.randn_like(x)
+    g = (torch.rand(cols, device="cuda") + 0.5).to(torch.bfloat16)
+    _, mean, rstd = tf.tf_layernorm_fwd(x, g, torch.zeros_like(g), 1e-5)
+    dx0, dg0, db0 = tf.tf_layernorm_bwd(x, g, dy, mean, rstd)
+    L = tf.lib()
+    n = L.tf_norm_bwd_workspace_bytes(rows, cols)
+    ws = torch.empty(n // 4 + 8, dtype=torch.float32, device="cuda")
+    dx, dg, db = torch.empty_like(x), torch.empty_like(g), torch.empty_like(g)
+    st = L.tf_layernorm_bwd(x.data_ptr(), g.data_ptr(), dy.data_ptr(), mean.data_ptr(), rstd.data_ptr(), dx.data_ptr(), dg.data_ptr(),
+                            db.data_ptr(), ws.data_ptr() + 4, n, rows, cols, BF16, torch.cuda.current_stream().cuda_stream)
+    assert st == 0
+    torch.cuda.synchronize()
+    tf.tf_device_status()
+    for a, b in ((dx0, dx), (dg0, dg), (db0, db)):
+        assert torch.equal(a.view(torch.uint16), b.view(torch.uint16))
+
+
 @pytest.mark.parametrize("rms,dt,rows,cols", [(True, BF16, 16384, 4096), (True, BF16, 16384, 8192), (True, F32, 16384, 4096), (False, BF16, 16384, 4096),
                                               (False, BF16, 65536, 1024), (False, F32, 8192, 8192), (False, BF16, 4096, 16384), (False, F32, 4096, 16384),
                                               (False, BF16, 2048, 32768)])
