@@ -461,7 +461,7 @@ __device__ __forceinline__ void lsm_cp_async16(uint4* dst, const uint4* src) {
 template <int N> __device__ __forceinline__ void lsm_cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 template <int DT, int NS, bool FULL>
-__global__ void __launch_bounds__(256, 4) k_logsoftmax_smem(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t rows, int nvec) {
+__global__ void __launch_bounds__(256, 4) k_logsoftmax_smem(const uint4* x, uint4* y, int64_t rows, int nvec) {
     using E = Elem<DT>;
     constexpr int NE = E::NE, U = 4;
     __shared__ float buf[2][32];
