@@ -880,11 +880,12 @@ def run_sine_table(args):
                 best = us if best is None else min(best, us)
             return best
 
+        us_default = timed(lambda k: tf.tf_sin_fwd(xs[k], ys[k]))
         grid = {}
         for threads in (32, 64, 128, 256, 512, 1024):
             for vpt in (1, 2, 4, 8):
                 grid[(threads, vpt)] = timed(lambda k: tf.tf_sin_fwd(xs[k], ys[k], threads, vpt))
-        us_default = timed(lambda k: tf.tf_sin_fwd(xs[k], ys[k]))
+        us_default = min(us_default, timed(lambda k: tf.tf_sin_fwd(xs[k], ys[k])))      # before and after the grid, like every entry the best region
         us_torch = timed(lambda k: torch.sin(xs[k], out=ys[k]))
         us_copy = timed(lambda k: tf.tf_copy(xs[k], ys[k]))
         tf.tf_device_status()

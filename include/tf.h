@@ -128,7 +128,7 @@ tf_status tf_copy(const void* x, void* y, int64_t bytes, void* cuda_stream);
 /* y[i] = sin(x[i]) over n elements: the element-wise kernel of the paper's Case Study 1, whose only tuning knob is
  * its launch geometry (the paper's baseline used blocks of 4 elements; the fix was an autotune over block sizes).
  * threads per CTA (multiple of 32, <= 1024) and 16-byte vectors per thread (1, 2, 4 or 8) are that knob here -- a
- * CTA covers threads x vectors_per_thread vectors, its "block size"; 0 selects the defaults (128 threads, 4 vectors
+ * CTA covers threads x vectors_per_thread vectors, its "block size"; 0 selects the defaults (64 threads, 4 vectors
  * per thread).
  * fp32 arithmetic with full range reduction, one rounding to the storage type (2-byte elements below 2^15 in
  * magnitude take a shorter fp32 evaluation whose rounded results are the same).  y == x is allowed. */

@@ -163,8 +163,8 @@ extern "C" tf_status tf_copy(const void* x, void* y, int64_t bytes, void* stream
 extern "C" tf_status tf_sin_fwd(const void* x, void* y, int64_t n, tf_dtype dt_, int threads, int vectors_per_thread, void* stream) {
     const int dt = dt_;
     if (n < 0 || (dt != DT_F32 && dt != DT_BF16) || (n > 0 && (!x || !y))) return TF_ERR_INVALID_ARG;
-    // defaults read off the geometry sweep (256 MiB of input): 128 threads with 4 vectors per thread
-    if (threads == 0) threads = 128;
+    // defaults read off the geometry sweep (256 MiB of input): 64 threads with 4 vectors per thread
+    if (threads == 0) threads = 64;
     int u = vectors_per_thread == 0 ? 4 : vectors_per_thread;
     if (threads < 32 || threads > 1024 || threads % 32 || (u != 1 && u != 2 && u != 4 && u != 8)) return TF_ERR_INVALID_ARG;
     if (n == 0) return TF_OK;
