@@ -287,6 +287,10 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
             // block.  LayerNorm bf16 rows of 64-512 columns: 81-82 us against 90-95 us for the pipeline (issue-bound there).
             q.variant = V_SROWS; q.threads = (nvec > 8 && nvec <= 16) ? 64 : 128;
             q.lanes = nvec <= 8 ? 2 : nvec <= 32 ? 4 : 8;
+            if (nvec & (nvec - 1)) {       // ragged rows: the fewest lanes with at most 8 vectors each (96 columns: 111 -> 93 us, 80: 84 -> 58)
+                q.lanes = 1;
+                while (q.lanes < 8 && (nvec + q.lanes - 1) / q.lanes > 8) q.lanes *= 2;
+            }
             const int64_t need = (nvec + q.lanes - 1) / q.lanes;
             q.vpt = need <= 4 ? 4 : need <= 8 ? 8 : 16;
             if (supports_srows(q, a, d)) return q;

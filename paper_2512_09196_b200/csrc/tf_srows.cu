@@ -90,6 +90,10 @@ __global__ void __launch_bounds__(256, 4) k_srows(const SArgs a) {       // 64 r
         const int rot = (G < 8) ? (r & (VPT - 1)) : 0;
         // (the walks are unrolled four vectors at a time: fully unrolled, the compiler hoists all of a pass's reads and spills)
         auto vec_of = [&](int k) { return g + G * ((k + rot) & (VPT - 1)); };
+        // the norms walk only the vectors the lane owns: all VPT of them in a full row (rotated), ceil((nvec - g) / G) in a
+        // ragged one (in order; no test per vector)
+        const int kend = FULL ? VPT : max(0, (nvec - g + G - 1) / G);
+        auto vec_at = [&](int k) { return FULL ? vec_of(k) : g + G * k; };
         const GroupRed<G> red;
         float mean = 0.f, scale = 0.f;
         if constexpr (OP == OP_SOFTMAX) {
@@ -131,43 +135,34 @@ __global__ void __launch_bounds__(256, 4) k_srows(const SArgs a) {       // 64 r
         } else if constexpr (OP == OP_LAYERNORM) {
             F2 s0 = f2(0.f), s1 = f2(0.f);
 #pragma unroll 4
-            for (int k = 0; k < VPT; ++k) {
-                const int j = vec_of(k);
-                if (FULL || j < nvec) {
-                    F2 w[NP];
-                    P::unpack(lds_again(rowp + j), w);
+            for (int k = 0; k < kend; ++k) {
+                F2 w[NP];
+                P::unpack(lds_again(rowp + vec_at(k)), w);
 #pragma unroll
-                    for (int i = 0; i < NP; i += 2) { s0 = add2(s0, w[i]); s1 = add2(s1, w[i + 1]); }
-                }
+                for (int i = 0; i < NP; i += 2) { s0 = add2(s0, w[i]); s1 = add2(s1, w[i + 1]); }
             }
             mean = fast_div(red.sum(hsum(add2(s0, s1)), 0), a.n);
             const F2 mm = f2(mean);
             F2 q0 = f2(0.f), q1 = f2(0.f);
 #pragma unroll 4
-            for (int k = 0; k < VPT; ++k) {
-                const int j = vec_of(k);
-                if (FULL || j < nvec) {
-                    F2 w[NP];
-                    P::unpack(lds_again(rowp + j), w);
+            for (int k = 0; k < kend; ++k) {
+                F2 w[NP];
+                P::unpack(lds_again(rowp + vec_at(k)), w);
 #pragma unroll
-                    for (int i = 0; i < NP; i += 2) {
-                        const F2 d0 = sub2(w[i], mm), d1 = sub2(w[i + 1], mm);
-                        q0 = fma2(d0, d0, q0); q1 = fma2(d1, d1, q1);
-                    }
+                for (int i = 0; i < NP; i += 2) {
+                    const F2 d0 = sub2(w[i], mm), d1 = sub2(w[i + 1], mm);
+                    q0 = fma2(d0, d0, q0); q1 = fma2(d1, d1, q1);
                 }
             }
             scale = fast_rsqrt(fast_div(red.sum(hsum(add2(q0, q1)), 0), a.n) + a.eps);
         } else {
             F2 q0 = f2(0.f), q1 = f2(0.f);
 #pragma unroll 4
-            for (int k = 0; k < VPT; ++k) {
-                const int j = vec_of(k);
-                if (FULL || j < nvec) {
-                    F2 w[NP];
-                    P::unpack(lds_again(rowp + j), w);
+            for (int k = 0; k < kend; ++k) {
+                F2 w[NP];
+                P::unpack(lds_again(rowp + vec_at(k)), w);
 #pragma unroll
-                    for (int i = 0; i < NP; i += 2) { q0 = fma2(w[i], w[i], q0); q1 = fma2(w[i + 1], w[i + 1], q1); }
-                }
+                for (int i = 0; i < NP; i += 2) { q0 = fma2(w[i], w[i], q0); q1 = fma2(w[i + 1], w[i + 1], q1); }
             }
             scale = fast_rsqrt(fast_div(red.sum(hsum(add2(q0, q1)), 0), a.n) + a.eps);
         }
@@ -179,10 +174,12 @@ __global__ void __launch_bounds__(256, 4) k_srows(const SArgs a) {       // 64 r
             }
             // LayerNorm: (mean, rstd); RMSNorm: (rrms, rrms)
             const F2 ta2 = f2(OP == OP_LAYERNORM ? mean : scale), tb2 = f2(scale);
+            if (live) {
 #pragma unroll 4
-            for (int k = 0; k < VPT; ++k) {
-                const int j = vec_of(k);
-                if (live && (FULL || j < nvec)) rowp[j] = apply_vec<OP, DT, true>(lds_again(rowp + j), params + j, params + nvec + j, ta2, tb2);
+                for (int k = 0; k < kend; ++k) {
+                    const int j = vec_at(k);
+                    rowp[j] = apply_vec<OP, DT, true>(lds_again(rowp + j), params + j, params + nvec + j, ta2, tb2);
+                }
             }
         }
     }
