@@ -243,6 +243,19 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
             else if (f32 && nvec >= 4096 && nvec < 8192) { ring(256, 4, 1, true); take = true; }
             else if (!f32 && nvec >= 8192) { ring(512, 3, 1, false); take = true; }
         }
+        // Widths between the sweep's powers of two that none of the rules above takes (20480-49152 columns; fp32 LayerNorm rows
+        // of 1-2 KiB that are not a power of two): what tf_tune keeps there is again the whole row in the ring, in up to four
+        // steps of up to 512 threads (softmax bf16 [3276, 20480]: 69 us for the pipeline, 43 us; LayerNorm bf16 [1638, 40960]:
+        // 73 us for the persistent clusters, 48 us).
+        const bool ragged = (nvec & (nvec - 1)) != 0;
+        if (!take && ragged &&
+            ((nvec > 4096 && nvec < 8192 && !(a.op == OP_RMSNORM && f32)) || (a.op == OP_SOFTMAX && !f32 && nvec > 2048 && nvec < 4096) ||
+             (a.op == OP_LAYERNORM && f32 && nvec >= 256 && nvec < 512))) {
+            int t = std::min(256, std::max(32, round_up(static_cast<int>((nvec + 7) / 8), 32)));
+            if ((nvec + 4 * t - 1) / (4 * t) > 4) t = round_up(static_cast<int>((nvec + 15) / 16), 32);
+            const int steps = static_cast<int>((nvec + 4 * t - 1) / (4 * t));
+            if (t <= 512 && steps <= 4) { ring(t, std::max(2, steps), 1, false); take = true; }
+        }
         if (take && a.rows >= 2LL * d.sms && supports_twopass(s, a, d)) return s;
     }
     // Rules read off the plans that tf_tune ends up with on the 84-point shape sweep (rows of 128 B to 256 KiB, three ops,
@@ -281,13 +294,17 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
             q.variant = V_CTA; q.cluster = 1; q.persist = 0; q.vpt = 8; q.threads = 64;
             if (supports_cta(q, a, d)) return q;
         }
-        if (nvec <= 128 && a.dt == DT_BF16 && a.op != OP_SOFTMAX && !(a.op == OP_RMSNORM && nvec > 64) && a.rows >= 64LL * d.sms) {
+        const bool ragged = (nvec & (nvec - 1)) != 0;
+        if (nvec <= 128 && a.op != OP_SOFTMAX && a.rows >= 64LL * d.sms &&
+            ((a.dt == DT_BF16 && !(a.op == OP_RMSNORM && nvec > 64)) || (ragged && !(ln && a.dt == DT_F32 && nvec < 32)))) {
+            // (ragged rows: either type, RMSNorm to 2 KiB -- RMSNorm fp32 rows of 72 columns 61 -> 42 us; fp32 LayerNorm rows below
+            // 512 B stay with the lane groups, which are 8-16 % ahead there)
             // bf16 LayerNorm rows up to 2 KiB and bf16 RMSNorm rows up to 1 KiB: blocks of rows resident in shared memory, a
             // few lanes per row walking 4-16 vectors each (no or few shuffles per row), y leaving as one bulk copy per
             // block.  LayerNorm bf16 rows of 64-512 columns: 81-82 us against 90-95 us for the pipeline (issue-bound there).
             q.variant = V_SROWS; q.threads = (nvec > 8 && nvec <= 16) ? 64 : 128;
             q.lanes = nvec <= 8 ? 2 : nvec <= 32 ? 4 : 8;
-            if (nvec & (nvec - 1)) {       // ragged rows: the fewest lanes with at most 8 vectors each (96 columns: 111 -> 93 us, 80: 84 -> 58)
+            if (ragged) {                  // ragged rows: the fewest lanes with at most 8 vectors each (96 columns: 111 -> 93 us, 80: 84 -> 58)
                 q.lanes = 1;
                 while (q.lanes < 8 && (nvec + q.lanes - 1) / q.lanes > 8) q.lanes *= 2;
             }
@@ -320,6 +337,7 @@ Plan heuristic(const Args& a, const DeviceInfo& d) {
             else if (nvec <= 64) { q.lanes = 32; q.vpt = 2; q.rpg = (a.dt == DT_F32 && a.op != OP_SOFTMAX) ? 2 : 1; }
             else if (nvec <= 128) { q.lanes = 32; q.vpt = 4; q.rpg = ((a.op == OP_RMSNORM && a.dt == DT_BF16) || (ln && a.dt == DT_F32)) ? 2 : 1; }
             else { q.lanes = 32; q.vpt = 8; }
+            if (ragged && a.op == OP_SOFTMAX && a.dt == DT_F32) q.threads = 256;      // (72 and 160 columns: 55-60 -> 44-45 us)
             if (supports_warp(q, a, d)) return q;
         } else if (!ln && nvec <= (a.dt == DT_BF16 ? 1024 : (a.op == OP_SOFTMAX ? 4096 : 3072))) {
             // softmax and RMSNorm from 4 KiB up to 16 KiB (bf16; eight bf16 vectors per thread cost too many registers) or
