@@ -230,6 +230,9 @@ Plan heuristic_addnorm(const Args& a, const DeviceInfo& d) {
         if (supports_addnorm(q, a, d)) return q;
         q = Plan();
     }
+    // rows beyond 64 KiB: the register-resident cluster forms lose to the plain add followed by the op's own long-row
+    // kernels (five tensors moved instead of four, but at the copy rate: bf16 LayerNorm [3276, 40960] 602 us fused)
+    if (nvec > 4096) return p;
     if (nvec <= 32) {
         q.variant = V_WARP; q.threads = 128; q.vpt = 1; q.rpg = 1;
         q.lanes = nvec <= 8 ? 8 : nvec <= 16 ? 16 : 32;
