@@ -208,8 +208,9 @@ tf_status tf_tune_norm_bwd_report(int* forms_timed, float* automatic_us, float* 
  * this is the residual-stream update of pre-norm transformer blocks.
  * x, r, h, y: [rows, cols] row-major, device memory, one element type; h may alias x or r, y may alias x; h and y must
  * not overlap each other.  gamma / beta / weight, mean / rstd, eps, errors and stream behaviour as for the unfused
- * calls, plus TF_ERR_INVALID_ARG for a null r or h.  Rows of up to 512 KiB on 16-byte aligned tensors run as one
- * kernel; anything else as an element-wise add followed by the unfused op (same results).  Allocates nothing. */
+ * calls, plus TF_ERR_INVALID_ARG for a null r or h.  Rows of up to 64 KiB on 16-byte aligned tensors run as one
+ * kernel; anything else as an element-wise add followed by the unfused op (same results; what the unfused op says
+ * about memory holds for that second step). */
 tf_status tf_add_layernorm_fwd(const void* x, const void* r, const void* gamma, const void* beta, void* h, void* y, float* mean,
                                float* rstd, int64_t rows, int64_t cols, float eps, tf_dtype dt, void* cuda_stream);
 tf_status tf_add_rmsnorm_fwd(const void* x, const void* r, const void* weight, void* h, void* y, float* rstd, int64_t rows,
