@@ -77,13 +77,18 @@ cudaError_t launch_softmax_len(const Plan& p, const Args& a, const DeviceInfo& d
 Plan heuristic_softmax_len(const Args& a, const DeviceInfo& d) {
     const int64_t nvec = a.cols * elem_size(a.dt) / 16;
     Plan q;
-    if (nvec <= 64) {
+    if (nvec < 256) {
+        // rows below 4 KiB: a lane group per row, the whole row loaded at once and the part behind the length discarded
+        // (65-255 vectors used to fall to a CTA per row with half its threads idle: bf16 rows of 1000 columns 154 us)
         q.variant = V_WARP; q.threads = 128; q.rpg = 1;
         if (nvec <= 8) { q.lanes = 8; q.vpt = 1; }
         else if (nvec <= 16) { q.lanes = 8; q.vpt = 2; }
         else if (nvec <= 32) { q.lanes = 16; q.vpt = 2; }
-        else { q.lanes = 32; q.vpt = 2; }
+        else if (nvec <= 64) { q.lanes = 32; q.vpt = 2; }
+        else if (nvec <= 128) { q.lanes = 32; q.vpt = 4; }
+        else { q.lanes = 32; q.vpt = 8; }
         if (supports_softmax_len(q, a, d)) return q;
+        q = Plan{};
     }
     if (nvec >= 256 && nvec <= 4096) {
         // rows of 4-64 KiB: the two-pass ring form with the whole row in the ring of one CTA copies only the live vectors of a
